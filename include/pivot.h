@@ -1,0 +1,169 @@
+/*
+ * pivot.h -- C ABI of the PIVOT group-shared indexer for NVIDIA B200 (sm_100a).
+ *
+ * The library produces, for every query token t, the index set T_t (k key positions) that a
+ * DSA-style sparse attention operator consumes.  It implements
+ *   - the dense lightning indexer  I_{t,s} = sum_j w_{t,j} ReLU(q_{t,j} . k_s), s <= t   (Eq. 1)
+ *     followed by T_t = TopK(I_{t,:}, k), and
+ *   - PIVOT (Algorithm 1): per group of g nearby queries one mean proxy (Eq. 4), one shared
+ *     prefix scan cut at the group's first position (Eq. 5), then either the proxy top-k for
+ *     the whole group (Reuse, Eq. 6) or a top-c candidate set (Eq. 7) re-scored by every member
+ *     with its own query and gate and reduced to a per-query top-k (Refine, Eq. 8-9).
+ * Groups are fixed-size runs of consecutive positions in prefill (Eq. 2) and the queries of one
+ * multi-token-prediction step in decode (Eq. 3).  Groups whose visible prefix is shorter than
+ * guard_len (default c) are scored densely per member (short-group guardrail of Algorithm 1).
+ *
+ * Conventions
+ *   - Positions are 0-indexed; query t sees keys 0..t inclusive.
+ *   - All pointers are DEVICE pointers owned by the caller unless a parameter says "host".
+ *     The library never allocates or frees device memory; scratch comes from the caller's
+ *     workspace (pivot_workspace_bytes / pivot_set_workspace, or the *_ex forms).
+ *   - All work is enqueued on `stream`; no entry point synchronises unless documented.
+ *   - Index output rows are SETS in unspecified order, no duplicates, every entry <= t.  When
+ *     fewer than k keys are visible (dense / guarded rows only) the valid entries come first
+ *     and the remainder is -1.
+ *   - Supported shapes: H_I = 64 indexer heads, d = 128, 1 <= k <= c <= 8192 (Refine) or
+ *     1 <= k <= 8192 (Reuse / dense).  Anything else returns PIVOT_ERR_UNSUPPORTED.
+ *   - Return value: PIVOT_OK or a positive error code; argument errors are detected on the host
+ *     before any launch.  Device-side conditions (a bounded wait that expired) are recorded in
+ *     a status word readable with pivot_device_status; kernels never trap.
+ */
+#ifndef PIVOT_H_
+#define PIVOT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* pivot_stream_t; /* a cudaStream_t */
+
+enum { PIVOT_BF16 = 0, PIVOT_FP8_E4M3 = 1 };
+enum { PIVOT_REUSE = 0, PIVOT_REFINE = 1 };
+enum { PIVOT_POOL_MEAN = 0, PIVOT_POOL_FIRST = 1, PIVOT_POOL_LAST = 2 };
+enum {
+  PIVOT_OK = 0,
+  PIVOT_ERR_INVALID_ARG = 1,
+  PIVOT_ERR_UNSUPPORTED = 2,
+  PIVOT_ERR_WORKSPACE = 3,   /* no workspace set, or too small */
+  PIVOT_ERR_CUDA = 4,        /* a CUDA runtime call failed; see pivot_last_cuda_error */
+  PIVOT_ERR_DEVICE = 5       /* device status word non-zero (pivot_device_status) */
+};
+
+/*
+ * A quantised operand.
+ *   data   row-major storage: bf16 bit patterns (2 B) or e4m3 codes (1 B).
+ *          queries: [L, H_I, d] (decode: [B, g, H_I, d]); key cache: [L, d] (decode: [B, Lmax, d]).
+ *   scale  NULL for bf16.  FP8: one fp32 scale per d-vector -- queries [L, H_I]
+ *          (decode [B, g, H_I]), keys [L] (decode [B, Lmax]); value = code * scale.
+ *   dtype  PIVOT_BF16 or PIVOT_FP8_E4M3; q and kcache must agree.
+ * data must be 16-byte aligned, scale 4-byte aligned.
+ */
+typedef struct pivot_tensor {
+  const void* data;
+  const float* scale;
+  int dtype;
+} pivot_tensor;
+
+/*
+ * Options of the *_ex entry points.  Zero-initialise, then set what is needed.
+ *   guard_len     groups with fewer visible keys than this are scored densely per member;
+ *                 -1 selects the default c (Algorithm 1 tests t0 < c).  0 disables the guardrail.
+ *   pool          proxy aggregation: mean (Eq. 4) or the first / last member (the paper's ablation).
+ *   dbg_cand      optional [n_groups, c] int32: candidate set of every group (Refine; rows of
+ *                 guarded groups are left untouched).  Unordered.
+ *   dbg_scores    optional fp32 buffer receiving the score that ranked each emitted index:
+ *                 same shape as out_idx ([rows, k]; -inf beside a -1 index).  For Refine these are
+ *                 the per-query re-scores (Eq. 8), for Reuse the proxy scores (Eq. 5), for dense
+ *                 and guarded rows Eq. 1.
+ *   dbg_cand_scores optional [n_groups, c] fp32: proxy score (Eq. 5) of each dbg_cand entry.
+ *   workspace     scratch of at least pivot_workspace_bytes(...) bytes, 256-byte aligned.
+ */
+typedef struct pivot_opts {
+  int guard_len;
+  int pool;
+  int32_t* dbg_cand;
+  float* dbg_scores;
+  float* dbg_cand_scores;
+  void* workspace;
+  size_t workspace_bytes;
+} pivot_opts;
+
+/* Bytes of scratch a call with these sizes needs.  rows = L for prefill / dense, B*g for decode;
+ * n_groups = ceil(L/g) or B.  Depends on the device's SM count (queried once). */
+size_t pivot_workspace_bytes(int rows, int n_groups, int c, int k);
+
+/* Registers the scratch buffer used by the short entry points below on the current device.
+ * The buffer stays owned by the caller and must outlive those calls.  Calls that share one
+ * workspace must not overlap on the GPU. */
+int pivot_set_workspace(void* workspace, size_t bytes);
+
+/*
+ * Prefill (Algorithm 1 with the grouping of Eq. 2) over one request of L positions.
+ *   q, kcache  operands as described at pivot_tensor; w is the gate [L, H_I] fp32 (the raw gate
+ *              times any positive constant; for FP8 NOT pre-multiplied by the query scale).
+ *   g          group size (>= 1; g = 1 is the dense indexer, Appendix A).
+ *   c, k       candidate budget and selection size; Refine needs k <= c.
+ *   mode       PIVOT_REUSE or PIVOT_REFINE.
+ *   out_idx    [L, k] int32.
+ */
+int pivot_index_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                        int L, int H_I, int d, int g, int c, int k, int mode,
+                        int32_t* out_idx, pivot_stream_t stream);
+int pivot_index_prefill_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                           int L, int H_I, int d, int g, int c, int k, int mode,
+                           int32_t* out_idx, pivot_stream_t stream, const pivot_opts* opts);
+
+/*
+ * Decode (Algorithm 1 with the grouping of Eq. 3): B independent sequences, each contributing
+ * the g queries of one MTP step at positions pos0[b] .. pos0[b]+g-1.
+ *   q       [B, g, H_I, d]; w [B, g, H_I]; kcache [B, Lmax, d] (+ scale [B, Lmax]); sequence b's
+ *           cache must hold keys 0 .. pos0[b]+g-1.
+ *   pos0    [B] int32, device.  The proxy scan is cut at pos0[b] (inclusive).
+ *   out_idx [B, g, k] int32.
+ */
+int pivot_index_decode(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                       const int32_t* pos0, int B, int Lmax, int H_I, int d, int g, int c, int k,
+                       int mode, int32_t* out_idx, pivot_stream_t stream);
+int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                          const int32_t* pos0, int B, int Lmax, int H_I, int d, int g, int c, int k,
+                          int mode, int32_t* out_idx, pivot_stream_t stream, const pivot_opts* opts);
+
+/*
+ * Dense control: Eq. 1 + TopK for every query of a request (prefill form) -- the O(L^2) indexer
+ * PIVOT replaces, run by the same kernels with one row per query.  out_idx [L, k].
+ */
+int dense_index(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                int L, int H_I, int d, int k, int32_t* out_idx, pivot_stream_t stream);
+int dense_index_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                   int L, int H_I, int d, int k, int32_t* out_idx, pivot_stream_t stream,
+                   const pivot_opts* opts);
+
+/*
+ * Host-buffer form of pivot_index_prefill: every tensor pointer (q, w, kcache, out_idx) is HOST
+ * memory (pinned for full copy speed).  The call copies the inputs into `arena` (device,
+ * at least pivot_prefill_host_arena_bytes(...) bytes, which includes the workspace), runs the
+ * device path, copies out_idx back and synchronises `stream` before returning.
+ */
+size_t pivot_prefill_host_arena_bytes(int L, int H_I, int d, int g, int c, int k, int dtype);
+int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                             int L, int H_I, int d, int g, int c, int k, int mode,
+                             int32_t* out_idx, void* arena, size_t arena_bytes,
+                             pivot_stream_t stream);
+
+/* Reads (and clears) the device status word of the workspace last used on this device after
+ * synchronising `stream`.  0 = no device-side condition. */
+int pivot_device_status(pivot_stream_t stream, int* status);
+
+/* Kernel launches issued by the library since the last call of this function (host counter). */
+long long pivot_launch_count_reset(void);
+
+const char* pivot_status_str(int code);
+int pivot_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PIVOT_H_ */

@@ -1,0 +1,197 @@
+"""ctypes binding of libpivot.so: argument marshalling only.
+
+Every function below has the name and argument order of the C entry point it forwards to
+(include/pivot.h); tensors are torch tensors whose device pointers are passed through.  torch
+is used for device memory and streams, nothing else: all arithmetic runs in the library's CUDA
+kernels.  Importing this module fails loudly when the shared library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpivot.so")
+
+BF16, FP8_E4M3 = 0, 1
+REUSE, REFINE = 0, 1
+POOL_MEAN, POOL_FIRST, POOL_LAST = 0, 1, 2
+OK = 0
+
+SYMBOLS = [
+    "pivot_workspace_bytes", "pivot_set_workspace", "pivot_index_prefill", "pivot_index_prefill_ex",
+    "pivot_index_decode", "pivot_index_decode_ex", "dense_index", "dense_index_ex",
+    "pivot_prefill_host_arena_bytes", "pivot_index_prefill_host", "pivot_device_status",
+    "pivot_launch_count_reset", "pivot_status_str", "pivot_last_cuda_error",
+]
+
+
+class pivot_tensor(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("scale", C.c_void_p), ("dtype", C.c_int)]
+
+
+class pivot_opts(C.Structure):
+    _fields_ = [("guard_len", C.c_int), ("pool", C.c_int), ("dbg_cand", C.c_void_p),
+                ("dbg_scores", C.c_void_p), ("dbg_cand_scores", C.c_void_p),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
+class PivotError(RuntimeError):
+    pass
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2607_24593_b200.build` "
+            "(there is no CPU fallback)")
+    lib = C.CDLL(LIB_PATH)
+    T, O, I, P, S = C.POINTER(pivot_tensor), C.POINTER(pivot_opts), C.c_int, C.c_void_p, C.c_size_t
+    lib.pivot_workspace_bytes.restype = S
+    lib.pivot_workspace_bytes.argtypes = [I, I, I, I]
+    lib.pivot_set_workspace.argtypes = [P, S]
+    lib.pivot_index_prefill.argtypes = [T, P, T, I, I, I, I, I, I, I, P, P]
+    lib.pivot_index_prefill_ex.argtypes = [T, P, T, I, I, I, I, I, I, I, P, P, O]
+    lib.pivot_index_decode.argtypes = [T, P, T, P, I, I, I, I, I, I, I, I, P, P]
+    lib.pivot_index_decode_ex.argtypes = [T, P, T, P, I, I, I, I, I, I, I, I, P, P, O]
+    lib.dense_index.argtypes = [T, P, T, I, I, I, I, P, P]
+    lib.dense_index_ex.argtypes = [T, P, T, I, I, I, I, P, P, O]
+    lib.pivot_prefill_host_arena_bytes.restype = S
+    lib.pivot_prefill_host_arena_bytes.argtypes = [I, I, I, I, I, I, I]
+    lib.pivot_index_prefill_host.argtypes = [T, P, T, I, I, I, I, I, I, I, P, P, S, P]
+    lib.pivot_device_status.argtypes = [P, C.POINTER(C.c_int)]
+    lib.pivot_launch_count_reset.restype = C.c_longlong
+    lib.pivot_status_str.restype = C.c_char_p
+    lib.pivot_status_str.argtypes = [I]
+    return lib
+
+
+lib = _load()
+_workspaces: dict[int, torch.Tensor] = {}
+
+
+def _check(rc: int):
+    if rc != OK:
+        extra = f" (cudaError {lib.pivot_last_cuda_error()})" if rc == 4 else ""
+        raise PivotError(f"libpivot: {lib.pivot_status_str(rc).decode()}{extra}")
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float8_e4m3fn:
+        return FP8_E4M3
+    raise TypeError(f"unsupported operand dtype {t.dtype}")
+
+
+def _tensor(data: torch.Tensor, scale) -> pivot_tensor:
+    assert data.is_contiguous() and (scale is None or (scale.is_contiguous() and scale.dtype == torch.float32))
+    return pivot_tensor(data.data_ptr(), None if scale is None else scale.data_ptr(), _dtype_code(data))
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace) -> pivot_opts:
+    p = lambda t: None if t is None else t.data_ptr()
+    return pivot_opts(-1 if guard_len is None else guard_len, pool, p(dbg_cand), p(dbg_scores),
+                      p(dbg_cand_scores), p(workspace), 0 if workspace is None else workspace.numel())
+
+
+def pivot_workspace_bytes(rows: int, n_groups: int, c: int, k: int) -> int:
+    return int(lib.pivot_workspace_bytes(rows, n_groups, c, k))
+
+
+def pivot_set_workspace(workspace: torch.Tensor | None):
+    """Registers a uint8 CUDA tensor as the scratch of the short entry points (kept alive here)."""
+    if workspace is None:
+        _check(lib.pivot_set_workspace(None, 0))
+        _workspaces.pop(torch.cuda.current_device(), None)
+        return
+    assert workspace.dtype == torch.uint8 and workspace.is_cuda
+    _check(lib.pivot_set_workspace(workspace.data_ptr(), workspace.numel()))
+    _workspaces[workspace.device.index] = workspace
+
+
+def ensure_workspace(rows: int, n_groups: int, c: int, k: int, device="cuda") -> torch.Tensor:
+    """Allocates (or reuses) a registered workspace large enough for these sizes."""
+    need = pivot_workspace_bytes(rows, n_groups, c, k)
+    dev = torch.device(device)
+    idx = dev.index if dev.index is not None else torch.cuda.current_device()
+    cur = _workspaces.get(idx)
+    if cur is None or cur.numel() < need:
+        with torch.cuda.device(idx):
+            cur = torch.empty(need, dtype=torch.uint8, device=f"cuda:{idx}")
+            pivot_set_workspace(cur)
+    return cur
+
+
+def pivot_index_prefill(q, w, kcache, L, H_I, d, g, c, k, mode, out_idx, stream=None, *,
+                        q_scale=None, k_scale=None, guard_len=None, pool=POOL_MEAN, dbg_cand=None,
+                        dbg_scores=None, dbg_cand_scores=None, workspace=None):
+    tq, tk = _tensor(q, q_scale), _tensor(kcache, k_scale)
+    assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and out_idx.numel() >= L * k
+    if workspace is None:
+        ensure_workspace(L, (L + g - 1) // g, c, k, q.device)
+    o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace)
+    _check(lib.pivot_index_prefill_ex(C.byref(tq), w.data_ptr(), C.byref(tk), L, H_I, d, g, c, k, mode,
+                                      out_idx.data_ptr(), _stream(stream), C.byref(o)))
+    return out_idx
+
+
+def dense_index(q, w, kcache, L, H_I, d, k, out_idx, stream=None, *, q_scale=None, k_scale=None,
+                dbg_scores=None, workspace=None):
+    tq, tk = _tensor(q, q_scale), _tensor(kcache, k_scale)
+    assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and out_idx.numel() >= L * k
+    if workspace is None:
+        ensure_workspace(L, L, k, k, q.device)
+    o = _opts(None, POOL_MEAN, None, dbg_scores, None, workspace)
+    _check(lib.dense_index_ex(C.byref(tq), w.data_ptr(), C.byref(tk), L, H_I, d, k, out_idx.data_ptr(),
+                              _stream(stream), C.byref(o)))
+    return out_idx
+
+
+def pivot_index_decode(q, w, kcache, pos0, B, Lmax, H_I, d, g, c, k, mode, out_idx, stream=None, *,
+                       q_scale=None, k_scale=None, guard_len=None, pool=POOL_MEAN, dbg_cand=None,
+                       dbg_scores=None, dbg_cand_scores=None, workspace=None):
+    tq, tk = _tensor(q, q_scale), _tensor(kcache, k_scale)
+    assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and pos0.dtype == torch.int32
+    assert out_idx.numel() >= B * g * k
+    if workspace is None:
+        ensure_workspace(B * g, B, c, k, q.device)
+    o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace)
+    _check(lib.pivot_index_decode_ex(C.byref(tq), w.data_ptr(), C.byref(tk), pos0.data_ptr(), B, Lmax,
+                                     H_I, d, g, c, k, mode, out_idx.data_ptr(), _stream(stream), C.byref(o)))
+    return out_idx
+
+
+def pivot_prefill_host_arena_bytes(L, H_I, d, g, c, k, dtype) -> int:
+    return int(lib.pivot_prefill_host_arena_bytes(L, H_I, d, g, c, k, dtype))
+
+
+def pivot_index_prefill_host(q, w, kcache, L, H_I, d, g, c, k, mode, out_idx, arena, stream=None, *,
+                             q_scale=None, k_scale=None):
+    """Host-buffer form: q / w / kcache / scales / out_idx are CPU tensors (pin them), `arena` a
+    uint8 CUDA tensor of at least pivot_prefill_host_arena_bytes(...) bytes.  Returns after the
+    result has landed in out_idx."""
+    for t in (q, w, kcache, out_idx):
+        assert not t.is_cuda
+    tq, tk = _tensor(q, q_scale), _tensor(kcache, k_scale)
+    _check(lib.pivot_index_prefill_host(C.byref(tq), w.data_ptr(), C.byref(tk), L, H_I, d, g, c, k, mode,
+                                        out_idx.data_ptr(), arena.data_ptr(), arena.numel(), _stream(stream)))
+    return out_idx
+
+
+def pivot_device_status(stream=None) -> int:
+    st = C.c_int(0)
+    _check(lib.pivot_device_status(_stream(stream), C.byref(st)))
+    return st.value
+
+
+def pivot_launch_count_reset() -> int:
+    return int(lib.pivot_launch_count_reset())

@@ -1,0 +1,334 @@
+// C ABI of the library (see include/pivot.h): argument checks, workspace carving, and the
+// launch sequence of Algorithm 1 -- proxy build (Eq. 4), planner, shared scan + streaming
+// select (Eq. 5-7), gather + re-score + top-k (Eq. 8-9).
+#include <stdio.h>
+#include <string.h>
+
+#include "../../include/pivot.h"
+#include "kernels.h"
+
+using namespace pivot;
+
+namespace {
+
+constexpr int kMaxSel = 8192;
+constexpr int kMaxDevices = 64;
+
+struct DeviceState {
+  void* ws = nullptr;
+  size_t ws_bytes = 0;
+  int sm_count = 0;
+  int* last_status = nullptr;
+};
+DeviceState g_dev[kMaxDevices];
+int g_last_cuda = 0;
+
+int cur_device() {
+  int d = 0;
+  cudaGetDevice(&d);
+  return (d >= 0 && d < kMaxDevices) ? d : 0;
+}
+
+int sm_count() {
+  DeviceState& ds = g_dev[cur_device()];
+  if (ds.sm_count == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, cur_device()) != cudaSuccess || n <= 0)
+      n = 148;
+    ds.sm_count = n;
+  }
+  return ds.sm_count;
+}
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+int cand_cap(int kmax) {
+  int cap = 2 * kmax;
+  if (cap < kmax + 1024) cap = kmax + 1024;
+  return (int)align_up((size_t)cap, 64);
+}
+
+struct Carve {
+  char* base;
+  size_t off = 0;
+  explicit Carve(void* p) : base((char*)p) {}
+  template <typename T>
+  T* take(size_t n) {
+    T* p = (T*)(base + off);
+    off = align_up(off + n * sizeof(T));
+    return p;
+  }
+};
+
+struct Workspace {
+  int* status;
+  int* counter;
+  void* proxy_q;
+  float* proxy_w;
+  int32_t* cand;
+  RowDesc* rows;
+  GroupDesc* groups;
+  ScanScratch scan;
+  size_t bytes;
+};
+
+// rows: scan-row slots; n_groups: groups (proxy rows / Refine groups).
+Workspace carve_workspace(void* base, int rows, int n_groups, int c, int k) {
+  Workspace w;
+  Carve cv(base);
+  const int kmax = c > k ? c : k;
+  int* head = cv.take<int>(64);
+  w.status = head;
+  w.counter = head + 1;
+  w.proxy_q = cv.take<uint16_t>((size_t)n_groups * kHeads * kDim);
+  w.proxy_w = cv.take<float>((size_t)n_groups * kHeads);
+  w.cand = cv.take<int32_t>((size_t)n_groups * c);
+  w.rows = cv.take<RowDesc>((size_t)rows + n_groups);
+  w.groups = cv.take<GroupDesc>((size_t)n_groups);
+  w.scan.n_cta = sm_count() * 4;
+  w.scan.cap = cand_cap(kmax);
+  w.scan.cand_key = cv.take<uint32_t>((size_t)w.scan.n_cta * 2 * w.scan.cap);
+  w.scan.cand_idx = cv.take<int32_t>((size_t)w.scan.n_cta * 2 * w.scan.cap);
+  w.scan.status = w.status;
+  w.scan.counter = w.counter;
+  w.bytes = cv.off;
+  return w;
+}
+
+int check_cuda(cudaError_t e) {
+  if (e == cudaSuccess) return PIVOT_OK;
+  g_last_cuda = (int)e;
+  return PIVOT_ERR_CUDA;
+}
+
+int check_common(const pivot_tensor* q, const float* w, const pivot_tensor* kc, int H, int d, int c,
+                 int k, int mode, const void* out) {
+  if (!q || !w || !kc || !out || !q->data || !kc->data) return PIVOT_ERR_INVALID_ARG;
+  if (q->dtype != kc->dtype) return PIVOT_ERR_INVALID_ARG;
+  if (q->dtype != PIVOT_BF16 && q->dtype != PIVOT_FP8_E4M3) return PIVOT_ERR_INVALID_ARG;
+  if (q->dtype == PIVOT_FP8_E4M3 && (!q->scale || !kc->scale)) return PIVOT_ERR_INVALID_ARG;
+  if (k < 1 || c < 1) return PIVOT_ERR_INVALID_ARG;
+  if (mode != PIVOT_REUSE && mode != PIVOT_REFINE) return PIVOT_ERR_INVALID_ARG;
+  if (mode == PIVOT_REFINE && k > c) return PIVOT_ERR_INVALID_ARG;
+  if (((uintptr_t)q->data | (uintptr_t)kc->data) & 15) return PIVOT_ERR_INVALID_ARG;
+  if (((uintptr_t)w | (uintptr_t)out | (uintptr_t)q->scale | (uintptr_t)kc->scale) & 3)
+    return PIVOT_ERR_INVALID_ARG;
+  if (H != kHeads || d != kDim) return PIVOT_ERR_UNSUPPORTED;
+  if (k > kMaxSel || c > kMaxSel) return PIVOT_ERR_UNSUPPORTED;
+  return PIVOT_OK;
+}
+
+int resolve_ws(const pivot_opts* o, size_t need, void** ws) {
+  void* p = o && o->workspace ? o->workspace : g_dev[cur_device()].ws;
+  size_t n = o && o->workspace ? o->workspace_bytes : g_dev[cur_device()].ws_bytes;
+  if (!p || n < need || ((uintptr_t)p & 255)) return PIVOT_ERR_WORKSPACE;
+  *ws = p;
+  return PIVOT_OK;
+}
+
+int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, int L, int g, int c,
+                int k, int mode, bool dense_only, int32_t* out_idx, cudaStream_t st,
+                const pivot_opts* o) {
+  const int nG = (L + g - 1) / g;
+  const size_t need = pivot_workspace_bytes(L, nG, c, k);
+  void* wsp = nullptr;
+  int rc = resolve_ws(o, need, &wsp);
+  if (rc) return rc;
+  Workspace ws = carve_workspace(wsp, L, nG, c, k);
+  g_dev[cur_device()].last_status = ws.status;
+
+  int guard = (o && o->guard_len >= 0) ? o->guard_len : c;
+  int first_group = guard <= 1 ? 0 : (guard - 1 + g - 1) / g;
+  if (first_group > nG) first_group = nG;
+  if (dense_only) first_group = nG;
+  long long nd = (long long)first_group * g;
+  PrefillPlan p;
+  p.q = q->data; p.w = w; p.qscale = q->scale;
+  p.kc = kc->data; p.kscale = kc->scale;
+  p.proxy_q = ws.proxy_q; p.proxy_w = ws.proxy_w;
+  p.cand = (o && o->dbg_cand) ? o->dbg_cand + (size_t)first_group * c : ws.cand;
+  p.cand_score = (o && o->dbg_cand_scores) ? o->dbg_cand_scores + (size_t)first_group * c : nullptr;
+  p.out = out_idx; p.out_score = o ? o->dbg_scores : nullptr;
+  p.L = L; p.g = g; p.c = c; p.k = k; p.mode = mode; p.dtype = q->dtype;
+  p.n_dense = (int)(nd < L ? nd : L);
+  p.first_group = first_group;
+  p.n_proxy = nG - first_group;
+
+  if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 2 * sizeof(int), st)))) return rc;
+  launch_proxy_build(q->data, q->scale, w, ws.proxy_q, ws.proxy_w, L, g, first_group, p.n_proxy,
+                     q->dtype, o ? o->pool : 0, st);
+  launch_plan_prefill(p, ws.rows, ws.groups, st);
+  launch_scan_simt(ws.rows, p.n_dense + p.n_proxy, q->dtype, ws.scan, st);
+  if (mode == PIVOT_REFINE) launch_refine_simt(ws.groups, p.n_proxy, q->dtype, ws.scan, st);
+  return check_cuda(cudaGetLastError());
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t pivot_workspace_bytes(int rows, int n_groups, int c, int k) {
+  if (rows < 1 || n_groups < 1 || c < 1 || k < 1) return 0;
+  return carve_workspace(nullptr, rows, n_groups, c, k).bytes;
+}
+
+int pivot_set_workspace(void* workspace, size_t bytes) {
+  if (workspace && ((uintptr_t)workspace & 255)) return PIVOT_ERR_INVALID_ARG;
+  DeviceState& ds = g_dev[cur_device()];
+  ds.ws = workspace;
+  ds.ws_bytes = workspace ? bytes : 0;
+  return PIVOT_OK;
+}
+
+int pivot_index_prefill_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kcache, int L,
+                           int H_I, int d, int g, int c, int k, int mode, int32_t* out_idx,
+                           pivot_stream_t stream, const pivot_opts* opts) {
+  int rc = check_common(q, w, kcache, H_I, d, c, k, mode, out_idx);
+  if (rc) return rc;
+  if (L < 1 || g < 1) return PIVOT_ERR_INVALID_ARG;
+  if (opts && (opts->pool < 0 || opts->pool > 2)) return PIVOT_ERR_INVALID_ARG;
+  return run_prefill(q, w, kcache, L, g, c, k, mode, false, out_idx, (cudaStream_t)stream, opts);
+}
+
+int pivot_index_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kcache, int L,
+                        int H_I, int d, int g, int c, int k, int mode, int32_t* out_idx,
+                        pivot_stream_t stream) {
+  return pivot_index_prefill_ex(q, w, kcache, L, H_I, d, g, c, k, mode, out_idx, stream, nullptr);
+}
+
+int dense_index_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kcache, int L, int H_I,
+                   int d, int k, int32_t* out_idx, pivot_stream_t stream, const pivot_opts* opts) {
+  int rc = check_common(q, w, kcache, H_I, d, k, k, PIVOT_REUSE, out_idx);
+  if (rc) return rc;
+  if (L < 1) return PIVOT_ERR_INVALID_ARG;
+  return run_prefill(q, w, kcache, L, 1, k, k, PIVOT_REUSE, true, out_idx, (cudaStream_t)stream, opts);
+}
+
+int dense_index(const pivot_tensor* q, const float* w, const pivot_tensor* kcache, int L, int H_I,
+                int d, int k, int32_t* out_idx, pivot_stream_t stream) {
+  return dense_index_ex(q, w, kcache, L, H_I, d, k, out_idx, stream, nullptr);
+}
+
+int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                          const int32_t* pos0, int B, int Lmax, int H_I, int d, int g, int c, int k,
+                          int mode, int32_t* out_idx, pivot_stream_t stream, const pivot_opts* o) {
+  int rc = check_common(q, w, kcache, H_I, d, c, k, mode, out_idx);
+  if (rc) return rc;
+  if (!pos0 || B < 1 || g < 1 || Lmax < g) return PIVOT_ERR_INVALID_ARG;
+  if (o && (o->pool < 0 || o->pool > 2)) return PIVOT_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t need = pivot_workspace_bytes(B * g, B, c, k);
+  void* wsp = nullptr;
+  if ((rc = resolve_ws(o, need, &wsp))) return rc;
+  Workspace ws = carve_workspace(wsp, B * g, B, c, k);
+  g_dev[cur_device()].last_status = ws.status;
+  DecodePlan p;
+  p.q = q->data; p.w = w; p.qscale = q->scale;
+  p.kc = kcache->data; p.kscale = kcache->scale;
+  p.pos0 = pos0;
+  p.proxy_q = ws.proxy_q; p.proxy_w = ws.proxy_w;
+  p.cand = (o && o->dbg_cand) ? o->dbg_cand : ws.cand;
+  p.cand_score = o ? o->dbg_cand_scores : nullptr;
+  p.out = out_idx; p.out_score = o ? o->dbg_scores : nullptr;
+  p.B = B; p.Lmax = Lmax; p.g = g; p.c = c; p.k = k; p.mode = mode; p.dtype = q->dtype;
+  p.guard_len = (o && o->guard_len >= 0) ? o->guard_len : c;
+  if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 2 * sizeof(int), st)))) return rc;
+  launch_proxy_build(q->data, q->scale, w, ws.proxy_q, ws.proxy_w, B * g, g, 0, B, q->dtype,
+                     o ? o->pool : 0, st);
+  launch_plan_decode(p, ws.rows, ws.groups, st);
+  launch_scan_simt(ws.rows, B + B * g, q->dtype, ws.scan, st);
+  if (mode == PIVOT_REFINE) launch_refine_simt(ws.groups, B, q->dtype, ws.scan, st);
+  return check_cuda(cudaGetLastError());
+}
+
+int pivot_index_decode(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                       const int32_t* pos0, int B, int Lmax, int H_I, int d, int g, int c, int k,
+                       int mode, int32_t* out_idx, pivot_stream_t stream) {
+  return pivot_index_decode_ex(q, w, kcache, pos0, B, Lmax, H_I, d, g, c, k, mode, out_idx, stream,
+                               nullptr);
+}
+
+size_t pivot_prefill_host_arena_bytes(int L, int H_I, int d, int g, int c, int k, int dtype) {
+  if (L < 1 || g < 1 || H_I < 1 || d < 1) return 0;
+  const size_t esz = dtype == PIVOT_FP8_E4M3 ? 1 : 2;
+  size_t n = 0;
+  n += align_up((size_t)L * H_I * d * esz);   // q
+  n += align_up((size_t)L * H_I * 4);         // q scale
+  n += align_up((size_t)L * H_I * 4);         // w
+  n += align_up((size_t)L * d * esz);         // k
+  n += align_up((size_t)L * 4);               // k scale
+  n += align_up((size_t)L * k * 4);           // out
+  n += pivot_workspace_bytes(L, (L + g - 1) / g, c, k);
+  return n;
+}
+
+int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_tensor* kcache, int L,
+                             int H_I, int d, int g, int c, int k, int mode, int32_t* out_idx,
+                             void* arena, size_t arena_bytes, pivot_stream_t stream) {
+  if (!q || !w || !kcache || !out_idx || !arena || L < 1 || g < 1) return PIVOT_ERR_INVALID_ARG;
+  if (((uintptr_t)arena & 255) || arena_bytes < pivot_prefill_host_arena_bytes(L, H_I, d, g, c, k, q->dtype))
+    return PIVOT_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const bool fp8 = q->dtype == PIVOT_FP8_E4M3;
+  const size_t esz = fp8 ? 1 : 2;
+  Carve cv(arena);
+  void* dq = cv.take<char>((size_t)L * H_I * d * esz);
+  float* dqs = cv.take<float>((size_t)L * H_I);
+  float* dw = cv.take<float>((size_t)L * H_I);
+  void* dk = cv.take<char>((size_t)L * d * esz);
+  float* dks = cv.take<float>((size_t)L);
+  int32_t* dout = cv.take<int32_t>((size_t)L * k);
+  void* dws = arena ? (char*)arena + cv.off : nullptr;
+  int rc;
+  if ((rc = check_cuda(cudaMemcpyAsync(dq, q->data, (size_t)L * H_I * d * esz, cudaMemcpyHostToDevice, st)))) return rc;
+  if ((rc = check_cuda(cudaMemcpyAsync(dw, w, (size_t)L * H_I * 4, cudaMemcpyHostToDevice, st)))) return rc;
+  if ((rc = check_cuda(cudaMemcpyAsync(dk, kcache->data, (size_t)L * d * esz, cudaMemcpyHostToDevice, st)))) return rc;
+  if (fp8) {
+    if (!q->scale || !kcache->scale) return PIVOT_ERR_INVALID_ARG;
+    if ((rc = check_cuda(cudaMemcpyAsync(dqs, q->scale, (size_t)L * H_I * 4, cudaMemcpyHostToDevice, st)))) return rc;
+    if ((rc = check_cuda(cudaMemcpyAsync(dks, kcache->scale, (size_t)L * 4, cudaMemcpyHostToDevice, st)))) return rc;
+  }
+  pivot_tensor tq{dq, fp8 ? dqs : nullptr, q->dtype};
+  pivot_tensor tk{dk, fp8 ? dks : nullptr, q->dtype};
+  pivot_opts o;
+  memset(&o, 0, sizeof(o));
+  o.guard_len = -1;
+  o.workspace = dws;
+  o.workspace_bytes = arena_bytes - cv.off;
+  rc = pivot_index_prefill_ex(&tq, dw, &tk, L, H_I, d, g, c, k, mode, dout, stream, &o);
+  if (rc) return rc;
+  if ((rc = check_cuda(cudaMemcpyAsync(out_idx, dout, (size_t)L * k * 4, cudaMemcpyDeviceToHost, st)))) return rc;
+  return check_cuda(cudaStreamSynchronize(st));
+}
+
+int pivot_device_status(pivot_stream_t stream, int* status) {
+  if (!status) return PIVOT_ERR_INVALID_ARG;
+  int* p = g_dev[cur_device()].last_status;
+  *status = 0;
+  if (!p) return PIVOT_OK;
+  int rc = check_cuda(cudaStreamSynchronize((cudaStream_t)stream));
+  if (rc) return rc;
+  return check_cuda(cudaMemcpy(status, p, sizeof(int), cudaMemcpyDeviceToHost));
+}
+
+long long pivot_launch_count_reset(void) {
+  long long n = launch_counter();
+  launch_counter() = 0;
+  return n;
+}
+
+const char* pivot_status_str(int code) {
+  switch (code) {
+    case PIVOT_OK: return "ok";
+    case PIVOT_ERR_INVALID_ARG: return "invalid argument";
+    case PIVOT_ERR_UNSUPPORTED: return "unsupported shape (H_I must be 64, d 128, k and c at most 8192)";
+    case PIVOT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case PIVOT_ERR_CUDA: return "CUDA runtime error (see pivot_last_cuda_error)";
+    case PIVOT_ERR_DEVICE: return "device-side condition recorded in the status word";
+    default: return "unknown status";
+  }
+}
+
+int pivot_last_cuda_error(void) { return g_last_cuda; }
+
+}  // extern "C"

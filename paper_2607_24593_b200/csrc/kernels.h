@@ -1,0 +1,71 @@
+// Host-callable launchers of the library's kernels (internal header).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "common.cuh"
+
+namespace pivot {
+
+// One group's fine step (Eq. 8-9): m members re-score the candidate list.
+struct GroupDesc {
+  const void* q;        // first member [m, H, d] codes, members contiguous
+  const float* w;       // [m, H]
+  const float* qscale;  // [m, H] or nullptr
+  const void* kbase;
+  const float* kscale;
+  const int32_t* cand;  // candidate key positions, valid entries first
+  int n_cand;           // valid candidates (0: group is skipped)
+  int m;                // members
+  int K;                // entries to select per member
+  int first_pos;        // position of the first member (slot i sits at first_pos + i)
+  int32_t* out;         // [m, out_stride]
+  float* out_score;     // optional
+  int out_stride;
+};
+
+// Geometry of a prefill-shaped call, shared by the planner kernels.
+struct PrefillPlan {
+  const void* q; const float* w; const float* qscale;   // raw per-query operands
+  const void* kc; const float* kscale;                  // key cache
+  void* proxy_q; float* proxy_w;                        // [nP, H, d], [nP, H]
+  int32_t* cand; float* cand_score;                     // [nP, c] (Refine)
+  int32_t* out; float* out_score;                       // [L, k]
+  int L, g, c, k, mode, dtype;
+  int n_dense;      // rows 0 .. n_dense-1 are scored densely (guarded groups or dense control)
+  int first_group;  // first group taking the proxy path
+  int n_proxy;      // groups on the proxy path
+};
+
+struct DecodePlan {
+  const void* q; const float* w; const float* qscale;   // [B, g, H, d] ...
+  const void* kc; const float* kscale;                  // [B, Lmax, d], [B, Lmax]
+  const int32_t* pos0;
+  void* proxy_q; float* proxy_w;                        // [B, H, d], [B, H]
+  int32_t* cand; float* cand_score;                     // [B, c]
+  int32_t* out; float* out_score;                       // [B, g, k]
+  int B, Lmax, g, c, k, mode, dtype, guard_len;
+};
+
+struct ScanScratch {
+  uint32_t* cand_key;   // [n_cta][2][cap]
+  int32_t* cand_idx;    // [n_cta][2][cap]
+  int cap;
+  int n_cta;
+  int* status;
+  int* counter;         // dynamic row scheduler
+};
+
+void launch_proxy_build(const void* q, const float* qscale, const float* w, void* proxy_q,
+                        float* proxy_w, int rows, int g, int first_group, int n_proxy, int dtype,
+                        int pool, cudaStream_t st);
+void launch_plan_prefill(const PrefillPlan& p, RowDesc* rows, GroupDesc* groups, cudaStream_t st);
+void launch_plan_decode(const DecodePlan& p, RowDesc* rows, GroupDesc* groups, cudaStream_t st);
+// Decode proxies need the guard test on device (pos0 lives there): rows of guarded sequences
+// get K = 0 and are skipped.
+void launch_scan_simt(const RowDesc* rows, int n_rows, int dtype, const ScanScratch& s, cudaStream_t st);
+void launch_refine_simt(const GroupDesc* groups, int n_groups, int dtype, const ScanScratch& s, cudaStream_t st);
+
+long long& launch_counter();
+
+}  // namespace pivot

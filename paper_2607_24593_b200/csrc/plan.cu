@@ -1,0 +1,148 @@
+// Planner kernels: turn a call's geometry into row descriptors (one per scan row) and group
+// descriptors (one per Refine group).  Grouping follows Eq. 2 (prefill) and Eq. 3 (decode);
+// the short-group guardrail of Algorithm 1 decides which rows are dense.
+#include "kernels.h"
+
+namespace pivot {
+
+// Scan-row order for prefill: rows [0, n_dense) are dense rows (row i = query i), rows
+// [n_dense, n_dense + n_proxy) are proxy rows.
+__global__ void plan_prefill_kernel(PrefillPlan p, RowDesc* rows, GroupDesc* groups) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t esz = p.dtype == DT_FP8 ? 1 : 2;
+  const size_t qrow = (size_t)kHeads * kDim * esz;
+  if (i < p.n_dense) {
+    RowDesc r;
+    r.q = (const char*)p.q + (size_t)i * qrow;
+    r.w = p.w + (size_t)i * kHeads;
+    r.qscale = p.qscale ? p.qscale + (size_t)i * kHeads : nullptr;
+    r.kbase = p.kc;
+    r.kscale = p.kscale;
+    r.n_vis = i + 1;
+    r.K = p.k;
+    r.out = p.out + (size_t)i * p.k;
+    r.out_score = p.out_score ? p.out_score + (size_t)i * p.k : nullptr;
+    r.out_rows = 1;
+    r.out_stride = p.k;
+    rows[i] = r;
+  } else if (i < p.n_dense + p.n_proxy) {
+    const int pr = i - p.n_dense;
+    const int t0 = (p.first_group + pr) * p.g;
+    const int m = min(p.g, p.L - t0);
+    RowDesc r;
+    r.q = (const char*)p.proxy_q + (size_t)pr * qrow;
+    r.w = p.proxy_w + (size_t)pr * kHeads;
+    r.qscale = nullptr;
+    r.kbase = p.kc;
+    r.kscale = p.kscale;
+    r.n_vis = t0 + 1;
+    if (p.mode == 0) {   // Reuse: the proxy top-k goes to every member (Eq. 6)
+      r.K = p.k;
+      r.out = p.out + (size_t)t0 * p.k;
+      r.out_score = p.out_score ? p.out_score + (size_t)t0 * p.k : nullptr;
+      r.out_rows = m;
+      r.out_stride = p.k;
+    } else {             // Refine: top-c candidate set (Eq. 7)
+      r.K = p.c;
+      r.out = p.cand + (size_t)pr * p.c;
+      r.out_score = p.cand_score ? p.cand_score + (size_t)pr * p.c : nullptr;
+      r.out_rows = 1;
+      r.out_stride = p.c;
+      GroupDesc gd;
+      gd.q = (const char*)p.q + (size_t)t0 * qrow;
+      gd.w = p.w + (size_t)t0 * kHeads;
+      gd.qscale = p.qscale ? p.qscale + (size_t)t0 * kHeads : nullptr;
+      gd.kbase = p.kc;
+      gd.kscale = p.kscale;
+      gd.cand = r.out;
+      gd.n_cand = min(p.c, r.n_vis);
+      gd.m = m;
+      gd.K = p.k;
+      gd.first_pos = t0;
+      gd.out = p.out + (size_t)t0 * p.k;
+      gd.out_score = p.out_score ? p.out_score + (size_t)t0 * p.k : nullptr;
+      gd.out_stride = p.k;
+      groups[pr] = gd;
+    }
+    rows[i] = r;
+  }
+}
+
+void launch_plan_prefill(const PrefillPlan& p, RowDesc* rows, GroupDesc* groups, cudaStream_t st) {
+  const int n = p.n_dense + p.n_proxy;
+  if (n <= 0) return;
+  plan_prefill_kernel<<<(n + 255) / 256, 256, 0, st>>>(p, rows, groups);
+  ++launch_counter();
+}
+
+// Decode: scan-row slot b is sequence b's proxy row; slots B + b*g + i are its dense rows.
+// Exactly one of the two kinds is live per sequence (the guard test runs here because pos0
+// lives on the device); dead slots get K = 0 and are skipped by the kernels.
+__global__ void plan_decode_kernel(DecodePlan p, RowDesc* rows, GroupDesc* groups) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= p.B) return;
+  const size_t esz = p.dtype == DT_FP8 ? 1 : 2;
+  const size_t qrow = (size_t)kHeads * kDim * esz;
+  const int p0 = p.pos0[b];
+  const int n0 = p0 + 1;
+  const bool guarded = n0 < p.guard_len;
+  const void* kb = (const char*)p.kc + (size_t)b * p.Lmax * kDim * esz;
+  const float* ksb = p.kscale ? p.kscale + (size_t)b * p.Lmax : nullptr;
+  int32_t* outb = p.out + (size_t)b * p.g * p.k;
+  float* outsb = p.out_score ? p.out_score + (size_t)b * p.g * p.k : nullptr;
+  RowDesc r;
+  r.q = (const char*)p.proxy_q + (size_t)b * qrow;
+  r.w = p.proxy_w + (size_t)b * kHeads;
+  r.qscale = nullptr;
+  r.kbase = kb;
+  r.kscale = ksb;
+  r.n_vis = n0;
+  GroupDesc gd;
+  gd.q = (const char*)p.q + (size_t)b * p.g * qrow;
+  gd.w = p.w + (size_t)b * p.g * kHeads;
+  gd.qscale = p.qscale ? p.qscale + (size_t)b * p.g * kHeads : nullptr;
+  gd.kbase = kb;
+  gd.kscale = ksb;
+  gd.cand = p.cand + (size_t)b * p.c;
+  gd.n_cand = 0;
+  gd.m = p.g;
+  gd.K = p.k;
+  gd.first_pos = p0;
+  gd.out = outb;
+  gd.out_score = outsb;
+  gd.out_stride = p.k;
+  if (guarded) {
+    r.K = 0; r.out = nullptr; r.out_score = nullptr; r.out_rows = 0; r.out_stride = 0;
+  } else if (p.mode == 0) {
+    r.K = p.k; r.out = outb; r.out_score = outsb; r.out_rows = p.g; r.out_stride = p.k;
+  } else {
+    r.K = p.c; r.out = p.cand + (size_t)b * p.c;
+    r.out_score = p.cand_score ? p.cand_score + (size_t)b * p.c : nullptr;
+    r.out_rows = 1; r.out_stride = p.c;
+    gd.n_cand = min(p.c, n0);
+  }
+  rows[b] = r;
+  groups[b] = gd;
+  for (int i = 0; i < p.g; ++i) {
+    RowDesc dr;
+    dr.q = (const char*)p.q + ((size_t)b * p.g + i) * qrow;
+    dr.w = p.w + ((size_t)b * p.g + i) * kHeads;
+    dr.qscale = p.qscale ? p.qscale + ((size_t)b * p.g + i) * kHeads : nullptr;
+    dr.kbase = kb;
+    dr.kscale = ksb;
+    dr.n_vis = p0 + i + 1;
+    dr.K = guarded ? p.k : 0;
+    dr.out = outb + (size_t)i * p.k;
+    dr.out_score = outsb ? outsb + (size_t)i * p.k : nullptr;
+    dr.out_rows = 1;
+    dr.out_stride = p.k;
+    rows[p.B + b * p.g + i] = dr;
+  }
+}
+
+void launch_plan_decode(const DecodePlan& p, RowDesc* rows, GroupDesc* groups, cudaStream_t st) {
+  plan_decode_kernel<<<(p.B + 127) / 128, 128, 0, st>>>(p, rows, groups);
+  ++launch_counter();
+}
+
+}  // namespace pivot

@@ -1,0 +1,134 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded
+inputs, element by element, under the acceptance rule of oracle/acceptance.py."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import acceptance as acc
+from oracle import pivot_oracle as po
+from paper_2607_24593_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pv():
+    from paper_2607_24593_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def gu():
+    import gpu_util
+    return gpu_util
+
+
+def _report(name, t):
+    print(f"\n[{name}] rows={t.rows} exact={t.exact_rows} band_swaps={t.band_swaps} "
+          f"scores={t.scores_checked} worst_score_err={t.max_score_err:.3f} x tol")
+
+
+# ---------------------------------------------------------------- small prefill, all groups
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+@pytest.mark.parametrize("mode", [po.MODE_REUSE, po.MODE_REFINE])
+@pytest.mark.parametrize("seed", [20260724, 11, 12])
+def test_prefill_small_full_parity(pv, gu, dtype, mode, seed):
+    """Config 1: L=2048, g=4, k=256, c=512 -- every group against the oracle."""
+    L, g, c, k = 2048, 4, 512, 256
+    x = inputs.make_prefill(L, dtype=dtype, seed=seed)
+    out, sc, cand, cs = gu.run_prefill(x, g=g, c=c, k=k, mode=mode)
+    t = acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=None, out_idx=out,
+                          out_scores=sc, cand=cand, cand_scores=cs)
+    _report(f"prefill {dtype} mode={mode} seed={seed}", t)
+    assert t.exact_rows >= 0.95 * t.rows
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+def test_dense_small_full_parity(pv, gu, dtype):
+    L, k = 1536, 256
+    x = inputs.make_prefill(L, dtype=dtype, seed=5)
+    out, sc = gu.run_dense(x, k=k)
+    t = acc.check_dense(x.codes(), k=k, out_idx=out, out_scores=sc)
+    _report(f"dense {dtype}", t)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+@pytest.mark.parametrize("L,g,c,k,guard", [
+    (1000, 4, 512, 256, None),     # ragged last tile
+    (1027, 3, 300, 77, None),      # odd sizes, short last group (m = 1)
+    (517, 8, 128, 128, 0),         # c == k, guardrail off: early groups see fewer than c keys
+    (260, 5, 64, 16, 1),           # tiny selection
+    (130, 1, 32, 8, None),         # g = 1
+    (64, 4, 512, 256, None),       # everything guarded, fewer keys than k
+    (1, 4, 8, 4, None),            # single token
+])
+def test_prefill_edge_shapes(pv, gu, dtype, L, g, c, k, guard):
+    x = inputs.make_prefill(L, dtype=dtype, seed=L)
+    for mode in (po.MODE_REUSE, po.MODE_REFINE):
+        out, sc, cand, cs = gu.run_prefill(x, g=g, c=c, k=k, mode=mode, guard_len=guard)
+        t = acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=guard, out_idx=out,
+                              out_scores=sc, cand=cand, cand_scores=cs)
+        _report(f"edge L={L} g={g} c={c} k={k} {dtype} mode={mode}", t)
+
+
+def test_group_of_one_equals_dense_on_gpu(pv, gu):
+    """Appendix A: g = 1 recovers the dense indexer -- on the GPU outputs themselves."""
+    x = inputs.make_prefill(700, dtype="bf16", seed=9)
+    a, _, _, _ = gu.run_prefill(x, g=1, c=128, k=64, mode=po.MODE_REUSE)
+    b, _ = gu.run_dense(x, k=64)
+    for t in range(700):
+        assert set(a[t].tolist()) == set(b[t].tolist())
+
+
+def test_ties_all_equal_scores(pv, gu):
+    """Zero gates make every score 0: the total order falls back to the lowest indices."""
+    x = inputs.make_prefill(900, dtype="bf16", seed=4)
+    x.w.zero_()
+    out, sc, cand, cs = gu.run_prefill(x, g=4, c=256, k=128, mode=po.MODE_REFINE)
+    for t in range(900):
+        n = min(128, t + 1)
+        assert sorted(out[t, :n].tolist()) == list(range(n))
+        assert (out[t, n:] == -1).all()
+
+
+def test_pool_variants(pv, gu):
+    x = inputs.make_prefill(600, dtype="fp8", seed=8)
+    for pool, name in ((pv.POOL_FIRST, "first"), (pv.POOL_LAST, "last")):
+        out, sc, cand, cs = gu.run_prefill(x, g=4, c=128, k=64, mode=po.MODE_REFINE, pool=pool)
+        acc.check_prefill(x.codes(), g=4, c=128, k=64, mode=po.MODE_REFINE, guard_len=None, out_idx=out,
+                          out_scores=sc, cand=cand, cand_scores=cs, pool=name)
+
+
+# ---------------------------------------------------------------- decode
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+@pytest.mark.parametrize("mode", [po.MODE_REUSE, po.MODE_REFINE])
+def test_decode_small_parity(pv, gu, dtype, mode):
+    x = inputs.make_decode(6, 2, 300, 3000, dtype=dtype, seed=21)
+    out, sc, cand, cs = gu.run_decode(x, c=512, k=256, mode=mode)     # mixes guarded and proxy sequences
+    t = acc.check_decode(x.codes(), c=512, k=256, mode=mode, guard_len=None, out_idx=out, out_scores=sc,
+                         cand=cand, cand_scores=cs)
+    _report(f"decode {dtype} mode={mode}", t)
+
+
+def test_decode_group_of_four(pv, gu):
+    x = inputs.make_decode(3, 4, 2000, 2600, dtype="fp8", seed=22)
+    out, sc, cand, cs = gu.run_decode(x, c=256, k=128, mode=po.MODE_REFINE)
+    acc.check_decode(x.codes(), c=256, k=128, mode=po.MODE_REFINE, guard_len=None, out_idx=out,
+                     out_scores=sc, cand=cand, cand_scores=cs)
+
+
+# ---------------------------------------------------------------- argument errors (host side)
+
+def test_argument_errors(pv):
+    x = inputs.make_prefill(64, dtype="bf16", seed=1)
+    q, w, k = x.q.cuda(), x.w.cuda(), x.k.cuda()
+    out = torch.empty((64, 8), dtype=torch.int32, device="cuda")
+    with pytest.raises(pv.PivotError, match="invalid"):
+        pv.pivot_index_prefill(q, w, k, 64, 64, 128, 4, 4, 8, pv.REFINE, out)      # k > c
+    with pytest.raises(pv.PivotError, match="unsupported"):
+        pv.pivot_index_prefill(q, w, k, 64, 32, 128, 4, 16, 8, pv.REFINE, out)     # H_I != 64
+    with pytest.raises(pv.PivotError, match="workspace"):
+        small = torch.empty(256, dtype=torch.uint8, device="cuda")
+        pv.pivot_index_prefill(q, w, k, 64, 64, 128, 4, 16, 8, pv.REFINE, out, workspace=small)
