@@ -80,6 +80,9 @@ typedef struct pivot_tensor {
  *                 and guarded rows Eq. 1.
  *   dbg_cand_scores optional [n_groups, c] fp32: proxy score (Eq. 5) of each dbg_cand entry.
  *   workspace     scratch of at least pivot_workspace_bytes(...) bytes, 256-byte aligned.
+ *   impl          0: tensor-core kernels (tcgen05; the product path).  1: the plain CUDA-core
+ *                 kernels that compute the same thing one key per thread -- a slow on-device
+ *                 cross-check, not a fallback: nothing selects it automatically.
  */
 typedef struct pivot_opts {
   int guard_len;
@@ -89,6 +92,7 @@ typedef struct pivot_opts {
   float* dbg_cand_scores;
   void* workspace;
   size_t workspace_bytes;
+  int impl;
 } pivot_opts;
 
 /* Bytes of scratch a call with these sizes needs.  rows = L for prefill / dense, B*g for decode;
@@ -156,6 +160,16 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
 /* Reads (and clears) the device status word of the workspace last used on this device after
  * synchronising `stream`.  0 = no device-side condition. */
 int pivot_device_status(pivot_stream_t stream, int* status);
+
+/*
+ * Per-stage timing, off by default.  While enabled, every call records CUDA events on its own
+ * stream around its stages; pivot_stage_times synchronises on the last call's final event and
+ * returns elapsed milliseconds: ms[0] proxy build (Eq. 4), ms[1] planner, ms[2] shared scan +
+ * streaming select (Eq. 5-7, and the dense rows), ms[3] gather + re-score + top-k (Eq. 8-9),
+ * ms[4] the whole call.  n must be at least 5.  Not thread-safe.
+ */
+int pivot_stage_timing(int enable);
+int pivot_stage_times(float* ms, int n);
 
 /* Kernel launches issued by the library since the last call of this function (host counter). */
 long long pivot_launch_count_reset(void);

@@ -24,7 +24,7 @@ SYMBOLS = [
     "pivot_workspace_bytes", "pivot_set_workspace", "pivot_index_prefill", "pivot_index_prefill_ex",
     "pivot_index_decode", "pivot_index_decode_ex", "dense_index", "dense_index_ex",
     "pivot_prefill_host_arena_bytes", "pivot_index_prefill_host", "pivot_device_status",
-    "pivot_launch_count_reset", "pivot_status_str", "pivot_last_cuda_error",
+    "pivot_stage_timing", "pivot_stage_times", "pivot_launch_count_reset", "pivot_status_str", "pivot_last_cuda_error",
 ]
 
 
@@ -35,7 +35,7 @@ class pivot_tensor(C.Structure):
 class pivot_opts(C.Structure):
     _fields_ = [("guard_len", C.c_int), ("pool", C.c_int), ("dbg_cand", C.c_void_p),
                 ("dbg_scores", C.c_void_p), ("dbg_cand_scores", C.c_void_p),
-                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("impl", C.c_int)]
 
 
 class PivotError(RuntimeError):
@@ -62,6 +62,8 @@ def _load():
     lib.pivot_prefill_host_arena_bytes.argtypes = [I, I, I, I, I, I, I]
     lib.pivot_index_prefill_host.argtypes = [T, P, T, I, I, I, I, I, I, I, P, P, S, P]
     lib.pivot_device_status.argtypes = [P, C.POINTER(C.c_int)]
+    lib.pivot_stage_timing.argtypes = [I]
+    lib.pivot_stage_times.argtypes = [C.POINTER(C.c_float), I]
     lib.pivot_launch_count_reset.restype = C.c_longlong
     lib.pivot_status_str.restype = C.c_char_p
     lib.pivot_status_str.argtypes = [I]
@@ -97,10 +99,13 @@ def _stream(stream) -> int:
     return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
 
 
-def _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace) -> pivot_opts:
+IMPL_TENSOR_CORE, IMPL_CUDA_CORE = 0, 1
+
+
+def _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl=0) -> pivot_opts:
     p = lambda t: None if t is None else t.data_ptr()
     return pivot_opts(-1 if guard_len is None else guard_len, pool, p(dbg_cand), p(dbg_scores),
-                      p(dbg_cand_scores), p(workspace), 0 if workspace is None else workspace.numel())
+                      p(dbg_cand_scores), p(workspace), 0 if workspace is None else workspace.numel(), impl)
 
 
 def pivot_workspace_bytes(rows: int, n_groups: int, c: int, k: int) -> int:
@@ -133,24 +138,24 @@ def ensure_workspace(rows: int, n_groups: int, c: int, k: int, device="cuda") ->
 
 def pivot_index_prefill(q, w, kcache, L, H_I, d, g, c, k, mode, out_idx, stream=None, *,
                         q_scale=None, k_scale=None, guard_len=None, pool=POOL_MEAN, dbg_cand=None,
-                        dbg_scores=None, dbg_cand_scores=None, workspace=None):
+                        dbg_scores=None, dbg_cand_scores=None, workspace=None, impl=0):
     tq, tk = _tensor(q, q_scale), _tensor(kcache, k_scale)
     assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and out_idx.numel() >= L * k
     if workspace is None:
         ensure_workspace(L, (L + g - 1) // g, c, k, q.device)
-    o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace)
+    o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl)
     _check(lib.pivot_index_prefill_ex(C.byref(tq), w.data_ptr(), C.byref(tk), L, H_I, d, g, c, k, mode,
                                       out_idx.data_ptr(), _stream(stream), C.byref(o)))
     return out_idx
 
 
 def dense_index(q, w, kcache, L, H_I, d, k, out_idx, stream=None, *, q_scale=None, k_scale=None,
-                dbg_scores=None, workspace=None):
+                dbg_scores=None, workspace=None, impl=0):
     tq, tk = _tensor(q, q_scale), _tensor(kcache, k_scale)
     assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and out_idx.numel() >= L * k
     if workspace is None:
         ensure_workspace(L, L, k, k, q.device)
-    o = _opts(None, POOL_MEAN, None, dbg_scores, None, workspace)
+    o = _opts(None, POOL_MEAN, None, dbg_scores, None, workspace, impl)
     _check(lib.dense_index_ex(C.byref(tq), w.data_ptr(), C.byref(tk), L, H_I, d, k, out_idx.data_ptr(),
                               _stream(stream), C.byref(o)))
     return out_idx
@@ -158,13 +163,13 @@ def dense_index(q, w, kcache, L, H_I, d, k, out_idx, stream=None, *, q_scale=Non
 
 def pivot_index_decode(q, w, kcache, pos0, B, Lmax, H_I, d, g, c, k, mode, out_idx, stream=None, *,
                        q_scale=None, k_scale=None, guard_len=None, pool=POOL_MEAN, dbg_cand=None,
-                       dbg_scores=None, dbg_cand_scores=None, workspace=None):
+                       dbg_scores=None, dbg_cand_scores=None, workspace=None, impl=0):
     tq, tk = _tensor(q, q_scale), _tensor(kcache, k_scale)
     assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and pos0.dtype == torch.int32
     assert out_idx.numel() >= B * g * k
     if workspace is None:
         ensure_workspace(B * g, B, c, k, q.device)
-    o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace)
+    o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl)
     _check(lib.pivot_index_decode_ex(C.byref(tq), w.data_ptr(), C.byref(tk), pos0.data_ptr(), B, Lmax,
                                      H_I, d, g, c, k, mode, out_idx.data_ptr(), _stream(stream), C.byref(o)))
     return out_idx
@@ -191,6 +196,17 @@ def pivot_device_status(stream=None) -> int:
     st = C.c_int(0)
     _check(lib.pivot_device_status(_stream(stream), C.byref(st)))
     return st.value
+
+
+def pivot_stage_timing(enable: bool):
+    _check(lib.pivot_stage_timing(1 if enable else 0))
+
+
+def pivot_stage_times() -> dict:
+    """Elapsed ms of the last call's stages (needs pivot_stage_timing(True) before the call)."""
+    ms = (C.c_float * 5)()
+    _check(lib.pivot_stage_times(ms, 5))
+    return dict(zip(("proxy_build", "plan", "scan_select", "refine", "total"), [float(v) for v in ms]))
 
 
 def pivot_launch_count_reset() -> int:

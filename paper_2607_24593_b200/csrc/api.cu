@@ -95,6 +95,13 @@ Workspace carve_workspace(void* base, int rows, int n_groups, int c, int k) {
   return w;
 }
 
+bool g_timing = false;
+cudaEvent_t g_ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+bool g_ev_valid = false;
+inline void mark(int i, cudaStream_t st) {
+  if (g_timing) { cudaEventRecord(g_ev[i], st); if (i == 4) g_ev_valid = true; }
+}
+
 int check_cuda(cudaError_t e) {
   if (e == cudaSuccess) return PIVOT_OK;
   g_last_cuda = (int)e;
@@ -155,11 +162,22 @@ int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, i
   p.n_proxy = nG - first_group;
 
   if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 2 * sizeof(int), st)))) return rc;
+  mark(0, st);
   launch_proxy_build(q->data, q->scale, w, ws.proxy_q, ws.proxy_w, L, g, first_group, p.n_proxy,
                      q->dtype, o ? o->pool : 0, st);
+  mark(1, st);
   launch_plan_prefill(p, ws.rows, ws.groups, st);
-  launch_scan_simt(ws.rows, p.n_dense + p.n_proxy, q->dtype, ws.scan, st);
+  mark(2, st);
+  if (o && o->impl == 1) {
+    launch_scan_simt(ws.rows, p.n_dense + p.n_proxy, q->dtype, ws.scan, st);
+  } else {
+    ScanOperands op{kc->data, L, q->data, L, ws.proxy_q, p.n_proxy, q->dtype};
+    if ((rc = check_cuda(launch_scan_tc(op, ws.rows, p.n_dense + p.n_proxy, 4, ws.scan, sm_count(), st))))
+      return rc;
+  }
+  mark(3, st);
   if (mode == PIVOT_REFINE) launch_refine_simt(ws.groups, p.n_proxy, q->dtype, ws.scan, st);
+  mark(4, st);
   return check_cuda(cudaGetLastError());
 }
 
@@ -186,7 +204,8 @@ int pivot_index_prefill_ex(const pivot_tensor* q, const float* w, const pivot_te
   int rc = check_common(q, w, kcache, H_I, d, c, k, mode, out_idx);
   if (rc) return rc;
   if (L < 1 || g < 1) return PIVOT_ERR_INVALID_ARG;
-  if (opts && (opts->pool < 0 || opts->pool > 2)) return PIVOT_ERR_INVALID_ARG;
+  if (opts && (opts->pool < 0 || opts->pool > 2 || opts->impl < 0 || opts->impl > 1))
+    return PIVOT_ERR_INVALID_ARG;
   return run_prefill(q, w, kcache, L, g, c, k, mode, false, out_idx, (cudaStream_t)stream, opts);
 }
 
@@ -233,11 +252,21 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
   p.B = B; p.Lmax = Lmax; p.g = g; p.c = c; p.k = k; p.mode = mode; p.dtype = q->dtype;
   p.guard_len = (o && o->guard_len >= 0) ? o->guard_len : c;
   if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 2 * sizeof(int), st)))) return rc;
+  mark(0, st);
   launch_proxy_build(q->data, q->scale, w, ws.proxy_q, ws.proxy_w, B * g, g, 0, B, q->dtype,
                      o ? o->pool : 0, st);
+  mark(1, st);
   launch_plan_decode(p, ws.rows, ws.groups, st);
-  launch_scan_simt(ws.rows, B + B * g, q->dtype, ws.scan, st);
+  mark(2, st);
+  if (o && o->impl == 1) {
+    launch_scan_simt(ws.rows, B + B * g, q->dtype, ws.scan, st);
+  } else {
+    ScanOperands op{kcache->data, (long long)B * Lmax, q->data, B * g, ws.proxy_q, B, q->dtype};
+    if ((rc = check_cuda(launch_scan_tc(op, ws.rows, B + B * g, 1, ws.scan, sm_count(), st)))) return rc;
+  }
+  mark(3, st);
   if (mode == PIVOT_REFINE) launch_refine_simt(ws.groups, B, q->dtype, ws.scan, st);
+  mark(4, st);
   return check_cuda(cudaGetLastError());
 }
 
@@ -309,6 +338,27 @@ int pivot_device_status(pivot_stream_t stream, int* status) {
   int rc = check_cuda(cudaStreamSynchronize((cudaStream_t)stream));
   if (rc) return rc;
   return check_cuda(cudaMemcpy(status, p, sizeof(int), cudaMemcpyDeviceToHost));
+}
+
+int pivot_stage_timing(int enable) {
+  if (enable && !g_ev[0]) {
+    for (int i = 0; i < 6; ++i) {
+      int rc = check_cuda(cudaEventCreate(&g_ev[i]));
+      if (rc) return rc;
+    }
+  }
+  g_timing = enable != 0;
+  g_ev_valid = false;
+  return PIVOT_OK;
+}
+
+int pivot_stage_times(float* ms, int n) {
+  if (!ms || n < 5 || !g_ev_valid) return PIVOT_ERR_INVALID_ARG;
+  int rc = check_cuda(cudaEventSynchronize(g_ev[4]));
+  if (rc) return rc;
+  for (int i = 0; i < 4; ++i)
+    if ((rc = check_cuda(cudaEventElapsedTime(&ms[i], g_ev[i], g_ev[i + 1])))) return rc;
+  return check_cuda(cudaEventElapsedTime(&ms[4], g_ev[0], g_ev[4]));
 }
 
 long long pivot_launch_count_reset(void) {

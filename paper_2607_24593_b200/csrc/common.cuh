@@ -53,6 +53,9 @@ struct RowDesc {
   float* out_score;     // optional, same layout
   int out_rows;
   int out_stride;
+  int q_map;            // which query tensor map holds q: 0 raw queries, 1 proxies
+  int q_row;            // query row (units of H x d) inside that tensor
+  int k_row0;           // first row of this sequence's keys inside the key-cache tensor
 };
 
 }  // namespace pivot

@@ -66,6 +66,17 @@ void launch_plan_decode(const DecodePlan& p, RowDesc* rows, GroupDesc* groups, c
 void launch_scan_simt(const RowDesc* rows, int n_rows, int dtype, const ScanScratch& s, cudaStream_t st);
 void launch_refine_simt(const GroupDesc* groups, int n_groups, int dtype, const ScanScratch& s, cudaStream_t st);
 
+// Operand tensors of a tensor-core scan, for the TMA tensor maps.
+struct ScanOperands {
+  const void* kc; long long k_rows;        // key cache [k_rows, d]
+  const void* q; int q_rows;               // raw queries [q_rows, H, d]
+  const void* proxy_q; int proxy_rows;     // proxies [proxy_rows, H, d]
+  int dtype;
+};
+// rows_per_block consecutive scan rows share one key stream (4 in prefill, 1 in decode).
+cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_rows, int rows_per_block,
+                           const ScanScratch& s, int sms, cudaStream_t st);
+
 long long& launch_counter();
 
 }  // namespace pivot

@@ -24,6 +24,7 @@ __global__ void plan_prefill_kernel(PrefillPlan p, RowDesc* rows, GroupDesc* gro
     r.out_score = p.out_score ? p.out_score + (size_t)i * p.k : nullptr;
     r.out_rows = 1;
     r.out_stride = p.k;
+    r.q_map = 0; r.q_row = i; r.k_row0 = 0;
     rows[i] = r;
   } else if (i < p.n_dense + p.n_proxy) {
     const int pr = i - p.n_dense;
@@ -36,6 +37,7 @@ __global__ void plan_prefill_kernel(PrefillPlan p, RowDesc* rows, GroupDesc* gro
     r.kbase = p.kc;
     r.kscale = p.kscale;
     r.n_vis = t0 + 1;
+    r.q_map = 1; r.q_row = pr; r.k_row0 = 0;
     if (p.mode == 0) {   // Reuse: the proxy top-k goes to every member (Eq. 6)
       r.K = p.k;
       r.out = p.out + (size_t)t0 * p.k;
@@ -97,6 +99,7 @@ __global__ void plan_decode_kernel(DecodePlan p, RowDesc* rows, GroupDesc* group
   r.kbase = kb;
   r.kscale = ksb;
   r.n_vis = n0;
+  r.q_map = 1; r.q_row = b; r.k_row0 = b * p.Lmax;
   GroupDesc gd;
   gd.q = (const char*)p.q + (size_t)b * p.g * qrow;
   gd.w = p.w + (size_t)b * p.g * kHeads;
@@ -136,6 +139,7 @@ __global__ void plan_decode_kernel(DecodePlan p, RowDesc* rows, GroupDesc* group
     dr.out_score = outsb ? outsb + (size_t)i * p.k : nullptr;
     dr.out_rows = 1;
     dr.out_stride = p.k;
+    dr.q_map = 0; dr.q_row = b * p.g + i; dr.k_row0 = b * p.Lmax;
     rows[p.B + b * p.g + i] = dr;
   }
 }

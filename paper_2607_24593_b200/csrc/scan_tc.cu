@@ -1,0 +1,448 @@
+// Kernels 2+3: shared prefix scan on tcgen05 tensor cores with the streaming top-K select
+// fused behind it, so the (rows x keys) score matrix never reaches HBM.
+//
+// Eq. 5 / Eq. 1 as a dense contraction: a tile is 128 keys (MMA M, one key per TMEM lane) by
+// NROWS x 64 heads (MMA N) by d = 128 (MMA K).  Keys stream through a TMA-fed shared-memory
+// ring; the query block (NROWS rows = NROWS consecutive proxies or queries) sits in shared
+// memory for the whole scan of its prefix.  The accumulator lives in TMEM, double-buffered:
+// while the tensor core fills one buffer, the epilogue warps drain the other -- each thread owns
+// one key, applies ReLU, the gate-weighted head sum, the key scale (Appendix A) and the causal
+// cut, and feeds the score to the row's streaming select (filter by the running K-th-best
+// threshold, append to an L2-resident candidate buffer, exact radix compaction when it fills).
+//
+// One persistent CTA per SM; warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner,
+// warps 2.. = epilogue (two warps per TMEM lane quarter, each pair of rows handled by its own
+// 128-thread team).  Row blocks are dealt to CTAs longest-first in snake order.
+#include <cuda.h>
+
+#include "kernels.h"
+#include "ptx.cuh"
+#include "select.cuh"
+
+namespace pivot {
+namespace {
+
+constexpr int TILE_KEYS = 128;
+constexpr int MAX_STAGES = 8;
+
+template <int DT, int NROWS>
+struct Cfg {
+  static constexpr bool FP8 = DT == DT_FP8;
+  static constexpr int ESZ = FP8 ? 1 : 2;
+  static constexpr int KHALVES = FP8 ? 1 : 2;                 // 128-byte K slices per row
+  static constexpr int HALF_TILE_BYTES = TILE_KEYS * 128;     // 16 KB: 128 keys x 128 B
+  static constexpr int STAGE_BYTES = KHALVES * HALF_TILE_BYTES;
+  static constexpr int QROW_HALF_BYTES = kHeads * 128;        // 8 KB: 64 heads x 128 B
+  static constexpr int QHALF_BYTES = NROWS * QROW_HALF_BYTES;
+  static constexpr int QBUF_BYTES = KHALVES * QHALF_BYTES;
+  static constexpr int N = NROWS * kHeads;
+  static constexpr int STAGES = FP8 ? 6 : (NROWS == 4 ? 2 : 4);
+  static constexpr int EPI_WARPS = NROWS == 4 ? 8 : 4;
+  static constexpr int ROWS_PER_TEAM = NROWS == 4 ? 2 : 1;
+  static constexpr int TEAMS = EPI_WARPS / 4;
+  static constexpr int THREADS = 64 + EPI_WARPS * 32;
+  static constexpr int TMEM_COLS = 2 * N < 32 ? 32 : 2 * N;
+  static constexpr int KSTEPS = 4;                            // 32 bytes of K per MMA
+  static constexpr uint32_t IDESC = ptx::make_idesc(FP8 ? 0u : 1u, TILE_KEYS, N);
+};
+
+struct Ctrl {
+  alignas(16) float w[4][kHeads];   // read as float4
+  uint64_t full[MAX_STAGES], empty[MAX_STAGES];
+  uint64_t q_full[2], q_empty[2], tmem_full[2], tmem_empty[2];
+  uint32_t tmem_base;
+  int abort;
+  int n_vis[4];
+  int K[4];
+  uint32_t count[4];
+  uint32_t thr[4];
+  int cur[4];
+  SelectSmem sel[2];
+};
+
+template <int DT, int NROWS>
+constexpr size_t smem_bytes() {
+  using C = Cfg<DT, NROWS>;
+  return 1024 + 2 * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(Ctrl);
+}
+
+// Block sequence of one CTA: blocks sorted longest-first are dealt in snake order.
+struct BlockIter {
+  int n_blocks, G, cta, round;
+  __device__ BlockIter(int nb, int g, int c) : n_blocks(nb), G(g), cta(c), round(0) {}
+  __device__ int next() {   // block index, or -1
+    const int pos = (round & 1) ? (G - 1 - cta) : cta;
+    const long long d = (long long)round * G + pos;
+    ++round;
+    if (d >= n_blocks) {
+      // a partial last round can still hold a block for this CTA on the other snake direction
+      return -1;
+    }
+    return n_blocks - 1 - (int)d;
+  }
+};
+
+__device__ __forceinline__ int block_tiles(const RowDesc* rows, int n_rows, int b, int nrows_blk, int* k_row0,
+                                           int* nv_max = nullptr) {
+  int mx = 0;
+  for (int r = 0; r < nrows_blk; ++r) {
+    const int ri = b * nrows_blk + r;
+    if (ri < n_rows) {
+      const int K = rows[ri].K;
+      const int nv = rows[ri].n_vis;
+      if (K > 0 && nv > mx) mx = nv;
+      if (r == 0) *k_row0 = rows[ri].k_row0;
+    }
+  }
+  if (nv_max) *nv_max = mx;
+  return (mx + TILE_KEYS - 1) / TILE_KEYS;
+}
+
+template <int DT, int NROWS>
+__global__ void __launch_bounds__(Cfg<DT, NROWS>::THREADS, 1)
+scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q0,
+                      const __grid_constant__ CUtensorMap tm_q1, const RowDesc* __restrict__ rows,
+                      int n_rows, ScanScratch sc) {
+  using C = Cfg<DT, NROWS>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* qbuf = smem;                                   // 2 x QBUF_BYTES
+  uint8_t* kring = smem + 2 * C::QBUF_BYTES;              // STAGES x STAGE_BYTES
+  Ctrl& ct = *reinterpret_cast<Ctrl*>(kring + C::STAGES * C::STAGE_BYTES);
+  volatile int* abort_flag = &ct.abort;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int n_blocks = (n_rows + NROWS - 1) / NROWS;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::STAGES; ++s) { ptx::mbar_init(&ct.full[s], 1); ptx::mbar_init(&ct.empty[s], 1); }
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(&ct.q_full[i], 1);
+      ptx::mbar_init(&ct.q_empty[i], 1);
+      ptx::mbar_init(&ct.tmem_full[i], 1);
+      ptx::mbar_init(&ct.tmem_empty[i], C::EPI_WARPS);
+    }
+    ct.abort = 0;
+    ptx::fence_barrier_init();
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(&ct.tmem_base, C::TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = ct.tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (ptx::elect_one()) {
+      ptx::prefetch_tensormap(&tm_k);
+      ptx::prefetch_tensormap(&tm_q0);
+      ptx::prefetch_tensormap(&tm_q1);
+      BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
+      uint32_t it = 0, blk = 0;
+      bool ok = true;
+      for (int b = bi.next(); b >= 0 && ok; b = bi.next()) {
+        int k_row0 = 0;
+        const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0);
+        if (ntiles == 0) continue;
+        const int qb = blk & 1;
+        ok = ptx::mbar_wait(&ct.q_empty[qb], ((blk >> 1) & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        int present = 0;
+        for (int r = 0; r < NROWS; ++r) present += (b * NROWS + r < n_rows) ? 1 : 0;
+        ptx::mbar_arrive_expect_tx(&ct.q_full[qb], present * C::KHALVES * C::QROW_HALF_BYTES);
+        for (int r = 0; r < NROWS; ++r) {
+          const int ri = b * NROWS + r;
+          if (ri >= n_rows) continue;
+          const CUtensorMap* tm = rows[ri].q_map ? &tm_q1 : &tm_q0;
+          const int y = rows[ri].q_row * kHeads;
+          for (int h = 0; h < C::KHALVES; ++h)
+            ptx::tma_load_2d(qbuf + qb * C::QBUF_BYTES + h * C::QHALF_BYTES + r * C::QROW_HALF_BYTES, tm,
+                             h * 64, y, &ct.q_full[qb]);
+        }
+        for (int t = 0; t < ntiles; ++t, ++it) {
+          const int s = it % C::STAGES;
+          const uint32_t ph = (it / C::STAGES) & 1;
+          ok = ptx::mbar_wait(&ct.empty[s], ph ^ 1, abort_flag);
+          if (!ok) break;
+          ptx::mbar_arrive_expect_tx(&ct.full[s], C::STAGE_BYTES);
+          for (int h = 0; h < C::KHALVES; ++h)
+            ptx::tma_load_2d(kring + s * C::STAGE_BYTES + h * C::HALF_TILE_BYTES, &tm_k, h * 64,
+                             k_row0 + t * TILE_KEYS, &ct.full[s]);
+        }
+        ++blk;
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (ptx::elect_one()) {
+      BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
+      uint32_t it = 0, blk = 0;
+      bool ok = true;
+      for (int b = bi.next(); b >= 0 && ok; b = bi.next()) {
+        int k_row0 = 0;
+        const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0);
+        if (ntiles == 0) continue;
+        const int qb = blk & 1;
+        ok = ptx::mbar_wait(&ct.q_full[qb], (blk >> 1) & 1, abort_flag);
+        if (!ok) break;
+        const uint32_t q_addr = ptx::smem_u32(qbuf + qb * C::QBUF_BYTES);
+        for (int t = 0; t < ntiles; ++t, ++it) {
+          const int s = it % C::STAGES;
+          const uint32_t ph = (it / C::STAGES) & 1;
+          const int buf = it & 1;
+          ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          ok = ptx::mbar_wait(&ct.full[s], ph, abort_flag);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          const uint32_t k_addr = ptx::smem_u32(kring + s * C::STAGE_BYTES);
+          const uint32_t d_tmem = tmem_base + buf * C::N;
+#pragma unroll
+          for (int h = 0; h < C::KHALVES; ++h)
+#pragma unroll
+            for (int ks = 0; ks < C::KSTEPS; ++ks) {
+              const uint64_t a = ptx::smem_desc_sw128(k_addr + h * C::HALF_TILE_BYTES + ks * 32);
+              const uint64_t bq = ptx::smem_desc_sw128(q_addr + h * C::QHALF_BYTES + ks * 32);
+              ptx::tc_mma<C::FP8>(d_tmem, a, bq, C::IDESC, (h | ks) ? 1u : 0u);
+            }
+          ptx::tc_commit(&ct.empty[s]);       // key stage free once these MMAs are done
+          ptx::tc_commit(&ct.tmem_full[buf]); // accumulator ready
+        }
+        ptx::tc_commit(&ct.q_empty[qb]);
+        ++blk;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue + select
+    const int ew = warp - 2;                       // 0 .. EPI_WARPS-1
+    const int team = ew >> 2;                      // which pair of rows
+    const int lq = warp & 3;                       // TMEM lane quarter this warp may read
+    const int key_in_tile = lq * 32 + lane;
+    const int tt = (ew & 3) * 32 + lane;           // rank inside the team (0..127)
+    const Team tm{tt, 128, 1 + team};
+    SelectSmem& sel = ct.sel[team];
+    const size_t cta_base = (size_t)blockIdx.x * NROWS * 2 * sc.cap;
+    BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
+    uint32_t it = 0;
+    // A failed wait never changes this role's control flow (the team barriers below must stay
+    // matched); once the abort flag is up every later wait returns at once.
+    for (int b = bi.next(); b >= 0; b = bi.next()) {
+      int k_row0 = 0, nv_max = 0;
+      const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0, &nv_max);
+      if (ntiles == 0) continue;
+      // ---- per-block state of this team's rows
+      tm.sync();
+      const float* kscale = nullptr;
+      {
+        const int rl = tt >> 6, j = tt & 63;
+        if (rl < C::ROWS_PER_TEAM) {
+          const int r = team * C::ROWS_PER_TEAM + rl;
+          const int ri = b * NROWS + r;
+          float wv = 0.f;
+          if (ri < n_rows && rows[ri].K > 0) {
+            wv = rows[ri].w[j];
+            if (rows[ri].qscale) wv = __fmul_rn(wv, rows[ri].qscale[j]);
+          }
+          ct.w[r][j] = wv;
+          if (j == 0) {
+            const bool live = ri < n_rows && rows[ri].K > 0;
+            ct.n_vis[r] = live ? rows[ri].n_vis : 0;
+            ct.K[r] = live ? rows[ri].K : 0;
+            ct.count[r] = 0;
+            ct.thr[r] = 0;
+            ct.cur[r] = 0;
+          }
+        }
+        const int r0 = b * NROWS;
+        kscale = rows[r0].kscale;
+      }
+      tm.sync();
+      for (int t = 0; t < ntiles; ++t, ++it) {
+        // ---- make room: exact compaction of a row whose buffer could overflow in this tile
+#pragma unroll
+        for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
+          const int r = team * C::ROWS_PER_TEAM + rl;
+          if ((int)ct.count[r] + TILE_KEYS > sc.cap) {
+            const int n = (int)ct.count[r];
+            const int cur = ct.cur[r];
+            uint32_t* kb = sc.cand_key + cta_base + (size_t)(r * 2) * sc.cap;
+            int32_t* ib = sc.cand_idx + cta_base + (size_t)(r * 2) * sc.cap;
+            tm.sync();
+            team_select_topk(tm, sel, kb + cur * sc.cap, ib + cur * sc.cap, n, ct.K[r],
+                             kb + (cur ^ 1) * sc.cap, ib + (cur ^ 1) * sc.cap, nullptr, &ct.thr[r]);
+            if (tt == 0) { ct.count[r] = (uint32_t)ct.K[r]; ct.cur[r] = cur ^ 1; }
+            tm.sync();
+          }
+        }
+        const int buf = it & 1;
+        const int s_key = t * TILE_KEYS + key_in_tile;
+        const float ksv = (kscale && s_key < nv_max) ? kscale[s_key] : 0.f;
+        (void)ptx::mbar_wait(&ct.tmem_full[buf], (it >> 1) & 1, abort_flag);
+        ptx::tc_fence_after();
+        float score[C::ROWS_PER_TEAM];
+#pragma unroll
+        for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
+          const int r = team * C::ROWS_PER_TEAM + rl;
+          const uint32_t taddr = tmem_base + ((uint32_t)(lq * 32) << 16) + buf * C::N + r * kHeads;
+          float acc = 0.f;
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            uint32_t v[32];
+            ptx::tmem_ld_32x32(taddr + half * 32, v);
+            ptx::tmem_wait_ld();
+            const float4* wp = reinterpret_cast<const float4*>(&ct.w[r][half * 32]);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float4 wv = wp[j];
+              acc = fmaf(wv.x, fmaxf(__uint_as_float(v[4 * j]), 0.f), acc);
+              acc = fmaf(wv.y, fmaxf(__uint_as_float(v[4 * j + 1]), 0.f), acc);
+              acc = fmaf(wv.z, fmaxf(__uint_as_float(v[4 * j + 2]), 0.f), acc);
+              acc = fmaf(wv.w, fmaxf(__uint_as_float(v[4 * j + 3]), 0.f), acc);
+            }
+          }
+          score[rl] = acc;
+        }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
+        // ---- filter + append
+#pragma unroll
+        for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
+          const int r = team * C::ROWS_PER_TEAM + rl;
+          const float sv = kscale ? score[rl] * ksv : score[rl];
+          const uint32_t key = score_to_key(sv);
+          const bool take = s_key < ct.n_vis[r] && key > ct.thr[r];
+          const uint32_t m = __ballot_sync(0xffffffffu, take);
+          if (m) {
+            uint32_t pos = 0;
+            const int leader = __ffs(m) - 1;
+            if (lane == leader) pos = atomicAdd(&ct.count[r], (uint32_t)__popc(m));
+            pos = __shfl_sync(0xffffffffu, pos, leader);
+            if (take) {
+              const uint32_t p = pos + __popc(m & ((1u << lane) - 1u));
+              const size_t o = cta_base + (size_t)(r * 2 + ct.cur[r]) * sc.cap + p;
+              sc.cand_key[o] = key;
+              sc.cand_idx[o] = s_key;
+            }
+          }
+        }
+        tm.sync();
+      }
+      // ---- end of the block: final exact select per row, then pad / replicate
+#pragma unroll
+      for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
+        const int r = team * C::ROWS_PER_TEAM + rl;
+        const int ri = b * NROWS + r;
+        const int K = ct.K[r];
+        if (K <= 0) continue;
+        const RowDesc rd = rows[ri];
+        const int n = (int)ct.count[r];
+        const uint32_t* kb = sc.cand_key + cta_base + (size_t)(r * 2 + ct.cur[r]) * sc.cap;
+        const int32_t* ib = sc.cand_idx + cta_base + (size_t)(r * 2 + ct.cur[r]) * sc.cap;
+        int n_valid = n;
+        if (n > K) {
+          team_select_topk(tm, sel, kb, ib, n, K, nullptr, rd.out, rd.out_score, nullptr);
+          n_valid = K;
+        } else {
+          for (int i = tt; i < n; i += 128) {
+            rd.out[i] = ib[i];
+            if (rd.out_score) rd.out_score[i] = key_to_score(kb[i]);
+          }
+        }
+        tm.sync();
+        for (int i = n_valid + tt; i < K; i += 128) {
+          rd.out[i] = -1;
+          if (rd.out_score) rd.out_score[i] = -INFINITY;
+        }
+        tm.sync();
+        for (int rr = 1; rr < rd.out_rows; ++rr)
+          for (int i = tt; i < K; i += 128) {
+            rd.out[(size_t)rr * rd.out_stride + i] = rd.out[i];
+            if (rd.out_score) rd.out_score[(size_t)rr * rd.out_stride + i] = rd.out_score[i];
+          }
+      }
+    }
+  }
+  // ------------------------------------------------------------------ teardown
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  if (warp == 1) ptx::tmem_dealloc(tmem_base, C::TMEM_COLS);
+  if (threadIdx.x == 0 && ct.abort) set_status(sc.status, DEV_WAIT_EXPIRED);
+}
+
+// ---------------------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// 2-D map over a row-major [rows, 128] operand tensor; box = 128 bytes x box_rows, 128B swizzle.
+bool make_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const bool fp8 = dtype == DT_FP8;
+  cuuint64_t dims[2] = {(cuuint64_t)kDim, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)(kDim * (fp8 ? 1 : 2))};
+  cuuint32_t box[2] = {(cuuint32_t)(fp8 ? 128 : 64), (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, dims,
+            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int DT, int NROWS>
+cudaError_t launch_one(const CUtensorMap& mk, const CUtensorMap& mq0, const CUtensorMap& mq1,
+                       const RowDesc* rows, int n_rows, const ScanScratch& s, int sms, cudaStream_t st) {
+  using C = Cfg<DT, NROWS>;
+  auto kern = scan_select_tc_kernel<DT, NROWS>;
+  static bool attr_set = false;
+  const size_t smem = smem_bytes<DT, NROWS>();
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int n_blocks = (n_rows + NROWS - 1) / NROWS;
+  const int grid = n_blocks < sms ? n_blocks : sms;
+  kern<<<grid, C::THREADS, smem, st>>>(mk, mq0, mq1, rows, n_rows, s);
+  ++launch_counter();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_rows, int rows_per_block,
+                           const ScanScratch& s, int sms, cudaStream_t st) {
+  if (n_rows <= 0) return cudaSuccess;
+  CUtensorMap mk, mq0, mq1;
+  if (!make_map(&mk, op.kc, op.k_rows, op.dtype, TILE_KEYS) ||
+      !make_map(&mq0, op.q, (long long)op.q_rows * kHeads, op.dtype, kHeads) ||
+      !make_map(&mq1, op.proxy_q, (long long)(op.proxy_rows > 0 ? op.proxy_rows : 1) * kHeads, op.dtype, kHeads))
+    return cudaErrorInvalidValue;
+  if (op.dtype == DT_FP8) {
+    return rows_per_block == 4 ? launch_one<DT_FP8, 4>(mk, mq0, mq1, rows, n_rows, s, sms, st)
+                               : launch_one<DT_FP8, 1>(mk, mq0, mq1, rows, n_rows, s, sms, st);
+  }
+  return rows_per_block == 4 ? launch_one<DT_BF16, 4>(mk, mq0, mq1, rows, n_rows, s, sms, st)
+                             : launch_one<DT_BF16, 1>(mk, mq0, mq1, rows, n_rows, s, sms, st);
+}
+
+}  // namespace pivot

@@ -12,7 +12,7 @@ namespace pivot {
 constexpr int SIMT_THREADS = 256;
 
 struct RowSmem {
-  float q[kHeads][kDim];   // decoded query codes
+  alignas(16) float q[kHeads][kDim];   // decoded query codes (read as float4)
   float w[kHeads];         // effective gate
   SelectSmem sel;
   uint32_t count;          // entries in the current candidate buffer
