@@ -1,0 +1,309 @@
+#!/usr/bin/env python
+"""Benchmark of the PIVOT group-shared indexer on B200.
+
+A "step" is one pass of the whole hot path (proxy build, shared scan + streaming select,
+gather + re-score + top-k, guarded dense rows) over one synthetic request.  Default workload:
+L = 131072 positions, FP8 e4m3 queries/keys with fp32 scales, Refine, g = 4, c = 4096, k = 2048
+(the configuration the headline metric "indexed query tokens/s" is quoted on).
+
+  python bench.py --gpus N --steps K --warmup W          the CUDA path (one JSON line)
+  python bench.py --impl reference ...                   the CPU oracle on a bounded sample
+
+With N > 1 (torchrun) every rank indexes its own request of the same shape (requests are
+independent: no data-path collective) and the line reports the aggregate -- weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_24593_b200 import inputs  # noqa: E402
+
+WORKLOADS = {
+    # name: (L, dtype, g, c, k, mode)
+    "prefill_128k_fp8_refine_g4": (131072, "fp8", 4, 4096, 2048, 1),
+    "prefill_128k_fp8_reuse_g4": (131072, "fp8", 4, 4096, 2048, 0),
+    "prefill_128k_fp8_refine_g8": (131072, "fp8", 8, 4096, 2048, 1),
+    "prefill_32k_bf16_refine_g4": (32768, "bf16", 4, 4096, 2048, 1),
+    "prefill_2k_bf16_refine_g4": (2048, "bf16", 4, 512, 256, 1),
+    "prefill_256k_fp8_refine_g4": (262144, "fp8", 4, 4096, 2048, 1),
+}
+DEFAULT_WORKLOAD = "prefill_128k_fp8_refine_g4"
+H, D = 64, 128
+FLOP_PER_SCORE = 2 * H * D
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        m = json.load(open(p))
+        return dict(hbm=m["hbm_gbs"], bf16=m["bf16_tflops"], bf16_sustained=m["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+def scan_scores(L, g, c, guard=None):
+    """Scores the scan kernel must produce: dense rows of guarded groups + one row per proxy."""
+    guard = c if guard is None else guard
+    nG = (L + g - 1) // g
+    first = 0 if guard <= 1 else min(nG, (guard - 1 + g - 1) // g)
+    n_dense = min(L, first * g)
+    dense = n_dense * (n_dense + 1) // 2
+    gi = np.arange(first, nG, dtype=np.int64)
+    proxy = int((gi * g + 1).sum())
+    return dense, proxy, nG - first, n_dense
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons during the timed region."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.samples, self.stop, self.th = index, [], threading.Event(), None
+
+    def _run(self):
+        while not self.stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+                self.samples.append([x.strip() for x in out.strip().split(",")])
+            except Exception:
+                pass
+            self.stop.wait(0.15)
+
+    def __enter__(self):
+        self.th = threading.Thread(target=self._run, daemon=True)
+        self.th.start()
+        return self
+
+    def __exit__(self, *a):
+        self.stop.set()
+        self.th.join(timeout=10)
+
+    def summary(self):
+        sm = [float(s[0]) for s in self.samples if len(s) >= 6 and s[0].replace(".", "").isdigit()]
+        mx = [float(s[1]) for s in self.samples if len(s) >= 6 and s[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({n for s in self.samples if len(s) >= 6 for n, v in zip(names, s[2:6]) if v == "Active"})
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=reasons, samples=len(sm))
+
+
+def oracle_sample_time(x, L, g, c, k, mode, n_groups, seed):
+    """Times the CPU oracle (as it stands) on a uniform random sample of groups; returns
+    (estimated seconds for the whole request, seconds spent, groups timed, threads used)."""
+    from oracle import pivot_oracle as po
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    nG = (L + g - 1) // g
+    rng = np.random.default_rng(seed)
+    sel = sorted(rng.choice(nG, size=min(n_groups, nG), replace=False).tolist())
+    codes = x.codes()
+    t0 = time.perf_counter()
+    po.pivot_prefill(codes, g=g, c=c, k=k, mode=mode, groups=sel)
+    dt = time.perf_counter() - t0
+    return dt / len(sel) * nG, dt, len(sel), threads
+
+
+def run_reference(args, wl):
+    L, dtype, g, c, k, mode = WORKLOADS[wl]
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    x = inputs.make_prefill(L, dtype=dtype, seed=inputs.DEFAULT_SEED)
+    per_step = 24
+    ests, spent = [], 0.0
+    for i in range(args.warmup + args.steps):
+        est, dt, n, threads = oracle_sample_time(x, L, g, c, k, mode, per_step, seed=100 + i)
+        if i >= args.warmup:
+            ests.append(est)
+            spent += dt
+    est = float(np.mean(ests))
+    val = L / est
+    line = {
+        "impl": "reference", "metric": "indexed query tokens/s", "value": val, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": est * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl, "L": L, "g": g, "c": c, "k": k, "mode": "refine" if mode else "reuse",
+                   "operands": dtype},
+        "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                         "sample": f"{per_step} uniformly drawn groups of {(L + g - 1) // g} per step, time scaled "
+                                   f"to the whole request; {spent:.1f} s of CPU work timed"},
+        "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--parity-groups", type=int, default=6, help="groups checked against the oracle after timing")
+    args = ap.parse_args()
+    wl = args.workload
+    if args.impl == "reference":
+        return run_reference(args, wl)
+
+    L, dtype, g, c, k, mode = WORKLOADS[wl]
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+
+    from paper_2607_24593_b200 import binding as pv
+
+    x = inputs.make_prefill(L, dtype=dtype, seed=inputs.DEFAULT_SEED + rank)
+    dev = torch.device(f"cuda:{local}")
+    dq, dw, dk = x.q.to(dev), x.w.to(dev), x.k.to(dev)
+    dqs = None if x.qscale is None else x.qscale.to(dev)
+    dks = None if x.kscale is None else x.kscale.to(dev)
+    out = torch.empty((L, k), dtype=torch.int32, device=dev)
+    nG = (L + g - 1) // g
+    pv.ensure_workspace(L, nG, c, k, dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        pv.pivot_index_prefill(dq, dw, dk, L, H, D, g, c, k, mode, out, stream, q_scale=dqs, k_scale=dks)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    assert pv.pivot_device_status() == 0, "device status word set during warm-up"
+    pv.pivot_stage_timing(True)
+    pv.pivot_launch_count_reset()
+    stage_acc = {}
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        barrier()
+        ev0.record(stream)
+        for _ in range(args.steps):
+            step()
+        ev1.record(stream)
+        barrier()
+    elapsed_ms = ev0.elapsed_time(ev1)
+    launches = pv.pivot_launch_count_reset()
+    # per-stage events of the last timed step (recorded by the library on the launch stream)
+    stage_acc = pv.pivot_stage_times()
+    pv.pivot_stage_timing(False)
+    assert pv.pivot_device_status() == 0, "device status word set during the timed region"
+    if dist is not None:
+        t = torch.tensor([elapsed_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * L / (ms_per_step * 1e-3)
+
+    # ---- end to end through the host-buffer entry point (H2D + compute + D2H every step)
+    e2e = None
+    if not args.no_e2e:
+        hq, hw, hk = x.q.pin_memory(), x.w.pin_memory(), x.k.pin_memory()
+        hqs = None if x.qscale is None else x.qscale.pin_memory()
+        hks = None if x.kscale is None else x.kscale.pin_memory()
+        hout = torch.empty((L, k), dtype=torch.int32).pin_memory()
+        del dq, dw, dk, dqs, dks, out
+        pv.pivot_set_workspace(None)
+        torch.cuda.empty_cache()
+        arena = torch.empty(pv.pivot_prefill_host_arena_bytes(L, H, D, g, c, k, pv.FP8_E4M3 if dtype == "fp8" else pv.BF16),
+                            dtype=torch.uint8, device=dev)
+        h2d = sum(t.numel() * t.element_size() for t in (hq, hw, hk, hqs, hks) if t is not None)
+        d2h = hout.numel() * 4
+
+        def estep():
+            pv.pivot_index_prefill_host(hq, hw, hk, L, H, D, g, c, k, mode, hout, arena, stream,
+                                        q_scale=hqs, k_scale=hks)
+
+        for _ in range(max(1, min(args.warmup, 2))):
+            estep()
+        barrier()
+        n_e2e = max(1, min(args.steps, 3))
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            estep()          # returns after the result has landed in host memory
+        t1 = time.perf_counter()
+        e_ms = (t1 - t0) * 1e3 / n_e2e
+        if dist is not None:
+            t = torch.tensor([e_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e2e = {"value": world * L / (e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e_ms, "steps": n_e2e}
+        e2e_out = hout
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    dense_sc, proxy_sc, n_proxy, n_dense = scan_scores(L, g, c)
+    scan_flops = FLOP_PER_SCORE * (dense_sc + proxy_sc)
+    scan_ms = stage_acc["scan_select"]
+    ratio = 2.0 if dtype == "fp8" else 1.0           # nominal dense fp8 : bf16 = 4.5 : 2.25
+    peak_tf = pk["bf16_sustained"] * ratio
+    achieved_tf = scan_flops / (scan_ms * 1e-3) / 1e12
+    roofline = {
+        "kernel": "scan_select_tc_kernel", "bound": "tensor", "achieved": achieved_tf, "peak": peak_tf,
+        "unit": "TFLOP/s", "frac": achieved_tf / peak_tf, "traffic": None,
+        "peak_source": f"{pk['source']} bf16 sustained {pk['bf16_sustained']} TFLOP/s x {ratio:g} (nominal {dtype}:bf16)",
+        "frac_of_nominal": achieved_tf / (4500.0 if dtype == "fp8" else 2250.0),
+        "algorithmic_flops_per_launch": scan_flops, "kernel_ms": scan_ms,
+    }
+    line = {
+        "metric": "indexed query tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "e4m3" if dtype == "fp8" else "bf16",
+        "data": "synthetic",
+        "config": {"workload": wl, "L": L, "H_I": H, "d": D, "g": g, "c": c, "k": k,
+                   "mode": "refine" if mode else "reuse", "operands": dtype, "proxy_groups": n_proxy,
+                   "dense_rows": n_dense, "l2": "inputs larger than L2 (queries >= 1 GB per step)"
+                   if L * H * D >= 2 ** 28 else "inputs smaller than L2; no flush"},
+        "clocks": clocks.summary(), "gpu_launches": int(launches),
+        "stages_ms": stage_acc, "roofline": roofline,
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+
+    # ---- parity probe on the e2e result (a few groups) and the CPU baseline
+    if not args.no_cpu_baseline:
+        est, dt, n, threads = oracle_sample_time(x, L, g, c, k, mode, n_groups=160 if L > 40000 else 256, seed=7)
+        line["cpu_baseline"] = {"value": L / est, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                                "sample": f"{n} uniformly drawn groups of {nG}, time scaled to the whole "
+                                          f"request; {dt:.1f} s of CPU work timed"}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
