@@ -84,7 +84,7 @@ Workspace carve_workspace(void* base, int rows, int n_groups, int c, int k) {
   w.proxy_w = cv.take<float>((size_t)n_groups * kHeads);
   w.cand = cv.take<int32_t>((size_t)n_groups * c);
   w.rows = cv.take<RowDesc>((size_t)rows + n_groups);
-  w.groups = cv.take<GroupDesc>((size_t)n_groups);
+  w.groups = cv.take<GroupDesc>((size_t)rows + n_groups);   // up to ceil(g/4) chunks per group
   w.scan.n_cta = sm_count() * 4;
   w.scan.cap = cand_cap(kmax);
   w.scan.cand_key = cv.take<uint32_t>((size_t)w.scan.n_cta * 2 * w.scan.cap);
@@ -176,7 +176,12 @@ int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, i
       return rc;
   }
   mark(3, st);
-  if (mode == PIVOT_REFINE) launch_refine_simt(ws.groups, p.n_proxy, q->dtype, ws.scan, st);
+  if (mode == PIVOT_REFINE) {
+    const int nd = p.n_proxy * group_chunks(g);
+    if (o && o->impl == 1) launch_refine_simt(ws.groups, nd, q->dtype, ws.scan, st);
+    else if ((rc = check_cuda(launch_refine_tc(q->data, L, q->dtype, ws.groups, nd, ws.scan, sm_count(), st))))
+      return rc;
+  }
   mark(4, st);
   return check_cuda(cudaGetLastError());
 }
@@ -265,7 +270,12 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
     if ((rc = check_cuda(launch_scan_tc(op, ws.rows, B + B * g, 1, ws.scan, sm_count(), st)))) return rc;
   }
   mark(3, st);
-  if (mode == PIVOT_REFINE) launch_refine_simt(ws.groups, B, q->dtype, ws.scan, st);
+  if (mode == PIVOT_REFINE) {
+    const int nd = B * group_chunks(g);
+    if (o && o->impl == 1) launch_refine_simt(ws.groups, nd, q->dtype, ws.scan, st);
+    else if ((rc = check_cuda(launch_refine_tc(q->data, B * g, q->dtype, ws.groups, nd, ws.scan, sm_count(), st))))
+      return rc;
+  }
   mark(4, st);
   return check_cuda(cudaGetLastError());
 }

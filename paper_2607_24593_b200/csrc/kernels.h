@@ -7,6 +7,9 @@
 
 namespace pivot {
 
+constexpr int kMembersPerDesc = 4;
+inline int group_chunks(int g) { return (g + kMembersPerDesc - 1) / kMembersPerDesc; }
+
 // One group's fine step (Eq. 8-9): m members re-score the candidate list.
 struct GroupDesc {
   const void* q;        // first member [m, H, d] codes, members contiguous
@@ -16,9 +19,10 @@ struct GroupDesc {
   const float* kscale;
   const int32_t* cand;  // candidate key positions, valid entries first
   int n_cand;           // valid candidates (0: group is skipped)
-  int m;                // members
+  int m;                // members (at most kMembersPerDesc per descriptor)
   int K;                // entries to select per member
   int first_pos;        // position of the first member (slot i sits at first_pos + i)
+  int q_row;            // row of the first member inside the raw query tensor (units of H x d)
   int32_t* out;         // [m, out_stride]
   float* out_score;     // optional
   int out_stride;
@@ -76,6 +80,9 @@ struct ScanOperands {
 // rows_per_block consecutive scan rows share one key stream (4 in prefill, 1 in decode).
 cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_rows, int rows_per_block,
                            const ScanScratch& s, int sms, cudaStream_t st);
+
+cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
+                             const ScanScratch& s, int sms, cudaStream_t st);
 
 long long& launch_counter();
 

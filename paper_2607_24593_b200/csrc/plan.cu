@@ -5,6 +5,29 @@
 
 namespace pivot {
 
+// The fine-step kernels take at most kMembersPerDesc members per descriptor (the MMA N side is
+// 4 x 64 heads); a larger group is split into chunks that share the candidate list.  Chunk
+// slots without members get n_cand = 0 and are skipped.
+__device__ __forceinline__ void put_group_chunks(GroupDesc* slots, const GroupDesc& full, int g, int dtype) {
+  const size_t esz = dtype == DT_FP8 ? 1 : 2;
+  const int chunks = (g + kMembersPerDesc - 1) / kMembersPerDesc;
+  for (int ch = 0; ch < chunks; ++ch) {
+    GroupDesc gd = full;
+    const int first = ch * kMembersPerDesc;
+    const int m = full.m - first;
+    gd.m = m < kMembersPerDesc ? (m > 0 ? m : 0) : kMembersPerDesc;
+    if (gd.m == 0) gd.n_cand = 0;
+    gd.q = (const char*)full.q + (size_t)first * kHeads * kDim * esz;
+    gd.w = full.w + (size_t)first * kHeads;
+    gd.qscale = full.qscale ? full.qscale + (size_t)first * kHeads : nullptr;
+    gd.first_pos = full.first_pos + first;
+    gd.q_row = full.q_row + first;
+    gd.out = full.out + (size_t)first * full.out_stride;
+    gd.out_score = full.out_score ? full.out_score + (size_t)first * full.out_stride : nullptr;
+    slots[ch] = gd;
+  }
+}
+
 // Scan-row order for prefill: rows [0, n_dense) are dense rows (row i = query i), rows
 // [n_dense, n_dense + n_proxy) are proxy rows.
 __global__ void plan_prefill_kernel(PrefillPlan p, RowDesc* rows, GroupDesc* groups) {
@@ -61,10 +84,12 @@ __global__ void plan_prefill_kernel(PrefillPlan p, RowDesc* rows, GroupDesc* gro
       gd.m = m;
       gd.K = p.k;
       gd.first_pos = t0;
+      gd.q_row = t0;
       gd.out = p.out + (size_t)t0 * p.k;
       gd.out_score = p.out_score ? p.out_score + (size_t)t0 * p.k : nullptr;
       gd.out_stride = p.k;
-      groups[pr] = gd;
+      const int chunks = (p.g + kMembersPerDesc - 1) / kMembersPerDesc;
+      put_group_chunks(groups + (size_t)pr * chunks, gd, p.g, p.dtype);
     }
     rows[i] = r;
   }
@@ -111,6 +136,7 @@ __global__ void plan_decode_kernel(DecodePlan p, RowDesc* rows, GroupDesc* group
   gd.m = p.g;
   gd.K = p.k;
   gd.first_pos = p0;
+  gd.q_row = b * p.g;
   gd.out = outb;
   gd.out_score = outsb;
   gd.out_stride = p.k;
@@ -125,7 +151,7 @@ __global__ void plan_decode_kernel(DecodePlan p, RowDesc* rows, GroupDesc* group
     gd.n_cand = min(p.c, n0);
   }
   rows[b] = r;
-  groups[b] = gd;
+  put_group_chunks(groups + (size_t)b * ((p.g + kMembersPerDesc - 1) / kMembersPerDesc), gd, p.g, p.dtype);
   for (int i = 0; i < p.g; ++i) {
     RowDesc dr;
     dr.q = (const char*)p.q + ((size_t)b * p.g + i) * qrow;

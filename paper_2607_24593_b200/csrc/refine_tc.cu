@@ -1,0 +1,340 @@
+// Kernel 4: candidate gather + per-query re-score on tcgen05 tensor cores + fused top-k
+// (Eq. 8-9).
+//
+// One group at a time per persistent CTA.  The group's m <= 4 member queries (m x 64 heads)
+// form the MMA N side and stay in shared memory; the c candidate keys are gathered from the
+// (L2-resident) key cache by four producer warps, 128 keys per tile, written straight into the
+// 128-byte-swizzled K-major layout the tensor core reads (cp.async, 16 bytes at a time).  The
+// epilogue is the scan's: one key per thread, ReLU, gate-weighted head sum, key scale.  Scores
+// go to a per-CTA buffer; after the last tile each member's exact top-k is selected from its c
+// scores and written out.
+//
+// Warps: 0 = query TMA, 1 = MMA issuer + TMEM owner, 2-5 = gather producers, 6-13 = epilogue.
+#include <cuda.h>
+
+#include "kernels.h"
+#include "ptx.cuh"
+#include "select.cuh"
+
+namespace pivot {
+namespace {
+
+constexpr int TILE_KEYS = 128;
+constexpr int MAX_STAGES = 8;
+constexpr int NMEM = 4;                       // members per MMA (N = 256)
+constexpr int GATHER_WARPS = 4;
+constexpr int EPI_WARPS = 8;
+constexpr int THREADS = (2 + GATHER_WARPS + EPI_WARPS) * 32;   // 448
+constexpr int N = NMEM * kHeads;
+constexpr int TMEM_COLS = 2 * N;
+
+template <int DT>
+struct RCfg {
+  static constexpr bool FP8 = DT == DT_FP8;
+  static constexpr int KHALVES = FP8 ? 1 : 2;
+  static constexpr int HALF_TILE_BYTES = TILE_KEYS * 128;
+  static constexpr int STAGE_BYTES = KHALVES * HALF_TILE_BYTES;
+  static constexpr int QROW_HALF_BYTES = kHeads * 128;
+  static constexpr int QHALF_BYTES = NMEM * QROW_HALF_BYTES;
+  static constexpr int QBUF_BYTES = KHALVES * QHALF_BYTES;
+  static constexpr int STAGES = FP8 ? 6 : 2;      // bf16: 2 x 64 KB of queries leave room for two
+  static constexpr int LOOKAHEAD = FP8 ? 3 : 1;   // gather tiles in flight per producer thread
+  static constexpr int ROW_BYTES = FP8 ? 128 : 256;
+  static constexpr uint32_t IDESC = ptx::make_idesc(FP8 ? 0u : 1u, TILE_KEYS, N);
+};
+
+struct RCtrl {
+  alignas(16) float w[NMEM][kHeads];
+  uint64_t full[MAX_STAGES], empty[MAX_STAGES];
+  uint64_t q_full[2], q_empty[2], tmem_full[2], tmem_empty[2];
+  uint32_t tmem_base;
+  int abort;
+  SelectSmem sel[2];
+};
+
+template <int DT>
+constexpr size_t rsmem_bytes() {
+  using C = RCfg<DT>;
+  return 1024 + 2 * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(RCtrl);
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int NPEND>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(NPEND) : "memory");
+}
+
+__device__ __forceinline__ int group_tiles(const GroupDesc& gd) {
+  return gd.n_cand > 0 ? (gd.n_cand + TILE_KEYS - 1) / TILE_KEYS : 0;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(THREADS, 1)
+refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __restrict__ groups, int n_groups,
+                 int q_rows_total, ScanScratch sc) {
+  using C = RCfg<DT>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* qbuf = smem;
+  uint8_t* kring = smem + 2 * C::QBUF_BYTES;
+  RCtrl& ct = *reinterpret_cast<RCtrl*>(kring + C::STAGES * C::STAGE_BYTES);
+  volatile int* abort_flag = &ct.abort;
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::STAGES; ++s) {
+      ptx::mbar_init(&ct.full[s], GATHER_WARPS);
+      ptx::mbar_init(&ct.empty[s], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(&ct.q_full[i], 1);
+      ptx::mbar_init(&ct.q_empty[i], 1);
+      ptx::mbar_init(&ct.tmem_full[i], 1);
+      ptx::mbar_init(&ct.tmem_empty[i], EPI_WARPS);
+    }
+    ct.abort = 0;
+    ptx::fence_barrier_init();
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(&ct.tmem_base, TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = ct.tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ member-query TMA
+    if (ptx::elect_one()) {
+      ptx::prefetch_tensormap(&tm_q);
+      uint32_t blk = 0;
+      for (int gi = blockIdx.x; gi < n_groups; gi += gridDim.x) {
+        const GroupDesc gd = groups[gi];
+        if (group_tiles(gd) == 0) continue;
+        const int qb = blk & 1;
+        if (!ptx::mbar_wait(&ct.q_empty[qb], ((blk >> 1) & 1) ^ 1, abort_flag)) break;
+        ptx::mbar_arrive_expect_tx(&ct.q_full[qb], gd.m * C::KHALVES * C::QROW_HALF_BYTES);
+        for (int r = 0; r < gd.m; ++r)
+          for (int h = 0; h < C::KHALVES; ++h)
+            ptx::tma_load_2d(qbuf + qb * C::QBUF_BYTES + h * C::QHALF_BYTES + r * C::QROW_HALF_BYTES, &tm_q,
+                             h * 64, (gd.q_row + r) * kHeads, &ct.q_full[qb]);
+        ++blk;
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (ptx::elect_one()) {
+      uint32_t it = 0, blk = 0;
+      bool ok = true;
+      for (int gi = blockIdx.x; gi < n_groups && ok; gi += gridDim.x) {
+        const int ntiles = group_tiles(groups[gi]);
+        if (ntiles == 0) continue;
+        const int qb = blk & 1;
+        ok = ptx::mbar_wait(&ct.q_full[qb], (blk >> 1) & 1, abort_flag);
+        if (!ok) break;
+        const uint32_t q_addr = ptx::smem_u32(qbuf + qb * C::QBUF_BYTES);
+        for (int t = 0; t < ntiles; ++t, ++it) {
+          const int s = it % C::STAGES;
+          const uint32_t ph = (it / C::STAGES) & 1;
+          const int buf = it & 1;
+          ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          ok = ptx::mbar_wait(&ct.full[s], ph, abort_flag);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          const uint32_t k_addr = ptx::smem_u32(kring + s * C::STAGE_BYTES);
+          const uint32_t d_tmem = tmem_base + buf * N;
+#pragma unroll
+          for (int h = 0; h < C::KHALVES; ++h)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+              const uint64_t a = ptx::smem_desc_sw128(k_addr + h * C::HALF_TILE_BYTES + ks * 32);
+              const uint64_t bq = ptx::smem_desc_sw128(q_addr + h * C::QHALF_BYTES + ks * 32);
+              ptx::tc_mma<C::FP8>(d_tmem, a, bq, C::IDESC, (h | ks) ? 1u : 0u);
+            }
+          ptx::tc_commit(&ct.empty[s]);
+          ptx::tc_commit(&ct.tmem_full[buf]);
+        }
+        ptx::tc_commit(&ct.q_empty[qb]);
+        ++blk;
+      }
+    }
+  } else if (warp < 2 + GATHER_WARPS) {
+    // ------------------------------------------------------------------ gather producers
+    // Thread j of the 128 copies candidate row j of each tile.  Tiles are committed as
+    // cp.async groups; a tile is published LOOKAHEAD tiles after it was issued.
+    const int j = (warp - 2) * 32 + lane;
+    const uint32_t swz = (uint32_t)(j & 7);
+    uint32_t it = 0;          // tiles issued
+    uint32_t pub = 0;         // tiles published
+    bool ok = true;
+    auto publish = [&](uint32_t p) {
+      ptx::fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&ct.full[p % C::STAGES]);
+    };
+    for (int gi = blockIdx.x; gi < n_groups; gi += gridDim.x) {
+      const GroupDesc gd = groups[gi];
+      const int ntiles = group_tiles(gd);
+      for (int t = 0; t < ntiles; ++t, ++it) {
+        const int s = it % C::STAGES;
+        const uint32_t ph = (it / C::STAGES) & 1;
+        const int slot = t * TILE_KEYS + j;
+        int idx = slot < gd.n_cand ? gd.cand[slot] : 0;
+        if (idx < 0) idx = 0;
+        if (ok) ok = ptx::mbar_wait(&ct.empty[s], ph ^ 1, abort_flag);
+        const uint8_t* src = (const uint8_t*)gd.kbase + (size_t)idx * C::ROW_BYTES;
+        const uint32_t dst = ptx::smem_u32(kring + s * C::STAGE_BYTES) + (uint32_t)j * 128u;
+#pragma unroll
+        for (int h = 0; h < C::KHALVES; ++h)
+#pragma unroll
+          for (int cidx = 0; cidx < 8; ++cidx)
+            cp_async16(dst + h * C::HALF_TILE_BYTES + ((cidx ^ swz) << 4), src + h * 128 + cidx * 16);
+        cp_async_commit();
+        if (it + 1 - pub > (uint32_t)C::LOOKAHEAD) {
+          cp_async_wait<C::LOOKAHEAD>();
+          publish(pub++);
+        }
+      }
+    }
+    cp_async_wait<0>();
+    while (pub < it) publish(pub++);
+  } else {
+    // ------------------------------------------------------------------ epilogue + top-k
+    const int ew = warp - (2 + GATHER_WARPS);
+    const int team = ew >> 2;
+    const int lq = warp & 3;
+    const int key_in_tile = lq * 32 + lane;
+    const int tt = (ew & 3) * 32 + lane;
+    const Team tm{tt, 128, 1 + team};
+    SelectSmem& sel = ct.sel[team];
+    // per-CTA score buffers: member r -> cand_key[cta][r][0 .. cap)
+    uint32_t* kbuf = sc.cand_key + (size_t)blockIdx.x * NMEM * 2 * sc.cap;
+    uint32_t it = 0;
+    for (int gi = blockIdx.x; gi < n_groups; gi += gridDim.x) {
+      const GroupDesc gd = groups[gi];
+      const int ntiles = group_tiles(gd);
+      if (ntiles == 0) continue;
+      tm.sync();
+      {
+        const int rl = tt >> 6, jh = tt & 63;
+        const int r = team * 2 + rl;
+        float wv = 0.f;
+        if (r < gd.m) {
+          wv = gd.w[r * kHeads + jh];
+          if (gd.qscale) wv = __fmul_rn(wv, gd.qscale[r * kHeads + jh]);
+        }
+        ct.w[r][jh] = wv;
+      }
+      tm.sync();
+      for (int t = 0; t < ntiles; ++t, ++it) {
+        const int buf = it & 1;
+        const int slot = t * TILE_KEYS + key_in_tile;
+        int idx = slot < gd.n_cand ? gd.cand[slot] : -1;
+        const float ksv = (gd.kscale && idx >= 0) ? gd.kscale[idx] : 1.f;
+        (void)ptx::mbar_wait(&ct.tmem_full[buf], (it >> 1) & 1, abort_flag);
+        ptx::tc_fence_after();
+        float score[2];
+#pragma unroll
+        for (int rl = 0; rl < 2; ++rl) {
+          const int r = team * 2 + rl;
+          const uint32_t taddr = tmem_base + ((uint32_t)(lq * 32) << 16) + buf * N + r * kHeads;
+          float acc = 0.f;
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            uint32_t v[32];
+            ptx::tmem_ld_32x32(taddr + half * 32, v);
+            ptx::tmem_wait_ld();
+            const float4* wp = reinterpret_cast<const float4*>(&ct.w[r][half * 32]);
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4) {
+              const float4 wv = wp[q4];
+              acc = fmaf(wv.x, fmaxf(__uint_as_float(v[4 * q4]), 0.f), acc);
+              acc = fmaf(wv.y, fmaxf(__uint_as_float(v[4 * q4 + 1]), 0.f), acc);
+              acc = fmaf(wv.z, fmaxf(__uint_as_float(v[4 * q4 + 2]), 0.f), acc);
+              acc = fmaf(wv.w, fmaxf(__uint_as_float(v[4 * q4 + 3]), 0.f), acc);
+            }
+          }
+          score[rl] = acc;
+        }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
+        if (slot < gd.n_cand) {
+#pragma unroll
+          for (int rl = 0; rl < 2; ++rl) {
+            const int r = team * 2 + rl;
+            if (r < gd.m) kbuf[(size_t)(r * 2) * sc.cap + slot] = score_to_key(gd.kscale ? score[rl] * ksv : score[rl]);
+          }
+        }
+      }
+      tm.sync();
+      // ---- per-member exact top-k over the candidate scores
+#pragma unroll
+      for (int rl = 0; rl < 2; ++rl) {
+        const int r = team * 2 + rl;
+        if (r >= gd.m) continue;
+        const uint32_t* kb = kbuf + (size_t)(r * 2) * sc.cap;
+        int32_t* out = gd.out + (size_t)r * gd.out_stride;
+        float* outs = gd.out_score ? gd.out_score + (size_t)r * gd.out_stride : nullptr;
+        int n_valid = gd.n_cand;
+        if (gd.n_cand > gd.K) {
+          team_select_topk(tm, sel, kb, gd.cand, gd.n_cand, gd.K, nullptr, out, outs, nullptr);
+          n_valid = gd.K;
+        } else {
+          for (int i = tt; i < gd.n_cand; i += 128) {
+            out[i] = gd.cand[i];
+            if (outs) outs[i] = key_to_score(kb[i]);
+          }
+        }
+        for (int i = n_valid + tt; i < gd.K; i += 128) {
+          out[i] = -1;
+          if (outs) outs[i] = -INFINITY;
+        }
+        tm.sync();
+      }
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  if (warp == 1) ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  if (threadIdx.x == 0 && ct.abort) set_status(sc.status, DEV_WAIT_EXPIRED);
+}
+
+template <int DT>
+cudaError_t launch_one(const CUtensorMap& mq, const GroupDesc* groups, int n_groups, int q_rows,
+                       const ScanScratch& s, int sms, cudaStream_t st) {
+  auto kern = refine_tc_kernel<DT>;
+  static bool attr_set = false;
+  const size_t smem = rsmem_bytes<DT>();
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int grid = n_groups < sms ? n_groups : sms;
+  kern<<<grid, THREADS, smem, st>>>(mq, groups, n_groups, q_rows, s);
+  ++launch_counter();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows);
+
+cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
+                             const ScanScratch& s, int sms, cudaStream_t st) {
+  if (n_groups <= 0) return cudaSuccess;
+  CUtensorMap mq;
+  if (!make_operand_map(&mq, q, (long long)q_rows * kHeads, dtype, kHeads)) return cudaErrorInvalidValue;
+  return dtype == DT_FP8 ? launch_one<DT_FP8>(mq, groups, n_groups, q_rows, s, sms, st)
+                         : launch_one<DT_BF16>(mq, groups, n_groups, q_rows, s, sms, st);
+}
+
+}  // namespace pivot

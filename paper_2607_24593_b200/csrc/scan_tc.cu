@@ -377,37 +377,6 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
 
 // ---------------------------------------------------------------------------- host side
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)p;
-  }
-  return fn;
-}
-
-// 2-D map over a row-major [rows, 128] operand tensor; box = 128 bytes x box_rows, 128B swizzle.
-bool make_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const bool fp8 = dtype == DT_FP8;
-  cuuint64_t dims[2] = {(cuuint64_t)kDim, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)(kDim * (fp8 ? 1 : 2))};
-  cuuint32_t box[2] = {(cuuint32_t)(fp8 ? 128 : 64), (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(m, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, dims,
-            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int DT, int NROWS>
 cudaError_t launch_one(const CUtensorMap& mk, const CUtensorMap& mq0, const CUtensorMap& mq1,
                        const RowDesc* rows, int n_rows, const ScanScratch& s, int sms, cudaStream_t st) {
@@ -429,13 +398,44 @@ cudaError_t launch_one(const CUtensorMap& mk, const CUtensorMap& mq0, const CUte
 
 }  // namespace
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// 2-D map over a row-major [rows, 128] operand tensor; box = 128 bytes x box_rows, 128B swizzle.
+bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const bool fp8 = dtype == DT_FP8;
+  cuuint64_t dims[2] = {(cuuint64_t)kDim, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)(kDim * (fp8 ? 1 : 2))};
+  cuuint32_t box[2] = {(cuuint32_t)(fp8 ? 128 : 64), (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, dims,
+            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_rows, int rows_per_block,
                            const ScanScratch& s, int sms, cudaStream_t st) {
   if (n_rows <= 0) return cudaSuccess;
   CUtensorMap mk, mq0, mq1;
-  if (!make_map(&mk, op.kc, op.k_rows, op.dtype, TILE_KEYS) ||
-      !make_map(&mq0, op.q, (long long)op.q_rows * kHeads, op.dtype, kHeads) ||
-      !make_map(&mq1, op.proxy_q, (long long)(op.proxy_rows > 0 ? op.proxy_rows : 1) * kHeads, op.dtype, kHeads))
+  if (!make_operand_map(&mk, op.kc, op.k_rows, op.dtype, TILE_KEYS) ||
+      !make_operand_map(&mq0, op.q, (long long)op.q_rows * kHeads, op.dtype, kHeads) ||
+      !make_operand_map(&mq1, op.proxy_q, (long long)(op.proxy_rows > 0 ? op.proxy_rows : 1) * kHeads, op.dtype, kHeads))
     return cudaErrorInvalidValue;
   if (op.dtype == DT_FP8) {
     return rows_per_block == 4 ? launch_one<DT_FP8, 4>(mk, mq0, mq1, rows, n_rows, s, sms, st)
