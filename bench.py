@@ -37,6 +37,7 @@ WORKLOADS = {
     "prefill_128k_fp8_reuse_g4": (131072, "fp8", 4, 4096, 2048, 0),
     "prefill_128k_fp8_refine_g8": (131072, "fp8", 8, 4096, 2048, 1),
     "prefill_32k_bf16_refine_g4": (32768, "bf16", 4, 4096, 2048, 1),
+    "prefill_32k_fp8_refine_g4": (32768, "fp8", 4, 4096, 2048, 1),
     "prefill_2k_bf16_refine_g4": (2048, "bf16", 4, 512, 256, 1),
     "prefill_256k_fp8_refine_g4": (262144, "fp8", 4, 4096, 2048, 1),
 }

@@ -87,8 +87,9 @@ Workspace carve_workspace(void* base, int rows, int n_groups, int c, int k) {
   w.groups = cv.take<GroupDesc>((size_t)rows + n_groups);   // up to ceil(g/4) chunks per group
   w.scan.n_cta = sm_count() * 4;
   w.scan.cap = cand_cap(kmax);
-  w.scan.cand_key = cv.take<uint32_t>((size_t)w.scan.n_cta * 2 * w.scan.cap);
-  w.scan.cand_idx = cv.take<int32_t>((size_t)w.scan.n_cta * 2 * w.scan.cap);
+  w.scan.cand64 = cv.take<unsigned long long>((size_t)w.scan.n_cta * 2 * w.scan.cap);
+  w.scan.cand_key = (uint32_t*)w.scan.cand64;
+  w.scan.cand_idx = (int32_t*)w.scan.cand64 + (size_t)w.scan.n_cta * 2 * w.scan.cap;
   w.scan.status = w.status;
   w.scan.counter = w.counter;
   w.bytes = cv.off;

@@ -52,8 +52,9 @@ struct DecodePlan {
 };
 
 struct ScanScratch {
-  uint32_t* cand_key;   // [n_cta][2][cap]
+  uint32_t* cand_key;   // [n_cta][2][cap]   (CUDA-core kernels: separate key / index arrays)
   int32_t* cand_idx;    // [n_cta][2][cap]
+  unsigned long long* cand64;   // the same memory seen as packed 64-bit entries (tensor-core kernels)
   int cap;
   int n_cta;
   int* status;

@@ -14,7 +14,7 @@
 
 #include "kernels.h"
 #include "ptx.cuh"
-#include "select.cuh"
+#include "segselect.cuh"
 
 namespace pivot {
 namespace {
@@ -49,7 +49,7 @@ struct RCtrl {
   uint64_t q_full[2], q_empty[2], tmem_full[2], tmem_empty[2];
   uint32_t tmem_base;
   int abort;
-  SelectSmem sel[2];
+  SegSelSmem sel[2];
 };
 
 template <int DT>
@@ -212,9 +212,12 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
     const int key_in_tile = lq * 32 + lane;
     const int tt = (ew & 3) * 32 + lane;
     const Team tm{tt, 128, 1 + team};
-    SelectSmem& sel = ct.sel[team];
-    // per-CTA score buffers: member r -> cand_key[cta][r][0 .. cap)
-    uint32_t* kbuf = sc.cand_key + (size_t)blockIdx.x * NMEM * 2 * sc.cap;
+    SegSelSmem& sel = ct.sel[team];
+    const int wq = ew & 3;
+    const int SEG = sc.cap >> 2;
+    // per-CTA score segments: (member r, warp wq) -> cand64[cta][r][0][wq][0 .. SEG)
+    const size_t cta_base = (size_t)blockIdx.x * NMEM * 2 * sc.cap;
+    auto seg_off = [&](int r) { return cta_base + ((size_t)(r * 2) * 4 + wq) * SEG; };
     uint32_t it = 0;
     for (int gi = blockIdx.x; gi < n_groups; gi += gridDim.x) {
       const GroupDesc gd = groups[gi];
@@ -265,12 +268,13 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
-        if (slot < gd.n_cand) {
+        // entry t*32+lane of this warp's segment; slots past the candidate list are padding
 #pragma unroll
-          for (int rl = 0; rl < 2; ++rl) {
-            const int r = team * 2 + rl;
-            if (r < gd.m) kbuf[(size_t)(r * 2) * sc.cap + slot] = score_to_key(gd.kscale ? score[rl] * ksv : score[rl]);
-          }
+        for (int rl = 0; rl < 2; ++rl) {
+          const int r = team * 2 + rl;
+          if (r < gd.m && t * 32 + lane < SEG)
+            sc.cand64[seg_off(r) + t * 32 + lane] =
+                idx >= 0 ? make_entry(score_to_key(gd.kscale ? score[rl] * ksv : score[rl]), idx) : kPadEntry;
         }
       }
       tm.sync();
@@ -279,19 +283,12 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       for (int rl = 0; rl < 2; ++rl) {
         const int r = team * 2 + rl;
         if (r >= gd.m) continue;
-        const uint32_t* kb = kbuf + (size_t)(r * 2) * sc.cap;
         int32_t* out = gd.out + (size_t)r * gd.out_stride;
         float* outs = gd.out_score ? gd.out_score + (size_t)r * gd.out_stride : nullptr;
-        int n_valid = gd.n_cand;
-        if (gd.n_cand > gd.K) {
-          team_select_topk(tm, sel, kb, gd.cand, gd.n_cand, gd.K, nullptr, out, outs, nullptr);
-          n_valid = gd.K;
-        } else {
-          for (int i = tt; i < gd.n_cand; i += 128) {
-            out[i] = gd.cand[i];
-            if (outs) outs[i] = key_to_score(kb[i]);
-          }
-        }
+        const int segcnt = min(ntiles * 32, SEG);
+        const Seg seg{sc.cand64 + seg_off(r), segcnt};
+        const int n_valid = SEG <= 2048 ? seg_emit<64, true>(tm, sel, seg, gd.n_cand, out, outs, gd.K)
+                                        : seg_emit<128, false>(tm, sel, seg, gd.n_cand, out, outs, gd.K);
         for (int i = n_valid + tt; i < gd.K; i += 128) {
           out[i] = -1;
           if (outs) outs[i] = -INFINITY;

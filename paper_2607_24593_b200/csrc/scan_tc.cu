@@ -17,9 +17,18 @@
 
 #include "kernels.h"
 #include "ptx.cuh"
-#include "select.cuh"
+#include "segselect.cuh"
 
 namespace pivot {
+#ifdef PIVOT_PROFILE
+// Developer build only: per-CTA cycle counters of the epilogue phases (team 0, thread 0).
+__device__ unsigned long long g_scan_prof[256 * 8];
+#define PROF_T(var) const long long var = clock64()
+#define PROF_ADD(slot, t0, t1) if (tt == 0 && team == 0) prof[slot] += (unsigned long long)((t1) - (t0))
+#else
+#define PROF_T(var)
+#define PROF_ADD(slot, t0, t1)
+#endif
 namespace {
 
 constexpr int TILE_KEYS = 128;
@@ -52,12 +61,9 @@ struct Ctrl {
   uint64_t q_full[2], q_empty[2], tmem_full[2], tmem_empty[2];
   uint32_t tmem_base;
   int abort;
-  int n_vis[4];
-  int K[4];
-  uint32_t count[4];
-  uint32_t thr[4];
-  int cur[4];
-  SelectSmem sel[2];
+  int abort_code;         // device status to report besides a timed-out wait
+  int flag[4];            // row r needs a compaction before the next tile
+  SegSelSmem sel[2];
 };
 
 template <int DT, int NROWS>
@@ -124,6 +130,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       ptx::mbar_init(&ct.tmem_empty[i], C::EPI_WARPS);
     }
     ct.abort = 0;
+    ct.abort_code = 0;
     ptx::fence_barrier_init();
   }
   if (warp == 1) {
@@ -220,14 +227,21 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     // ------------------------------------------------------------------ epilogue + select
     const int ew = warp - 2;                       // 0 .. EPI_WARPS-1
     const int team = ew >> 2;                      // which pair of rows
+    const int wq = ew & 3;                         // warp inside the team = candidate segment
     const int lq = warp & 3;                       // TMEM lane quarter this warp may read
     const int key_in_tile = lq * 32 + lane;
-    const int tt = (ew & 3) * 32 + lane;           // rank inside the team (0..127)
+    const int tt = wq * 32 + lane;                 // rank inside the team (0..127)
     const Team tm{tt, 128, 1 + team};
-    SelectSmem& sel = ct.sel[team];
+    SegSelSmem& sel = ct.sel[team];
+    const int SEG = sc.cap >> 2;                   // entries per warp segment
     const size_t cta_base = (size_t)blockIdx.x * NROWS * 2 * sc.cap;
+    // segment of (row r, ping-pong half pp) owned by this warp
+    auto seg_off = [&](int r, int pp) { return cta_base + ((size_t)(r * 2 + pp) * 4 + wq) * SEG; };
     BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
     uint32_t it = 0;
+#ifdef PIVOT_PROFILE
+    unsigned long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#endif
     // A failed wait never changes this role's control flow (the team barriers below must stay
     // matched); once the abort flag is up every later wait returns at once.
     for (int b = bi.next(); b >= 0; b = bi.next()) {
@@ -236,7 +250,9 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       if (ntiles == 0) continue;
       // ---- per-block state of this team's rows
       tm.sync();
-      const float* kscale = nullptr;
+      const float* kscale = rows[b * NROWS].kscale;
+      int n_vis[C::ROWS_PER_TEAM], Ksel[C::ROWS_PER_TEAM], cnt[C::ROWS_PER_TEAM], cur[C::ROWS_PER_TEAM];
+      uint32_t thr[C::ROWS_PER_TEAM];
       {
         const int rl = tt >> 6, j = tt & 63;
         if (rl < C::ROWS_PER_TEAM) {
@@ -248,112 +264,123 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             if (rows[ri].qscale) wv = __fmul_rn(wv, rows[ri].qscale[j]);
           }
           ct.w[r][j] = wv;
-          if (j == 0) {
-            const bool live = ri < n_rows && rows[ri].K > 0;
-            ct.n_vis[r] = live ? rows[ri].n_vis : 0;
-            ct.K[r] = live ? rows[ri].K : 0;
-            ct.count[r] = 0;
-            ct.thr[r] = 0;
-            ct.cur[r] = 0;
-          }
+          if (j == 0) ct.flag[r] = 0;
         }
-        const int r0 = b * NROWS;
-        kscale = rows[r0].kscale;
+      }
+#pragma unroll
+      for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
+        const int ri = b * NROWS + team * C::ROWS_PER_TEAM + rl;
+        const bool live = ri < n_rows && rows[ri].K > 0;
+        n_vis[rl] = live ? rows[ri].n_vis : 0;
+        Ksel[rl] = live ? rows[ri].K : 0;
+        cnt[rl] = 0; cur[rl] = 0; thr[rl] = 0;
       }
       tm.sync();
       for (int t = 0; t < ntiles; ++t, ++it) {
-        // ---- make room: exact compaction of a row whose buffer could overflow in this tile
+        PROF_T(p0);
+        // ---- make room: exact compaction of a row one of whose segments is nearly full
 #pragma unroll
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
           const int r = team * C::ROWS_PER_TEAM + rl;
-          if ((int)ct.count[r] + TILE_KEYS > sc.cap) {
-            const int n = (int)ct.count[r];
-            const int cur = ct.cur[r];
-            uint32_t* kb = sc.cand_key + cta_base + (size_t)(r * 2) * sc.cap;
-            int32_t* ib = sc.cand_idx + cta_base + (size_t)(r * 2) * sc.cap;
-            tm.sync();
-            team_select_topk(tm, sel, kb + cur * sc.cap, ib + cur * sc.cap, n, ct.K[r],
-                             kb + (cur ^ 1) * sc.cap, ib + (cur ^ 1) * sc.cap, nullptr, &ct.thr[r]);
-            if (tt == 0) { ct.count[r] = (uint32_t)ct.K[r]; ct.cur[r] = cur ^ 1; }
+          if (ct.flag[r]) {
+            const Seg seg{sc.cand64 + seg_off(r, cur[rl]), cnt[rl]};
+            entry_t* dst = sc.cand64 + seg_off(r, cur[rl] ^ 1);
+            entry_t cut;
+            cnt[rl] = SEG <= 2048 ? seg_compact<64, true>(tm, sel, seg, dst, Ksel[rl], &cut)
+                                  : seg_compact<128, false>(tm, sel, seg, dst, Ksel[rl], &cut);
+            cur[rl] ^= 1;
+            thr[rl] = entry_key(cut);
+            if (tt == 0) ct.flag[r] = 0;
+#ifdef PIVOT_PROFILE
+            if (tt == 0 && team == 0) prof[7] += 1;
+#endif
             tm.sync();
           }
         }
+        PROF_T(p1);
+        PROF_ADD(0, p0, p1);
         const int buf = it & 1;
         const int s_key = t * TILE_KEYS + key_in_tile;
         const float ksv = (kscale && s_key < nv_max) ? kscale[s_key] : 0.f;
         (void)ptx::mbar_wait(&ct.tmem_full[buf], (it >> 1) & 1, abort_flag);
         ptx::tc_fence_after();
+        PROF_T(p2);
+        PROF_ADD(1, p1, p2);
         float score[C::ROWS_PER_TEAM];
 #pragma unroll
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
           const int r = team * C::ROWS_PER_TEAM + rl;
           const uint32_t taddr = tmem_base + ((uint32_t)(lq * 32) << 16) + buf * C::N + r * kHeads;
-          float acc = 0.f;
+          uint32_t v0[32], v1[32];
+          ptx::tmem_ld_32x32(taddr, v0);
+          ptx::tmem_ld_32x32(taddr + 32, v1);
+          ptx::tmem_wait_ld();
+          float a0 = 0.f, a1 = 0.f;
+          const float4* wp = reinterpret_cast<const float4*>(&ct.w[r][0]);
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            uint32_t v[32];
-            ptx::tmem_ld_32x32(taddr + half * 32, v);
-            ptx::tmem_wait_ld();
-            const float4* wp = reinterpret_cast<const float4*>(&ct.w[r][half * 32]);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const float4 wv = wp[j];
-              acc = fmaf(wv.x, fmaxf(__uint_as_float(v[4 * j]), 0.f), acc);
-              acc = fmaf(wv.y, fmaxf(__uint_as_float(v[4 * j + 1]), 0.f), acc);
-              acc = fmaf(wv.z, fmaxf(__uint_as_float(v[4 * j + 2]), 0.f), acc);
-              acc = fmaf(wv.w, fmaxf(__uint_as_float(v[4 * j + 3]), 0.f), acc);
-            }
+          for (int j = 0; j < 8; ++j) {
+            const float4 wa = wp[j], wb = wp[8 + j];
+            a0 = fmaf(wa.x, fmaxf(__uint_as_float(v0[4 * j]), 0.f), a0);
+            a1 = fmaf(wb.x, fmaxf(__uint_as_float(v1[4 * j]), 0.f), a1);
+            a0 = fmaf(wa.y, fmaxf(__uint_as_float(v0[4 * j + 1]), 0.f), a0);
+            a1 = fmaf(wb.y, fmaxf(__uint_as_float(v1[4 * j + 1]), 0.f), a1);
+            a0 = fmaf(wa.z, fmaxf(__uint_as_float(v0[4 * j + 2]), 0.f), a0);
+            a1 = fmaf(wb.z, fmaxf(__uint_as_float(v1[4 * j + 2]), 0.f), a1);
+            a0 = fmaf(wa.w, fmaxf(__uint_as_float(v0[4 * j + 3]), 0.f), a0);
+            a1 = fmaf(wb.w, fmaxf(__uint_as_float(v1[4 * j + 3]), 0.f), a1);
           }
-          score[rl] = acc;
+          score[rl] = a0 + a1;
         }
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
-        // ---- filter + append
+        PROF_T(p3);
+        PROF_ADD(2, p2, p3);
+        // ---- filter + append to this warp's own segment (register cursor, no atomics)
 #pragma unroll
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
           const int r = team * C::ROWS_PER_TEAM + rl;
           const float sv = kscale ? score[rl] * ksv : score[rl];
           const uint32_t key = score_to_key(sv);
-          const bool take = s_key < ct.n_vis[r] && key > ct.thr[r];
+          const bool take = s_key < n_vis[rl] && key > thr[rl];
           const uint32_t m = __ballot_sync(0xffffffffu, take);
-          if (m) {
-            uint32_t pos = 0;
-            const int leader = __ffs(m) - 1;
-            if (lane == leader) pos = atomicAdd(&ct.count[r], (uint32_t)__popc(m));
-            pos = __shfl_sync(0xffffffffu, pos, leader);
-            if (take) {
-              const uint32_t p = pos + __popc(m & ((1u << lane) - 1u));
-              const size_t o = cta_base + (size_t)(r * 2 + ct.cur[r]) * sc.cap + p;
-              sc.cand_key[o] = key;
-              sc.cand_idx[o] = s_key;
+          if (take) {
+            const int p = cnt[rl] + __popc(m & ((1u << lane) - 1u));
+            if (p < SEG) {
+              sc.cand64[seg_off(r, cur[rl]) + p] = make_entry(key, s_key);
+            } else {
+              ct.abort_code = DEV_CAND_OVERFLOW;
             }
           }
+          cnt[rl] = min(cnt[rl] + __popc(m), SEG);
+          if (lane == 0 && cnt[rl] + 32 > SEG) ct.flag[r] = 1;
         }
+        PROF_T(p4);
+        PROF_ADD(3, p3, p4);
         tm.sync();
+        PROF_T(p5);
+        PROF_ADD(4, p4, p5);
+#ifdef PIVOT_PROFILE
+        if (tt == 0 && team == 0) prof[6] += 1;
+#endif
       }
+      PROF_T(p6);
       // ---- end of the block: final exact select per row, then pad / replicate
 #pragma unroll
       for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
         const int r = team * C::ROWS_PER_TEAM + rl;
         const int ri = b * NROWS + r;
-        const int K = ct.K[r];
+        const int K = Ksel[rl];
         if (K <= 0) continue;
         const RowDesc rd = rows[ri];
-        const int n = (int)ct.count[r];
-        const uint32_t* kb = sc.cand_key + cta_base + (size_t)(r * 2 + ct.cur[r]) * sc.cap;
-        const int32_t* ib = sc.cand_idx + cta_base + (size_t)(r * 2 + ct.cur[r]) * sc.cap;
-        int n_valid = n;
-        if (n > K) {
-          team_select_topk(tm, sel, kb, ib, n, K, nullptr, rd.out, rd.out_score, nullptr);
-          n_valid = K;
-        } else {
-          for (int i = tt; i < n; i += 128) {
-            rd.out[i] = ib[i];
-            if (rd.out_score) rd.out_score[i] = key_to_score(kb[i]);
-          }
-        }
+        if (tt == 0) sel.total = 0;
         tm.sync();
+        if (lane == 0) atomicAdd(&sel.total, (uint32_t)cnt[rl]);
+        tm.sync();
+        const int n = (int)sel.total;
+        const Seg seg{sc.cand64 + seg_off(r, cur[rl]), cnt[rl]};
+        const int n_valid = SEG <= 2048 ? seg_emit<64, true>(tm, sel, seg, n, rd.out, rd.out_score, K)
+                                        : seg_emit<128, false>(tm, sel, seg, n, rd.out, rd.out_score, K);
         for (int i = n_valid + tt; i < K; i += 128) {
           rd.out[i] = -1;
           if (rd.out_score) rd.out_score[i] = -INFINITY;
@@ -365,7 +392,13 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             if (rd.out_score) rd.out_score[(size_t)rr * rd.out_stride + i] = rd.out_score[i];
           }
       }
+      PROF_T(p7);
+      PROF_ADD(5, p6, p7);
     }
+#ifdef PIVOT_PROFILE
+    if (tt == 0 && team == 0)
+      for (int i = 0; i < 8; ++i) g_scan_prof[blockIdx.x * 8 + i] = prof[i];
+#endif
   }
   // ------------------------------------------------------------------ teardown
   ptx::tc_fence_before();
@@ -373,6 +406,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
   ptx::tc_fence_after();
   if (warp == 1) ptx::tmem_dealloc(tmem_base, C::TMEM_COLS);
   if (threadIdx.x == 0 && ct.abort) set_status(sc.status, DEV_WAIT_EXPIRED);
+  if (threadIdx.x == 0 && ct.abort_code) set_status(sc.status, ct.abort_code);
 }
 
 // ---------------------------------------------------------------------------- host side
@@ -428,6 +462,15 @@ bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtyp
             strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+
+#ifdef PIVOT_PROFILE
+extern "C" int pivot_profile_read(unsigned long long* host, int n) {
+  return (int)cudaMemcpyFromSymbol(host, g_scan_prof, sizeof(unsigned long long) * (size_t)n);
+}
+extern "C" int pivot_profile_read_sel(unsigned long long* host) {
+  return (int)cudaMemcpyFromSymbol(host, g_sel_prof, sizeof(unsigned long long) * 16);
+}
+#endif
 
 cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_rows, int rows_per_block,
                            const ScanScratch& s, int sms, cudaStream_t st) {
