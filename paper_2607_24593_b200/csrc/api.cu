@@ -48,6 +48,12 @@ int cand_cap(int kmax) {
   return (int)align_up((size_t)cap, 64);
 }
 
+int tc_cap(int kmax) {
+  size_t cap = (size_t)6 * kmax;
+  if (cap < 4096) cap = 4096;
+  return (int)align_up(cap, 128);
+}
+
 struct Carve {
   char* base;
   size_t off = 0;
@@ -61,6 +67,7 @@ struct Carve {
 };
 
 struct Workspace {
+  int tc_cap;
   int* status;
   int* counter;
   void* proxy_q;
@@ -85,15 +92,29 @@ Workspace carve_workspace(void* base, int rows, int n_groups, int c, int k) {
   w.cand = cv.take<int32_t>((size_t)n_groups * c);
   w.rows = cv.take<RowDesc>((size_t)rows + n_groups);
   w.groups = cv.take<GroupDesc>((size_t)rows + n_groups);   // up to ceil(g/4) chunks per group
+  // Candidate scratch.  Tensor-core kernels: one CTA per SM, 4 rows x cap packed entries each,
+  // cap = 6 K (a tight running threshold admits about K (1 + ln(n / K)) entries per row).
+  // CUDA-core kernels: 4 CTAs per SM, two buffers of 2 K (key, index) pairs each.  The
+  // region is sized for the larger of the two and shared.
   w.scan.n_cta = sm_count() * 4;
   w.scan.cap = cand_cap(kmax);
-  w.scan.cand64 = cv.take<unsigned long long>((size_t)w.scan.n_cta * 2 * w.scan.cap);
+  w.tc_cap = tc_cap(kmax);
+  const size_t simt_entries = (size_t)w.scan.n_cta * 2 * w.scan.cap;
+  const size_t tc_entries = (size_t)sm_count() * 4 * w.tc_cap;
+  w.scan.cand64 = cv.take<unsigned long long>(simt_entries > tc_entries ? simt_entries : tc_entries);
   w.scan.cand_key = (uint32_t*)w.scan.cand64;
-  w.scan.cand_idx = (int32_t*)w.scan.cand64 + (size_t)w.scan.n_cta * 2 * w.scan.cap;
+  w.scan.cand_idx = (int32_t*)w.scan.cand64 + simt_entries;
   w.scan.status = w.status;
   w.scan.counter = w.counter;
   w.bytes = cv.off;
   return w;
+}
+
+// The scratch as the tensor-core kernels see it: per-row capacity of packed entries.
+ScanScratch tc_scratch(const Workspace& ws) {
+  ScanScratch s = ws.scan;
+  s.cap = ws.tc_cap;
+  return s;
 }
 
 bool g_timing = false;
@@ -173,14 +194,14 @@ int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, i
     launch_scan_simt(ws.rows, p.n_dense + p.n_proxy, q->dtype, ws.scan, st);
   } else {
     ScanOperands op{kc->data, L, q->data, L, ws.proxy_q, p.n_proxy, q->dtype};
-    if ((rc = check_cuda(launch_scan_tc(op, ws.rows, p.n_dense + p.n_proxy, 4, ws.scan, sm_count(), st))))
+    if ((rc = check_cuda(launch_scan_tc(op, ws.rows, p.n_dense + p.n_proxy, 4, tc_scratch(ws), sm_count(), st))))
       return rc;
   }
   mark(3, st);
   if (mode == PIVOT_REFINE) {
     const int nd = p.n_proxy * group_chunks(g);
     if (o && o->impl == 1) launch_refine_simt(ws.groups, nd, q->dtype, ws.scan, st);
-    else if ((rc = check_cuda(launch_refine_tc(q->data, L, q->dtype, ws.groups, nd, ws.scan, sm_count(), st))))
+    else if ((rc = check_cuda(launch_refine_tc(q->data, L, q->dtype, ws.groups, nd, tc_scratch(ws), sm_count(), st))))
       return rc;
   }
   mark(4, st);
@@ -268,13 +289,13 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
     launch_scan_simt(ws.rows, B + B * g, q->dtype, ws.scan, st);
   } else {
     ScanOperands op{kcache->data, (long long)B * Lmax, q->data, B * g, ws.proxy_q, B, q->dtype};
-    if ((rc = check_cuda(launch_scan_tc(op, ws.rows, B + B * g, 1, ws.scan, sm_count(), st)))) return rc;
+    if ((rc = check_cuda(launch_scan_tc(op, ws.rows, B + B * g, 1, tc_scratch(ws), sm_count(), st)))) return rc;
   }
   mark(3, st);
   if (mode == PIVOT_REFINE) {
     const int nd = B * group_chunks(g);
     if (o && o->impl == 1) launch_refine_simt(ws.groups, nd, q->dtype, ws.scan, st);
-    else if ((rc = check_cuda(launch_refine_tc(q->data, B * g, q->dtype, ws.groups, nd, ws.scan, sm_count(), st))))
+    else if ((rc = check_cuda(launch_refine_tc(q->data, B * g, q->dtype, ws.groups, nd, tc_scratch(ws), sm_count(), st))))
       return rc;
   }
   mark(4, st);

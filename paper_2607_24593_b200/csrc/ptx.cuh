@@ -60,12 +60,16 @@ constexpr uint64_t kWaitLimitNs = 4000000000ull;  // 4 s: far beyond any legitim
 
 // Waits for the phase with the given parity to complete.  Returns false if `*abort_flag`
 // became non-zero or the time limit ran out (the flag is then set for everybody else).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// `backoff_ns` > 0 puts the thread to sleep between polls: single-thread roles (TMA producer,
+// MMA issuer) share a scheduler with epilogue warps and must not eat their issue slots.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned backoff_ns = 0) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   uint32_t spins = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (backoff_ns) __nanosleep(backoff_ns);
     if (*abort_flag) return false;
     if ((++spins & 255u) == 0) {
       if (globaltimer_ns() - t0 > kWaitLimitNs) {

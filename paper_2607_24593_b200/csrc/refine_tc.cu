@@ -215,9 +215,9 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
     SegSelSmem& sel = ct.sel[team];
     const int wq = ew & 3;
     const int SEG = sc.cap >> 2;
-    // per-CTA score segments: (member r, warp wq) -> cand64[cta][r][0][wq][0 .. SEG)
-    const size_t cta_base = (size_t)blockIdx.x * NMEM * 2 * sc.cap;
-    auto seg_off = [&](int r) { return cta_base + ((size_t)(r * 2) * 4 + wq) * SEG; };
+    // per-CTA score segments: (member r, warp wq) -> cand64[cta][r][wq][0 .. SEG)
+    const size_t cta_base = (size_t)blockIdx.x * NMEM * sc.cap;
+    auto seg_off = [&](int r) { return cta_base + ((size_t)r * 4 + wq) * SEG; };
     uint32_t it = 0;
     for (int gi = blockIdx.x; gi < n_groups; gi += gridDim.x) {
       const GroupDesc gd = groups[gi];
@@ -287,8 +287,8 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         float* outs = gd.out_score ? gd.out_score + (size_t)r * gd.out_stride : nullptr;
         const int segcnt = min(ntiles * 32, SEG);
         const Seg seg{sc.cand64 + seg_off(r), segcnt};
-        const int n_valid = SEG <= 2048 ? seg_emit<64, true>(tm, sel, seg, gd.n_cand, out, outs, gd.K)
-                                        : seg_emit<128, false>(tm, sel, seg, gd.n_cand, out, outs, gd.K);
+        const int n_valid = segcnt <= 32 * kSelEpt ? seg_emit<true>(tm, sel, seg, gd.n_cand, out, outs, gd.K)
+                                                   : seg_emit<false>(tm, sel, seg, gd.n_cand, out, outs, gd.K);
         for (int i = n_valid + tt; i < gd.K; i += 128) {
           out[i] = -1;
           if (outs) outs[i] = -INFINITY;

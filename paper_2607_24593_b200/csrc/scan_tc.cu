@@ -45,7 +45,8 @@ struct Cfg {
   static constexpr int QHALF_BYTES = NROWS * QROW_HALF_BYTES;
   static constexpr int QBUF_BYTES = KHALVES * QHALF_BYTES;
   static constexpr int N = NROWS * kHeads;
-  static constexpr int STAGES = FP8 ? 6 : (NROWS == 4 ? 2 : 4);
+  static constexpr int QBUFS = (!FP8 && NROWS == 4) ? 1 : 2;   // bf16 x 4 rows: 64 KB per query buffer
+  static constexpr int STAGES = FP8 ? 6 : (NROWS == 4 ? 3 : 4);
   static constexpr int EPI_WARPS = NROWS == 4 ? 8 : 4;
   static constexpr int ROWS_PER_TEAM = NROWS == 4 ? 2 : 1;
   static constexpr int TEAMS = EPI_WARPS / 4;
@@ -55,21 +56,24 @@ struct Cfg {
   static constexpr uint32_t IDESC = ptx::make_idesc(FP8 ? 0u : 1u, TILE_KEYS, N);
 };
 
+template <int NROWS>
 struct Ctrl {
-  alignas(16) float w[4][kHeads];   // read as float4
+  alignas(16) float w[4][kHeads];       // effective gates of the block's rows (read as float4)
+  uint32_t rhist[NROWS][kSelBins];      // per row: histogram of every score seen so far
   uint64_t full[MAX_STAGES], empty[MAX_STAGES];
   uint64_t q_full[2], q_empty[2], tmem_full[2], tmem_empty[2];
   uint32_t tmem_base;
   int abort;
   int abort_code;         // device status to report besides a timed-out wait
-  int flag[4];            // row r needs a compaction before the next tile
+  int flag[4];            // row r: a candidate segment is nearly full
+  uint32_t rowmax[4];     // row r: largest score key of the first tile (anchors the histogram)
   SegSelSmem sel[2];
 };
 
 template <int DT, int NROWS>
 constexpr size_t smem_bytes() {
   using C = Cfg<DT, NROWS>;
-  return 1024 + 2 * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(Ctrl);
+  return 1024 + C::QBUFS * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(Ctrl<NROWS>);
 }
 
 // Block sequence of one CTA: blocks sorted longest-first are dealt in snake order.
@@ -112,9 +116,9 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
   using C = Cfg<DT, NROWS>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* qbuf = smem;                                   // 2 x QBUF_BYTES
-  uint8_t* kring = smem + 2 * C::QBUF_BYTES;              // STAGES x STAGE_BYTES
-  Ctrl& ct = *reinterpret_cast<Ctrl*>(kring + C::STAGES * C::STAGE_BYTES);
+  uint8_t* qbuf = smem;                                   // QBUFS x QBUF_BYTES
+  uint8_t* kring = smem + C::QBUFS * C::QBUF_BYTES;       // STAGES x STAGE_BYTES
+  Ctrl<NROWS>& ct = *reinterpret_cast<Ctrl<NROWS>*>(kring + C::STAGES * C::STAGE_BYTES);
   volatile int* abort_flag = &ct.abort;
 
   const int warp = threadIdx.x >> 5;
@@ -155,8 +159,8 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         int k_row0 = 0;
         const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0);
         if (ntiles == 0) continue;
-        const int qb = blk & 1;
-        ok = ptx::mbar_wait(&ct.q_empty[qb], ((blk >> 1) & 1) ^ 1, abort_flag);
+        const int qb = blk % C::QBUFS;
+        ok = ptx::mbar_wait(&ct.q_empty[qb], ((blk / C::QBUFS) & 1) ^ 1, abort_flag, 64);
         if (!ok) break;
         int present = 0;
         for (int r = 0; r < NROWS; ++r) present += (b * NROWS + r < n_rows) ? 1 : 0;
@@ -173,7 +177,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         for (int t = 0; t < ntiles; ++t, ++it) {
           const int s = it % C::STAGES;
           const uint32_t ph = (it / C::STAGES) & 1;
-          ok = ptx::mbar_wait(&ct.empty[s], ph ^ 1, abort_flag);
+          ok = ptx::mbar_wait(&ct.empty[s], ph ^ 1, abort_flag, 64);
           if (!ok) break;
           ptx::mbar_arrive_expect_tx(&ct.full[s], C::STAGE_BYTES);
           for (int h = 0; h < C::KHALVES; ++h)
@@ -193,17 +197,17 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         int k_row0 = 0;
         const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0);
         if (ntiles == 0) continue;
-        const int qb = blk & 1;
-        ok = ptx::mbar_wait(&ct.q_full[qb], (blk >> 1) & 1, abort_flag);
+        const int qb = blk % C::QBUFS;
+        ok = ptx::mbar_wait(&ct.q_full[qb], (blk / C::QBUFS) & 1, abort_flag, 32);
         if (!ok) break;
         const uint32_t q_addr = ptx::smem_u32(qbuf + qb * C::QBUF_BYTES);
         for (int t = 0; t < ntiles; ++t, ++it) {
           const int s = it % C::STAGES;
           const uint32_t ph = (it / C::STAGES) & 1;
           const int buf = it & 1;
-          ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag);
+          ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, 32);
           if (!ok) break;
-          ok = ptx::mbar_wait(&ct.full[s], ph, abort_flag);
+          ok = ptx::mbar_wait(&ct.full[s], ph, abort_flag, 32);
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t k_addr = ptx::smem_u32(kring + s * C::STAGE_BYTES);
@@ -234,9 +238,38 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     const Team tm{tt, 128, 1 + team};
     SegSelSmem& sel = ct.sel[team];
     const int SEG = sc.cap >> 2;                   // entries per warp segment
-    const size_t cta_base = (size_t)blockIdx.x * NROWS * 2 * sc.cap;
-    // segment of (row r, ping-pong half pp) owned by this warp
-    auto seg_off = [&](int r, int pp) { return cta_base + ((size_t)(r * 2 + pp) * 4 + wq) * SEG; };
+    const size_t cta_base = (size_t)blockIdx.x * NROWS * sc.cap;
+    auto seg_ptr = [&](int r) { return sc.cand64 + cta_base + ((size_t)r * 4 + wq) * SEG; };
+    // Score key -> histogram bin: 256 bins per octave (8 mantissa bits), 2048 bins anchored two
+    // octaves above the row's first-tile maximum; keys outside land in the end bins.
+    auto key_bin = [](uint32_t key, int base) {
+      const int b = (int)(key >> 15) - base;
+      return b < 0 ? 0 : (b > kSelBins - 1 ? kSelBins - 1 : b);
+    };
+    // Lower bound on the K-th best score seen so far, read off the row histogram: the largest
+    // bin edge with at least K scores at or above it.  Returned as a key threshold t such that
+    // only keys > t can still belong to the top K.
+    auto hist_threshold = [&](int r, int K, int base) -> uint32_t {
+      hist_boundary(tm, sel, ct.rhist[r], (uint32_t)K);
+      const uint32_t b = sel.bin;
+      return b > 0 ? (((uint32_t)((int)b + base)) << 15) - 1u : 0u;
+    };
+    auto team_max = [&](int v) -> int {          // max of a warp-uniform value over the team
+      tm.sync();
+      if (tt == 0) sel.maxcnt = 0;
+      tm.sync();
+      if (lane == 0) atomicMax(&sel.maxcnt, (uint32_t)v);
+      tm.sync();
+      return (int)sel.maxcnt;
+    };
+    auto team_sum = [&](int v) -> int {          // sum of a warp-uniform value over the team
+      tm.sync();
+      if (tt == 0) sel.total = 0;
+      tm.sync();
+      if (lane == 0) atomicAdd(&sel.total, (uint32_t)v);
+      tm.sync();
+      return (int)sel.total;
+    };
     BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
     uint32_t it = 0;
 #ifdef PIVOT_PROFILE
@@ -251,7 +284,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       // ---- per-block state of this team's rows
       tm.sync();
       const float* kscale = rows[b * NROWS].kscale;
-      int n_vis[C::ROWS_PER_TEAM], Ksel[C::ROWS_PER_TEAM], cnt[C::ROWS_PER_TEAM], cur[C::ROWS_PER_TEAM];
+      int n_vis[C::ROWS_PER_TEAM], Ksel[C::ROWS_PER_TEAM], cnt[C::ROWS_PER_TEAM], base[C::ROWS_PER_TEAM];
       uint32_t thr[C::ROWS_PER_TEAM];
       {
         const int rl = tt >> 6, j = tt & 63;
@@ -263,38 +296,43 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             wv = rows[ri].w[j];
             if (rows[ri].qscale) wv = __fmul_rn(wv, rows[ri].qscale[j]);
           }
-          ct.w[r][j] = wv;
-          if (j == 0) ct.flag[r] = 0;
+          ct.w[r][j] = 0.5f * wv;       // halved: see the epilogue's ReLU identity
+          if (j == 0) { ct.flag[r] = 0; ct.rowmax[r] = 0; }
         }
       }
 #pragma unroll
       for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
-        const int ri = b * NROWS + team * C::ROWS_PER_TEAM + rl;
+        const int r = team * C::ROWS_PER_TEAM + rl;
+        const int ri = b * NROWS + r;
         const bool live = ri < n_rows && rows[ri].K > 0;
         n_vis[rl] = live ? rows[ri].n_vis : 0;
         Ksel[rl] = live ? rows[ri].K : 0;
-        cnt[rl] = 0; cur[rl] = 0; thr[rl] = 0;
+        cnt[rl] = 0; base[rl] = 0; thr[rl] = 0;
+        for (int i = tt; i < kSelBins; i += 128) ct.rhist[r][i] = 0;
       }
       tm.sync();
       for (int t = 0; t < ntiles; ++t, ++it) {
         PROF_T(p0);
-        // ---- make room: exact compaction of a row one of whose segments is nearly full
+        // ---- a segment is nearly full: tighten the threshold and drop what fell below it;
+        //      if that is not enough (ties, adversarial order) compact exactly to the K best
 #pragma unroll
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
           const int r = team * C::ROWS_PER_TEAM + rl;
           if (ct.flag[r]) {
-            const Seg seg{sc.cand64 + seg_off(r, cur[rl]), cnt[rl]};
-            entry_t* dst = sc.cand64 + seg_off(r, cur[rl] ^ 1);
-            entry_t cut;
-            cnt[rl] = SEG <= 2048 ? seg_compact<64, true>(tm, sel, seg, dst, Ksel[rl], &cut)
-                                  : seg_compact<128, false>(tm, sel, seg, dst, Ksel[rl], &cut);
-            cur[rl] ^= 1;
-            thr[rl] = entry_key(cut);
+            const uint32_t th = hist_threshold(r, Ksel[rl], base[rl]);
+            thr[rl] = th > thr[rl] ? th : thr[rl];
+            const uint32_t tcur = thr[rl];
+            cnt[rl] = seg_filter_inplace(seg_ptr(r), cnt[rl], lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
+            if (team_max(cnt[rl]) + 32 > SEG) {
+              entry_t cut;
+              cnt[rl] = seg_compact<false>(tm, sel, Seg{seg_ptr(r), cnt[rl]}, Ksel[rl], &cut);
+              thr[rl] = entry_key(cut) > thr[rl] ? entry_key(cut) : thr[rl];
+            }
             if (tt == 0) ct.flag[r] = 0;
+            tm.sync();
 #ifdef PIVOT_PROFILE
             if (tt == 0 && team == 0) prof[7] += 1;
 #endif
-            tm.sync();
           }
         }
         PROF_T(p1);
@@ -315,42 +353,65 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
           ptx::tmem_ld_32x32(taddr, v0);
           ptx::tmem_ld_32x32(taddr + 32, v1);
           ptx::tmem_wait_ld();
-          float a0 = 0.f, a1 = 0.f;
+          // w ReLU(x) = (w/2) x + (w/2) |x|: two full-rate FMAs per element (|x| is a free
+          // operand modifier) instead of a half-rate max plus an FMA; ct.w holds w/2.
+          // Eight independent accumulation chains keep the FMA pipe busy.
+          float ap[4] = {0.f, 0.f, 0.f, 0.f}, an[4] = {0.f, 0.f, 0.f, 0.f};
           const float4* wp = reinterpret_cast<const float4*>(&ct.w[r][0]);
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const float4 wa = wp[j], wb = wp[8 + j];
-            a0 = fmaf(wa.x, fmaxf(__uint_as_float(v0[4 * j]), 0.f), a0);
-            a1 = fmaf(wb.x, fmaxf(__uint_as_float(v1[4 * j]), 0.f), a1);
-            a0 = fmaf(wa.y, fmaxf(__uint_as_float(v0[4 * j + 1]), 0.f), a0);
-            a1 = fmaf(wb.y, fmaxf(__uint_as_float(v1[4 * j + 1]), 0.f), a1);
-            a0 = fmaf(wa.z, fmaxf(__uint_as_float(v0[4 * j + 2]), 0.f), a0);
-            a1 = fmaf(wb.z, fmaxf(__uint_as_float(v1[4 * j + 2]), 0.f), a1);
-            a0 = fmaf(wa.w, fmaxf(__uint_as_float(v0[4 * j + 3]), 0.f), a0);
-            a1 = fmaf(wb.w, fmaxf(__uint_as_float(v1[4 * j + 3]), 0.f), a1);
+            const float x0 = __uint_as_float(v0[4 * j]), x1 = __uint_as_float(v0[4 * j + 1]);
+            const float x2 = __uint_as_float(v0[4 * j + 2]), x3 = __uint_as_float(v0[4 * j + 3]);
+            const float y0 = __uint_as_float(v1[4 * j]), y1 = __uint_as_float(v1[4 * j + 1]);
+            const float y2 = __uint_as_float(v1[4 * j + 2]), y3 = __uint_as_float(v1[4 * j + 3]);
+            ap[0] = fmaf(fabsf(x0), wa.x, ap[0]); an[0] = fmaf(x0, wa.x, an[0]);
+            ap[1] = fmaf(fabsf(x1), wa.y, ap[1]); an[1] = fmaf(x1, wa.y, an[1]);
+            ap[2] = fmaf(fabsf(x2), wa.z, ap[2]); an[2] = fmaf(x2, wa.z, an[2]);
+            ap[3] = fmaf(fabsf(x3), wa.w, ap[3]); an[3] = fmaf(x3, wa.w, an[3]);
+            ap[0] = fmaf(fabsf(y0), wb.x, ap[0]); an[0] = fmaf(y0, wb.x, an[0]);
+            ap[1] = fmaf(fabsf(y1), wb.y, ap[1]); an[1] = fmaf(y1, wb.y, an[1]);
+            ap[2] = fmaf(fabsf(y2), wb.z, ap[2]); an[2] = fmaf(y2, wb.z, an[2]);
+            ap[3] = fmaf(fabsf(y3), wb.w, ap[3]); an[3] = fmaf(y3, wb.w, an[3]);
           }
-          score[rl] = a0 + a1;
+          score[rl] = ((ap[0] + an[0]) + (ap[1] + an[1])) + ((ap[2] + an[2]) + (ap[3] + an[3]));
         }
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
         PROF_T(p3);
         PROF_ADD(2, p2, p3);
-        // ---- filter + append to this warp's own segment (register cursor, no atomics)
+        // ---- count every score in the row histogram, append the ones above the threshold
+        uint32_t key[C::ROWS_PER_TEAM];
+        bool valid[C::ROWS_PER_TEAM];
+#pragma unroll
+        for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
+          key[rl] = score_to_key(kscale ? score[rl] * ksv : score[rl]);
+          valid[rl] = s_key < n_vis[rl];
+        }
+        if (t == 0) {          // anchor the histogram range on the first tile's maximum
+#pragma unroll
+          for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
+            const uint32_t mx = __reduce_max_sync(0xffffffffu, valid[rl] ? key[rl] : 0u);
+            if (lane == 0) atomicMax(&ct.rowmax[team * C::ROWS_PER_TEAM + rl], mx);
+          }
+          tm.sync();
+#pragma unroll
+          for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
+            const int top = (int)(ct.rowmax[team * C::ROWS_PER_TEAM + rl] >> 15) + 512 - (kSelBins - 1);
+            base[rl] = top > 0 ? top : 0;
+          }
+        }
 #pragma unroll
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
           const int r = team * C::ROWS_PER_TEAM + rl;
-          const float sv = kscale ? score[rl] * ksv : score[rl];
-          const uint32_t key = score_to_key(sv);
-          const bool take = s_key < n_vis[rl] && key > thr[rl];
+          if (valid[rl]) atomicAdd(&ct.rhist[r][key_bin(key[rl], base[rl])], 1u);
+          const bool take = valid[rl] && key[rl] > thr[rl];
           const uint32_t m = __ballot_sync(0xffffffffu, take);
           if (take) {
             const int p = cnt[rl] + __popc(m & ((1u << lane) - 1u));
-            if (p < SEG) {
-              sc.cand64[seg_off(r, cur[rl]) + p] = make_entry(key, s_key);
-            } else {
-              ct.abort_code = DEV_CAND_OVERFLOW;
-            }
+            if (p < SEG) seg_ptr(r)[p] = make_entry(key[rl], s_key);
+            else ct.abort_code = DEV_CAND_OVERFLOW;
           }
           cnt[rl] = min(cnt[rl] + __popc(m), SEG);
           if (lane == 0 && cnt[rl] + 32 > SEG) ct.flag[r] = 1;
@@ -358,6 +419,15 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         PROF_T(p4);
         PROF_ADD(3, p3, p4);
         tm.sync();
+        if ((t & 31) == 31) {  // refresh the thresholds from the histograms
+#pragma unroll
+          for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
+            if (Ksel[rl] > 0) {
+              const uint32_t th = hist_threshold(team * C::ROWS_PER_TEAM + rl, Ksel[rl], base[rl]);
+              thr[rl] = th > thr[rl] ? th : thr[rl];
+            }
+          }
+        }
         PROF_T(p5);
         PROF_ADD(4, p4, p5);
 #ifdef PIVOT_PROFILE
@@ -373,14 +443,18 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         const int K = Ksel[rl];
         if (K <= 0) continue;
         const RowDesc rd = rows[ri];
-        if (tt == 0) sel.total = 0;
-        tm.sync();
-        if (lane == 0) atomicAdd(&sel.total, (uint32_t)cnt[rl]);
-        tm.sync();
-        const int n = (int)sel.total;
-        const Seg seg{sc.cand64 + seg_off(r, cur[rl]), cnt[rl]};
-        const int n_valid = SEG <= 2048 ? seg_emit<64, true>(tm, sel, seg, n, rd.out, rd.out_score, K)
-                                        : seg_emit<128, false>(tm, sel, seg, n, rd.out, rd.out_score, K);
+        int n = team_sum(cnt[rl]);
+        int mxc = team_max(cnt[rl]);
+        if (mxc > 32 * kSelEpt) {     // too many for the register-resident select: drop the dead ones first
+          const uint32_t th = hist_threshold(r, K, base[rl]);
+          const uint32_t tcur = th > thr[rl] ? th : thr[rl];
+          cnt[rl] = seg_filter_inplace(seg_ptr(r), cnt[rl], lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
+          n = team_sum(cnt[rl]);
+          mxc = team_max(cnt[rl]);
+        }
+        const Seg seg{seg_ptr(r), cnt[rl]};
+        const int n_valid = mxc <= 32 * kSelEpt ? seg_emit<true>(tm, sel, seg, n, rd.out, rd.out_score, K)
+                                                : seg_emit<false>(tm, sel, seg, n, rd.out, rd.out_score, K);
         for (int i = n_valid + tt; i < K; i += 128) {
           rd.out[i] = -1;
           if (rd.out_score) rd.out_score[i] = -INFINITY;

@@ -7,14 +7,16 @@
 //
 // The streaming select of the tensor-core kernels keeps, per row, one candidate segment per
 // epilogue warp: warp w appends only to its own segment (cursor in a register, no atomics), and
-// entry e of a segment belongs to lane e % 32.  A selection loads every lane's entries into
-// registers once and then finds the K-th largest entry of the union by histogramming:
+// entry e of a segment belongs to lane e % 32.  A selection finds the K-th largest entry of the
+// union of the four segments by histogramming:
 //   1. reduce the range [lo, hi] of the entries;
 //   2. 2048 bins, linear over [lo, hi]; count; walk the bins from the top to the one that holds
 //      the K-th entry (the boundary bin);
 //   3. if the boundary bin is small (<= 256 entries) rank its entries by brute force, else
 //      narrow [lo, hi] to that bin and repeat (the width shrinks 2048-fold per round).
 // The result is the cut: an entry is among the K best iff entry >= cut.
+// Lanes hold their entries in registers when a segment has at most 32 * EPT entries
+// (CACHED = true, loops unrolled) and re-read them from memory otherwise (rolled loops).
 #pragma once
 #include "common.cuh"
 #include "select.cuh"
@@ -33,6 +35,7 @@ __device__ unsigned long long g_sel_prof[16];
 
 constexpr int kSelBins = 2048;
 constexpr int kSelSmall = 256;
+constexpr int kSelEpt = 64;      // register-cached entries per lane
 
 typedef unsigned long long entry_t;
 
@@ -41,8 +44,7 @@ __device__ __forceinline__ entry_t make_entry(uint32_t key, int32_t pos) {
 }
 __device__ __forceinline__ uint32_t entry_key(entry_t e) { return (uint32_t)(e >> 32); }
 __device__ __forceinline__ int32_t entry_pos(entry_t e) { return (int32_t)(~(uint32_t)e); }
-// Padding entry: lowest possible, position -1.
-constexpr entry_t kPadEntry = 0ull;
+constexpr entry_t kPadEntry = 0ull;   // lowest possible entry, position -1: never selected
 
 struct SegSelSmem {
   uint32_t hist[kSelBins];
@@ -54,48 +56,104 @@ struct SegSelSmem {
   uint32_t list_n;
   uint32_t out_count;
   uint32_t total;
+  uint32_t maxcnt;
 };
 
 // One warp's view of its segment (warp-uniform count).
 struct Seg {
-  const entry_t* e;
+  entry_t* e;
   int cnt;
 };
 
-// A lane's entries: cached in registers (EPT entries at most) or re-read on each use.
-template <int EPT, bool CACHED>
+// A lane's entries: entry j of the lane is segment element j * 32 + lane.
+template <bool CACHED>
 struct SegRegs {
-  entry_t v[CACHED ? EPT : 1];
+  entry_t v[CACHED ? kSelEpt : 1];
   const entry_t* base;
-  __device__ __forceinline__ void load(const Seg& s, int lane, int nj) {
+  int nj;      // this lane's entry count
+  __device__ __forceinline__ void load(const Seg& s, int lane) {
     base = s.e + lane;
+    nj = s.cnt > lane ? (s.cnt - lane + 31) >> 5 : 0;
     if constexpr (CACHED) {
 #pragma unroll
-      for (int j = 0; j < EPT; ++j) v[j] = j < nj ? __ldcg(s.e + j * 32 + lane) : kPadEntry;
+      for (int j = 0; j < kSelEpt; ++j) v[j] = j < nj ? __ldcg(base + j * 32) : kPadEntry;
     }
   }
-  __device__ __forceinline__ entry_t get(int j) const {
-    if constexpr (CACHED) return v[j];
-    else return __ldcg(base + j * 32);
+  template <typename F>
+  __device__ __forceinline__ void for_each(F f) const {
+    if constexpr (CACHED) {
+#pragma unroll
+      for (int j = 0; j < kSelEpt; ++j)
+        if (j < nj) f(v[j]);
+    } else {
+#pragma unroll 4
+      for (int j = 0; j < nj; ++j) f(__ldcg(base + j * 32));
+    }
+  }
+  // Warp-uniform trip count njw = ceil(cnt / 32): f(x, valid) runs for every lane.
+  template <typename F>
+  __device__ __forceinline__ void for_each_uniform(int njw, F f) const {
+    if constexpr (CACHED) {
+#pragma unroll
+      for (int j = 0; j < kSelEpt; ++j)
+        if (j < njw) f(j < nj ? v[j] : kPadEntry, j < nj);
+    } else {
+      for (int j = 0; j < njw; ++j) f(j < nj ? __ldcg(base + j * 32) : kPadEntry, j < nj);
+    }
   }
 };
 
-// Finds the K-th largest entry among the team's segments (more than K entries in total).
-// All 128 threads call; the cut is returned (and left in sm.cut).
-template <int EPT, bool CACHED>
-__device__ __forceinline__ entry_t seg_find_cut(const Team& tm, SegSelSmem& sm, const SegRegs<EPT, CACHED>& regs,
-                                                int nj, int K) {
+// Boundary bin of a 2048-bin histogram walked from the top: the largest bin b such that the
+// bins >= b hold at least `need` entries.  Leaves (bin, need inside that bin, its population)
+// in sm.bin / sm.need / sm.pop; if the histogram holds fewer than `need` entries, bin = 0 and
+// pop = need = 0.  All 128 threads call.
+__device__ __forceinline__ void hist_boundary(const Team& tm, SegSelSmem& sm, const uint32_t* hist, uint32_t need) {
   const int lane = tm.tid & 31;
   const int wq = tm.tid >> 5;
+  tm.sync();          // everyone is done with the previous result, and the histogram is complete
+  uint32_t loc[16];
+  uint32_t s = 0;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) { loc[i] = hist[kSelBins - 1 - 16 * tm.tid - i]; s += loc[i]; }
+  uint32_t incl = s;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) sm.wsum[wq] = incl;
+  if (tm.tid == 0) { sm.bin = 0; sm.need = 0; sm.pop = 0; }
+  tm.sync();
+  uint32_t base = 0;
+  for (int w = 0; w < wq; ++w) base += sm.wsum[w];
+  const uint32_t excl = base + incl - s;
+  if (excl < need && need <= excl + s) {
+    uint32_t cum = excl;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      if (cum + loc[i] >= need) {
+        sm.bin = (uint32_t)(kSelBins - 1 - 16 * tm.tid - i);
+        sm.need = need - cum;
+        sm.pop = loc[i];
+        break;
+      }
+      cum += loc[i];
+    }
+  }
+  tm.sync();
+}
+
+// Finds the K-th largest entry among the team's segments (more than K real entries in total).
+// All 128 threads call; the cut is returned (and left in sm.cut).
+template <bool CACHED>
+__device__ __forceinline__ entry_t seg_find_cut(const Team& tm, SegSelSmem& sm, const SegRegs<CACHED>& regs, int K) {
+  const int lane = tm.tid & 31;
   SELP_T(q0);
   entry_t mn = ~0ull, mx = 0ull;
-#pragma unroll
-  for (int j = 0; j < EPT; ++j)
-    if (j < nj) {
-      const entry_t x = regs.get(j);
-      mn = (x < mn && x != kPadEntry) ? x : mn;     // padding never bounds the range
-      mx = x > mx ? x : mx;
-    }
+  regs.for_each([&](entry_t x) {
+    mn = (x < mn && x != kPadEntry) ? x : mn;     // padding never bounds the range
+    mx = x > mx ? x : mx;
+  });
   if (tm.tid == 0) { sm.vmin = ~0ull; sm.vmax = 0ull; }
   tm.sync();
 #pragma unroll
@@ -118,45 +176,13 @@ __device__ __forceinline__ entry_t seg_find_cut(const Team& tm, SegSelSmem& sm, 
     const int shift = bitsw > 11 ? bitsw - 11 : 0;
     for (int i = tm.tid; i < kSelBins; i += tm.nthr) sm.hist[i] = 0;
     tm.sync();
-#pragma unroll
-    for (int j = 0; j < EPT; ++j)
-      if (j < nj) {
-        const entry_t x = regs.get(j);
-        if (x >= lo && x <= hi) atomicAdd(&sm.hist[(uint32_t)((x - lo) >> shift)], 1u);
-      }
+    regs.for_each([&](entry_t x) {
+      if (x >= lo && x <= hi) atomicAdd(&sm.hist[(uint32_t)((x - lo) >> shift)], 1u);
+    });
     tm.sync();
     SELP_T(r1);
     SELP_ADD(1, r0, r1);
-    // boundary bin, walking from the top: thread t owns bins 2047-16t .. 2032-16t
-    uint32_t loc[16];
-    uint32_t s = 0;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) { loc[i] = sm.hist[kSelBins - 1 - 16 * tm.tid - i]; s += loc[i]; }
-    uint32_t incl = s;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += v;
-    }
-    if (lane == 31) sm.wsum[wq] = incl;
-    tm.sync();
-    uint32_t base = 0;
-    for (int w = 0; w < wq; ++w) base += sm.wsum[w];
-    const uint32_t excl = base + incl - s;
-    if (excl < need && need <= excl + s) {
-      uint32_t cum = excl;
-#pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        if (cum + loc[i] >= need) {
-          sm.bin = (uint32_t)(kSelBins - 1 - 16 * tm.tid - i);
-          sm.need = need - cum;
-          sm.pop = loc[i];
-          break;
-        }
-        cum += loc[i];
-      }
-    }
-    tm.sync();
+    hist_boundary(tm, sm, sm.hist, need);
     const uint32_t b = sm.bin, pop = sm.pop;
     need = sm.need;
     const entry_t lo2 = lo + ((entry_t)b << shift);
@@ -175,15 +201,12 @@ __device__ __forceinline__ entry_t seg_find_cut(const Team& tm, SegSelSmem& sm, 
     if (pop <= (uint32_t)kSelSmall) {   // rank the boundary bin's entries by brute force
       if (tm.tid == 0) sm.list_n = 0;
       tm.sync();
-#pragma unroll
-      for (int j = 0; j < EPT; ++j)
-        if (j < nj) {
-          const entry_t x = regs.get(j);
-          if (x >= lo2 && x <= hi2) {
-            const uint32_t p = atomicAdd(&sm.list_n, 1u);
-            if (p < (uint32_t)kSelSmall) sm.list[p] = x;
-          }
+      regs.for_each([&](entry_t x) {
+        if (x >= lo2 && x <= hi2) {
+          const uint32_t p = atomicAdd(&sm.list_n, 1u);
+          if (p < (uint32_t)kSelSmall) sm.list[p] = x;
         }
+      });
       tm.sync();
       const int P = min((int)sm.list_n, kSelSmall);
       for (int t = tm.tid; t < P; t += tm.nthr) {
@@ -205,87 +228,82 @@ __device__ __forceinline__ entry_t seg_find_cut(const Team& tm, SegSelSmem& sm, 
   return lo;
 }
 
-// Compaction: keeps the K best entries; every warp rewrites its survivors into `dst` (its own
-// segment of the other ping-pong half) and returns its new count.  *cut_out gets the cut.
-template <int EPT, bool CACHED>
-__device__ __forceinline__ int seg_compact(const Team& tm, SegSelSmem& sm, const Seg& seg, entry_t* dst, int K,
-                                           entry_t* cut_out) {
-  const int lane = tm.tid & 31;
-  const int nj = seg.cnt > lane ? (seg.cnt - lane + 31) >> 5 : 0;
-  SegRegs<EPT, CACHED> regs;
-  regs.load(seg, lane, nj);
-  SELP_T(c1);
-  const entry_t cut = seg_find_cut<EPT, CACHED>(tm, sm, regs, nj, K);
-  SELP_T(c2);
-  SELP_ADD(5, c1, c2);
+// In-place filter of one warp's segment: keeps the entries for which pred holds, in order,
+// and returns the new count.  Safe in place: writes never pass the read position.  Warp-local.
+template <typename Pred>
+__device__ __forceinline__ int seg_filter_inplace(entry_t* e, int cnt, int lane, Pred pred) {
   int out = 0;
-  const int njw = (seg.cnt + 31) >> 5;          // warp-uniform trip count
+  for (int j0 = 0; j0 < cnt; j0 += 128) {        // four rows of 32 in flight
+    entry_t x[4];
 #pragma unroll
-  for (int j = 0; j < EPT; ++j) {
-    if (j < njw) {
-      const entry_t x = j < nj ? regs.get(j) : kPadEntry;
-      const bool keep = j < nj && x >= cut;
+    for (int u = 0; u < 4; ++u) {
+      const int i = j0 + u * 32 + lane;
+      x[u] = i < cnt ? __ldcg(e + i) : kPadEntry;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const bool keep = (j0 + u * 32 + lane) < cnt && pred(x[u]);
       const uint32_t m = __ballot_sync(0xffffffffu, keep);
-      if (keep) dst[out + __popc(m & ((1u << lane) - 1u))] = x;
+      if (keep) e[out + __popc(m & ((1u << lane) - 1u))] = x[u];
       out += __popc(m);
     }
+    __syncwarp();
   }
-  *cut_out = cut;
-  SELP_T(c3);
-  SELP_ADD(6, c2, c3);
-#ifdef PIVOT_PROFILE
-  if (tm.tid == 0 && tm.bar == 1 && blockIdx.x == 0) g_sel_prof[10] += 1;
-#endif
   return out;
 }
 
-// Writes the positions (and optionally scores) of the entries flagged by `pred` through the
-// team cursor sm.out_count; entries at position -1 (padding) are skipped.
-template <int EPT, bool CACHED, typename Pred>
-__device__ __forceinline__ void seg_write_out(const Team& tm, SegSelSmem& sm, const SegRegs<EPT, CACHED>& regs,
-                                              int nj, int njw, int32_t* out, float* out_score, int K, Pred pred) {
+// Exact compaction in place: keeps the K best entries of the team's segments; returns this
+// warp's new count and the cut through *cut_out.  Needs more than K real entries in total.
+template <bool CACHED>
+__device__ __forceinline__ int seg_compact(const Team& tm, SegSelSmem& sm, const Seg& seg, int K, entry_t* cut_out) {
   const int lane = tm.tid & 31;
-#pragma unroll
-  for (int j = 0; j < EPT; ++j) {
-    if (j < njw) {
-      const entry_t x = j < nj ? regs.get(j) : kPadEntry;
-      const bool keep = j < nj && entry_pos(x) >= 0 && pred(x);
+  SegRegs<CACHED> regs;
+  regs.load(seg, lane);
+  const entry_t cut = seg_find_cut<CACHED>(tm, sm, regs, K);
+  *cut_out = cut;
+  if constexpr (CACHED) {
+    int out = 0;
+    regs.for_each_uniform((seg.cnt + 31) >> 5, [&](entry_t x, bool valid) {
+      const bool keep = valid && x >= cut;
       const uint32_t m = __ballot_sync(0xffffffffu, keep);
-      if (m) {
-        uint32_t pos = 0;
-        const int leader = __ffs(m) - 1;
-        if (lane == leader) pos = atomicAdd(&sm.out_count, (uint32_t)__popc(m));
-        pos = __shfl_sync(0xffffffffu, pos, leader);
-        if (keep) {
-          const uint32_t p = pos + __popc(m & ((1u << lane) - 1u));
-          if (p < (uint32_t)K) {
-            out[p] = entry_pos(x);
-            if (out_score) out_score[p] = key_to_score(entry_key(x));
-          }
-        }
-      }
-    }
+      if (keep) seg.e[out + __popc(m & ((1u << lane) - 1u))] = x;
+      out += __popc(m);
+    });
+    return out;
+  } else {
+    return seg_filter_inplace(seg.e, seg.cnt, lane, [cut](entry_t x) { return x >= cut; });
   }
 }
 
 // Final selection of a row: writes min(K, n_valid) positions (unordered) to out, returns how
 // many.  n_valid = real (non-padding) entries in the team's segments.
-template <int EPT, bool CACHED>
+template <bool CACHED>
 __device__ __forceinline__ int seg_emit(const Team& tm, SegSelSmem& sm, const Seg& seg, int n_valid, int32_t* out,
                                         float* out_score, int K) {
   const int lane = tm.tid & 31;
-  const int nj = seg.cnt > lane ? (seg.cnt - lane + 31) >> 5 : 0;
-  const int njw = (seg.cnt + 31) >> 5;
-  SegRegs<EPT, CACHED> regs;
-  regs.load(seg, lane, nj);
+  SegRegs<CACHED> regs;
+  regs.load(seg, lane);
   if (tm.tid == 0) sm.out_count = 0;
   tm.sync();
-  if (n_valid > K) {
-    const entry_t cut = seg_find_cut<EPT, CACHED>(tm, sm, regs, nj, K);
-    seg_write_out<EPT, CACHED>(tm, sm, regs, nj, njw, out, out_score, K, [cut](entry_t x) { return x >= cut; });
-  } else {
-    seg_write_out<EPT, CACHED>(tm, sm, regs, nj, njw, out, out_score, K, [](entry_t) { return true; });
-  }
+  entry_t cut = 0ull;
+  if (n_valid > K) cut = seg_find_cut<CACHED>(tm, sm, regs, K);
+  regs.for_each_uniform((seg.cnt + 31) >> 5, [&](entry_t x, bool valid) {
+    const bool keep = valid && entry_pos(x) >= 0 && x >= cut;
+    const uint32_t m = __ballot_sync(0xffffffffu, keep);
+    if (m) {
+      uint32_t pos = 0;
+      const int leader = __ffs(m) - 1;
+      if (lane == leader) pos = atomicAdd(&sm.out_count, (uint32_t)__popc(m));
+      pos = __shfl_sync(0xffffffffu, pos, leader);
+      if (keep) {
+        const uint32_t p = pos + __popc(m & ((1u << lane) - 1u));
+        if (p < (uint32_t)K) {
+          out[p] = entry_pos(x);
+          if (out_score) out_score[p] = key_to_score(entry_key(x));
+        }
+      }
+    }
+  });
   tm.sync();
   return n_valid > K ? K : n_valid;
 }
