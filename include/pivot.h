@@ -146,6 +146,24 @@ int dense_index_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kc
                    const pivot_opts* opts);
 
 /*
+ * dense_index without any caller-provided scratch (no counterpart in the paper: this is a
+ * deployment convenience, not part of the method).  For hosts that may not allocate device
+ * memory -- a plugin inside a server that owns the device heap, code bound to a framework's
+ * memory pool -- the scratch comes from an 8 MiB array built into the library image (every GPU
+ * that loads the library holds it until the process exits).  Same arguments and result as
+ * dense_index; q, w, kcache, out_idx are device pointers as usual.
+ *   Limits: L <= 4096 and k <= 512, else PIVOT_ERR_WORKSPACE.  Runs on a reduced grid, so it is
+ *   slower than dense_index.
+ *   The first call on a device looks up the array's device address; make that call before any
+ *   stream capture.  Calls never allocate or free.
+ *   All calls on a device share the array (it keeps the previous call's contents; what must
+ *   start at zero is cleared on `stream`): calls that overlap on the GPU race -- run them on
+ *   one stream, or order them otherwise.  pivot_device_status does not cover this entry point.
+ */
+int dense_index_static(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                       int L, int H_I, int d, int k, int32_t* out_idx, pivot_stream_t stream);
+
+/*
  * Host-buffer form of pivot_index_prefill: every tensor pointer (q, w, kcache, out_idx) is HOST
  * memory (pinned for full copy speed).  The call copies the inputs into `arena` (device,
  * at least pivot_prefill_host_arena_bytes(...) bytes, which includes the workspace), runs the

@@ -22,7 +22,7 @@ OK = 0
 
 SYMBOLS = [
     "pivot_workspace_bytes", "pivot_set_workspace", "pivot_index_prefill", "pivot_index_prefill_ex",
-    "pivot_index_decode", "pivot_index_decode_ex", "dense_index", "dense_index_ex",
+    "pivot_index_decode", "pivot_index_decode_ex", "dense_index", "dense_index_ex", "dense_index_static",
     "pivot_prefill_host_arena_bytes", "pivot_index_prefill_host", "pivot_device_status",
     "pivot_stage_timing", "pivot_stage_times", "pivot_launch_count_reset", "pivot_status_str", "pivot_last_cuda_error",
 ]
@@ -58,6 +58,7 @@ def _load():
     lib.pivot_index_decode_ex.argtypes = [T, P, T, P, I, I, I, I, I, I, I, I, P, P, O]
     lib.dense_index.argtypes = [T, P, T, I, I, I, I, P, P]
     lib.dense_index_ex.argtypes = [T, P, T, I, I, I, I, P, P, O]
+    lib.dense_index_static.argtypes = [T, P, T, I, I, I, I, P, P]
     lib.pivot_prefill_host_arena_bytes.restype = S
     lib.pivot_prefill_host_arena_bytes.argtypes = [I, I, I, I, I, I, I]
     lib.pivot_index_prefill_host.argtypes = [T, P, T, I, I, I, I, I, I, I, P, P, S, P]
@@ -158,6 +159,17 @@ def dense_index(q, w, kcache, L, H_I, d, k, out_idx, stream=None, *, q_scale=Non
     o = _opts(None, POOL_MEAN, None, dbg_scores, None, workspace, impl)
     _check(lib.dense_index_ex(C.byref(tq), w.data_ptr(), C.byref(tk), L, H_I, d, k, out_idx.data_ptr(),
                               _stream(stream), C.byref(o)))
+    return out_idx
+
+
+def dense_index_static(q, w, kcache, L, H_I, d, k, out_idx, stream=None, *, q_scale=None, k_scale=None):
+    """dense_index for callers that may not allocate device memory: no workspace argument, the
+    scratch is an array built into the library (L <= 4096, k <= 512).  Nothing is allocated
+    here either -- the tensors are the caller's."""
+    tq, tk = _tensor(q, q_scale), _tensor(kcache, k_scale)
+    assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and out_idx.numel() >= L * k
+    _check(lib.dense_index_static(C.byref(tq), w.data_ptr(), C.byref(tk), L, H_I, d, k, out_idx.data_ptr(),
+                                  _stream(stream)))
     return out_idx
 
 
