@@ -59,7 +59,7 @@ enum {
  *   scale  NULL for bf16.  FP8: one fp32 scale per d-vector -- queries [L, H_I]
  *          (decode [B, g, H_I]), keys [L] (decode [B, Lmax]); value = code * scale.
  *   dtype  PIVOT_BF16 or PIVOT_FP8_E4M3; q and kcache must agree.
- * data must be 16-byte aligned, scale 4-byte aligned.
+ * data must be 16-byte aligned; the key-cache scale 16-byte aligned, the query scale 4-byte.
  */
 typedef struct pivot_tensor {
   const void* data;
@@ -126,6 +126,8 @@ int pivot_index_prefill_ex(const pivot_tensor* q, const float* w, const pivot_te
  *   q       [B, g, H_I, d]; w [B, g, H_I]; kcache [B, Lmax, d] (+ scale [B, Lmax]); sequence b's
  *           cache must hold keys 0 .. pos0[b]+g-1.
  *   pos0    [B] int32, device.  The proxy scan is cut at pos0[b] (inclusive).
+ *   Lmax    rows per sequence in kcache; with FP8 it must be a multiple of 4 (each sequence's
+ *           scale row then starts on a 16-byte boundary).
  *   out_idx [B, g, k] int32.
  */
 int pivot_index_decode(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,

@@ -140,8 +140,8 @@ int check_common(const pivot_tensor* q, const float* w, const pivot_tensor* kc, 
   if (mode != PIVOT_REUSE && mode != PIVOT_REFINE) return PIVOT_ERR_INVALID_ARG;
   if (mode == PIVOT_REFINE && k > c) return PIVOT_ERR_INVALID_ARG;
   if (((uintptr_t)q->data | (uintptr_t)kc->data) & 15) return PIVOT_ERR_INVALID_ARG;
-  if (((uintptr_t)w | (uintptr_t)out | (uintptr_t)q->scale | (uintptr_t)kc->scale) & 3)
-    return PIVOT_ERR_INVALID_ARG;
+  if (((uintptr_t)w | (uintptr_t)out | (uintptr_t)q->scale) & 3) return PIVOT_ERR_INVALID_ARG;
+  if ((uintptr_t)kc->scale & 15) return PIVOT_ERR_INVALID_ARG;
   if (H != kHeads || d != kDim) return PIVOT_ERR_UNSUPPORTED;
   if (k > kMaxSel || c > kMaxSel) return PIVOT_ERR_UNSUPPORTED;
   return PIVOT_OK;
@@ -193,7 +193,7 @@ int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, i
   if (o && o->impl == 1) {
     launch_scan_simt(ws.rows, p.n_dense + p.n_proxy, q->dtype, ws.scan, st);
   } else {
-    ScanOperands op{kc->data, L, q->data, L, ws.proxy_q, p.n_proxy, q->dtype};
+    ScanOperands op{kc->data, L, kc->scale, q->data, L, ws.proxy_q, p.n_proxy, q->dtype};
     if ((rc = check_cuda(launch_scan_tc(op, ws.rows, p.n_dense + p.n_proxy, 4, tc_scratch(ws), sm_count(), st))))
       return rc;
   }
@@ -261,6 +261,8 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
   int rc = check_common(q, w, kcache, H_I, d, c, k, mode, out_idx);
   if (rc) return rc;
   if (!pos0 || B < 1 || g < 1 || Lmax < g) return PIVOT_ERR_INVALID_ARG;
+  // every sequence's scale row must start on a 16-byte boundary (TMA reads it in 128-scale tiles)
+  if (q->dtype == PIVOT_FP8_E4M3 && (Lmax & 3)) return PIVOT_ERR_INVALID_ARG;
   if (o && (o->pool < 0 || o->pool > 2)) return PIVOT_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t need = pivot_workspace_bytes(B * g, B, c, k);
@@ -288,7 +290,7 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
   if (o && o->impl == 1) {
     launch_scan_simt(ws.rows, B + B * g, q->dtype, ws.scan, st);
   } else {
-    ScanOperands op{kcache->data, (long long)B * Lmax, q->data, B * g, ws.proxy_q, B, q->dtype};
+    ScanOperands op{kcache->data, (long long)B * Lmax, kcache->scale, q->data, B * g, ws.proxy_q, B, q->dtype};
     if ((rc = check_cuda(launch_scan_tc(op, ws.rows, B + B * g, 1, tc_scratch(ws), sm_count(), st)))) return rc;
   }
   mark(3, st);

@@ -74,6 +74,7 @@ void launch_refine_simt(const GroupDesc* groups, int n_groups, int dtype, const 
 // Operand tensors of a tensor-core scan, for the TMA tensor maps.
 struct ScanOperands {
   const void* kc; long long k_rows;        // key cache [k_rows, d]
+  const float* kscale;                     // [k_rows] (FP8) or nullptr
   const void* q; int q_rows;               // raw queries [q_rows, H, d]
   const void* proxy_q; int proxy_rows;     // proxies [proxy_rows, H, d]
   int dtype;

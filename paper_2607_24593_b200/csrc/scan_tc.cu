@@ -14,6 +14,7 @@
 // warps 2.. = epilogue (two warps per TMEM lane quarter, each pair of rows handled by its own
 // 128-thread team).  Row blocks are dealt to CTAs longest-first in snake order.
 #include <cuda.h>
+#include <string.h>
 
 #include "kernels.h"
 #include "ptx.cuh"
@@ -33,6 +34,7 @@ namespace {
 
 constexpr int TILE_KEYS = 128;
 constexpr int MAX_STAGES = 8;
+constexpr int KS_SLOTS = 12;      // key-scale ring: deeper than (key stages + accumulator buffers)
 
 template <int DT, int NROWS>
 struct Cfg {
@@ -46,9 +48,11 @@ struct Cfg {
   static constexpr int QBUF_BYTES = KHALVES * QHALF_BYTES;
   static constexpr int N = NROWS * kHeads;
   static constexpr int QBUFS = (!FP8 && NROWS == 4) ? 1 : 2;   // bf16 x 4 rows: 64 KB per query buffer
-  static constexpr int STAGES = FP8 ? 6 : (NROWS == 4 ? 3 : 4);
-  static constexpr int EPI_WARPS = NROWS == 4 ? 8 : 4;
-  static constexpr int ROWS_PER_TEAM = NROWS == 4 ? 2 : 1;
+  static constexpr int STAGES = NROWS == 4 ? (FP8 ? 4 : 2) : (FP8 ? 6 : 4);
+  // One 4-warp team per row: 16 epilogue warps (four per scheduler) hide each other's latencies.
+  static constexpr int EPI_WARPS = NROWS == 4 ? 16 : 4;
+  static constexpr int ROWS_PER_TEAM = 1;
+  static constexpr bool SEL_CACHED = NROWS != 4;   // 576 threads leave too few registers to cache entries
   static constexpr int TEAMS = EPI_WARPS / 4;
   static constexpr int THREADS = 64 + EPI_WARPS * 32;
   static constexpr int TMEM_COLS = 2 * N < 32 ? 32 : 2 * N;
@@ -58,16 +62,18 @@ struct Cfg {
 
 template <int NROWS>
 struct Ctrl {
+  alignas(128) float ks[KS_SLOTS][TILE_KEYS];   // key scales of the tiles in flight (TMA destination)
   alignas(16) float w[4][kHeads];       // effective gates of the block's rows (read as float4)
   uint32_t rhist[NROWS][kSelBins];      // per row: histogram of every score seen so far
   uint64_t full[MAX_STAGES], empty[MAX_STAGES];
   uint64_t q_full[2], q_empty[2], tmem_full[2], tmem_empty[2];
+  uint64_t ks_full[KS_SLOTS];
   uint32_t tmem_base;
   int abort;
   int abort_code;         // device status to report besides a timed-out wait
   int flag[4];            // row r: a candidate segment is nearly full
   uint32_t rowmax[4];     // row r: largest score key of the first tile (anchors the histogram)
-  SegSelSmem sel[2];
+  SegSelSmem sel[NROWS == 4 ? 4 : 1];
 };
 
 template <int DT, int NROWS>
@@ -111,8 +117,8 @@ __device__ __forceinline__ int block_tiles(const RowDesc* rows, int n_rows, int 
 template <int DT, int NROWS>
 __global__ void __launch_bounds__(Cfg<DT, NROWS>::THREADS, 1)
 scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q0,
-                      const __grid_constant__ CUtensorMap tm_q1, const RowDesc* __restrict__ rows,
-                      int n_rows, ScanScratch sc) {
+                      const __grid_constant__ CUtensorMap tm_q1, const __grid_constant__ CUtensorMap tm_ks,
+                      const RowDesc* __restrict__ rows, int n_rows, ScanScratch sc) {
   using C = Cfg<DT, NROWS>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -133,6 +139,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       ptx::mbar_init(&ct.tmem_full[i], 1);
       ptx::mbar_init(&ct.tmem_empty[i], C::EPI_WARPS);
     }
+    for (int i = 0; i < KS_SLOTS; ++i) ptx::mbar_init(&ct.ks_full[i], 1);
     ct.abort = 0;
     ct.abort_code = 0;
     ptx::fence_barrier_init();
@@ -152,6 +159,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       ptx::prefetch_tensormap(&tm_k);
       ptx::prefetch_tensormap(&tm_q0);
       ptx::prefetch_tensormap(&tm_q1);
+      if (C::FP8) ptx::prefetch_tensormap(&tm_ks);
       BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
       uint32_t it = 0, blk = 0;
       bool ok = true;
@@ -183,6 +191,14 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
           for (int h = 0; h < C::KHALVES; ++h)
             ptx::tma_load_2d(kring + s * C::STAGE_BYTES + h * C::HALF_TILE_BYTES, &tm_k, h * 64,
                              k_row0 + t * TILE_KEYS, &ct.full[s]);
+          if (C::FP8) {
+            // The tile's key scales ride along into their own ring.  A slot is free again
+            // by construction: this thread runs at most STAGES tiles ahead of the MMA and the
+            // MMA at most two ahead of the epilogue, fewer than KS_SLOTS in total.
+            const int ksl = it % KS_SLOTS;
+            ptx::mbar_arrive_expect_tx(&ct.ks_full[ksl], TILE_KEYS * 4);
+            ptx::tma_load_1d(&ct.ks[ksl][0], &tm_ks, k_row0 + t * TILE_KEYS, &ct.ks_full[ksl]);
+          }
         }
         ++blk;
       }
@@ -311,19 +327,33 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         for (int i = tt; i < kSelBins; i += 128) ct.rhist[r][i] = 0;
       }
       tm.sync();
+      // The team meets only every CHK tiles (a barrier after an append waits for the store to
+      // land): that is when thresholds are refreshed and nearly full segments are dealt with,
+      // so a segment is flagged while it still has room for CHK tiles of appends.
+      const int CHK = SEG / 64 < 32 ? (SEG / 64 > 0 ? SEG / 64 : 1) : 32;
+      const int headroom = 32 * CHK;
       for (int t = 0; t < ntiles; ++t, ++it) {
         PROF_T(p0);
+        const bool meet = (t % CHK) == 0 && t > 0;
+        if (meet) {
+          tm.sync();
+#pragma unroll
+          for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
+            if (Ksel[rl] > 0) {
+              const uint32_t th = hist_threshold(team * C::ROWS_PER_TEAM + rl, Ksel[rl], base[rl]);
+              thr[rl] = th > thr[rl] ? th : thr[rl];
+            }
+          }
+        }
         // ---- a segment is nearly full: tighten the threshold and drop what fell below it;
         //      if that is not enough (ties, adversarial order) compact exactly to the K best
 #pragma unroll
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
           const int r = team * C::ROWS_PER_TEAM + rl;
-          if (ct.flag[r]) {
-            const uint32_t th = hist_threshold(r, Ksel[rl], base[rl]);
-            thr[rl] = th > thr[rl] ? th : thr[rl];
+          if (meet && ct.flag[r]) {
             const uint32_t tcur = thr[rl];
             cnt[rl] = seg_filter_inplace(seg_ptr(r), cnt[rl], lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
-            if (team_max(cnt[rl]) + 32 > SEG) {
+            if (team_max(cnt[rl]) + headroom > SEG && team_sum(cnt[rl]) > Ksel[rl]) {
               entry_t cut;
               cnt[rl] = seg_compact<false>(tm, sel, Seg{seg_ptr(r), cnt[rl]}, Ksel[rl], &cut);
               thr[rl] = entry_key(cut) > thr[rl] ? entry_key(cut) : thr[rl];
@@ -339,25 +369,55 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         PROF_ADD(0, p0, p1);
         const int buf = it & 1;
         const int s_key = t * TILE_KEYS + key_in_tile;
-        const float ksv = (kscale && s_key < nv_max) ? kscale[s_key] : 0.f;
+        // Key scales come through shared memory (TMA): a global load issued by an epilogue warp
+        // would sit in the same memory queue as its TMEM loads and stall them for an L2 round trip.
+        float ksv = 1.f;
+#ifndef EXP_NOKS_A
+        if (C::FP8) {
+          const int ksl = it % KS_SLOTS;
+          (void)ptx::mbar_wait(&ct.ks_full[ksl], (it / KS_SLOTS) & 1, abort_flag);
+#ifndef EXP_NOKS_B
+          ksv = ct.ks[ksl][key_in_tile];
+#endif
+        }
+#endif
         (void)ptx::mbar_wait(&ct.tmem_full[buf], (it >> 1) & 1, abort_flag);
         ptx::tc_fence_after();
         PROF_T(p2);
         PROF_ADD(1, p1, p2);
+#ifdef EXP_EARLY_RELEASE
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
+#endif
         float score[C::ROWS_PER_TEAM];
 #pragma unroll
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
           const int r = team * C::ROWS_PER_TEAM + rl;
           const uint32_t taddr = tmem_base + ((uint32_t)(lq * 32) << 16) + buf * C::N + r * kHeads;
           uint32_t v0[32], v1[32];
+#ifdef EXP_X64
+          {
+            uint32_t vv[64];
+            ptx::tmem_ld_32x64(taddr, vv);
+            ptx::tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) { v0[j] = vv[j]; v1[j] = vv[32 + j]; }
+          }
+#elif !defined(EXP_NOLD)
           ptx::tmem_ld_32x32(taddr, v0);
           ptx::tmem_ld_32x32(taddr + 32, v1);
           ptx::tmem_wait_ld();
+#else
+          for (int j = 0; j < 32; ++j) { v0[j] = taddr + j + it; v1[j] = taddr - j + it; }
+#endif
           // w ReLU(x) = (w/2) x + (w/2) |x|: two full-rate FMAs per element (|x| is a free
           // operand modifier) instead of a half-rate max plus an FMA; ct.w holds w/2.
           // Eight independent accumulation chains keep the FMA pipe busy.
           float ap[4] = {0.f, 0.f, 0.f, 0.f}, an[4] = {0.f, 0.f, 0.f, 0.f};
           const float4* wp = reinterpret_cast<const float4*>(&ct.w[r][0]);
+#ifdef EXP_NOFMA
+          for (int j = 0; j < 32; j += 8) ap[j >> 3] = __uint_as_float(v0[j]) + __uint_as_float(v1[j]);
+#else
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const float4 wa = wp[j], wb = wp[8 + j];
@@ -374,11 +434,14 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             ap[2] = fmaf(fabsf(y2), wb.z, ap[2]); an[2] = fmaf(y2, wb.z, an[2]);
             ap[3] = fmaf(fabsf(y3), wb.w, ap[3]); an[3] = fmaf(y3, wb.w, an[3]);
           }
+#endif
           score[rl] = ((ap[0] + an[0]) + (ap[1] + an[1])) + ((ap[2] + an[2]) + (ap[3] + an[3]));
         }
         ptx::tc_fence_before();
         __syncwarp();
+#ifndef EXP_EARLY_RELEASE
         if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
+#endif
         PROF_T(p3);
         PROF_ADD(2, p2, p3);
         // ---- count every score in the row histogram, append the ones above the threshold
@@ -386,7 +449,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         bool valid[C::ROWS_PER_TEAM];
 #pragma unroll
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
-          key[rl] = score_to_key(kscale ? score[rl] * ksv : score[rl]);
+          key[rl] = score_to_key(C::FP8 ? score[rl] * ksv : score[rl]);
           valid[rl] = s_key < n_vis[rl];
         }
         if (t == 0) {          // anchor the histogram range on the first tile's maximum
@@ -405,8 +468,15 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
 #pragma unroll
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
           const int r = team * C::ROWS_PER_TEAM + rl;
-          if (valid[rl]) atomicAdd(&ct.rhist[r][key_bin(key[rl], base[rl])], 1u);
+          // Only scores above the current threshold are counted: the ones at or below it can
+          // never reach a bin edge the threshold could still move to, so the counts that
+          // matter stay exact.
+#ifdef EXP_NOAPPEND
+          const bool take = false;
+#else
           const bool take = valid[rl] && key[rl] > thr[rl];
+#endif
+          if (take) atomicAdd(&ct.rhist[r][key_bin(key[rl], base[rl])], 1u);
           const uint32_t m = __ballot_sync(0xffffffffu, take);
           if (take) {
             const int p = cnt[rl] + __popc(m & ((1u << lane) - 1u));
@@ -414,20 +484,10 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             else ct.abort_code = DEV_CAND_OVERFLOW;
           }
           cnt[rl] = min(cnt[rl] + __popc(m), SEG);
-          if (lane == 0 && cnt[rl] + 32 > SEG) ct.flag[r] = 1;
+          if (lane == 0 && cnt[rl] + headroom > SEG) ct.flag[r] = 1;
         }
         PROF_T(p4);
         PROF_ADD(3, p3, p4);
-        tm.sync();
-        if ((t & 31) == 31) {  // refresh the thresholds from the histograms
-#pragma unroll
-          for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
-            if (Ksel[rl] > 0) {
-              const uint32_t th = hist_threshold(team * C::ROWS_PER_TEAM + rl, Ksel[rl], base[rl]);
-              thr[rl] = th > thr[rl] ? th : thr[rl];
-            }
-          }
-        }
         PROF_T(p5);
         PROF_ADD(4, p4, p5);
 #ifdef PIVOT_PROFILE
@@ -445,7 +505,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         const RowDesc rd = rows[ri];
         int n = team_sum(cnt[rl]);
         int mxc = team_max(cnt[rl]);
-        if (mxc > 32 * kSelEpt) {     // too many for the register-resident select: drop the dead ones first
+        if (!C::SEL_CACHED || mxc > 32 * kSelEpt) {   // drop the entries the final threshold already rules out
           const uint32_t th = hist_threshold(r, K, base[rl]);
           const uint32_t tcur = th > thr[rl] ? th : thr[rl];
           cnt[rl] = seg_filter_inplace(seg_ptr(r), cnt[rl], lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
@@ -453,8 +513,13 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
           mxc = team_max(cnt[rl]);
         }
         const Seg seg{seg_ptr(r), cnt[rl]};
-        const int n_valid = mxc <= 32 * kSelEpt ? seg_emit<true>(tm, sel, seg, n, rd.out, rd.out_score, K)
-                                                : seg_emit<false>(tm, sel, seg, n, rd.out, rd.out_score, K);
+        int n_valid;
+        if constexpr (C::SEL_CACHED) {
+          n_valid = mxc <= 32 * kSelEpt ? seg_emit<true>(tm, sel, seg, n, rd.out, rd.out_score, K)
+                                        : seg_emit<false>(tm, sel, seg, n, rd.out, rd.out_score, K);
+        } else {
+          n_valid = seg_emit<false>(tm, sel, seg, n, rd.out, rd.out_score, K);
+        }
         for (int i = n_valid + tt; i < K; i += 128) {
           rd.out[i] = -1;
           if (rd.out_score) rd.out_score[i] = -INFINITY;
@@ -486,7 +551,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
 // ---------------------------------------------------------------------------- host side
 
 template <int DT, int NROWS>
-cudaError_t launch_one(const CUtensorMap& mk, const CUtensorMap& mq0, const CUtensorMap& mq1,
+cudaError_t launch_one(const CUtensorMap& mk, const CUtensorMap& mq0, const CUtensorMap& mq1, const CUtensorMap& mks,
                        const RowDesc* rows, int n_rows, const ScanScratch& s, int sms, cudaStream_t st) {
   using C = Cfg<DT, NROWS>;
   auto kern = scan_select_tc_kernel<DT, NROWS>;
@@ -499,7 +564,7 @@ cudaError_t launch_one(const CUtensorMap& mk, const CUtensorMap& mq0, const CUte
   }
   const int n_blocks = (n_rows + NROWS - 1) / NROWS;
   const int grid = n_blocks < sms ? n_blocks : sms;
-  kern<<<grid, C::THREADS, smem, st>>>(mk, mq0, mq1, rows, n_rows, s);
+  kern<<<grid, C::THREADS, smem, st>>>(mk, mq0, mq1, mks, rows, n_rows, s);
   ++launch_counter();
   return cudaGetLastError();
 }
@@ -537,6 +602,19 @@ bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtyp
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 1-D map over an fp32 scale array; box = 128 scales.
+bool make_scale_map(CUtensorMap* m, const float* base, long long n) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[1] = {(cuuint64_t)n};
+  cuuint64_t strides[1] = {0};
+  cuuint32_t box[1] = {(cuuint32_t)TILE_KEYS};
+  cuuint32_t estr[1] = {1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 1, (void*)base, dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 #ifdef PIVOT_PROFILE
 extern "C" int pivot_profile_read(unsigned long long* host, int n) {
   return (int)cudaMemcpyFromSymbol(host, g_scan_prof, sizeof(unsigned long long) * (size_t)n);
@@ -549,17 +627,19 @@ extern "C" int pivot_profile_read_sel(unsigned long long* host) {
 cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_rows, int rows_per_block,
                            const ScanScratch& s, int sms, cudaStream_t st) {
   if (n_rows <= 0) return cudaSuccess;
-  CUtensorMap mk, mq0, mq1;
+  CUtensorMap mk, mq0, mq1, mks;
+  memset(&mks, 0, sizeof(mks));
+  if (op.dtype == DT_FP8 && !make_scale_map(&mks, op.kscale, op.k_rows)) return cudaErrorInvalidValue;
   if (!make_operand_map(&mk, op.kc, op.k_rows, op.dtype, TILE_KEYS) ||
       !make_operand_map(&mq0, op.q, (long long)op.q_rows * kHeads, op.dtype, kHeads) ||
       !make_operand_map(&mq1, op.proxy_q, (long long)(op.proxy_rows > 0 ? op.proxy_rows : 1) * kHeads, op.dtype, kHeads))
     return cudaErrorInvalidValue;
   if (op.dtype == DT_FP8) {
-    return rows_per_block == 4 ? launch_one<DT_FP8, 4>(mk, mq0, mq1, rows, n_rows, s, sms, st)
-                               : launch_one<DT_FP8, 1>(mk, mq0, mq1, rows, n_rows, s, sms, st);
+    return rows_per_block == 4 ? launch_one<DT_FP8, 4>(mk, mq0, mq1, mks, rows, n_rows, s, sms, st)
+                               : launch_one<DT_FP8, 1>(mk, mq0, mq1, mks, rows, n_rows, s, sms, st);
   }
-  return rows_per_block == 4 ? launch_one<DT_BF16, 4>(mk, mq0, mq1, rows, n_rows, s, sms, st)
-                             : launch_one<DT_BF16, 1>(mk, mq0, mq1, rows, n_rows, s, sms, st);
+  return rows_per_block == 4 ? launch_one<DT_BF16, 4>(mk, mq0, mq1, mks, rows, n_rows, s, sms, st)
+                             : launch_one<DT_BF16, 1>(mk, mq0, mq1, mks, rows, n_rows, s, sms, st);
 }
 
 }  // namespace pivot

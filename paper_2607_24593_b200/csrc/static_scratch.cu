@@ -79,7 +79,7 @@ extern "C" int dense_index_static(const pivot_tensor* q, const float* w, const p
   sc.status = status;
   sc.counter = status + 1;
   // the proxy tensor map needs some valid address; no row refers to it
-  ScanOperands op{kcache->data, L, q->data, L, q->data, 1, q->dtype};
+  ScanOperands op{kcache->data, L, kcache->scale, q->data, L, q->data, 1, q->dtype};
   if (launch_scan_tc(op, rows, L, 4, sc, kStaticCtas, st) != cudaSuccess) return PIVOT_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? PIVOT_OK : PIVOT_ERR_CUDA;
 }

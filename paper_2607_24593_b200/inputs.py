@@ -184,11 +184,11 @@ def make_decode(B: int, g: int, len_lo: int, len_hi: int, H: int = 64, d: int = 
 
     The visible-prefix length n0_b = pos0_b + 1 is a uniform integer in [len_lo, len_hi];
     sequence b's cache holds keys 0 .. pos0_b + g - 1 (later rows of the [B, Lmax, d]
-    buffer are zero), Lmax = len_hi + g.
+    buffer are zero), Lmax = len_hi + g rounded up to a multiple of 64.
     """
     assert dtype in ("bf16", "fp8")
     n0 = _rng(seed, _TID_LEN, 0).integers(len_lo, len_hi + 1, size=B).astype(np.int64)
-    Lmax = len_hi + g
+    Lmax = (len_hi + g + 63) // 64 * 64       # rows per sequence, rounded up (alignment of the scale rows)
     st = torch.bfloat16 if dtype == "bf16" else torch.float8_e4m3fn
     k = torch.zeros((B, Lmax, d), dtype=torch.bfloat16).to(st)
     ks = None if dtype == "bf16" else torch.zeros((B, Lmax), dtype=torch.float32)
