@@ -238,8 +238,13 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       for (int t = 0; t < ntiles; ++t, ++it) {
         const int buf = it & 1;
         const int slot = t * TILE_KEYS + key_in_tile;
+#ifdef EXP_R_NOLOADS
+        int idx = slot < gd.n_cand ? slot : -1;
+        const float ksv = 1.f;
+#else
         int idx = slot < gd.n_cand ? gd.cand[slot] : -1;
         const float ksv = (gd.kscale && idx >= 0) ? gd.kscale[idx] : 1.f;
+#endif
         (void)ptx::mbar_wait(&ct.tmem_full[buf], (it >> 1) & 1, abort_flag);
         ptx::tc_fence_after();
         float score[2];
@@ -287,8 +292,13 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         float* outs = gd.out_score ? gd.out_score + (size_t)r * gd.out_stride : nullptr;
         const int segcnt = min(ntiles * 32, SEG);
         const Seg seg{sc.cand64 + seg_off(r), segcnt};
-        const int n_valid = segcnt <= 32 * kSelEpt ? seg_emit<true>(tm, sel, seg, gd.n_cand, out, outs, gd.K)
-                                                   : seg_emit<false>(tm, sel, seg, gd.n_cand, out, outs, gd.K);
+#ifdef EXP_R_NOSELECT
+        const int n_valid = gd.K;
+#else
+        // 32 entries per lane (c <= 4096) fit the registers this kernel has; beyond that re-read
+        const int n_valid = segcnt <= 32 * 32 ? seg_emit<true, 32>(tm, sel, seg, gd.n_cand, out, outs, gd.K)
+                                              : seg_emit<false>(tm, sel, seg, gd.n_cand, out, outs, gd.K);
+#endif
         for (int i = n_valid + tt; i < gd.K; i += 128) {
           out[i] = -1;
           if (outs) outs[i] = -INFINITY;

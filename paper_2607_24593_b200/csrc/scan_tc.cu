@@ -49,10 +49,17 @@ struct Cfg {
   static constexpr int N = NROWS * kHeads;
   static constexpr int QBUFS = (!FP8 && NROWS == 4) ? 1 : 2;   // bf16 x 4 rows: 64 KB per query buffer
   static constexpr int STAGES = NROWS == 4 ? (FP8 ? 4 : 2) : (FP8 ? 6 : 4);
-  // One 4-warp team per row: 16 epilogue warps (four per scheduler) hide each other's latencies.
+  // Eight epilogue warps, two rows per 4-warp team (measured faster than one team per row with
+  // sixteen warps, which leaves only 96 registers per thread).
+#ifndef PIVOT_EPI16
+  static constexpr int EPI_WARPS = NROWS == 4 ? 8 : 4;
+  static constexpr int ROWS_PER_TEAM = NROWS == 4 ? 2 : 1;
+  static constexpr bool SEL_CACHED = true;
+#else
   static constexpr int EPI_WARPS = NROWS == 4 ? 16 : 4;
   static constexpr int ROWS_PER_TEAM = 1;
   static constexpr bool SEL_CACHED = NROWS != 4;   // 576 threads leave too few registers to cache entries
+#endif
   static constexpr int TEAMS = EPI_WARPS / 4;
   static constexpr int THREADS = 64 + EPI_WARPS * 32;
   static constexpr int TMEM_COLS = 2 * N < 32 ? 32 : 2 * N;
@@ -476,12 +483,16 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
 #else
           const bool take = valid[rl] && key[rl] > thr[rl];
 #endif
+#ifndef EXP_NOHIST
           if (take) atomicAdd(&ct.rhist[r][key_bin(key[rl], base[rl])], 1u);
+#endif
           const uint32_t m = __ballot_sync(0xffffffffu, take);
           if (take) {
             const int p = cnt[rl] + __popc(m & ((1u << lane) - 1u));
+#ifndef EXP_NOSTORE
             if (p < SEG) seg_ptr(r)[p] = make_entry(key[rl], s_key);
             else ct.abort_code = DEV_CAND_OVERFLOW;
+#endif
           }
           cnt[rl] = min(cnt[rl] + __popc(m), SEG);
           if (lane == 0 && cnt[rl] + headroom > SEG) ct.flag[r] = 1;

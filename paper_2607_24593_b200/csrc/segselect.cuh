@@ -66,9 +66,9 @@ struct Seg {
 };
 
 // A lane's entries: entry j of the lane is segment element j * 32 + lane.
-template <bool CACHED>
+template <bool CACHED, int EPT = kSelEpt>
 struct SegRegs {
-  entry_t v[CACHED ? kSelEpt : 1];
+  entry_t v[CACHED ? EPT : 1];
   const entry_t* base;
   int nj;      // this lane's entry count
   __device__ __forceinline__ void load(const Seg& s, int lane) {
@@ -76,14 +76,14 @@ struct SegRegs {
     nj = s.cnt > lane ? (s.cnt - lane + 31) >> 5 : 0;
     if constexpr (CACHED) {
 #pragma unroll
-      for (int j = 0; j < kSelEpt; ++j) v[j] = j < nj ? __ldcg(base + j * 32) : kPadEntry;
+      for (int j = 0; j < EPT; ++j) v[j] = j < nj ? __ldcg(base + j * 32) : kPadEntry;
     }
   }
   template <typename F>
   __device__ __forceinline__ void for_each(F f) const {
     if constexpr (CACHED) {
 #pragma unroll
-      for (int j = 0; j < kSelEpt; ++j)
+      for (int j = 0; j < EPT; ++j)
         if (j < nj) f(v[j]);
     } else {
 #pragma unroll 4
@@ -95,7 +95,7 @@ struct SegRegs {
   __device__ __forceinline__ void for_each_uniform(int njw, F f) const {
     if constexpr (CACHED) {
 #pragma unroll
-      for (int j = 0; j < kSelEpt; ++j)
+      for (int j = 0; j < EPT; ++j)
         if (j < njw) f(j < nj ? v[j] : kPadEntry, j < nj);
     } else {
       for (int j = 0; j < njw; ++j) f(j < nj ? __ldcg(base + j * 32) : kPadEntry, j < nj);
@@ -145,8 +145,8 @@ __device__ __forceinline__ void hist_boundary(const Team& tm, SegSelSmem& sm, co
 
 // Finds the K-th largest entry among the team's segments (more than K real entries in total).
 // All 128 threads call; the cut is returned (and left in sm.cut).
-template <bool CACHED>
-__device__ __forceinline__ entry_t seg_find_cut(const Team& tm, SegSelSmem& sm, const SegRegs<CACHED>& regs, int K) {
+template <bool CACHED, int EPT = kSelEpt>
+__device__ __forceinline__ entry_t seg_find_cut(const Team& tm, SegSelSmem& sm, const SegRegs<CACHED, EPT>& regs, int K) {
   const int lane = tm.tid & 31;
   SELP_T(q0);
   entry_t mn = ~0ull, mx = 0ull;
@@ -254,12 +254,12 @@ __device__ __forceinline__ int seg_filter_inplace(entry_t* e, int cnt, int lane,
 
 // Exact compaction in place: keeps the K best entries of the team's segments; returns this
 // warp's new count and the cut through *cut_out.  Needs more than K real entries in total.
-template <bool CACHED>
+template <bool CACHED, int EPT = kSelEpt>
 __device__ __forceinline__ int seg_compact(const Team& tm, SegSelSmem& sm, const Seg& seg, int K, entry_t* cut_out) {
   const int lane = tm.tid & 31;
-  SegRegs<CACHED> regs;
+  SegRegs<CACHED, EPT> regs;
   regs.load(seg, lane);
-  const entry_t cut = seg_find_cut<CACHED>(tm, sm, regs, K);
+  const entry_t cut = seg_find_cut<CACHED, EPT>(tm, sm, regs, K);
   *cut_out = cut;
   if constexpr (CACHED) {
     int out = 0;
@@ -277,16 +277,16 @@ __device__ __forceinline__ int seg_compact(const Team& tm, SegSelSmem& sm, const
 
 // Final selection of a row: writes min(K, n_valid) positions (unordered) to out, returns how
 // many.  n_valid = real (non-padding) entries in the team's segments.
-template <bool CACHED>
+template <bool CACHED, int EPT = kSelEpt>
 __device__ __forceinline__ int seg_emit(const Team& tm, SegSelSmem& sm, const Seg& seg, int n_valid, int32_t* out,
                                         float* out_score, int K) {
   const int lane = tm.tid & 31;
-  SegRegs<CACHED> regs;
+  SegRegs<CACHED, EPT> regs;
   regs.load(seg, lane);
   if (tm.tid == 0) sm.out_count = 0;
   tm.sync();
   entry_t cut = 0ull;
-  if (n_valid > K) cut = seg_find_cut<CACHED>(tm, sm, regs, K);
+  if (n_valid > K) cut = seg_find_cut<CACHED, EPT>(tm, sm, regs, K);
   regs.for_each_uniform((seg.cnt + 31) >> 5, [&](entry_t x, bool valid) {
     const bool keep = valid && entry_pos(x) >= 0 && x >= cut;
     const uint32_t m = __ballot_sync(0xffffffffu, keep);
