@@ -122,6 +122,52 @@ class ClockSampler:
                     reasons=reasons, samples=len(sm))
 
 
+def decode_bench(pv, dev, steps, warmup, pk):
+    """Batched MTP decode step (32 sequences, prefix lengths uniform in [64K, 128K], FP8 cache,
+    g = 2, Refine, c = 4096, k = 2048): microseconds per step, device-timed, plus the HBM
+    roofline of the step (every visible key and its scale are read once per step)."""
+    B, g, c, k = 32, 2, 4096, 2048
+    x = inputs.make_decode(B, g, 65536, 131072, dtype="fp8")
+    Lmax = x.k.shape[1]
+    q, w, kc, p0 = x.q.to(dev), x.w.to(dev), x.k.to(dev), x.pos0.to(dev)
+    qs, ks = x.qscale.to(dev), x.kscale.to(dev)
+    out = torch.empty((B, g, k), dtype=torch.int32, device=dev)
+    pv.ensure_workspace(B * g, B, c, k, dev, need=pv.pivot_decode_workspace_bytes(B, Lmax, g, c, k))
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)     # > L2: evict the key cache between steps
+
+    def step():
+        pv.pivot_index_decode(q, w, kc, p0, B, Lmax, H, D, g, c, k, pv.REFINE, out, stream, q_scale=qs, k_scale=ks)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    times = []
+    pv.pivot_launch_count_reset()
+    for _ in range(steps):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) * 1e3)
+    launches = pv.pivot_launch_count_reset()
+    assert pv.pivot_device_status() == 0
+    us = float(np.median(times))
+    n0 = (x.pos0.numpy().astype(np.int64) + 1)
+    key_bytes = int(n0.sum()) * (D + 4)                      # e4m3 key + fp32 scale, read once per step
+    gather_bytes = B * c * (D + 4)
+    alg = key_bytes + gather_bytes + B * g * H * (D + 8) + B * g * k * 4
+    return {"metric": "us per MTP decode step", "value": us, "unit": "us", "min_us": float(min(times)),
+            "steps": steps, "higher_is_better": False, "gpu_launches_per_step": launches / max(steps, 1),
+            "config": {"workload": "decode_mtp_b32_64k-128k_fp8_g2_refine", "B": B, "g": g, "c": c, "k": k,
+                       "visible_keys": int(n0.sum()), "l2": "256 MB flush between steps"},
+            "roofline": {"bound": "hbm", "achieved": alg / (us * 1e-6) / 1e9, "peak": pk["hbm"], "unit": "GB/s",
+                         "frac": alg / (us * 1e-6) / 1e9 / pk["hbm"], "traffic": None,
+                         "algorithmic_bytes_per_step": alg, "peak_source": pk["source"] + " STREAM copy"}}
+
+
 def oracle_sample_time(x, L, g, c, k, mode, n_groups, seed):
     """Times the CPU oracle (as it stands) on a uniform random sample of groups; returns
     (estimated seconds for the whole request, seconds spent, groups timed, threads used)."""
@@ -180,6 +226,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-decode", action="store_true")
     args = ap.parse_args()
     wl = args.workload
     if args.impl == "reference":
@@ -305,6 +352,13 @@ def main():
     }
     if e2e is not None:
         line["e2e"] = e2e
+    if not args.no_decode:
+        try:
+            del arena
+        except NameError:
+            pass
+        torch.cuda.empty_cache()
+        line["decode"] = decode_bench(pv, dev, steps=max(args.steps, 5), warmup=max(args.warmup, 3), pk=pk)
 
     # ---- parity probe on the e2e result (a few groups) and the CPU baseline
     if not args.no_cpu_baseline:

@@ -95,9 +95,13 @@ typedef struct pivot_opts {
   int impl;
 } pivot_opts;
 
-/* Bytes of scratch a call with these sizes needs.  rows = L for prefill / dense, B*g for decode;
- * n_groups = ceil(L/g) or B.  Depends on the device's SM count (queried once). */
+/* Bytes of scratch a prefill / dense call with these sizes needs: rows = L, n_groups = ceil(L/g)
+ * (L for dense_index).  Depends on the device's SM count (queried once).  Decode calls need
+ * pivot_decode_workspace_bytes. */
 size_t pivot_workspace_bytes(int rows, int n_groups, int c, int k);
+
+/* Scratch of a decode call (adds the per-key score array and histograms of the decode path). */
+size_t pivot_decode_workspace_bytes(int B, int Lmax, int g, int c, int k);
 
 /* Registers the scratch buffer used by the short entry points below on the current device.
  * The buffer stays owned by the caller and must outlive those calls.  Calls that share one

@@ -21,7 +21,7 @@ POOL_MEAN, POOL_FIRST, POOL_LAST = 0, 1, 2
 OK = 0
 
 SYMBOLS = [
-    "pivot_workspace_bytes", "pivot_set_workspace", "pivot_index_prefill", "pivot_index_prefill_ex",
+    "pivot_workspace_bytes", "pivot_decode_workspace_bytes", "pivot_set_workspace", "pivot_index_prefill", "pivot_index_prefill_ex",
     "pivot_index_decode", "pivot_index_decode_ex", "dense_index", "dense_index_ex", "dense_index_static",
     "pivot_prefill_host_arena_bytes", "pivot_index_prefill_host", "pivot_device_status",
     "pivot_stage_timing", "pivot_stage_times", "pivot_launch_count_reset", "pivot_status_str", "pivot_last_cuda_error",
@@ -51,6 +51,8 @@ def _load():
     T, O, I, P, S = C.POINTER(pivot_tensor), C.POINTER(pivot_opts), C.c_int, C.c_void_p, C.c_size_t
     lib.pivot_workspace_bytes.restype = S
     lib.pivot_workspace_bytes.argtypes = [I, I, I, I]
+    lib.pivot_decode_workspace_bytes.restype = S
+    lib.pivot_decode_workspace_bytes.argtypes = [I, I, I, I, I]
     lib.pivot_set_workspace.argtypes = [P, S]
     lib.pivot_index_prefill.argtypes = [T, P, T, I, I, I, I, I, I, I, P, P]
     lib.pivot_index_prefill_ex.argtypes = [T, P, T, I, I, I, I, I, I, I, P, P, O]
@@ -124,9 +126,13 @@ def pivot_set_workspace(workspace: torch.Tensor | None):
     _workspaces[workspace.device.index] = workspace
 
 
-def ensure_workspace(rows: int, n_groups: int, c: int, k: int, device="cuda") -> torch.Tensor:
+def pivot_decode_workspace_bytes(B: int, Lmax: int, g: int, c: int, k: int) -> int:
+    return int(lib.pivot_decode_workspace_bytes(B, Lmax, g, c, k))
+
+
+def ensure_workspace(rows: int, n_groups: int, c: int, k: int, device="cuda", need: int | None = None) -> torch.Tensor:
     """Allocates (or reuses) a registered workspace large enough for these sizes."""
-    need = pivot_workspace_bytes(rows, n_groups, c, k)
+    need = pivot_workspace_bytes(rows, n_groups, c, k) if need is None else need
     dev = torch.device(device)
     idx = dev.index if dev.index is not None else torch.cuda.current_device()
     cur = _workspaces.get(idx)
@@ -180,7 +186,7 @@ def pivot_index_decode(q, w, kcache, pos0, B, Lmax, H_I, d, g, c, k, mode, out_i
     assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and pos0.dtype == torch.int32
     assert out_idx.numel() >= B * g * k
     if workspace is None:
-        ensure_workspace(B * g, B, c, k, q.device)
+        ensure_workspace(B * g, B, c, k, q.device, need=pivot_decode_workspace_bytes(B, Lmax, g, c, k))
     o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl)
     _check(lib.pivot_index_decode_ex(C.byref(tq), w.data_ptr(), C.byref(tk), pos0.data_ptr(), B, Lmax,
                                      H_I, d, g, c, k, mode, out_idx.data_ptr(), _stream(stream), C.byref(o)))

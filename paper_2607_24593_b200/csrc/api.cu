@@ -217,6 +217,11 @@ size_t pivot_workspace_bytes(int rows, int n_groups, int c, int k) {
   return carve_workspace(nullptr, rows, n_groups, c, k).bytes;
 }
 
+size_t pivot_decode_workspace_bytes(int B, int Lmax, int g, int c, int k) {
+  if (B < 1 || Lmax < 1 || g < 1 || c < 1 || k < 1) return 0;
+  return pivot_workspace_bytes(B * g, B, c, k) + decode_fast_bytes(B, Lmax, g, c);
+}
+
 int pivot_set_workspace(void* workspace, size_t bytes) {
   if (workspace && ((uintptr_t)workspace & 255)) return PIVOT_ERR_INVALID_ARG;
   DeviceState& ds = g_dev[cur_device()];
@@ -265,7 +270,8 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
   if (q->dtype == PIVOT_FP8_E4M3 && (Lmax & 3)) return PIVOT_ERR_INVALID_ARG;
   if (o && (o->pool < 0 || o->pool > 2)) return PIVOT_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
-  const size_t need = pivot_workspace_bytes(B * g, B, c, k);
+  const size_t base_bytes = pivot_workspace_bytes(B * g, B, c, k);
+  const size_t need = base_bytes + decode_fast_bytes(B, Lmax, g, c);
   void* wsp = nullptr;
   if ((rc = resolve_ws(o, need, &wsp))) return rc;
   Workspace ws = carve_workspace(wsp, B * g, B, c, k);
@@ -290,15 +296,23 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
   if (o && o->impl == 1) {
     launch_scan_simt(ws.rows, B + B * g, q->dtype, ws.scan, st);
   } else {
+    // proxy rows: key-tile-split scan, per-sequence select, chunked re-score, final top-k
+    DecodeFast df;
+    df.prox = ws.rows; df.groups = ws.groups;
+    df.kc = kcache->data; df.kscale = kcache->scale; df.q = q->data; df.proxy_q = ws.proxy_q;
+    df.B = B; df.Lmax = Lmax; df.g = g; df.c = c; df.k = k; df.mode = mode; df.dtype = q->dtype;
+    df.sms = sm_count();
+    df.scratch = (char*)wsp + base_bytes;
+    df.scratch_tc = tc_scratch(ws);
+    df.status = ws.status;
+    if ((rc = check_cuda(launch_decode_fast(df, st)))) return rc;
+    // dense rows of guarded (short) sequences, if any: the generic scan, one row per block
     ScanOperands op{kcache->data, (long long)B * Lmax, kcache->scale, q->data, B * g, ws.proxy_q, B, q->dtype};
-    if ((rc = check_cuda(launch_scan_tc(op, ws.rows, B + B * g, 1, tc_scratch(ws), sm_count(), st)))) return rc;
+    if ((rc = check_cuda(launch_scan_tc(op, ws.rows + B, B * g, 1, tc_scratch(ws), sm_count(), st)))) return rc;
   }
   mark(3, st);
-  if (mode == PIVOT_REFINE) {
-    const int nd = B * group_chunks(g);
-    if (o && o->impl == 1) launch_refine_simt(ws.groups, nd, q->dtype, ws.scan, st);
-    else if ((rc = check_cuda(launch_refine_tc(q->data, B * g, q->dtype, ws.groups, nd, tc_scratch(ws), sm_count(), st))))
-      return rc;
+  if (mode == PIVOT_REFINE && o && o->impl == 1) {
+    launch_refine_simt(ws.groups, B * group_chunks(g), q->dtype, ws.scan, st);
   }
   mark(4, st);
   return check_cuda(cudaGetLastError());

@@ -1,0 +1,466 @@
+// Decode path (Algorithm 1 with the grouping of Eq. 3), built for HBM bandwidth.
+//
+// One MTP step scores one proxy per sequence against that sequence's whole key cache, so the
+// step is a single pass over every visible key (128 B + 4 B scale): memory bound.  The work is
+// therefore split by KEY TILES, not by rows:
+//   decode_scan_kernel   every SM takes an equal, contiguous share of all (sequence, 128-key
+//                        tile) pairs; per tile: TMA -> tcgen05 MMA (128 keys x 64 heads x d) ->
+//                        epilogue (ReLU, gate-weighted head sum, key scale) -> one fp32 score per
+//                        key to an L2-resident score array (3 % of the bytes read), plus a
+//                        16384-bin histogram of the scores' top 14 key bits per sequence.
+//   decode_select_kernel one 1024-thread CTA per sequence: the histogram gives the bin holding
+//                        the K-th best score; if that leaves too many candidates the bin is
+//                        refined 12 bits at a time with further passes over the scores; the
+//                        survivors are collected in shared memory and the exact top-K (Eq. 6 / 7)
+//                        is taken there.
+//   entries_topk_kernel  exact top-k (Eq. 9) of each query's re-scored candidates, which the
+//                        gather + re-score kernel leaves as packed entries (refine_tc.cu, chunked
+//                        over candidates so that all SMs take part).
+#include <cuda.h>
+#include <string.h>
+
+#include "blockselect.cuh"
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace pivot {
+namespace {
+
+constexpr int TILE_KEYS = 128;
+constexpr int DKS_SLOTS = 14;
+constexpr int DHIST = 16384;            // top 14 bits of the score key
+constexpr int D_N = kHeads;             // MMA N: one proxy
+constexpr int D_THREADS = 64 + 128;     // TMA warp, MMA warp, four epilogue warps
+constexpr int SEL_CAP = 12288;          // candidates collected in shared memory per sequence
+
+template <int DT>
+struct DCfg {
+  static constexpr bool FP8 = DT == DT_FP8;
+  static constexpr int KHALVES = FP8 ? 1 : 2;
+  static constexpr int HALF_TILE_BYTES = TILE_KEYS * 128;
+  static constexpr int STAGE_BYTES = KHALVES * HALF_TILE_BYTES;
+  static constexpr int QHALF_BYTES = kHeads * 128;
+  static constexpr int QBUF_BYTES = KHALVES * QHALF_BYTES;
+  static constexpr int STAGES = FP8 ? 8 : 3;
+  static constexpr uint32_t IDESC = ptx::make_idesc(FP8 ? 0u : 1u, TILE_KEYS, D_N);
+};
+
+struct DCtrl {
+  alignas(128) float ks[DKS_SLOTS][TILE_KEYS];
+  alignas(16) float w[2][kHeads];
+  uint32_t hist[DHIST];
+  uint64_t full[8], empty[8], q_full[2], q_empty[2], tmem_full[2], tmem_empty[2], ks_full[DKS_SLOTS];
+  uint32_t tmem_base;
+  int abort;
+};
+
+template <int DT>
+constexpr size_t dsmem_bytes() {
+  return 1024 + 2 * DCfg<DT>::QBUF_BYTES + DCfg<DT>::STAGES * DCfg<DT>::STAGE_BYTES + sizeof(DCtrl);
+}
+
+// Walks the global tile index space: sequence b owns tiles [prefix[b], prefix[b+1]).
+struct TileWalk {
+  const int* prefix;
+  int B, b;
+  __device__ TileWalk(const int* p, int nb) : prefix(p), B(nb), b(0) {}
+  __device__ __forceinline__ int seq_of(int g) {     // g non-decreasing between calls
+    while (b + 1 < B && g >= prefix[b + 1]) ++b;
+    return b;
+  }
+};
+
+template <int DT>
+__global__ void __launch_bounds__(D_THREADS, 1)
+decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
+                   const __grid_constant__ CUtensorMap tm_ks, const RowDesc* __restrict__ prox,
+                   const int* __restrict__ tile_prefix, int B, int Lmax, float* __restrict__ scores,
+                   uint32_t* __restrict__ ghist, int* status) {
+  using C = DCfg<DT>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* qbuf = smem;
+  uint8_t* kring = smem + 2 * C::QBUF_BYTES;
+  DCtrl& ct = *reinterpret_cast<DCtrl*>(kring + C::STAGES * C::STAGE_BYTES);
+  volatile int* abort_flag = &ct.abort;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::STAGES; ++s) { ptx::mbar_init(&ct.full[s], 1); ptx::mbar_init(&ct.empty[s], 1); }
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(&ct.q_full[i], 1);
+      ptx::mbar_init(&ct.q_empty[i], 1);
+      ptx::mbar_init(&ct.tmem_full[i], 1);
+      ptx::mbar_init(&ct.tmem_empty[i], 4);
+    }
+    for (int i = 0; i < DKS_SLOTS; ++i) ptx::mbar_init(&ct.ks_full[i], 1);
+    ct.abort = 0;
+    ptx::fence_barrier_init();
+  }
+  for (int i = threadIdx.x; i < DHIST; i += D_THREADS) ct.hist[i] = 0;
+  if (warp == 1) { ptx::tmem_alloc(&ct.tmem_base, 2 * D_N); ptx::tmem_relinquish(); }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = ct.tmem_base;
+
+  const int total = tile_prefix[B];
+  const int g_lo = (int)((long long)blockIdx.x * total / gridDim.x);
+  const int g_hi = (int)((long long)(blockIdx.x + 1) * total / gridDim.x);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (ptx::elect_one()) {
+      ptx::prefetch_tensormap(&tm_k);
+      ptx::prefetch_tensormap(&tm_q);
+      if (C::FP8) ptx::prefetch_tensormap(&tm_ks);
+      TileWalk tw(tile_prefix, B);
+      int cur_b = -1;
+      uint32_t it = 0, blk = 0;
+      for (int g = g_lo; g < g_hi; ++g, ++it) {
+        const int b = tw.seq_of(g);
+        const int t = g - tile_prefix[b];
+        if (b != cur_b) {             // new sequence: its proxy becomes the MMA's B operand
+          const int qb = blk & 1;
+          if (!ptx::mbar_wait(&ct.q_empty[qb], ((blk >> 1) & 1) ^ 1, abort_flag, 64)) break;
+          ptx::mbar_arrive_expect_tx(&ct.q_full[qb], C::QBUF_BYTES);
+          for (int h = 0; h < C::KHALVES; ++h)
+            ptx::tma_load_2d(qbuf + qb * C::QBUF_BYTES + h * C::QHALF_BYTES, &tm_q, h * 64, prox[b].q_row * kHeads,
+                             &ct.q_full[qb]);
+          ++blk;
+          cur_b = b;
+        }
+        const int s = it % C::STAGES;
+        if (!ptx::mbar_wait(&ct.empty[s], ((it / C::STAGES) & 1) ^ 1, abort_flag, 64)) break;
+        ptx::mbar_arrive_expect_tx(&ct.full[s], C::STAGE_BYTES);
+        for (int h = 0; h < C::KHALVES; ++h)
+          ptx::tma_load_2d(kring + s * C::STAGE_BYTES + h * C::HALF_TILE_BYTES, &tm_k, h * 64,
+                           prox[b].k_row0 + t * TILE_KEYS, &ct.full[s]);
+        if (C::FP8) {
+          const int ksl = it % DKS_SLOTS;       // free by construction (see the prefill scan)
+          ptx::mbar_arrive_expect_tx(&ct.ks_full[ksl], TILE_KEYS * 4);
+          ptx::tma_load_1d(&ct.ks[ksl][0], &tm_ks, prox[b].k_row0 + t * TILE_KEYS, &ct.ks_full[ksl]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (ptx::elect_one()) {
+      TileWalk tw(tile_prefix, B);
+      int cur_b = -1, qb = 0;
+      uint32_t it = 0, blk = 0;
+      bool ok = true;
+      for (int g = g_lo; g < g_hi && ok; ++g, ++it) {
+        const int b = tw.seq_of(g);
+        if (b != cur_b) {
+          if (cur_b >= 0) ptx::tc_commit(&ct.q_empty[qb]);     // previous proxy no longer needed
+          qb = blk & 1;
+          ok = ptx::mbar_wait(&ct.q_full[qb], (blk >> 1) & 1, abort_flag, 32);
+          if (!ok) break;
+          ++blk;
+          cur_b = b;
+        }
+        const int s = it % C::STAGES;
+        const int buf = it & 1;
+        ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, 32);
+        if (!ok) break;
+        ok = ptx::mbar_wait(&ct.full[s], (it / C::STAGES) & 1, abort_flag, 32);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t k_addr = ptx::smem_u32(kring + s * C::STAGE_BYTES);
+        const uint32_t q_addr = ptx::smem_u32(qbuf + qb * C::QBUF_BYTES);
+        const uint32_t d_tmem = tmem_base + buf * D_N;
+#pragma unroll
+        for (int h = 0; h < C::KHALVES; ++h)
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            ptx::tc_mma<C::FP8>(d_tmem, ptx::smem_desc_sw128(k_addr + h * C::HALF_TILE_BYTES + ks * 32),
+                                ptx::smem_desc_sw128(q_addr + h * C::QHALF_BYTES + ks * 32), C::IDESC,
+                                (h | ks) ? 1u : 0u);
+        ptx::tc_commit(&ct.empty[s]);
+        ptx::tc_commit(&ct.tmem_full[buf]);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int tt = threadIdx.x - 64;                 // 0..127 = key inside the tile
+    const int lq = warp & 3;
+    const int key_in_tile = lq * 32 + lane;
+    const Team tm{tt, 128, 1};
+    TileWalk tw(tile_prefix, B);
+    int cur_b = -1, wb = 0, n_vis = 0;
+    uint32_t it = 0, blk = 0;
+    auto flush_hist = [&](int b) {
+      tm.sync();
+      for (int i = tt; i < DHIST; i += 128) {
+        const uint32_t h = ct.hist[i];
+        if (h) { atomicAdd(&ghist[(size_t)b * DHIST + i], h); ct.hist[i] = 0; }
+      }
+      tm.sync();
+    };
+    for (int g = g_lo; g < g_hi; ++g, ++it) {
+      const int b = tw.seq_of(g);
+      const int t = g - tile_prefix[b];
+      if (b != cur_b) {
+        if (cur_b >= 0) flush_hist(cur_b);
+        wb = blk & 1;
+        ++blk;
+        cur_b = b;
+        n_vis = prox[b].n_vis;
+        tm.sync();
+        if (tt < kHeads) ct.w[wb][tt] = 0.5f * prox[b].w[tt];      // proxy gate, halved (ReLU identity)
+        tm.sync();
+      }
+      const int buf = it & 1;
+      float ksv = 1.f;
+      if (C::FP8) {
+        const int ksl = it % DKS_SLOTS;
+        (void)ptx::mbar_wait(&ct.ks_full[ksl], (it / DKS_SLOTS) & 1, abort_flag);
+        ksv = ct.ks[ksl][key_in_tile];
+      }
+      (void)ptx::mbar_wait(&ct.tmem_full[buf], (it >> 1) & 1, abort_flag);
+      ptx::tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(lq * 32) << 16) + buf * D_N;
+      uint32_t v0[32], v1[32];
+      ptx::tmem_ld_32x32(taddr, v0);
+      ptx::tmem_ld_32x32(taddr + 32, v1);
+      ptx::tmem_wait_ld();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
+      float ap[4] = {0.f, 0.f, 0.f, 0.f}, an[4] = {0.f, 0.f, 0.f, 0.f};
+      const float4* wp = reinterpret_cast<const float4*>(&ct.w[wb][0]);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float4 wa = wp[j], wbv = wp[8 + j];
+        const float x0 = __uint_as_float(v0[4 * j]), x1 = __uint_as_float(v0[4 * j + 1]);
+        const float x2 = __uint_as_float(v0[4 * j + 2]), x3 = __uint_as_float(v0[4 * j + 3]);
+        const float y0 = __uint_as_float(v1[4 * j]), y1 = __uint_as_float(v1[4 * j + 1]);
+        const float y2 = __uint_as_float(v1[4 * j + 2]), y3 = __uint_as_float(v1[4 * j + 3]);
+        ap[0] = fmaf(fabsf(x0), wa.x, ap[0]); an[0] = fmaf(x0, wa.x, an[0]);
+        ap[1] = fmaf(fabsf(x1), wa.y, ap[1]); an[1] = fmaf(x1, wa.y, an[1]);
+        ap[2] = fmaf(fabsf(x2), wa.z, ap[2]); an[2] = fmaf(x2, wa.z, an[2]);
+        ap[3] = fmaf(fabsf(x3), wa.w, ap[3]); an[3] = fmaf(x3, wa.w, an[3]);
+        ap[0] = fmaf(fabsf(y0), wbv.x, ap[0]); an[0] = fmaf(y0, wbv.x, an[0]);
+        ap[1] = fmaf(fabsf(y1), wbv.y, ap[1]); an[1] = fmaf(y1, wbv.y, an[1]);
+        ap[2] = fmaf(fabsf(y2), wbv.z, ap[2]); an[2] = fmaf(y2, wbv.z, an[2]);
+        ap[3] = fmaf(fabsf(y3), wbv.w, ap[3]); an[3] = fmaf(y3, wbv.w, an[3]);
+      }
+      float sv = ((ap[0] + an[0]) + (ap[1] + an[1])) + ((ap[2] + an[2]) + (ap[3] + an[3]));
+      if (C::FP8) sv *= ksv;
+      const int s_key = t * TILE_KEYS + key_in_tile;
+      if (s_key < n_vis) {
+        scores[(size_t)b * Lmax + s_key] = sv;
+        atomicAdd(&ct.hist[score_to_key(sv) >> 18], 1u);
+      }
+    }
+    if (cur_b >= 0) flush_hist(cur_b);
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  if (warp == 1) ptx::tmem_dealloc(tmem_base, 2 * D_N);
+  if (threadIdx.x == 0 && ct.abort) set_status(status, DEV_WAIT_EXPIRED);
+}
+
+// ------------------------------------------------------------------------------ per-sequence select
+
+struct SelSmem {
+  BlkSelSmem blk;
+  entry_t list[SEL_CAP];
+};
+
+__global__ void __launch_bounds__(kBlk, 1)
+decode_select_kernel(const RowDesc* __restrict__ prox, int Lmax, const float* __restrict__ scores,
+                     const uint32_t* __restrict__ ghist) {
+  extern __shared__ uint8_t sel_raw[];
+  SelSmem& sm = *reinterpret_cast<SelSmem*>(((uintptr_t)sel_raw + 15) & ~(uintptr_t)15);
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
+  const RowDesc rd = prox[b];
+  const int K = rd.K, n0 = rd.n_vis;
+  if (K <= 0) return;
+  const float* sc = scores + (size_t)b * Lmax;
+  auto entry_at = [&](int i) { return make_entry(score_to_key(__ldcg(sc + i)), i); };
+  // ---- narrow the candidates: entries whose top `pbits` bits are >= prefix
+  unsigned long long prefix = 0;
+  int pbits = 0;
+  if (n0 > SEL_CAP) {
+    blk_boundary(sm.blk, ghist + (size_t)b * DHIST, DHIST, (uint32_t)K);
+    uint32_t need = sm.blk.need, pop = sm.blk.pop;
+    prefix = sm.blk.bin;
+    pbits = 14;
+    while ((uint32_t)K - need + pop > (uint32_t)SEL_CAP && pbits < 64) {
+      const int wbits = 64 - pbits < 12 ? 64 - pbits : 12;
+      __syncthreads();
+      for (int i = tid; i < 4096; i += kBlk) sm.blk.hist[i] = 0;
+      __syncthreads();
+      for (int i = tid; i < n0; i += kBlk) {
+        const entry_t e = entry_at(i);
+        if ((e >> (64 - pbits)) == prefix) atomicAdd(&sm.blk.hist[(uint32_t)((e >> (64 - pbits - wbits)) & ((1u << wbits) - 1u))], 1u);
+      }
+      blk_boundary(sm.blk, sm.blk.hist, 4096, need);
+      need = sm.blk.need;
+      pop = sm.blk.pop;
+      prefix = (prefix << wbits) | sm.blk.bin;
+      pbits += wbits;
+    }
+  }
+  // ---- collect them in shared memory
+  if (tid == 0) sm.blk.list_n = 0;
+  __syncthreads();
+  for (int i0 = 0; i0 < n0; i0 += kBlk) {
+    const int i = i0 + tid;
+    entry_t e = 0;
+    bool keep = false;
+    if (i < n0) {
+      e = entry_at(i);
+      keep = pbits == 0 || (e >> (64 - pbits)) >= prefix;
+    }
+    const uint32_t m = __ballot_sync(0xffffffffu, keep);
+    if (m) {
+      uint32_t pos = 0;
+      const int leader = __ffs(m) - 1;
+      if (lane == leader) pos = atomicAdd(&sm.blk.list_n, (uint32_t)__popc(m));
+      pos = __shfl_sync(0xffffffffu, pos, leader);
+      if (keep) {
+        const uint32_t p = pos + __popc(m & ((1u << lane) - 1u));
+        if (p < (uint32_t)SEL_CAP) sm.list[p] = e;
+      }
+    }
+  }
+  __syncthreads();
+  const int n = min((int)sm.blk.list_n, SEL_CAP);
+  blk_emit_topk(sm.blk, sm.list, n, n, K, rd.out, rd.out_score, rd.out_rows, rd.out_stride);
+}
+
+// ------------------------------------------------------------------------------ top-k of entry lists
+
+__global__ void __launch_bounds__(kBlk, 1) entries_topk_kernel(const EntryList* __restrict__ lists) {
+  __shared__ BlkSelSmem sm;
+  const EntryList el = lists[blockIdx.x];
+  if (el.K <= 0) return;
+  blk_emit_topk(sm, (const entry_t*)el.list, el.n, el.n, el.K, el.out, el.out_score, 1, el.K);
+}
+
+// ------------------------------------------------------------------------------ setup
+
+__global__ void decode_setup_kernel(const RowDesc* __restrict__ prox, const GroupDesc* __restrict__ groups, int B,
+                                    int g, int c, int k, int mode, int* tile_prefix, GroupDesc* chunks,
+                                    EntryList* lists, unsigned long long* entries) {
+  __shared__ int tiles[1024];
+  const int tid = threadIdx.x;
+  for (int b = tid; b < B; b += blockDim.x)
+    tiles[b] = prox[b].K > 0 ? (prox[b].n_vis + TILE_KEYS - 1) / TILE_KEYS : 0;
+  __syncthreads();
+  if (tid == 0) {
+    int acc = 0;
+    for (int b = 0; b < B; ++b) { tile_prefix[b] = acc; acc += tiles[b]; }
+    tile_prefix[B] = acc;
+  }
+  if (mode != 1) return;
+  // Refine: split every (sequence, member chunk) into candidate chunks so all SMs re-score,
+  // each leaving packed entries; one entry list per query for the final top-k.
+  const int mc = (g + kMembersPerDesc - 1) / kMembersPerDesc;
+  const int ncc = (c + kDecodeCandChunk - 1) / kDecodeCandChunk;
+  for (int i = tid; i < B * mc * ncc; i += blockDim.x) {
+    const int gi = i / ncc, cc = i % ncc;
+    GroupDesc gd = groups[gi];
+    const int left = gd.n_cand - cc * kDecodeCandChunk;
+    gd.cand = gd.cand + cc * kDecodeCandChunk;
+    gd.n_cand = left > 0 ? (left < kDecodeCandChunk ? left : kDecodeCandChunk) : 0;
+    gd.ent_out = entries + (size_t)gd.q_row * c;
+    gd.ent_stride = c;
+    gd.slot0 = cc * kDecodeCandChunk;
+    chunks[i] = gd;
+  }
+  for (int i = tid; i < B * g; i += blockDim.x) {
+    const int b = i / g;
+    const GroupDesc gd = groups[b * mc];
+    EntryList el;
+    el.list = entries + (size_t)i * c;
+    el.n = gd.n_cand;
+    el.K = gd.n_cand > 0 ? k : 0;
+    el.out = groups[b * mc].out + (size_t)(i - b * g) * gd.out_stride;
+    el.out_score = gd.out_score ? groups[b * mc].out_score + (size_t)(i - b * g) * gd.out_stride : nullptr;
+    lists[i] = el;
+  }
+}
+
+template <int DT>
+cudaError_t launch_scan(const CUtensorMap& mk, const CUtensorMap& mq, const CUtensorMap& mks, const RowDesc* prox,
+                        const int* tile_prefix, int B, int Lmax, float* scores, uint32_t* ghist, int* status,
+                        int sms, cudaStream_t st) {
+  auto kern = decode_scan_kernel<DT>;
+  static bool attr_set = false;
+  const size_t smem = dsmem_bytes<DT>();
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  kern<<<sms, D_THREADS, smem, st>>>(mk, mq, mks, prox, tile_prefix, B, Lmax, scores, ghist, status);
+  ++launch_counter();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows);
+bool make_scale_map(CUtensorMap* m, const float* base, long long n);
+
+size_t decode_fast_bytes(int B, int Lmax, int g, int c) {
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  const int mc = group_chunks(g);
+  const int ncc = (c + kDecodeCandChunk - 1) / kDecodeCandChunk;
+  return up((size_t)B * Lmax * 4) + up((size_t)B * DHIST * 4) + up((size_t)(B + 1) * 4) +
+         up((size_t)B * mc * ncc * sizeof(GroupDesc)) + up((size_t)B * g * sizeof(EntryList)) +
+         up((size_t)B * g * c * 8);
+}
+
+cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  char* p = (char*)d.scratch;
+  float* scores = (float*)p;                 p += up((size_t)d.B * d.Lmax * 4);
+  uint32_t* ghist = (uint32_t*)p;            p += up((size_t)d.B * DHIST * 4);
+  int* tile_prefix = (int*)p;                p += up((size_t)(d.B + 1) * 4);
+  const int mc = group_chunks(d.g);
+  const int ncc = (d.c + kDecodeCandChunk - 1) / kDecodeCandChunk;
+  GroupDesc* chunks = (GroupDesc*)p;         p += up((size_t)d.B * mc * ncc * sizeof(GroupDesc));
+  EntryList* lists = (EntryList*)p;          p += up((size_t)d.B * d.g * sizeof(EntryList));
+  unsigned long long* entries = (unsigned long long*)p;
+
+  cudaError_t e = cudaMemsetAsync(ghist, 0, (size_t)d.B * DHIST * 4, st);
+  if (e != cudaSuccess) return e;
+  decode_setup_kernel<<<1, 1024, 0, st>>>(d.prox, d.groups, d.B, d.g, d.c, d.k, d.mode, tile_prefix, chunks, lists,
+                                          entries);
+  ++launch_counter();
+  CUtensorMap mk, mq, mks;
+  memset(&mks, 0, sizeof(mks));
+  if (d.dtype == DT_FP8 && !make_scale_map(&mks, d.kscale, (long long)d.B * d.Lmax)) return cudaErrorInvalidValue;
+  if (!make_operand_map(&mk, d.kc, (long long)d.B * d.Lmax, d.dtype, TILE_KEYS) ||
+      !make_operand_map(&mq, d.proxy_q, (long long)d.B * kHeads, d.dtype, kHeads))
+    return cudaErrorInvalidValue;
+  e = d.dtype == DT_FP8
+          ? launch_scan<DT_FP8>(mk, mq, mks, d.prox, tile_prefix, d.B, d.Lmax, scores, ghist, d.status, d.sms, st)
+          : launch_scan<DT_BF16>(mk, mq, mks, d.prox, tile_prefix, d.B, d.Lmax, scores, ghist, d.status, d.sms, st);
+  if (e != cudaSuccess) return e;
+  static bool sel_attr = false;
+  const size_t sel_smem = sizeof(SelSmem) + 16;
+  if (!sel_attr) {
+    e = cudaFuncSetAttribute(decode_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sel_smem);
+    if (e != cudaSuccess) return e;
+    sel_attr = true;
+  }
+  decode_select_kernel<<<d.B, kBlk, sel_smem, st>>>(d.prox, d.Lmax, scores, ghist);
+  ++launch_counter();
+  if (d.mode == 1) {
+    ScanScratch sc = d.scratch_tc;
+    e = launch_refine_tc(d.q, d.B * d.g, d.dtype, chunks, d.B * mc * ncc, sc, d.sms, st);
+    if (e != cudaSuccess) return e;
+    entries_topk_kernel<<<d.B * d.g, kBlk, 0, st>>>(lists);
+    ++launch_counter();
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace pivot

@@ -26,6 +26,22 @@ struct GroupDesc {
   int32_t* out;         // [m, out_stride]
   float* out_score;     // optional
   int out_stride;
+  // Chunked mode (decode): when ent_out is set the kernel does not select; member r's packed
+  // entries go to ent_out[r * ent_stride + slot0 + slot] for a later top-k over the whole list.
+  unsigned long long* ent_out;
+  int ent_stride;
+  int slot0;
+};
+
+constexpr int kDecodeCandChunk = 512;   // candidates per re-score work item in decode
+
+// One query's re-scored candidates (packed entries) awaiting the final top-k.
+struct EntryList {
+  const unsigned long long* list;
+  int n;
+  int K;
+  int32_t* out;
+  float* out_score;
 };
 
 // Geometry of a prefill-shaped call, shared by the planner kernels.
@@ -85,6 +101,19 @@ cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_ro
 
 cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
                              const ScanScratch& s, int sms, cudaStream_t st);
+
+// Decode fast path: key-tile-split scan -> per-sequence select -> chunked re-score -> top-k.
+struct DecodeFast {
+  const RowDesc* prox;        // [B] proxy rows (K = 0: guarded sequence, skipped)
+  const GroupDesc* groups;    // [B * group_chunks(g)]
+  const void* kc; const float* kscale; const void* q; const void* proxy_q;
+  int B, Lmax, g, c, k, mode, dtype, sms;
+  void* scratch;              // decode_fast_bytes(...) bytes
+  ScanScratch scratch_tc;     // candidate scratch of the re-score kernel
+  int* status;
+};
+size_t decode_fast_bytes(int B, int Lmax, int g, int c);
+cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st);
 
 long long& launch_counter();
 

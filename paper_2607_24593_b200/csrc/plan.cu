@@ -88,6 +88,7 @@ __global__ void plan_prefill_kernel(PrefillPlan p, RowDesc* rows, GroupDesc* gro
       gd.out = p.out + (size_t)t0 * p.k;
       gd.out_score = p.out_score ? p.out_score + (size_t)t0 * p.k : nullptr;
       gd.out_stride = p.k;
+      gd.ent_out = nullptr; gd.ent_stride = 0; gd.slot0 = 0;
       const int chunks = (p.g + kMembersPerDesc - 1) / kMembersPerDesc;
       put_group_chunks(groups + (size_t)pr * chunks, gd, p.g, p.dtype);
     }
@@ -140,6 +141,7 @@ __global__ void plan_decode_kernel(DecodePlan p, RowDesc* rows, GroupDesc* group
   gd.out = outb;
   gd.out_score = outsb;
   gd.out_stride = p.k;
+  gd.ent_out = nullptr; gd.ent_stride = 0; gd.slot0 = 0;
   if (guarded) {
     r.K = 0; r.out = nullptr; r.out_score = nullptr; r.out_rows = 0; r.out_stride = 0;
   } else if (p.mode == 0) {

@@ -277,12 +277,17 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
 #pragma unroll
         for (int rl = 0; rl < 2; ++rl) {
           const int r = team * 2 + rl;
-          if (r < gd.m && t * 32 + lane < SEG)
-            sc.cand64[seg_off(r) + t * 32 + lane] =
-                idx >= 0 ? make_entry(score_to_key(gd.kscale ? score[rl] * ksv : score[rl]), idx) : kPadEntry;
+          const entry_t e =
+              idx >= 0 ? make_entry(score_to_key(gd.kscale ? score[rl] * ksv : score[rl]), idx) : kPadEntry;
+          if (gd.ent_out) {            // chunked mode: leave the entries for a later top-k
+            if (r < gd.m && slot < gd.n_cand) gd.ent_out[(size_t)r * gd.ent_stride + gd.slot0 + slot] = e;
+          } else if (r < gd.m && t * 32 + lane < SEG) {
+            sc.cand64[seg_off(r) + t * 32 + lane] = e;
+          }
         }
       }
       tm.sync();
+      if (gd.ent_out) continue;
       // ---- per-member exact top-k over the candidate scores
 #pragma unroll
       for (int rl = 0; rl < 2; ++rl) {
