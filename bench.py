@@ -227,6 +227,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--decode-only", action="store_true", help="only the MTP decode step (prints its object)")
     args = ap.parse_args()
     wl = args.workload
     if args.impl == "reference":
@@ -244,6 +245,10 @@ def main():
 
     from paper_2607_24593_b200 import binding as pv
 
+    if args.decode_only:
+        print(json.dumps(decode_bench(pv, torch.device(f"cuda:{local}"), steps=max(args.steps, 5),
+                                      warmup=max(args.warmup, 3), pk=peaks())))
+        return
     x = inputs.make_prefill(L, dtype=dtype, seed=rank_seed(rank))
     dev = torch.device(f"cuda:{local}")
     dq, dw, dk = x.q.to(dev), x.w.to(dev), x.k.to(dev)

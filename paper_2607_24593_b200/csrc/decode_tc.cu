@@ -28,10 +28,11 @@ namespace {
 
 constexpr int TILE_KEYS = 128;
 constexpr int DKS_SLOTS = 14;
-constexpr int DHIST = 16384;            // top 14 bits of the score key
+constexpr int DHIST_BITS = 13;          // histogram digit: top 13 bits of the score key (16 bins per octave)
+constexpr int DHIST = 1 << DHIST_BITS;
 constexpr int D_N = kHeads;             // MMA N: one proxy
-constexpr int D_THREADS = 64 + 128;     // TMA warp, MMA warp, four epilogue warps
-constexpr int SEL_CAP = 12288;          // candidates collected in shared memory per sequence
+constexpr int D_THREADS = 64 + 256;     // TMA warp, MMA warp, two sets of four epilogue warps
+constexpr int SEL_CAP = 16384;          // candidates collected in shared memory per sequence
 
 template <int DT>
 struct DCfg {
@@ -47,8 +48,8 @@ struct DCfg {
 
 struct DCtrl {
   alignas(128) float ks[DKS_SLOTS][TILE_KEYS];
-  alignas(16) float w[2][kHeads];
-  uint32_t hist[DHIST];
+  alignas(16) float w[2][kHeads];       // per epilogue set: gate of its current sequence
+  uint32_t hist[2][DHIST];              // per epilogue set: histogram of its current sequence
   uint64_t full[8], empty[8], q_full[2], q_empty[2], tmem_full[2], tmem_empty[2], ks_full[DKS_SLOTS];
   uint32_t tmem_base;
   int abort;
@@ -91,13 +92,13 @@ decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       ptx::mbar_init(&ct.q_full[i], 1);
       ptx::mbar_init(&ct.q_empty[i], 1);
       ptx::mbar_init(&ct.tmem_full[i], 1);
-      ptx::mbar_init(&ct.tmem_empty[i], 4);
+      ptx::mbar_init(&ct.tmem_empty[i], 4);   // the four warps of the set that owns buffer i
     }
     for (int i = 0; i < DKS_SLOTS; ++i) ptx::mbar_init(&ct.ks_full[i], 1);
     ct.abort = 0;
     ptx::fence_barrier_init();
   }
-  for (int i = threadIdx.x; i < DHIST; i += D_THREADS) ct.hist[i] = 0;
+  for (int i = threadIdx.x; i < 2 * DHIST; i += D_THREADS) (&ct.hist[0][0])[i] = 0;
   if (warp == 1) { ptx::tmem_alloc(&ct.tmem_base, 2 * D_N); ptx::tmem_relinquish(); }
   ptx::tc_fence_before();
   __syncthreads();
@@ -183,35 +184,36 @@ decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     }
   } else {
     // ------------------------------------------------------------------ epilogue
-    const int tt = threadIdx.x - 64;                 // 0..127 = key inside the tile
+    // Two sets of four warps take alternate tiles (set s drains accumulator buffer s), so one
+    // set's head sum overlaps the other's wait; each set keeps its own gate copy and histogram.
+    const int set = (warp - 2) >> 2;
+    const int tt = (threadIdx.x - 64) & 127;         // 0..127 inside the set
     const int lq = warp & 3;
     const int key_in_tile = lq * 32 + lane;
-    const Team tm{tt, 128, 1};
+    const Team tm{tt, 128, 1 + set};
     TileWalk tw(tile_prefix, B);
-    int cur_b = -1, wb = 0, n_vis = 0;
-    uint32_t it = 0, blk = 0;
+    int cur_b = -1, n_vis = 0;
     auto flush_hist = [&](int b) {
       tm.sync();
       for (int i = tt; i < DHIST; i += 128) {
-        const uint32_t h = ct.hist[i];
-        if (h) { atomicAdd(&ghist[(size_t)b * DHIST + i], h); ct.hist[i] = 0; }
+        const uint32_t h = ct.hist[set][i];
+        if (h) { atomicAdd(&ghist[(size_t)b * DHIST + i], h); ct.hist[set][i] = 0; }
       }
       tm.sync();
     };
-    for (int g = g_lo; g < g_hi; ++g, ++it) {
+    for (int g = g_lo + set; g < g_hi; g += 2) {
+      const uint32_t it = (uint32_t)(g - g_lo);
       const int b = tw.seq_of(g);
       const int t = g - tile_prefix[b];
       if (b != cur_b) {
         if (cur_b >= 0) flush_hist(cur_b);
-        wb = blk & 1;
-        ++blk;
         cur_b = b;
         n_vis = prox[b].n_vis;
         tm.sync();
-        if (tt < kHeads) ct.w[wb][tt] = 0.5f * prox[b].w[tt];      // proxy gate, halved (ReLU identity)
+        if (tt < kHeads) ct.w[set][tt] = 0.5f * prox[b].w[tt];      // proxy gate, halved (ReLU identity)
         tm.sync();
       }
-      const int buf = it & 1;
+      const int buf = it & 1;                        // == set
       float ksv = 1.f;
       if (C::FP8) {
         const int ksl = it % DKS_SLOTS;
@@ -229,7 +231,7 @@ decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
       float ap[4] = {0.f, 0.f, 0.f, 0.f}, an[4] = {0.f, 0.f, 0.f, 0.f};
-      const float4* wp = reinterpret_cast<const float4*>(&ct.w[wb][0]);
+      const float4* wp = reinterpret_cast<const float4*>(&ct.w[set][0]);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const float4 wa = wp[j], wbv = wp[8 + j];
@@ -251,7 +253,7 @@ decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       const int s_key = t * TILE_KEYS + key_in_tile;
       if (s_key < n_vis) {
         scores[(size_t)b * Lmax + s_key] = sv;
-        atomicAdd(&ct.hist[score_to_key(sv) >> 18], 1u);
+        atomicAdd(&ct.hist[set][score_to_key(sv) >> (32 - DHIST_BITS)], 1u);
       }
     }
     if (cur_b >= 0) flush_hist(cur_b);
@@ -280,7 +282,6 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Lmax, const float* __
   const int K = rd.K, n0 = rd.n_vis;
   if (K <= 0) return;
   const float* sc = scores + (size_t)b * Lmax;
-  auto entry_at = [&](int i) { return make_entry(score_to_key(__ldcg(sc + i)), i); };
   // ---- narrow the candidates: entries whose top `pbits` bits are >= prefix
   unsigned long long prefix = 0;
   int pbits = 0;
@@ -288,15 +289,32 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Lmax, const float* __
     blk_boundary(sm.blk, ghist + (size_t)b * DHIST, DHIST, (uint32_t)K);
     uint32_t need = sm.blk.need, pop = sm.blk.pop;
     prefix = sm.blk.bin;
-    pbits = 14;
+    pbits = DHIST_BITS;
     while ((uint32_t)K - need + pop > (uint32_t)SEL_CAP && pbits < 64) {
       const int wbits = 64 - pbits < 12 ? 64 - pbits : 12;
       __syncthreads();
       for (int i = tid; i < 4096; i += kBlk) sm.blk.hist[i] = 0;
       __syncthreads();
-      for (int i = tid; i < n0; i += kBlk) {
-        const entry_t e = entry_at(i);
-        if ((e >> (64 - pbits)) == prefix) atomicAdd(&sm.blk.hist[(uint32_t)((e >> (64 - pbits - wbits)) & ((1u << wbits) - 1u))], 1u);
+      for (int i0 = 0; i0 < n0; i0 += 16 * kBlk) {     // four 16-byte loads in flight per thread
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + (u * kBlk + tid) * 4;
+          v[u] = i < n0 ? __ldcg(reinterpret_cast<const float4*>(sc + i)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float vv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+          for (int e4 = 0; e4 < 4; ++e4) {
+            const int i = i0 + (u * kBlk + tid) * 4 + e4;
+            if (i < n0) {
+              const entry_t e = make_entry(score_to_key(vv[e4]), i);
+              if ((e >> (64 - pbits)) == prefix)
+                atomicAdd(&sm.blk.hist[(uint32_t)((e >> (64 - pbits - wbits)) & ((1u << wbits) - 1u))], 1u);
+            }
+          }
+        }
       }
       blk_boundary(sm.blk, sm.blk.hist, 4096, need);
       need = sm.blk.need;
@@ -308,23 +326,30 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Lmax, const float* __
   // ---- collect them in shared memory
   if (tid == 0) sm.blk.list_n = 0;
   __syncthreads();
-  for (int i0 = 0; i0 < n0; i0 += kBlk) {
-    const int i = i0 + tid;
-    entry_t e = 0;
-    bool keep = false;
-    if (i < n0) {
-      e = entry_at(i);
-      keep = pbits == 0 || (e >> (64 - pbits)) >= prefix;
+  for (int i0 = 0; i0 < n0; i0 += 16 * kBlk) {         // four 16-byte loads in flight per thread
+    float4 v4[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + (u * kBlk + tid) * 4;
+      v4[u] = i < n0 ? __ldcg(reinterpret_cast<const float4*>(sc + i)) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    const uint32_t m = __ballot_sync(0xffffffffu, keep);
-    if (m) {
-      uint32_t pos = 0;
-      const int leader = __ffs(m) - 1;
-      if (lane == leader) pos = atomicAdd(&sm.blk.list_n, (uint32_t)__popc(m));
-      pos = __shfl_sync(0xffffffffu, pos, leader);
-      if (keep) {
-        const uint32_t p = pos + __popc(m & ((1u << lane) - 1u));
-        if (p < (uint32_t)SEL_CAP) sm.list[p] = e;
+#pragma unroll
+    for (int u = 0; u < 16; ++u) {
+      const float4 q4 = v4[u >> 2];
+      const float vu = (u & 3) == 0 ? q4.x : (u & 3) == 1 ? q4.y : (u & 3) == 2 ? q4.z : q4.w;
+      const int i = i0 + ((u >> 2) * kBlk + tid) * 4 + (u & 3);
+      const entry_t e = make_entry(score_to_key(vu), i);
+      const bool keep = i < n0 && (pbits == 0 || (e >> (64 - pbits)) >= prefix);
+      const uint32_t m = __ballot_sync(0xffffffffu, keep);
+      if (m) {
+        uint32_t pos = 0;
+        const int leader = __ffs(m) - 1;
+        if (lane == leader) pos = atomicAdd(&sm.blk.list_n, (uint32_t)__popc(m));
+        pos = __shfl_sync(0xffffffffu, pos, leader);
+        if (keep) {
+          const uint32_t p = pos + __popc(m & ((1u << lane) - 1u));
+          if (p < (uint32_t)SEL_CAP) sm.list[p] = e;
+        }
       }
     }
   }
