@@ -118,7 +118,8 @@ ScanScratch tc_scratch(const Workspace& ws) {
 }
 
 bool g_timing = false;
-cudaEvent_t g_ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+cudaEvent_t g_ev[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+bool g_ev_decode_scan = false;
 bool g_ev_valid = false;
 inline void mark(int i, cudaStream_t st) {
   if (g_timing) { cudaEventRecord(g_ev[i], st); if (i == 4) g_ev_valid = true; }
@@ -305,6 +306,9 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
     df.scratch = (char*)wsp + base_bytes;
     df.scratch_tc = tc_scratch(ws);
     df.status = ws.status;
+    df.ev_scan_begin = g_timing ? g_ev[6] : nullptr;
+    df.ev_scan_end = g_timing ? g_ev[7] : nullptr;
+    g_ev_decode_scan = g_timing;
     if ((rc = check_cuda(launch_decode_fast(df, st)))) return rc;
     // dense rows of guarded (short) sequences, if any: the generic scan, one row per block
     ScanOperands op{kcache->data, (long long)B * Lmax, kcache->scale, q->data, B * g, ws.proxy_q, B, q->dtype};
@@ -390,13 +394,14 @@ int pivot_device_status(pivot_stream_t stream, int* status) {
 
 int pivot_stage_timing(int enable) {
   if (enable && !g_ev[0]) {
-    for (int i = 0; i < 6; ++i) {
+    for (int i = 0; i < 8; ++i) {
       int rc = check_cuda(cudaEventCreate(&g_ev[i]));
       if (rc) return rc;
     }
   }
   g_timing = enable != 0;
   g_ev_valid = false;
+  g_ev_decode_scan = false;
   return PIVOT_OK;
 }
 
@@ -406,7 +411,12 @@ int pivot_stage_times(float* ms, int n) {
   if (rc) return rc;
   for (int i = 0; i < 4; ++i)
     if ((rc = check_cuda(cudaEventElapsedTime(&ms[i], g_ev[i], g_ev[i + 1])))) return rc;
-  return check_cuda(cudaEventElapsedTime(&ms[4], g_ev[0], g_ev[4]));
+  if ((rc = check_cuda(cudaEventElapsedTime(&ms[4], g_ev[0], g_ev[4])))) return rc;
+  if (n >= 6) {
+    ms[5] = 0.f;
+    if (g_ev_decode_scan && (rc = check_cuda(cudaEventElapsedTime(&ms[5], g_ev[6], g_ev[7])))) return rc;
+  }
+  return PIVOT_OK;
 }
 
 long long pivot_launch_count_reset(void) {

@@ -465,10 +465,12 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   if (!make_operand_map(&mk, d.kc, (long long)d.B * d.Lmax, d.dtype, TILE_KEYS) ||
       !make_operand_map(&mq, d.proxy_q, (long long)d.B * kHeads, d.dtype, kHeads))
     return cudaErrorInvalidValue;
+  if (d.ev_scan_begin) cudaEventRecord(d.ev_scan_begin, st);
   e = d.dtype == DT_FP8
           ? launch_scan<DT_FP8>(mk, mq, mks, d.prox, tile_prefix, d.B, d.Lmax, scores, ghist, d.status, d.sms, st)
           : launch_scan<DT_BF16>(mk, mq, mks, d.prox, tile_prefix, d.B, d.Lmax, scores, ghist, d.status, d.sms, st);
   if (e != cudaSuccess) return e;
+  if (d.ev_scan_end) cudaEventRecord(d.ev_scan_end, st);
   static bool sel_attr = false;
   const size_t sel_smem = sizeof(SelSmem) + 16;
   if (!sel_attr) {

@@ -111,6 +111,7 @@ struct DecodeFast {
   void* scratch;              // decode_fast_bytes(...) bytes
   ScanScratch scratch_tc;     // candidate scratch of the re-score kernel
   int* status;
+  cudaEvent_t ev_scan_begin, ev_scan_end;   // optional: recorded around the scan kernel
 };
 size_t decode_fast_bytes(int B, int Lmax, int g, int c);
 cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st);
