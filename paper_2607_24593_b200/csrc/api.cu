@@ -49,9 +49,9 @@ int cand_cap(int kmax) {
 }
 
 int tc_cap(int kmax) {
-  size_t cap = (size_t)6 * kmax;
-  if (cap < 4096) cap = 4096;
-  return (int)align_up(cap, 128);
+  size_t cap = (size_t)8 * kmax;     // eight warp segments of K entries each
+  if (cap < 8192) cap = 8192;
+  return (int)align_up(cap, 256);
 }
 
 struct Carve {
@@ -93,7 +93,8 @@ Workspace carve_workspace(void* base, int rows, int n_groups, int c, int k) {
   w.rows = cv.take<RowDesc>((size_t)rows + n_groups);
   w.groups = cv.take<GroupDesc>((size_t)rows + n_groups);   // up to ceil(g/4) chunks per group
   // Candidate scratch.  Tensor-core kernels: one CTA per SM, 4 rows x cap packed entries each,
-  // cap = 6 K (a tight running threshold admits about K (1 + ln(n / K)) entries per row).
+  // cap = 8 K (a tight running threshold admits about K (1 + ln(n / K)) entries per row; one
+  // segment per epilogue warp, each able to hold K).
   // CUDA-core kernels: 4 CTAs per SM, two buffers of 2 K (key, index) pairs each.  The
   // region is sized for the larger of the two and shared.
   w.scan.n_cta = sm_count() * 4;

@@ -37,14 +37,23 @@ struct RCfg {
   static constexpr int QROW_HALF_BYTES = kHeads * 128;
   static constexpr int QHALF_BYTES = NMEM * QROW_HALF_BYTES;
   static constexpr int QBUF_BYTES = KHALVES * QHALF_BYTES;
-  static constexpr int STAGES = FP8 ? 6 : 2;      // bf16: 2 x 64 KB of queries leave room for two
-  static constexpr int LOOKAHEAD = FP8 ? 3 : 1;   // gather tiles in flight per producer thread
+  static constexpr int STAGES = FP8 ? 7 : 2;      // bf16: 2 x 64 KB of queries leave room for two
+  static constexpr int LOOKAHEAD = FP8 ? 5 : 1;   // gather tiles in flight per producer thread
   static constexpr int ROW_BYTES = FP8 ? 128 : 256;
   static constexpr uint32_t IDESC = ptx::make_idesc(FP8 ? 0u : 1u, TILE_KEYS, N);
 };
 
+constexpr int META_SLOTS = MAX_STAGES + 3;    // deeper than (key stages + accumulator buffers)
+
+// What the epilogue needs to know about a gathered key: its position and scale.
+struct KeyMeta {
+  int idx;       // key position, -1 for a padding slot
+  float ks;      // key scale (1 for bf16)
+};
+
 struct RCtrl {
   alignas(16) float w[NMEM][kHeads];
+  KeyMeta meta[META_SLOTS][TILE_KEYS];   // written by the gather warps, read by the epilogue
   uint64_t full[MAX_STAGES], empty[MAX_STAGES];
   uint64_t q_full[2], q_empty[2], tmem_full[2], tmem_empty[2];
   uint32_t tmem_base;
@@ -181,13 +190,27 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
     for (int gi = blockIdx.x; gi < n_groups; gi += gridDim.x) {
       const GroupDesc gd = groups[gi];
       const int ntiles = group_tiles(gd);
+      if (ntiles == 0) continue;
+      // Candidate positions are fetched two tiles ahead and key scales one tile ahead, so
+      // neither round trip sits on this thread's issue path.
+      auto load_idx = [&](int tile) -> int {
+        const int sl = tile * TILE_KEYS + j;
+        return (tile < ntiles && sl < gd.n_cand) ? __ldg(gd.cand + sl) : -1;
+      };
+      auto load_ks = [&](int ix) -> float { return (gd.kscale && ix >= 0) ? __ldg(gd.kscale + ix) : 1.f; };
+      int idx0 = load_idx(0), idx1 = load_idx(1);
+      float ks0 = load_ks(idx0);
       for (int t = 0; t < ntiles; ++t, ++it) {
         const int s = it % C::STAGES;
         const uint32_t ph = (it / C::STAGES) & 1;
-        const int slot = t * TILE_KEYS + j;
-        int idx = slot < gd.n_cand ? gd.cand[slot] : 0;
-        if (idx < 0) idx = 0;
+        const int idx_meta = idx0;
+        const float ks_meta = ks0;
+        const int idx2 = load_idx(t + 2);
+        const float ks1 = load_ks(idx1);
+        const int idx = idx_meta < 0 ? 0 : idx_meta;
         if (ok) ok = ptx::mbar_wait(&ct.empty[s], ph ^ 1, abort_flag);
+        ct.meta[it % META_SLOTS][j] = KeyMeta{idx_meta, ks_meta};
+        idx0 = idx1; idx1 = idx2; ks0 = ks1;
         const uint8_t* src = (const uint8_t*)gd.kbase + (size_t)idx * C::ROW_BYTES;
         const uint32_t dst = ptx::smem_u32(kring + s * C::STAGE_BYTES) + (uint32_t)j * 128u;
 #pragma unroll
@@ -232,43 +255,48 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
           wv = gd.w[r * kHeads + jh];
           if (gd.qscale) wv = __fmul_rn(wv, gd.qscale[r * kHeads + jh]);
         }
-        ct.w[r][jh] = wv;
+        ct.w[r][jh] = 0.5f * wv;       // halved: see the ReLU identity in the tile loop
       }
       tm.sync();
       for (int t = 0; t < ntiles; ++t, ++it) {
         const int buf = it & 1;
         const int slot = t * TILE_KEYS + key_in_tile;
-#ifdef EXP_R_NOLOADS
-        int idx = slot < gd.n_cand ? slot : -1;
-        const float ksv = 1.f;
-#else
-        int idx = slot < gd.n_cand ? gd.cand[slot] : -1;
-        const float ksv = (gd.kscale && idx >= 0) ? gd.kscale[idx] : 1.f;
-#endif
         (void)ptx::mbar_wait(&ct.tmem_full[buf], (it >> 1) & 1, abort_flag);
         ptx::tc_fence_after();
+        // position and scale of this thread's key, left in shared memory by the gather warps
+        // (no global load here: it would queue behind nothing good next to the TMEM loads)
+        const KeyMeta mt = ct.meta[it % META_SLOTS][key_in_tile];
+        const int idx = mt.idx;
+        const float ksv = mt.ks;
         float score[2];
 #pragma unroll
         for (int rl = 0; rl < 2; ++rl) {
           const int r = team * 2 + rl;
           const uint32_t taddr = tmem_base + ((uint32_t)(lq * 32) << 16) + buf * N + r * kHeads;
-          float acc = 0.f;
+          uint32_t v0[32], v1[32];
+          ptx::tmem_ld_32x32(taddr, v0);
+          ptx::tmem_ld_32x32(taddr + 32, v1);
+          ptx::tmem_wait_ld();
+          // w ReLU(x) = (w/2) x + (w/2) |x| (ct.w holds w/2): full-rate FMAs, eight chains
+          float ap[4] = {0.f, 0.f, 0.f, 0.f}, an[4] = {0.f, 0.f, 0.f, 0.f};
+          const float4* wp = reinterpret_cast<const float4*>(&ct.w[r][0]);
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            uint32_t v[32];
-            ptx::tmem_ld_32x32(taddr + half * 32, v);
-            ptx::tmem_wait_ld();
-            const float4* wp = reinterpret_cast<const float4*>(&ct.w[r][half * 32]);
-#pragma unroll
-            for (int q4 = 0; q4 < 8; ++q4) {
-              const float4 wv = wp[q4];
-              acc = fmaf(wv.x, fmaxf(__uint_as_float(v[4 * q4]), 0.f), acc);
-              acc = fmaf(wv.y, fmaxf(__uint_as_float(v[4 * q4 + 1]), 0.f), acc);
-              acc = fmaf(wv.z, fmaxf(__uint_as_float(v[4 * q4 + 2]), 0.f), acc);
-              acc = fmaf(wv.w, fmaxf(__uint_as_float(v[4 * q4 + 3]), 0.f), acc);
-            }
+          for (int q4 = 0; q4 < 8; ++q4) {
+            const float4 wa = wp[q4], wb = wp[8 + q4];
+            const float x0 = __uint_as_float(v0[4 * q4]), x1 = __uint_as_float(v0[4 * q4 + 1]);
+            const float x2 = __uint_as_float(v0[4 * q4 + 2]), x3 = __uint_as_float(v0[4 * q4 + 3]);
+            const float y0 = __uint_as_float(v1[4 * q4]), y1 = __uint_as_float(v1[4 * q4 + 1]);
+            const float y2 = __uint_as_float(v1[4 * q4 + 2]), y3 = __uint_as_float(v1[4 * q4 + 3]);
+            ap[0] = fmaf(fabsf(x0), wa.x, ap[0]); an[0] = fmaf(x0, wa.x, an[0]);
+            ap[1] = fmaf(fabsf(x1), wa.y, ap[1]); an[1] = fmaf(x1, wa.y, an[1]);
+            ap[2] = fmaf(fabsf(x2), wa.z, ap[2]); an[2] = fmaf(x2, wa.z, an[2]);
+            ap[3] = fmaf(fabsf(x3), wa.w, ap[3]); an[3] = fmaf(x3, wa.w, an[3]);
+            ap[0] = fmaf(fabsf(y0), wb.x, ap[0]); an[0] = fmaf(y0, wb.x, an[0]);
+            ap[1] = fmaf(fabsf(y1), wb.y, ap[1]); an[1] = fmaf(y1, wb.y, an[1]);
+            ap[2] = fmaf(fabsf(y2), wb.z, ap[2]); an[2] = fmaf(y2, wb.z, an[2]);
+            ap[3] = fmaf(fabsf(y3), wb.w, ap[3]); an[3] = fmaf(y3, wb.w, an[3]);
           }
-          score[rl] = acc;
+          score[rl] = ((ap[0] + an[0]) + (ap[1] + an[1])) + ((ap[2] + an[2]) + (ap[3] + an[3]));
         }
         ptx::tc_fence_before();
         __syncwarp();
@@ -297,13 +325,9 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         float* outs = gd.out_score ? gd.out_score + (size_t)r * gd.out_stride : nullptr;
         const int segcnt = min(ntiles * 32, SEG);
         const Seg seg{sc.cand64 + seg_off(r), segcnt};
-#ifdef EXP_R_NOSELECT
-        const int n_valid = gd.K;
-#else
         // 32 entries per lane (c <= 4096) fit the registers this kernel has; beyond that re-read
         const int n_valid = segcnt <= 32 * 32 ? seg_emit<true, 32>(tm, sel, seg, gd.n_cand, out, outs, gd.K)
                                               : seg_emit<false>(tm, sel, seg, gd.n_cand, out, outs, gd.K);
-#endif
         for (int i = n_valid + tt; i < gd.K; i += 128) {
           out[i] = -1;
           if (outs) outs[i] = -INFINITY;

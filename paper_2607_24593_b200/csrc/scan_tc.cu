@@ -21,15 +21,6 @@
 #include "segselect.cuh"
 
 namespace pivot {
-#ifdef PIVOT_PROFILE
-// Developer build only: per-CTA cycle counters of the epilogue phases (team 0, thread 0).
-__device__ unsigned long long g_scan_prof[256 * 8];
-#define PROF_T(var) const long long var = clock64()
-#define PROF_ADD(slot, t0, t1) if (tt == 0 && team == 0) prof[slot] += (unsigned long long)((t1) - (t0))
-#else
-#define PROF_T(var)
-#define PROF_ADD(slot, t0, t1)
-#endif
 namespace {
 
 constexpr int TILE_KEYS = 128;
@@ -295,9 +286,6 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     };
     BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
     uint32_t it = 0;
-#ifdef PIVOT_PROFILE
-    unsigned long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-#endif
     // A failed wait never changes this role's control flow (the team barriers below must stay
     // matched); once the abort flag is up every later wait returns at once.
     for (int b = bi.next(); b >= 0; b = bi.next()) {
@@ -340,7 +328,6 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       const int CHK = SEG / 64 < 32 ? (SEG / 64 > 0 ? SEG / 64 : 1) : 32;
       const int headroom = 32 * CHK;
       for (int t = 0; t < ntiles; ++t, ++it) {
-        PROF_T(p0);
         const bool meet = (t % CHK) == 0 && t > 0;
         if (meet) {
           tm.sync();
@@ -367,64 +354,34 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             }
             if (tt == 0) ct.flag[r] = 0;
             tm.sync();
-#ifdef PIVOT_PROFILE
-            if (tt == 0 && team == 0) prof[7] += 1;
-#endif
           }
         }
-        PROF_T(p1);
-        PROF_ADD(0, p0, p1);
         const int buf = it & 1;
         const int s_key = t * TILE_KEYS + key_in_tile;
         // Key scales come through shared memory (TMA): a global load issued by an epilogue warp
         // would sit in the same memory queue as its TMEM loads and stall them for an L2 round trip.
         float ksv = 1.f;
-#ifndef EXP_NOKS_A
         if (C::FP8) {
           const int ksl = it % KS_SLOTS;
           (void)ptx::mbar_wait(&ct.ks_full[ksl], (it / KS_SLOTS) & 1, abort_flag);
-#ifndef EXP_NOKS_B
           ksv = ct.ks[ksl][key_in_tile];
-#endif
         }
-#endif
         (void)ptx::mbar_wait(&ct.tmem_full[buf], (it >> 1) & 1, abort_flag);
         ptx::tc_fence_after();
-        PROF_T(p2);
-        PROF_ADD(1, p1, p2);
-#ifdef EXP_EARLY_RELEASE
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
-#endif
         float score[C::ROWS_PER_TEAM];
 #pragma unroll
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
           const int r = team * C::ROWS_PER_TEAM + rl;
           const uint32_t taddr = tmem_base + ((uint32_t)(lq * 32) << 16) + buf * C::N + r * kHeads;
           uint32_t v0[32], v1[32];
-#ifdef EXP_X64
-          {
-            uint32_t vv[64];
-            ptx::tmem_ld_32x64(taddr, vv);
-            ptx::tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 32; ++j) { v0[j] = vv[j]; v1[j] = vv[32 + j]; }
-          }
-#elif !defined(EXP_NOLD)
           ptx::tmem_ld_32x32(taddr, v0);
           ptx::tmem_ld_32x32(taddr + 32, v1);
           ptx::tmem_wait_ld();
-#else
-          for (int j = 0; j < 32; ++j) { v0[j] = taddr + j + it; v1[j] = taddr - j + it; }
-#endif
           // w ReLU(x) = (w/2) x + (w/2) |x|: two full-rate FMAs per element (|x| is a free
           // operand modifier) instead of a half-rate max plus an FMA; ct.w holds w/2.
           // Eight independent accumulation chains keep the FMA pipe busy.
           float ap[4] = {0.f, 0.f, 0.f, 0.f}, an[4] = {0.f, 0.f, 0.f, 0.f};
           const float4* wp = reinterpret_cast<const float4*>(&ct.w[r][0]);
-#ifdef EXP_NOFMA
-          for (int j = 0; j < 32; j += 8) ap[j >> 3] = __uint_as_float(v0[j]) + __uint_as_float(v1[j]);
-#else
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const float4 wa = wp[j], wb = wp[8 + j];
@@ -441,16 +398,11 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             ap[2] = fmaf(fabsf(y2), wb.z, ap[2]); an[2] = fmaf(y2, wb.z, an[2]);
             ap[3] = fmaf(fabsf(y3), wb.w, ap[3]); an[3] = fmaf(y3, wb.w, an[3]);
           }
-#endif
           score[rl] = ((ap[0] + an[0]) + (ap[1] + an[1])) + ((ap[2] + an[2]) + (ap[3] + an[3]));
         }
         ptx::tc_fence_before();
         __syncwarp();
-#ifndef EXP_EARLY_RELEASE
         if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
-#endif
-        PROF_T(p3);
-        PROF_ADD(2, p2, p3);
         // ---- count every score in the row histogram, append the ones above the threshold
         uint32_t key[C::ROWS_PER_TEAM];
         bool valid[C::ROWS_PER_TEAM];
@@ -478,34 +430,18 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
           // Only scores above the current threshold are counted: the ones at or below it can
           // never reach a bin edge the threshold could still move to, so the counts that
           // matter stay exact.
-#ifdef EXP_NOAPPEND
-          const bool take = false;
-#else
           const bool take = valid[rl] && key[rl] > thr[rl];
-#endif
-#ifndef EXP_NOHIST
           if (take) atomicAdd(&ct.rhist[r][key_bin(key[rl], base[rl])], 1u);
-#endif
           const uint32_t m = __ballot_sync(0xffffffffu, take);
           if (take) {
             const int p = cnt[rl] + __popc(m & ((1u << lane) - 1u));
-#ifndef EXP_NOSTORE
             if (p < SEG) seg_ptr(r)[p] = make_entry(key[rl], s_key);
             else ct.abort_code = DEV_CAND_OVERFLOW;
-#endif
           }
           cnt[rl] = min(cnt[rl] + __popc(m), SEG);
           if (lane == 0 && cnt[rl] + headroom > SEG) ct.flag[r] = 1;
         }
-        PROF_T(p4);
-        PROF_ADD(3, p3, p4);
-        PROF_T(p5);
-        PROF_ADD(4, p4, p5);
-#ifdef PIVOT_PROFILE
-        if (tt == 0 && team == 0) prof[6] += 1;
-#endif
       }
-      PROF_T(p6);
       // ---- end of the block: final exact select per row, then pad / replicate
 #pragma unroll
       for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
@@ -542,13 +478,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             if (rd.out_score) rd.out_score[(size_t)rr * rd.out_stride + i] = rd.out_score[i];
           }
       }
-      PROF_T(p7);
-      PROF_ADD(5, p6, p7);
     }
-#ifdef PIVOT_PROFILE
-    if (tt == 0 && team == 0)
-      for (int i = 0; i < 8; ++i) g_scan_prof[blockIdx.x * 8 + i] = prof[i];
-#endif
   }
   // ------------------------------------------------------------------ teardown
   ptx::tc_fence_before();
@@ -626,14 +556,6 @@ bool make_scale_map(CUtensorMap* m, const float* base, long long n) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-#ifdef PIVOT_PROFILE
-extern "C" int pivot_profile_read(unsigned long long* host, int n) {
-  return (int)cudaMemcpyFromSymbol(host, g_scan_prof, sizeof(unsigned long long) * (size_t)n);
-}
-extern "C" int pivot_profile_read_sel(unsigned long long* host) {
-  return (int)cudaMemcpyFromSymbol(host, g_sel_prof, sizeof(unsigned long long) * 16);
-}
-#endif
 
 cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_rows, int rows_per_block,
                            const ScanScratch& s, int sms, cudaStream_t st) {

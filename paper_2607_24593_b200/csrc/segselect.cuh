@@ -23,15 +23,6 @@
 
 namespace pivot {
 
-#ifdef PIVOT_PROFILE
-__device__ unsigned long long g_sel_prof[16];
-#define SELP_T(var) const long long var = clock64()
-#define SELP_ADD(slot, t0, t1) \
-  if (tm.tid == 0 && tm.bar == 1 && blockIdx.x == 0) g_sel_prof[slot] += (unsigned long long)((t1) - (t0))
-#else
-#define SELP_T(var)
-#define SELP_ADD(slot, t0, t1)
-#endif
 
 constexpr int kSelBins = 2048;
 constexpr int kSelSmall = 256;
@@ -51,7 +42,7 @@ struct SegSelSmem {
   entry_t list[kSelSmall];
   entry_t vmin, vmax;
   entry_t cut;
-  uint32_t wsum[4];
+  uint32_t wsum[8];
   uint32_t bin, need, pop;
   uint32_t list_n;
   uint32_t out_count;
@@ -106,15 +97,14 @@ struct SegRegs {
 // Boundary bin of a 2048-bin histogram walked from the top: the largest bin b such that the
 // bins >= b hold at least `need` entries.  Leaves (bin, need inside that bin, its population)
 // in sm.bin / sm.need / sm.pop; if the histogram holds fewer than `need` entries, bin = 0 and
-// pop = need = 0.  All 128 threads call.
+// pop = need = 0.  All threads of the team call (128 or 256 threads).
 __device__ __forceinline__ void hist_boundary(const Team& tm, SegSelSmem& sm, const uint32_t* hist, uint32_t need) {
   const int lane = tm.tid & 31;
   const int wq = tm.tid >> 5;
+  const int per = kSelBins / tm.nthr;       // bins per thread: 16 or 8
   tm.sync();          // everyone is done with the previous result, and the histogram is complete
-  uint32_t loc[16];
   uint32_t s = 0;
-#pragma unroll
-  for (int i = 0; i < 16; ++i) { loc[i] = hist[kSelBins - 1 - 16 * tm.tid - i]; s += loc[i]; }
+  for (int i = 0; i < per; ++i) s += hist[kSelBins - 1 - per * tm.tid - i];
   uint32_t incl = s;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -129,15 +119,15 @@ __device__ __forceinline__ void hist_boundary(const Team& tm, SegSelSmem& sm, co
   const uint32_t excl = base + incl - s;
   if (excl < need && need <= excl + s) {
     uint32_t cum = excl;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      if (cum + loc[i] >= need) {
-        sm.bin = (uint32_t)(kSelBins - 1 - 16 * tm.tid - i);
+    for (int i = 0; i < per; ++i) {
+      const uint32_t h = hist[kSelBins - 1 - per * tm.tid - i];
+      if (cum + h >= need) {
+        sm.bin = (uint32_t)(kSelBins - 1 - per * tm.tid - i);
         sm.need = need - cum;
-        sm.pop = loc[i];
+        sm.pop = h;
         break;
       }
-      cum += loc[i];
+      cum += h;
     }
   }
   tm.sync();
@@ -148,7 +138,6 @@ __device__ __forceinline__ void hist_boundary(const Team& tm, SegSelSmem& sm, co
 template <bool CACHED, int EPT = kSelEpt>
 __device__ __forceinline__ entry_t seg_find_cut(const Team& tm, SegSelSmem& sm, const SegRegs<CACHED, EPT>& regs, int K) {
   const int lane = tm.tid & 31;
-  SELP_T(q0);
   entry_t mn = ~0ull, mx = 0ull;
   regs.for_each([&](entry_t x) {
     mn = (x < mn && x != kPadEntry) ? x : mn;     // padding never bounds the range
@@ -167,10 +156,7 @@ __device__ __forceinline__ entry_t seg_find_cut(const Team& tm, SegSelSmem& sm, 
   tm.sync();
   entry_t lo = sm.vmin, hi = sm.vmax;
   uint32_t need = (uint32_t)K;
-  SELP_T(q1);
-  SELP_ADD(0, q0, q1);
   for (int iter = 0; iter < 8; ++iter) {
-    SELP_T(r0);
     const entry_t span = hi - lo;
     const int bitsw = span ? 64 - __clzll((long long)span) : 0;
     const int shift = bitsw > 11 ? bitsw - 11 : 0;
@@ -180,19 +166,12 @@ __device__ __forceinline__ entry_t seg_find_cut(const Team& tm, SegSelSmem& sm, 
       if (x >= lo && x <= hi) atomicAdd(&sm.hist[(uint32_t)((x - lo) >> shift)], 1u);
     });
     tm.sync();
-    SELP_T(r1);
-    SELP_ADD(1, r0, r1);
     hist_boundary(tm, sm, sm.hist, need);
     const uint32_t b = sm.bin, pop = sm.pop;
     need = sm.need;
     const entry_t lo2 = lo + ((entry_t)b << shift);
     const entry_t width1 = shift ? (((entry_t)1 << shift) - 1ull) : 0ull;
     const entry_t hi2 = (hi - lo2) < width1 ? hi : lo2 + width1;
-    SELP_T(r2);
-    SELP_ADD(2, r1, r2);
-#ifdef PIVOT_PROFILE
-    if (tm.tid == 0 && tm.bar == 1 && blockIdx.x == 0) { g_sel_prof[8] += 1; g_sel_prof[9] += pop; }
-#endif
     if (pop == need) {          // the whole boundary bin is wanted
       if (tm.tid == 0) sm.cut = lo2;
       tm.sync();
@@ -216,8 +195,6 @@ __device__ __forceinline__ entry_t seg_find_cut(const Team& tm, SegSelSmem& sm, 
         if (rank == need - 1) sm.cut = xt;
       }
       tm.sync();
-      SELP_T(r3);
-      SELP_ADD(3, r2, r3);
       return sm.cut;
     }
     lo = lo2;

@@ -21,6 +21,7 @@ constexpr size_t kStaticBytes = (size_t)8 << 20;          // 8 MiB per GPU
 constexpr int kStaticMaxL = 4096;
 constexpr int kStaticMaxK = 512;
 constexpr int kStaticCtas = 48;                           // grid cap: 48 x 4 rows x 4096 entries x 8 B = 6 MiB
+// (4096 entries per row = eight warp segments of 512 = the largest k this entry point accepts)
 constexpr int kStaticCap = 4096;                          // candidate entries per row
 constexpr int kMaxDev = 64;
 
