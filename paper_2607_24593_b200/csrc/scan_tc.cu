@@ -45,11 +45,9 @@ struct Cfg {
 #ifndef PIVOT_EPI16
   static constexpr int EPI_WARPS = NROWS == 4 ? 8 : 4;
   static constexpr int ROWS_PER_TEAM = NROWS == 4 ? 2 : 1;
-  static constexpr bool SEL_CACHED = true;
 #else
   static constexpr int EPI_WARPS = NROWS == 4 ? 16 : 4;
   static constexpr int ROWS_PER_TEAM = 1;
-  static constexpr bool SEL_CACHED = NROWS != 4;   // 576 threads leave too few registers to cache entries
 #endif
   static constexpr int TEAMS = EPI_WARPS / 4;
   static constexpr int THREADS = 64 + EPI_WARPS * 32;
@@ -263,9 +261,9 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     // Lower bound on the K-th best score seen so far, read off the row histogram: the largest
     // bin edge with at least K scores at or above it.  Returned as a key threshold t such that
     // only keys > t can still belong to the top K.
-    auto hist_threshold = [&](int r, int K, int base) -> uint32_t {
-      hist_boundary(tm, sel, ct.rhist[r], (uint32_t)K);
-      const uint32_t b = sel.bin;
+    auto hist_threshold = [&](int r, int K, int base) -> uint32_t {   // warp-local, no barrier
+      uint32_t b, need_in, pop;
+      if (!warp_hist_boundary(ct.rhist[r], (uint32_t)K, lane, &b, &need_in, &pop)) return 0u;
       return b > 0 ? (((uint32_t)((int)b + base)) << 15) - 1u : 0u;
     };
     auto team_max = [&](int v) -> int {          // max of a warp-uniform value over the team
@@ -442,7 +440,10 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
           if (lane == 0 && cnt[rl] + headroom > SEG) ct.flag[r] = 1;
         }
       }
-      // ---- end of the block: final exact select per row, then pad / replicate
+      // ---- end of the block: final exact select per row, then pad / replicate.  The row
+      //      histogram is exact for every entry still held, so one pass over the segments
+      //      suffices; a boundary bin too crowded to rank takes the general path.
+      tm.sync();
 #pragma unroll
       for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
         const int r = team * C::ROWS_PER_TEAM + rl;
@@ -450,22 +451,15 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         const int K = Ksel[rl];
         if (K <= 0) continue;
         const RowDesc rd = rows[ri];
-        int n = team_sum(cnt[rl]);
-        int mxc = team_max(cnt[rl]);
-        if (!C::SEL_CACHED || mxc > 32 * kSelEpt) {   // drop the entries the final threshold already rules out
-          const uint32_t th = hist_threshold(r, K, base[rl]);
+        const int rbase = base[rl];
+        int n_valid = seg_emit_hist(tm, sel, Seg{seg_ptr(r), cnt[rl]}, ct.rhist[r],
+                                    [&](uint32_t key) { return key_bin(key, rbase); }, rd.out, rd.out_score, K);
+        if (n_valid < 0) {
+          const uint32_t th = hist_threshold(r, K, rbase);
           const uint32_t tcur = th > thr[rl] ? th : thr[rl];
           cnt[rl] = seg_filter_inplace(seg_ptr(r), cnt[rl], lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
-          n = team_sum(cnt[rl]);
-          mxc = team_max(cnt[rl]);
-        }
-        const Seg seg{seg_ptr(r), cnt[rl]};
-        int n_valid;
-        if constexpr (C::SEL_CACHED) {
-          n_valid = mxc <= 32 * kSelEpt ? seg_emit<true>(tm, sel, seg, n, rd.out, rd.out_score, K)
-                                        : seg_emit<false>(tm, sel, seg, n, rd.out, rd.out_score, K);
-        } else {
-          n_valid = seg_emit<false>(tm, sel, seg, n, rd.out, rd.out_score, K);
+          const int n = team_sum(cnt[rl]);
+          n_valid = seg_emit<false>(tm, sel, Seg{seg_ptr(r), cnt[rl]}, n, rd.out, rd.out_score, K);
         }
         for (int i = n_valid + tt; i < K; i += 128) {
           rd.out[i] = -1;

@@ -133,6 +133,56 @@ __device__ __forceinline__ void hist_boundary(const Team& tm, SegSelSmem& sm, co
   tm.sync();
 }
 
+// Warp-local boundary bin of a 2048-bin histogram (16-byte aligned, shared memory), walked from
+// the top: the largest bin b such that the bins >= b hold at least `need` entries.  Returns
+// false if the histogram holds fewer than `need`.  No barrier: other warps may keep adding to
+// the histogram meanwhile; counts only grow, so a torn snapshot can only give a lower bin, which
+// is still a valid bound.  *need_in and *pop describe the boundary bin (entries still wanted
+// from it, and its population as read).
+__device__ __forceinline__ bool warp_hist_boundary(const uint32_t* hist, uint32_t need, int lane, uint32_t* bin,
+                                                   uint32_t* need_in, uint32_t* pop) {
+  const uint4* h4 = reinterpret_cast<const uint4*>(hist);
+  uint32_t cum = 0;
+  int jsel = -1;
+  // level 1: chunks of 128 bins, lane holds four consecutive bins of each chunk
+#pragma unroll
+  for (int j = kSelBins / 128 - 1; j >= 0; --j) {
+    const uint4 v = h4[j * 32 + lane];
+    const uint32_t c = __reduce_add_sync(0xffffffffu, (v.x + v.y) + (v.z + v.w));
+    if (jsel < 0) {
+      if (cum + c >= need) jsel = j;
+      else cum += c;
+    }
+  }
+  if (jsel < 0) { *bin = 0; *need_in = 0; *pop = 0; return false; }
+  // level 2: inside the chunk, suffix sums over the lanes
+  const uint4 v = h4[jsel * 32 + lane];
+  const uint32_t s = (v.x + v.y) + (v.z + v.w);
+  uint32_t incl = s;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_down_sync(0xffffffffu, incl, o);
+    if (lane + o < 32) incl += t;
+  }
+  const uint32_t above = cum + incl - s;              // entries in bins above this lane's four
+  const bool here = above < need && need <= above + s;
+  uint32_t b = 0, ni = 0, pp = 0;
+  if (here) {
+    uint32_t c = above;
+    if (c + v.w >= need) { b = 3; ni = need - c; pp = v.w; }
+    else if ((c += v.w) + v.z >= need) { b = 2; ni = need - c; pp = v.z; }
+    else if ((c += v.z) + v.y >= need) { b = 1; ni = need - c; pp = v.y; }
+    else { c += v.y; b = 0; ni = need - c; pp = v.x; }
+    b += (uint32_t)(jsel * 128 + lane * 4);
+  }
+  const uint32_t m = __ballot_sync(0xffffffffu, here);
+  const int src = __ffs(m) - 1;                        // exactly one lane
+  *bin = __shfl_sync(0xffffffffu, b, src);
+  *need_in = __shfl_sync(0xffffffffu, ni, src);
+  *pop = __shfl_sync(0xffffffffu, pp, src);
+  return true;
+}
+
 // Finds the K-th largest entry among the team's segments (more than K real entries in total).
 // All 128 threads call; the cut is returned (and left in sm.cut).
 template <bool CACHED, int EPT = kSelEpt>
@@ -283,6 +333,76 @@ __device__ __forceinline__ int seg_emit(const Team& tm, SegSelSmem& sm, const Se
   });
   tm.sync();
   return n_valid > K ? K : n_valid;
+}
+
+// Final selection of a row straight from its score histogram: `hist` counted every entry that
+// was ever appended and bin_of(key) is the bin it was counted in.  Entries in bins above the
+// boundary bin are emitted in one pass over the segments; the boundary bin's entries are ranked
+// by brute force.  Returns how many positions were written (K, or fewer when the segments hold
+// fewer than K), or -1 when the boundary bin holds more than kSelSmall entries (the caller then
+// takes the general path; `out` may hold partial results).  All threads of the team call, after
+// a team barrier that follows the last append.
+template <typename BinFn>
+__device__ __forceinline__ int seg_emit_hist(const Team& tm, SegSelSmem& sm, const Seg& seg, const uint32_t* hist,
+                                             BinFn bin_of, int32_t* out, float* out_score, int K) {
+  const int lane = tm.tid & 31;
+  uint32_t b = 0, need_b = 0, pop = 0;
+  const bool found = warp_hist_boundary(hist, (uint32_t)K, lane, &b, &need_b, &pop);
+  const int bsel = found ? (int)b : -1;
+  if (tm.tid == 0) { sm.out_count = 0; sm.list_n = 0; }
+  tm.sync();
+  for (int j0 = 0; j0 < seg.cnt; j0 += 256) {        // eight rows of 32 in flight
+    entry_t x[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = j0 + u * 32 + lane;
+      x[u] = i < seg.cnt ? __ldcg(seg.e + i) : kPadEntry;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const bool valid = (j0 + u * 32 + lane) < seg.cnt && entry_pos(x[u]) >= 0;
+      const int bn = (int)bin_of(entry_key(x[u]));
+      const bool emit = valid && bn > bsel;
+      const uint32_t m = __ballot_sync(0xffffffffu, emit);
+      if (m) {
+        uint32_t pos = 0;
+        const int leader = __ffs(m) - 1;
+        if (lane == leader) pos = atomicAdd(&sm.out_count, (uint32_t)__popc(m));
+        pos = __shfl_sync(0xffffffffu, pos, leader);
+        if (emit) {
+          const uint32_t p = pos + __popc(m & ((1u << lane) - 1u));
+          if (p < (uint32_t)K) {
+            out[p] = entry_pos(x[u]);
+            if (out_score) out_score[p] = key_to_score(entry_key(x[u]));
+          }
+        }
+      }
+      if (valid && bn == bsel) {
+        const uint32_t q = atomicAdd(&sm.list_n, 1u);
+        if (q < (uint32_t)kSelSmall) sm.list[q] = x[u];
+      }
+    }
+  }
+  tm.sync();
+  if (found) {
+    const uint32_t P = sm.list_n;
+    if (P > (uint32_t)kSelSmall) return -1;
+    for (uint32_t t = tm.tid; t < P; t += tm.nthr) {
+      const entry_t xt = sm.list[t];
+      uint32_t rank = 0;
+      for (uint32_t u = 0; u < P; ++u) rank += sm.list[u] > xt ? 1u : 0u;
+      if (rank < need_b) {
+        const uint32_t p = atomicAdd(&sm.out_count, 1u);
+        if (p < (uint32_t)K) {
+          out[p] = entry_pos(xt);
+          if (out_score) out_score[p] = key_to_score(entry_key(xt));
+        }
+      }
+    }
+    tm.sync();
+  }
+  const int n = (int)sm.out_count;
+  return n < K ? n : K;
 }
 
 }  // namespace pivot
