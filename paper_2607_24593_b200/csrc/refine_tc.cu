@@ -22,9 +22,9 @@ namespace {
 constexpr int TILE_KEYS = 128;
 constexpr int MAX_STAGES = 8;
 constexpr int NMEM = 4;                       // members per MMA (N = 256)
-constexpr int GATHER_WARPS = 4;
+constexpr int GATHER_WARPS = 2;       // each producer thread copies two rows of a tile
 constexpr int EPI_WARPS = 8;
-constexpr int THREADS = (2 + GATHER_WARPS + EPI_WARPS) * 32;   // 448
+constexpr int THREADS = (2 + GATHER_WARPS + EPI_WARPS) * 32;   // 384: 168 registers per thread
 constexpr int N = NMEM * kHeads;
 constexpr int TMEM_COLS = 2 * N;
 
@@ -175,10 +175,9 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
     }
   } else if (warp < 2 + GATHER_WARPS) {
     // ------------------------------------------------------------------ gather producers
-    // Thread j of the 128 copies candidate row j of each tile.  Tiles are committed as
-    // cp.async groups; a tile is published LOOKAHEAD tiles after it was issued.
+    // Thread j of the 64 copies candidate rows j and j + 64 of each tile.  Tiles are committed
+    // as cp.async groups; a tile is published LOOKAHEAD tiles after it was issued.
     const int j = (warp - 2) * 32 + lane;
-    const uint32_t swz = (uint32_t)(j & 7);
     uint32_t it = 0;          // tiles issued
     uint32_t pub = 0;         // tiles published
     bool ok = true;
@@ -193,31 +192,34 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       if (ntiles == 0) continue;
       // Candidate positions are fetched two tiles ahead and key scales one tile ahead, so
       // neither round trip sits on this thread's issue path.
-      auto load_idx = [&](int tile) -> int {
-        const int sl = tile * TILE_KEYS + j;
+      auto load_idx = [&](int tile, int half) -> int {
+        const int sl = tile * TILE_KEYS + half * 64 + j;
         return (tile < ntiles && sl < gd.n_cand) ? __ldg(gd.cand + sl) : -1;
       };
       auto load_ks = [&](int ix) -> float { return (gd.kscale && ix >= 0) ? __ldg(gd.kscale + ix) : 1.f; };
-      int idx0 = load_idx(0), idx1 = load_idx(1);
-      float ks0 = load_ks(idx0);
+      int idx0[2] = {load_idx(0, 0), load_idx(0, 1)}, idx1[2] = {load_idx(1, 0), load_idx(1, 1)};
+      float ks0[2] = {load_ks(idx0[0]), load_ks(idx0[1])};
       for (int t = 0; t < ntiles; ++t, ++it) {
         const int s = it % C::STAGES;
         const uint32_t ph = (it / C::STAGES) & 1;
-        const int idx_meta = idx0;
-        const float ks_meta = ks0;
-        const int idx2 = load_idx(t + 2);
-        const float ks1 = load_ks(idx1);
-        const int idx = idx_meta < 0 ? 0 : idx_meta;
+        const int idx2[2] = {load_idx(t + 2, 0), load_idx(t + 2, 1)};
+        const float ks1[2] = {load_ks(idx1[0]), load_ks(idx1[1])};
         if (ok) ok = ptx::mbar_wait(&ct.empty[s], ph ^ 1, abort_flag);
-        ct.meta[it % META_SLOTS][j] = KeyMeta{idx_meta, ks_meta};
-        idx0 = idx1; idx1 = idx2; ks0 = ks1;
-        const uint8_t* src = (const uint8_t*)gd.kbase + (size_t)idx * C::ROW_BYTES;
-        const uint32_t dst = ptx::smem_u32(kring + s * C::STAGE_BYTES) + (uint32_t)j * 128u;
 #pragma unroll
-        for (int h = 0; h < C::KHALVES; ++h)
+        for (int half = 0; half < 2; ++half) {
+          const int row = half * 64 + j;
+          ct.meta[it % META_SLOTS][row] = KeyMeta{idx0[half], ks0[half]};
+          const int idx = idx0[half] < 0 ? 0 : idx0[half];
+          const uint32_t swz = (uint32_t)(row & 7);
+          const uint8_t* src = (const uint8_t*)gd.kbase + (size_t)idx * C::ROW_BYTES;
+          const uint32_t dst = ptx::smem_u32(kring + s * C::STAGE_BYTES) + (uint32_t)row * 128u;
 #pragma unroll
-          for (int cidx = 0; cidx < 8; ++cidx)
-            cp_async16(dst + h * C::HALF_TILE_BYTES + ((cidx ^ swz) << 4), src + h * 128 + cidx * 16);
+          for (int h = 0; h < C::KHALVES; ++h)
+#pragma unroll
+            for (int cidx = 0; cidx < 8; ++cidx)
+              cp_async16(dst + h * C::HALF_TILE_BYTES + ((cidx ^ swz) << 4), src + h * 128 + cidx * 16);
+          idx0[half] = idx1[half]; idx1[half] = idx2[half]; ks0[half] = ks1[half];
+        }
         cp_async_commit();
         if (it + 1 - pub > (uint32_t)C::LOOKAHEAD) {
           cp_async_wait<C::LOOKAHEAD>();
