@@ -37,13 +37,21 @@ struct RCfg {
   static constexpr int QROW_HALF_BYTES = kHeads * 128;
   static constexpr int QHALF_BYTES = NMEM * QROW_HALF_BYTES;
   static constexpr int QBUF_BYTES = KHALVES * QHALF_BYTES;
-  static constexpr int STAGES = FP8 ? 7 : 2;      // bf16: 2 x 64 KB of queries leave room for two
-  static constexpr int LOOKAHEAD = FP8 ? 5 : 1;   // gather tiles in flight per producer thread
+  // FP8 keeps the group's score keys in shared memory (4 members x 4096 slots x 4 B) for the
+  // final top-k; bf16 has no room for that next to 2 x 64 KB of queries and goes through the
+  // per-CTA global segments instead.
+  static constexpr bool SMEM_SCORES = FP8;
+  // With the score rows resident, one query buffer (the next group's queries load while the
+  // key ring refills) buys two more gather stages, which matter more.
+  static constexpr int QBUFS = SMEM_SCORES ? 1 : 2;
+  static constexpr int STAGES = FP8 ? 6 : 2;
+  static constexpr int LOOKAHEAD = FP8 ? 4 : 1;   // gather tiles in flight per producer thread
   static constexpr int ROW_BYTES = FP8 ? 128 : 256;
   static constexpr uint32_t IDESC = ptx::make_idesc(FP8 ? 0u : 1u, TILE_KEYS, N);
 };
 
 constexpr int META_SLOTS = MAX_STAGES + 3;    // deeper than (key stages + accumulator buffers)
+constexpr int SCORE_SLOTS = 4096;             // shared-memory score row: candidates per member
 
 // What the epilogue needs to know about a gathered key: its position and scale.
 struct KeyMeta {
@@ -64,8 +72,10 @@ struct RCtrl {
 template <int DT>
 constexpr size_t rsmem_bytes() {
   using C = RCfg<DT>;
-  return 1024 + 2 * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(RCtrl);
+  return 1024 + C::QBUFS * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(RCtrl) +
+         (C::SMEM_SCORES ? (size_t)NMEM * SCORE_SLOTS * 4 : 0);
 }
+static_assert(rsmem_bytes<DT_FP8>() <= 232448 && rsmem_bytes<DT_BF16>() <= 232448, "shared memory budget");
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -88,8 +98,9 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* qbuf = smem;
-  uint8_t* kring = smem + 2 * C::QBUF_BYTES;
+  uint8_t* kring = smem + C::QBUFS * C::QBUF_BYTES;
   RCtrl& ct = *reinterpret_cast<RCtrl*>(kring + C::STAGES * C::STAGE_BYTES);
+  uint32_t* skey = reinterpret_cast<uint32_t*>(kring + C::STAGES * C::STAGE_BYTES + sizeof(RCtrl));   // [NMEM][SCORE_SLOTS]
   volatile int* abort_flag = &ct.abort;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -125,8 +136,8 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       for (int gi = blockIdx.x; gi < n_groups; gi += gridDim.x) {
         const GroupDesc gd = groups[gi];
         if (group_tiles(gd) == 0) continue;
-        const int qb = blk & 1;
-        if (!ptx::mbar_wait(&ct.q_empty[qb], ((blk >> 1) & 1) ^ 1, abort_flag)) break;
+        const int qb = blk % C::QBUFS;
+        if (!ptx::mbar_wait(&ct.q_empty[qb], ((blk / C::QBUFS) & 1) ^ 1, abort_flag)) break;
         ptx::mbar_arrive_expect_tx(&ct.q_full[qb], gd.m * C::KHALVES * C::QROW_HALF_BYTES);
         for (int r = 0; r < gd.m; ++r)
           for (int h = 0; h < C::KHALVES; ++h)
@@ -143,8 +154,8 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       for (int gi = blockIdx.x; gi < n_groups && ok; gi += gridDim.x) {
         const int ntiles = group_tiles(groups[gi]);
         if (ntiles == 0) continue;
-        const int qb = blk & 1;
-        ok = ptx::mbar_wait(&ct.q_full[qb], (blk >> 1) & 1, abort_flag);
+        const int qb = blk % C::QBUFS;
+        ok = ptx::mbar_wait(&ct.q_full[qb], (blk / C::QBUFS) & 1, abort_flag);
         if (!ok) break;
         const uint32_t q_addr = ptx::smem_u32(qbuf + qb * C::QBUF_BYTES);
         for (int t = 0; t < ntiles; ++t, ++it) {
@@ -248,6 +259,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       const GroupDesc gd = groups[gi];
       const int ntiles = group_tiles(gd);
       if (ntiles == 0) continue;
+      const bool smem_sel = C::SMEM_SCORES && !gd.ent_out && ntiles * TILE_KEYS <= SCORE_SLOTS;
       tm.sync();
       {
         const int rl = tt >> 6, jh = tt & 63;
@@ -307,8 +319,12 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
 #pragma unroll
         for (int rl = 0; rl < 2; ++rl) {
           const int r = team * 2 + rl;
-          const entry_t e =
-              idx >= 0 ? make_entry(score_to_key(gd.kscale ? score[rl] * ksv : score[rl]), idx) : kPadEntry;
+          const uint32_t key = score_to_key(gd.kscale ? score[rl] * ksv : score[rl]);
+          if (smem_sel) {              // key only; the position is looked up again at the end
+            if (r < gd.m) skey[r * SCORE_SLOTS + slot] = idx >= 0 ? key : 0u;
+            continue;
+          }
+          const entry_t e = idx >= 0 ? make_entry(key, idx) : kPadEntry;
           if (gd.ent_out) {            // chunked mode: leave the entries for a later top-k
             if (r < gd.m && slot < gd.n_cand) gd.ent_out[(size_t)r * gd.ent_stride + gd.slot0 + slot] = e;
           } else if (r < gd.m && t * 32 + lane < SEG) {
@@ -327,9 +343,24 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         float* outs = gd.out_score ? gd.out_score + (size_t)r * gd.out_stride : nullptr;
         const int segcnt = min(ntiles * 32, SEG);
         const Seg seg{sc.cand64 + seg_off(r), segcnt};
+        int n_valid = -1;
+        if (smem_sel) {
+          const uint32_t* keys = skey + r * SCORE_SLOTS;
+          n_valid = smem_row_topk(tm, sel, keys, ntiles * TILE_KEYS, gd.cand, gd.n_cand, out, outs, gd.K);
+          if (n_valid < 0) {           // crowded boundary bin (ties): spell the entries out and re-select
+            for (int i = 0; i < ntiles; ++i) {
+              const int sl = i * TILE_KEYS + tt;
+              const uint32_t k = keys[sl];
+              const int ci = __ldg(gd.cand + (sl < gd.n_cand ? sl : 0));
+              if (i * 32 + lane < SEG) sc.cand64[seg_off(r) + i * 32 + lane] = k ? make_entry(k, ci) : kPadEntry;
+            }
+            tm.sync();
+          }
+        }
         // 32 entries per lane (c <= 4096) fit the registers this kernel has; beyond that re-read
-        const int n_valid = segcnt <= 32 * 32 ? seg_emit<true, 32>(tm, sel, seg, gd.n_cand, out, outs, gd.K)
-                                              : seg_emit<false>(tm, sel, seg, gd.n_cand, out, outs, gd.K);
+        if (n_valid < 0)
+          n_valid = segcnt <= 32 * 32 ? seg_emit<true, 32>(tm, sel, seg, gd.n_cand, out, outs, gd.K)
+                                      : seg_emit<false>(tm, sel, seg, gd.n_cand, out, outs, gd.K);
         for (int i = n_valid + tt; i < gd.K; i += 128) {
           out[i] = -1;
           if (outs) outs[i] = -INFINITY;

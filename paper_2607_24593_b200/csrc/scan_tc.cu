@@ -263,7 +263,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     // only keys > t can still belong to the top K.
     auto hist_threshold = [&](int r, int K, int base) -> uint32_t {   // warp-local, no barrier
       uint32_t b, need_in, pop;
-      if (!warp_hist_boundary(ct.rhist[r], (uint32_t)K, lane, &b, &need_in, &pop)) return 0u;
+      if (!warp_hist_boundary<false>(ct.rhist[r], (uint32_t)K, lane, &b, &need_in, &pop)) return 0u;
       return b > 0 ? (((uint32_t)((int)b + base)) << 15) - 1u : 0u;
     };
     auto team_max = [&](int v) -> int {          // max of a warp-uniform value over the team

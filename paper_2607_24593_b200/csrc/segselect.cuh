@@ -38,7 +38,7 @@ __device__ __forceinline__ int32_t entry_pos(entry_t e) { return (int32_t)(~(uin
 constexpr entry_t kPadEntry = 0ull;   // lowest possible entry, position -1: never selected
 
 struct SegSelSmem {
-  uint32_t hist[kSelBins];
+  alignas(16) uint32_t hist[kSelBins];   // read as uint4 by warp_hist_boundary
   entry_t list[kSelSmall];
   entry_t vmin, vmax;
   entry_t cut;
@@ -48,6 +48,7 @@ struct SegSelSmem {
   uint32_t out_count;
   uint32_t total;
   uint32_t maxcnt;
+  uint32_t kmin, kmax;    // key range of a shared-memory score row
 };
 
 // One warp's view of its segment (warp-uniform count).
@@ -139,19 +140,42 @@ __device__ __forceinline__ void hist_boundary(const Team& tm, SegSelSmem& sm, co
 // the histogram meanwhile; counts only grow, so a torn snapshot can only give a lower bin, which
 // is still a valid bound.  *need_in and *pop describe the boundary bin (entries still wanted
 // from it, and its population as read).
+// BATCHED issues all level-1 loads before the reductions (faster, 16 more live registers);
+// the serial form is for callers inside a register-bound loop.
+template <bool BATCHED = true>
 __device__ __forceinline__ bool warp_hist_boundary(const uint32_t* hist, uint32_t need, int lane, uint32_t* bin,
                                                    uint32_t* need_in, uint32_t* pop) {
   const uint4* h4 = reinterpret_cast<const uint4*>(hist);
   uint32_t cum = 0;
   int jsel = -1;
-  // level 1: chunks of 128 bins, lane holds four consecutive bins of each chunk
+  // level 1: chunks of 128 bins, lane holds four consecutive bins of each chunk.  All loads
+  // first, then all reductions, so their latencies overlap.
+  constexpr int NCH = kSelBins / 128;
+  if constexpr (BATCHED) {
+    uint32_t part[NCH];
 #pragma unroll
-  for (int j = kSelBins / 128 - 1; j >= 0; --j) {
-    const uint4 v = h4[j * 32 + lane];
-    const uint32_t c = __reduce_add_sync(0xffffffffu, (v.x + v.y) + (v.z + v.w));
-    if (jsel < 0) {
-      if (cum + c >= need) jsel = j;
-      else cum += c;
+    for (int j = 0; j < NCH; ++j) {
+      const uint4 v = h4[j * 32 + lane];
+      part[j] = (v.x + v.y) + (v.z + v.w);
+    }
+#pragma unroll
+    for (int j = 0; j < NCH; ++j) part[j] = __reduce_add_sync(0xffffffffu, part[j]);
+#pragma unroll
+    for (int j = NCH - 1; j >= 0; --j) {
+      if (jsel < 0) {
+        if (cum + part[j] >= need) jsel = j;
+        else cum += part[j];
+      }
+    }
+  } else {
+#pragma unroll
+    for (int j = NCH - 1; j >= 0; --j) {
+      const uint4 v = h4[j * 32 + lane];
+      const uint32_t c = __reduce_add_sync(0xffffffffu, (v.x + v.y) + (v.z + v.w));
+      if (jsel < 0) {
+        if (cum + c >= need) jsel = j;
+        else cum += c;
+      }
     }
   }
   if (jsel < 0) { *bin = 0; *need_in = 0; *pop = 0; return false; }
@@ -347,7 +371,7 @@ __device__ __forceinline__ int seg_emit_hist(const Team& tm, SegSelSmem& sm, con
                                              BinFn bin_of, int32_t* out, float* out_score, int K) {
   const int lane = tm.tid & 31;
   uint32_t b = 0, need_b = 0, pop = 0;
-  const bool found = warp_hist_boundary(hist, (uint32_t)K, lane, &b, &need_b, &pop);
+  const bool found = warp_hist_boundary<false>(hist, (uint32_t)K, lane, &b, &need_b, &pop);
   const int bsel = found ? (int)b : -1;
   if (tm.tid == 0) { sm.out_count = 0; sm.list_n = 0; }
   tm.sync();
@@ -403,6 +427,122 @@ __device__ __forceinline__ int seg_emit_hist(const Team& tm, SegSelSmem& sm, con
   }
   const int n = (int)sm.out_count;
   return n < K ? n : K;
+}
+
+// Exact top-K of a row of score keys held in shared memory (0 = padding slot); the position of
+// slot s is cand[s] (s < n_cand).  One linear 2048-bin histogram over the row's key range finds
+// the boundary bin; the slots above it are emitted in a second pass and the boundary bin's
+// slots are ranked by (key, position).  Returns how many positions were written, or -1 --
+// before writing anything -- when the boundary bin is too crowded to rank (the caller takes the
+// general path).  At most 32 slots per thread (nslots <= 32 x team size, a multiple of the team
+// size); all threads of the team call.
+__device__ __forceinline__ int smem_row_topk(const Team& tm, SegSelSmem& sm, const uint32_t* keys, int nslots,
+                                             const int32_t* __restrict__ cand, int n_cand, int32_t* out,
+                                             float* out_score, int K) {
+  const int lane = tm.tid & 31;
+  const int per = nslots / tm.nthr;       // slots of this thread: i * nthr + tid, i < per
+  // positions first: their global-memory round trip hides behind the histogram passes
+  int ci[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const int s = i * tm.nthr + tm.tid;
+    ci[i] = (i < per && s < n_cand) ? __ldg(cand + s) : -1;
+  }
+  // ... and the keys: every pass below runs on registers
+  uint32_t kreg[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) kreg[i] = i < per ? keys[i * tm.nthr + tm.tid] : 0u;
+  uint32_t mn = 0xffffffffu, mx = 0u, nv = 0u;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const uint32_t k = kreg[i];
+    mn = (k && k < mn) ? k : mn;
+    mx = k > mx ? k : mx;
+    nv += k ? 1u : 0u;
+  }
+  if (tm.tid == 0) { sm.kmin = 0xffffffffu; sm.kmax = 0u; sm.total = 0u; sm.out_count = 0u; sm.list_n = 0u; }
+  for (int i = tm.tid; i < kSelBins; i += tm.nthr) sm.hist[i] = 0;
+  tm.sync();
+  mn = __reduce_min_sync(0xffffffffu, mn);
+  mx = __reduce_max_sync(0xffffffffu, mx);
+  nv = __reduce_add_sync(0xffffffffu, nv);
+  if (lane == 0) { atomicMin(&sm.kmin, mn); atomicMax(&sm.kmax, mx); atomicAdd(&sm.total, nv); }
+  tm.sync();
+  const uint32_t lo = sm.kmin, hi = sm.kmax;
+  const int n_valid = (int)sm.total;
+  int bsel = -1;            // emit every bin above bsel
+  uint32_t need_b = 0;
+  bool whole_bin = false;   // the boundary bin is wanted entirely
+  int shift = 0;
+  if (n_valid > K) {
+    const uint32_t span = hi - lo;
+    const int bitsw = span ? 32 - __clz(span) : 0;
+    shift = bitsw > 11 ? bitsw - 11 : 0;
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+      if (kreg[i]) atomicAdd(&sm.hist[(kreg[i] - lo) >> shift], 1u);
+    tm.sync();
+    uint32_t b, pop;
+    warp_hist_boundary(sm.hist, (uint32_t)K, lane, &b, &need_b, &pop);   // same result in every warp
+    if (pop != need_b && pop > (uint32_t)kSelSmall) return -1;
+    bsel = (int)b;
+    whole_bin = pop == need_b;
+  }
+  // Which of this thread's slots go out: counted first, then a scan over the team hands every
+  // thread a contiguous run of output positions (no atomics, no votes in the write loop).
+  uint32_t emit_mask = 0u;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const uint32_t k = kreg[i];
+    const bool valid = k != 0u;
+    const int bn = valid ? (int)((k - lo) >> shift) : -2;
+    if (valid && (bn > bsel || (whole_bin && bn == bsel))) emit_mask |= 1u << i;
+    if (valid && bn == bsel && !whole_bin) {
+      const uint32_t q = atomicAdd(&sm.list_n, 1u);
+      if (q < (uint32_t)kSelSmall) sm.list[q] = make_entry(k, ci[i]);
+    }
+  }
+  const uint32_t mine = (uint32_t)__popc(emit_mask);
+  uint32_t incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  const int wq = tm.tid >> 5;
+  if (lane == 31) sm.wsum[wq] = incl;
+  tm.sync();
+  uint32_t p = incl - mine;
+  for (int w = 0; w < wq; ++w) p += sm.wsum[w];
+  if (tm.tid == tm.nthr - 1) sm.out_count = p + mine;      // emitted so far; the ranked ones follow
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    if ((emit_mask >> i) & 1u) {
+      if (p < (uint32_t)K) {
+        out[p] = ci[i];
+        if (out_score) out_score[p] = key_to_score(kreg[i]);
+      }
+      ++p;
+    }
+  }
+  tm.sync();
+  if (bsel >= 0 && !whole_bin) {
+    const uint32_t P = sm.list_n < (uint32_t)kSelSmall ? sm.list_n : (uint32_t)kSelSmall;
+    for (uint32_t t = tm.tid; t < P; t += tm.nthr) {
+      const entry_t xt = sm.list[t];
+      uint32_t rank = 0;
+      for (uint32_t u = 0; u < P; ++u) rank += sm.list[u] > xt ? 1u : 0u;
+      if (rank < need_b) {
+        const uint32_t p = atomicAdd(&sm.out_count, 1u);
+        if (p < (uint32_t)K) {
+          out[p] = entry_pos(xt);
+          if (out_score) out_score[p] = key_to_score(entry_key(xt));
+        }
+      }
+    }
+    tm.sync();
+  }
+  return n_valid < K ? n_valid : K;
 }
 
 }  // namespace pivot
