@@ -137,7 +137,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         const GroupDesc gd = groups[gi];
         if (group_tiles(gd) == 0) continue;
         const int qb = blk % C::QBUFS;
-        if (!ptx::mbar_wait(&ct.q_empty[qb], ((blk / C::QBUFS) & 1) ^ 1, abort_flag)) break;
+        if (!ptx::mbar_wait(&ct.q_empty[qb], ((blk / C::QBUFS) & 1) ^ 1, abort_flag, 128)) break;
         ptx::mbar_arrive_expect_tx(&ct.q_full[qb], gd.m * C::KHALVES * C::QROW_HALF_BYTES);
         for (int r = 0; r < gd.m; ++r)
           for (int h = 0; h < C::KHALVES; ++h)
@@ -155,16 +155,16 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         const int ntiles = group_tiles(groups[gi]);
         if (ntiles == 0) continue;
         const int qb = blk % C::QBUFS;
-        ok = ptx::mbar_wait(&ct.q_full[qb], (blk / C::QBUFS) & 1, abort_flag);
+        ok = ptx::mbar_wait(&ct.q_full[qb], (blk / C::QBUFS) & 1, abort_flag, 32);
         if (!ok) break;
         const uint32_t q_addr = ptx::smem_u32(qbuf + qb * C::QBUF_BYTES);
         for (int t = 0; t < ntiles; ++t, ++it) {
           const int s = it % C::STAGES;
           const uint32_t ph = (it / C::STAGES) & 1;
           const int buf = it & 1;
-          ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag);
+          ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, 32);
           if (!ok) break;
-          ok = ptx::mbar_wait(&ct.full[s], ph, abort_flag);
+          ok = ptx::mbar_wait(&ct.full[s], ph, abort_flag, 32);
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t k_addr = ptx::smem_u32(kring + s * C::STAGE_BYTES);
@@ -215,7 +215,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         const uint32_t ph = (it / C::STAGES) & 1;
         const int idx2[2] = {load_idx(t + 2, 0), load_idx(t + 2, 1)};
         const float ks1[2] = {load_ks(idx1[0]), load_ks(idx1[1])};
-        if (ok) ok = ptx::mbar_wait(&ct.empty[s], ph ^ 1, abort_flag);
+        if (ok) ok = ptx::mbar_wait(&ct.empty[s], ph ^ 1, abort_flag, 64);   // whole warps wait here: sleep, do not spin
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
           const int row = half * 64 + j;

@@ -366,37 +366,45 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         }
         (void)ptx::mbar_wait(&ct.tmem_full[buf], (it >> 1) & 1, abort_flag);
         ptx::tc_fence_after();
+        // The accumulator comes over in 32-column chunks, two register sets in turn: while one
+        // chunk goes through the FMAs the next is already on its way from TMEM.
+        // w ReLU(x) = (w/2) x + (w/2) |x|: two full-rate FMAs per element (|x| is a free operand
+        // modifier) instead of a half-rate max plus an FMA; ct.w holds w/2.  Eight independent
+        // accumulation chains per row keep the FMA pipe busy.
         float score[C::ROWS_PER_TEAM];
-#pragma unroll
-        for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
-          const int r = team * C::ROWS_PER_TEAM + rl;
-          const uint32_t taddr = tmem_base + ((uint32_t)(lq * 32) << 16) + buf * C::N + r * kHeads;
-          uint32_t v0[32], v1[32];
-          ptx::tmem_ld_32x32(taddr, v0);
-          ptx::tmem_ld_32x32(taddr + 32, v1);
-          ptx::tmem_wait_ld();
-          // w ReLU(x) = (w/2) x + (w/2) |x|: two full-rate FMAs per element (|x| is a free
-          // operand modifier) instead of a half-rate max plus an FMA; ct.w holds w/2.
-          // Eight independent accumulation chains keep the FMA pipe busy.
-          float ap[4] = {0.f, 0.f, 0.f, 0.f}, an[4] = {0.f, 0.f, 0.f, 0.f};
-          const float4* wp = reinterpret_cast<const float4*>(&ct.w[r][0]);
+        constexpr int NCHUNK = 2 * C::ROWS_PER_TEAM;            // 32-column chunks of this warp
+        const uint32_t tbase = tmem_base + ((uint32_t)(lq * 32) << 16) + buf * C::N + team * C::ROWS_PER_TEAM * kHeads;
+        uint32_t va[32], vb[32];
+        float ap[4], an[4];
+        auto fma_chunk = [&](const uint32_t (&v)[32], const float* wrow) {
+          const float4* wp = reinterpret_cast<const float4*>(wrow);
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            const float4 wa = wp[j], wb = wp[8 + j];
-            const float x0 = __uint_as_float(v0[4 * j]), x1 = __uint_as_float(v0[4 * j + 1]);
-            const float x2 = __uint_as_float(v0[4 * j + 2]), x3 = __uint_as_float(v0[4 * j + 3]);
-            const float y0 = __uint_as_float(v1[4 * j]), y1 = __uint_as_float(v1[4 * j + 1]);
-            const float y2 = __uint_as_float(v1[4 * j + 2]), y3 = __uint_as_float(v1[4 * j + 3]);
-            ap[0] = fmaf(fabsf(x0), wa.x, ap[0]); an[0] = fmaf(x0, wa.x, an[0]);
-            ap[1] = fmaf(fabsf(x1), wa.y, ap[1]); an[1] = fmaf(x1, wa.y, an[1]);
-            ap[2] = fmaf(fabsf(x2), wa.z, ap[2]); an[2] = fmaf(x2, wa.z, an[2]);
-            ap[3] = fmaf(fabsf(x3), wa.w, ap[3]); an[3] = fmaf(x3, wa.w, an[3]);
-            ap[0] = fmaf(fabsf(y0), wb.x, ap[0]); an[0] = fmaf(y0, wb.x, an[0]);
-            ap[1] = fmaf(fabsf(y1), wb.y, ap[1]); an[1] = fmaf(y1, wb.y, an[1]);
-            ap[2] = fmaf(fabsf(y2), wb.z, ap[2]); an[2] = fmaf(y2, wb.z, an[2]);
-            ap[3] = fmaf(fabsf(y3), wb.w, ap[3]); an[3] = fmaf(y3, wb.w, an[3]);
+            const float4 wv = wp[j];
+            const float x0 = __uint_as_float(v[4 * j]), x1 = __uint_as_float(v[4 * j + 1]);
+            const float x2 = __uint_as_float(v[4 * j + 2]), x3 = __uint_as_float(v[4 * j + 3]);
+            ap[0] = fmaf(fabsf(x0), wv.x, ap[0]); an[0] = fmaf(x0, wv.x, an[0]);
+            ap[1] = fmaf(fabsf(x1), wv.y, ap[1]); an[1] = fmaf(x1, wv.y, an[1]);
+            ap[2] = fmaf(fabsf(x2), wv.z, ap[2]); an[2] = fmaf(x2, wv.z, an[2]);
+            ap[3] = fmaf(fabsf(x3), wv.w, ap[3]); an[3] = fmaf(x3, wv.w, an[3]);
           }
-          score[rl] = ((ap[0] + an[0]) + (ap[1] + an[1])) + ((ap[2] + an[2]) + (ap[3] + an[3]));
+        };
+        ptx::tmem_ld_32x32(tbase, va);
+#pragma unroll
+        for (int c = 0; c < NCHUNK; ++c) {
+          ptx::tmem_wait_ld();                                  // chunk c has landed
+          if (c + 1 < NCHUNK) {
+            if (c & 1) ptx::tmem_ld_32x32(tbase + (c + 1) * 32, va);
+            else ptx::tmem_ld_32x32(tbase + (c + 1) * 32, vb);
+          }
+          if ((c & 1) == 0) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { ap[i] = 0.f; an[i] = 0.f; }
+          }
+          const float* wrow = &ct.w[team * C::ROWS_PER_TEAM + (c >> 1)][(c & 1) * 32];
+          if (c & 1) fma_chunk(vb, wrow);
+          else fma_chunk(va, wrow);
+          if (c & 1) score[c >> 1] = ((ap[0] + an[0]) + (ap[1] + an[1])) + ((ap[2] + an[2]) + (ap[3] + an[3]));
         }
         ptx::tc_fence_before();
         __syncwarp();
