@@ -83,6 +83,11 @@ typedef struct pivot_tensor {
  *   impl          0: tensor-core kernels (tcgen05; the product path).  1: the plain CUDA-core
  *                 kernels that compute the same thing one key per thread -- a slow on-device
  *                 cross-check, not a fallback: nothing selects it automatically.
+ *   row_begin, row_end  prefill / dense only: index just the query rows row_begin .. row_end-1 of
+ *                 the request (chunked prefill; the other rows of out_idx are left untouched).
+ *                 Both 0 = all rows.  row_begin must be a multiple of g, row_end a multiple of g
+ *                 or L.  Tensor arguments keep their full-request shapes; a chunk's result is the
+ *                 same as the corresponding rows of one whole call (groups never straddle chunks).
  */
 typedef struct pivot_opts {
   int guard_len;
@@ -93,6 +98,7 @@ typedef struct pivot_opts {
   void* workspace;
   size_t workspace_bytes;
   int impl;
+  int row_begin, row_end;
 } pivot_opts;
 
 /* Bytes of scratch a prefill / dense call with these sizes needs: rows = L, n_groups = ceil(L/g)
@@ -171,9 +177,14 @@ int dense_index_static(const pivot_tensor* q, const float* w, const pivot_tensor
 
 /*
  * Host-buffer form of pivot_index_prefill: every tensor pointer (q, w, kcache, out_idx) is HOST
- * memory (pinned for full copy speed).  The call copies the inputs into `arena` (device,
- * at least pivot_prefill_host_arena_bytes(...) bytes, which includes the workspace), runs the
- * device path, copies out_idx back and synchronises `stream` before returning.
+ * memory (pinned, else the copies are neither asynchronous nor fast).  The call copies the inputs
+ * into `arena` (device, at least pivot_prefill_host_arena_bytes(...) bytes, which includes the
+ * workspace), runs the device path and copies out_idx back; it returns after everything has
+ * finished.  Keys and gates go first; the queries then travel in row chunks on a copy stream of
+ * the library's own while earlier chunks are indexed on `stream` (row_begin / row_end of
+ * pivot_opts) and their results return on a second copy stream, so the PCIe transfers in both
+ * directions overlap the kernels.  The first call on a device creates the two copy streams and
+ * their events (kept until the process exits).
  */
 size_t pivot_prefill_host_arena_bytes(int L, int H_I, int d, int g, int c, int k, int dtype);
 int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,

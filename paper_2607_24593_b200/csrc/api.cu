@@ -14,11 +14,16 @@ namespace {
 constexpr int kMaxSel = 8192;
 constexpr int kMaxDevices = 64;
 
+constexpr int kHostChunks = 8;       // query-row chunks of the host-buffer prefill pipeline
+
 struct DeviceState {
   void* ws = nullptr;
   size_t ws_bytes = 0;
   int sm_count = 0;
   int* last_status = nullptr;
+  // host-buffer prefill: copy streams and events, created on first use
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;
+  cudaEvent_t ev_entry = nullptr, ev_in[kHostChunks] = {}, ev_done[kHostChunks] = {};
 };
 DeviceState g_dev[kMaxDevices];
 int g_last_cuda = 0;
@@ -172,22 +177,34 @@ int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, i
   int first_group = guard <= 1 ? 0 : (guard - 1 + g - 1) / g;
   if (first_group > nG) first_group = nG;
   if (dense_only) first_group = nG;
-  long long nd = (long long)first_group * g;
+  long long nd = (long long)first_group * g;      // rows below nd are scored densely
+  if (nd > L) nd = L;
+  // optional row range (chunked prefill): groups never straddle a chunk boundary
+  int r0 = 0, r1 = L;
+  if (o && (o->row_begin || o->row_end)) {
+    r0 = o->row_begin; r1 = o->row_end;
+    if (r0 < 0 || r1 <= r0 || r1 > L || r0 % g || (r1 % g && r1 != L)) return PIVOT_ERR_INVALID_ARG;
+  }
+  const int g_begin = r0 / g, g_end = (r1 + g - 1) / g;
+  const int dense0 = r0 < nd ? r0 : (int)nd;
+  const int dense1 = r1 < nd ? r1 : (int)nd;
+  const int pg0 = g_begin > first_group ? g_begin : first_group;   // first proxy group of this call
   PrefillPlan p;
   p.q = q->data; p.w = w; p.qscale = q->scale;
   p.kc = kc->data; p.kscale = kc->scale;
   p.proxy_q = ws.proxy_q; p.proxy_w = ws.proxy_w;
-  p.cand = (o && o->dbg_cand) ? o->dbg_cand + (size_t)first_group * c : ws.cand;
-  p.cand_score = (o && o->dbg_cand_scores) ? o->dbg_cand_scores + (size_t)first_group * c : nullptr;
+  p.cand = (o && o->dbg_cand) ? o->dbg_cand + (size_t)pg0 * c : ws.cand;
+  p.cand_score = (o && o->dbg_cand_scores) ? o->dbg_cand_scores + (size_t)pg0 * c : nullptr;
   p.out = out_idx; p.out_score = o ? o->dbg_scores : nullptr;
   p.L = L; p.g = g; p.c = c; p.k = k; p.mode = mode; p.dtype = q->dtype;
-  p.n_dense = (int)(nd < L ? nd : L);
-  p.first_group = first_group;
-  p.n_proxy = nG - first_group;
+  p.dense_begin = dense0;
+  p.n_dense = dense1 - dense0;
+  p.first_group = pg0;
+  p.n_proxy = g_end > pg0 ? g_end - pg0 : 0;
 
   if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 2 * sizeof(int), st)))) return rc;
   mark(0, st);
-  launch_proxy_build(q->data, q->scale, w, ws.proxy_q, ws.proxy_w, L, g, first_group, p.n_proxy,
+  launch_proxy_build(q->data, q->scale, w, ws.proxy_q, ws.proxy_w, L, g, pg0, p.n_proxy,
                      q->dtype, o ? o->pool : 0, st);
   mark(1, st);
   launch_plan_prefill(p, ws.rows, ws.groups, st);
@@ -352,35 +369,75 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
     return PIVOT_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   const bool fp8 = q->dtype == PIVOT_FP8_E4M3;
+  if (fp8 && (!q->scale || !kcache->scale)) return PIVOT_ERR_INVALID_ARG;
   const size_t esz = fp8 ? 1 : 2;
+  int rc;
+  DeviceState& ds = g_dev[cur_device()];
+  if (!ds.copy_in) {
+    if ((rc = check_cuda(cudaStreamCreateWithFlags(&ds.copy_in, cudaStreamNonBlocking)))) return rc;
+    if ((rc = check_cuda(cudaStreamCreateWithFlags(&ds.copy_out, cudaStreamNonBlocking)))) return rc;
+    if ((rc = check_cuda(cudaEventCreateWithFlags(&ds.ev_entry, cudaEventDisableTiming)))) return rc;
+    for (int i = 0; i < kHostChunks; ++i) {
+      if ((rc = check_cuda(cudaEventCreateWithFlags(&ds.ev_in[i], cudaEventDisableTiming)))) return rc;
+      if ((rc = check_cuda(cudaEventCreateWithFlags(&ds.ev_done[i], cudaEventDisableTiming)))) return rc;
+    }
+  }
   Carve cv(arena);
-  void* dq = cv.take<char>((size_t)L * H_I * d * esz);
+  char* dq = cv.take<char>((size_t)L * H_I * d * esz);
   float* dqs = cv.take<float>((size_t)L * H_I);
   float* dw = cv.take<float>((size_t)L * H_I);
   void* dk = cv.take<char>((size_t)L * d * esz);
   float* dks = cv.take<float>((size_t)L);
   int32_t* dout = cv.take<int32_t>((size_t)L * k);
-  void* dws = arena ? (char*)arena + cv.off : nullptr;
-  int rc;
-  if ((rc = check_cuda(cudaMemcpyAsync(dq, q->data, (size_t)L * H_I * d * esz, cudaMemcpyHostToDevice, st)))) return rc;
-  if ((rc = check_cuda(cudaMemcpyAsync(dw, w, (size_t)L * H_I * 4, cudaMemcpyHostToDevice, st)))) return rc;
+  void* dws = (char*)arena + cv.off;
+
+  // Row chunks: whole groups, at least 8192 rows each, at most kHostChunks of them.
+  const int nG = (L + g - 1) / g;
+  int n_chunks = L / 8192;
+  n_chunks = n_chunks < 1 ? 1 : (n_chunks > kHostChunks ? kHostChunks : n_chunks);
+  const int chunk_rows = ((nG + n_chunks - 1) / n_chunks) * g;
+  n_chunks = (L + chunk_rows - 1) / chunk_rows;
+
+  // The copy-in stream may not touch the arena before earlier work on `stream` has left it.
+  if ((rc = check_cuda(cudaEventRecord(ds.ev_entry, st)))) return rc;
+  if ((rc = check_cuda(cudaStreamWaitEvent(ds.copy_in, ds.ev_entry, 0)))) return rc;
+  // keys, gates and scales: small, ahead of the first chunk on the compute stream
   if ((rc = check_cuda(cudaMemcpyAsync(dk, kcache->data, (size_t)L * d * esz, cudaMemcpyHostToDevice, st)))) return rc;
+  if ((rc = check_cuda(cudaMemcpyAsync(dw, w, (size_t)L * H_I * 4, cudaMemcpyHostToDevice, st)))) return rc;
   if (fp8) {
-    if (!q->scale || !kcache->scale) return PIVOT_ERR_INVALID_ARG;
     if ((rc = check_cuda(cudaMemcpyAsync(dqs, q->scale, (size_t)L * H_I * 4, cudaMemcpyHostToDevice, st)))) return rc;
     if ((rc = check_cuda(cudaMemcpyAsync(dks, kcache->scale, (size_t)L * 4, cudaMemcpyHostToDevice, st)))) return rc;
   }
+  // queries: chunk by chunk on the copy-in stream
+  const size_t qrow = (size_t)H_I * d * esz;
+  for (int i = 0; i < n_chunks; ++i) {
+    const int r0 = i * chunk_rows, r1 = (r0 + chunk_rows < L) ? r0 + chunk_rows : L;
+    if ((rc = check_cuda(cudaMemcpyAsync(dq + (size_t)r0 * qrow, (const char*)q->data + (size_t)r0 * qrow,
+                                         (size_t)(r1 - r0) * qrow, cudaMemcpyHostToDevice, ds.copy_in))))
+      return rc;
+    if ((rc = check_cuda(cudaEventRecord(ds.ev_in[i], ds.copy_in)))) return rc;
+  }
   pivot_tensor tq{dq, fp8 ? dqs : nullptr, q->dtype};
   pivot_tensor tk{dk, fp8 ? dks : nullptr, q->dtype};
-  pivot_opts o;
-  memset(&o, 0, sizeof(o));
-  o.guard_len = -1;
-  o.workspace = dws;
-  o.workspace_bytes = arena_bytes - cv.off;
-  rc = pivot_index_prefill_ex(&tq, dw, &tk, L, H_I, d, g, c, k, mode, dout, stream, &o);
-  if (rc) return rc;
-  if ((rc = check_cuda(cudaMemcpyAsync(out_idx, dout, (size_t)L * k * 4, cudaMemcpyDeviceToHost, st)))) return rc;
-  return check_cuda(cudaStreamSynchronize(st));
+  for (int i = 0; i < n_chunks; ++i) {
+    const int r0 = i * chunk_rows, r1 = (r0 + chunk_rows < L) ? r0 + chunk_rows : L;
+    pivot_opts o;
+    memset(&o, 0, sizeof(o));
+    o.guard_len = -1;
+    o.workspace = dws;
+    o.workspace_bytes = arena_bytes - cv.off;
+    if (n_chunks > 1) { o.row_begin = r0; o.row_end = r1; }
+    if ((rc = check_cuda(cudaStreamWaitEvent(st, ds.ev_in[i], 0)))) return rc;
+    rc = pivot_index_prefill_ex(&tq, dw, &tk, L, H_I, d, g, c, k, mode, dout, stream, &o);
+    if (rc) return rc;
+    if ((rc = check_cuda(cudaEventRecord(ds.ev_done[i], st)))) return rc;
+    if ((rc = check_cuda(cudaStreamWaitEvent(ds.copy_out, ds.ev_done[i], 0)))) return rc;
+    if ((rc = check_cuda(cudaMemcpyAsync(out_idx + (size_t)r0 * k, dout + (size_t)r0 * k, (size_t)(r1 - r0) * k * 4,
+                                         cudaMemcpyDeviceToHost, ds.copy_out))))
+      return rc;
+  }
+  if ((rc = check_cuda(cudaStreamSynchronize(st)))) return rc;
+  return check_cuda(cudaStreamSynchronize(ds.copy_out));
 }
 
 int pivot_device_status(pivot_stream_t stream, int* status) {

@@ -52,7 +52,8 @@ struct PrefillPlan {
   int32_t* cand; float* cand_score;                     // [nP, c] (Refine)
   int32_t* out; float* out_score;                       // [L, k]
   int L, g, c, k, mode, dtype;
-  int n_dense;      // rows 0 .. n_dense-1 are scored densely (guarded groups or dense control)
+  int dense_begin;  // first densely scored row of this call
+  int n_dense;      // rows dense_begin .. dense_begin+n_dense-1 are scored densely (guarded groups or dense control)
   int first_group;  // first group taking the proxy path
   int n_proxy;      // groups on the proxy path
 };

@@ -35,19 +35,20 @@ __global__ void plan_prefill_kernel(PrefillPlan p, RowDesc* rows, GroupDesc* gro
   const size_t esz = p.dtype == DT_FP8 ? 1 : 2;
   const size_t qrow = (size_t)kHeads * kDim * esz;
   if (i < p.n_dense) {
+    const int t = p.dense_begin + i;      // query row (= position) of this dense row
     RowDesc r;
-    r.q = (const char*)p.q + (size_t)i * qrow;
-    r.w = p.w + (size_t)i * kHeads;
-    r.qscale = p.qscale ? p.qscale + (size_t)i * kHeads : nullptr;
+    r.q = (const char*)p.q + (size_t)t * qrow;
+    r.w = p.w + (size_t)t * kHeads;
+    r.qscale = p.qscale ? p.qscale + (size_t)t * kHeads : nullptr;
     r.kbase = p.kc;
     r.kscale = p.kscale;
-    r.n_vis = i + 1;
+    r.n_vis = t + 1;
     r.K = p.k;
-    r.out = p.out + (size_t)i * p.k;
-    r.out_score = p.out_score ? p.out_score + (size_t)i * p.k : nullptr;
+    r.out = p.out + (size_t)t * p.k;
+    r.out_score = p.out_score ? p.out_score + (size_t)t * p.k : nullptr;
     r.out_rows = 1;
     r.out_stride = p.k;
-    r.q_map = 0; r.q_row = i; r.k_row0 = 0;
+    r.q_map = 0; r.q_row = t; r.k_row0 = 0;
     rows[i] = r;
   } else if (i < p.n_dense + p.n_proxy) {
     const int pr = i - p.n_dense;

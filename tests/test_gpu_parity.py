@@ -132,3 +132,56 @@ def test_argument_errors(pv):
     with pytest.raises(pv.PivotError, match="workspace"):
         small = torch.empty(256, dtype=torch.uint8, device="cuda")
         pv.pivot_index_prefill(q, w, k, 64, 64, 128, 4, 16, 8, pv.REFINE, out, workspace=small)
+
+
+# ---------------------------------------------------------------- chunked prefill / host pipeline
+
+def _sorted_rows(a):
+    return np.sort(a, axis=1)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+@pytest.mark.parametrize("mode", [po.MODE_REUSE, po.MODE_REFINE])
+def test_prefill_row_ranges_match_whole_call(pv, dtype, mode):
+    """Chunks of query rows (row_begin / row_end) give the rows of one whole call: same sets
+    (the order inside a row is free), rows outside the chunk untouched."""
+    L, g, c, k = 1900, 4, 256, 64
+    x = inputs.make_prefill(L, dtype=dtype, seed=77)
+    q, w, kk = x.q.cuda(), x.w.cuda(), x.k.cuda()
+    sc = dict(q_scale=None if x.qscale is None else x.qscale.cuda(),
+              k_scale=None if x.kscale is None else x.kscale.cuda())
+    whole = torch.full((L, k), -7, dtype=torch.int32, device="cuda")
+    pv.pivot_index_prefill(q, w, kk, L, 64, 128, g, c, k, mode, whole, **sc)
+    parts = torch.full((L, k), -7, dtype=torch.int32, device="cuda")
+    bounds = [0, 128, 260, 1000, 1524, L]          # chunks inside, across and past the guardrail (c = 256)
+    for r0, r1 in zip(bounds[:-1], bounds[1:]):
+        before = parts.clone()
+        pv.pivot_index_prefill(q, w, kk, L, 64, 128, g, c, k, mode, parts, rows=(r0, r1), **sc)
+        torch.cuda.synchronize()
+        assert pv.pivot_device_status() == 0
+        untouched = torch.ones(L, dtype=torch.bool, device="cuda")
+        untouched[r0:r1] = False
+        assert torch.equal(parts[untouched], before[untouched])
+    assert np.array_equal(_sorted_rows(parts.cpu().numpy()), _sorted_rows(whole.cpu().numpy()))
+    for bad in [(2, 8), (0, 6), (8, 8), (0, L + 4), (-4, 8)]:
+        with pytest.raises(pv.PivotError, match="invalid"):
+            pv.pivot_index_prefill(q, w, kk, L, 64, 128, g, c, k, mode, parts, rows=bad, **sc)
+
+
+def test_prefill_host_pipeline_matches_device_call(pv):
+    """The host-buffer entry point (chunked copies overlapping the kernels) returns what the
+    device entry point returns for the same request; large enough for several chunks."""
+    L, g, c, k = 20000, 4, 512, 128
+    x = inputs.make_prefill(L, dtype="fp8", seed=5)
+    dev = torch.full((L, k), -7, dtype=torch.int32, device="cuda")
+    pv.pivot_index_prefill(x.q.cuda(), x.w.cuda(), x.k.cuda(), L, 64, 128, g, c, k, pv.REFINE, dev,
+                           q_scale=x.qscale.cuda(), k_scale=x.kscale.cuda())
+    torch.cuda.synchronize()
+    pin = lambda t: t.contiguous().pin_memory()
+    hq, hw, hk, hqs, hks = pin(x.q), pin(x.w), pin(x.k), pin(x.qscale), pin(x.kscale)
+    hout = torch.full((L, k), -7, dtype=torch.int32).pin_memory()
+    arena = torch.empty(pv.pivot_prefill_host_arena_bytes(L, 64, 128, g, c, k, pv.FP8_E4M3), dtype=torch.uint8, device="cuda")
+    for _ in range(2):          # second call: the arena and the copy streams are reused
+        hout.fill_(-7)
+        pv.pivot_index_prefill_host(hq, hw, hk, L, 64, 128, g, c, k, pv.REFINE, hout, arena, q_scale=hqs, k_scale=hks)
+        assert np.array_equal(_sorted_rows(hout.numpy()), _sorted_rows(dev.cpu().numpy()))
