@@ -7,7 +7,7 @@
 //                        tile) pairs; per tile: TMA -> tcgen05 MMA (128 keys x 64 heads x d) ->
 //                        epilogue (ReLU, gate-weighted head sum, key scale) -> one fp32 score per
 //                        key to an L2-resident score array (3 % of the bytes read), plus a
-//                        16384-bin histogram of the scores' top 14 key bits per sequence.
+//                        8192-bin histogram of the scores' top 13 key bits per sequence.
 //   decode_select_kernel one 1024-thread CTA per sequence: the histogram gives the bin holding
 //                        the K-th best score; if that leaves too many candidates the bin is
 //                        refined 12 bits at a time with further passes over the scores; the
