@@ -10,9 +10,17 @@
 // cut, and feeds the score to the row's streaming select (filter by the running K-th-best
 // threshold, append to an L2-resident candidate buffer, exact radix compaction when it fills).
 //
-// One persistent CTA per SM; warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner,
-// warps 2.. = epilogue (two warps per TMEM lane quarter, each pair of rows handled by its own
-// 128-thread team).  Row blocks are dealt to CTAs longest-first in snake order.
+// One persistent CTA per SM; warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, then the
+// SCORE warps (two per TMEM lane quarter, each computing two rows of a tile), then one APPEND
+// warp per row.  A score warp compares its 32 scores of a row with the row's published
+// threshold and leaves the survivors, compacted, in a small double-buffered shared-memory
+// queue; the row's append warp counts them in the row histogram, moves them to the row's
+// candidate segment (L2-resident scratch) and keeps the threshold fresh -- alone, without
+// barriers.  Splitting the epilogue this way puts more warps on every scheduler within the
+// register file (the score warps carry no select state) and takes the histogram atomics, the
+// global stores and the threshold refresh off the warps that feed the tensor core.  At the end
+// of a block the score-warp teams (128 threads per pair of rows) do the final exact select.
+// Row blocks are dealt to CTAs longest-first in snake order.
 #include <cuda.h>
 #include <string.h>
 
@@ -26,6 +34,7 @@ namespace {
 constexpr int TILE_KEYS = 128;
 constexpr int MAX_STAGES = 8;
 constexpr int KS_SLOTS = 12;      // key-scale ring: deeper than (key stages + accumulator buffers)
+constexpr int QDEPTH = 4;         // survivor-queue buffers between the score warps and the append warps
 
 template <int DT, int NROWS>
 struct Cfg {
@@ -40,17 +49,14 @@ struct Cfg {
   static constexpr int N = NROWS * kHeads;
   static constexpr int QBUFS = (!FP8 && NROWS == 4) ? 1 : 2;   // bf16 x 4 rows: 64 KB per query buffer
   static constexpr int STAGES = NROWS == 4 ? (FP8 ? 4 : 2) : (FP8 ? 6 : 4);
-  // Eight epilogue warps, two rows per 4-warp team (measured faster than one team per row with
-  // sixteen warps, which leaves only 96 registers per thread).
-#ifndef PIVOT_EPI16
+  // Eight score warps, two rows per 4-warp team (one team per row with sixteen warps leaves too
+  // few registers per thread), and one select warp per row.
   static constexpr int EPI_WARPS = NROWS == 4 ? 8 : 4;
   static constexpr int ROWS_PER_TEAM = NROWS == 4 ? 2 : 1;
-#else
-  static constexpr int EPI_WARPS = NROWS == 4 ? 16 : 4;
-  static constexpr int ROWS_PER_TEAM = 1;
-#endif
   static constexpr int TEAMS = EPI_WARPS / 4;
-  static constexpr int THREADS = 64 + EPI_WARPS * 32;
+  static constexpr int SEL_WARPS = NROWS;                     // append warps, one per row
+  static constexpr int RDV_THREADS = 128 + ROWS_PER_TEAM * 32; // a team plus the append warps of its rows
+  static constexpr int THREADS = 64 + (EPI_WARPS + SEL_WARPS) * 32;
   static constexpr int TMEM_COLS = 2 * N < 32 ? 32 : 2 * N;
   static constexpr int KSTEPS = 4;                            // 32 bytes of K per MMA
   static constexpr uint32_t IDESC = ptx::make_idesc(FP8 ? 0u : 1u, TILE_KEYS, N);
@@ -64,12 +70,17 @@ struct Ctrl {
   uint64_t full[MAX_STAGES], empty[MAX_STAGES];
   uint64_t q_full[2], q_empty[2], tmem_full[2], tmem_empty[2];
   uint64_t ks_full[KS_SLOTS];
+  uint64_t sc_full[QDEPTH], sc_empty[QDEPTH];     // survivor queues: score warps -> append warps
+  alignas(16) unsigned long long q[QDEPTH][NROWS][4][32];   // [tile % QDEPTH][row][lane quarter]: packed entries
+  alignas(16) uint32_t qn[QDEPTH][NROWS][4];                // their counts
+  volatile uint32_t thr[NROWS];         // published append threshold of each row (only grows)
+  int rowcnt[NROWS];                    // end of a block: entries held in the row's segment
+  int rowbase[NROWS];                   // ... the row histogram's anchor
+  uint32_t rowthr[NROWS];               // ... and the row's final threshold
   uint32_t tmem_base;
   int abort;
   int abort_code;         // device status to report besides a timed-out wait
-  int flag[4];            // row r: a candidate segment is nearly full
-  uint32_t rowmax[4];     // row r: largest score key of the first tile (anchors the histogram)
-  SegSelSmem sel[NROWS == 4 ? 4 : 1];
+  SegSelSmem sel[NROWS];  // one per select warp
 };
 
 template <int DT, int NROWS>
@@ -136,8 +147,13 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       ptx::mbar_init(&ct.tmem_empty[i], C::EPI_WARPS);
     }
     for (int i = 0; i < KS_SLOTS; ++i) ptx::mbar_init(&ct.ks_full[i], 1);
+    for (int i = 0; i < QDEPTH; ++i) {
+      ptx::mbar_init(&ct.sc_full[i], C::EPI_WARPS);
+      ptx::mbar_init(&ct.sc_empty[i], C::SEL_WARPS);
+    }
     ct.abort = 0;
     ct.abort_code = 0;
+    for (int r = 0; r < NROWS; ++r) ct.thr[r] = 0u;
     ptx::fence_barrier_init();
   }
   if (warp == 1) {
@@ -239,62 +255,27 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         ++blk;
       }
     }
-  } else {
-    // ------------------------------------------------------------------ epilogue + select
+  } else if (warp < 2 + C::EPI_WARPS) {
+    // ------------------------------------------------------------------ score warps
     const int ew = warp - 2;                       // 0 .. EPI_WARPS-1
     const int team = ew >> 2;                      // which pair of rows
-    const int wq = ew & 3;                         // warp inside the team = candidate segment
+    const int wq = ew & 3;
     const int lq = warp & 3;                       // TMEM lane quarter this warp may read
     const int key_in_tile = lq * 32 + lane;
     const int tt = wq * 32 + lane;                 // rank inside the team (0..127)
     const Team tm{tt, 128, 1 + team};
-    SegSelSmem& sel = ct.sel[team];
-    const int SEG = sc.cap >> 2;                   // entries per warp segment
-    const size_t cta_base = (size_t)blockIdx.x * NROWS * sc.cap;
-    auto seg_ptr = [&](int r) { return sc.cand64 + cta_base + ((size_t)r * 4 + wq) * SEG; };
-    // Score key -> histogram bin: 256 bins per octave (8 mantissa bits), 2048 bins anchored two
-    // octaves above the row's first-tile maximum; keys outside land in the end bins.
-    auto key_bin = [](uint32_t key, int base) {
-      const int b = (int)(key >> 15) - base;
-      return b < 0 ? 0 : (b > kSelBins - 1 ? kSelBins - 1 : b);
-    };
-    // Lower bound on the K-th best score seen so far, read off the row histogram: the largest
-    // bin edge with at least K scores at or above it.  Returned as a key threshold t such that
-    // only keys > t can still belong to the top K.
-    auto hist_threshold = [&](int r, int K, int base) -> uint32_t {   // warp-local, no barrier
-      uint32_t b, need_in, pop;
-      if (!warp_hist_boundary<false>(ct.rhist[r], (uint32_t)K, lane, &b, &need_in, &pop)) return 0u;
-      return b > 0 ? (((uint32_t)((int)b + base)) << 15) - 1u : 0u;
-    };
-    auto team_max = [&](int v) -> int {          // max of a warp-uniform value over the team
-      tm.sync();
-      if (tt == 0) sel.maxcnt = 0;
-      tm.sync();
-      if (lane == 0) atomicMax(&sel.maxcnt, (uint32_t)v);
-      tm.sync();
-      return (int)sel.maxcnt;
-    };
-    auto team_sum = [&](int v) -> int {          // sum of a warp-uniform value over the team
-      tm.sync();
-      if (tt == 0) sel.total = 0;
-      tm.sync();
-      if (lane == 0) atomicAdd(&sel.total, (uint32_t)v);
-      tm.sync();
-      return (int)sel.total;
-    };
+    const Team rdv{0, C::RDV_THREADS, 7 + team};   // this team and the append warps of its rows
+    const uint32_t lt_mask = (1u << lane) - 1u;
     BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
     uint32_t it = 0;
     // A failed wait never changes this role's control flow (the team barriers below must stay
     // matched); once the abort flag is up every later wait returns at once.
     for (int b = bi.next(); b >= 0; b = bi.next()) {
-      int k_row0 = 0, nv_max = 0;
-      const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0, &nv_max);
+      int k_row0 = 0;
+      const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0);
       if (ntiles == 0) continue;
-      // ---- per-block state of this team's rows
+      // ---- effective gates of this team's rows
       tm.sync();
-      const float* kscale = rows[b * NROWS].kscale;
-      int n_vis[C::ROWS_PER_TEAM], Ksel[C::ROWS_PER_TEAM], cnt[C::ROWS_PER_TEAM], base[C::ROWS_PER_TEAM];
-      uint32_t thr[C::ROWS_PER_TEAM];
       {
         const int rl = tt >> 6, j = tt & 63;
         if (rl < C::ROWS_PER_TEAM) {
@@ -305,59 +286,22 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             wv = rows[ri].w[j];
             if (rows[ri].qscale) wv = __fmul_rn(wv, rows[ri].qscale[j]);
           }
-          ct.w[r][j] = 0.5f * wv;       // halved: see the epilogue's ReLU identity
-          if (j == 0) { ct.flag[r] = 0; ct.rowmax[r] = 0; }
+          ct.w[r][j] = 0.5f * wv;       // halved: see the ReLU identity below
         }
       }
+      int n_vis[C::ROWS_PER_TEAM], Ksel[C::ROWS_PER_TEAM];
 #pragma unroll
       for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
-        const int r = team * C::ROWS_PER_TEAM + rl;
-        const int ri = b * NROWS + r;
+        const int ri = b * NROWS + team * C::ROWS_PER_TEAM + rl;
         const bool live = ri < n_rows && rows[ri].K > 0;
         n_vis[rl] = live ? rows[ri].n_vis : 0;
         Ksel[rl] = live ? rows[ri].K : 0;
-        cnt[rl] = 0; base[rl] = 0; thr[rl] = 0;
-        for (int i = tt; i < kSelBins; i += 128) ct.rhist[r][i] = 0;
       }
       tm.sync();
-      // The team meets only every CHK tiles (a barrier after an append waits for the store to
-      // land): that is when thresholds are refreshed and nearly full segments are dealt with,
-      // so a segment is flagged while it still has room for CHK tiles of appends.
-      const int CHK = SEG / 64 < 32 ? (SEG / 64 > 0 ? SEG / 64 : 1) : 32;
-      const int headroom = 32 * CHK;
       for (int t = 0; t < ntiles; ++t, ++it) {
-        const bool meet = (t % CHK) == 0 && t > 0;
-        if (meet) {
-          tm.sync();
-#pragma unroll
-          for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
-            if (Ksel[rl] > 0) {
-              const uint32_t th = hist_threshold(team * C::ROWS_PER_TEAM + rl, Ksel[rl], base[rl]);
-              thr[rl] = th > thr[rl] ? th : thr[rl];
-            }
-          }
-        }
-        // ---- a segment is nearly full: tighten the threshold and drop what fell below it;
-        //      if that is not enough (ties, adversarial order) compact exactly to the K best
-#pragma unroll
-        for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
-          const int r = team * C::ROWS_PER_TEAM + rl;
-          if (meet && ct.flag[r]) {
-            const uint32_t tcur = thr[rl];
-            cnt[rl] = seg_filter_inplace(seg_ptr(r), cnt[rl], lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
-            if (team_max(cnt[rl]) + headroom > SEG && team_sum(cnt[rl]) > Ksel[rl]) {
-              entry_t cut;
-              cnt[rl] = seg_compact<false>(tm, sel, Seg{seg_ptr(r), cnt[rl]}, Ksel[rl], &cut);
-              thr[rl] = entry_key(cut) > thr[rl] ? entry_key(cut) : thr[rl];
-            }
-            if (tt == 0) ct.flag[r] = 0;
-            tm.sync();
-          }
-        }
         const int buf = it & 1;
-        const int s_key = t * TILE_KEYS + key_in_tile;
-        // Key scales come through shared memory (TMA): a global load issued by an epilogue warp
-        // would sit in the same memory queue as its TMEM loads and stall them for an L2 round trip.
+        // Key scales come through shared memory (TMA): a global load issued by this warp would
+        // sit in the same memory queue as its TMEM loads and stall them for an L2 round trip.
         float ksv = 1.f;
         if (C::FP8) {
           const int ksl = it % KS_SLOTS;
@@ -389,13 +333,14 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             ap[3] = fmaf(fabsf(x3), wv.w, ap[3]); an[3] = fmaf(x3, wv.w, an[3]);
           }
         };
-        ptx::tmem_ld_32x32(tbase, va);
+        ptx::tmem_ld_32x32_async(tbase, va);
 #pragma unroll
         for (int c = 0; c < NCHUNK; ++c) {
-          ptx::tmem_wait_ld();                                  // chunk c has landed
+          if (c & 1) ptx::tmem_wait_ld_regs(vb);                // chunk c has landed
+          else ptx::tmem_wait_ld_regs(va);
           if (c + 1 < NCHUNK) {
-            if (c & 1) ptx::tmem_ld_32x32(tbase + (c + 1) * 32, va);
-            else ptx::tmem_ld_32x32(tbase + (c + 1) * 32, vb);
+            if (c & 1) ptx::tmem_ld_32x32_async(tbase + (c + 1) * 32, va);
+            else ptx::tmem_ld_32x32_async(tbase + (c + 1) * 32, vb);
           }
           if ((c & 1) == 0) {
 #pragma unroll
@@ -409,49 +354,26 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
-        // ---- count every score in the row histogram, append the ones above the threshold
-        uint32_t key[C::ROWS_PER_TEAM];
-        bool valid[C::ROWS_PER_TEAM];
-#pragma unroll
-        for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
-          key[rl] = score_to_key(C::FP8 ? score[rl] * ksv : score[rl]);
-          valid[rl] = s_key < n_vis[rl];
-        }
-        if (t == 0) {          // anchor the histogram range on the first tile's maximum
-#pragma unroll
-          for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
-            const uint32_t mx = __reduce_max_sync(0xffffffffu, valid[rl] ? key[rl] : 0u);
-            if (lane == 0) atomicMax(&ct.rowmax[team * C::ROWS_PER_TEAM + rl], mx);
-          }
-          tm.sync();
-#pragma unroll
-          for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
-            const int top = (int)(ct.rowmax[team * C::ROWS_PER_TEAM + rl] >> 15) + 512 - (kSelBins - 1);
-            base[rl] = top > 0 ? top : 0;
-          }
-        }
+        // ---- survivors of this warp's 32 keys (key scale applied, Appendix A) go to the row queues
+        const int qb = it % QDEPTH;
+        (void)ptx::mbar_wait(&ct.sc_empty[qb], ((it / QDEPTH) & 1) ^ 1, abort_flag);
+        const int s_key = t * TILE_KEYS + key_in_tile;
 #pragma unroll
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
           const int r = team * C::ROWS_PER_TEAM + rl;
-          // Only scores above the current threshold are counted: the ones at or below it can
-          // never reach a bin edge the threshold could still move to, so the counts that
-          // matter stay exact.
-          const bool take = valid[rl] && key[rl] > thr[rl];
-          if (take) atomicAdd(&ct.rhist[r][key_bin(key[rl], base[rl])], 1u);
+          const uint32_t key = score_to_key(C::FP8 ? score[rl] * ksv : score[rl]);
+          const bool take = s_key < n_vis[rl] && key > ct.thr[r];
           const uint32_t m = __ballot_sync(0xffffffffu, take);
-          if (take) {
-            const int p = cnt[rl] + __popc(m & ((1u << lane) - 1u));
-            if (p < SEG) seg_ptr(r)[p] = make_entry(key[rl], s_key);
-            else ct.abort_code = DEV_CAND_OVERFLOW;
-          }
-          cnt[rl] = min(cnt[rl] + __popc(m), SEG);
-          if (lane == 0 && cnt[rl] + headroom > SEG) ct.flag[r] = 1;
+          if (take) ct.q[qb][r][lq][__popc(m & lt_mask)] = make_entry(key, s_key);
+          if (lane == 0) ct.qn[qb][r][lq] = (uint32_t)__popc(m);
         }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&ct.sc_full[qb]);
       }
-      // ---- end of the block: final exact select per row, then pad / replicate.  The row
-      //      histogram is exact for every entry still held, so one pass over the segments
-      //      suffices; a boundary bin too crowded to rank takes the general path.
-      tm.sync();
+      // ---- end of the block: the team takes the final exact select of its rows.  The append
+      //      warps have counted every entry they hold, so the row histogram is exact and one pass
+      //      over the segment suffices; a boundary bin too crowded to rank takes the general path.
+      rdv.sync();                                  // append warps are done with the last tile
 #pragma unroll
       for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
         const int r = team * C::ROWS_PER_TEAM + rl;
@@ -459,15 +381,26 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         const int K = Ksel[rl];
         if (K <= 0) continue;
         const RowDesc rd = rows[ri];
-        const int rbase = base[rl];
-        int n_valid = seg_emit_hist(tm, sel, Seg{seg_ptr(r), cnt[rl]}, ct.rhist[r],
-                                    [&](uint32_t key) { return key_bin(key, rbase); }, rd.out, rd.out_score, K);
+        SegSelSmem& sel = ct.sel[r];               // the row's append warp is idle now
+        entry_t* const seg = sc.cand64 + ((size_t)blockIdx.x * NROWS + r) * sc.cap;
+        const int total = ct.rowcnt[r];
+        const int rbase = ct.rowbase[r];
+        const int lo = (int)(((long long)total * wq) >> 2), hi = (int)(((long long)total * (wq + 1)) >> 2);
+        int mine = hi - lo;                        // this warp's slice of the row segment
+        auto key_bin = [rbase](uint32_t key) {
+          const int bb = (int)(key >> 15) - rbase;
+          return bb < 0 ? 0 : (bb > kSelBins - 1 ? kSelBins - 1 : bb);
+        };
+        int n_valid = seg_emit_hist(tm, sel, Seg{seg + lo, mine}, ct.rhist[r], key_bin, rd.out, rd.out_score, K);
         if (n_valid < 0) {
-          const uint32_t th = hist_threshold(r, K, rbase);
-          const uint32_t tcur = th > thr[rl] ? th : thr[rl];
-          cnt[rl] = seg_filter_inplace(seg_ptr(r), cnt[rl], lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
-          const int n = team_sum(cnt[rl]);
-          n_valid = seg_emit<false>(tm, sel, Seg{seg_ptr(r), cnt[rl]}, n, rd.out, rd.out_score, K);
+          const uint32_t tcur = ct.rowthr[r];
+          mine = seg_filter_inplace(seg + lo, mine, lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
+          tm.sync();
+          if (tt == 0) sel.total = 0;
+          tm.sync();
+          if (lane == 0) atomicAdd(&sel.total, (uint32_t)mine);
+          tm.sync();
+          n_valid = seg_emit<false>(tm, sel, Seg{seg + lo, mine}, (int)sel.total, rd.out, rd.out_score, K);
         }
         for (int i = n_valid + tt; i < K; i += 128) {
           rd.out[i] = -1;
@@ -480,6 +413,104 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             if (rd.out_score) rd.out_score[(size_t)rr * rd.out_stride + i] = rd.out_score[i];
           }
       }
+      rdv.sync();                                  // rows' histograms and segments may be reused
+    }
+  } else {
+    // ------------------------------------------------------------------ append warps: one row each
+    const int r = warp - 2 - C::EPI_WARPS;
+    const Team tm{lane, 32, 3 + r};
+    const Team rdv{0, C::RDV_THREADS, 7 + r / C::ROWS_PER_TEAM};
+    SegSelSmem& sel = ct.sel[r];
+    const int CAP = sc.cap;                        // entries of this row's candidate segment
+    entry_t* const seg = sc.cand64 + ((size_t)blockIdx.x * NROWS + r) * CAP;
+    uint32_t* const rhist = ct.rhist[r];
+    // Score key -> histogram bin: 256 bins per octave (8 mantissa bits), 2048 bins anchored two
+    // octaves above the row's first-tile maximum; keys outside land in the end bins.
+    auto key_bin = [](uint32_t key, int base) {
+      const int b = (int)(key >> 15) - base;
+      return b < 0 ? 0 : (b > kSelBins - 1 ? kSelBins - 1 : b);
+    };
+    // Lower bound on the K-th best score seen so far, read off the row histogram: the largest
+    // bin edge with at least K scores at or above it.  Returned as a key threshold t such that
+    // only keys > t can still belong to the top K.
+    auto hist_threshold = [&](int K, int base) -> uint32_t {
+      uint32_t b, need_in, pop;
+      if (!warp_hist_boundary<2>(rhist, (uint32_t)K, lane, &b, &need_in, &pop)) return 0u;
+      return b > 0 ? (((uint32_t)((int)b + base)) << 15) - 1u : 0u;
+    };
+    // The threshold is refreshed every CHK tiles; a tile adds at most TILE_KEYS entries, so a
+    // segment checked then always has room until the next check.
+    const int CHK = CAP / (2 * TILE_KEYS) < 16 ? (CAP / (2 * TILE_KEYS) > 0 ? CAP / (2 * TILE_KEYS) : 1) : 16;
+    const int headroom = TILE_KEYS * CHK;
+    BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
+    uint32_t it = 0;
+    for (int b = bi.next(); b >= 0; b = bi.next()) {
+      int k_row0 = 0;
+      const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0);
+      if (ntiles == 0) continue;
+      const int ri = b * NROWS + r;
+      const bool live = ri < n_rows && rows[ri].K > 0;
+      const int K = live ? rows[ri].K : 0;
+      int cnt = 0, base = 0;
+      uint32_t thr = 0;
+      for (int i = lane; i < kSelBins; i += 32) rhist[i] = 0;
+      __syncwarp();
+      for (int t = 0; t < ntiles; ++t, ++it) {
+        if (K > 0 && t > 0 && (t % CHK) == 0) {
+          const uint32_t th = hist_threshold(K, base);
+          thr = th > thr ? th : thr;
+          if (cnt + headroom > CAP) {
+            // nearly full: drop what fell below the threshold; if that is not enough (ties,
+            // adversarial order) compact exactly to the K best
+            const uint32_t tcur = thr;
+            cnt = seg_filter_inplace(seg, cnt, lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
+            if (cnt + headroom > CAP && cnt > K) {
+              entry_t cut;
+              cnt = seg_compact<false>(tm, sel, Seg{seg, cnt}, K, &cut);
+              thr = entry_key(cut) > thr ? entry_key(cut) : thr;
+            }
+          }
+          if (lane == 0) ct.thr[r] = thr;
+        }
+        const int sb = it % QDEPTH;
+        (void)ptx::mbar_wait(&ct.sc_full[sb], (it / QDEPTH) & 1, abort_flag);
+        const uint4 n4 = *reinterpret_cast<const uint4*>(&ct.qn[sb][r][0]);
+        const uint32_t nq[4] = {n4.x, n4.y, n4.z, n4.w};
+        entry_t e[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) e[j] = (uint32_t)lane < nq[j] ? ct.q[sb][r][j][lane] : kPadEntry;
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&ct.sc_empty[sb]);
+        if (K <= 0) continue;                    // a dead row still takes part in the handshake
+        if (t == 0) {          // anchor the histogram range on the first tile's maximum
+          uint32_t mx = 0;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) mx = entry_key(e[j]) > mx ? entry_key(e[j]) : mx;
+          mx = __reduce_max_sync(0xffffffffu, mx);
+          const int top = (int)(mx >> 15) + 512 - (kSelBins - 1);
+          base = top > 0 ? top : 0;
+        }
+        // Every entry that reaches the segment is counted: the ones the score warps dropped were
+        // at or below a valid threshold and can never reach a bin edge the threshold could still
+        // move to, so the counts that matter stay exact.
+        int p = cnt + lane;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if ((uint32_t)lane < nq[j]) {
+            atomicAdd(&rhist[key_bin(entry_key(e[j]), base)], 1u);
+            if (p < CAP) seg[p] = e[j];
+            else ct.abort_code = DEV_CAND_OVERFLOW;
+          }
+          p += (int)nq[j];
+        }
+        cnt = min(cnt + (int)(nq[0] + nq[1] + nq[2] + nq[3]), CAP);
+      }
+      // ---- end of the block: hand the row to the team's final select, wait until it is done
+      if (lane == 0) { ct.rowcnt[r] = cnt; ct.rowbase[r] = base; ct.rowthr[r] = thr; }
+      __syncwarp();
+      rdv.sync();
+      if (lane == 0) ct.thr[r] = 0u;             // the next block starts from scratch (read after the barrier below)
+      rdv.sync();
     }
   }
   // ------------------------------------------------------------------ teardown
