@@ -46,7 +46,7 @@ H, D = 64, 128
 FLOP_PER_SCORE = 2 * H * D
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/ (same workloads as the ones timed here)
-TRAFFIC_BYTES = {"prefill_128k_fp8_refine_g4": 2489417984 + 4554478848,
+TRAFFIC_BYTES = {"prefill_128k_fp8_refine_g4": 2638740736 + 4181647360,
                  "decode_scan_kernel": 403583488 + 12487936}
 
 
@@ -233,6 +233,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--window", type=int, default=0, help="local window W of Appendix B (device-timed value only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
@@ -269,7 +270,8 @@ def main():
     stream = torch.cuda.current_stream()
 
     def step():
-        pv.pivot_index_prefill(dq, dw, dk, L, H, D, g, c, k, mode, out, stream, q_scale=dqs, k_scale=dks)
+        pv.pivot_index_prefill(dq, dw, dk, L, H, D, g, c, k, mode, out, stream, q_scale=dqs, k_scale=dks,
+                               W=args.window)
 
     def barrier():
         torch.cuda.synchronize()
@@ -358,7 +360,7 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "e4m3" if dtype == "fp8" else "bf16",
         "data": "synthetic",
         "config": {"workload": wl, "L": L, "H_I": H, "d": D, "g": g, "c": c, "k": k,
-                   "mode": "refine" if mode else "reuse", "operands": dtype, "proxy_groups": n_proxy,
+                   "mode": "refine" if mode else "reuse", "operands": dtype, "W": args.window, "proxy_groups": n_proxy,
                    "dense_rows": n_dense, "l2": "inputs larger than L2 (queries >= 1 GB per step)"
                    if L * H * D >= 2 ** 28 else "inputs smaller than L2; no flush"},
         "clocks": clocks.summary(), "gpu_launches": int(launches),

@@ -84,19 +84,23 @@ def check_selection(got_idx, scores, index, K, rtol, tally: Tally, what="", got_
 
 
 def check_group(x: dict, kd, kscale, members, *, c, k, mode, guard_len, out_idx, out_scores=None,
-                cand=None, cand_scores=None, q_rows=None, pool="mean") -> Tally:
-    """Checks one group's rows of out_idx ([m, k]) (and candidates [c]) against the oracle."""
+                cand=None, cand_scores=None, q_rows=None, pool="mean", W=0) -> Tally:
+    """Checks one group's rows of out_idx ([m, k]) (and candidates [c]) against the oracle.
+
+    With a local window (Appendix B, W > 0) the proxy part of the candidate set is checked
+    against the shortened scan, the window slots must hold t0-W+1 .. t0+m-1 in ascending order,
+    and every member is checked on the slots it may see (positions <= its own)."""
     rtol = RTOL[x["dtype"]]
     t = Tally()
     r = po.pivot_group(x, members, kd, kscale, c=c, k=k, mode=mode, guard_len=guard_len, pool=pool,
-                       q_rows=q_rows)
+                       q_rows=q_rows, W=W)
     m = len(r.members)
     if r.guarded:
         for i, tq in enumerate(r.members):
             check_selection(out_idx[i], r.member_scores[i], np.arange(tq + 1), k, rtol, t,
                             f"dense row t={tq}", None if out_scores is None else out_scores[i])
         return t
-    n0 = r.t0 + 1
+    n0 = r.t0 + 1 if W == 0 else max(r.t0 - W + 1, 0)      # keys the proxy scan ranks
     if mode == po.MODE_REUSE:
         for i, tq in enumerate(r.members):
             check_selection(out_idx[i], r.proxy_scores, np.arange(n0), k, rtol, t,
@@ -104,20 +108,28 @@ def check_group(x: dict, kd, kscale, members, *, c, k, mode, guard_len, out_idx,
             assert sorted(out_idx[i].tolist()) == sorted(out_idx[0].tolist()), "reuse rows must share one set"
         return t
     assert cand is not None, "Refine parity needs the candidate set"
-    check_selection(cand, r.proxy_scores, np.arange(n0), c, rtol, t, f"candidates t0={r.t0}", cand_scores)
-    C = np.asarray(cand[: min(c, n0)], dtype=np.int64)
+    w_g = W + m - 1 if W > 0 else 0
+    cp = c - w_g                                            # slots filled by the proxy scan
+    check_selection(cand[:cp], r.proxy_scores, np.arange(n0), cp, rtol, t, f"candidates t0={r.t0}",
+                    None if cand_scores is None else cand_scores[:cp])
+    C = np.asarray(cand[: min(cp, n0)], dtype=np.int64)
+    if w_g:
+        win = np.arange(max(r.t0 - W + 1, 0), r.t0 + m, dtype=np.int64)
+        got_win = np.asarray(cand[cp:], dtype=np.int64)
+        assert np.array_equal(got_win[got_win >= 0], win), f"window slots of group t0={r.t0}"
+        C = np.concatenate([C, win])
     rows = r.members if q_rows is None else np.asarray(q_rows)
     qs = None if x["qscale"] is None else x["qscale"][rows]
     qd, weff = po.member_operands(x["q"][rows], qs, x["w"][rows], x["dtype"])
     for i, tq in enumerate(r.members):
-        s, _, _ = po.refine_on_candidates(qd[i], weff[i], kd, kscale, C, k)
-        check_selection(out_idx[i], s, C, k, rtol, t, f"refine row t={tq}",
+        s, _, ok = po.refine_on_candidates(qd[i], weff[i], kd, kscale, C, k, t_member=int(tq) if w_g else None)
+        check_selection(out_idx[i], s[ok], C[ok], k, rtol, t, f"refine row t={tq}",
                         None if out_scores is None else out_scores[i])
     return t
 
 
 def check_prefill(x: dict, *, g, c, k, mode, guard_len, out_idx, out_scores=None, cand=None,
-                  cand_scores=None, groups=None, pool="mean") -> Tally:
+                  cand_scores=None, groups=None, pool="mean", W=0) -> Tally:
     L = x["q"].shape[0]
     kd = po.decode_operand(x["k"], x["dtype"])
     allg = po.prefill_groups(L, g)
@@ -128,7 +140,7 @@ def check_prefill(x: dict, *, g, c, k, mode, guard_len, out_idx, out_scores=None
             x, kd, x["kscale"], mem, c=c, k=k, mode=mode, guard_len=guard_len,
             out_idx=out_idx[mem], out_scores=None if out_scores is None else out_scores[mem],
             cand=None if cand is None else cand[gi],
-            cand_scores=None if cand_scores is None else cand_scores[gi], pool=pool))
+            cand_scores=None if cand_scores is None else cand_scores[gi], pool=pool, W=W))
     return total
 
 

@@ -36,7 +36,7 @@ class pivot_opts(C.Structure):
     _fields_ = [("guard_len", C.c_int), ("pool", C.c_int), ("dbg_cand", C.c_void_p),
                 ("dbg_scores", C.c_void_p), ("dbg_cand_scores", C.c_void_p),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("impl", C.c_int),
-                ("row_begin", C.c_int), ("row_end", C.c_int)]
+                ("row_begin", C.c_int), ("row_end", C.c_int), ("W", C.c_int)]
 
 
 class PivotError(RuntimeError):
@@ -106,12 +106,12 @@ def _stream(stream) -> int:
 IMPL_TENSOR_CORE, IMPL_CUDA_CORE = 0, 1
 
 
-def _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl=0, rows=None) -> pivot_opts:
+def _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl=0, rows=None, W=0) -> pivot_opts:
     p = lambda t: None if t is None else t.data_ptr()
     r0, r1 = (0, 0) if rows is None else rows
     return pivot_opts(-1 if guard_len is None else guard_len, pool, p(dbg_cand), p(dbg_scores),
                       p(dbg_cand_scores), p(workspace), 0 if workspace is None else workspace.numel(), impl,
-                      r0, r1)
+                      r0, r1, W)
 
 
 def pivot_workspace_bytes(rows: int, n_groups: int, c: int, k: int) -> int:
@@ -148,13 +148,14 @@ def ensure_workspace(rows: int, n_groups: int, c: int, k: int, device="cuda", ne
 
 def pivot_index_prefill(q, w, kcache, L, H_I, d, g, c, k, mode, out_idx, stream=None, *,
                         q_scale=None, k_scale=None, guard_len=None, pool=POOL_MEAN, dbg_cand=None,
-                        dbg_scores=None, dbg_cand_scores=None, workspace=None, impl=0, rows=None):
-    """rows=(row_begin, row_end) indexes just that chunk of query rows (chunked prefill)."""
+                        dbg_scores=None, dbg_cand_scores=None, workspace=None, impl=0, rows=None, W=0):
+    """rows=(row_begin, row_end) indexes just that chunk of query rows (chunked prefill); W is
+    the local window of Appendix B (0 = off)."""
     tq, tk = _tensor(q, q_scale), _tensor(kcache, k_scale)
     assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and out_idx.numel() >= L * k
     if workspace is None:
         ensure_workspace(L, (L + g - 1) // g, c, k, q.device)
-    o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl, rows)
+    o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl, rows, W)
     _check(lib.pivot_index_prefill_ex(C.byref(tq), w.data_ptr(), C.byref(tk), L, H_I, d, g, c, k, mode,
                                       out_idx.data_ptr(), _stream(stream), C.byref(o)))
     return out_idx

@@ -185,6 +185,10 @@ int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, i
     r0 = o->row_begin; r1 = o->row_end;
     if (r0 < 0 || r1 <= r0 || r1 > L || r0 % g || (r1 % g && r1 != L)) return PIVOT_ERR_INVALID_ARG;
   }
+  // local window (Appendix B): needs room in the candidate set and a scan of at least one key
+  const int W = (o && !dense_only) ? o->W : 0;
+  if (W < 0) return PIVOT_ERR_INVALID_ARG;
+  if (W > 0 && (W + g - 1 >= c || guard < W + g || (o && o->impl == 1))) return PIVOT_ERR_INVALID_ARG;
   const int g_begin = r0 / g, g_end = (r1 + g - 1) / g;
   const int dense0 = r0 < nd ? r0 : (int)nd;
   const int dense1 = r1 < nd ? r1 : (int)nd;
@@ -197,6 +201,7 @@ int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, i
   p.cand_score = (o && o->dbg_cand_scores) ? o->dbg_cand_scores + (size_t)pg0 * c : nullptr;
   p.out = out_idx; p.out_score = o ? o->dbg_scores : nullptr;
   p.L = L; p.g = g; p.c = c; p.k = k; p.mode = mode; p.dtype = q->dtype;
+  p.W = W;
   p.dense_begin = dense0;
   p.n_dense = dense1 - dense0;
   p.first_group = pg0;
@@ -287,7 +292,7 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
   if (!pos0 || B < 1 || g < 1 || Lmax < g) return PIVOT_ERR_INVALID_ARG;
   // every sequence's scale row must start on a 16-byte boundary (TMA reads it in 128-scale tiles)
   if (q->dtype == PIVOT_FP8_E4M3 && (Lmax & 3)) return PIVOT_ERR_INVALID_ARG;
-  if (o && (o->pool < 0 || o->pool > 2)) return PIVOT_ERR_INVALID_ARG;
+  if (o && (o->pool < 0 || o->pool > 2 || o->W != 0)) return PIVOT_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t base_bytes = pivot_workspace_bytes(B * g, B, c, k);
   const size_t need = base_bytes + decode_fast_bytes(B, Lmax, g, c);

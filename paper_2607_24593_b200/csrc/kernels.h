@@ -52,6 +52,7 @@ struct PrefillPlan {
   int32_t* cand; float* cand_score;                     // [nP, c] (Refine)
   int32_t* out; float* out_score;                       // [L, k]
   int L, g, c, k, mode, dtype;
+  int W;            // local window (Appendix B); 0 = off
   int dense_begin;  // first densely scored row of this call
   int n_dense;      // rows dense_begin .. dense_begin+n_dense-1 are scored densely (guarded groups or dense control)
   int first_group;  // first group taking the proxy path

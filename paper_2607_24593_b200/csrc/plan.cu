@@ -60,7 +60,9 @@ __global__ void plan_prefill_kernel(PrefillPlan p, RowDesc* rows, GroupDesc* gro
     r.qscale = nullptr;
     r.kbase = p.kc;
     r.kscale = p.kscale;
-    r.n_vis = t0 + 1;
+    // With a local window the proxy ranks s <= t0 - W only (Appendix B); the window itself is
+    // appended to the candidate set below.
+    r.n_vis = p.W > 0 ? max(t0 - p.W + 1, 0) : t0 + 1;
     r.q_map = 1; r.q_row = pr; r.k_row0 = 0;
     if (p.mode == 0) {   // Reuse: the proxy top-k goes to every member (Eq. 6)
       r.K = p.k;
@@ -69,8 +71,14 @@ __global__ void plan_prefill_kernel(PrefillPlan p, RowDesc* rows, GroupDesc* gro
       r.out_rows = m;
       r.out_stride = p.k;
     } else {             // Refine: top-c candidate set (Eq. 7)
-      r.K = p.c;
+      const int w_g = p.W > 0 ? p.W + m - 1 : 0;      // slots reserved for the window union
+      r.K = p.c - w_g;
       r.out = p.cand + (size_t)pr * p.c;
+      for (int j = 0; j < w_g; ++j) {                 // t0-W+1 .. t0+m-1, ascending
+        const int s = t0 - p.W + 1 + j;
+        p.cand[(size_t)pr * p.c + (p.c - w_g) + j] = s >= 0 ? s : -1;
+        if (p.cand_score) p.cand_score[(size_t)pr * p.c + (p.c - w_g) + j] = __int_as_float(0x7fc00000);
+      }
       r.out_score = p.cand_score ? p.cand_score + (size_t)pr * p.c : nullptr;
       r.out_rows = 1;
       r.out_stride = p.c;
@@ -81,7 +89,7 @@ __global__ void plan_prefill_kernel(PrefillPlan p, RowDesc* rows, GroupDesc* gro
       gd.kbase = p.kc;
       gd.kscale = p.kscale;
       gd.cand = r.out;
-      gd.n_cand = min(p.c, r.n_vis);
+      gd.n_cand = p.W > 0 ? p.c : min(p.c, r.n_vis);   // with a window every slot is read (pads are skipped)
       gd.m = m;
       gd.K = p.k;
       gd.first_pos = t0;

@@ -320,11 +320,13 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         for (int rl = 0; rl < 2; ++rl) {
           const int r = team * 2 + rl;
           const uint32_t key = score_to_key(gd.kscale ? score[rl] * ksv : score[rl]);
+          // a member never sees a key beyond its own position (only window slots can be: Appendix B)
+          const bool seen = idx >= 0 && idx <= gd.first_pos + r;
           if (smem_sel) {              // key only; the position is looked up again at the end
-            if (r < gd.m) skey[r * SCORE_SLOTS + slot] = idx >= 0 ? key : 0u;
+            if (r < gd.m) skey[r * SCORE_SLOTS + slot] = seen ? key : 0u;
             continue;
           }
-          const entry_t e = idx >= 0 ? make_entry(key, idx) : kPadEntry;
+          const entry_t e = seen ? make_entry(key, idx) : kPadEntry;
           if (gd.ent_out) {            // chunked mode: leave the entries for a later top-k
             if (r < gd.m && slot < gd.n_cand) gd.ent_out[(size_t)r * gd.ent_stride + gd.slot0 + slot] = e;
           } else if (r < gd.m && t * 32 + lane < SEG) {

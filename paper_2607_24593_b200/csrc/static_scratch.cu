@@ -69,7 +69,7 @@ extern "C" int dense_index_static(const pivot_tensor* q, const float* w, const p
   p.proxy_q = nullptr; p.proxy_w = nullptr; p.cand = nullptr; p.cand_score = nullptr;
   p.out = out_idx; p.out_score = nullptr;
   p.L = L; p.g = 1; p.c = k; p.k = k; p.mode = 0; p.dtype = q->dtype;
-  p.dense_begin = 0; p.n_dense = L; p.first_group = L; p.n_proxy = 0;
+  p.W = 0; p.dense_begin = 0; p.n_dense = L; p.first_group = L; p.n_proxy = 0;
   launch_plan_prefill(p, rows, nullptr, st);
 
   ScanScratch sc;

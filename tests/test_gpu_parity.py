@@ -185,3 +185,32 @@ def test_prefill_host_pipeline_matches_device_call(pv):
         hout.fill_(-7)
         pv.pivot_index_prefill_host(hq, hw, hk, L, 64, 128, g, c, k, pv.REFINE, hout, arena, q_scale=hqs, k_scale=hks)
         assert np.array_equal(_sorted_rows(hout.numpy()), _sorted_rows(dev.cpu().numpy()))
+
+
+# ---------------------------------------------------------------- local window (Appendix B)
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+@pytest.mark.parametrize("mode", [po.MODE_REUSE, po.MODE_REFINE])
+@pytest.mark.parametrize("g,W", [(4, 4), (8, 3), (3, 1)])
+def test_prefill_local_window_parity(pv, gu, dtype, mode, g, W):
+    """W > 0: shortened proxy scan, window slots at the end of the candidate set, per-member
+    causal mask over the window -- every group against the oracle's Appendix B steps."""
+    L, c, k = 1000 + g - 1, 256, 96          # short last group
+    x = inputs.make_prefill(L, dtype=dtype, seed=31)
+    out, scores, cand, cs = gu.run_prefill(x, g=g, c=c, k=k, mode=mode, W=W)
+    t = acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=None, out_idx=out, out_scores=scores,
+                          cand=cand, cand_scores=cs, W=W)
+    _report(f"window {dtype} mode={mode} g={g} W={W}", t)
+    assert t.rows > 0
+
+
+def test_local_window_argument_errors(pv):
+    x = inputs.make_prefill(256, dtype="bf16", seed=1)
+    q, w, k = x.q.cuda(), x.w.cuda(), x.k.cuda()
+    out = torch.empty((256, 8), dtype=torch.int32, device="cuda")
+    with pytest.raises(pv.PivotError, match="invalid"):
+        pv.pivot_index_prefill(q, w, k, 256, 64, 128, 4, 16, 8, pv.REFINE, out, W=13)        # W + g - 1 >= c
+    with pytest.raises(pv.PivotError, match="invalid"):
+        pv.pivot_index_prefill(q, w, k, 256, 64, 128, 4, 16, 8, pv.REFINE, out, W=4, guard_len=4)   # guardrail < W + g
+    with pytest.raises(pv.PivotError, match="invalid"):
+        pv.pivot_index_prefill(q, w, k, 256, 64, 128, 4, 16, 8, pv.REFINE, out, W=-1)

@@ -317,3 +317,35 @@ def test_decode_group_equals_prefill_group_on_same_tensors():
     b = po.pivot_prefill(x, g=g, c=12, k=6, mode=po.MODE_REFINE, groups=[p0 // g])[p0 // g]
     np.testing.assert_array_equal(a.T, b.T)
     np.testing.assert_array_equal(a.C, b.C)
+
+
+# ---------------------------------------------------------------- acceptance rule with a local window
+
+def test_acceptance_rule_with_window_accepts_the_oracle_and_rejects_mutations():
+    """The window form of the acceptance check (Appendix B) passes on the oracle's own output,
+    and fails when a window slot is wrong or a member selects a key beyond its own position."""
+    from oracle import acceptance as acc
+    from paper_2607_24593_b200 import inputs
+    L, g, c, k, W = 120, 4, 32, 12, 3
+    x = inputs.make_prefill(L, dtype="bf16", seed=3).codes()
+    res = po.pivot_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE, W=W)
+    out = np.full((L, k), -1, np.int32)
+    cand = np.full((len(res), c), -1, np.int32)
+    for gi, r in res.items():
+        out[r.members] = r.T
+        if r.C is not None:
+            cand[gi, : len(r.C)] = r.C
+    t = acc.check_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE, guard_len=None, out_idx=out, cand=cand, W=W)
+    assert t.rows > 0 and t.exact_rows == t.rows
+    gi = len(res) - 1                       # a group past the guardrail
+    r = res[gi]
+    assert not r.guarded
+    bad = cand.copy()
+    bad[gi, c - 1] -= 1                     # last window slot must be t0 + m - 1
+    with pytest.raises(AssertionError):
+        acc.check_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE, guard_len=None, out_idx=out, cand=bad, W=W, groups=[gi])
+    bad_out = out.copy()
+    first = int(r.members[0])
+    bad_out[first, 0] = first + 1           # a key the first member may not see
+    with pytest.raises(AssertionError):
+        acc.check_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE, guard_len=None, out_idx=bad_out, cand=cand, W=W, groups=[gi])
