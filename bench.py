@@ -146,27 +146,58 @@ def decode_bench(pv, dev, steps, warmup, pk):
     for _ in range(warmup):
         step()
     torch.cuda.synchronize()
-    times, scan_us = [], []
+
+    def timed(run, n):
+        ts = []
+        for _ in range(n):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            run()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return ts
+
     pv.pivot_launch_count_reset()
-    pv.pivot_stage_timing(True)
-    for _ in range(steps):
-        flush.fill_(1)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        step()
-        e1.record(stream)
-        torch.cuda.synchronize()
-        times.append(e0.elapsed_time(e1) * 1e3)
-        scan_us.append(pv.pivot_stage_times()["decode_scan"] * 1e3)    # events around the scan launch
-    pv.pivot_stage_timing(False)
+    times = timed(step, steps)                                         # the step as a caller launches it
     launches = pv.pivot_launch_count_reset()
+    scan_us = []
+    pv.pivot_stage_timing(True)                                        # extra steps with events around the scan launch
+    for _ in range(max(3, min(steps, 5))):
+        flush.fill_(1)
+        step()
+        torch.cuda.synchronize()
+        scan_us.append(pv.pivot_stage_times()["decode_scan"] * 1e3)
+    pv.pivot_stage_timing(False)
     assert pv.pivot_device_status() == 0
+    # the same step replayed from a CUDA graph (what a serving loop would do): launch gaps gone
+    graph_us, graph_note = None, None
+    try:
+        gstream = torch.cuda.Stream(device=dev)
+        gstream.wait_stream(stream)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(gstream):
+            gs = torch.cuda.current_stream()
+            pv.pivot_index_decode(q, w, kc, p0, B, Lmax, H, D, g, c, k, pv.REFINE, out, gs, q_scale=qs, k_scale=ks)
+            gs.synchronize()
+            with torch.cuda.graph(graph, stream=gstream):
+                pv.pivot_index_decode(q, w, kc, p0, B, Lmax, H, D, g, c, k, pv.REFINE, out,
+                                      torch.cuda.current_stream(), q_scale=qs, k_scale=ks)
+        stream.wait_stream(gstream)
+        torch.cuda.synchronize()
+        graph_us = float(np.median(timed(graph.replay, steps)))
+        assert pv.pivot_device_status() == 0
+    except Exception as e:                                              # capture refused: say why, keep the stream number
+        graph_note = f"{type(e).__name__}: {e}"[:200]
+        torch.cuda.synchronize()
     us = float(np.median(times))
     scan = float(np.mean(scan_us))
     n0 = (x.pos0.numpy().astype(np.int64) + 1)
     key_bytes = int(n0.sum()) * (D + 4)                      # e4m3 key + fp32 scale, read once per step
     return {"metric": "us per MTP decode step", "value": us, "unit": "us", "min_us": float(min(times)),
             "steps": steps, "higher_is_better": False, "gpu_launches_per_step": launches / max(steps, 1),
+            "graph_replay_us": graph_us, "graph_note": graph_note,
             "config": {"workload": "decode_mtp_b32_64k-128k_fp8_g2_refine", "B": B, "g": g, "c": c, "k": k,
                        "visible_keys": int(n0.sum()), "l2": "256 MB flush between steps"},
             # dominant kernel: the key-streaming scan; algorithmic bytes = visible keys x 132 B

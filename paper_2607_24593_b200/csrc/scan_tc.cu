@@ -138,6 +138,13 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
   const int lane = threadIdx.x & 31;
   const int n_blocks = (n_rows + NROWS - 1) / NROWS;
 
+  // A small launch whose rows are all dead (decode: no guarded sequence in the batch) leaves
+  // before any barrier or TMEM is set up.
+  if (n_rows <= (int)blockDim.x) {
+    const bool live = (int)threadIdx.x < n_rows && rows[threadIdx.x].K > 0 && rows[threadIdx.x].n_vis > 0;
+    if (!__syncthreads_or(live)) return;
+  }
+
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) { ptx::mbar_init(&ct.full[s], 1); ptx::mbar_init(&ct.empty[s], 1); }
     for (int i = 0; i < 2; ++i) {
