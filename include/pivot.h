@@ -80,9 +80,15 @@ typedef struct pivot_tensor {
  *                 and guarded rows Eq. 1.
  *   dbg_cand_scores optional [n_groups, c] fp32: proxy score (Eq. 5) of each dbg_cand entry.
  *   workspace     scratch of at least pivot_workspace_bytes(...) bytes, 256-byte aligned.
- *   impl          0: tensor-core kernels (tcgen05; the product path).  1: the plain CUDA-core
- *                 kernels that compute the same thing one key per thread -- a slow on-device
- *                 cross-check, not a fallback: nothing selects it automatically.
+ *   impl          0: tensor-core kernels (tcgen05; the product path).  In FP8 prefill the shared
+ *                 scan also takes the gate-weighted head sum of Eq. 5 on the tensor core: ReLU
+ *                 values rounded to bf16, gates carried as two bf16 terms, fp32 accumulation -- a
+ *                 relative score error of about 2^-9, inside the FP8 acceptance band.
+ *                 2: the same kernels with that head sum in fp32 FMAs (slower; the scores then
+ *                 differ from exact arithmetic by fp32 summation order only).
+ *                 1: the plain CUDA-core kernels that compute the same thing one key per thread
+ *                 -- a slow on-device cross-check, not a fallback: nothing selects it
+ *                 automatically.
  *   row_begin, row_end  prefill / dense only: index just the query rows row_begin .. row_end-1 of
  *                 the request (chunked prefill; the other rows of out_idx are left untouched).
  *                 Both 0 = all rows.  row_begin must be a multiple of g, row_end a multiple of g

@@ -103,7 +103,7 @@ def _stream(stream) -> int:
     return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
 
 
-IMPL_TENSOR_CORE, IMPL_CUDA_CORE = 0, 1
+IMPL_TENSOR_CORE, IMPL_CUDA_CORE, IMPL_TENSOR_CORE_FP32_HEAD_SUM = 0, 1, 2
 
 
 def _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl=0, rows=None, W=0) -> pivot_opts:

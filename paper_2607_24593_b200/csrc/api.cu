@@ -218,7 +218,8 @@ int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, i
     launch_scan_simt(ws.rows, p.n_dense + p.n_proxy, q->dtype, ws.scan, st);
   } else {
     ScanOperands op{kc->data, L, kc->scale, q->data, L, ws.proxy_q, p.n_proxy, q->dtype};
-    if ((rc = check_cuda(launch_scan_tc(op, ws.rows, p.n_dense + p.n_proxy, 4, tc_scratch(ws), sm_count(), st))))
+    if ((rc = check_cuda(launch_scan_tc(op, ws.rows, p.n_dense + p.n_proxy, 4, tc_scratch(ws), sm_count(), st,
+                                        o && o->impl == 2))))
       return rc;
   }
   mark(3, st);
@@ -260,7 +261,7 @@ int pivot_index_prefill_ex(const pivot_tensor* q, const float* w, const pivot_te
   int rc = check_common(q, w, kcache, H_I, d, c, k, mode, out_idx);
   if (rc) return rc;
   if (L < 1 || g < 1) return PIVOT_ERR_INVALID_ARG;
-  if (opts && (opts->pool < 0 || opts->pool > 2 || opts->impl < 0 || opts->impl > 1))
+  if (opts && (opts->pool < 0 || opts->pool > 2 || opts->impl < 0 || opts->impl > 2))
     return PIVOT_ERR_INVALID_ARG;
   return run_prefill(q, w, kcache, L, g, c, k, mode, false, out_idx, (cudaStream_t)stream, opts);
 }

@@ -98,8 +98,10 @@ struct ScanOperands {
   int dtype;
 };
 // rows_per_block consecutive scan rows share one key stream (4 in prefill, 1 in decode).
+// fp32_head_sum: keep the gate-weighted head sum in fp32 FMAs even where the tensor-core form
+// (FP8, four rows per block) is available.
 cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_rows, int rows_per_block,
-                           const ScanScratch& s, int sms, cudaStream_t st);
+                           const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum = false);
 
 cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
                              const ScanScratch& s, int sms, cudaStream_t st);

@@ -36,7 +36,9 @@ constexpr int MAX_STAGES = 8;
 constexpr int KS_SLOTS = 12;      // key-scale ring: deeper than (key stages + accumulator buffers)
 constexpr int QDEPTH = 4;         // survivor-queue buffers between the score warps and the append warps
 
-template <int DT, int NROWS>
+// EPI: 1 = the gate-weighted head sum runs on the tensor core where the configuration allows it
+// (FP8, four rows); 0 = fp32 FMA epilogue everywhere.
+template <int DT, int NROWS, int EPI = 1>
 struct Cfg {
   static constexpr bool FP8 = DT == DT_FP8;
   static constexpr int ESZ = FP8 ? 1 : 2;
@@ -58,21 +60,35 @@ struct Cfg {
   static constexpr int RDV_THREADS = 128 + ROWS_PER_TEAM * 32; // a team plus the append warps of its rows
   static constexpr int THREADS = 64 + (EPI_WARPS + SEL_WARPS) * 32;
   static constexpr int TMEM_COLS = 2 * N < 32 ? 32 : 2 * N;
+  // FP8, four rows: the gate-weighted head sum itself runs on the tensor core (see the kernel
+  // header).  Other configurations keep the fp32 FMA epilogue.
+  static constexpr bool MMA2 = FP8 && NROWS == 4 && EPI == 1;
+  static constexpr int QD = MMA2 ? 2 : QDEPTH;                 // survivor-queue depth
+  static constexpr int TMEM_EMPTY_ARRIVALS = MMA2 ? 4 : EPI_WARPS;
+  static constexpr int SC_FULL_ARRIVALS = MMA2 ? 4 : EPI_WARPS;
+  static constexpr uint32_t IDESC2 = ptx::make_idesc(1u, TILE_KEYS, 16);   // bf16 x bf16, N = 16
   static constexpr int KSTEPS = 4;                            // 32 bytes of K per MMA
   static constexpr uint32_t IDESC = ptx::make_idesc(FP8 ? 0u : 1u, TILE_KEYS, N);
 };
 
-template <int NROWS>
+template <int NROWS, bool MMA2>
 struct Ctrl {
+  static constexpr int QD = MMA2 ? 2 : QDEPTH;
+  // MMA2: the block's gate matrix W [16 x 256] bf16, K-major with 128-byte swizzle (4 slabs of 64
+  // columns, 16 rows x 128 B each): row r < 4 holds the bf16 head of row r's effective gates in
+  // columns 64 r .. 64 r + 63, row 4 + r the bf16 remainder (so the gates enter with 16 mantissa
+  // bits), everything else is zero.  B operand of the second MMA.
+  alignas(1024) uint8_t wmat[MMA2 ? 8192 : 16];
+  uint64_t a_ready[2], s_ready[2], w_ready;      // MMA2 handshakes (see the kernel)
   alignas(128) float ks[KS_SLOTS][TILE_KEYS];   // key scales of the tiles in flight (TMA destination)
   alignas(16) float w[4][kHeads];       // effective gates of the block's rows (read as float4)
   uint32_t rhist[NROWS][kSelBins];      // per row: histogram of every score seen so far
   uint64_t full[MAX_STAGES], empty[MAX_STAGES];
   uint64_t q_full[2], q_empty[2], tmem_full[2], tmem_empty[2];
   uint64_t ks_full[KS_SLOTS];
-  uint64_t sc_full[QDEPTH], sc_empty[QDEPTH];     // survivor queues: score warps -> append warps
-  alignas(16) unsigned long long q[QDEPTH][NROWS][4][32];   // [tile % QDEPTH][row][lane quarter]: packed entries
-  alignas(16) uint32_t qn[QDEPTH][NROWS][4];                // their counts
+  uint64_t sc_full[QD], sc_empty[QD];     // survivor queues: score warps -> append warps
+  alignas(16) unsigned long long q[QD][NROWS][4][32];   // [tile % QD][row][lane quarter]: packed entries
+  alignas(16) uint32_t qn[QD][NROWS][4];                // their counts
   volatile uint32_t thr[NROWS];         // published append threshold of each row (only grows)
   int rowcnt[NROWS];                    // end of a block: entries held in the row's segment
   int rowbase[NROWS];                   // ... the row histogram's anchor
@@ -83,11 +99,13 @@ struct Ctrl {
   SegSelSmem sel[NROWS];  // one per select warp
 };
 
-template <int DT, int NROWS>
+template <int DT, int NROWS, int EPI = 1>
 constexpr size_t smem_bytes() {
-  using C = Cfg<DT, NROWS>;
-  return 1024 + C::QBUFS * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(Ctrl<NROWS>);
+  using C = Cfg<DT, NROWS, EPI>;
+  return 1024 + C::QBUFS * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(Ctrl<NROWS, C::MMA2>);
 }
+static_assert(smem_bytes<DT_FP8, 4, 1>() <= 232448 && smem_bytes<DT_FP8, 4, 0>() <= 232448 &&
+              smem_bytes<DT_BF16, 4>() <= 232448, "shared memory budget");
 
 // Block sequence of one CTA: blocks sorted longest-first are dealt in snake order.
 struct BlockIter {
@@ -121,17 +139,19 @@ __device__ __forceinline__ int block_tiles(const RowDesc* rows, int n_rows, int 
   return (mx + TILE_KEYS - 1) / TILE_KEYS;
 }
 
-template <int DT, int NROWS>
-__global__ void __launch_bounds__(Cfg<DT, NROWS>::THREADS, 1)
+template <int DT, int NROWS, int EPI>
+__global__ void __launch_bounds__(Cfg<DT, NROWS, EPI>::THREADS, 1)
 scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q0,
                       const __grid_constant__ CUtensorMap tm_q1, const __grid_constant__ CUtensorMap tm_ks,
                       const RowDesc* __restrict__ rows, int n_rows, ScanScratch sc) {
-  using C = Cfg<DT, NROWS>;
+  using C = Cfg<DT, NROWS, EPI>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* qbuf = smem;                                   // QBUFS x QBUF_BYTES
   uint8_t* kring = smem + C::QBUFS * C::QBUF_BYTES;       // STAGES x STAGE_BYTES
-  Ctrl<NROWS>& ct = *reinterpret_cast<Ctrl<NROWS>*>(kring + C::STAGES * C::STAGE_BYTES);
+  using CtrlT = Ctrl<NROWS, C::MMA2>;
+  CtrlT& ct = *reinterpret_cast<CtrlT*>(kring + C::STAGES * C::STAGE_BYTES);
+  constexpr int QD = C::QD;
   volatile int* abort_flag = &ct.abort;
 
   const int warp = threadIdx.x >> 5;
@@ -151,11 +171,14 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       ptx::mbar_init(&ct.q_full[i], 1);
       ptx::mbar_init(&ct.q_empty[i], 1);
       ptx::mbar_init(&ct.tmem_full[i], 1);
-      ptx::mbar_init(&ct.tmem_empty[i], C::EPI_WARPS);
+      ptx::mbar_init(&ct.tmem_empty[i], C::TMEM_EMPTY_ARRIVALS);
+      ptx::mbar_init(&ct.a_ready[i], 4);
+      ptx::mbar_init(&ct.s_ready[i], 1);
     }
+    ptx::mbar_init(&ct.w_ready, 1);
     for (int i = 0; i < KS_SLOTS; ++i) ptx::mbar_init(&ct.ks_full[i], 1);
-    for (int i = 0; i < QDEPTH; ++i) {
-      ptx::mbar_init(&ct.sc_full[i], C::EPI_WARPS);
+    for (int i = 0; i < QD; ++i) {
+      ptx::mbar_init(&ct.sc_full[i], C::SC_FULL_ARRIVALS);
       ptx::mbar_init(&ct.sc_empty[i], C::SEL_WARPS);
     }
     ct.abort = 0;
@@ -167,6 +190,8 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     ptx::tmem_alloc(&ct.tmem_base, C::TMEM_COLS);
     ptx::tmem_relinquish();
   }
+  if constexpr (C::MMA2)        // off-diagonal blocks and rows 4..15 of the gate matrix stay zero
+    for (int i = threadIdx.x; i < 8192 / 16; i += blockDim.x) reinterpret_cast<uint4*>(ct.wmat)[i] = make_uint4(0, 0, 0, 0);
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
@@ -228,6 +253,29 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
       uint32_t it = 0, blk = 0;
       bool ok = true;
+      // MMA2: the gate-weighted head sum of tile it-1, S[128 keys x 16] = ReLU(X)[128 x 256] . W^T,
+      // is issued right after the first MMA of tile it (its operand -- the accumulator turned into
+      // bf16 ReLU values in place -- is produced while that MMA runs).
+      bool pend = false;
+      uint32_t pend_it = 0, pend_blk = 0, w_blk = 0xffffffffu;
+      auto issue_mma2 = [&]() -> bool {
+        if (pend_blk != w_blk) {                 // first tile of a block: its gate matrix must be in place
+          if (!ptx::mbar_wait(&ct.w_ready, pend_blk & 1, abort_flag, 32)) return false;
+          w_blk = pend_blk;
+        }
+        const int pb = pend_it & 1;
+        if (!ptx::mbar_wait(&ct.a_ready[pb], (pend_it >> 1) & 1, abort_flag, 32)) return false;
+        ptx::tc_fence_after();
+        const uint32_t w_addr = ptx::smem_u32(ct.wmat);
+        const uint32_t a_tmem = tmem_base + pb * C::N;
+#pragma unroll
+        for (int ks = 0; ks < 16; ++ks)          // 16 bf16 of K per step: 8 TMEM columns, 32 bytes of W
+          ptx::tc_mma_a_tmem_bf16(a_tmem + 128, a_tmem + ks * 8,
+                                  ptx::smem_desc_sw128(w_addr + (ks >> 2) * 2048 + (ks & 3) * 32), C::IDESC2,
+                                  ks ? 1u : 0u);
+        ptx::tc_commit(&ct.s_ready[pb]);
+        return true;
+      };
       for (int b = bi.next(); b >= 0 && ok; b = bi.next()) {
         int k_row0 = 0;
         const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0);
@@ -257,9 +305,16 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             }
           ptx::tc_commit(&ct.empty[s]);       // key stage free once these MMAs are done
           ptx::tc_commit(&ct.tmem_full[buf]); // accumulator ready
+          if constexpr (C::MMA2) {
+            if (pend) { ok = issue_mma2(); if (!ok) break; }
+            pend = true; pend_it = it; pend_blk = blk;
+          }
         }
         ptx::tc_commit(&ct.q_empty[qb]);
         ++blk;
+      }
+      if constexpr (C::MMA2) {
+        if (pend && ok) (void)issue_mma2();
       }
     }
   } else if (warp < 2 + C::EPI_WARPS) {
@@ -283,7 +338,31 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       if (ntiles == 0) continue;
       // ---- effective gates of this team's rows
       tm.sync();
-      {
+      if constexpr (C::MMA2) {
+        // team 1 (the compact warps) writes the four diagonal blocks of the gate matrix; the last
+        // second MMA of the previous block is through (its scores have been read)
+        if (team == 1) {
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int i = tt + u * 128, r = i >> 6, j = i & 63;
+            const int ri = b * NROWS + r;
+            float wv = 0.f;
+            if (ri < n_rows && rows[ri].K > 0) {
+              wv = rows[ri].w[j];
+              if (rows[ri].qscale) wv = __fmul_rn(wv, rows[ri].qscale[j]);
+            }
+            // gate = hi + lo in bf16: matrix rows r and 4 + r (both inside slab r, the row's 64 columns)
+            const __nv_bfloat16 hi = __float2bfloat16_rn(wv);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(wv - __bfloat162float(hi));
+            const uint32_t in_row = (j & 7) * 2;
+            *reinterpret_cast<__nv_bfloat16*>(ct.wmat + r * 2048 + r * 128 + (((j >> 3) ^ (r & 7)) << 4) + in_row) = hi;
+            *reinterpret_cast<__nv_bfloat16*>(ct.wmat + r * 2048 + (4 + r) * 128 + (((j >> 3) ^ ((4 + r) & 7)) << 4) + in_row) = lo;
+          }
+          ptx::fence_proxy_async_smem();         // generic-proxy writes -> tensor-core reads
+          tm.sync();
+          if (tt == 0) ptx::mbar_arrive(&ct.w_ready);
+        }
+      } else {
         const int rl = tt >> 6, j = tt & 63;
         if (rl < C::ROWS_PER_TEAM) {
           const int r = team * C::ROWS_PER_TEAM + rl;
@@ -305,6 +384,83 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         Ksel[rl] = live ? rows[ri].K : 0;
       }
       tm.sync();
+      if constexpr (C::MMA2) {
+        if (team == 0) {
+          // ---- ReLU warps: turn the fp32 accumulator into bf16 ReLU values in place.  Thread =
+          // key (TMEM lane); 32 columns at a time come in, 16 packed columns go back to the start
+          // of the buffer (writes trail the reads: column 16 c + 16 <= 32 c + 32).
+          // Rows missing from a partial block have no queries in shared memory: whatever the first
+          // MMA made of the stale bytes there (possibly NaN) must not reach the second one, whose
+          // sums run over all 256 columns -- those columns are written as zeros.
+          const int present = n_rows - b * NROWS;
+          for (int t = 0; t < ntiles; ++t, ++it) {
+            const int buf = it & 1;
+            (void)ptx::mbar_wait(&ct.tmem_full[buf], (it >> 1) & 1, abort_flag);
+            ptx::tc_fence_after();
+            const uint32_t xb = tmem_base + ((uint32_t)(lq * 32) << 16) + buf * C::N;
+            uint32_t va[32], vb[32];
+            ptx::tmem_ld_32x32_async(xb, va);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              if (c & 1) ptx::tmem_wait_ld_regs(vb);
+              else ptx::tmem_wait_ld_regs(va);
+              if (c + 1 < 8) {
+                if (c & 1) ptx::tmem_ld_32x32_async(xb + (c + 1) * 32, va);
+                else ptx::tmem_ld_32x32_async(xb + (c + 1) * 32, vb);
+              }
+              uint32_t pk[16];
+              const bool have_row = (c >> 1) < present;        // chunk c holds heads of row c / 2
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                pk[i] = (c & 1) ? ptx::relu_pack_bf16x2(__uint_as_float(vb[2 * i]), __uint_as_float(vb[2 * i + 1]))
+                                : ptx::relu_pack_bf16x2(__uint_as_float(va[2 * i]), __uint_as_float(va[2 * i + 1]));
+                pk[i] = have_row ? pk[i] : 0u;
+              }
+              ptx::tmem_st_32x16(xb + c * 16, pk);
+            }
+            ptx::tmem_wait_st();
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&ct.a_ready[buf]);
+          }
+        } else {
+          // ---- compact warps: read the four row scores of this thread's key, free the
+          // accumulator buffer, leave the survivors in the row queues
+          int nv4[NROWS];
+#pragma unroll
+          for (int r = 0; r < NROWS; ++r) {
+            const int ri = b * NROWS + r;
+            nv4[r] = (ri < n_rows && rows[ri].K > 0) ? rows[ri].n_vis : 0;
+          }
+          for (int t = 0; t < ntiles; ++t, ++it) {
+            const int buf = it & 1;
+            const int ksl = it % KS_SLOTS;
+            (void)ptx::mbar_wait(&ct.ks_full[ksl], (it / KS_SLOTS) & 1, abort_flag);
+            const float ksv = ct.ks[ksl][key_in_tile];
+            (void)ptx::mbar_wait(&ct.s_ready[buf], (it >> 1) & 1, abort_flag);
+            ptx::tc_fence_after();
+            uint32_t sv[8];          // columns r: sum with the gates' bf16 heads, 4 + r: with their remainders
+            ptx::tmem_ld_32x8(tmem_base + ((uint32_t)(lq * 32) << 16) + buf * C::N + 128, sv);
+            ptx::tmem_wait_ld();
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
+            const int qb = it % QD;
+            (void)ptx::mbar_wait(&ct.sc_empty[qb], ((it / QD) & 1) ^ 1, abort_flag);
+            const int s_key = t * TILE_KEYS + key_in_tile;
+#pragma unroll
+            for (int r = 0; r < NROWS; ++r) {
+              const uint32_t key = score_to_key((__uint_as_float(sv[r]) + __uint_as_float(sv[4 + r])) * ksv);
+              const bool take = s_key < nv4[r] && key > ct.thr[r];
+              const uint32_t m = __ballot_sync(0xffffffffu, take);
+              if (take) ct.q[qb][r][lq][__popc(m & lt_mask)] = make_entry(key, s_key);
+              if (lane == 0) ct.qn[qb][r][lq] = (uint32_t)__popc(m);
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&ct.sc_full[qb]);
+          }
+        }
+      } else
       for (int t = 0; t < ntiles; ++t, ++it) {
         const int buf = it & 1;
         // Key scales come through shared memory (TMA): a global load issued by this warp would
@@ -362,8 +518,8 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
         // ---- survivors of this warp's 32 keys (key scale applied, Appendix A) go to the row queues
-        const int qb = it % QDEPTH;
-        (void)ptx::mbar_wait(&ct.sc_empty[qb], ((it / QDEPTH) & 1) ^ 1, abort_flag);
+        const int qb = it % QD;
+        (void)ptx::mbar_wait(&ct.sc_empty[qb], ((it / QD) & 1) ^ 1, abort_flag);
         const int s_key = t * TILE_KEYS + key_in_tile;
 #pragma unroll
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
@@ -479,8 +635,8 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
           }
           if (lane == 0) ct.thr[r] = thr;
         }
-        const int sb = it % QDEPTH;
-        (void)ptx::mbar_wait(&ct.sc_full[sb], (it / QDEPTH) & 1, abort_flag);
+        const int sb = it % QD;
+        (void)ptx::mbar_wait(&ct.sc_full[sb], (it / QD) & 1, abort_flag);
         const uint4 n4 = *reinterpret_cast<const uint4*>(&ct.qn[sb][r][0]);
         const uint32_t nq[4] = {n4.x, n4.y, n4.z, n4.w};
         entry_t e[4];
@@ -531,13 +687,13 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
 
 // ---------------------------------------------------------------------------- host side
 
-template <int DT, int NROWS>
+template <int DT, int NROWS, int EPI = 1>
 cudaError_t launch_one(const CUtensorMap& mk, const CUtensorMap& mq0, const CUtensorMap& mq1, const CUtensorMap& mks,
                        const RowDesc* rows, int n_rows, const ScanScratch& s, int sms, cudaStream_t st) {
-  using C = Cfg<DT, NROWS>;
-  auto kern = scan_select_tc_kernel<DT, NROWS>;
+  using C = Cfg<DT, NROWS, EPI>;
+  auto kern = scan_select_tc_kernel<DT, NROWS, EPI>;
   static bool attr_set = false;
-  const size_t smem = smem_bytes<DT, NROWS>();
+  const size_t smem = smem_bytes<DT, NROWS, EPI>();
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -598,7 +754,7 @@ bool make_scale_map(CUtensorMap* m, const float* base, long long n) {
 
 
 cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_rows, int rows_per_block,
-                           const ScanScratch& s, int sms, cudaStream_t st) {
+                           const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum) {
   if (n_rows <= 0) return cudaSuccess;
   CUtensorMap mk, mq0, mq1, mks;
   memset(&mks, 0, sizeof(mks));
@@ -608,8 +764,9 @@ cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_ro
       !make_operand_map(&mq1, op.proxy_q, (long long)(op.proxy_rows > 0 ? op.proxy_rows : 1) * kHeads, op.dtype, kHeads))
     return cudaErrorInvalidValue;
   if (op.dtype == DT_FP8) {
-    return rows_per_block == 4 ? launch_one<DT_FP8, 4>(mk, mq0, mq1, mks, rows, n_rows, s, sms, st)
-                               : launch_one<DT_FP8, 1>(mk, mq0, mq1, mks, rows, n_rows, s, sms, st);
+    if (rows_per_block != 4) return launch_one<DT_FP8, 1>(mk, mq0, mq1, mks, rows, n_rows, s, sms, st);
+    return fp32_head_sum ? launch_one<DT_FP8, 4, 0>(mk, mq0, mq1, mks, rows, n_rows, s, sms, st)
+                         : launch_one<DT_FP8, 4, 1>(mk, mq0, mq1, mks, rows, n_rows, s, sms, st);
   }
   return rows_per_block == 4 ? launch_one<DT_BF16, 4>(mk, mq0, mq1, mks, rows, n_rows, s, sms, st)
                              : launch_one<DT_BF16, 1>(mk, mq0, mq1, mks, rows, n_rows, s, sms, st);

@@ -13,7 +13,7 @@ def to_cuda(x):
     return d
 
 
-def run_prefill(x, *, g, c, k, mode, guard_len=None, pool=pv.POOL_MEAN, debug=True, W=0):
+def run_prefill(x, *, g, c, k, mode, guard_len=None, pool=pv.POOL_MEAN, debug=True, W=0, impl=0):
     d = to_cuda(x)
     L, H, dd = x.q.shape
     nG = (L + g - 1) // g
@@ -23,7 +23,7 @@ def run_prefill(x, *, g, c, k, mode, guard_len=None, pool=pv.POOL_MEAN, debug=Tr
     cs = torch.full((nG, c), float("nan"), dtype=torch.float32, device="cuda") if cand is not None else None
     pv.pivot_index_prefill(d["q"], d["w"], d["k"], L, H, dd, g, c, k, mode, out, q_scale=d["qscale"],
                            k_scale=d["kscale"], guard_len=guard_len, pool=pool, dbg_cand=cand,
-                           dbg_scores=scores, dbg_cand_scores=cs, W=W)
+                           dbg_scores=scores, dbg_cand_scores=cs, W=W, impl=impl)
     torch.cuda.synchronize()
     assert pv.pivot_device_status() == 0
     f = lambda t: None if t is None else t.cpu().numpy()
