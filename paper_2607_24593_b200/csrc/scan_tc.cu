@@ -603,7 +603,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     };
     // The threshold is refreshed every CHK tiles; a tile adds at most TILE_KEYS entries, so a
     // segment checked then always has room until the next check.
-    const int CHK = CAP / (2 * TILE_KEYS) < 16 ? (CAP / (2 * TILE_KEYS) > 0 ? CAP / (2 * TILE_KEYS) : 1) : 16;
+    const int CHK = CAP / (2 * TILE_KEYS) < 32 ? (CAP / (2 * TILE_KEYS) > 0 ? CAP / (2 * TILE_KEYS) : 1) : 32;
     const int headroom = TILE_KEYS * CHK;
     BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
     uint32_t it = 0;
