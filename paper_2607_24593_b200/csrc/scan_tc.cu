@@ -21,6 +21,14 @@
 // global stores and the threshold refresh off the warps that feed the tensor core.  At the end
 // of a block the score-warp teams (128 threads per pair of rows) do the final exact select.
 // Row blocks are dealt to CTAs longest-first in snake order.
+//
+// FP8 with four rows per block (the prefill configuration) takes the gate-weighted head sum of
+// Eq. 5 on the tensor core as well: it is the contraction ReLU(X) [128 keys x 256] . W^T with a
+// block-diagonal gate matrix W [16 x 256].  The eight score warps then split into four ReLU
+// warps, which turn the fp32 accumulator into packed bf16 ReLU values in place in tensor memory,
+// and four compact warps, which read the row scores the second MMA (A operand in tensor memory,
+// W in shared memory) leaves in 16 columns of the same buffer.  The fp32 FMA head sum remains for
+// bf16 operands, one-row blocks and on request.
 #include <cuda.h>
 #include <string.h>
 
