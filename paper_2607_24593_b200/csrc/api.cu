@@ -226,7 +226,8 @@ int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, i
   if (mode == PIVOT_REFINE) {
     const int nd = p.n_proxy * group_chunks(g);
     if (o && o->impl == 1) launch_refine_simt(ws.groups, nd, q->dtype, ws.scan, st);
-    else if ((rc = check_cuda(launch_refine_tc(q->data, L, q->dtype, ws.groups, nd, tc_scratch(ws), sm_count(), st))))
+    else if ((rc = check_cuda(launch_refine_tc(q->data, L, q->dtype, ws.groups, nd, tc_scratch(ws), sm_count(), st,
+                                               o && o->impl == 2))))
       return rc;
   }
   mark(4, st);

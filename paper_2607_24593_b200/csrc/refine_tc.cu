@@ -28,7 +28,8 @@ constexpr int THREADS = (2 + GATHER_WARPS + EPI_WARPS) * 32;   // 384: 168 regis
 constexpr int N = NMEM * kHeads;
 constexpr int TMEM_COLS = 2 * N;
 
-template <int DT>
+// EPI: 1 = tensor-core head sum where available (FP8), 0 = fp32 FMA head sum.
+template <int DT, int EPI = 1>
 struct RCfg {
   static constexpr bool FP8 = DT == DT_FP8;
   static constexpr int KHALVES = FP8 ? 1 : 2;
@@ -48,9 +49,16 @@ struct RCfg {
   static constexpr int LOOKAHEAD = FP8 ? 4 : 1;   // gather tiles in flight per producer thread
   static constexpr int ROW_BYTES = FP8 ? 128 : 256;
   static constexpr uint32_t IDESC = ptx::make_idesc(FP8 ? 0u : 1u, TILE_KEYS, N);
+  // FP8: the gate-weighted head sum of Eq. 8 runs on the tensor core, as in the shared scan (a
+  // second MMA over bf16 ReLU values written in place in tensor memory against a block-diagonal
+  // gate matrix).  bf16 operands keep the fp32 FMA head sum.
+  static constexpr bool MMA2 = FP8 && EPI == 1;
+  static constexpr uint32_t IDESC2 = ptx::make_idesc(1u, TILE_KEYS, 16);
+  static constexpr int TMEM_EMPTY_ARRIVALS = MMA2 ? 4 : EPI_WARPS;
 };
 
-constexpr int META_SLOTS = MAX_STAGES + 3;    // deeper than (key stages + accumulator buffers)
+constexpr int META_SLOTS = 8;     // key stages in flight (<= 6) + accumulator buffers (2)
+static_assert(META_SLOTS >= 6 + 2, "meta ring");
 constexpr int SCORE_SLOTS = 4096;             // shared-memory score row: candidates per member
 
 // What the epilogue needs to know about a gathered key: its position and scale.
@@ -59,8 +67,18 @@ struct KeyMeta {
   float ks;      // key scale (1 for bf16)
 };
 
-struct RCtrl {
-  alignas(16) float w[NMEM][kHeads];
+// MMA2: the group's gate matrix, bf16, K-major with 128-byte swizzle, in the compact form the
+// second MMA reads: 4 slabs (64 columns each) of 8 rows x 128 B -- row r = bf16 head of member r's
+// effective gates (in slab r only), row 4 + r = their bf16 remainder -- followed by one 1 KB block
+// of zeros that serves as rows 8..15 of every slab (the descriptor's stride between the two 8-row
+// groups is set per slab).
+constexpr int WMAT_BYTES = 5120;
+
+template <bool MMA2>
+struct RCtrlT {
+  alignas(1024) uint8_t wmat[MMA2 ? WMAT_BYTES : 16];
+  uint64_t a_ready[2], s_ready[2], w_ready;      // MMA2 handshakes
+  alignas(16) float w[MMA2 ? 1 : NMEM][kHeads];
   KeyMeta meta[META_SLOTS][TILE_KEYS];   // written by the gather warps, read by the epilogue
   uint64_t full[MAX_STAGES], empty[MAX_STAGES];
   uint64_t q_full[2], q_empty[2], tmem_full[2], tmem_empty[2];
@@ -69,13 +87,14 @@ struct RCtrl {
   SegSelSmem sel[2];
 };
 
-template <int DT>
+template <int DT, int EPI = 1>
 constexpr size_t rsmem_bytes() {
-  using C = RCfg<DT>;
-  return 1024 + C::QBUFS * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(RCtrl) +
+  using C = RCfg<DT, EPI>;
+  return 1024 + C::QBUFS * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(RCtrlT<C::MMA2>) +
          (C::SMEM_SCORES ? (size_t)NMEM * SCORE_SLOTS * 4 : 0);
 }
-static_assert(rsmem_bytes<DT_FP8>() <= 232448 && rsmem_bytes<DT_BF16>() <= 232448, "shared memory budget");
+static_assert(rsmem_bytes<DT_FP8, 1>() <= 232448 && rsmem_bytes<DT_FP8, 0>() <= 232448 &&
+              rsmem_bytes<DT_BF16>() <= 232448, "shared memory budget");
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -90,15 +109,16 @@ __device__ __forceinline__ int group_tiles(const GroupDesc& gd) {
   return gd.n_cand > 0 ? (gd.n_cand + TILE_KEYS - 1) / TILE_KEYS : 0;
 }
 
-template <int DT>
+template <int DT, int EPI>
 __global__ void __launch_bounds__(THREADS, 1)
 refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __restrict__ groups, int n_groups,
                  int q_rows_total, ScanScratch sc) {
-  using C = RCfg<DT>;
+  using C = RCfg<DT, EPI>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* qbuf = smem;
   uint8_t* kring = smem + C::QBUFS * C::QBUF_BYTES;
+  using RCtrl = RCtrlT<C::MMA2>;
   RCtrl& ct = *reinterpret_cast<RCtrl*>(kring + C::STAGES * C::STAGE_BYTES);
   uint32_t* skey = reinterpret_cast<uint32_t*>(kring + C::STAGES * C::STAGE_BYTES + sizeof(RCtrl));   // [NMEM][SCORE_SLOTS]
   volatile int* abort_flag = &ct.abort;
@@ -114,8 +134,11 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       ptx::mbar_init(&ct.q_full[i], 1);
       ptx::mbar_init(&ct.q_empty[i], 1);
       ptx::mbar_init(&ct.tmem_full[i], 1);
-      ptx::mbar_init(&ct.tmem_empty[i], EPI_WARPS);
+      ptx::mbar_init(&ct.tmem_empty[i], C::TMEM_EMPTY_ARRIVALS);
+      ptx::mbar_init(&ct.a_ready[i], 4);
+      ptx::mbar_init(&ct.s_ready[i], 1);
     }
+    ptx::mbar_init(&ct.w_ready, 1);
     ct.abort = 0;
     ptx::fence_barrier_init();
   }
@@ -123,6 +146,8 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
     ptx::tmem_alloc(&ct.tmem_base, TMEM_COLS);
     ptx::tmem_relinquish();
   }
+  if constexpr (C::MMA2)        // everything but the diagonal blocks of the gate matrix stays zero
+    for (int i = threadIdx.x; i < WMAT_BYTES / 16; i += blockDim.x) reinterpret_cast<uint4*>(ct.wmat)[i] = make_uint4(0, 0, 0, 0);
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
@@ -151,6 +176,30 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
     if (ptx::elect_one()) {
       uint32_t it = 0, blk = 0;
       bool ok = true;
+      // MMA2: the head sum of tile it-1 follows the first MMA of tile it (see the shared scan)
+      bool pend = false;
+      uint32_t pend_it = 0, pend_blk = 0, w_blk = 0xffffffffu;
+      auto issue_mma2 = [&]() -> bool {
+        if (pend_blk != w_blk) {                 // first tile of a group: its gate matrix must be in place
+          if (!ptx::mbar_wait(&ct.w_ready, pend_blk & 1, abort_flag, 32)) return false;
+          w_blk = pend_blk;
+        }
+        const int pb = pend_it & 1;
+        if (!ptx::mbar_wait(&ct.a_ready[pb], (pend_it >> 1) & 1, abort_flag, 32)) return false;
+        ptx::tc_fence_after();
+        const uint32_t w_addr = ptx::smem_u32(ct.wmat);
+        const uint32_t a_tmem = tmem_base + pb * N;
+#pragma unroll
+        for (int ks = 0; ks < 16; ++ks) {        // 16 bf16 of K per step: 8 TMEM columns, 32 bytes of W
+          const int slab = ks >> 2;
+          uint64_t d = ptx::smem_desc_sw128(w_addr + slab * 1024 + (ks & 3) * 32);
+          d &= ~((uint64_t)0x3FFF << 32);        // rows 8..15 of the slab: the shared zero block
+          d |= (uint64_t)(((4096 - slab * 1024) >> 4) & 0x3FFF) << 32;
+          ptx::tc_mma_a_tmem_bf16(a_tmem + 128, a_tmem + ks * 8, d, C::IDESC2, ks ? 1u : 0u);
+        }
+        ptx::tc_commit(&ct.s_ready[pb]);
+        return true;
+      };
       for (int gi = blockIdx.x; gi < n_groups && ok; gi += gridDim.x) {
         const int ntiles = group_tiles(groups[gi]);
         if (ntiles == 0) continue;
@@ -179,6 +228,14 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
             }
           ptx::tc_commit(&ct.empty[s]);
           ptx::tc_commit(&ct.tmem_full[buf]);
+          if constexpr (C::MMA2) {
+            if (pend) { ok = issue_mma2(); if (!ok) break; }
+            pend = true; pend_it = it; pend_blk = blk;
+          }
+        }
+        if constexpr (C::MMA2) {                 // the group's last tile: nothing left to overlap it with
+          if (pend && ok) ok = issue_mma2();
+          pend = false;
         }
         ptx::tc_commit(&ct.q_empty[qb]);
         ++blk;
@@ -248,6 +305,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
     const int key_in_tile = lq * 32 + lane;
     const int tt = (ew & 3) * 32 + lane;
     const Team tm{tt, 128, 1 + team};
+    const Team all{ew * 32 + lane, EPI_WARPS * 32, 3};   // both teams
     SegSelSmem& sel = ct.sel[team];
     const int wq = ew & 3;
     const int SEG = sc.cap >> 2;
@@ -260,8 +318,32 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       const int ntiles = group_tiles(gd);
       if (ntiles == 0) continue;
       const bool smem_sel = C::SMEM_SCORES && !gd.ent_out && ntiles * TILE_KEYS <= SCORE_SLOTS;
-      tm.sync();
-      {
+      if constexpr (C::MMA2) {
+        // team 1 scores all four members (so both teams meet around the tile loop: the other team
+        // selects from what it wrote) and writes the diagonal blocks of the gate matrix; the last
+        // second MMA of the previous group is through (its scores have been read)
+        all.sync();
+        if (team == 1) {
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int i = tt + u * 128, r = i >> 6, j = i & 63;
+            float wv = 0.f;
+            if (r < gd.m) {
+              wv = gd.w[r * kHeads + j];
+              if (gd.qscale) wv = __fmul_rn(wv, gd.qscale[r * kHeads + j]);
+            }
+            const __nv_bfloat16 hi = __float2bfloat16_rn(wv);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(wv - __bfloat162float(hi));
+            const uint32_t in_row = (j & 7) * 2;
+            *reinterpret_cast<__nv_bfloat16*>(ct.wmat + r * 1024 + r * 128 + (((j >> 3) ^ (r & 7)) << 4) + in_row) = hi;
+            *reinterpret_cast<__nv_bfloat16*>(ct.wmat + r * 1024 + (4 + r) * 128 + (((j >> 3) ^ ((4 + r) & 7)) << 4) + in_row) = lo;
+          }
+          ptx::fence_proxy_async_smem();         // generic-proxy writes -> tensor-core reads
+          tm.sync();
+          if (tt == 0) ptx::mbar_arrive(&ct.w_ready);
+        }
+      } else {
+        tm.sync();
         const int rl = tt >> 6, jh = tt & 63;
         const int r = team * 2 + rl;
         float wv = 0.f;
@@ -270,8 +352,80 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
           if (gd.qscale) wv = __fmul_rn(wv, gd.qscale[r * kHeads + jh]);
         }
         ct.w[r][jh] = 0.5f * wv;       // halved: see the ReLU identity in the tile loop
+        tm.sync();
       }
-      tm.sync();
+      // One member row's result: a key never seen by the member (beyond its own position: only
+      // window slots can be, Appendix B) or a padding slot counts as empty.
+      auto put = [&](int r, int t, int slot, int idx, uint32_t key) {
+        const bool seen = idx >= 0 && idx <= gd.first_pos + r;
+        if (smem_sel) {                // key only; the position is looked up again at the end
+          if (r < gd.m) skey[r * SCORE_SLOTS + slot] = seen ? key : 0u;
+          return;
+        }
+        const entry_t e = seen ? make_entry(key, idx) : kPadEntry;
+        if (gd.ent_out) {              // chunked mode: leave the entries for a later top-k
+          if (r < gd.m && slot < gd.n_cand) gd.ent_out[(size_t)r * gd.ent_stride + gd.slot0 + slot] = e;
+        } else if (r < gd.m && t * 32 + lane < SEG) {
+          sc.cand64[seg_off(r) + t * 32 + lane] = e;   // entry t*32+lane of segment (r, lane quarter)
+        }
+      };
+      if constexpr (C::MMA2) {
+        if (team == 0) {
+          // ---- ReLU warps: fp32 accumulator -> packed bf16 ReLU values, in place (thread = key)
+          for (int t = 0; t < ntiles; ++t, ++it) {
+            const int buf = it & 1;
+            (void)ptx::mbar_wait(&ct.tmem_full[buf], (it >> 1) & 1, abort_flag);
+            ptx::tc_fence_after();
+            const uint32_t xb = tmem_base + ((uint32_t)(lq * 32) << 16) + buf * N;
+            uint32_t va[32], vb[32];
+            ptx::tmem_ld_32x32_async(xb, va);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              if (c & 1) ptx::tmem_wait_ld_regs(vb);
+              else ptx::tmem_wait_ld_regs(va);
+              if (c + 1 < 8) {
+                if (c & 1) ptx::tmem_ld_32x32_async(xb + (c + 1) * 32, va);
+                else ptx::tmem_ld_32x32_async(xb + (c + 1) * 32, vb);
+              }
+              uint32_t pk[16];
+              const bool have_row = (c >> 1) < gd.m;           // members missing from the group: zeros
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                pk[i] = (c & 1) ? ptx::relu_pack_bf16x2(__uint_as_float(vb[2 * i]), __uint_as_float(vb[2 * i + 1]))
+                                : ptx::relu_pack_bf16x2(__uint_as_float(va[2 * i]), __uint_as_float(va[2 * i + 1]));
+                pk[i] = have_row ? pk[i] : 0u;
+              }
+              ptx::tmem_st_32x16(xb + c * 16, pk);
+            }
+            ptx::tmem_wait_st();
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&ct.a_ready[buf]);
+          }
+        } else {
+          // ---- score warps: the four member scores of this thread's key
+          for (int t = 0; t < ntiles; ++t, ++it) {
+            const int buf = it & 1;
+            const int slot = t * TILE_KEYS + key_in_tile;
+            (void)ptx::mbar_wait(&ct.s_ready[buf], (it >> 1) & 1, abort_flag);
+            ptx::tc_fence_after();
+            // position and scale of this thread's key, left in shared memory by the gather warps
+            const KeyMeta mt = ct.meta[it % META_SLOTS][key_in_tile];
+            uint32_t s8[8];            // columns r: sums with the gates' bf16 heads, 4 + r: with their remainders
+            ptx::tmem_ld_32x8(tmem_base + ((uint32_t)(lq * 32) << 16) + buf * N + 128, s8);
+            ptx::tmem_wait_ld();
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
+#pragma unroll
+            for (int r = 0; r < NMEM; ++r) {
+              const float sc_r = __uint_as_float(s8[r]) + __uint_as_float(s8[4 + r]);
+              put(r, t, slot, mt.idx, score_to_key(gd.kscale ? sc_r * mt.ks : sc_r));
+            }
+          }
+        }
+        all.sync();
+      } else {
       for (int t = 0; t < ntiles; ++t, ++it) {
         const int buf = it & 1;
         const int slot = t * TILE_KEYS + key_in_tile;
@@ -315,26 +469,12 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
-        // entry t*32+lane of this warp's segment; slots past the candidate list are padding
 #pragma unroll
-        for (int rl = 0; rl < 2; ++rl) {
-          const int r = team * 2 + rl;
-          const uint32_t key = score_to_key(gd.kscale ? score[rl] * ksv : score[rl]);
-          // a member never sees a key beyond its own position (only window slots can be: Appendix B)
-          const bool seen = idx >= 0 && idx <= gd.first_pos + r;
-          if (smem_sel) {              // key only; the position is looked up again at the end
-            if (r < gd.m) skey[r * SCORE_SLOTS + slot] = seen ? key : 0u;
-            continue;
-          }
-          const entry_t e = seen ? make_entry(key, idx) : kPadEntry;
-          if (gd.ent_out) {            // chunked mode: leave the entries for a later top-k
-            if (r < gd.m && slot < gd.n_cand) gd.ent_out[(size_t)r * gd.ent_stride + gd.slot0 + slot] = e;
-          } else if (r < gd.m && t * 32 + lane < SEG) {
-            sc.cand64[seg_off(r) + t * 32 + lane] = e;
-          }
-        }
+        for (int rl = 0; rl < 2; ++rl)
+          put(team * 2 + rl, t, slot, idx, score_to_key(gd.kscale ? score[rl] * ksv : score[rl]));
       }
       tm.sync();
+      }
       if (gd.ent_out) continue;
       // ---- per-member exact top-k over the candidate scores
 #pragma unroll
@@ -378,12 +518,12 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
   if (threadIdx.x == 0 && ct.abort) set_status(sc.status, DEV_WAIT_EXPIRED);
 }
 
-template <int DT>
+template <int DT, int EPI = 1>
 cudaError_t launch_one(const CUtensorMap& mq, const GroupDesc* groups, int n_groups, int q_rows,
                        const ScanScratch& s, int sms, cudaStream_t st) {
-  auto kern = refine_tc_kernel<DT>;
+  auto kern = refine_tc_kernel<DT, EPI>;
   static bool attr_set = false;
-  const size_t smem = rsmem_bytes<DT>();
+  const size_t smem = rsmem_bytes<DT, EPI>();
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -400,12 +540,13 @@ cudaError_t launch_one(const CUtensorMap& mq, const GroupDesc* groups, int n_gro
 bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows);
 
 cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
-                             const ScanScratch& s, int sms, cudaStream_t st) {
+                             const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum) {
   if (n_groups <= 0) return cudaSuccess;
   CUtensorMap mq;
   if (!make_operand_map(&mq, q, (long long)q_rows * kHeads, dtype, kHeads)) return cudaErrorInvalidValue;
-  return dtype == DT_FP8 ? launch_one<DT_FP8>(mq, groups, n_groups, q_rows, s, sms, st)
-                         : launch_one<DT_BF16>(mq, groups, n_groups, q_rows, s, sms, st);
+  if (dtype != DT_FP8) return launch_one<DT_BF16>(mq, groups, n_groups, q_rows, s, sms, st);
+  return fp32_head_sum ? launch_one<DT_FP8, 0>(mq, groups, n_groups, q_rows, s, sms, st)
+                       : launch_one<DT_FP8, 1>(mq, groups, n_groups, q_rows, s, sms, st);
 }
 
 }  // namespace pivot
