@@ -382,28 +382,37 @@ __device__ __forceinline__ int seg_emit_hist(const Team& tm, SegSelSmem& sm, con
       const int i = j0 + u * 32 + lane;
       x[u] = i < seg.cnt ? __ldcg(seg.e + i) : kPadEntry;
     }
+    // one cursor bump per batch: the eight votes first, then a single atomic for their total
+    uint32_t m[8];
+    uint32_t batch = 0;
+    uint32_t emit_bits = 0;
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       const bool valid = (j0 + u * 32 + lane) < seg.cnt && entry_pos(x[u]) >= 0;
       const int bn = (int)bin_of(entry_key(x[u]));
       const bool emit = valid && bn > bsel;
-      const uint32_t m = __ballot_sync(0xffffffffu, emit);
-      if (m) {
-        uint32_t pos = 0;
-        const int leader = __ffs(m) - 1;
-        if (lane == leader) pos = atomicAdd(&sm.out_count, (uint32_t)__popc(m));
-        pos = __shfl_sync(0xffffffffu, pos, leader);
-        if (emit) {
-          const uint32_t p = pos + __popc(m & ((1u << lane) - 1u));
+      m[u] = __ballot_sync(0xffffffffu, emit);
+      batch += (uint32_t)__popc(m[u]);
+      emit_bits |= emit ? 1u << u : 0u;
+      if (valid && bn == bsel) {
+        const uint32_t q = atomicAdd(&sm.list_n, 1u);
+        if (q < (uint32_t)kSelSmall) sm.list[q] = x[u];
+      }
+    }
+    if (batch) {
+      uint32_t pos = 0;
+      if (lane == 0) pos = atomicAdd(&sm.out_count, batch);
+      pos = __shfl_sync(0xffffffffu, pos, 0);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if ((emit_bits >> u) & 1u) {
+          const uint32_t p = pos + __popc(m[u] & ((1u << lane) - 1u));
           if (p < (uint32_t)K) {
             out[p] = entry_pos(x[u]);
             if (out_score) out_score[p] = key_to_score(entry_key(x[u]));
           }
         }
-      }
-      if (valid && bn == bsel) {
-        const uint32_t q = atomicAdd(&sm.list_n, 1u);
-        if (q < (uint32_t)kSelSmall) sm.list[q] = x[u];
+        pos += (uint32_t)__popc(m[u]);
       }
     }
   }
