@@ -266,6 +266,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--window", type=int, default=0, help="local window W of Appendix B (device-timed value only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense-indexer control")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--decode-only", action="store_true", help="only the MTP decode step (prints its object)")
@@ -335,6 +336,33 @@ def main():
     ms_per_step = elapsed_ms / args.steps
     value = job_throughput(world, L, ms_per_step)
 
+    # ---- the dense indexer (Eq. 1 for every query: the O(L^2) control PIVOT replaces) on the same
+    #      inputs, same kernels, same GPU: gives the PIVOT / dense ratio to set beside the paper's
+    dense = None
+    if not args.no_dense and rank == 0:
+        dout = torch.empty((L, k), dtype=torch.int32, device=dev)
+        dstep = lambda: pv.dense_index(dq, dw, dk, L, H, D, k, dout, stream, q_scale=dqs, k_scale=dks)
+        dstep()
+        torch.cuda.synchronize()
+        n_d = 2
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record(stream)
+        for _ in range(n_d):
+            dstep()
+        d1.record(stream)
+        torch.cuda.synchronize()
+        d_ms = d0.elapsed_time(d1) / n_d
+        assert pv.pivot_device_status() == 0
+        dense_scores = L * (L + 1) // 2
+        dense = {"entry": "dense_index", "ms_per_step": d_ms, "tokens_per_s": L / (d_ms * 1e-3), "steps": n_d,
+                 "tflops": FLOP_PER_SCORE * dense_scores / (d_ms * 1e-3) / 1e12,
+                 "pivot_speedup_over_dense": d_ms / ms_per_step,
+                 "paper_h20_speedup_context": "PIVOT-Refine 0.93x at 16K .. 3.87x at 256K, PIVOT-Reuse about 4x (H20, FP8)"}
+        del dout
+        pv.pivot_set_workspace(None)
+        torch.cuda.empty_cache()
+        pv.ensure_workspace(L, nG, c, k, dev)
+
     # ---- end to end through the host-buffer entry point (H2D + compute + D2H every step)
     e2e = None
     if not args.no_e2e:
@@ -399,6 +427,8 @@ def main():
     }
     if e2e is not None:
         line["e2e"] = e2e
+    if dense is not None:
+        line["dense_control"] = dense
     if not args.no_decode:
         try:
             del arena
