@@ -371,7 +371,7 @@ __device__ __forceinline__ int seg_emit_hist(const Team& tm, SegSelSmem& sm, con
                                              BinFn bin_of, int32_t* out, float* out_score, int K) {
   const int lane = tm.tid & 31;
   uint32_t b = 0, need_b = 0, pop = 0;
-  const bool found = warp_hist_boundary<false>(hist, (uint32_t)K, lane, &b, &need_b, &pop);
+  const bool found = warp_hist_boundary<0>(hist, (uint32_t)K, lane, &b, &need_b, &pop);
   const int bsel = found ? (int)b : -1;
   if (tm.tid == 0) { sm.out_count = 0; sm.list_n = 0; }
   tm.sync();
