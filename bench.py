@@ -439,7 +439,7 @@ def main():
 
     # ---- parity probe on the e2e result (a few groups) and the CPU baseline
     if not args.no_cpu_baseline:
-        est, dt, n, threads = oracle_sample_time(x, L, g, c, k, mode, n_groups=160 if L > 40000 else 256, seed=7)
+        est, dt, n, threads = oracle_sample_time(x, L, g, c, k, mode, n_groups=512 if L > 40000 else 768, seed=7)
         line["cpu_baseline"] = {"value": L / est, "unit": "tokens/s", "cores": threads, "kind": "oracle",
                                 "sample": f"{n} uniformly drawn groups of {nG}, time scaled to the whole "
                                           f"request; {dt:.1f} s of CPU work timed"}
