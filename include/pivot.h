@@ -146,6 +146,22 @@ int pivot_index_prefill_ex(const pivot_tensor* q, const float* w, const pivot_te
                            int32_t* out_idx, pivot_stream_t stream, const pivot_opts* opts);
 
 /*
+ * Batched prefill of several requests packed back to back (the request boundaries of Eq. 2:
+ * groups and causal prefixes never cross from one request into the next).
+ *   cu_seqlens   HOST array [n_req + 1], non-decreasing, cu_seqlens[0] = 0: request i owns rows
+ *                cu_seqlens[i] .. cu_seqlens[i+1]-1 of q / w / kcache / out_idx (total rows =
+ *                cu_seqlens[n_req]).  With FP8 every request must start on a multiple of 4 rows
+ *                (the key-scale rows are read in 16-byte units); empty requests are allowed.
+ *   out_idx      [total rows, k]; positions are relative to the start of the row's own request.
+ * Each request is indexed by the prefill path above, one after the other on `stream`, sharing
+ * one workspace sized for the longest request (opts->workspace, else the registered one).
+ * opts may be NULL; row_begin / row_end and the debug buffers are not available here.
+ */
+int pivot_index_prefill_varlen(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                               const int32_t* cu_seqlens, int n_req, int H_I, int d, int g, int c, int k,
+                               int mode, int32_t* out_idx, pivot_stream_t stream, const pivot_opts* opts);
+
+/*
  * Decode (Algorithm 1 with the grouping of Eq. 3): B independent sequences, each contributing
  * the g queries of one MTP step at positions pos0[b] .. pos0[b]+g-1.
  *   q       [B, g, H_I, d]; w [B, g, H_I]; kcache [B, Lmax, d] (+ scale [B, Lmax]); sequence b's

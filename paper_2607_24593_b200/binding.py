@@ -22,6 +22,7 @@ OK = 0
 
 SYMBOLS = [
     "pivot_workspace_bytes", "pivot_decode_workspace_bytes", "pivot_set_workspace", "pivot_index_prefill", "pivot_index_prefill_ex",
+    "pivot_index_prefill_varlen",
     "pivot_index_decode", "pivot_index_decode_ex", "dense_index", "dense_index_ex", "dense_index_static",
     "pivot_prefill_host_arena_bytes", "pivot_index_prefill_host", "pivot_device_status",
     "pivot_stage_timing", "pivot_stage_times", "pivot_launch_count_reset", "pivot_status_str", "pivot_last_cuda_error",
@@ -57,6 +58,7 @@ def _load():
     lib.pivot_set_workspace.argtypes = [P, S]
     lib.pivot_index_prefill.argtypes = [T, P, T, I, I, I, I, I, I, I, P, P]
     lib.pivot_index_prefill_ex.argtypes = [T, P, T, I, I, I, I, I, I, I, P, P, O]
+    lib.pivot_index_prefill_varlen.argtypes = [T, P, T, C.POINTER(C.c_int32), I, I, I, I, I, I, I, P, P, O]
     lib.pivot_index_decode.argtypes = [T, P, T, P, I, I, I, I, I, I, I, I, P, P]
     lib.pivot_index_decode_ex.argtypes = [T, P, T, P, I, I, I, I, I, I, I, I, P, P, O]
     lib.dense_index.argtypes = [T, P, T, I, I, I, I, P, P]
@@ -158,6 +160,24 @@ def pivot_index_prefill(q, w, kcache, L, H_I, d, g, c, k, mode, out_idx, stream=
     o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl, rows, W)
     _check(lib.pivot_index_prefill_ex(C.byref(tq), w.data_ptr(), C.byref(tk), L, H_I, d, g, c, k, mode,
                                       out_idx.data_ptr(), _stream(stream), C.byref(o)))
+    return out_idx
+
+
+def pivot_index_prefill_varlen(q, w, kcache, cu_seqlens, H_I, d, g, c, k, mode, out_idx, stream=None, *,
+                               q_scale=None, k_scale=None, guard_len=None, pool=POOL_MEAN, workspace=None, impl=0, W=0):
+    """Several requests packed back to back; cu_seqlens is a host sequence [n_req + 1] starting at 0.
+    Positions in out_idx are relative to each row's own request."""
+    cu = [int(v) for v in cu_seqlens]
+    n_req = len(cu) - 1
+    tq, tk = _tensor(q, q_scale), _tensor(kcache, k_scale)
+    assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and out_idx.numel() >= cu[-1] * k
+    if workspace is None:
+        Lmax = max((b - a for a, b in zip(cu[:-1], cu[1:])), default=1)
+        ensure_workspace(max(Lmax, 1), (max(Lmax, 1) + g - 1) // g, c, k, q.device)
+    o = _opts(guard_len, pool, None, None, None, workspace, impl, None, W)
+    arr = (C.c_int32 * (n_req + 1))(*cu)
+    _check(lib.pivot_index_prefill_varlen(C.byref(tq), w.data_ptr(), C.byref(tk), arr, n_req, H_I, d, g, c, k, mode,
+                                          out_idx.data_ptr(), _stream(stream), C.byref(o)))
     return out_idx
 
 

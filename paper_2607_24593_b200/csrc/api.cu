@@ -273,6 +273,32 @@ int pivot_index_prefill(const pivot_tensor* q, const float* w, const pivot_tenso
   return pivot_index_prefill_ex(q, w, kcache, L, H_I, d, g, c, k, mode, out_idx, stream, nullptr);
 }
 
+int pivot_index_prefill_varlen(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                               const int32_t* cu_seqlens, int n_req, int H_I, int d, int g, int c, int k,
+                               int mode, int32_t* out_idx, pivot_stream_t stream, const pivot_opts* opts) {
+  int rc = check_common(q, w, kcache, H_I, d, c, k, mode, out_idx);
+  if (rc) return rc;
+  if (!cu_seqlens || n_req < 1 || g < 1 || cu_seqlens[0] != 0) return PIVOT_ERR_INVALID_ARG;
+  if (opts && (opts->row_begin || opts->row_end || opts->dbg_cand || opts->dbg_scores || opts->dbg_cand_scores))
+    return PIVOT_ERR_INVALID_ARG;
+  const bool fp8 = q->dtype == PIVOT_FP8_E4M3;
+  for (int i = 0; i < n_req; ++i) {
+    if (cu_seqlens[i + 1] < cu_seqlens[i]) return PIVOT_ERR_INVALID_ARG;
+    if (fp8 && (cu_seqlens[i] & 3)) return PIVOT_ERR_INVALID_ARG;
+  }
+  const size_t esz = fp8 ? 1 : 2;
+  for (int i = 0; i < n_req; ++i) {
+    const size_t r0 = (size_t)cu_seqlens[i];
+    const int L = cu_seqlens[i + 1] - cu_seqlens[i];
+    if (L == 0) continue;
+    pivot_tensor tq{(const char*)q->data + r0 * H_I * d * esz, q->scale ? q->scale + r0 * H_I : nullptr, q->dtype};
+    pivot_tensor tk{(const char*)kcache->data + r0 * d * esz, kcache->scale ? kcache->scale + r0 : nullptr, q->dtype};
+    rc = pivot_index_prefill_ex(&tq, w + r0 * H_I, &tk, L, H_I, d, g, c, k, mode, out_idx + r0 * k, stream, opts);
+    if (rc) return rc;
+  }
+  return PIVOT_OK;
+}
+
 int dense_index_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kcache, int L, int H_I,
                    int d, int k, int32_t* out_idx, pivot_stream_t stream, const pivot_opts* opts) {
   int rc = check_common(q, w, kcache, H_I, d, k, k, PIVOT_REUSE, out_idx);

@@ -224,3 +224,36 @@ def test_local_window_argument_errors(pv):
         pv.pivot_index_prefill(q, w, k, 256, 64, 128, 4, 16, 8, pv.REFINE, out, W=4, guard_len=4)   # guardrail < W + g
     with pytest.raises(pv.PivotError, match="invalid"):
         pv.pivot_index_prefill(q, w, k, 256, 64, 128, 4, 16, 8, pv.REFINE, out, W=-1)
+
+
+# ---------------------------------------------------------------- packed requests (Eq. 2 boundaries)
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+def test_prefill_varlen_equals_per_request_calls(pv, dtype):
+    """Requests packed back to back give, row for row, what separate calls give: groups and causal
+    prefixes stop at the request boundaries, positions are relative to the request."""
+    lens = [700, 0, 1028, 300]            # starts at multiples of 4 (FP8 scale rows), one empty request
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(int)
+    g, c, k, mode = 4, 256, 64, pv.REFINE
+    xs = [inputs.make_prefill(n, dtype=dtype, seed=100 + i) if n else None for i, n in enumerate(lens)]
+    cat = lambda name: torch.cat([getattr(x, name) for x in xs if x is not None]).cuda()
+    q, w, kk = cat("q"), cat("w"), cat("k")
+    sc = dict(q_scale=cat("qscale"), k_scale=cat("kscale")) if dtype == "fp8" else {}
+    packed = torch.full((int(cu[-1]), k), -7, dtype=torch.int32, device="cuda")
+    pv.pivot_index_prefill_varlen(q, w, kk, cu, 64, 128, g, c, k, mode, packed, **sc)
+    torch.cuda.synchronize()
+    assert pv.pivot_device_status() == 0
+    for i, x in enumerate(xs):
+        if x is None:
+            continue
+        one = torch.full((lens[i], k), -7, dtype=torch.int32, device="cuda")
+        s1 = dict(q_scale=x.qscale.cuda(), k_scale=x.kscale.cuda()) if dtype == "fp8" else {}
+        pv.pivot_index_prefill(x.q.cuda(), x.w.cuda(), x.k.cuda(), lens[i], 64, 128, g, c, k, mode, one, **s1)
+        got = packed[cu[i]:cu[i + 1]].cpu().numpy()
+        assert np.array_equal(_sorted_rows(got), _sorted_rows(one.cpu().numpy())), f"request {i}"
+        assert got.max() < lens[i]
+    if dtype == "fp8":
+        with pytest.raises(pv.PivotError, match="invalid"):
+            pv.pivot_index_prefill_varlen(q, w, kk, [0, 702, int(cu[-1])], 64, 128, g, c, k, mode, packed, **sc)
+    with pytest.raises(pv.PivotError, match="invalid"):
+        pv.pivot_index_prefill_varlen(q, w, kk, [0, 800, 400], 64, 128, g, c, k, mode, packed, **sc)
