@@ -257,6 +257,51 @@ def run_reference(args, wl):
     print(json.dumps(line))
 
 
+def sweep(pv, dev, L, dtype, steps):
+    """Group size / candidate budget / pooling / window sweep on one synthetic request: milliseconds
+    per request and recall of the dense indexer's top-k (the library's own dense_index on the same
+    inputs), averaged over a sample of query rows.  A stand-in for the paper's ablation tables, whose
+    accuracy numbers need the models and evaluation suites: recall on the synthetic generator says how
+    close the selection stays to the dense one, nothing about task accuracy.  One JSON line per case."""
+    k = 2048
+    x = inputs.make_prefill(L, dtype=dtype, seed=rank_seed(0))
+    q, w, kc = x.q.to(dev), x.w.to(dev), x.k.to(dev)
+    sc = dict(q_scale=None if x.qscale is None else x.qscale.to(dev), k_scale=None if x.kscale is None else x.kscale.to(dev))
+    stream = torch.cuda.current_stream()
+    dense = torch.empty((L, k), dtype=torch.int32, device=dev)
+    pv.dense_index(q, w, kc, L, H, D, k, dense, stream, **sc)
+    torch.cuda.synchronize()
+    rows = torch.arange(8192 + 37, L, max(1, (L - 8192) // 512), device=dev)        # past every guardrail
+    dsel = torch.zeros((len(rows), L), dtype=torch.bool, device=dev)
+    dsel.scatter_(1, dense[rows].long().clamp_(min=0), True)
+    out = torch.empty((L, k), dtype=torch.int32, device=dev)
+    cases = [dict(g=g, c=4096, mode=m, pool=0, W=0) for g in (2, 4, 8, 16) for m in (1, 0)]
+    cases += [dict(g=4, c=c, mode=1, pool=0, W=0) for c in (3072, 6144, 8192)]
+    cases += [dict(g=4, c=4096, mode=1, pool=p, W=0) for p in (1, 2)]
+    cases += [dict(g=4, c=4096, mode=m, pool=0, W=4) for m in (1, 0)]
+    for cs in cases:
+        g, c = cs["g"], cs["c"]
+        pv.ensure_workspace(L, (L + g - 1) // g, c, k, dev)
+        run = lambda: pv.pivot_index_prefill(q, w, kc, L, H, D, g, c, k, cs["mode"], out, stream, pool=cs["pool"],
+                                             W=cs["W"], **sc)
+        run()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            run()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        assert pv.pivot_device_status() == 0
+        got = out[rows].long()
+        hit = torch.gather(dsel, 1, got.clamp(min=0)) & (got >= 0)
+        recall = float(hit.sum(1).float().mean() / k)
+        print(json.dumps({"sweep": f"prefill_{L // 1024}k_{dtype}", "g": g, "c": c, "k": k,
+                          "mode": "refine" if cs["mode"] else "reuse", "pool": ["mean", "first", "last"][cs["pool"]],
+                          "W": cs["W"], "ms_per_request": e0.elapsed_time(e1) / steps,
+                          "recall_of_dense_topk": recall, "rows_sampled": int(len(rows))}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -270,6 +315,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--decode-only", action="store_true", help="only the MTP decode step (prints its object)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="g / c / pooling / window sweep with recall of the dense top-k (one JSON line per case)")
     args = ap.parse_args()
     wl = args.workload
     if args.impl == "reference":
@@ -287,6 +334,9 @@ def main():
 
     from paper_2607_24593_b200 import binding as pv
 
+    if args.sweep:
+        sweep(pv, torch.device(f"cuda:{local}"), L, dtype, max(1, min(args.steps, 3)))
+        return
     if args.decode_only:
         print(json.dumps(decode_bench(pv, torch.device(f"cuda:{local}"), steps=max(args.steps, 5),
                                       warmup=max(args.warmup, 3), pk=peaks())))
