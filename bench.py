@@ -191,6 +191,41 @@ def decode_bench(pv, dev, steps, warmup, pk):
     except Exception as e:                                              # capture refused: say why, keep the stream number
         graph_note = f"{type(e).__name__}: {e}"[:200]
         torch.cuda.synchronize()
+    # the same step over a paged copy of the cache (128-key pages scattered over a pool)
+    mp = (Lmax + 127) // 128
+    pages = torch.zeros((B, mp * 128, D), dtype=torch.uint8, device=dev)
+    pages[:, :Lmax] = kc.view(torch.uint8)
+    pscale = torch.zeros((B, mp * 128), dtype=torch.float32, device=dev)
+    pscale[:, :Lmax] = ks
+    perm = torch.randperm(B * mp, generator=torch.Generator().manual_seed(1)).to(dev)
+    pool = torch.empty((B * mp, 128, D), dtype=torch.uint8, device=dev)
+    pool[perm] = pages.view(B * mp, 128, D)
+    pool_s = torch.empty((B * mp, 128), dtype=torch.float32, device=dev)
+    pool_s[perm] = pscale.view(B * mp, 128)
+    del pages, pscale
+    pool = pool.view(B * mp * 128, D).view(kc.dtype)
+    pool_s = pool_s.view(-1)
+    bt = perm.to(torch.int32).view(B, mp).contiguous()
+    out_p = torch.empty_like(out)
+
+    def step_paged():
+        pv.pivot_index_decode_paged(q, w, pool, bt, p0, B, mp, B * mp, H, D, g, c, k, pv.REFINE, out_p, stream,
+                                    q_scale=qs, k_scale=pool_s)
+
+    for _ in range(warmup):
+        step_paged()
+    torch.cuda.synchronize()
+    paged_times = timed(step_paged, steps)
+    same = bool((torch.sort(out_p, dim=2).values == torch.sort(out, dim=2).values).all().item())
+    pv.pivot_stage_timing(True)
+    paged_scan = []
+    for _ in range(3):
+        flush.fill_(1)
+        step_paged()
+        torch.cuda.synchronize()
+        paged_scan.append(pv.pivot_stage_times()["decode_scan"] * 1e3)
+    pv.pivot_stage_timing(False)
+    assert pv.pivot_device_status() == 0
     us = float(np.median(times))
     scan = float(np.mean(scan_us))
     n0 = (x.pos0.numpy().astype(np.int64) + 1)
@@ -198,6 +233,8 @@ def decode_bench(pv, dev, steps, warmup, pk):
     return {"metric": "us per MTP decode step", "value": us, "unit": "us", "min_us": float(min(times)),
             "steps": steps, "higher_is_better": False, "gpu_launches_per_step": launches / max(steps, 1),
             "graph_replay_us": graph_us, "graph_note": graph_note,
+            "paged": {"value": float(np.median(paged_times)), "unit": "us", "scan_kernel_us": float(np.mean(paged_scan)),
+                      "page_keys": 128, "pool_pages": B * mp, "same_positions_as_contiguous": same},
             "config": {"workload": "decode_mtp_b32_64k-128k_fp8_g2_refine", "B": B, "g": g, "c": c, "k": k,
                        "visible_keys": int(n0.sum()), "l2": "256 MB flush between steps"},
             # dominant kernel: the key-streaming scan; algorithmic bytes = visible keys x 132 B

@@ -179,6 +179,27 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
                           int mode, int32_t* out_idx, pivot_stream_t stream, const pivot_opts* opts);
 
 /*
+ * Decode over a PAGED key cache (the layout a serving engine's block manager keeps; the method
+ * itself, Algorithm 1 with the grouping of Eq. 3, is unchanged).
+ *   kpages       the page pool: data [n_pages * 128, d] (+ scale [n_pages * 128]); a page holds
+ *                128 consecutive key positions of one sequence.
+ *   block_table  [B, max_pages] int32, device: block_table[b][p] is the pool page holding keys
+ *                128 p .. 128 p + 127 of sequence b.  Entries for pages past pos0[b] + g - 1 are
+ *                never read.  An entry outside [0, n_pages) faults nothing: its keys read as
+ *                zeros in the scan and are dropped as holes by the re-score.
+ *   pos0, q, w, out_idx, c, k, mode   as in pivot_index_decode; returned positions are LOGICAL
+ *                key positions of the sequence.
+ * Differences from the contiguous form: the short-sequence guardrail is off (opts->guard_len is
+ * ignored) -- a sequence with fewer than c visible keys takes the proxy path with every visible
+ * key as a candidate, so Refine is still exact for it over the keys up to pos0 -- and
+ * opts->impl = 1 is rejected.  Workspace: pivot_decode_workspace_bytes(B, max_pages * 128, ...).
+ */
+int pivot_index_decode_paged(const pivot_tensor* q, const float* w, const pivot_tensor* kpages,
+                             const int32_t* block_table, const int32_t* pos0, int B, int max_pages,
+                             int n_pages, int H_I, int d, int g, int c, int k, int mode,
+                             int32_t* out_idx, pivot_stream_t stream, const pivot_opts* opts);
+
+/*
  * Dense control: Eq. 1 + TopK for every query of a request (prefill form) -- the O(L^2) indexer
  * PIVOT replaces, run by the same kernels with one row per query.  out_idx [L, k].
  */

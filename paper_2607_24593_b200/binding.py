@@ -23,7 +23,7 @@ OK = 0
 SYMBOLS = [
     "pivot_workspace_bytes", "pivot_decode_workspace_bytes", "pivot_set_workspace", "pivot_index_prefill", "pivot_index_prefill_ex",
     "pivot_index_prefill_varlen",
-    "pivot_index_decode", "pivot_index_decode_ex", "dense_index", "dense_index_ex", "dense_index_static",
+    "pivot_index_decode", "pivot_index_decode_ex", "pivot_index_decode_paged", "dense_index", "dense_index_ex", "dense_index_static",
     "pivot_prefill_host_arena_bytes", "pivot_index_prefill_host", "pivot_device_status",
     "pivot_stage_timing", "pivot_stage_times", "pivot_launch_count_reset", "pivot_status_str", "pivot_last_cuda_error",
 ]
@@ -61,6 +61,7 @@ def _load():
     lib.pivot_index_prefill_varlen.argtypes = [T, P, T, C.POINTER(C.c_int32), I, I, I, I, I, I, I, P, P, O]
     lib.pivot_index_decode.argtypes = [T, P, T, P, I, I, I, I, I, I, I, I, P, P]
     lib.pivot_index_decode_ex.argtypes = [T, P, T, P, I, I, I, I, I, I, I, I, P, P, O]
+    lib.pivot_index_decode_paged.argtypes = [T, P, T, P, P, I, I, I, I, I, I, I, I, I, P, P, O]
     lib.dense_index.argtypes = [T, P, T, I, I, I, I, P, P]
     lib.dense_index_ex.argtypes = [T, P, T, I, I, I, I, P, P, O]
     lib.dense_index_static.argtypes = [T, P, T, I, I, I, I, P, P]
@@ -215,6 +216,22 @@ def pivot_index_decode(q, w, kcache, pos0, B, Lmax, H_I, d, g, c, k, mode, out_i
     o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl)
     _check(lib.pivot_index_decode_ex(C.byref(tq), w.data_ptr(), C.byref(tk), pos0.data_ptr(), B, Lmax,
                                      H_I, d, g, c, k, mode, out_idx.data_ptr(), _stream(stream), C.byref(o)))
+    return out_idx
+
+
+def pivot_index_decode_paged(q, w, kpages, block_table, pos0, B, max_pages, n_pages, H_I, d, g, c, k, mode,
+                             out_idx, stream=None, *, q_scale=None, k_scale=None, pool=POOL_MEAN, dbg_cand=None,
+                             dbg_scores=None, dbg_cand_scores=None, workspace=None, impl=0):
+    tq, tk = _tensor(q, q_scale), _tensor(kpages, k_scale)
+    assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and pos0.dtype == torch.int32
+    assert block_table.dtype == torch.int32 and block_table.is_contiguous() and block_table.numel() >= B * max_pages
+    assert out_idx.numel() >= B * g * k
+    if workspace is None:
+        ensure_workspace(B * g, B, c, k, q.device, need=pivot_decode_workspace_bytes(B, max_pages * 128, g, c, k))
+    o = _opts(None, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl)
+    _check(lib.pivot_index_decode_paged(C.byref(tq), w.data_ptr(), C.byref(tk), block_table.data_ptr(),
+                                        pos0.data_ptr(), B, max_pages, n_pages, H_I, d, g, c, k, mode,
+                                        out_idx.data_ptr(), _stream(stream), C.byref(o)))
     return out_idx
 
 

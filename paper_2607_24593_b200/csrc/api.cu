@@ -312,15 +312,19 @@ int dense_index(const pivot_tensor* q, const float* w, const pivot_tensor* kcach
   return dense_index_ex(q, w, kcache, L, H_I, d, k, out_idx, stream, nullptr);
 }
 
-int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
-                          const int32_t* pos0, int B, int Lmax, int H_I, int d, int g, int c, int k,
-                          int mode, int32_t* out_idx, pivot_stream_t stream, const pivot_opts* o) {
+// One MTP decode step.  block_table == nullptr: kcache is [B, Lmax, d]; otherwise kcache is a
+// pool of n_pages pages of 128 keys and block_table [B, Lmax / 128] names each sequence's pages.
+static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor* kcache, const int32_t* pos0,
+                      int B, int Lmax, int H_I, int d, int g, int c, int k, int mode, int32_t* out_idx,
+                      pivot_stream_t stream, const pivot_opts* o, const int32_t* block_table, int n_pages) {
   int rc = check_common(q, w, kcache, H_I, d, c, k, mode, out_idx);
   if (rc) return rc;
   if (!pos0 || B < 1 || g < 1 || Lmax < g) return PIVOT_ERR_INVALID_ARG;
   // every sequence's scale row must start on a 16-byte boundary (TMA reads it in 128-scale tiles)
   if (q->dtype == PIVOT_FP8_E4M3 && (Lmax & 3)) return PIVOT_ERR_INVALID_ARG;
   if (o && (o->pool < 0 || o->pool > 2 || o->W != 0)) return PIVOT_ERR_INVALID_ARG;
+  const bool paged = block_table != nullptr;
+  if (paged && (n_pages < 1 || (Lmax & 127) || (o && o->impl == 1))) return PIVOT_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t base_bytes = pivot_workspace_bytes(B * g, B, c, k);
   const size_t need = base_bytes + decode_fast_bytes(B, Lmax, g, c);
@@ -338,6 +342,12 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
   p.out = out_idx; p.out_score = o ? o->dbg_scores : nullptr;
   p.B = B; p.Lmax = Lmax; p.g = g; p.c = c; p.k = k; p.mode = mode; p.dtype = q->dtype;
   p.guard_len = (o && o->guard_len >= 0) ? o->guard_len : c;
+  // Paged: a short sequence's dense rows would need a contiguous prefix, so the guardrail is
+  // off and short sequences take the proxy path with every visible key as a candidate.
+  if (paged) p.guard_len = 0;
+  p.block_table = block_table;
+  p.n_pages = n_pages;
+  const long long k_rows = paged ? (long long)n_pages * 128 : (long long)B * Lmax;
   if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 2 * sizeof(int), st)))) return rc;
   mark(0, st);
   launch_proxy_build(q->data, q->scale, w, ws.proxy_q, ws.proxy_w, B * g, g, 0, B, q->dtype,
@@ -353,6 +363,7 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
     df.prox = ws.rows; df.groups = ws.groups;
     df.kc = kcache->data; df.kscale = kcache->scale; df.q = q->data; df.proxy_q = ws.proxy_q;
     df.B = B; df.Lmax = Lmax; df.g = g; df.c = c; df.k = k; df.mode = mode; df.dtype = q->dtype;
+    df.k_rows = k_rows;
     df.sms = sm_count();
     df.scratch = (char*)wsp + base_bytes;
     df.scratch_tc = tc_scratch(ws);
@@ -362,8 +373,10 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
     g_ev_decode_scan = g_timing;
     if ((rc = check_cuda(launch_decode_fast(df, st)))) return rc;
     // dense rows of guarded (short) sequences, if any: the generic scan, one row per block
-    ScanOperands op{kcache->data, (long long)B * Lmax, kcache->scale, q->data, B * g, ws.proxy_q, B, q->dtype};
-    if ((rc = check_cuda(launch_scan_tc(op, ws.rows + B, B * g, 1, tc_scratch(ws), sm_count(), st)))) return rc;
+    if (!paged) {
+      ScanOperands op{kcache->data, k_rows, kcache->scale, q->data, B * g, ws.proxy_q, B, q->dtype};
+      if ((rc = check_cuda(launch_scan_tc(op, ws.rows + B, B * g, 1, tc_scratch(ws), sm_count(), st)))) return rc;
+    }
   }
   mark(3, st);
   if (mode == PIVOT_REFINE && o && o->impl == 1) {
@@ -371,6 +384,21 @@ int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_ten
   }
   mark(4, st);
   return check_cuda(cudaGetLastError());
+}
+
+int pivot_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                          const int32_t* pos0, int B, int Lmax, int H_I, int d, int g, int c, int k,
+                          int mode, int32_t* out_idx, pivot_stream_t stream, const pivot_opts* o) {
+  return run_decode(q, w, kcache, pos0, B, Lmax, H_I, d, g, c, k, mode, out_idx, stream, o, nullptr, 0);
+}
+
+int pivot_index_decode_paged(const pivot_tensor* q, const float* w, const pivot_tensor* kpages,
+                             const int32_t* block_table, const int32_t* pos0, int B, int max_pages,
+                             int n_pages, int H_I, int d, int g, int c, int k, int mode, int32_t* out_idx,
+                             pivot_stream_t stream, const pivot_opts* o) {
+  if (!block_table || max_pages < 1 || max_pages > (1 << 23)) return PIVOT_ERR_INVALID_ARG;
+  return run_decode(q, w, kpages, pos0, B, max_pages * 128, H_I, d, g, c, k, mode, out_idx, stream, o,
+                    block_table, n_pages);
 }
 
 int pivot_index_decode(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,

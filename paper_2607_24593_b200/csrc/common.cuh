@@ -56,6 +56,8 @@ struct RowDesc {
   int q_map;            // which query tensor map holds q: 0 raw queries, 1 proxies
   int q_row;            // query row (units of H x d) inside that tensor
   int k_row0;           // first row of this sequence's keys inside the key-cache tensor
+  // Paged key cache (decode): key tile t of this row is pool page pages[t]; nullptr = contiguous.
+  const int32_t* pages = nullptr;
 };
 
 }  // namespace pivot

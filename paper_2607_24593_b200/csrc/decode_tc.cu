@@ -131,16 +131,19 @@ decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
           ++blk;
           cur_b = b;
         }
+        // Row of the tile inside the key tensor.  Paged cache: the sequence's block table names
+        // the pool page (a page outside the pool reads as zero fill, like any out-of-range box).
+        const int32_t* pages = prox[b].pages;
+        const int krow = pages ? __ldg(pages + t) * TILE_KEYS : prox[b].k_row0 + t * TILE_KEYS;
         const int s = it % C::STAGES;
         if (!ptx::mbar_wait(&ct.empty[s], ((it / C::STAGES) & 1) ^ 1, abort_flag, 64)) break;
         ptx::mbar_arrive_expect_tx(&ct.full[s], C::STAGE_BYTES);
         for (int h = 0; h < C::KHALVES; ++h)
-          ptx::tma_load_2d(kring + s * C::STAGE_BYTES + h * C::HALF_TILE_BYTES, &tm_k, h * 64,
-                           prox[b].k_row0 + t * TILE_KEYS, &ct.full[s]);
+          ptx::tma_load_2d(kring + s * C::STAGE_BYTES + h * C::HALF_TILE_BYTES, &tm_k, h * 64, krow, &ct.full[s]);
         if (C::FP8) {
           const int ksl = it % DKS_SLOTS;       // free by construction (see the prefill scan)
           ptx::mbar_arrive_expect_tx(&ct.ks_full[ksl], TILE_KEYS * 4);
-          ptx::tma_load_1d(&ct.ks[ksl][0], &tm_ks, prox[b].k_row0 + t * TILE_KEYS, &ct.ks_full[ksl]);
+          ptx::tma_load_1d(&ct.ks[ksl][0], &tm_ks, krow, &ct.ks_full[ksl]);
         }
       }
     }
@@ -461,8 +464,8 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   ++launch_counter();
   CUtensorMap mk, mq, mks;
   memset(&mks, 0, sizeof(mks));
-  if (d.dtype == DT_FP8 && !make_scale_map(&mks, d.kscale, (long long)d.B * d.Lmax)) return cudaErrorInvalidValue;
-  if (!make_operand_map(&mk, d.kc, (long long)d.B * d.Lmax, d.dtype, TILE_KEYS) ||
+  if (d.dtype == DT_FP8 && !make_scale_map(&mks, d.kscale, d.k_rows)) return cudaErrorInvalidValue;
+  if (!make_operand_map(&mk, d.kc, d.k_rows, d.dtype, TILE_KEYS) ||
       !make_operand_map(&mq, d.proxy_q, (long long)d.B * kHeads, d.dtype, kHeads))
     return cudaErrorInvalidValue;
   if (d.ev_scan_begin) cudaEventRecord(d.ev_scan_begin, st);

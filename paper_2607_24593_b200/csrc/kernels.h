@@ -31,6 +31,10 @@ struct GroupDesc {
   unsigned long long* ent_out;
   int ent_stride;
   int slot0;
+  // Paged key cache (decode): kbase / kscale are the page pool and key position s lives in pool
+  // row pages[s / 128] * 128 + s % 128; pages == nullptr means one contiguous cache.
+  const int32_t* pages = nullptr;
+  int n_pages = 0;      // pages in the pool (entries outside [0, n_pages) are treated as holes)
 };
 
 constexpr int kDecodeCandChunk = 512;   // candidates per re-score work item in decode
@@ -67,6 +71,8 @@ struct DecodePlan {
   int32_t* cand; float* cand_score;                     // [B, c]
   int32_t* out; float* out_score;                       // [B, g, k]
   int B, Lmax, g, c, k, mode, dtype, guard_len;
+  const int32_t* block_table = nullptr;                 // paged cache: [B, Lmax / 128] pool pages
+  int n_pages = 0;
 };
 
 struct ScanScratch {
@@ -112,6 +118,7 @@ struct DecodeFast {
   const GroupDesc* groups;    // [B * group_chunks(g)]
   const void* kc; const float* kscale; const void* q; const void* proxy_q;
   int B, Lmax, g, c, k, mode, dtype, sms;
+  long long k_rows;           // rows of the key tensor (B * Lmax, or pool pages * 128 when paged)
   void* scratch;              // decode_fast_bytes(...) bytes
   ScanScratch scratch_tc;     // candidate scratch of the re-score kernel
   int* status;

@@ -123,8 +123,11 @@ __global__ void plan_decode_kernel(DecodePlan p, RowDesc* rows, GroupDesc* group
   const int p0 = p.pos0[b];
   const int n0 = p0 + 1;
   const bool guarded = n0 < p.guard_len;
-  const void* kb = (const char*)p.kc + (size_t)b * p.Lmax * kDim * esz;
-  const float* ksb = p.kscale ? p.kscale + (size_t)b * p.Lmax : nullptr;
+  // Paged cache: descriptors point at the page pool and carry the sequence's block-table row.
+  const bool paged = p.block_table != nullptr;
+  const int32_t* pages = paged ? p.block_table + (size_t)b * (p.Lmax / 128) : nullptr;
+  const void* kb = paged ? p.kc : (const char*)p.kc + (size_t)b * p.Lmax * kDim * esz;
+  const float* ksb = !p.kscale ? nullptr : paged ? p.kscale : p.kscale + (size_t)b * p.Lmax;
   int32_t* outb = p.out + (size_t)b * p.g * p.k;
   float* outsb = p.out_score ? p.out_score + (size_t)b * p.g * p.k : nullptr;
   RowDesc r;
@@ -134,8 +137,11 @@ __global__ void plan_decode_kernel(DecodePlan p, RowDesc* rows, GroupDesc* group
   r.kbase = kb;
   r.kscale = ksb;
   r.n_vis = n0;
-  r.q_map = 1; r.q_row = b; r.k_row0 = b * p.Lmax;
+  r.q_map = 1; r.q_row = b; r.k_row0 = paged ? 0 : b * p.Lmax;
+  r.pages = pages;
   GroupDesc gd;
+  gd.pages = pages;
+  gd.n_pages = p.n_pages;
   gd.q = (const char*)p.q + (size_t)b * p.g * qrow;
   gd.w = p.w + (size_t)b * p.g * kHeads;
   gd.qscale = p.qscale ? p.qscale + (size_t)b * p.g * kHeads : nullptr;

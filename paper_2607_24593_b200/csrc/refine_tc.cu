@@ -258,35 +258,46 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       const GroupDesc gd = groups[gi];
       const int ntiles = group_tiles(gd);
       if (ntiles == 0) continue;
-      // Candidate positions are fetched two tiles ahead and key scales one tile ahead, so
-      // neither round trip sits on this thread's issue path.
+      // Candidate positions are fetched three tiles ahead, their rows in the key tensor (a
+      // block-table lookup when the cache is paged) two tiles ahead and key scales one tile
+      // ahead, so no round trip sits on this thread's issue path.
       auto load_idx = [&](int tile, int half) -> int {
         const int sl = tile * TILE_KEYS + half * 64 + j;
         return (tile < ntiles && sl < gd.n_cand) ? __ldg(gd.cand + sl) : -1;
       };
-      auto load_ks = [&](int ix) -> float { return (gd.kscale && ix >= 0) ? __ldg(gd.kscale + ix) : 1.f; };
+      auto key_row = [&](int ix) -> int {      // -1: padding slot, or a page outside the pool
+        if (!gd.pages || ix < 0) return ix;
+        const uint32_t pg = (uint32_t)__ldg(gd.pages + (ix >> 7));
+        return pg < (uint32_t)gd.n_pages ? (int)(pg * 128u + (uint32_t)(ix & 127)) : -1;
+      };
+      auto load_ks = [&](int row) -> float { return (gd.kscale && row >= 0) ? __ldg(gd.kscale + row) : 1.f; };
       int idx0[2] = {load_idx(0, 0), load_idx(0, 1)}, idx1[2] = {load_idx(1, 0), load_idx(1, 1)};
-      float ks0[2] = {load_ks(idx0[0]), load_ks(idx0[1])};
+      int idx2[2] = {load_idx(2, 0), load_idx(2, 1)};
+      int row0[2] = {key_row(idx0[0]), key_row(idx0[1])}, row1[2] = {key_row(idx1[0]), key_row(idx1[1])};
+      float ks0[2] = {load_ks(row0[0]), load_ks(row0[1])};
       for (int t = 0; t < ntiles; ++t, ++it) {
         const int s = it % C::STAGES;
         const uint32_t ph = (it / C::STAGES) & 1;
-        const int idx2[2] = {load_idx(t + 2, 0), load_idx(t + 2, 1)};
-        const float ks1[2] = {load_ks(idx1[0]), load_ks(idx1[1])};
+        const int idx3[2] = {load_idx(t + 3, 0), load_idx(t + 3, 1)};
+        const int row2[2] = {key_row(idx2[0]), key_row(idx2[1])};
+        const float ks1[2] = {load_ks(row1[0]), load_ks(row1[1])};
         if (ok) ok = ptx::mbar_wait(&ct.empty[s], ph ^ 1, abort_flag, 64);   // whole warps wait here: sleep, do not spin
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
           const int row = half * 64 + j;
-          ct.meta[it % META_SLOTS][row] = KeyMeta{idx0[half], ks0[half]};
-          const int idx = idx0[half] < 0 ? 0 : idx0[half];
+          ct.meta[it % META_SLOTS][row] = KeyMeta{row0[half] < 0 ? -1 : idx0[half], ks0[half]};
+          const int krow = row0[half] < 0 ? 0 : row0[half];
           const uint32_t swz = (uint32_t)(row & 7);
-          const uint8_t* src = (const uint8_t*)gd.kbase + (size_t)idx * C::ROW_BYTES;
+          const uint8_t* src = (const uint8_t*)gd.kbase + (size_t)krow * C::ROW_BYTES;
           const uint32_t dst = ptx::smem_u32(kring + s * C::STAGE_BYTES) + (uint32_t)row * 128u;
 #pragma unroll
           for (int h = 0; h < C::KHALVES; ++h)
 #pragma unroll
             for (int cidx = 0; cidx < 8; ++cidx)
               cp_async16(dst + h * C::HALF_TILE_BYTES + ((cidx ^ swz) << 4), src + h * 128 + cidx * 16);
-          idx0[half] = idx1[half]; idx1[half] = idx2[half]; ks0[half] = ks1[half];
+          idx0[half] = idx1[half]; idx1[half] = idx2[half]; idx2[half] = idx3[half];
+          row0[half] = row1[half]; row1[half] = row2[half];
+          ks0[half] = ks1[half];
         }
         cp_async_commit();
         if (it + 1 - pub > (uint32_t)C::LOOKAHEAD) {

@@ -129,6 +129,47 @@ def test_decode_group_of_four(pv, gu):
                      out_scores=sc, cand=cand, cand_scores=cs)
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+@pytest.mark.parametrize("mode", [po.MODE_REUSE, po.MODE_REFINE])
+def test_decode_paged_matches_contiguous(pv, gu, dtype, mode):
+    """Paged key cache: same step as the contiguous cache with the guardrail off, page by page
+    scattered over a pool -- oracle parity, and the same positions as the contiguous call."""
+    x = inputs.make_decode(5, 2, 200, 3000, dtype=dtype, seed=23)     # some sequences shorter than c
+    out, sc, cand, cs = gu.run_decode_paged(x, c=512, k=256, mode=mode, seed=5)
+    t = acc.check_decode(x.codes(), c=512, k=256, mode=mode, guard_len=0, out_idx=out, out_scores=sc,
+                         cand=cand, cand_scores=cs)
+    _report(f"decode paged {dtype} mode={mode}", t)
+    ref, _, rcand, _ = gu.run_decode(x, c=512, k=256, mode=mode, guard_len=0)
+    assert np.array_equal(np.sort(out, axis=2), np.sort(ref, axis=2))
+    if cand is not None:
+        assert np.array_equal(np.sort(cand, axis=1), np.sort(rcand, axis=1))
+
+
+def test_decode_paged_bad_page_is_a_hole(pv, gu):
+    """A block-table entry outside the pool faults nothing: the page's keys are never returned by
+    Refine (the scan sees zeros there, the re-score drops them)."""
+    x = inputs.make_decode(2, 2, 1500, 2000, dtype="fp8", seed=24)
+    out, _, _, _ = gu.run_decode_paged(x, c=512, k=256, mode=po.MODE_REFINE, seed=6, bad_entry=(1, 3))
+    hole = (out[1] >= 3 * 128) & (out[1] < 4 * 128)
+    assert not hole.any()
+    assert (out[0] >= 0).all()
+
+
+def test_decode_paged_argument_errors(pv):
+    x = inputs.make_decode(2, 2, 300, 600, dtype="bf16", seed=25)
+    q, w, k, pos0 = x.q.cuda(), x.w.cuda(), x.k.cuda(), x.pos0.cuda()
+    B, g = 2, 2
+    mp = k.shape[1] // 128
+    pool = k[:, : mp * 128].reshape(B * mp * 128, 128).contiguous()
+    bt = torch.arange(B * mp, dtype=torch.int32, device="cuda").reshape(B, mp)
+    out = torch.empty((B, g, 64), dtype=torch.int32, device="cuda")
+    with pytest.raises(pv.PivotError, match="invalid"):
+        pv.pivot_index_decode_paged(q, w, pool, bt, pos0, B, mp, 0, 64, 128, g, 128, 64, pv.REFINE, out)   # empty pool
+    with pytest.raises(pv.PivotError, match="invalid"):
+        pv.pivot_index_decode_paged(q, w, pool, bt, pos0, B, mp, B * mp, 64, 128, g, 128, 64, pv.REFINE, out,
+                                    impl=pv.IMPL_CUDA_CORE)
+
+
 # ---------------------------------------------------------------- argument errors (host side)
 
 def test_argument_errors(pv):
