@@ -399,12 +399,13 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
                 else ptx::tmem_ld_32x32_async(xb + (c + 1) * 32, vb);
               }
               uint32_t pk[16];
-              const bool have_row = (c >> 1) < gd.m;           // members missing from the group: zeros
 #pragma unroll
-              for (int i = 0; i < 16; ++i) {
+              for (int i = 0; i < 16; ++i)
                 pk[i] = (c & 1) ? ptx::relu_pack_bf16x2(__uint_as_float(vb[2 * i]), __uint_as_float(vb[2 * i + 1]))
                                 : ptx::relu_pack_bf16x2(__uint_as_float(va[2 * i]), __uint_as_float(va[2 * i + 1]));
-                pk[i] = have_row ? pk[i] : 0u;
+              if ((c >> 1) >= gd.m) {                          // members missing from the group: zeros (warp-uniform)
+#pragma unroll
+                for (int i = 0; i < 16; ++i) pk[i] = 0u;
               }
               ptx::tmem_st_32x16(xb + c * 16, pk);
             }
