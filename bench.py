@@ -226,6 +226,16 @@ def decode_bench(pv, dev, steps, warmup, pk):
         paged_scan.append(pv.pivot_stage_times()["decode_scan"] * 1e3)
     pv.pivot_stage_timing(False)
     assert pv.pivot_device_status() == 0
+    # ... and with the local window of Appendix B (decode form, the paper's W = 4)
+    def step_window():
+        pv.pivot_index_decode(q, w, kc, p0, B, Lmax, H, D, g, c, k, pv.REFINE, out_p, stream, q_scale=qs, k_scale=ks,
+                              W=4)
+
+    for _ in range(warmup):
+        step_window()
+    torch.cuda.synchronize()
+    window_times = timed(step_window, steps)
+    assert pv.pivot_device_status() == 0
     us = float(np.median(times))
     scan = float(np.mean(scan_us))
     n0 = (x.pos0.numpy().astype(np.int64) + 1)
@@ -235,6 +245,7 @@ def decode_bench(pv, dev, steps, warmup, pk):
             "graph_replay_us": graph_us, "graph_note": graph_note,
             "paged": {"value": float(np.median(paged_times)), "unit": "us", "scan_kernel_us": float(np.mean(paged_scan)),
                       "page_keys": 128, "pool_pages": B * mp, "same_positions_as_contiguous": same},
+            "local_window": {"W": 4, "value": float(np.median(window_times)), "unit": "us"},
             "config": {"workload": "decode_mtp_b32_64k-128k_fp8_g2_refine", "B": B, "g": g, "c": c, "k": k,
                        "visible_keys": int(n0.sum()), "l2": "256 MB flush between steps"},
             # dominant kernel: the key-streaming scan; algorithmic bytes = visible keys x 132 B

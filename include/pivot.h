@@ -94,14 +94,19 @@ typedef struct pivot_tensor {
  *                 Both 0 = all rows.  row_begin must be a multiple of g, row_end a multiple of g
  *                 or L.  Tensor arguments keep their full-request shapes; a chunk's result is the
  *                 same as the corresponding rows of one whole call (groups never straddle chunks).
- *   W             prefill only: local window of Appendix B (0 = off, the default; the paper's
- *                 setting is 4).  The proxy scan of a group at t0 then ranks the keys s <= t0 - W
+ *   W             local window of Appendix B (0 = off, the default; the paper's setting is 4).
+ *                 Prefill: the proxy scan of a group at t0 then ranks the keys s <= t0 - W
  *                 only.  Refine: the proxy fills c - (W + m - 1) candidate slots (m = members of
  *                 the group) and the last W + m - 1 slots hold the window positions
  *                 t0-W+1 .. t0+m-1 in ascending order; every member re-scores all slots and
  *                 ignores window slots beyond its own position.  Reuse: the shared top-k comes
  *                 from the shortened scan.  Needs W + g - 1 < c and a guardrail of at least
- *                 W + g (the default c is); not available in decode calls or with impl = 1.
+ *                 W + g (the default c is).
+ *                 Decode (Refine only): the pool is still the proxy's top-c over s <= pos0, and
+ *                 the query at t re-scores pool U [t-W+1, t] (duplicates counted once).  Needs
+ *                 W >= g (the window then covers the keys written inside the step) and
+ *                 W + g - 1 <= 512.  Sequences under the guardrail are scored densely as usual.
+ *                 Not available with impl = 1.
  */
 typedef struct pivot_opts {
   int guard_len;

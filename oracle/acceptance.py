@@ -84,16 +84,21 @@ def check_selection(got_idx, scores, index, K, rtol, tally: Tally, what="", got_
 
 
 def check_group(x: dict, kd, kscale, members, *, c, k, mode, guard_len, out_idx, out_scores=None,
-                cand=None, cand_scores=None, q_rows=None, pool="mean", W=0) -> Tally:
+                cand=None, cand_scores=None, q_rows=None, pool="mean", W=0, per_query_window=False) -> Tally:
     """Checks one group's rows of out_idx ([m, k]) (and candidates [c]) against the oracle.
 
     With a local window (Appendix B, W > 0) the proxy part of the candidate set is checked
     against the shortened scan, the window slots must hold t0-W+1 .. t0+m-1 in ascending order,
-    and every member is checked on the slots it may see (positions <= its own)."""
+    and every member is checked on the slots it may see (positions <= its own).
+    per_query_window (decode form): `cand` is the pool of c entries, checked as for W = 0, and
+    each member is checked on the produced pool united with its own window [t-W+1, t]."""
     rtol = RTOL[x["dtype"]]
     t = Tally()
     r = po.pivot_group(x, members, kd, kscale, c=c, k=k, mode=mode, guard_len=guard_len, pool=pool,
-                       q_rows=q_rows, W=W)
+                       q_rows=q_rows, W=W, per_query_window=per_query_window)
+    W_own = W if per_query_window else 0
+    if per_query_window:
+        W = 0                      # pool and scan are those of the plain method
     m = len(r.members)
     if r.guarded:
         for i, tq in enumerate(r.members):
@@ -122,8 +127,12 @@ def check_group(x: dict, kd, kscale, members, *, c, k, mode, guard_len, out_idx,
     qs = None if x["qscale"] is None else x["qscale"][rows]
     qd, weff = po.member_operands(x["q"][rows], qs, x["w"][rows], x["dtype"])
     for i, tq in enumerate(r.members):
-        s, _, ok = po.refine_on_candidates(qd[i], weff[i], kd, kscale, C, k, t_member=int(tq) if w_g else None)
-        check_selection(out_idx[i], s[ok], C[ok], k, rtol, t, f"refine row t={tq}",
+        Ci = C
+        if W_own:
+            win = np.arange(max(int(tq) - W_own + 1, 0), int(tq) + 1, dtype=np.int64)
+            Ci = np.concatenate([C, np.setdiff1d(win, C)])
+        s, _, ok = po.refine_on_candidates(qd[i], weff[i], kd, kscale, Ci, k, t_member=int(tq) if w_g else None)
+        check_selection(out_idx[i], s[ok], Ci[ok], k, rtol, t, f"refine row t={tq}",
                         None if out_scores is None else out_scores[i])
     return t
 
@@ -155,7 +164,7 @@ def check_dense(x: dict, *, k, out_idx, out_scores=None, rows=None) -> Tally:
 
 
 def check_decode(x: dict, *, c, k, mode, guard_len, out_idx, out_scores=None, cand=None,
-                 cand_scores=None, seqs=None) -> Tally:
+                 cand_scores=None, seqs=None, W=0) -> Tally:
     B, g = x["q"].shape[0], x["q"].shape[1]
     total = Tally()
     for b in (range(B) if seqs is None else seqs):
@@ -169,5 +178,6 @@ def check_decode(x: dict, *, c, k, mode, guard_len, out_idx, out_scores=None, ca
             xb, kd, ks, np.arange(p0, p0 + g), c=c, k=k, mode=mode, guard_len=guard_len,
             out_idx=out_idx[b], out_scores=None if out_scores is None else out_scores[b],
             cand=None if cand is None else cand[b],
-            cand_scores=None if cand_scores is None else cand_scores[b], q_rows=np.arange(g)))
+            cand_scores=None if cand_scores is None else cand_scores[b], q_rows=np.arange(g),
+            W=W, per_query_window=W > 0))
     return total

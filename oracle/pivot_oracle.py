@@ -9,7 +9,9 @@ What it computes, with the passage each function follows:
   top_set             TopK of Eq. 1 / 6 / 7 / 9, total order (score desc, index asc)
   build_proxy         Eq. 4 (per-head mean of queries and gates over the group)
   pivot_group         Algorithm 1, one group: guardrail, Eq. 5 scan, Eq. 6 Reuse, Eq. 7-9 Refine,
-                      local window of Appendix B when W > 0
+                      local window of Appendix B when W > 0 (prefill form: one shared candidate
+                      set with reserved window slots; decode form: pool united with each query's
+                      own window)
   refine_on_candidates Eq. 8-9 on a candidate set supplied from outside
   pivot_prefill / pivot_decode / dense_index   drivers over groups (Eq. 2 / Eq. 3 grouping)
 
@@ -32,9 +34,11 @@ Readings taken where the paper is silent (each also listed in the design notes):
 
 Pins: every function is pinned by tests that do not call it to produce their expectation
 (hand-worked example, torch einsum/topk restatement, g = 1 identity, c >= n0 identity,
-identical-member identity, coverage identity, brute-force select, codec tables).  The window
-variant's slot layout rests on the reading above alone: parity unpinned for W > 0 beyond the
-W = 0 reduction and the containment/coverage invariants.
+identical-member identity, coverage identity, brute-force select, codec tables).  The prefill
+window variant's slot layout rests on the reading above alone: parity unpinned for W > 0 beyond
+the W = 0 reduction and the containment/coverage invariants.  The decode window variant is
+pinned by its reduction to the dense definition when pool and window cover every visible key,
+and by a set-membership restatement of "pool united with the query's own window".
 """
 from __future__ import annotations
 
@@ -201,6 +205,7 @@ class GroupResult:
     proxy_scores: np.ndarray | None = None   # [n0] float64, Eq. 5
     member_scores: np.ndarray | None = None  # Refine: [m, |C|] float64 (Eq. 8); guarded: list of [t+1]
     C_mask: np.ndarray | None = None    # [m, |C|] bool, False where a window slot lies beyond t
+    member_C: list | None = None        # decode window form: each member's own candidate positions
 
 
 def refine_on_candidates(qd, weff, kd_all, kscale_all, C: np.ndarray, k: int, t_member=None):
@@ -222,8 +227,11 @@ def refine_on_candidates(qd, weff, kd_all, kscale_all, C: np.ndarray, k: int, t_
 
 def pivot_group(x: dict, members: np.ndarray, kd: np.ndarray, kscale, *, c: int, k: int, mode: int,
                 guard_len: int | None = None, W: int = 0, pool: str = "mean",
-                q_rows: np.ndarray | None = None) -> GroupResult:
+                q_rows: np.ndarray | None = None, per_query_window: bool = False) -> GroupResult:
     """Algorithm 1 for one group.
+
+    per_query_window selects the decode form of Appendix B's local window: the scan and the
+    pool C are those of W = 0, and the member at t refines over C united with [t-W+1, t].
 
     x: dict with "dtype", "q" [.., H, d] codes, "qscale", "w" indexed by q_rows (defaults to
     `members`, the query positions; decode passes slot indices instead).  kd / kscale: decoded
@@ -250,9 +258,9 @@ def pivot_group(x: dict, members: np.ndarray, kd: np.ndarray, kscale, *, c: int,
 
     pq_codes, pweff = build_proxy(x["q"][rows], qs, x["w"][rows], dtype, pool)        # Eq. 4
     pqd = decode_operand(pq_codes, dtype)
-    # Eq. 5: one scan, cut at the group's first position (t0 - W with a window: the window
-    # part then covers the rest without duplicates)
-    n_scan = n0 if W == 0 else max(t0 - W + 1, 0)
+    # Eq. 5: one scan, cut at the group's first position (prefill form of the window: t0 - W,
+    # the window part then covers the rest without duplicates)
+    n_scan = n0 if (W == 0 or per_query_window) else max(t0 - W + 1, 0)
     pscores = indexer_scores(pqd, pweff, kd[:n_scan], None if kscale is None else kscale[:n_scan])
 
     if mode == MODE_REUSE:                           # Eq. 6: the proxy top-k serves every member
@@ -262,6 +270,19 @@ def pivot_group(x: dict, members: np.ndarray, kd: np.ndarray, kscale, *, c: int,
 
     # Refine.  Eq. 7 candidate set; with a window, the proxy fills c - w_g slots and the
     # union of the members' windows [t0-W+1, t0+m-1] takes the rest (Appendix B).
+    if W > 0 and per_query_window:
+        # decode form: every query keeps the pool and adds its own W most recent positions
+        C = top_set(pscores, c)
+        T = np.empty((m, k), np.int32)
+        ms, member_C = [], []
+        for i, t in enumerate(members):
+            win = np.arange(max(int(t) - W + 1, 0), int(t) + 1, dtype=np.int64)
+            Ci = np.concatenate([C, win[~np.isin(win, C)]])          # duplicates counted once
+            s, Ti, _ = refine_on_candidates(qd[i], weff[i], kd, kscale, Ci, k)
+            T[i] = _pad(Ti, k)
+            ms.append(s)
+            member_C.append(Ci)
+        return GroupResult(t0, members, False, T, C=C, proxy_scores=pscores, member_scores=ms, member_C=member_C)
     if W == 0:
         C = top_set(pscores, c)
     else:
@@ -300,9 +321,9 @@ def pivot_decode(x: dict, *, c: int, k: int, mode: int, guard_len=None, W: int =
     """Algorithm 1 in decode (Eq. 3): sequence b's group is its g queries at positions
     pos0_b .. pos0_b + g - 1, scanned against that sequence's own key cache, cut at pos0_b.
     Returns {b: GroupResult}."""
-    if W:
-        raise NotImplementedError("decode window (pool united with each query's own window) not built")
     B, g = x["q"].shape[0], x["q"].shape[1]
+    if W and W < g:
+        raise ValueError("the decode window must cover the step: W >= g (Appendix B)")
     out = {}
     for b in (range(B) if seqs is None else seqs):
         p0 = int(x["pos0"][b])
@@ -312,7 +333,8 @@ def pivot_decode(x: dict, *, c: int, k: int, mode: int, guard_len=None, W: int =
         xb = dict(dtype=x["dtype"], q=x["q"][b], qscale=None if x["qscale"] is None else x["qscale"][b],
                   w=x["w"][b])
         out[b] = pivot_group(xb, np.arange(p0, p0 + g), kd, ks, c=c, k=k, mode=mode,
-                             guard_len=guard_len, W=W, pool=pool, q_rows=np.arange(g))
+                             guard_len=guard_len, W=W, pool=pool, q_rows=np.arange(g),
+                             per_query_window=True)
     return out
 
 

@@ -207,13 +207,13 @@ def dense_index_static(q, w, kcache, L, H_I, d, k, out_idx, stream=None, *, q_sc
 
 def pivot_index_decode(q, w, kcache, pos0, B, Lmax, H_I, d, g, c, k, mode, out_idx, stream=None, *,
                        q_scale=None, k_scale=None, guard_len=None, pool=POOL_MEAN, dbg_cand=None,
-                       dbg_scores=None, dbg_cand_scores=None, workspace=None, impl=0):
+                       dbg_scores=None, dbg_cand_scores=None, workspace=None, impl=0, W=0):
     tq, tk = _tensor(q, q_scale), _tensor(kcache, k_scale)
     assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and pos0.dtype == torch.int32
     assert out_idx.numel() >= B * g * k
     if workspace is None:
         ensure_workspace(B * g, B, c, k, q.device, need=pivot_decode_workspace_bytes(B, Lmax, g, c, k))
-    o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl)
+    o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl, W=W)
     _check(lib.pivot_index_decode_ex(C.byref(tq), w.data_ptr(), C.byref(tk), pos0.data_ptr(), B, Lmax,
                                      H_I, d, g, c, k, mode, out_idx.data_ptr(), _stream(stream), C.byref(o)))
     return out_idx
@@ -221,14 +221,14 @@ def pivot_index_decode(q, w, kcache, pos0, B, Lmax, H_I, d, g, c, k, mode, out_i
 
 def pivot_index_decode_paged(q, w, kpages, block_table, pos0, B, max_pages, n_pages, H_I, d, g, c, k, mode,
                              out_idx, stream=None, *, q_scale=None, k_scale=None, pool=POOL_MEAN, dbg_cand=None,
-                             dbg_scores=None, dbg_cand_scores=None, workspace=None, impl=0):
+                             dbg_scores=None, dbg_cand_scores=None, workspace=None, impl=0, W=0):
     tq, tk = _tensor(q, q_scale), _tensor(kpages, k_scale)
     assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and pos0.dtype == torch.int32
     assert block_table.dtype == torch.int32 and block_table.is_contiguous() and block_table.numel() >= B * max_pages
     assert out_idx.numel() >= B * g * k
     if workspace is None:
         ensure_workspace(B * g, B, c, k, q.device, need=pivot_decode_workspace_bytes(B, max_pages * 128, g, c, k))
-    o = _opts(None, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl)
+    o = _opts(None, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl, W=W)
     _check(lib.pivot_index_decode_paged(C.byref(tq), w.data_ptr(), C.byref(tk), block_table.data_ptr(),
                                         pos0.data_ptr(), B, max_pages, n_pages, H_I, d, g, c, k, mode,
                                         out_idx.data_ptr(), _stream(stream), C.byref(o)))

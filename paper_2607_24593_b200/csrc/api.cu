@@ -322,7 +322,12 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
   if (!pos0 || B < 1 || g < 1 || Lmax < g) return PIVOT_ERR_INVALID_ARG;
   // every sequence's scale row must start on a 16-byte boundary (TMA reads it in 128-scale tiles)
   if (q->dtype == PIVOT_FP8_E4M3 && (Lmax & 3)) return PIVOT_ERR_INVALID_ARG;
-  if (o && (o->pool < 0 || o->pool > 2 || o->W != 0)) return PIVOT_ERR_INVALID_ARG;
+  if (o && (o->pool < 0 || o->pool > 2)) return PIVOT_ERR_INVALID_ARG;
+  // local window, decode form (Appendix B): every query adds its own last W positions to the
+  // pool, so W must cover the step (W >= g); Refine only
+  const int W = o ? o->W : 0;
+  if (W < 0 || (W > 0 && (mode != PIVOT_REFINE || W < g || W + g - 1 > kDecodeWinMax || o->impl == 1)))
+    return PIVOT_ERR_INVALID_ARG;
   const bool paged = block_table != nullptr;
   if (paged && (n_pages < 1 || (Lmax & 127) || (o && o->impl == 1))) return PIVOT_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
@@ -364,6 +369,7 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
     df.kc = kcache->data; df.kscale = kcache->scale; df.q = q->data; df.proxy_q = ws.proxy_q;
     df.B = B; df.Lmax = Lmax; df.g = g; df.c = c; df.k = k; df.mode = mode; df.dtype = q->dtype;
     df.k_rows = k_rows;
+    df.W = W;
     df.sms = sm_count();
     df.scratch = (char*)wsp + base_bytes;
     df.scratch_tc = tc_scratch(ws);

@@ -13,6 +13,9 @@
 //                        refined 12 bits at a time with further passes over the scores; the
 //                        survivors are collected in shared memory and the exact top-K (Eq. 6 / 7)
 //                        is taken there.
+//   decode_window_kernel (only with a local window, Appendix B) the union of the step's per-query
+//                        windows as one more candidate chunk per sequence, minus the positions
+//                        the pool already holds.
 //   entries_topk_kernel  exact top-k (Eq. 9) of each query's re-scored candidates, which the
 //                        gather + re-score kernel leaves as packed entries (refine_tc.cu, chunked
 //                        over candidates so that all SMs take part).
@@ -373,8 +376,8 @@ __global__ void __launch_bounds__(kBlk, 1) entries_topk_kernel(const EntryList* 
 // ------------------------------------------------------------------------------ setup
 
 __global__ void decode_setup_kernel(const RowDesc* __restrict__ prox, const GroupDesc* __restrict__ groups, int B,
-                                    int g, int c, int k, int mode, int* tile_prefix, GroupDesc* chunks,
-                                    EntryList* lists, unsigned long long* entries) {
+                                    int g, int c, int k, int mode, int W, int* tile_prefix, GroupDesc* chunks,
+                                    EntryList* lists, unsigned long long* entries, const int32_t* wcand) {
   __shared__ int tiles[1024];
   const int tid = threadIdx.x;
   for (int b = tid; b < B; b += blockDim.x)
@@ -390,27 +393,62 @@ __global__ void decode_setup_kernel(const RowDesc* __restrict__ prox, const Grou
   // each leaving packed entries; one entry list per query for the final top-k.
   const int mc = (g + kMembersPerDesc - 1) / kMembersPerDesc;
   const int ncc = (c + kDecodeCandChunk - 1) / kDecodeCandChunk;
-  for (int i = tid; i < B * mc * ncc; i += blockDim.x) {
-    const int gi = i / ncc, cc = i % ncc;
+  const int nch = ncc + (W > 0 ? 1 : 0);           // with a window: one more chunk, the window slots
+  const int w_g = W > 0 ? W + g - 1 : 0;
+  const int stride = c + kDecodeWinMax;            // entries per query
+  for (int i = tid; i < B * mc * nch; i += blockDim.x) {
+    const int gi = i / nch, cc = i % nch;
     GroupDesc gd = groups[gi];
-    const int left = gd.n_cand - cc * kDecodeCandChunk;
-    gd.cand = gd.cand + cc * kDecodeCandChunk;
-    gd.n_cand = left > 0 ? (left < kDecodeCandChunk ? left : kDecodeCandChunk) : 0;
-    gd.ent_out = entries + (size_t)gd.q_row * c;
-    gd.ent_stride = c;
-    gd.slot0 = cc * kDecodeCandChunk;
+    gd.ent_out = entries + (size_t)gd.q_row * stride;
+    gd.ent_stride = stride;
+    if (cc < ncc) {
+      const int left = gd.n_cand - cc * kDecodeCandChunk;
+      gd.cand = gd.cand + cc * kDecodeCandChunk;
+      gd.n_cand = left > 0 ? (left < kDecodeCandChunk ? left : kDecodeCandChunk) : 0;
+      gd.slot0 = cc * kDecodeCandChunk;
+    } else {                 // window slots follow the pool's valid entries
+      gd.slot0 = gd.n_cand;
+      gd.cand = wcand + (size_t)(gi / mc) * kDecodeWinMax;
+      gd.n_cand = gd.n_cand > 0 ? w_g : 0;
+      gd.win_span = W;
+    }
     chunks[i] = gd;
   }
   for (int i = tid; i < B * g; i += blockDim.x) {
     const int b = i / g;
     const GroupDesc gd = groups[b * mc];
     EntryList el;
-    el.list = entries + (size_t)i * c;
-    el.n = gd.n_cand;
+    el.list = entries + (size_t)i * stride;
+    el.n = gd.n_cand > 0 ? gd.n_cand + w_g : 0;
     el.K = gd.n_cand > 0 ? k : 0;
     el.out = groups[b * mc].out + (size_t)(i - b * g) * gd.out_stride;
     el.out_score = gd.out_score ? groups[b * mc].out_score + (size_t)(i - b * g) * gd.out_stride : nullptr;
     lists[i] = el;
+  }
+}
+
+// Decode form of the local window (Appendix B): the queries of the step at pos0 .. pos0 + g - 1
+// each add their own window [t - W + 1, t] to the pool.  The union of those windows,
+// pos0 - W + 1 .. pos0 + g - 1, becomes one more candidate chunk of the sequence; positions the
+// pool already holds (and positions before the start of the sequence) are left out as -1, and
+// the re-score kernel masks every slot to the members whose window covers it.
+__global__ void decode_window_kernel(const GroupDesc* __restrict__ groups, int mc, int g, int W,
+                                     int32_t* __restrict__ wcand) {
+  __shared__ int dup[kDecodeWinMax];
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const GroupDesc gd = groups[b * mc];
+  if (gd.n_cand <= 0) return;                      // guarded sequence: scored densely
+  const int pos0 = gd.first_pos, lo = pos0 - W + 1, w_g = W + g - 1;
+  for (int j = tid; j < w_g; j += blockDim.x) dup[j] = 0;
+  __syncthreads();
+  for (int i = tid; i < gd.n_cand; i += blockDim.x) {
+    const int p = gd.cand[i];
+    if (p >= lo && p <= pos0) dup[p - lo] = 1;
+  }
+  __syncthreads();
+  for (int j = tid; j < w_g; j += blockDim.x) {
+    const int s = lo + j;
+    wcand[(size_t)b * kDecodeWinMax + j] = (s < 0 || dup[j]) ? -1 : s;
   }
 }
 
@@ -441,8 +479,8 @@ size_t decode_fast_bytes(int B, int Lmax, int g, int c) {
   const int mc = group_chunks(g);
   const int ncc = (c + kDecodeCandChunk - 1) / kDecodeCandChunk;
   return up((size_t)B * Lmax * 4) + up((size_t)B * DHIST * 4) + up((size_t)(B + 1) * 4) +
-         up((size_t)B * mc * ncc * sizeof(GroupDesc)) + up((size_t)B * g * sizeof(EntryList)) +
-         up((size_t)B * g * c * 8);
+         up((size_t)B * mc * (ncc + 1) * sizeof(GroupDesc)) + up((size_t)B * g * sizeof(EntryList)) +
+         up((size_t)B * kDecodeWinMax * 4) + up((size_t)B * g * (c + kDecodeWinMax) * 8);
 }
 
 cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
@@ -453,14 +491,17 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   int* tile_prefix = (int*)p;                p += up((size_t)(d.B + 1) * 4);
   const int mc = group_chunks(d.g);
   const int ncc = (d.c + kDecodeCandChunk - 1) / kDecodeCandChunk;
-  GroupDesc* chunks = (GroupDesc*)p;         p += up((size_t)d.B * mc * ncc * sizeof(GroupDesc));
+  const int W = d.mode == 1 ? d.W : 0;
+  const int nch = ncc + (W > 0 ? 1 : 0);
+  GroupDesc* chunks = (GroupDesc*)p;         p += up((size_t)d.B * mc * (ncc + 1) * sizeof(GroupDesc));
   EntryList* lists = (EntryList*)p;          p += up((size_t)d.B * d.g * sizeof(EntryList));
+  int32_t* wcand = (int32_t*)p;              p += up((size_t)d.B * kDecodeWinMax * 4);
   unsigned long long* entries = (unsigned long long*)p;
 
   cudaError_t e = cudaMemsetAsync(ghist, 0, (size_t)d.B * DHIST * 4, st);
   if (e != cudaSuccess) return e;
-  decode_setup_kernel<<<1, 1024, 0, st>>>(d.prox, d.groups, d.B, d.g, d.c, d.k, d.mode, tile_prefix, chunks, lists,
-                                          entries);
+  decode_setup_kernel<<<1, 1024, 0, st>>>(d.prox, d.groups, d.B, d.g, d.c, d.k, d.mode, W, tile_prefix, chunks,
+                                          lists, entries, wcand);
   ++launch_counter();
   CUtensorMap mk, mq, mks;
   memset(&mks, 0, sizeof(mks));
@@ -484,8 +525,12 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   decode_select_kernel<<<d.B, kBlk, sel_smem, st>>>(d.prox, d.Lmax, scores, ghist);
   ++launch_counter();
   if (d.mode == 1) {
+    if (W > 0) {
+      decode_window_kernel<<<d.B, 128, 0, st>>>(d.groups, mc, d.g, W, wcand);
+      ++launch_counter();
+    }
     ScanScratch sc = d.scratch_tc;
-    e = launch_refine_tc(d.q, d.B * d.g, d.dtype, chunks, d.B * mc * ncc, sc, d.sms, st);
+    e = launch_refine_tc(d.q, d.B * d.g, d.dtype, chunks, d.B * mc * nch, sc, d.sms, st);
     if (e != cudaSuccess) return e;
     entries_topk_kernel<<<d.B * d.g, kBlk, 0, st>>>(lists);
     ++launch_counter();

@@ -35,7 +35,12 @@ struct GroupDesc {
   // row pages[s / 128] * 128 + s % 128; pages == nullptr means one contiguous cache.
   const int32_t* pages = nullptr;
   int n_pages = 0;      // pages in the pool (entries outside [0, n_pages) are treated as holes)
+  // Per-query window slots (decode form of Appendix B): the member at position t takes a slot
+  // only if t - win_span < position <= t.  The default never excludes anything below t.
+  int win_span = 1 << 30;
 };
+
+constexpr int kDecodeWinMax = 512;      // most window slots (W + g - 1) of a decode step
 
 constexpr int kDecodeCandChunk = 512;   // candidates per re-score work item in decode
 
@@ -73,6 +78,7 @@ struct DecodePlan {
   int B, Lmax, g, c, k, mode, dtype, guard_len;
   const int32_t* block_table = nullptr;                 // paged cache: [B, Lmax / 128] pool pages
   int n_pages = 0;
+  int W = 0;                                            // per-query local window (Appendix B, decode form)
 };
 
 struct ScanScratch {
@@ -119,6 +125,7 @@ struct DecodeFast {
   const void* kc; const float* kscale; const void* q; const void* proxy_q;
   int B, Lmax, g, c, k, mode, dtype, sms;
   long long k_rows;           // rows of the key tensor (B * Lmax, or pool pages * 128 when paged)
+  int W = 0;                  // per-query local window (Appendix B, decode form); Refine only
   void* scratch;              // decode_fast_bytes(...) bytes
   ScanScratch scratch_tc;     // candidate scratch of the re-score kernel
   int* status;

@@ -365,10 +365,12 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         ct.w[r][jh] = 0.5f * wv;       // halved: see the ReLU identity in the tile loop
         tm.sync();
       }
-      // One member row's result: a key never seen by the member (beyond its own position: only
-      // window slots can be, Appendix B) or a padding slot counts as empty.
+      // One member row's result: a key never seen by the member (beyond its own position, or
+      // before its own window in a chunk of per-query window slots: Appendix B) or a padding
+      // slot counts as empty.
       auto put = [&](int r, int t, int slot, int idx, uint32_t key) {
-        const bool seen = idx >= 0 && idx <= gd.first_pos + r;
+        const int t_r = gd.first_pos + r;
+        const bool seen = idx >= 0 && idx <= t_r && idx + gd.win_span > t_r;
         if (smem_sel) {                // key only; the position is looked up again at the end
           if (r < gd.m) skey[r * SCORE_SLOTS + slot] = seen ? key : 0u;
           return;

@@ -42,7 +42,7 @@ def run_dense(x, *, k):
     return out.cpu().numpy(), scores.cpu().numpy()
 
 
-def run_decode(x, *, c, k, mode, guard_len=None):
+def run_decode(x, *, c, k, mode, guard_len=None, W=0):
     d = to_cuda(x)
     B, g, H, dd = x.q.shape
     Lmax = x.k.shape[1]
@@ -52,14 +52,14 @@ def run_decode(x, *, c, k, mode, guard_len=None):
     cs = torch.full((B, c), float("nan"), dtype=torch.float32, device="cuda") if cand is not None else None
     pv.pivot_index_decode(d["q"], d["w"], d["k"], d["pos0"], B, Lmax, H, dd, g, c, k, mode, out,
                           q_scale=d["qscale"], k_scale=d["kscale"], guard_len=guard_len, dbg_cand=cand,
-                          dbg_scores=scores, dbg_cand_scores=cs)
+                          dbg_scores=scores, dbg_cand_scores=cs, W=W)
     torch.cuda.synchronize()
     assert pv.pivot_device_status() == 0
     f = lambda t: None if t is None else t.cpu().numpy()
     return f(out), f(scores), f(cand), f(cs)
 
 
-def run_decode_paged(x, *, c, k, mode, seed=0, bad_entry=None):
+def run_decode_paged(x, *, c, k, mode, seed=0, bad_entry=None, W=0):
     """The same decode step over a paged copy of x's key cache: pages scattered over a pool by a
     seeded permutation, spare pool pages filled with large codes (a wrong page read shows up)."""
     d = to_cuda(x)
@@ -93,7 +93,7 @@ def run_decode_paged(x, *, c, k, mode, seed=0, bad_entry=None):
     cs = torch.full((B, c), float("nan"), dtype=torch.float32, device="cuda") if cand is not None else None
     pv.pivot_index_decode_paged(d["q"], d["w"], pool, bt, d["pos0"], B, mp, n_pages, H, dd, g, c, k, mode, out,
                                 q_scale=d["qscale"], k_scale=pool_s, dbg_cand=cand, dbg_scores=scores,
-                                dbg_cand_scores=cs)
+                                dbg_cand_scores=cs, W=W)
     torch.cuda.synchronize()
     assert pv.pivot_device_status() == 0
     f = lambda t: None if t is None else t.cpu().numpy()

@@ -145,6 +145,44 @@ def test_decode_paged_matches_contiguous(pv, gu, dtype, mode):
         assert np.array_equal(np.sort(cand, axis=1), np.sort(rcand, axis=1))
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+@pytest.mark.parametrize("g,W", [(2, 4), (4, 4), (3, 64)])
+def test_decode_local_window_parity(pv, gu, dtype, g, W):
+    """Decode form of the local window (Appendix B): pool of c from the scan up to pos0, each
+    query re-scores pool U [t-W+1, t]; mixes guarded (dense) and proxy sequences."""
+    x = inputs.make_decode(5, g, 300, 2600, dtype=dtype, seed=26)
+    out, sc, cand, cs = gu.run_decode(x, c=512, k=256, mode=po.MODE_REFINE, W=W)
+    t = acc.check_decode(x.codes(), c=512, k=256, mode=po.MODE_REFINE, guard_len=None, out_idx=out,
+                         out_scores=sc, cand=cand, cand_scores=cs, W=W)
+    _report(f"decode window {dtype} g={g} W={W}", t)
+    # the step's own keys are reachable now: the last query's newest key is its own position
+    ref, _, _, _ = gu.run_decode(x, c=512, k=256, mode=po.MODE_REFINE)
+    p0 = x.pos0.numpy()
+    assert all(ref[b].max() <= p0[b] or p0[b] + 1 < 512 for b in range(5))
+    assert any(out[b, g - 1].max() > p0[b] for b in range(5))
+
+
+def test_decode_local_window_paged_matches_contiguous(pv, gu):
+    x = inputs.make_decode(4, 2, 700, 2600, dtype="fp8", seed=27)
+    out, _, cand, _ = gu.run_decode_paged(x, c=512, k=256, mode=po.MODE_REFINE, seed=7, W=4)
+    ref, _, rcand, _ = gu.run_decode(x, c=512, k=256, mode=po.MODE_REFINE, guard_len=0, W=4)
+    assert np.array_equal(np.sort(out, axis=2), np.sort(ref, axis=2))
+    assert np.array_equal(np.sort(cand, axis=1), np.sort(rcand, axis=1))
+
+
+def test_decode_local_window_argument_errors(pv):
+    x = inputs.make_decode(2, 4, 300, 600, dtype="bf16", seed=28)
+    q, w, k, pos0 = x.q.cuda(), x.w.cuda(), x.k.cuda(), x.pos0.cuda()
+    out = torch.empty((2, 4, 64), dtype=torch.int32, device="cuda")
+    args = (q, w, k, pos0, 2, k.shape[1], 64, 128, 4, 128, 64)
+    with pytest.raises(pv.PivotError, match="invalid"):
+        pv.pivot_index_decode(*args, pv.REFINE, out, W=3)              # W < g
+    with pytest.raises(pv.PivotError, match="invalid"):
+        pv.pivot_index_decode(*args, pv.REUSE, out, W=4)               # Reuse has no candidate set to widen
+    with pytest.raises(pv.PivotError, match="invalid"):
+        pv.pivot_index_decode(*args, pv.REFINE, out, W=510)            # W + g - 1 > 512
+
+
 def test_decode_paged_bad_page_is_a_hole(pv, gu):
     """A block-table entry outside the pool faults nothing: the page's keys are never returned by
     Refine (the scan sees zeros there, the re-score drops them)."""

@@ -319,6 +319,72 @@ def test_decode_group_equals_prefill_group_on_same_tensors():
     np.testing.assert_array_equal(a.C, b.C)
 
 
+def _decode_view(x, p0, g):
+    return dict(dtype=x["dtype"], q=x["q"][None, p0:p0 + g],
+                qscale=None if x["qscale"] is None else x["qscale"][None, p0:p0 + g],
+                w=x["w"][None, p0:p0 + g], k=x["k"][None],
+                kscale=None if x["kscale"] is None else x["kscale"][None], pos0=np.array([p0], np.int32))
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+def test_decode_window_covering_everything_is_the_dense_indexer(dtype):
+    """Decode form of Appendix B: with the pool holding every key up to pos0 (c >= pos0 + 1) and
+    W >= g, pool united with [t-W+1, t] is the whole visible prefix of t, so every query of the
+    step must get the dense indexer's set (torch restatement), including the keys written
+    inside the step, which the pool cannot hold."""
+    x = tiny(L=80, H=4, d=8, dtype=dtype)
+    g, p0, k = 3, 50, 9
+    _, sets = _torch_dense(x, k)
+    r = po.pivot_decode(_decode_view(x, p0, g), c=64, k=k, mode=po.MODE_REFINE, guard_len=0, W=3)[0]
+    assert not r.guarded
+    for i in range(g):
+        assert set(r.T[i].tolist()) == sets[p0 + i]
+    # without the window the later queries cannot see the step's own keys
+    r0 = po.pivot_decode(_decode_view(x, p0, g), c=64, k=k, mode=po.MODE_REFINE, guard_len=0)[0]
+    assert r0.T.max() <= p0
+
+
+def test_decode_window_is_pool_united_with_own_window():
+    """Set-membership restatement: each query's result is the top-k, by its own dense scores
+    (torch restatement), over exactly pool U [t-W+1, t] -- a recent key outside the pool is
+    eligible for the queries whose window covers it and for no other."""
+    x = tiny(L=96, H=4, d=8, dtype="bf16", seed=5)
+    g, p0, c, k, W = 3, 80, 10, 6, 4
+    I, _ = _torch_dense(x, k)
+    r = po.pivot_decode(_decode_view(x, p0, g), c=c, k=k, mode=po.MODE_REFINE, guard_len=0, W=W)[0]
+    pool = set(r.C.tolist())
+    assert len(pool) == c and max(pool) <= p0
+    r_plain = po.pivot_decode(_decode_view(x, p0, g), c=c, k=k, mode=po.MODE_REFINE, guard_len=0)[0]
+    np.testing.assert_array_equal(r.C, r_plain.C)                  # the pool is the plain method's
+    for i in range(g):
+        t = p0 + i
+        allowed = sorted(pool | set(range(t - W + 1, t + 1)))
+        sc = I[t, allowed].numpy()
+        order = sorted(range(len(allowed)), key=lambda j: (-sc[j], allowed[j]))[:k]
+        assert set(r.T[i].tolist()) == {allowed[j] for j in order}
+        assert sorted(r.member_C[i].tolist()) == allowed
+    with pytest.raises(ValueError):
+        po.pivot_decode(_decode_view(x, p0, g), c=c, k=k, mode=po.MODE_REFINE, guard_len=0, W=2)   # W < g
+
+
+def test_acceptance_rule_decode_window_accepts_the_oracle_and_rejects_a_stale_row():
+    from oracle import acceptance as acc
+    x = inputs.make_decode(3, 2, 200, 400, dtype="bf16", seed=9).codes()
+    c, k, W = 64, 24, 4
+    res = po.pivot_decode(x, c=c, k=k, mode=po.MODE_REFINE, guard_len=0, W=W)
+    out = np.stack([res[b].T for b in range(3)])
+    cand = np.stack([res[b].C for b in range(3)]).astype(np.int32)
+    t = acc.check_decode(x, c=c, k=k, mode=po.MODE_REFINE, guard_len=0, out_idx=out, cand=cand, W=W)
+    assert t.rows > 0 and t.exact_rows == t.rows
+    plain = po.pivot_decode(x, c=c, k=k, mode=po.MODE_REFINE, guard_len=0)
+    differs = [b for b in range(3) if not np.array_equal(np.sort(plain[b].T), np.sort(res[b].T))]
+    assert differs, "the window must change at least one row of this case"
+    bad = out.copy()
+    bad[differs[0]] = plain[differs[0]].T                           # result computed without the window
+    with pytest.raises(AssertionError):
+        acc.check_decode(x, c=c, k=k, mode=po.MODE_REFINE, guard_len=0, out_idx=bad, cand=cand, W=W)
+
+
 # ---------------------------------------------------------------- acceptance rule with a local window
 
 def test_acceptance_rule_with_window_accepts_the_oracle_and_rejects_mutations():
