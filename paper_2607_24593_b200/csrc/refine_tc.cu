@@ -243,9 +243,14 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
     }
   } else if (warp < 2 + GATHER_WARPS) {
     // ------------------------------------------------------------------ gather producers
-    // Thread j of the 64 copies candidate rows j and j + 64 of each tile.  Tiles are committed
-    // as cp.async groups; a tile is published LOOKAHEAD tiles after it was issued.
-    const int j = (warp - 2) * 32 + lane;
+    // Each gather warp fills 64 rows of a tile.  A lane looks up two of them (position, row in
+    // the key tensor, scale: rows wrow0 + lane and wrow0 + 32 + lane); the copies themselves go
+    // eight lanes to a row, one 16-byte chunk each, so that one warp instruction reads four whole
+    // 128-byte lines (a lane-per-row copy would touch 32 lines for the same bytes and is bound
+    // by the L1's tag rate).  Tiles are committed as cp.async groups; a tile is published
+    // LOOKAHEAD tiles after it was issued.
+    const int wrow0 = (warp - 2) * 64;
+    const int sub = lane >> 3, chunk = lane & 7;
     uint32_t it = 0;          // tiles issued
     uint32_t pub = 0;         // tiles published
     bool ok = true;
@@ -262,7 +267,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       // block-table lookup when the cache is paged) two tiles ahead and key scales one tile
       // ahead, so no round trip sits on this thread's issue path.
       auto load_idx = [&](int tile, int half) -> int {
-        const int sl = tile * TILE_KEYS + half * 64 + j;
+        const int sl = tile * TILE_KEYS + wrow0 + half * 32 + lane;
         return (tile < ntiles && sl < gd.n_cand) ? __ldg(gd.cand + sl) : -1;
       };
       auto key_row = [&](int ix) -> int {      // -1: padding slot, or a page outside the pool
@@ -282,22 +287,26 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         const int row2[2] = {key_row(idx2[0]), key_row(idx2[1])};
         const float ks1[2] = {load_ks(row1[0]), load_ks(row1[1])};
         if (ok) ok = ptx::mbar_wait(&ct.empty[s], ph ^ 1, abort_flag, 64);   // whole warps wait here: sleep, do not spin
+        int krow[2];
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
-          const int row = half * 64 + j;
+          const int row = wrow0 + half * 32 + lane;
           ct.meta[it % META_SLOTS][row] = KeyMeta{row0[half] < 0 ? -1 : idx0[half], ks0[half]};
-          const int krow = row0[half] < 0 ? 0 : row0[half];
-          const uint32_t swz = (uint32_t)(row & 7);
-          const uint8_t* src = (const uint8_t*)gd.kbase + (size_t)krow * C::ROW_BYTES;
-          const uint32_t dst = ptx::smem_u32(kring + s * C::STAGE_BYTES) + (uint32_t)row * 128u;
-#pragma unroll
-          for (int h = 0; h < C::KHALVES; ++h)
-#pragma unroll
-            for (int cidx = 0; cidx < 8; ++cidx)
-              cp_async16(dst + h * C::HALF_TILE_BYTES + ((cidx ^ swz) << 4), src + h * 128 + cidx * 16);
+          krow[half] = row0[half] < 0 ? 0 : row0[half];
           idx0[half] = idx1[half]; idx1[half] = idx2[half]; idx2[half] = idx3[half];
           row0[half] = row1[half]; row1[half] = row2[half];
           ks0[half] = ks1[half];
+        }
+        const uint32_t dst0 = ptx::smem_u32(kring + s * C::STAGE_BYTES);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {                 // four rows per pass
+          const int rl = i * 4 + sub;                  // row inside this warp's 64
+          const int kr = __shfl_sync(0xffffffffu, krow[i >> 3], rl & 31);
+          const int row = wrow0 + rl;
+          const uint8_t* src = (const uint8_t*)gd.kbase + (size_t)kr * C::ROW_BYTES + chunk * 16;
+          const uint32_t dst = dst0 + (uint32_t)row * 128u + (uint32_t)((chunk ^ (row & 7)) << 4);
+#pragma unroll
+          for (int h = 0; h < C::KHALVES; ++h) cp_async16(dst + h * C::HALF_TILE_BYTES, src + h * 128);
         }
         cp_async_commit();
         if (it + 1 - pub > (uint32_t)C::LOOKAHEAD) {
