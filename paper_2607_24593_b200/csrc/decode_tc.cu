@@ -339,22 +339,40 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Lmax, const float* __
       const int i = i0 + (u * kBlk + tid) * 4;
       v4[u] = i < n0 ? __ldcg(reinterpret_cast<const float4*>(sc + i)) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-#pragma unroll
-    for (int u = 0; u < 16; ++u) {
+    // One list-cursor bump per warp and pass: each thread counts its keepers among its sixteen
+    // scores, a warp scan turns the counts into offsets (a bump per keeper group would queue
+    // hundreds of same-address atomics per pass).
+    auto entry_of = [&](int u) -> entry_t {
       const float4 q4 = v4[u >> 2];
       const float vu = (u & 3) == 0 ? q4.x : (u & 3) == 1 ? q4.y : (u & 3) == 2 ? q4.z : q4.w;
+      return make_entry(score_to_key(vu), i0 + ((u >> 2) * kBlk + tid) * 4 + (u & 3));
+    };
+    uint32_t keepmask = 0;
+#pragma unroll
+    for (int u = 0; u < 16; ++u) {
       const int i = i0 + ((u >> 2) * kBlk + tid) * 4 + (u & 3);
-      const entry_t e = make_entry(score_to_key(vu), i);
+      const entry_t e = entry_of(u);
       const bool keep = i < n0 && (pbits == 0 || (e >> (64 - pbits)) >= prefix);
-      const uint32_t m = __ballot_sync(0xffffffffu, keep);
-      if (m) {
-        uint32_t pos = 0;
-        const int leader = __ffs(m) - 1;
-        if (lane == leader) pos = atomicAdd(&sm.blk.list_n, (uint32_t)__popc(m));
-        pos = __shfl_sync(0xffffffffu, pos, leader);
-        if (keep) {
-          const uint32_t p = pos + __popc(m & ((1u << lane) - 1u));
-          if (p < (uint32_t)SEL_CAP) sm.list[p] = e;
+      keepmask |= keep ? 1u << u : 0u;
+    }
+    const uint32_t cnt = (uint32_t)__popc(keepmask);
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
+    if (tot) {                                           // warp-uniform
+      uint32_t base = 0;
+      if (lane == 31) base = atomicAdd(&sm.blk.list_n, tot);
+      base = __shfl_sync(0xffffffffu, base, 31);
+      uint32_t p = base + incl - cnt;
+#pragma unroll
+      for (int u = 0; u < 16; ++u) {
+        if ((keepmask >> u) & 1u) {
+          if (p < (uint32_t)SEL_CAP) sm.list[p] = entry_of(u);
+          ++p;
         }
       }
     }
