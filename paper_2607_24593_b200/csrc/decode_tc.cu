@@ -8,11 +8,13 @@
 //                        epilogue (ReLU, gate-weighted head sum, key scale) -> one fp32 score per
 //                        key to an L2-resident score array (3 % of the bytes read), plus a
 //                        8192-bin histogram of the scores' top 13 key bits per sequence.
-//   decode_select_kernel one 1024-thread CTA per sequence: the histogram gives the bin holding
-//                        the K-th best score; if that leaves too many candidates the bin is
-//                        refined 12 bits at a time with further passes over the scores; the
-//                        survivors are collected in shared memory and the exact top-K (Eq. 6 / 7)
-//                        is taken there.
+//   decode_select_kernel four 1024-thread CTAs per sequence: the histogram gives the bin holding
+//                        the K-th best score; each CTA collects the survivors of its quarter of
+//                        the score array and appends them to the sequence's list in global
+//                        memory; the CTA that finishes last takes the exact top-K (Eq. 6 / 7) of
+//                        the list in shared memory (nobody waits for anybody).  If the boundary
+//                        bin leaves too many candidates, one CTA alone refines it 12 bits at a
+//                        time with further passes over the scores.
 //   decode_window_kernel (only with a local window, Appendix B) the union of the step's per-query
 //                        windows as one more candidate chunk per sequence, minus the positions
 //                        the pool already holds.
@@ -36,6 +38,7 @@ constexpr int DHIST = 1 << DHIST_BITS;
 constexpr int D_N = kHeads;             // MMA N: one proxy
 constexpr int D_THREADS = 64 + 256;     // TMA warp, MMA warp, two sets of four epilogue warps
 constexpr int SEL_CAP = 16384;          // candidates collected in shared memory per sequence
+constexpr int SEL_SPLIT = 4;            // CTAs sharing the collection pass of one sequence
 
 template <int DT>
 struct DCfg {
@@ -278,24 +281,31 @@ struct SelSmem {
   entry_t list[SEL_CAP];
 };
 
+// sel_ctr[2 b] = entries in sequence b's global list, sel_ctr[2 b + 1] = CTAs that have
+// delivered their share (both zeroed with the histograms before every step).
 __global__ void __launch_bounds__(kBlk, 1)
-decode_select_kernel(const RowDesc* __restrict__ prox, int Lmax, const float* __restrict__ scores,
-                     const uint32_t* __restrict__ ghist) {
+decode_select_kernel(const RowDesc* __restrict__ prox, int Ls, const float* __restrict__ scores,
+                     const uint32_t* __restrict__ ghist, entry_t* __restrict__ glist, uint32_t* sel_ctr) {
   extern __shared__ uint8_t sel_raw[];
   SelSmem& sm = *reinterpret_cast<SelSmem*>(((uintptr_t)sel_raw + 15) & ~(uintptr_t)15);
-  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
+  const int split = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31;
   const RowDesc rd = prox[b];
   const int K = rd.K, n0 = rd.n_vis;
   if (K <= 0) return;
-  const float* sc = scores + (size_t)b * Lmax;
+  const float* sc = scores + (size_t)b * Ls;
   // ---- narrow the candidates: entries whose top `pbits` bits are >= prefix
   unsigned long long prefix = 0;
   int pbits = 0;
+  bool solo = false;              // this CTA handles the whole sequence by itself
   if (n0 > SEL_CAP) {
     blk_boundary(sm.blk, ghist + (size_t)b * DHIST, DHIST, (uint32_t)K);
     uint32_t need = sm.blk.need, pop = sm.blk.pop;
     prefix = sm.blk.bin;
     pbits = DHIST_BITS;
+    // too crowded a boundary bin (every CTA of the sequence sees the same histogram): the
+    // refinement passes need the whole score array, CTA 0 takes the sequence alone
+    solo = (uint32_t)K - need + pop > (uint32_t)SEL_CAP;
+    if (solo && split != 0) return;
     while ((uint32_t)K - need + pop > (uint32_t)SEL_CAP && pbits < 64) {
       const int wbits = 64 - pbits < 12 ? 64 - pbits : 12;
       __syncthreads();
@@ -329,15 +339,17 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Lmax, const float* __
       pbits += wbits;
     }
   }
-  // ---- collect them in shared memory
+  // ---- collect them in shared memory: this CTA's share of the scores (multiples of four)
+  const int lo = solo ? 0 : (int)(((long long)n0 * split / SEL_SPLIT) & ~3ll);
+  const int hi = (solo || split == SEL_SPLIT - 1) ? n0 : (int)(((long long)n0 * (split + 1) / SEL_SPLIT) & ~3ll);
   if (tid == 0) sm.blk.list_n = 0;
   __syncthreads();
-  for (int i0 = 0; i0 < n0; i0 += 16 * kBlk) {         // four 16-byte loads in flight per thread
+  for (int i0 = lo; i0 < hi; i0 += 16 * kBlk) {        // four 16-byte loads in flight per thread
     float4 v4[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int i = i0 + (u * kBlk + tid) * 4;
-      v4[u] = i < n0 ? __ldcg(reinterpret_cast<const float4*>(sc + i)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      v4[u] = i < hi ? __ldcg(reinterpret_cast<const float4*>(sc + i)) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     // One list-cursor bump per warp and pass: each thread counts its keepers among its sixteen
     // scores, a warp scan turns the counts into offsets (a bump per keeper group would queue
@@ -352,7 +364,7 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Lmax, const float* __
     for (int u = 0; u < 16; ++u) {
       const int i = i0 + ((u >> 2) * kBlk + tid) * 4 + (u & 3);
       const entry_t e = entry_of(u);
-      const bool keep = i < n0 && (pbits == 0 || (e >> (64 - pbits)) >= prefix);
+      const bool keep = i < hi && (pbits == 0 || (e >> (64 - pbits)) >= prefix);
       keepmask |= keep ? 1u << u : 0u;
     }
     const uint32_t cnt = (uint32_t)__popc(keepmask);
@@ -378,7 +390,25 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Lmax, const float* __
     }
   }
   __syncthreads();
-  const int n = min((int)sm.blk.list_n, SEL_CAP);
+  int n = min((int)sm.blk.list_n, SEL_CAP);
+  if (!solo) {
+    // ---- hand the share over; whoever delivers last holds the complete list
+    entry_t* const gl = glist + (size_t)b * SEL_CAP;
+    if (tid == 0) sm.blk.small_n = n ? atomicAdd(&sel_ctr[2 * b], (uint32_t)n) : 0u;
+    __syncthreads();
+    const uint32_t at = sm.blk.small_n;
+    for (int i = tid; i < n; i += kBlk)
+      if (at + i < (uint32_t)SEL_CAP) gl[at + i] = sm.list[i];
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) sm.blk.small_n = atomicAdd(&sel_ctr[2 * b + 1], 1u);
+    __syncthreads();
+    if (sm.blk.small_n != (uint32_t)(SEL_SPLIT - 1)) return;
+    __threadfence();
+    n = min((int)*reinterpret_cast<volatile uint32_t*>(&sel_ctr[2 * b]), SEL_CAP);
+    for (int i = tid; i < n; i += kBlk) sm.list[i] = __ldcg(gl + i);
+    __syncthreads();
+  }
   blk_emit_topk(sm.blk, sm.list, n, n, K, rd.out, rd.out_score, rd.out_rows, rd.out_stride);
 }
 
@@ -459,9 +489,16 @@ __global__ void decode_window_kernel(const GroupDesc* __restrict__ groups, int m
   const int pos0 = gd.first_pos, lo = pos0 - W + 1, w_g = W + g - 1;
   for (int j = tid; j < w_g; j += blockDim.x) dup[j] = 0;
   __syncthreads();
-  for (int i = tid; i < gd.n_cand; i += blockDim.x) {
-    const int p = gd.cand[i];
-    if (p >= lo && p <= pos0) dup[p - lo] = 1;
+  for (int i0 = 0; i0 < gd.n_cand; i0 += 4 * blockDim.x) {      // four independent loads per thread
+    int p[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u * blockDim.x + tid;
+      p[u] = i < gd.n_cand ? __ldcg(gd.cand + i) : -1;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (p[u] >= lo && p[u] <= pos0) dup[p[u] - lo] = 1;
   }
   __syncthreads();
   for (int j = tid; j < w_g; j += blockDim.x) {
@@ -496,7 +533,8 @@ size_t decode_fast_bytes(int B, int Lmax, int g, int c) {
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
   const int mc = group_chunks(g);
   const int ncc = (c + kDecodeCandChunk - 1) / kDecodeCandChunk;
-  return up((size_t)B * Lmax * 4) + up((size_t)B * DHIST * 4) + up((size_t)(B + 1) * 4) +
+  const size_t Ls = ((size_t)Lmax + 3) & ~(size_t)3;     // score rows start on 16-byte boundaries
+  return up(B * Ls * 4) + up((size_t)B * (DHIST + 2) * 4) + up((size_t)(B + 1) * 4) + up((size_t)B * SEL_CAP * 8) +
          up((size_t)B * mc * (ncc + 1) * sizeof(GroupDesc)) + up((size_t)B * g * sizeof(EntryList)) +
          up((size_t)B * kDecodeWinMax * 4) + up((size_t)B * g * (c + kDecodeWinMax) * 8);
 }
@@ -504,9 +542,12 @@ size_t decode_fast_bytes(int B, int Lmax, int g, int c) {
 cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
   char* p = (char*)d.scratch;
-  float* scores = (float*)p;                 p += up((size_t)d.B * d.Lmax * 4);
-  uint32_t* ghist = (uint32_t*)p;            p += up((size_t)d.B * DHIST * 4);
+  const int Ls = (d.Lmax + 3) & ~3;
+  float* scores = (float*)p;                 p += up((size_t)d.B * Ls * 4);
+  uint32_t* ghist = (uint32_t*)p;            p += up((size_t)d.B * (DHIST + 2) * 4);
+  uint32_t* sel_ctr = ghist + (size_t)d.B * DHIST;       // zeroed together with the histograms
   int* tile_prefix = (int*)p;                p += up((size_t)(d.B + 1) * 4);
+  entry_t* glist = (entry_t*)p;              p += up((size_t)d.B * SEL_CAP * 8);
   const int mc = group_chunks(d.g);
   const int ncc = (d.c + kDecodeCandChunk - 1) / kDecodeCandChunk;
   const int W = d.mode == 1 ? d.W : 0;
@@ -516,7 +557,7 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   int32_t* wcand = (int32_t*)p;              p += up((size_t)d.B * kDecodeWinMax * 4);
   unsigned long long* entries = (unsigned long long*)p;
 
-  cudaError_t e = cudaMemsetAsync(ghist, 0, (size_t)d.B * DHIST * 4, st);
+  cudaError_t e = cudaMemsetAsync(ghist, 0, (size_t)d.B * (DHIST + 2) * 4, st);
   if (e != cudaSuccess) return e;
   decode_setup_kernel<<<1, 1024, 0, st>>>(d.prox, d.groups, d.B, d.g, d.c, d.k, d.mode, W, tile_prefix, chunks,
                                           lists, entries, wcand);
@@ -529,8 +570,8 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
     return cudaErrorInvalidValue;
   if (d.ev_scan_begin) cudaEventRecord(d.ev_scan_begin, st);
   e = d.dtype == DT_FP8
-          ? launch_scan<DT_FP8>(mk, mq, mks, d.prox, tile_prefix, d.B, d.Lmax, scores, ghist, d.status, d.sms, st)
-          : launch_scan<DT_BF16>(mk, mq, mks, d.prox, tile_prefix, d.B, d.Lmax, scores, ghist, d.status, d.sms, st);
+          ? launch_scan<DT_FP8>(mk, mq, mks, d.prox, tile_prefix, d.B, Ls, scores, ghist, d.status, d.sms, st)
+          : launch_scan<DT_BF16>(mk, mq, mks, d.prox, tile_prefix, d.B, Ls, scores, ghist, d.status, d.sms, st);
   if (e != cudaSuccess) return e;
   if (d.ev_scan_end) cudaEventRecord(d.ev_scan_end, st);
   static bool sel_attr = false;
@@ -540,11 +581,11 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     sel_attr = true;
   }
-  decode_select_kernel<<<d.B, kBlk, sel_smem, st>>>(d.prox, d.Lmax, scores, ghist);
+  decode_select_kernel<<<dim3(SEL_SPLIT, d.B), kBlk, sel_smem, st>>>(d.prox, Ls, scores, ghist, glist, sel_ctr);
   ++launch_counter();
   if (d.mode == 1) {
     if (W > 0) {
-      decode_window_kernel<<<d.B, 128, 0, st>>>(d.groups, mc, d.g, W, wcand);
+      decode_window_kernel<<<d.B, 1024, 0, st>>>(d.groups, mc, d.g, W, wcand);
       ++launch_counter();
     }
     ScanScratch sc = d.scratch_tc;

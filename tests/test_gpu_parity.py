@@ -122,6 +122,35 @@ def test_decode_small_parity(pv, gu, dtype, mode):
     _report(f"decode {dtype} mode={mode}", t)
 
 
+def test_decode_ties_beyond_the_select_list(pv, gu):
+    """Zero gates make all scores equal: with more visible keys than the select's shared-memory
+    list holds, the boundary bin is the whole sequence and one CTA refines it down to the
+    position bits -- the total order must still return the lowest positions."""
+    x = inputs.make_decode(2, 2, 20000, 24000, dtype="bf16", seed=29)
+    x.w.zero_()
+    out, _, cand, _ = gu.run_decode(x, c=512, k=256, mode=po.MODE_REFINE)
+    for b in range(2):
+        assert sorted(cand[b].tolist()) == list(range(512))
+        for i in range(2):
+            assert sorted(out[b, i].tolist()) == list(range(256))
+
+
+def test_decode_cache_rows_not_a_multiple_of_four(pv):
+    """bf16 caches may have any Lmax: the per-sequence score rows are padded inside the library."""
+    x = inputs.make_decode(3, 2, 700, 1200, dtype="bf16", seed=30)
+    Lmax = x.k.shape[1] - 3                                      # 1213: odd
+    k = x.k[:, :Lmax].contiguous().cuda()
+    q, w, pos0 = x.q.cuda(), x.w.cuda(), x.pos0.cuda()
+    out = torch.full((3, 2, 128), -7, dtype=torch.int32, device="cuda")
+    pv.pivot_index_decode(q, w, k, pos0, 3, Lmax, 64, 128, 2, 256, 128, pv.REFINE, out)
+    torch.cuda.synchronize()
+    assert pv.pivot_device_status() == 0
+    ref = torch.full((3, 2, 128), -7, dtype=torch.int32, device="cuda")
+    pv.pivot_index_decode(q, w, x.k.cuda(), pos0, 3, x.k.shape[1], 64, 128, 2, 256, 128, pv.REFINE, ref)
+    torch.cuda.synchronize()
+    assert torch.equal(torch.sort(out, dim=2).values, torch.sort(ref, dim=2).values)
+
+
 def test_decode_group_of_four(pv, gu):
     x = inputs.make_decode(3, 4, 2000, 2600, dtype="fp8", seed=22)
     out, sc, cand, cs = gu.run_decode(x, c=256, k=128, mode=po.MODE_REFINE)
