@@ -237,10 +237,11 @@ int dense_index_static(const pivot_tensor* q, const float* w, const pivot_tensor
  * memory (pinned, else the copies are neither asynchronous nor fast).  The call copies the inputs
  * into `arena` (device, at least pivot_prefill_host_arena_bytes(...) bytes, which includes the
  * workspace), runs the device path and copies out_idx back; it returns after everything has
- * finished.  Keys and gates go first; the queries then travel in row chunks on a copy stream of
- * the library's own while earlier chunks are indexed on `stream` (row_begin / row_end of
- * pivot_opts) and their results return on a second copy stream, so the PCIe transfers in both
- * directions overlap the kernels.  The first call on a device creates the two copy streams and
+ * finished.  Keys and key scales go first; queries, gates and query scales then travel in row
+ * chunks on a copy stream of the library's own while earlier chunks are indexed on `stream`
+ * (row_begin / row_end of pivot_opts) and their results return on a second copy stream, so the
+ * PCIe transfers in both directions overlap the kernels.  Chunks are taken alternately from the
+ * end and the start of the request (late rows cost the most compute per byte copied).  The first call on a device creates the two copy streams and
  * their events (kept until the process exits).
  */
 size_t pivot_prefill_host_arena_bytes(int L, int H_I, int d, int g, int c, int k, int dtype);

@@ -468,17 +468,29 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
   // The copy-in stream may not touch the arena before earlier work on `stream` has left it.
   if ((rc = check_cuda(cudaEventRecord(ds.ev_entry, st)))) return rc;
   if ((rc = check_cuda(cudaStreamWaitEvent(ds.copy_in, ds.ev_entry, 0)))) return rc;
-  // keys, gates and scales: small, ahead of the first chunk on the compute stream
+  // keys and their scales: every chunk needs all of them; small, ahead of the first chunk on
+  // the compute stream
   if ((rc = check_cuda(cudaMemcpyAsync(dk, kcache->data, (size_t)L * d * esz, cudaMemcpyHostToDevice, st)))) return rc;
-  if ((rc = check_cuda(cudaMemcpyAsync(dw, w, (size_t)L * H_I * 4, cudaMemcpyHostToDevice, st)))) return rc;
-  if (fp8) {
-    if ((rc = check_cuda(cudaMemcpyAsync(dqs, q->scale, (size_t)L * H_I * 4, cudaMemcpyHostToDevice, st)))) return rc;
-    if ((rc = check_cuda(cudaMemcpyAsync(dks, kcache->scale, (size_t)L * 4, cudaMemcpyHostToDevice, st)))) return rc;
-  }
+  if (fp8 && (rc = check_cuda(cudaMemcpyAsync(dks, kcache->scale, (size_t)L * 4, cudaMemcpyHostToDevice, st)))) return rc;
+  // Order of the chunks: a chunk's cost grows with its position in the request (longer prefixes)
+  // while its copies do not.  In row order the first chunks finish long before the next input
+  // has arrived; back to front, the last (cheap) chunks finish faster than their results can
+  // leave.  Alternating the two ends (last, first, last but one, second, ...) keeps both the
+  // compute stream and the copy-out stream fed.
+  int order[kHostChunks];
+  for (int j = 0; j < n_chunks; ++j) order[j] = (j & 1) ? j / 2 : n_chunks - 1 - j / 2;
   // queries: chunk by chunk on the copy-in stream
   const size_t qrow = (size_t)H_I * d * esz;
-  for (int i = 0; i < n_chunks; ++i) {
+  for (int j = 0; j < n_chunks; ++j) {
+    const int i = order[j];
     const int r0 = i * chunk_rows, r1 = (r0 + chunk_rows < L) ? r0 + chunk_rows : L;
+    // a chunk's queries, gates and query scales travel together
+    if ((rc = check_cuda(cudaMemcpyAsync(dw + (size_t)r0 * H_I, w + (size_t)r0 * H_I, (size_t)(r1 - r0) * H_I * 4,
+                                         cudaMemcpyHostToDevice, ds.copy_in))))
+      return rc;
+    if (fp8 && (rc = check_cuda(cudaMemcpyAsync(dqs + (size_t)r0 * H_I, q->scale + (size_t)r0 * H_I,
+                                                (size_t)(r1 - r0) * H_I * 4, cudaMemcpyHostToDevice, ds.copy_in))))
+      return rc;
     if ((rc = check_cuda(cudaMemcpyAsync(dq + (size_t)r0 * qrow, (const char*)q->data + (size_t)r0 * qrow,
                                          (size_t)(r1 - r0) * qrow, cudaMemcpyHostToDevice, ds.copy_in))))
       return rc;
@@ -486,7 +498,8 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
   }
   pivot_tensor tq{dq, fp8 ? dqs : nullptr, q->dtype};
   pivot_tensor tk{dk, fp8 ? dks : nullptr, q->dtype};
-  for (int i = 0; i < n_chunks; ++i) {
+  for (int j = 0; j < n_chunks; ++j) {
+    const int i = order[j];
     const int r0 = i * chunk_rows, r1 = (r0 + chunk_rows < L) ? r0 + chunk_rows : L;
     pivot_opts o;
     memset(&o, 0, sizeof(o));
