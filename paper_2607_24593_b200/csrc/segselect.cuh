@@ -499,17 +499,23 @@ __device__ __forceinline__ int smem_row_topk(const Team& tm, SegSelSmem& sm, con
   }
   // Which of this thread's slots go out: counted first, then a scan over the team hands every
   // thread a contiguous run of output positions (no atomics, no votes in the write loop).
-  uint32_t emit_mask = 0u;
+  uint32_t emit_mask = 0u, edge_mask = 0u;
 #pragma unroll
-  for (int i = 0; i < 32; ++i) {
+  for (int i = 0; i < 32; ++i) {             // branch-free: two bit masks per thread
     const uint32_t k = kreg[i];
     const bool valid = k != 0u;
     const int bn = valid ? (int)((k - lo) >> shift) : -2;
-    if (valid && (bn > bsel || (whole_bin && bn == bsel))) emit_mask |= 1u << i;
-    if (valid && bn == bsel && !whole_bin) {
-      const uint32_t q = atomicAdd(&sm.list_n, 1u);
-      if (q < (uint32_t)kSelSmall) sm.list[q] = make_entry(k, ci[i]);
-    }
+    emit_mask |= (valid && (bn > bsel || (whole_bin && bn == bsel))) ? 1u << i : 0u;
+    edge_mask |= (valid && bn == bsel && !whole_bin) ? 1u << i : 0u;
+  }
+  // the boundary bin's slots (a handful per row) go to the list that is ranked below; kept out
+  // of the loop above, where a rarely taken branch per slot cost more than everything else in it
+  while (edge_mask) {
+    const int i = __ffs(edge_mask) - 1;
+    edge_mask &= edge_mask - 1u;
+    const int sl = i * tm.nthr + tm.tid;
+    const uint32_t q = atomicAdd(&sm.list_n, 1u);
+    if (q < (uint32_t)kSelSmall) sm.list[q] = make_entry(keys[sl], sl < n_cand ? __ldg(cand + sl) : -1);
   }
   const uint32_t mine = (uint32_t)__popc(emit_mask);
   uint32_t incl = mine;
