@@ -530,14 +530,38 @@ __device__ __forceinline__ int smem_row_topk(const Team& tm, SegSelSmem& sm, con
   uint32_t p = incl - mine;
   for (int w = 0; w < wq; ++w) p += sm.wsum[w];
   if (tm.tid == tm.nthr - 1) sm.out_count = p + mine;      // emitted so far; the ranked ones follow
+  if (K <= kSelBins && out_score == nullptr) {
+    // Positions are lined up in output order in shared memory first (the histogram is no longer
+    // needed: every warp has its boundary, see the barrier above) and leave as whole 16-byte
+    // rows; written straight from the loop below they would go out as scattered 4-byte stores.
+    int32_t* const stage = reinterpret_cast<int32_t*>(sm.hist);
 #pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    if ((emit_mask >> i) & 1u) {
-      if (p < (uint32_t)K) {
-        out[p] = ci[i];
-        if (out_score) out_score[p] = key_to_score(kreg[i]);
+    for (int i = 0; i < 32; ++i) {
+      if ((emit_mask >> i) & 1u) {
+        if (p < (uint32_t)K) stage[p] = ci[i];
+        ++p;
       }
-      ++p;
+    }
+    tm.sync();
+    const int n_out = (int)(sm.out_count < (uint32_t)K ? sm.out_count : (uint32_t)K);
+    const int n4 = n_out >> 2;
+    if ((reinterpret_cast<uintptr_t>(out) & 15) == 0) {
+      for (int t = tm.tid; t < n4; t += tm.nthr)
+        reinterpret_cast<int4*>(out)[t] = reinterpret_cast<const int4*>(stage)[t];
+      for (int t = (n4 << 2) + tm.tid; t < n_out; t += tm.nthr) out[t] = stage[t];
+    } else {
+      for (int t = tm.tid; t < n_out; t += tm.nthr) out[t] = stage[t];
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      if ((emit_mask >> i) & 1u) {
+        if (p < (uint32_t)K) {
+          out[p] = ci[i];
+          if (out_score) out_score[p] = key_to_score(kreg[i]);
+        }
+        ++p;
+      }
     }
   }
   tm.sync();

@@ -259,6 +259,17 @@ def _sorted_rows(a):
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+def test_plain_call_matches_the_call_with_debug_buffers(pv, gu, dtype):
+    """The oracle parity tests pass score / candidate buffers, which take other store paths in
+    the kernels than a caller's plain call: both must return the same sets."""
+    L, g, c, k = 2500, 4, 512, 256
+    x = inputs.make_prefill(L, dtype=dtype, seed=78)
+    dbg, _, _, _ = gu.run_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE)
+    plain, _, _, _ = gu.run_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE, debug=False)
+    assert np.array_equal(_sorted_rows(plain), _sorted_rows(dbg))
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
 @pytest.mark.parametrize("mode", [po.MODE_REUSE, po.MODE_REFINE])
 def test_prefill_row_ranges_match_whole_call(pv, dtype, mode):
     """Chunks of query rows (row_begin / row_end) give the rows of one whole call: same sets
