@@ -426,16 +426,31 @@ __global__ void __launch_bounds__(kBlk, 1) entries_topk_kernel(const EntryList* 
 __global__ void decode_setup_kernel(const RowDesc* __restrict__ prox, const GroupDesc* __restrict__ groups, int B,
                                     int g, int c, int k, int mode, int W, int* tile_prefix, GroupDesc* chunks,
                                     EntryList* lists, unsigned long long* entries, const int32_t* wcand) {
-  __shared__ int tiles[1024];
-  const int tid = threadIdx.x;
-  for (int b = tid; b < B; b += blockDim.x)
-    tiles[b] = prox[b].K > 0 ? (prox[b].n_vis + TILE_KEYS - 1) / TILE_KEYS : 0;
+  // tile_prefix = exclusive prefix sum of the sequences' tile counts (any B: 1024 at a time)
+  __shared__ int wsum[32];
+  __shared__ int carry;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  if (tid == 0) carry = 0;
   __syncthreads();
-  if (tid == 0) {
-    int acc = 0;
-    for (int b = 0; b < B; ++b) { tile_prefix[b] = acc; acc += tiles[b]; }
-    tile_prefix[B] = acc;
+  for (int b0 = 0; b0 < B; b0 += 1024) {
+    const int b = b0 + tid;
+    const int v = (b < B && prox[b].K > 0) ? (prox[b].n_vis + TILE_KEYS - 1) / TILE_KEYS : 0;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int u = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += u;
+    }
+    if (lane == 31) wsum[wid] = incl;
+    __syncthreads();
+    int base = carry;
+    for (int w = 0; w < wid; ++w) base += wsum[w];
+    if (b < B) tile_prefix[b] = base + incl - v;
+    __syncthreads();
+    if (tid == 1023) carry = base + incl;
+    __syncthreads();
   }
+  if (tid == 0) tile_prefix[B] = carry;
   if (mode != 1) return;
   // Refine: split every (sequence, member chunk) into candidate chunks so all SMs re-score,
   // each leaving packed entries; one entry list per query for the final top-k.

@@ -151,6 +151,15 @@ def test_decode_cache_rows_not_a_multiple_of_four(pv):
     assert torch.equal(torch.sort(out, dim=2).values, torch.sort(ref, dim=2).values)
 
 
+def test_decode_more_than_1024_sequences(pv, gu):
+    """Batch sizes beyond one block's worth of sequences in the setup kernel."""
+    x = inputs.make_decode(1100, 2, 40, 200, dtype="bf16", seed=31)
+    out, sc, cand, cs = gu.run_decode(x, c=32, k=16, mode=po.MODE_REFINE)
+    t = acc.check_decode(x.codes(), c=32, k=16, mode=po.MODE_REFINE, guard_len=None, out_idx=out, out_scores=sc,
+                         cand=cand, cand_scores=cs, seqs=[0, 5, 511, 1023, 1024, 1025, 1099])
+    assert t.rows > 0
+
+
 def test_decode_group_of_four(pv, gu):
     x = inputs.make_decode(3, 4, 2000, 2600, dtype="fp8", seed=22)
     out, sc, cand, cs = gu.run_decode(x, c=256, k=128, mode=po.MODE_REFINE)
