@@ -72,6 +72,7 @@ def test_dense_small_full_parity(pv, gu, dtype):
     (130, 1, 32, 8, None),         # g = 1
     (64, 4, 512, 256, None),       # everything guarded, fewer keys than k
     (1, 4, 8, 4, None),            # single token
+    (700, 3, 101, 37, None),       # odd sizes: output rows not 16-byte aligned, g does not divide L
 ])
 def test_prefill_edge_shapes(pv, gu, dtype, L, g, c, k, guard):
     x = inputs.make_prefill(L, dtype=dtype, seed=L)
@@ -80,6 +81,22 @@ def test_prefill_edge_shapes(pv, gu, dtype, L, g, c, k, guard):
         t = acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=guard, out_idx=out,
                               out_scores=sc, cand=cand, cand_scores=cs)
         _report(f"edge L={L} g={g} c={c} k={k} {dtype} mode={mode}", t)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+def test_prefill_candidate_budget_beyond_the_shared_memory_rows(pv, gu, dtype):
+    """c above 4096 (and not a multiple of the tile): the re-score keeps its score rows in the
+    global segments instead of shared memory, the scan selects more than 4096 per row."""
+    L, g, c, k = 9000, 4, 5000, 2500
+    x = inputs.make_prefill(L, dtype=dtype, seed=32)
+    out, sc, cand, cs = gu.run_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE)
+    nG = (L + g - 1) // g
+    groups = [0, 1, 1249, 1250, 1251, 1500, 2000, nG - 1]           # guarded, at the guardrail, proxy groups
+    t = acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=po.MODE_REFINE, guard_len=None, out_idx=out,
+                          out_scores=sc, cand=cand, cand_scores=cs, groups=groups)
+    _report(f"large c {dtype}", t)
+    plain, _, _, _ = gu.run_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE, debug=False)
+    assert np.array_equal(np.sort(plain, axis=1), np.sort(out, axis=1))
 
 
 def test_group_of_one_equals_dense_on_gpu(pv, gu):
