@@ -181,11 +181,13 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       uint32_t pend_it = 0, pend_blk = 0, w_blk = 0xffffffffu;
       auto issue_mma2 = [&]() -> bool {
         if (pend_blk != w_blk) {                 // first tile of a group: its gate matrix must be in place
-          if (!ptx::mbar_wait(&ct.w_ready, pend_blk & 1, abort_flag, 32)) return false;
+          if (!ptx::mbar_wait(&ct.w_ready, pend_blk & 1, abort_flag, 0)) return false;
           w_blk = pend_blk;
         }
         const int pb = pend_it & 1;
-        if (!ptx::mbar_wait(&ct.a_ready[pb], (pend_it >> 1) & 1, abort_flag, 32)) return false;
+        // no sleep between polls here or on the accumulator / key-stage waits below: this thread's
+        // wake-up latency sits on the tile loop's critical path (four handoffs per tile)
+        if (!ptx::mbar_wait(&ct.a_ready[pb], (pend_it >> 1) & 1, abort_flag, 0)) return false;
         ptx::tc_fence_after();
         const uint32_t w_addr = ptx::smem_u32(ct.wmat);
         const uint32_t a_tmem = tmem_base + pb * N;
@@ -211,9 +213,9 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
           const int s = it % C::STAGES;
           const uint32_t ph = (it / C::STAGES) & 1;
           const int buf = it & 1;
-          ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, 32);
+          ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, 0);
           if (!ok) break;
-          ok = ptx::mbar_wait(&ct.full[s], ph, abort_flag, 32);
+          ok = ptx::mbar_wait(&ct.full[s], ph, abort_flag, 0);
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t k_addr = ptx::smem_u32(kring + s * C::STAGE_BYTES);
