@@ -187,7 +187,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         const int pb = pend_it & 1;
         // no sleep between polls here or on the accumulator / key-stage waits below: this thread's
         // wake-up latency sits on the tile loop's critical path (four handoffs per tile)
-        if (!ptx::mbar_wait(&ct.a_ready[pb], (pend_it >> 1) & 1, abort_flag, 0)) return false;
+        if (!ptx::mbar_wait_poll(&ct.a_ready[pb], (pend_it >> 1) & 1, abort_flag)) return false;
         ptx::tc_fence_after();
         const uint32_t w_addr = ptx::smem_u32(ct.wmat);
         const uint32_t a_tmem = tmem_base + pb * N;
@@ -213,9 +213,9 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
           const int s = it % C::STAGES;
           const uint32_t ph = (it / C::STAGES) & 1;
           const int buf = it & 1;
-          ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, 0);
+          ok = ptx::mbar_wait_poll(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag);
           if (!ok) break;
-          ok = ptx::mbar_wait(&ct.full[s], ph, abort_flag, 0);
+          ok = ptx::mbar_wait_poll(&ct.full[s], ph, abort_flag);
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t k_addr = ptx::smem_u32(kring + s * C::STAGE_BYTES);
