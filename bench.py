@@ -46,7 +46,7 @@ H, D = 64, 128
 FLOP_PER_SCORE = 2 * H * D
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/ (same workloads as the ones timed here)
-TRAFFIC_BYTES = {"prefill_128k_fp8_refine_g4": 2772653568 + 4299215616,
+TRAFFIC_BYTES = {"prefill_128k_fp8_refine_g4": 2780454144 + 4301106432,
                  "decode_scan_kernel": 403583488 + 12487936}
 
 
