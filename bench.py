@@ -382,6 +382,9 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-indexer control")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--shard-request", action="store_true",
+                    help="N > 1: all ranks share ONE request (row blocks dealt in snake order, one all-gather of the "
+                         "index sets per step) instead of one request per rank; reported as strong scaling")
     ap.add_argument("--decode-only", action="store_true", help="only the MTP decode step (prints its object)")
     ap.add_argument("--sweep", action="store_true",
                     help="g / c / pooling / window sweep with recall of the dense top-k (one JSON line per case)")
@@ -409,7 +412,10 @@ def main():
         print(json.dumps(decode_bench(pv, torch.device(f"cuda:{local}"), steps=max(args.steps, 5),
                                       warmup=max(args.warmup, 3), pk=peaks())))
         return
-    x = inputs.make_prefill(L, dtype=dtype, seed=rank_seed(rank))
+    shard = args.shard_request
+    if shard:                                   # the strong-scaling line carries the device-timed value only
+        args.no_e2e = args.no_decode = args.no_dense = args.no_cpu_baseline = True
+    x = inputs.make_prefill(L, dtype=dtype, seed=rank_seed(0 if shard else rank))
     dev = torch.device(f"cuda:{local}")
     dq, dw, dk = x.q.to(dev), x.w.to(dev), x.k.to(dev)
     dqs = None if x.qscale is None else x.qscale.to(dev)
@@ -420,6 +426,13 @@ def main():
     stream = torch.cuda.current_stream()
 
     def step():
+        if shard:
+            from paper_2607_24593_b200 import sharded
+            sharded.pivot_index_prefill_sharded(dq, dw, dk, L, H, D, g, c, k, mode, out, rank=rank, world=world,
+                                                stream=stream, q_scale=dqs, k_scale=dks, W=args.window)
+            if world > 1:
+                sharded.all_gather_rows(out, L, g, world, rank)
+            return
         pv.pivot_index_prefill(dq, dw, dk, L, H, D, g, c, k, mode, out, stream, q_scale=dqs, k_scale=dks,
                                W=args.window)
 
@@ -452,7 +465,7 @@ def main():
     assert pv.pivot_device_status() == 0, "device status word set during the timed region"
     elapsed_ms = max_over_ranks(elapsed_ms, dist, dev)
     ms_per_step = elapsed_ms / args.steps
-    value = job_throughput(world, L, ms_per_step)
+    value = job_throughput(1 if shard else world, L, ms_per_step)     # sharded: one request, whoever indexes it
 
     # ---- the dense indexer (Eq. 1 for every query: the O(L^2) control PIVOT replaces) on the same
     #      inputs, same kernels, same GPU: gives the PIVOT / dense ratio to set beside the paper's
@@ -534,9 +547,9 @@ def main():
     line = {
         "metric": "indexed query tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "e4m3" if dtype == "fp8" else "bf16",
+        "scaling": "strong" if shard else "weak", "vs_baseline": None, "dtype": "e4m3" if dtype == "fp8" else "bf16",
         "data": "synthetic",
-        "config": {"workload": wl, "L": L, "H_I": H, "d": D, "g": g, "c": c, "k": k,
+        "config": {"workload": wl, "sharding": "one request over all ranks" if shard else "one request per rank", "L": L, "H_I": H, "d": D, "g": g, "c": c, "k": k,
                    "mode": "refine" if mode else "reuse", "operands": dtype, "W": args.window, "proxy_groups": n_proxy,
                    "dense_rows": n_dense, "l2": "inputs larger than L2 (queries >= 1 GB per step)"
                    if L * H * D >= 2 ** 28 else "inputs smaller than L2; no flush"},

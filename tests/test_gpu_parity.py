@@ -295,6 +295,26 @@ def test_plain_call_matches_the_call_with_debug_buffers(pv, gu, dtype):
     assert np.array_equal(_sorted_rows(plain), _sorted_rows(dbg))
 
 
+def test_sharded_request_blocks_match_whole_call(pv):
+    """The multi-GPU form of one request (row blocks dealt to ranks in snake order), with the
+    ranks' shares indexed one after the other on this GPU: together they give the whole call."""
+    from paper_2607_24593_b200 import sharded
+    L, g, c, k = 3000, 4, 256, 128
+    x = inputs.make_prefill(L, dtype="fp8", seed=79)
+    q, w, kk, qs, ks = x.q.cuda(), x.w.cuda(), x.k.cuda(), x.qscale.cuda(), x.kscale.cuda()
+    whole = torch.full((L, k), -7, dtype=torch.int32, device="cuda")
+    pv.pivot_index_prefill(q, w, kk, L, 64, 128, g, c, k, pv.REFINE, whole, q_scale=qs, k_scale=ks)
+    parts = torch.full((L, k), -7, dtype=torch.int32, device="cuda")
+    covered = 0
+    for rank in range(3):
+        mine = sharded.pivot_index_prefill_sharded(q, w, kk, L, 64, 128, g, c, k, pv.REFINE, parts, rank=rank, world=3,
+                                                   block_rows=400, q_scale=qs, k_scale=ks)
+        covered += sum(r1 - r0 for r0, r1 in mine)
+    torch.cuda.synchronize()
+    assert covered == L and pv.pivot_device_status() == 0
+    assert np.array_equal(_sorted_rows(parts.cpu().numpy()), _sorted_rows(whole.cpu().numpy()))
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "fp8"])
 @pytest.mark.parametrize("mode", [po.MODE_REUSE, po.MODE_REFINE])
 def test_prefill_row_ranges_match_whole_call(pv, dtype, mode):

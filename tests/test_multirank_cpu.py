@@ -44,3 +44,63 @@ def test_two_ranks_index_independent_requests():
         assert ret["slowest"] == 20.0                       # max over ranks, not the mean
         assert abs(ret["value"] - 2 * 256 / 20e-3) < 1e-6   # all ranks' tokens over the slowest time
         assert ret["digests"][0] != ret["digests"][1]       # different requests per rank
+
+
+# ---------------------------------------------------------------- one request sharded over the ranks
+
+def test_row_blocks_cover_the_request_and_balance():
+    from paper_2607_24593_b200 import sharded
+    for L, g, world, br in [(131072, 4, 8, 8192), (1000, 3, 2, 64), (7, 4, 4, 8), (50000, 8, 3, 4096)]:
+        blocks = sharded.row_blocks(L, g, br)
+        assert blocks[0][0] == 0 and blocks[-1][1] == L
+        assert all(a[1] == b[0] for a, b in zip(blocks[:-1], blocks[1:]))
+        assert all(r0 % g == 0 for r0, _ in blocks)                       # whole groups
+        seen = sorted(b for r in range(world) for b in sharded.my_blocks(L, g, world, r, br))
+        assert seen == blocks                                             # every block has exactly one owner
+    assert [sharded.owner(i, 4) for i in range(10)] == [0, 1, 2, 3, 3, 2, 1, 0, 0, 1]
+    assert sharded.imbalance(131072, 4, 8) < 1.01                         # snake order pairs cheap with expensive blocks
+    assert sharded.imbalance(131072, 4, 8) < sum(
+        sharded.block_cost(b) for i, b in enumerate(sharded.row_blocks(131072, 4)) if i % 8 == 7) / (
+        sum(sharded.block_cost(b) for b in sharded.row_blocks(131072, 4)) / 8)   # plain cyclic is worse
+
+
+def _shard_worker(rank, world, port, ret):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    from oracle import pivot_oracle as po
+    from paper_2607_24593_b200 import inputs, sharded
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    L, g, c, k, br = 300, 4, 32, 16, 40
+    x = inputs.make_prefill(L, 4, 8, dtype="bf16", seed=5, threads=1).codes()      # the same request on every rank
+    out = torch.full((L, k), -7, dtype=torch.int32)
+
+    def index_rows(b):                      # stands in for the library's chunked prefill (rows=(r0, r1))
+        r0, r1 = b
+        res = po.pivot_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE, groups=range(r0 // g, (r1 + g - 1) // g))
+        for gr in res.values():
+            out[torch.from_numpy(gr.members)] = torch.from_numpy(gr.T)
+
+    mine = sharded.index_my_rows(index_rows, L, g, world, rank, br)
+    untouched = torch.ones(L, dtype=torch.bool)
+    for r0, r1 in mine:
+        untouched[r0:r1] = False
+    assert (out[untouched] == -7).all()     # a rank writes its own rows only
+    sharded.all_gather_rows(out, L, g, world, rank, br)
+    if rank == 0:
+        ret["out"] = out.numpy().copy()
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_one_request_sharded_over_two_ranks_matches_one_process():
+    from oracle import pivot_oracle as po
+    from paper_2607_24593_b200 import inputs
+    with mp.Manager() as m:
+        ret = m.dict()
+        port = 31500 + (os.getpid() % 2000)
+        mp.spawn(_shard_worker, args=(2, port, ret), nprocs=2, join=True)
+        got = ret["out"]
+    L, g, c, k = 300, 4, 32, 16
+    x = inputs.make_prefill(L, 4, 8, dtype="bf16", seed=5, threads=1).codes()
+    want = po.assemble(po.pivot_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE), L, k)
+    assert np.array_equal(got, want)
