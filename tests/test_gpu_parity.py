@@ -99,6 +99,40 @@ def test_prefill_candidate_budget_beyond_the_shared_memory_rows(pv, gu, dtype):
     assert np.array_equal(np.sort(plain, axis=1), np.sort(out, axis=1))
 
 
+def _random_configs(n, seed):
+    rng = np.random.default_rng(seed)
+    cfgs = []
+    while len(cfgs) < n:
+        L = int(rng.integers(1, 1400))
+        g = int(rng.integers(1, 10))
+        k = int(rng.integers(1, 300))
+        c = int(k + rng.integers(0, 400))
+        mode = int(rng.integers(0, 2))
+        dtype = ("bf16", "fp8")[int(rng.integers(0, 2))]
+        guard = (None, 0, int(rng.integers(1, c + 50)))[int(rng.integers(0, 3))]
+        W = 0
+        if rng.integers(0, 3) == 0:                              # a third of the cases with a local window
+            W = int(rng.integers(1, 9))
+            eff_guard = c if guard is None else guard
+            if W + g - 1 >= c or eff_guard < W + g:
+                continue
+        pool = ("mean", "first", "last")[int(rng.integers(0, 3))]
+        cfgs.append((L, g, c, k, mode, dtype, guard, W, pool))
+    return cfgs
+
+
+@pytest.mark.parametrize("cfg", _random_configs(28, 20260724), ids=lambda c: "L{}-g{}-c{}-k{}-m{}-{}-gd{}-W{}-{}".format(*c))
+def test_prefill_random_small_configs(pv, gu, cfg):
+    """Seeded random shapes (lengths, group sizes, budgets, guardrails, windows, pooling, both
+    operand types and variants): the whole request against the oracle."""
+    L, g, c, k, mode, dtype, guard, W, pool = cfg
+    x = inputs.make_prefill(L, dtype=dtype, seed=1000 + L)
+    pools = {"mean": pv.POOL_MEAN, "first": pv.POOL_FIRST, "last": pv.POOL_LAST}
+    out, sc, cand, cs = gu.run_prefill(x, g=g, c=c, k=k, mode=mode, guard_len=guard, pool=pools[pool], W=W)
+    acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=guard, out_idx=out, out_scores=sc,
+                      cand=cand, cand_scores=cs, pool=pool, W=W)
+
+
 def test_group_of_one_equals_dense_on_gpu(pv, gu):
     """Appendix A: g = 1 recovers the dense indexer -- on the GPU outputs themselves."""
     x = inputs.make_prefill(700, dtype="bf16", seed=9)
