@@ -211,6 +211,42 @@ def test_decode_more_than_1024_sequences(pv, gu):
     assert t.rows > 0
 
 
+def _random_decode_configs(n, seed):
+    rng = np.random.default_rng(seed)
+    cfgs = []
+    while len(cfgs) < n:
+        B = int(rng.integers(1, 7))
+        g = int(rng.integers(1, 6))
+        lo = int(rng.integers(1, 1500))
+        hi = lo + int(rng.integers(0, 1500))
+        k = int(rng.integers(1, 200))
+        c = int(k + rng.integers(0, 300))
+        mode = int(rng.integers(0, 2))
+        dtype = ("bf16", "fp8")[int(rng.integers(0, 2))]
+        paged = bool(rng.integers(0, 3) == 0)
+        guard = 0 if paged else (None, 0, int(rng.integers(1, c + 50)))[int(rng.integers(0, 3))]
+        W = 0
+        if mode == 1 and rng.integers(0, 3) == 0:
+            W = int(g + rng.integers(0, 12))
+        cfgs.append((B, g, lo, hi, c, k, mode, dtype, guard, W, paged))
+    return cfgs
+
+
+@pytest.mark.parametrize("cfg", _random_decode_configs(20, 20260725),
+                         ids=lambda c: "B{}-g{}-n{}..{}-c{}-k{}-m{}-{}-gd{}-W{}-pg{}".format(*c))
+def test_decode_random_small_configs(pv, gu, cfg):
+    """Seeded random decode steps (batch, MTP width, prefix lengths, budgets, guardrails, window,
+    contiguous or paged cache, both operand types and variants) against the oracle."""
+    B, g, lo, hi, c, k, mode, dtype, guard, W, paged = cfg
+    x = inputs.make_decode(B, g, lo, hi, dtype=dtype, seed=2000 + lo)
+    if paged:
+        out, sc, cand, cs = gu.run_decode_paged(x, c=c, k=k, mode=mode, seed=lo, W=W)
+    else:
+        out, sc, cand, cs = gu.run_decode(x, c=c, k=k, mode=mode, guard_len=guard, W=W)
+    acc.check_decode(x.codes(), c=c, k=k, mode=mode, guard_len=guard, out_idx=out, out_scores=sc,
+                     cand=cand, cand_scores=cs, W=W)
+
+
 def test_decode_group_of_four(pv, gu):
     x = inputs.make_decode(3, 4, 2000, 2600, dtype="fp8", seed=22)
     out, sc, cand, cs = gu.run_decode(x, c=256, k=128, mode=po.MODE_REFINE)
