@@ -98,9 +98,8 @@ class ClockSampler:
     def __init__(self, index):
         self.index, self.samples, self.stop, self.th = index, [], threading.Event(), None
 
-    def _run(self):
-        # NVML queries (reads only) take well under a millisecond, so even a timed region of a few
-        # steps is sampled many times; nvidia-smi (one process per sample) is the fallback.
+    def _nvml_open(self):
+        """NVML handle and constants, opened before the timed region (the first init takes a while)."""
         try:
             import pynvml
             pynvml.nvmlInit()
@@ -108,17 +107,28 @@ class ClockSampler:
             mx = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
             get_reasons = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
                 pynvml.nvmlDeviceGetCurrentClocksThrottleReasons
-            bits = ((0x8, 2), (0x40, 3), (0x20, 4), (0x4, 5))     # hw_slowdown, hw_thermal, sw_thermal, sw_power_cap
-            while not self.stop.is_set():
-                r = int(get_reasons(h))
-                row = [str(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)), str(mx), "", "", "", ""]
-                for bit, col in bits:
-                    row[col] = "Active" if r & bit else "Not Active"
-                self.samples.append(row)
-                self.stop.wait(0.01)
-            return
+            get_reasons(h)
+            return pynvml, h, mx, get_reasons
         except Exception:
-            pass
+            return None
+
+    def _run(self):
+        # NVML queries (reads only) take well under a millisecond, so even a timed region of a few
+        # steps is sampled many times; nvidia-smi (one process per sample) is the fallback.
+        if self.nvml is not None:
+            pynvml, h, mx, get_reasons = self.nvml
+            bits = ((0x8, 2), (0x40, 3), (0x20, 4), (0x4, 5))     # hw_slowdown, hw_thermal, sw_thermal, sw_power_cap
+            try:
+                while not self.stop.is_set():
+                    r = int(get_reasons(h))
+                    row = [str(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)), str(mx), "", "", "", ""]
+                    for bit, col in bits:
+                        row[col] = "Active" if r & bit else "Not Active"
+                    self.samples.append(row)
+                    self.stop.wait(0.005)
+                return
+            except Exception:
+                pass
         while not self.stop.is_set():
             try:
                 out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
@@ -129,6 +139,7 @@ class ClockSampler:
             self.stop.wait(0.15)
 
     def __enter__(self):
+        self.nvml = self._nvml_open()
         self.th = threading.Thread(target=self._run, daemon=True)
         self.th.start()
         return self
