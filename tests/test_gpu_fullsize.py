@@ -76,6 +76,13 @@ def test_config5_prefill_256k_fp8_refine():
     _run_and_check(262144, "fp8", 4, 4096, 2048, po.MODE_REFINE, n_random=12)
 
 
+def test_prefill_512k_fp8_refine_beyond_the_benchmark_sizes():
+    """Four times the headline length (4.3 GB of queries, 131072 groups): sizes and offsets past
+    the benchmark's, same launch path."""
+    _run_and_check(524288, "fp8", 4, 4096, 2048, po.MODE_REFINE, n_random=2)
+    _cache.clear()
+
+
 def test_config4_decode_mtp_groups():
     """32 sequences, prefix lengths uniform in [64K, 128K], FP8 cache, g = 2, Refine."""
     import gpu_util
