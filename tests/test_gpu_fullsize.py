@@ -98,3 +98,13 @@ def test_config4_decode_mtp_groups():
         for i in range(2):
             assert out[b, i].min() >= 0 and out[b, i].max() <= pos0[b] + i
             assert len(np.unique(out[b, i])) == 2048
+
+
+def test_decode_million_key_sequences():
+    """Two sequences of about a million keys each (eight times the benchmark's longest)."""
+    import gpu_util
+    x = inputs.make_decode(2, 2, 900000, 1048000, dtype="fp8", seed=41)
+    out, sc, cand, cs = gpu_util.run_decode(x, c=4096, k=2048, mode=po.MODE_REFINE)
+    t = acc.check_decode(x.codes(), c=4096, k=2048, mode=po.MODE_REFINE, guard_len=None, out_idx=out,
+                         out_scores=sc, cand=cand, cand_scores=cs)
+    assert t.rows == 6          # per sequence: the candidate set and its two queries
