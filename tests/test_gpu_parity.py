@@ -365,6 +365,33 @@ def test_plain_call_matches_the_call_with_debug_buffers(pv, gu, dtype):
     assert np.array_equal(_sorted_rows(plain), _sorted_rows(dbg))
 
 
+def test_two_streams_with_their_own_workspaces(pv):
+    """Two requests indexed at the same time on two streams, each call with its own workspace
+    (pivot_opts.workspace): same results as one after the other."""
+    L, g, c, k = 6000, 4, 512, 256
+    xs = [inputs.make_prefill(L, dtype="fp8", seed=80 + i) for i in range(2)]
+    dev = [dict(q=x.q.cuda(), w=x.w.cuda(), k=x.k.cuda(), qs=x.qscale.cuda(), ks=x.kscale.cuda()) for x in xs]
+    nG = (L + g - 1) // g
+    ws = [torch.empty(pv.pivot_workspace_bytes(L, nG, c, k), dtype=torch.uint8, device="cuda") for _ in range(2)]
+    serial = []
+    for d, wsp in zip(dev, ws):
+        o = torch.full((L, k), -7, dtype=torch.int32, device="cuda")
+        pv.pivot_index_prefill(d["q"], d["w"], d["k"], L, 64, 128, g, c, k, pv.REFINE, o, q_scale=d["qs"],
+                               k_scale=d["ks"], workspace=wsp)
+        serial.append(o)
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    both = [torch.full((L, k), -7, dtype=torch.int32, device="cuda") for _ in range(2)]
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for d, wsp, st, o in zip(dev, ws, streams, both):
+            pv.pivot_index_prefill(d["q"], d["w"], d["k"], L, 64, 128, g, c, k, pv.REFINE, o, st, q_scale=d["qs"],
+                                   k_scale=d["ks"], workspace=wsp)
+    torch.cuda.synchronize()
+    for a, b in zip(serial, both):
+        assert np.array_equal(_sorted_rows(a.cpu().numpy()), _sorted_rows(b.cpu().numpy()))
+
+
 def test_sharded_request_blocks_match_whole_call(pv):
     """The multi-GPU form of one request (row blocks dealt to ranks in snake order), with the
     ranks' shares indexed one after the other on this GPU: together they give the whole call."""
