@@ -353,18 +353,19 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
   p.block_table = block_table;
   p.n_pages = n_pages;
   const long long k_rows = paged ? (long long)n_pages * 128 : (long long)B * Lmax;
-  if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 2 * sizeof(int), st)))) return rc;
+  if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 3 * sizeof(int), st)))) return rc;   // status, row counter, prepare ticket
   mark(0, st);
   launch_proxy_build(q->data, q->scale, w, ws.proxy_q, ws.proxy_w, B * g, g, 0, B, q->dtype,
                      o ? o->pool : 0, st);
   mark(1, st);
-  launch_plan_decode(p, ws.rows, ws.groups, st);
+  if (o && o->impl == 1) launch_plan_decode(p, ws.rows, ws.groups, st);   // the tensor-core path plans inside its prepare kernel
   mark(2, st);
   if (o && o->impl == 1) {
     launch_scan_simt(ws.rows, B + B * g, q->dtype, ws.scan, st);
   } else {
     // proxy rows: key-tile-split scan, per-sequence select, chunked re-score, final top-k
     DecodeFast df;
+    df.plan = p; df.ticket = ws.status + 2;
     df.prox = ws.rows; df.groups = ws.groups;
     df.kc = kcache->data; df.kscale = kcache->scale; df.q = q->data; df.proxy_q = ws.proxy_q;
     df.B = B; df.Lmax = Lmax; df.g = g; df.c = c; df.k = k; df.mode = mode; df.dtype = q->dtype;

@@ -26,6 +26,7 @@
 
 #include "blockselect.cuh"
 #include "kernels.h"
+#include "plan.cuh"
 #include "ptx.cuh"
 
 namespace pivot {
@@ -423,9 +424,32 @@ __global__ void __launch_bounds__(kBlk, 1) entries_topk_kernel(const EntryList* 
 
 // ------------------------------------------------------------------------------ setup
 
-__global__ void decode_setup_kernel(const RowDesc* __restrict__ prox, const GroupDesc* __restrict__ groups, int B,
-                                    int g, int c, int k, int mode, int W, int* tile_prefix, GroupDesc* chunks,
-                                    EntryList* lists, unsigned long long* entries, const int32_t* wcand) {
+// One launch prepares a decode step: block b clears sequence b's histogram and list counters and
+// plans the sequence (row and group descriptors, guard test on the device-resident pos0); the
+// block that finishes last -- nobody waits for anybody -- then has every descriptor in front of
+// it and derives what spans sequences: the tile prefix of the key-split scan, the candidate
+// chunks of the re-score and the entry lists of the final top-k.  1024 threads per block.
+__global__ void __launch_bounds__(1024)
+decode_prepare_kernel(DecodePlan p, RowDesc* rows, GroupDesc* plan_groups, uint32_t* ghist, int* ticket, int W,
+                      int* tile_prefix, GroupDesc* chunks, EntryList* lists, unsigned long long* entries,
+                      const int32_t* wcand) {
+  {
+    const int b = blockIdx.x;
+    for (int i = threadIdx.x; i < DHIST; i += blockDim.x) ghist[(size_t)b * DHIST + i] = 0u;
+    if (threadIdx.x < 2) ghist[(size_t)p.B * DHIST + 2 * b + threadIdx.x] = 0u;      // list length, delivered shares
+    if (threadIdx.x == 0) plan_decode_sequence(p, b, rows, plan_groups);
+    __threadfence();
+    __shared__ int is_last;
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = atomicAdd(ticket, 1) == (int)gridDim.x - 1;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    if (threadIdx.x == 0) *ticket = 0;              // ready for the next step
+  }
+  const RowDesc* prox = rows;
+  const GroupDesc* groups = plan_groups;
+  const int B = p.B, g = p.g, c = p.c, k = p.k, mode = p.mode;
   // tile_prefix = exclusive prefix sum of the sequences' tile counts (any B: 1024 at a time)
   __shared__ int wsum[32];
   __shared__ int carry;
@@ -572,11 +596,11 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   int32_t* wcand = (int32_t*)p;              p += up((size_t)d.B * kDecodeWinMax * 4);
   unsigned long long* entries = (unsigned long long*)p;
 
-  cudaError_t e = cudaMemsetAsync(ghist, 0, (size_t)d.B * (DHIST + 2) * 4, st);
-  if (e != cudaSuccess) return e;
-  decode_setup_kernel<<<1, 1024, 0, st>>>(d.prox, d.groups, d.B, d.g, d.c, d.k, d.mode, W, tile_prefix, chunks,
-                                          lists, entries, wcand);
+  decode_prepare_kernel<<<d.B, 1024, 0, st>>>(d.plan, d.prox, d.groups, ghist, d.ticket, W, tile_prefix, chunks, lists,
+                                              entries, wcand);
   ++launch_counter();
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
   CUtensorMap mk, mq, mks;
   memset(&mks, 0, sizeof(mks));
   if (d.dtype == DT_FP8 && !make_scale_map(&mks, d.kscale, d.k_rows)) return cudaErrorInvalidValue;

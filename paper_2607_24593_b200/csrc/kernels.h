@@ -120,8 +120,10 @@ cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDe
 
 // Decode fast path: key-tile-split scan -> per-sequence select -> chunked re-score -> top-k.
 struct DecodeFast {
-  const RowDesc* prox;        // [B] proxy rows (K = 0: guarded sequence, skipped)
-  const GroupDesc* groups;    // [B * group_chunks(g)]
+  DecodePlan plan;            // the call's geometry: the prepare kernel plans the sequences itself
+  int* ticket;                // one zeroed int (counts the prepare kernel's finished blocks)
+  RowDesc* prox;              // [B + B * g] row slots; [0, B) = proxy rows (K = 0: guarded sequence, skipped)
+  GroupDesc* groups;          // [B * group_chunks(g)]
   const void* kc; const float* kscale; const void* q; const void* proxy_q;
   int B, Lmax, g, c, k, mode, dtype, sms;
   long long k_rows;           // rows of the key tensor (B * Lmax, or pool pages * 128 when paged)
