@@ -3,6 +3,8 @@
 // One MTP step scores one proxy per sequence against that sequence's whole key cache, so the
 // step is a single pass over every visible key (128 B + 4 B scale): memory bound.  The work is
 // therefore split by KEY TILES, not by rows:
+//   decode_prepare_kernel one block per sequence clears its histogram and plans it; the block that
+//                        finishes last derives the tile prefix, candidate chunks and entry lists.
 //   decode_scan_kernel   every SM takes an equal, contiguous share of all (sequence, 128-key
 //                        tile) pairs; per tile: TMA -> tcgen05 MMA (128 keys x 64 heads x d) ->
 //                        epilogue (ReLU, gate-weighted head sum, key scale) -> one fp32 score per
