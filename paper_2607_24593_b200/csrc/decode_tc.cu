@@ -630,7 +630,7 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
       ++launch_counter();
     }
     ScanScratch sc = d.scratch_tc;
-    e = launch_refine_tc(d.q, d.B * d.g, d.dtype, chunks, d.B * mc * nch, sc, d.sms, st);
+    e = launch_refine_tc(d.q, d.B * d.g, d.dtype, chunks, d.B * mc * nch, sc, d.sms, st, false, true);
     if (e != cudaSuccess) return e;
     entries_topk_kernel<<<d.B * d.g, kBlk, 0, st>>>(lists);
     ++launch_counter();

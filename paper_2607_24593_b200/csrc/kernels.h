@@ -116,7 +116,8 @@ cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_ro
                            const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum = false);
 
 cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
-                             const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum = false);
+                             const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum = false,
+                             bool chunked = false);
 
 // Decode fast path: key-tile-split scan -> per-sequence select -> chunked re-score -> top-k.
 struct DecodeFast {

@@ -28,7 +28,10 @@ constexpr int THREADS = (2 + GATHER_WARPS + EPI_WARPS) * 32;   // 384: 168 regis
 constexpr int N = NMEM * kHeads;
 constexpr int TMEM_COLS = 2 * N;
 
-// EPI: 1 = tensor-core head sum where available (FP8), 0 = fp32 FMA head sum.
+// EPI: 1 = tensor-core head sum where available (FP8), 0 = fp32 FMA head sum, 2 = as 1 for the
+// candidate chunks of a decode step: those leave packed entries for a later top-k, so the score
+// rows need no shared memory and a second query buffer takes their place (the next chunk's
+// queries load while the current one is re-scored).
 template <int DT, int EPI = 1>
 struct RCfg {
   static constexpr bool FP8 = DT == DT_FP8;
@@ -41,7 +44,7 @@ struct RCfg {
   // FP8 keeps the group's score keys in shared memory (4 members x 4096 slots x 4 B) for the
   // final top-k; bf16 has no room for that next to 2 x 64 KB of queries and goes through the
   // per-CTA global segments instead.
-  static constexpr bool SMEM_SCORES = FP8;
+  static constexpr bool SMEM_SCORES = FP8 && EPI != 2;
   // With the score rows resident, one query buffer (the next group's queries load while the
   // key ring refills) buys two more gather stages, which matter more.
   static constexpr int QBUFS = SMEM_SCORES ? 1 : 2;
@@ -52,7 +55,7 @@ struct RCfg {
   // FP8: the gate-weighted head sum of Eq. 8 runs on the tensor core, as in the shared scan (a
   // second MMA over bf16 ReLU values written in place in tensor memory against a block-diagonal
   // gate matrix).  bf16 operands keep the fp32 FMA head sum.
-  static constexpr bool MMA2 = FP8 && EPI == 1;
+  static constexpr bool MMA2 = FP8 && EPI != 0;
   static constexpr uint32_t IDESC2 = ptx::make_idesc(1u, TILE_KEYS, 16);
   static constexpr int TMEM_EMPTY_ARRIVALS = MMA2 ? 4 : EPI_WARPS;
 };
@@ -93,7 +96,7 @@ constexpr size_t rsmem_bytes() {
   return 1024 + C::QBUFS * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(RCtrlT<C::MMA2>) +
          (C::SMEM_SCORES ? (size_t)NMEM * SCORE_SLOTS * 4 : 0);
 }
-static_assert(rsmem_bytes<DT_FP8, 1>() <= 232448 && rsmem_bytes<DT_FP8, 0>() <= 232448 &&
+static_assert(rsmem_bytes<DT_FP8, 1>() <= 232448 && rsmem_bytes<DT_FP8, 0>() <= 232448 && rsmem_bytes<DT_FP8, 2>() <= 232448 &&
               rsmem_bytes<DT_BF16>() <= 232448, "shared memory budget");
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -565,13 +568,14 @@ cudaError_t launch_one(const CUtensorMap& mq, const GroupDesc* groups, int n_gro
 bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows);
 
 cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
-                             const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum) {
+                             const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum, bool chunked) {
   if (n_groups <= 0) return cudaSuccess;
   CUtensorMap mq;
   if (!make_operand_map(&mq, q, (long long)q_rows * kHeads, dtype, kHeads)) return cudaErrorInvalidValue;
   if (dtype != DT_FP8) return launch_one<DT_BF16>(mq, groups, n_groups, q_rows, s, sms, st);
-  return fp32_head_sum ? launch_one<DT_FP8, 0>(mq, groups, n_groups, q_rows, s, sms, st)
-                       : launch_one<DT_FP8, 1>(mq, groups, n_groups, q_rows, s, sms, st);
+  if (fp32_head_sum) return launch_one<DT_FP8, 0>(mq, groups, n_groups, q_rows, s, sms, st);
+  return chunked ? launch_one<DT_FP8, 2>(mq, groups, n_groups, q_rows, s, sms, st)
+                 : launch_one<DT_FP8, 1>(mq, groups, n_groups, q_rows, s, sms, st);
 }
 
 }  // namespace pivot
