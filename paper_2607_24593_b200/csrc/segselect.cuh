@@ -326,8 +326,9 @@ __device__ __forceinline__ int seg_compact(const Team& tm, SegSelSmem& sm, const
   }
 }
 
-// Final selection of a row: writes min(K, n_valid) positions (unordered) to out, returns how
-// many.  n_valid = real (non-padding) entries in the team's segments.
+// Final selection of a row: writes the K best real entries (fewer if the segments hold fewer;
+// unordered) to out and returns how many.  n_valid = an upper bound on the real (non-padding)
+// entries in the team's segments, used only to skip the cut search when everything fits.
 template <bool CACHED, int EPT = kSelEpt>
 __device__ __forceinline__ int seg_emit(const Team& tm, SegSelSmem& sm, const Seg& seg, int n_valid, int32_t* out,
                                         float* out_score, int K) {
@@ -356,7 +357,10 @@ __device__ __forceinline__ int seg_emit(const Team& tm, SegSelSmem& sm, const Se
     }
   });
   tm.sync();
-  return n_valid > K ? K : n_valid;
+  // what was really written: n_valid is an upper bound only (masked window slots and slots of a
+  // short prefix are padding entries), and the caller pads the row from the returned count on
+  const int n_out = (int)sm.out_count;
+  return n_out > K ? K : n_out;
 }
 
 // Final selection of a row straight from its score histogram: `hist` counted every entry that

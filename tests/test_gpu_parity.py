@@ -133,6 +133,24 @@ def test_prefill_random_small_configs(pv, gu, cfg):
                       cand=cand, cand_scores=cs, pool=pool, W=W)
 
 
+@pytest.mark.parametrize("cfg", [
+    (5802, 1, 2378, 1105, 72, 5, "last"),      # guardrail far below c: rows with fewer valid candidates than k
+    (900, 4, 64, 64, None, 3, "mean"),         # c == k: the window slots a member may not see leave it short of k
+])
+def test_window_rows_with_fewer_candidates_than_k_are_padded(pv, gu, cfg):
+    """bf16 Refine with a local window: a member whose visible candidates number fewer than k
+    gets them all, and -1 after them (the row's tail must not keep what the buffer held)."""
+    L, g, c, k, guard, W, pool = cfg
+    pools = {"mean": pv.POOL_MEAN, "last": pv.POOL_LAST}
+    x = inputs.make_prefill(L, dtype="bf16", seed=5)
+    out, sc, cand, cs = gu.run_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE, guard_len=guard, pool=pools[pool], W=W)
+    assert (out >= -1).all()                                   # the -7 the buffer was filled with is gone everywhere
+    nG = (L + g - 1) // g
+    groups = sorted({0, 1, 20, 100 // g, 613 // g, nG // 2, nG - 1})
+    acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=po.MODE_REFINE, guard_len=guard, out_idx=out, out_scores=sc,
+                      cand=cand, cand_scores=cs, pool=pool, W=W, groups=groups)
+
+
 def test_group_of_one_equals_dense_on_gpu(pv, gu):
     """Appendix A: g = 1 recovers the dense indexer -- on the GPU outputs themselves."""
     x = inputs.make_prefill(700, dtype="bf16", seed=9)
