@@ -37,6 +37,24 @@ while time.time() - t0 < float(sys.argv[2]) if len(sys.argv) > 2 else 300:
         groups = sorted(set(rng.integers(0, nG, 12).tolist() + [0, nG - 1]))
         acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=guard, out_idx=out, out_scores=sc, cand=cand,
                           cand_scores=cs, pool=pool, W=W, groups=groups)
+        # the same request through other forms of the call: fp32 head sum, two row chunks, dense control
+        import torch
+        if dtype == "fp8" and rng.integers(0, 3) == 0:
+            o2 = gu.run_prefill(x, g=g, c=c, k=k, mode=mode, guard_len=guard, pool=pools[pool], W=W, impl=2)
+            acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=guard, out_idx=o2[0], out_scores=o2[1],
+                              cand=o2[2], cand_scores=o2[3], pool=pool, W=W, groups=groups)
+        if nG > 1 and rng.integers(0, 2) == 0:
+            d = gu.to_cuda(x)
+            cut = int(rng.integers(1, nG)) * g
+            parts = torch.full((L, k), -7, dtype=torch.int32, device="cuda")
+            for rows_ in ((0, cut), (cut, L)):
+                pv.pivot_index_prefill(d["q"], d["w"], d["k"], L, 64, 128, g, c, k, mode, parts, q_scale=d["qscale"],
+                                       k_scale=d["kscale"], guard_len=guard, pool=pools[pool], W=W, rows=rows_)
+            torch.cuda.synchronize()
+            assert np.array_equal(np.sort(parts.cpu().numpy(), axis=1), np.sort(out, axis=1)), "row chunks differ from the whole call"
+        if L <= 3000 and rng.integers(0, 3) == 0:
+            do, ds = gu.run_dense(x, k=k)
+            acc.check_dense(x.codes(), k=k, out_idx=do, out_scores=ds, rows=sorted(set(rng.integers(0, L, 10).tolist() + [0, L - 1])))
     except Exception as e:
         fails += 1
         print("FAIL prefill", cfg, repr(e)[:300]); traceback.print_exc(limit=2)
