@@ -1,6 +1,6 @@
 """Randomised parity soak (run by hand on a GPU machine; pytest does not collect it):
 
-    python tests/soak_gpu.py [seed] [seconds]
+    python tests/soak_gpu.py [seed] [seconds] [decode length scale]
 
 draws prefill and decode configurations at random from the seed -- lengths, group sizes, budgets,
 guardrails, local windows, pooling, operand types, contiguous or paged caches -- runs each through
@@ -17,6 +17,7 @@ from oracle import acceptance as acc, pivot_oracle as po
 from paper_2607_24593_b200 import inputs, binding as pv
 rng = np.random.default_rng(int(sys.argv[1]) if len(sys.argv) > 1 else 7)
 pools = {"mean": pv.POOL_MEAN, "first": pv.POOL_FIRST, "last": pv.POOL_LAST}
+DEC_MAX = int(sys.argv[3]) if len(sys.argv) > 3 else 6000        # decode prefix lengths up to about twice this
 fails = 0
 t0 = time.time()
 n = 0
@@ -60,7 +61,7 @@ while time.time() - t0 < float(sys.argv[2]) if len(sys.argv) > 2 else 300:
         print("FAIL prefill", cfg, repr(e)[:300]); traceback.print_exc(limit=2)
     n += 1
     # a decode step
-    B = int(rng.integers(1, 9)); gd = int(rng.integers(1, 7)); lo = int(rng.integers(1, 6000)); hi = lo + int(rng.integers(0, 6000))
+    B = int(rng.integers(1, 9)); gd = int(rng.integers(1, 7)); lo = int(rng.integers(1, DEC_MAX)); hi = lo + int(rng.integers(0, DEC_MAX))
     kd = int(rng.integers(1, 600)); cd = int(kd + rng.integers(0, 900)); md = int(rng.integers(0, 2)); paged = bool(rng.integers(0, 3) == 0)
     gdl = 0 if paged else (None, 0, int(rng.integers(1, cd + 50)))[int(rng.integers(0, 3))]
     Wd = int(gd + rng.integers(0, 12)) if (md == 1 and rng.integers(0, 3) == 0) else 0
