@@ -19,7 +19,7 @@ PIVOT approximates the dense indexer, so this oracle is the algorithm's steps in
 order, not the dense definition -- except for g = 1 and for guarded (short) groups, where it is
 the dense definition itself.
 
-Readings taken where the paper is silent (each also listed in the design notes):
+Readings taken where the paper is silent:
   * positions are 0-indexed here; a query at t sees keys s <= t (inclusive);
   * the proxy scan is cut at the group's first position t0, n0 = t0 + 1 keys visible;
   * guardrail: dense per member iff n0 < guard_len (default c), for both variants;
@@ -34,11 +34,14 @@ Readings taken where the paper is silent (each also listed in the design notes):
 
 Pins: every function is pinned by tests that do not call it to produce their expectation
 (hand-worked example, torch einsum/topk restatement, g = 1 identity, c >= n0 identity,
-identical-member identity, coverage identity, brute-force select, codec tables).  The prefill
-window variant's slot layout rests on the reading above alone: parity unpinned for W > 0 beyond
-the W = 0 reduction and the containment/coverage invariants.  The decode window variant is
-pinned by its reduction to the dense definition when pool and window cover every visible key,
-and by a set-membership restatement of "pool united with the query's own window".
+identical-member identity, coverage identity, brute-force select, codec tables; first / last
+pooling against the dense indexer's row of that member; the rounded proxy against the exact
+fp64 mean inside the score band).  The prefill window variant is pinned by its reduction to the
+dense definition over [0, t] when the proxy part and the window slots together hold every
+visible key, and by a torch restatement of its slot layout; the decode window variant by the
+same reduction and by a set-membership restatement of "pool united with the query's own
+window".  Parity unpinned: only the reading that the short-group guardrail also applies to
+Reuse (Algorithm 1 tests it before the variant branch; nothing else in the paper fixes it).
 """
 from __future__ import annotations
 

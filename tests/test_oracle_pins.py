@@ -415,3 +415,119 @@ def test_acceptance_rule_with_window_accepts_the_oracle_and_rejects_mutations():
     bad_out[first, 0] = first + 1           # a key the first member may not see
     with pytest.raises(AssertionError):
         acc.check_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE, guard_len=None, out_idx=bad_out, cand=cand, W=W, groups=[gi])
+
+
+# ---------------------------------------------------------------- pooling variants, prefill window, proxy rounding
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+def test_first_and_last_pooling_reduce_to_a_member_row_of_the_dense_indexer(dtype):
+    """Endpoint proxies of the pooling ablation: with pool = "first" the proxy IS the group's first
+    query, whose visible prefix is exactly the scan's [0, t0], so Reuse must return the dense
+    indexer's top-k of row t0 (torch restatement); with pool = "last" it is the last member's
+    query scored over [0, t0] only.  (bf16: the proxy is the member bit for bit; fp8: values that
+    already sit on the e4m3 grid re-quantise to themselves.)"""
+    L, g, k = 72, 4, 6
+    x = tiny(L=L, H=4, d=8, dtype=dtype)
+    I, sets = _torch_dense(x, k)
+    first = po.pivot_prefill(x, g=g, c=12, k=k, mode=po.MODE_REUSE, guard_len=0, pool="first")
+    last = po.pivot_prefill(x, g=g, c=12, k=k, mode=po.MODE_REUSE, guard_len=0, pool="last")
+    mean = po.pivot_prefill(x, g=g, c=12, k=k, mode=po.MODE_REUSE, guard_len=0)
+    differs = 0
+    for gi in first:
+        t0, tl = int(first[gi].t0), int(first[gi].members[-1])
+        if t0 + 1 < k:
+            continue
+        for T in first[gi].T:
+            assert set(T.tolist()) == sets[t0]
+        want_last = set(torch.topk(I[tl, : t0 + 1], k).indices.tolist())
+        for T in last[gi].T:
+            assert set(T.tolist()) == want_last
+        differs += set(mean[gi].T[0].tolist()) != sets[t0]
+    assert differs > 0, "mean pooling must differ from the first-member proxy somewhere in this case"
+    # Refine with the first-member proxy: the candidate set is row t0's dense top-c
+    r = po.pivot_prefill(x, g=g, c=12, k=k, mode=po.MODE_REFINE, guard_len=0, pool="first", groups=[10])[10]
+    assert set(r.C.tolist()) == set(torch.topk(I[r.t0, : r.t0 + 1], 12).indices.tolist())
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+@pytest.mark.parametrize("g,W", [(4, 4), (4, 2), (3, 5)])
+def test_prefill_window_covering_everything_is_the_dense_indexer(dtype, g, W):
+    """Prefill form of Appendix B: the proxy part ranks s <= t0 - W and fills c - (W + m - 1) slots,
+    the window union [t0 - W + 1, t0 + m - 1] takes the rest.  With the guardrail off and
+    c - (W + m - 1) >= t0 - W + 1 the two parts together hold every key up to t0 + m - 1, each
+    member masks the slots beyond its own position, and so every member must get the dense
+    indexer's top-k over [0, t] (torch restatement) -- including the keys of its own group, which
+    the plain method (W = 0) cannot reach."""
+    L, k, c = 61, 5, 80
+    x = tiny(L=L, H=4, d=8, dtype=dtype)
+    _, sets = _torch_dense(x, k)
+    res = po.pivot_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE, guard_len=0, W=W)
+    reached_own_group = 0
+    for r in res.values():
+        assert not r.guarded
+        m = len(r.members)
+        assert len(r.C) == min(c, r.t0 + m) and sorted(r.C.tolist()) == list(range(r.t0 + m))
+        for i, t in enumerate(r.members):
+            T = r.T[i]
+            assert set(T[T >= 0].tolist()) == sets[t], (r.t0, i)
+            assert (T[min(k, t + 1):] == -1).all()
+            reached_own_group += int(T.max() > r.t0)
+    assert reached_own_group > 0
+    plain = po.pivot_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE, guard_len=0, W=0)
+    assert all(r.T.max() <= r.t0 for r in plain.values())
+
+
+def test_prefill_window_slot_layout_with_a_short_candidate_budget():
+    """The same form when the proxy part does NOT cover its prefix: the last W + m - 1 slots are
+    the window positions in ascending order, the first c - (W + m - 1) are the top of the proxy
+    scores over s <= t0 - W (recomputed here from build_proxy + torch), and no slot repeats."""
+    L, g, c, k, W = 96, 4, 24, 8, 4
+    x = tiny(L=L, H=4, d=8)
+    kk = torch.from_numpy(x["k"].view(np.int16)).view(torch.bfloat16).double()
+    res = po.pivot_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE, W=W)
+    checked = 0
+    for r in res.values():
+        if r.guarded:
+            continue
+        m, t0 = len(r.members), r.t0
+        w_g = W + m - 1
+        assert r.C[c - w_g:].tolist() == list(range(t0 - W + 1, t0 + m))
+        pq, pw = po.build_proxy(x["q"][r.members], None, x["w"][r.members], "bf16")
+        pqt = torch.from_numpy(pq.view(np.int16)).view(torch.bfloat16).double()
+        n_scan = t0 - W + 1
+        s = (torch.relu(kk[:n_scan] @ pqt.T) * torch.from_numpy(pw).double()).sum(1)
+        want = set(torch.topk(s, c - w_g).indices.tolist())
+        assert set(r.C[: c - w_g].tolist()) == want
+        assert len(set(r.C.tolist())) == c
+        checked += 1
+    assert checked > 5
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+def test_rounded_proxy_stays_inside_the_score_band_of_the_exact_mean(dtype):
+    """Eq. 4 is real-valued; the oracle rounds the mean proxy back to the storage type (the rounding
+    points of a kernel that feeds a low-precision scan).  This bounds that reading from the oracle's
+    side: Eq. 5 scores of the rounded proxy against those of the unrounded fp64 mean of the
+    de-quantised members, at the real head count and width, stay inside the acceptance band."""
+    from oracle import acceptance as acc
+    L, g = 640, 4
+    x = inputs.make_prefill(L, dtype=dtype, seed=17, threads=1).codes()
+    kd = po.decode_operand(x["k"], dtype)
+    ks = x["kscale"]
+    worst = 0.0
+    for t0 in (128, 300, 636):
+        rows = np.arange(t0, t0 + g)
+        qs = None if x["qscale"] is None else x["qscale"][rows]
+        pq, pw = po.build_proxy(x["q"][rows], qs, x["w"][rows], dtype)
+        s_round = po.indexer_scores(po.decode_operand(pq, dtype), pw, kd[: t0 + 1], None if ks is None else ks[: t0 + 1])
+        qd = po.decode_operand(x["q"][rows], dtype)
+        if dtype == "fp8":
+            qd = qd * qs.astype(np.float64)[..., None]
+        qbar = qd.mean(axis=0)                                    # exact Eq. 4, fp64
+        wbar = x["w"][rows].astype(np.float64).mean(axis=0)
+        s_exact = np.maximum(kd[: t0 + 1] @ qbar.T, 0.0) @ wbar
+        if ks is not None:
+            s_exact = s_exact * ks[: t0 + 1].astype(np.float64)
+        err = np.abs(s_round - s_exact) / (acc.ATOL + acc.RTOL[dtype] * np.abs(s_exact))
+        worst = max(worst, float(err.max()))
+    assert worst <= 1.0, worst
