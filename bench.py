@@ -44,10 +44,12 @@ WORKLOADS = {
 DEFAULT_WORKLOAD = "prefill_128k_fp8_refine_g4"
 H, D = 64, 128
 FLOP_PER_SCORE = 2 * H * D
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
-# profiles/ (same workloads as the ones timed here)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch: STORED figures from the ncu captures
+# summarised under profiles/ (same workloads as the ones timed here); not re-measured by this run,
+# and labelled so in the line ("traffic_source").
 TRAFFIC_BYTES = {"prefill_128k_fp8_refine_g4": 2780454144 + 4301106432,
                  "decode_scan_kernel": 403583488 + 12487936}
+TRAFFIC_SOURCE = "stored ncu capture (profiles/), not re-measured in this run"
 
 
 def peaks():
@@ -267,22 +269,46 @@ def decode_bench(pv, dev, steps, warmup, pk):
     torch.cuda.synchronize()
     window_times = timed(step_window, steps)
     assert pv.pivot_device_status() == 0
+    # the dense control of the same step (Eq. 1 + TopK for each of the g queries; the queries of a
+    # sequence share one pass over its keys), same inputs, same GPU
+    dout = torch.empty_like(out)
+    pv.ensure_workspace(B * g, B, k, k, dev, need=pv.pivot_decode_workspace_bytes(B, Lmax, g, max(c, k), k))
+
+    def step_dense():
+        pv.dense_index_decode(q, w, kc, p0, B, Lmax, H, D, g, k, dout, stream, q_scale=qs, k_scale=ks)
+
+    for _ in range(warmup):
+        step_dense()
+    torch.cuda.synchronize()
+    dense_times = timed(step_dense, steps)
+    assert pv.pivot_device_status() == 0
     us = float(np.median(times))
     scan = float(np.mean(scan_us))
     n0 = (x.pos0.numpy().astype(np.int64) + 1)
     key_bytes = int(n0.sum()) * (D + 4)                      # e4m3 key + fp32 scale, read once per step
+    # whole step: every visible key once, the c gathered candidates of each sequence once more, and
+    # the step's own operands and result (queries, gates, scales, positions, index rows)
+    step_bytes = key_bytes + B * c * (D + 4) + B * g * (H * D + 2 * H * 4 + k * 4) + B * 4
+    dense_us = float(np.median(dense_times))
     return {"metric": "us per MTP decode step", "value": us, "unit": "us", "min_us": float(min(times)),
             "steps": steps, "higher_is_better": False, "gpu_launches_per_step": launches / max(steps, 1),
             "graph_replay_us": graph_us, "graph_note": graph_note,
             "paged": {"value": float(np.median(paged_times)), "unit": "us", "scan_kernel_us": float(np.mean(paged_scan)),
                       "page_keys": 128, "pool_pages": B * mp, "same_positions_as_contiguous": same},
             "local_window": {"W": 4, "value": float(np.median(window_times)), "unit": "us"},
+            "dense_control": {"entry": "dense_index_decode", "value": dense_us, "unit": "us",
+                              "pivot_speedup_over_dense": dense_us / us,
+                              "paper_h20_speedup_context": "PIVOT-Refine decode 1.40x at 16K .. 3.42x at 256K (H20, FP8, MTP g = 4)"},
+            "roofline_step": {"bound": "hbm", "achieved": step_bytes / (us * 1e-6) / 1e9, "peak": pk["hbm"], "unit": "GB/s",
+                              "frac": step_bytes / (us * 1e-6) / 1e9 / pk["hbm"], "algorithmic_bytes_per_step": step_bytes,
+                              "frac_of_nominal_8TBs": step_bytes / (us * 1e-6) / 8e12,
+                              "peak_source": pk["source"] + " STREAM copy"},
             "config": {"workload": "decode_mtp_b32_64k-128k_fp8_g2_refine", "B": B, "g": g, "c": c, "k": k,
                        "visible_keys": int(n0.sum()), "l2": "256 MB flush between steps"},
             # dominant kernel: the key-streaming scan; algorithmic bytes = visible keys x 132 B
             "roofline": {"kernel": "decode_scan_kernel", "bound": "hbm", "achieved": key_bytes / (scan * 1e-6) / 1e9,
                          "peak": pk["hbm"], "unit": "GB/s", "frac": key_bytes / (scan * 1e-6) / 1e9 / pk["hbm"],
-                         "traffic": TRAFFIC_BYTES["decode_scan_kernel"], "kernel_us": scan,
+                         "traffic": TRAFFIC_BYTES["decode_scan_kernel"], "traffic_source": TRAFFIC_SOURCE, "kernel_us": scan,
                          "algorithmic_bytes_per_launch": key_bytes, "peak_source": pk["source"] + " STREAM copy",
                          "frac_of_nominal_8TBs": key_bytes / (scan * 1e-6) / 8e12}}
 
@@ -381,6 +407,54 @@ def sweep(pv, dev, L, dtype, steps):
                           "recall_of_dense_topk": recall, "rows_sampled": int(len(rows))}))
 
 
+def spawn_ranks(n: int) -> int:
+    """Re-runs this command line as n ranks of one node under torch.distributed.run (one process per
+    GPU, rendezvous on 127.0.0.1); returns the launcher's exit code."""
+    have = torch.cuda.device_count()
+    if have < n:
+        print(json.dumps({"error": f"--gpus {n} asked for, {have} CUDA device(s) visible"}))
+        return 2
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def parity_probe(pv, dev, x, L, dtype, g, c, k, mode, result, n_groups=16, seed=11):
+    """Oracle check of a result the benchmark produced (index rows `result`, a CPU tensor [L, k]) on a
+    seeded sample of groups.  Refine's acceptance rule needs the candidate sets the kernels ranked:
+    one extra call with debug buffers on the same inputs supplies them (outside every timed region)."""
+    from oracle import acceptance as acc
+    nG = (L + g - 1) // g
+    first = (c - 1 + g - 1) // g
+    rng = np.random.default_rng(seed)
+    picks = sorted({0, min(first, nG - 1), nG - 1} | set(rng.integers(0, nG, max(n_groups - 3, 1)).tolist()))
+    dq, dw, dk = x.q.to(dev), x.w.to(dev), x.k.to(dev)
+    dqs = None if x.qscale is None else x.qscale.to(dev)
+    dks = None if x.kscale is None else x.kscale.to(dev)
+    pv.ensure_workspace(L, nG, c, k, dev)
+    tmp = torch.empty((L, k), dtype=torch.int32, device=dev)
+    cand = torch.full((nG, c), -7, dtype=torch.int32, device=dev) if mode == 1 else None
+    cs = torch.zeros((nG, c), dtype=torch.float32, device=dev) if mode == 1 else None
+    pv.pivot_index_prefill(dq, dw, dk, L, H, D, g, c, k, mode, tmp, q_scale=dqs, k_scale=dks, dbg_cand=cand,
+                           dbg_cand_scores=cs)
+    torch.cuda.synchronize()
+    f = lambda t: None if t is None else t[torch.tensor(picks, device=dev)].cpu().numpy()
+    cand_np = None
+    cs_np = None
+    if cand is not None:                       # only the sampled groups' rows travel
+        cand_np = np.full((nG, c), -7, np.int32)
+        cs_np = np.zeros((nG, c), np.float32)
+        cand_np[picks], cs_np[picks] = f(cand), f(cs)
+    t = acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=None, out_idx=result.numpy(),
+                          cand=cand_np, cand_scores=cs_np, groups=picks)
+    return {"groups": len(picks), "rows": t.rows, "exact": t.exact_rows, "band_swaps": t.band_swaps,
+            "max_score_err_x_tol": t.max_score_err, "checked": "e2e result" , "passed": True}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -393,10 +467,14 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-indexer control")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-parity-probe", action="store_true")
     ap.add_argument("--shard-request", action="store_true",
                     help="N > 1: all ranks share ONE request (row blocks dealt in snake order, one all-gather of the "
                          "index sets per step) instead of one request per rank; reported as strong scaling")
     ap.add_argument("--decode-only", action="store_true", help="only the MTP decode step (prints its object)")
+    ap.add_argument("--mma-model", action="store_true",
+                    help="one-SM timing probe behind the per-tile model of the scan (tensor pipe, tensor-memory port, "
+                         "hand-overs): prints one JSON object of clocks per tile")
     ap.add_argument("--sweep", action="store_true",
                     help="g / c / pooling / window sweep with recall of the dense top-k (one JSON line per case)")
     args = ap.parse_args()
@@ -404,6 +482,9 @@ def main():
     if args.impl == "reference":
         return run_reference(args, wl)
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain `python bench.py --gpus N`: become N ranks, one per GPU
+        sys.exit(spawn_ranks(args.gpus))
     L, dtype, g, c, k, mode = WORKLOADS[wl]
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -416,6 +497,9 @@ def main():
 
     from paper_2607_24593_b200 import binding as pv
 
+    if args.mma_model:
+        print(json.dumps({"mma_model": pv.pivot_debug_mma_model()}, indent=1))
+        return
     if args.sweep:
         sweep(pv, torch.device(f"cuda:{local}"), L, dtype, max(1, min(args.steps, 3)))
         return
@@ -507,6 +591,7 @@ def main():
 
     # ---- end to end through the host-buffer entry point (H2D + compute + D2H every step)
     e2e = None
+    probe_result, probe_what = (out.cpu() if rank == 0 and not shard else None), "device-timed result"
     if not args.no_e2e:
         hq, hw, hk = x.q.pin_memory(), x.w.pin_memory(), x.k.pin_memory()
         hqs = None if x.qscale is None else x.qscale.pin_memory()
@@ -536,6 +621,8 @@ def main():
         e_ms = max_over_ranks(e_ms, dist, dev)
         e2e = {"value": job_throughput(world, L, e_ms), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": e_ms, "steps": n_e2e}
+        if rank == 0:
+            probe_result, probe_what = hout.clone(), "e2e result"
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -551,8 +638,10 @@ def main():
     roofline = {
         "kernel": "scan_select_tc_kernel", "bound": "tensor", "achieved": achieved_tf, "peak": peak_tf,
         "unit": "TFLOP/s", "frac": achieved_tf / peak_tf, "traffic": TRAFFIC_BYTES.get(wl),
+        "traffic_source": TRAFFIC_SOURCE if wl in TRAFFIC_BYTES else None,
         "peak_source": f"{pk['source']} bf16 sustained {pk['bf16_sustained']} TFLOP/s x {ratio:g} (nominal {dtype}:bf16)",
         "frac_of_nominal": achieved_tf / (4500.0 if dtype == "fp8" else 2250.0),
+        "frac_of_measured_burst": achieved_tf / (pk["bf16"] * ratio),
         "algorithmic_flops_per_launch": scan_flops, "kernel_ms": scan_ms,
     }
     line = {
@@ -579,7 +668,13 @@ def main():
         torch.cuda.empty_cache()
         line["decode"] = decode_bench(pv, dev, steps=max(args.steps, 5), warmup=max(args.warmup, 3), pk=pk)
 
-    # ---- parity probe on the e2e result (a few groups) and the CPU baseline
+    # ---- parity probe: the oracle's acceptance rule on sampled groups of what the benchmark computed
+    if not args.no_parity_probe and probe_result is not None:
+        torch.cuda.empty_cache()
+        pp = parity_probe(pv, dev, x, L, dtype, g, c, k, mode, probe_result)
+        pp["checked"] = probe_what
+        line["parity_probe"] = pp
+    # ---- the CPU baseline
     if not args.no_cpu_baseline:
         est, dt, n, threads = oracle_sample_time(x, L, g, c, k, mode, n_groups=512 if L > 40000 else 768, seed=7)
         line["cpu_baseline"] = {"value": L / est, "unit": "tokens/s", "cores": threads, "kind": "oracle",

@@ -51,6 +51,14 @@ enum {
   PIVOT_ERR_CUDA = 4,        /* a CUDA runtime call failed; see pivot_last_cuda_error */
   PIVOT_ERR_DEVICE = 5       /* device status word non-zero (pivot_device_status) */
 };
+/* Values of the device status word (pivot_device_status); the first condition of a call wins. */
+enum {
+  PIVOT_DEV_OK = 0,
+  PIVOT_DEV_WAIT_EXPIRED = 1,  /* a bounded wait inside a kernel ran out; the kernel ended early, results invalid */
+  PIVOT_DEV_CAND_OVERFLOW = 2, /* a candidate buffer would have overflowed (internal error; the entry was dropped) */
+  PIVOT_DEV_BAD_POS = 3,       /* decode: some pos0[b] outside [0, Lmax - g]; that sequence's rows are all -1 */
+  PIVOT_DEV_BOUNDS = 4         /* checked builds (-DPIVOT_DEBUG) only: an index failed a bounds check, access skipped */
+};
 
 /*
  * A quantised operand.
@@ -171,7 +179,10 @@ int pivot_index_prefill_varlen(const pivot_tensor* q, const float* w, const pivo
  * the g queries of one MTP step at positions pos0[b] .. pos0[b]+g-1.
  *   q       [B, g, H_I, d]; w [B, g, H_I]; kcache [B, Lmax, d] (+ scale [B, Lmax]); sequence b's
  *           cache must hold keys 0 .. pos0[b]+g-1.
- *   pos0    [B] int32, device.  The proxy scan is cut at pos0[b] (inclusive).
+ *   pos0    [B] int32, device.  The proxy scan is cut at pos0[b] (inclusive).  Must lie in
+ *           [0, Lmax - g]; a sequence whose pos0 does not is not indexed: its g output rows are
+ *           filled with -1 and the status word reads PIVOT_DEV_BAD_POS (nothing is read out of
+ *           range, nothing traps).
  *   Lmax    rows per sequence in kcache; with FP8 it must be a multiple of 4 (each sequence's
  *           scale row then starts on a 16-byte boundary).
  *   out_idx [B, g, k] int32.
@@ -215,6 +226,21 @@ int dense_index_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kc
                    const pivot_opts* opts);
 
 /*
+ * Dense control, decode form: Eq. 1 + TopK for each of the g queries of one MTP step (the grouping
+ * of Eq. 3) of B sequences -- what a DSA decode step costs without PIVOT.  Arguments as in
+ * pivot_index_decode (contiguous cache); the query at position pos0[b] + i ranks keys
+ * 0 .. pos0[b] + i of sequence b.  The queries of one sequence share one pass over its keys
+ * (rows are packed four to a scan block per sequence).  out_idx [B, g, k] int32.  Workspace:
+ * pivot_decode_workspace_bytes(B, Lmax, g, k, k).  opts: dbg_scores, workspace, impl (0 / 2).
+ */
+int dense_index_decode(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                       const int32_t* pos0, int B, int Lmax, int H_I, int d, int g, int k,
+                       int32_t* out_idx, pivot_stream_t stream);
+int dense_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
+                          const int32_t* pos0, int B, int Lmax, int H_I, int d, int g, int k,
+                          int32_t* out_idx, pivot_stream_t stream, const pivot_opts* opts);
+
+/*
  * dense_index without any caller-provided scratch (no counterpart in the paper: this is a
  * deployment convenience, not part of the method).  For hosts that may not allocate device
  * memory -- a plugin inside a server that owns the device heap, code bound to a framework's
@@ -251,8 +277,30 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
                              pivot_stream_t stream);
 
 /* Reads (and clears) the device status word of the workspace last used on this device after
- * synchronising `stream`.  0 = no device-side condition. */
+ * synchronising `stream`.  0 = no device-side condition, else a PIVOT_DEV_* value. */
 int pivot_device_status(pivot_stream_t stream, int* status);
+
+/*
+ * Diagnostic (no counterpart in the paper): runs a one-block kernel whose threads wait, through the
+ * library's own bounded-wait routines, for a barrier that nothing completes, with a limit of
+ * limit_ns nanoseconds (1 us .. 1 s) instead of the library's 4 s.  The waits run out, the kernel
+ * returns normally and pivot_device_status then reads PIVOT_DEV_WAIT_EXPIRED -- the path every
+ * tensor-core kernel here takes instead of hanging should one of its hand-shakes ever break.
+ * Uses the status word of the registered workspace (pivot_set_workspace; PIVOT_ERR_WORKSPACE if
+ * there is none).  The GPU context stays usable; later calls are unaffected.
+ */
+int pivot_debug_wait_expiry(unsigned long long limit_ns, pivot_stream_t stream);
+
+/*
+ * Diagnostic (no counterpart in the paper): times, on one SM, the tensor-core instruction streams
+ * the shared scan (Eq. 5) and the re-score (Eq. 8) are built from -- the 128 x 256 x 128 FP8
+ * product, the head-sum product with its A operand in tensor memory in several operand widths,
+ * both interleaved -- alone and while other warps keep the tensor-memory port busy, plus the
+ * latency of a warp-to-warp mbarrier hand-over.  out_device: 256 int64 slots in device memory,
+ * clocks per tile; `bench.py --mma-model` prints them with their labels.  Operands are zeros: this
+ * measures time only.
+ */
+int pivot_debug_mma_model(long long* out_device, pivot_stream_t stream);
 
 /*
  * Per-stage timing, off by default.  While enabled, every call records CUDA events on its own

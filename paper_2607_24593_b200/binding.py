@@ -26,7 +26,9 @@ SYMBOLS = [
     "pivot_index_decode", "pivot_index_decode_ex", "pivot_index_decode_paged", "dense_index", "dense_index_ex", "dense_index_static",
     "pivot_prefill_host_arena_bytes", "pivot_index_prefill_host", "pivot_device_status",
     "pivot_stage_timing", "pivot_stage_times", "pivot_launch_count_reset", "pivot_status_str", "pivot_last_cuda_error",
+    "dense_index_decode", "dense_index_decode_ex", "pivot_debug_wait_expiry", "pivot_debug_mma_model",
 ]
+DEV_OK, DEV_WAIT_EXPIRED, DEV_CAND_OVERFLOW, DEV_BAD_POS, DEV_BOUNDS = 0, 1, 2, 3, 4
 
 
 class pivot_tensor(C.Structure):
@@ -65,6 +67,10 @@ def _load():
     lib.dense_index.argtypes = [T, P, T, I, I, I, I, P, P]
     lib.dense_index_ex.argtypes = [T, P, T, I, I, I, I, P, P, O]
     lib.dense_index_static.argtypes = [T, P, T, I, I, I, I, P, P]
+    lib.dense_index_decode.argtypes = [T, P, T, P, I, I, I, I, I, I, P, P]
+    lib.dense_index_decode_ex.argtypes = [T, P, T, P, I, I, I, I, I, I, P, P, O]
+    lib.pivot_debug_wait_expiry.argtypes = [C.c_ulonglong, P]
+    lib.pivot_debug_mma_model.argtypes = [P, P]
     lib.pivot_prefill_host_arena_bytes.restype = S
     lib.pivot_prefill_host_arena_bytes.argtypes = [I, I, I, I, I, I, I]
     lib.pivot_index_prefill_host.argtypes = [T, P, T, I, I, I, I, I, I, I, P, P, S, P]
@@ -233,6 +239,49 @@ def pivot_index_decode_paged(q, w, kpages, block_table, pos0, B, max_pages, n_pa
                                         pos0.data_ptr(), B, max_pages, n_pages, H_I, d, g, c, k, mode,
                                         out_idx.data_ptr(), _stream(stream), C.byref(o)))
     return out_idx
+
+
+def dense_index_decode(q, w, kcache, pos0, B, Lmax, H_I, d, g, k, out_idx, stream=None, *, q_scale=None, k_scale=None,
+                       dbg_scores=None, workspace=None, impl=0):
+    """Dense control of a decode step: Eq. 1 + TopK for each of the g queries of every sequence."""
+    tq, tk = _tensor(q, q_scale), _tensor(kcache, k_scale)
+    assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and pos0.dtype == torch.int32
+    assert out_idx.numel() >= B * g * k
+    if workspace is None:
+        ensure_workspace(B * g, B, k, k, q.device, need=pivot_decode_workspace_bytes(B, Lmax, g, k, k))
+    o = _opts(None, POOL_MEAN, None, dbg_scores, None, workspace, impl)
+    _check(lib.dense_index_decode_ex(C.byref(tq), w.data_ptr(), C.byref(tk), pos0.data_ptr(), B, Lmax, H_I, d, g, k,
+                                     out_idx.data_ptr(), _stream(stream), C.byref(o)))
+    return out_idx
+
+
+def pivot_debug_wait_expiry(limit_ns: int, stream=None):
+    """Diagnostic: lets the library's bounded device waits run out after limit_ns (see pivot.h)."""
+    _check(lib.pivot_debug_wait_expiry(int(limit_ns), _stream(stream)))
+
+
+MMA_MODEL_VARIANTS = ["M1 fp8 N=256 (4 K-steps)", "M1 fp8 N=192", "M1 fp8 2 x N=128", "M2 bf16 A in TMEM, 16 K-steps",
+                      "M2 bf16 A in TMEM, 8 K-steps", "M2 fp8 A in TMEM, 8 K-steps", "M2 int8 A in TMEM, 8 K-steps",
+                      "M1 + M2 bf16 x16", "M1 + M2 bf16 x8", "M1 + M2 int8 x8", "M1 N=192 + M2 int8 x6",
+                      "linear block fp8 N=16 (4 K-steps)", "M1 + linear block"]
+MMA_MODEL_PHASES = ["alone", "with ReLU-pass traffic (4 warps: load 32 cols, pack, store 16)",
+                    "with load-only traffic (4 warps)", "with load-only traffic (8 warps)"]
+
+
+def pivot_debug_mma_model(stream=None) -> dict:
+    """Runs the one-SM timing probe (see pivot.h) and labels its numbers: clocks per tile."""
+    out = torch.zeros(256, dtype=torch.int64, device="cuda")
+    _check(lib.pivot_debug_mma_model(out.data_ptr(), _stream(stream)))
+    torch.cuda.synchronize()
+    v = out.cpu().tolist()
+    res = {"abort_flag": v[254], "handover_clk": {"mbarrier try_wait, one way": v[128], "mbarrier test_wait, one way": v[129],
+                                                  "tcgen05.commit -> waiter -> arrive -> issuer, round trip": v[130]}}
+    for ph, pname in enumerate(MMA_MODEL_PHASES):
+        d = {name: v[ph * 32 + i] for i, name in enumerate(MMA_MODEL_VARIANTS)}
+        if ph:
+            d["traffic warps: clk per 256-column pass"] = [x for x in v[ph * 32 + 16: ph * 32 + 24] if x]
+        res[pname] = d
+    return res
 
 
 def pivot_prefill_host_arena_bytes(L, H_I, d, g, c, k, dtype) -> int:

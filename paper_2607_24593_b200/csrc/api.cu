@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include "../../include/pivot.h"
+#include "api_internal.h"
 #include "kernels.h"
 
 using namespace pivot;
@@ -24,6 +25,9 @@ struct DeviceState {
   // host-buffer prefill: copy streams and events, created on first use
   cudaStream_t copy_in = nullptr, copy_out = nullptr;
   cudaEvent_t ev_entry = nullptr, ev_in[kHostChunks] = {}, ev_done[kHostChunks] = {};
+  // stage-timing events (created on this device on first use) and what the last call recorded
+  cudaEvent_t ev[8] = {};
+  bool ev_valid = false, ev_decode_scan = false;
 };
 DeviceState g_dev[kMaxDevices];
 int g_last_cuda = 0;
@@ -124,21 +128,40 @@ ScanScratch tc_scratch(const Workspace& ws) {
 }
 
 bool g_timing = false;
-cudaEvent_t g_ev[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
-bool g_ev_decode_scan = false;
-bool g_ev_valid = false;
+// Events belong to the device that was current when they were created: one set per device.
+cudaEvent_t* timing_events() {
+  DeviceState& ds = g_dev[cur_device()];
+  if (!ds.ev[0])
+    for (int i = 0; i < 8; ++i)
+      if (cudaEventCreate(&ds.ev[i]) != cudaSuccess) { ds.ev[0] = nullptr; return nullptr; }
+  return ds.ev;
+}
 inline void mark(int i, cudaStream_t st) {
-  if (g_timing) { cudaEventRecord(g_ev[i], st); if (i == 4) g_ev_valid = true; }
+  if (!g_timing) return;
+  cudaEvent_t* ev = timing_events();
+  if (!ev) return;
+  cudaEventRecord(ev[i], st);
+  if (i == 4) g_dev[cur_device()].ev_valid = true;
 }
 
-int check_cuda(cudaError_t e) {
+inline int check_cuda(cudaError_t e) { return pivot::record_cuda(e); }
+inline int check_common(const pivot_tensor* q, const float* w, const pivot_tensor* kc, int H, int d, int c,
+                        int k, int mode, const void* out) {
+  return pivot::check_operands(q, w, kc, H, d, c, k, mode, out);
+}
+
+}  // namespace
+
+namespace pivot {
+
+int record_cuda(cudaError_t e) {
   if (e == cudaSuccess) return PIVOT_OK;
   g_last_cuda = (int)e;
   return PIVOT_ERR_CUDA;
 }
 
-int check_common(const pivot_tensor* q, const float* w, const pivot_tensor* kc, int H, int d, int c,
-                 int k, int mode, const void* out) {
+int check_operands(const pivot_tensor* q, const float* w, const pivot_tensor* kc, int H, int d, int c,
+                   int k, int mode, const void* out) {
   if (!q || !w || !kc || !out || !q->data || !kc->data) return PIVOT_ERR_INVALID_ARG;
   if (q->dtype != kc->dtype) return PIVOT_ERR_INVALID_ARG;
   if (q->dtype != PIVOT_BF16 && q->dtype != PIVOT_FP8_E4M3) return PIVOT_ERR_INVALID_ARG;
@@ -153,6 +176,10 @@ int check_common(const pivot_tensor* q, const float* w, const pivot_tensor* kc, 
   if (k > kMaxSel || c > kMaxSel) return PIVOT_ERR_UNSUPPORTED;
   return PIVOT_OK;
 }
+
+}  // namespace pivot
+
+namespace {
 
 int resolve_ws(const pivot_opts* o, size_t need, void** ws) {
   void* p = o && o->workspace ? o->workspace : g_dev[cur_device()].ws;
@@ -243,9 +270,13 @@ size_t pivot_workspace_bytes(int rows, int n_groups, int c, int k) {
   return carve_workspace(nullptr, rows, n_groups, c, k).bytes;
 }
 
+// Row slots of a decode call: the step's B * g queries, padded per sequence to a multiple of four
+// (the dense control packs a sequence's rows into four-row blocks).
+static int decode_row_slots(int B, int g) { return B * ((g + 3) / 4 * 4); }
+
 size_t pivot_decode_workspace_bytes(int B, int Lmax, int g, int c, int k) {
   if (B < 1 || Lmax < 1 || g < 1 || c < 1 || k < 1) return 0;
-  return pivot_workspace_bytes(B * g, B, c, k) + decode_fast_bytes(B, Lmax, g, c);
+  return pivot_workspace_bytes(decode_row_slots(B, g), B, c, k) + decode_fast_bytes(B, Lmax, g, c);
 }
 
 int pivot_set_workspace(void* workspace, size_t bytes) {
@@ -331,11 +362,11 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
   const bool paged = block_table != nullptr;
   if (paged && (n_pages < 1 || (Lmax & 127) || (o && o->impl == 1))) return PIVOT_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
-  const size_t base_bytes = pivot_workspace_bytes(B * g, B, c, k);
+  const size_t base_bytes = pivot_workspace_bytes(decode_row_slots(B, g), B, c, k);
   const size_t need = base_bytes + decode_fast_bytes(B, Lmax, g, c);
   void* wsp = nullptr;
   if ((rc = resolve_ws(o, need, &wsp))) return rc;
-  Workspace ws = carve_workspace(wsp, B * g, B, c, k);
+  Workspace ws = carve_workspace(wsp, decode_row_slots(B, g), B, c, k);
   g_dev[cur_device()].last_status = ws.status;
   DecodePlan p;
   p.q = q->data; p.w = w; p.qscale = q->scale;
@@ -352,6 +383,8 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
   if (paged) p.guard_len = 0;
   p.block_table = block_table;
   p.n_pages = n_pages;
+  p.status = ws.status;
+  p.W = W;
   const long long k_rows = paged ? (long long)n_pages * 128 : (long long)B * Lmax;
   if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 3 * sizeof(int), st)))) return rc;   // status, row counter, prepare ticket
   mark(0, st);
@@ -375,9 +408,10 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
     df.scratch = (char*)wsp + base_bytes;
     df.scratch_tc = tc_scratch(ws);
     df.status = ws.status;
-    df.ev_scan_begin = g_timing ? g_ev[6] : nullptr;
-    df.ev_scan_end = g_timing ? g_ev[7] : nullptr;
-    g_ev_decode_scan = g_timing;
+    cudaEvent_t* tev = g_timing ? timing_events() : nullptr;
+    df.ev_scan_begin = tev ? tev[6] : nullptr;
+    df.ev_scan_end = tev ? tev[7] : nullptr;
+    g_dev[cur_device()].ev_decode_scan = tev != nullptr;
     if ((rc = check_cuda(launch_decode_fast(df, st)))) return rc;
     // dense rows of guarded (short) sequences, if any: the generic scan, one row per block
     if (!paged) {
@@ -415,6 +449,65 @@ int pivot_index_decode(const pivot_tensor* q, const float* w, const pivot_tensor
                                nullptr);
 }
 
+int dense_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kcache, const int32_t* pos0,
+                          int B, int Lmax, int H_I, int d, int g, int k, int32_t* out_idx, pivot_stream_t stream,
+                          const pivot_opts* o) {
+  int rc = check_common(q, w, kcache, H_I, d, k, k, PIVOT_REUSE, out_idx);
+  if (rc) return rc;
+  if (!pos0 || B < 1 || g < 1 || Lmax < g) return PIVOT_ERR_INVALID_ARG;
+  if (q->dtype == PIVOT_FP8_E4M3 && (Lmax & 3)) return PIVOT_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int gp = (g + 3) / 4 * 4;
+  const size_t need = pivot_decode_workspace_bytes(B, Lmax, g, k, k);
+  void* wsp = nullptr;
+  if ((rc = resolve_ws(o, need, &wsp))) return rc;
+  Workspace ws = carve_workspace(wsp, decode_row_slots(B, g), B, k, k);
+  g_dev[cur_device()].last_status = ws.status;
+  DecodePlan p;
+  p.q = q->data; p.w = w; p.qscale = q->scale;
+  p.kc = kcache->data; p.kscale = kcache->scale;
+  p.pos0 = pos0;
+  p.proxy_q = nullptr; p.proxy_w = nullptr; p.cand = nullptr; p.cand_score = nullptr;
+  p.out = out_idx; p.out_score = o ? o->dbg_scores : nullptr;
+  p.B = B; p.Lmax = Lmax; p.g = g; p.c = k; p.k = k; p.mode = PIVOT_REUSE; p.dtype = q->dtype;
+  p.guard_len = 0;
+  p.status = ws.status;
+  if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 3 * sizeof(int), st)))) return rc;
+  mark(0, st);
+  mark(1, st);
+  launch_plan_dense_decode(p, ws.rows, gp, st);
+  mark(2, st);
+  // the proxy tensor map needs some valid address; no row refers to it
+  ScanOperands op{kcache->data, (long long)B * Lmax, kcache->scale, q->data, B * g, q->data, 1, q->dtype};
+  if ((rc = check_cuda(launch_scan_tc(op, ws.rows, B * gp, 4, tc_scratch(ws), sm_count(), st, o && o->impl == 2))))
+    return rc;
+  mark(3, st);
+  mark(4, st);
+  return check_cuda(cudaGetLastError());
+}
+
+int dense_index_decode(const pivot_tensor* q, const float* w, const pivot_tensor* kcache, const int32_t* pos0,
+                       int B, int Lmax, int H_I, int d, int g, int k, int32_t* out_idx, pivot_stream_t stream) {
+  return dense_index_decode_ex(q, w, kcache, pos0, B, Lmax, H_I, d, g, k, out_idx, stream, nullptr);
+}
+
+int pivot_debug_wait_expiry(unsigned long long limit_ns, pivot_stream_t stream) {
+  if (limit_ns < 1000ull || limit_ns > 1000000000ull) return PIVOT_ERR_INVALID_ARG;      // 1 us .. 1 s
+  DeviceState& ds = g_dev[cur_device()];
+  if (!ds.ws || ds.ws_bytes < 256) return PIVOT_ERR_WORKSPACE;
+  int* status = (int*)ds.ws;                     // the status word is the first word of every workspace
+  ds.last_status = status;
+  cudaStream_t st = (cudaStream_t)stream;
+  int rc = check_cuda(cudaMemsetAsync(status, 0, sizeof(int), st));
+  if (rc) return rc;
+  return check_cuda(launch_wait_expiry_probe(status, limit_ns, st));
+}
+
+int pivot_debug_mma_model(long long* out_device, pivot_stream_t stream) {
+  if (!out_device || ((uintptr_t)out_device & 7)) return PIVOT_ERR_INVALID_ARG;
+  return check_cuda(launch_mma_model_probe(out_device, (cudaStream_t)stream));
+}
+
 size_t pivot_prefill_host_arena_bytes(int L, int H_I, int d, int g, int c, int k, int dtype) {
   if (L < 1 || g < 1 || H_I < 1 || d < 1) return 0;
   const size_t esz = dtype == PIVOT_FP8_E4M3 ? 1 : 2;
@@ -433,13 +526,14 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
                              int H_I, int d, int g, int c, int k, int mode, int32_t* out_idx,
                              void* arena, size_t arena_bytes, pivot_stream_t stream) {
   if (!q || !w || !kcache || !out_idx || !arena || L < 1 || g < 1) return PIVOT_ERR_INVALID_ARG;
+  // every argument check of the device entry point runs here, before the first copy is enqueued
+  int rc = check_common(q, w, kcache, H_I, d, c, k, mode, out_idx);
+  if (rc) return rc;
   if (((uintptr_t)arena & 255) || arena_bytes < pivot_prefill_host_arena_bytes(L, H_I, d, g, c, k, q->dtype))
     return PIVOT_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   const bool fp8 = q->dtype == PIVOT_FP8_E4M3;
-  if (fp8 && (!q->scale || !kcache->scale)) return PIVOT_ERR_INVALID_ARG;
   const size_t esz = fp8 ? 1 : 2;
-  int rc;
   DeviceState& ds = g_dev[cur_device()];
   if (!ds.copy_in) {
     if ((rc = check_cuda(cudaStreamCreateWithFlags(&ds.copy_in, cudaStreamNonBlocking)))) return rc;
@@ -450,6 +544,9 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
       if ((rc = check_cuda(cudaEventCreateWithFlags(&ds.ev_done[i], cudaEventDisableTiming)))) return rc;
     }
   }
+  // From here on copies are in flight on three streams: an error return must not leave them
+  // running on the caller's pinned buffers and arena.
+  auto body = [&]() -> int {
   Carve cv(arena);
   char* dq = cv.take<char>((size_t)L * H_I * d * esz);
   float* dqs = cv.take<float>((size_t)L * H_I);
@@ -519,6 +616,14 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
   }
   if ((rc = check_cuda(cudaStreamSynchronize(st)))) return rc;
   return check_cuda(cudaStreamSynchronize(ds.copy_out));
+  };
+  rc = body();
+  if (rc) {
+    cudaStreamSynchronize(ds.copy_in);
+    cudaStreamSynchronize(st);
+    cudaStreamSynchronize(ds.copy_out);
+  }
+  return rc;
 }
 
 int pivot_device_status(pivot_stream_t stream, int* status) {
@@ -528,32 +633,30 @@ int pivot_device_status(pivot_stream_t stream, int* status) {
   if (!p) return PIVOT_OK;
   int rc = check_cuda(cudaStreamSynchronize((cudaStream_t)stream));
   if (rc) return rc;
-  return check_cuda(cudaMemcpy(status, p, sizeof(int), cudaMemcpyDeviceToHost));
+  if ((rc = check_cuda(cudaMemcpy(status, p, sizeof(int), cudaMemcpyDeviceToHost)))) return rc;
+  if (*status) rc = check_cuda(cudaMemset(p, 0, sizeof(int)));     // read and cleared
+  return rc;
 }
 
 int pivot_stage_timing(int enable) {
-  if (enable && !g_ev[0]) {
-    for (int i = 0; i < 8; ++i) {
-      int rc = check_cuda(cudaEventCreate(&g_ev[i]));
-      if (rc) return rc;
-    }
-  }
+  if (enable && !timing_events()) { (void)check_cuda(cudaGetLastError()); return PIVOT_ERR_CUDA; }
   g_timing = enable != 0;
-  g_ev_valid = false;
-  g_ev_decode_scan = false;
+  for (DeviceState& ds : g_dev) { ds.ev_valid = false; ds.ev_decode_scan = false; }
   return PIVOT_OK;
 }
 
 int pivot_stage_times(float* ms, int n) {
-  if (!ms || n < 5 || !g_ev_valid) return PIVOT_ERR_INVALID_ARG;
-  int rc = check_cuda(cudaEventSynchronize(g_ev[4]));
+  DeviceState& ds = g_dev[cur_device()];
+  if (!ms || n < 5 || !ds.ev_valid) return PIVOT_ERR_INVALID_ARG;
+  cudaEvent_t* ev = ds.ev;
+  int rc = check_cuda(cudaEventSynchronize(ev[4]));
   if (rc) return rc;
   for (int i = 0; i < 4; ++i)
-    if ((rc = check_cuda(cudaEventElapsedTime(&ms[i], g_ev[i], g_ev[i + 1])))) return rc;
-  if ((rc = check_cuda(cudaEventElapsedTime(&ms[4], g_ev[0], g_ev[4])))) return rc;
+    if ((rc = check_cuda(cudaEventElapsedTime(&ms[i], ev[i], ev[i + 1])))) return rc;
+  if ((rc = check_cuda(cudaEventElapsedTime(&ms[4], ev[0], ev[4])))) return rc;
   if (n >= 6) {
     ms[5] = 0.f;
-    if (g_ev_decode_scan && (rc = check_cuda(cudaEventElapsedTime(&ms[5], g_ev[6], g_ev[7])))) return rc;
+    if (ds.ev_decode_scan && (rc = check_cuda(cudaEventElapsedTime(&ms[5], ev[6], ev[7])))) return rc;
   }
   return PIVOT_OK;
 }

@@ -16,6 +16,8 @@ constexpr int DT_FP8 = 1;
 constexpr int DEV_OK = 0;
 constexpr int DEV_WAIT_EXPIRED = 1;   // a bounded barrier wait ran out
 constexpr int DEV_CAND_OVERFLOW = 2;  // a candidate buffer would have overflowed (logic error)
+constexpr int DEV_BAD_POS = 3;        // decode: a sequence's pos0 lies outside [0, Lmax - g]; its rows are all -1
+constexpr int DEV_BOUNDS = 4;         // PIVOT_DEBUG builds: an index, page or cursor failed its bounds check (access skipped)
 
 // fp32 score -> uint32 key whose unsigned order equals the float order (-inf lowest).
 __device__ __forceinline__ uint32_t score_to_key(float s) {

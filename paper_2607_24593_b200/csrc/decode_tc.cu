@@ -439,9 +439,11 @@ decode_prepare_kernel(DecodePlan p, RowDesc* rows, GroupDesc* plan_groups, uint3
     const int b = blockIdx.x;
     for (int i = threadIdx.x; i < DHIST; i += blockDim.x) ghist[(size_t)b * DHIST + i] = 0u;
     if (threadIdx.x < 2) ghist[(size_t)p.B * DHIST + 2 * b + threadIdx.x] = 0u;      // list length, delivered shares
-    if (threadIdx.x == 0) plan_decode_sequence(p, b, rows, plan_groups);
+    __shared__ int is_last, seq_ok;
+    if (threadIdx.x == 0) seq_ok = plan_decode_sequence(p, b, rows, plan_groups) ? 1 : 0;
+    __syncthreads();
+    if (!seq_ok) fill_decode_rows_empty(p, b, threadIdx.x, blockDim.x);     // pos0 outside the cache: rows of -1
     __threadfence();
-    __shared__ int is_last;
     __syncthreads();
     if (threadIdx.x == 0) is_last = atomicAdd(ticket, 1) == (int)gridDim.x - 1;
     __syncthreads();
@@ -553,13 +555,9 @@ cudaError_t launch_scan(const CUtensorMap& mk, const CUtensorMap& mq, const CUte
                         const int* tile_prefix, int B, int Lmax, float* scores, uint32_t* ghist, int* status,
                         int sms, cudaStream_t st) {
   auto kern = decode_scan_kernel<DT>;
-  static bool attr_set = false;
+  static bool attr_set[kMaxDevices] = {};
   const size_t smem = dsmem_bytes<DT>();
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  if (cudaError_t e = opt_in_dynamic_smem(kern, smem, attr_set); e != cudaSuccess) return e;
   kern<<<sms, D_THREADS, smem, st>>>(mk, mq, mks, prox, tile_prefix, B, Lmax, scores, ghist, status);
   ++launch_counter();
   return cudaGetLastError();
@@ -615,13 +613,9 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
           : launch_scan<DT_BF16>(mk, mq, mks, d.prox, tile_prefix, d.B, Ls, scores, ghist, d.status, d.sms, st);
   if (e != cudaSuccess) return e;
   if (d.ev_scan_end) cudaEventRecord(d.ev_scan_end, st);
-  static bool sel_attr = false;
+  static bool sel_attr[kMaxDevices] = {};
   const size_t sel_smem = sizeof(SelSmem) + 16;
-  if (!sel_attr) {
-    e = cudaFuncSetAttribute(decode_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sel_smem);
-    if (e != cudaSuccess) return e;
-    sel_attr = true;
-  }
+  if ((e = opt_in_dynamic_smem(decode_select_kernel, sel_smem, sel_attr)) != cudaSuccess) return e;
   decode_select_kernel<<<dim3(SEL_SPLIT, d.B), kBlk, sel_smem, st>>>(d.prox, Ls, scores, ghist, glist, sel_ctr);
   ++launch_counter();
   if (d.mode == 1) {

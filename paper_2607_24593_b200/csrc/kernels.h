@@ -79,6 +79,7 @@ struct DecodePlan {
   const int32_t* block_table = nullptr;                 // paged cache: [B, Lmax / 128] pool pages
   int n_pages = 0;
   int W = 0;                                            // per-query local window (Appendix B, decode form)
+  int* status = nullptr;                                // device status word (a bad pos0 is reported there)
 };
 
 struct ScanScratch {
@@ -138,5 +139,27 @@ size_t decode_fast_bytes(int B, int Lmax, int g, int c);
 cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st);
 
 long long& launch_counter();
+
+// Diagnostic: a kernel whose bounded waits run out after limit_ns (see debug_probe.cu).
+cudaError_t launch_wait_expiry_probe(int* status, unsigned long long limit_ns, cudaStream_t st);
+// Diagnostic: tensor-pipe / tensor-memory / hand-over timings of one SM (see debug_probe.cu); out = 256 slots.
+cudaError_t launch_mma_model_probe(long long* out, cudaStream_t st);
+// Dense control of a decode step: rows of a sequence padded to blocks of four that share a key stream.
+void launch_plan_dense_decode(const DecodePlan& p, RowDesc* rows, int gp, cudaStream_t st);
+
+// The opt-in to more than 48 KB of dynamic shared memory is an attribute of (function, device):
+// remembered per device, so that a process driving several GPUs sets it on each of them.
+constexpr int kMaxDevices = 64;
+template <typename Kern>
+inline cudaError_t opt_in_dynamic_smem(Kern kern, size_t bytes, bool (&done)[kMaxDevices]) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool tracked = dev >= 0 && dev < kMaxDevices;
+  if (tracked && done[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess && tracked) done[dev] = true;
+  return e;
+}
 
 }  // namespace pivot

@@ -30,10 +30,17 @@ __device__ __forceinline__ void put_group_chunks(GroupDesc* slots, const GroupDe
 // Decode, one sequence: scan-row slot b is sequence b's proxy row; slots B + b*g + i are its dense rows.
 // Exactly one of the two kinds is live per sequence (the guard test runs here because pos0
 // lives on the device); dead slots get K = 0 and are skipped by the kernels.
-__device__ __forceinline__ void plan_decode_sequence(const DecodePlan& p, int b, RowDesc* rows, GroupDesc* groups) {
+// The cache of a sequence holds Lmax rows and the step reads keys 0 .. pos0 + g - 1: a pos0 outside
+// [0, Lmax - g] would send the scan past the sequence's rows (into the next sequence, or past the
+// block table).  Such a sequence gets no live slot at all, the status word reports DEV_BAD_POS, and
+// the function returns false so that the caller fills the sequence's output rows with -1.
+__device__ __forceinline__ bool plan_decode_sequence(const DecodePlan& p, int b, RowDesc* rows, GroupDesc* groups) {
   const size_t esz = p.dtype == DT_FP8 ? 1 : 2;
   const size_t qrow = (size_t)kHeads * kDim * esz;
-  const int p0 = p.pos0[b];
+  const int p_in = p.pos0[b];
+  const bool bad = p_in < 0 || p_in > p.Lmax - p.g;
+  if (bad) set_status(p.status, DEV_BAD_POS);
+  const int p0 = bad ? 0 : p_in;
   const int n0 = p0 + 1;
   const bool guarded = n0 < p.guard_len;
   // Paged cache: descriptors point at the page pool and carry the sequence's block-table row.
@@ -70,7 +77,7 @@ __device__ __forceinline__ void plan_decode_sequence(const DecodePlan& p, int b,
   gd.out_score = outsb;
   gd.out_stride = p.k;
   gd.ent_out = nullptr; gd.ent_stride = 0; gd.slot0 = 0;
-  if (guarded) {
+  if (guarded || bad) {
     r.K = 0; r.out = nullptr; r.out_score = nullptr; r.out_rows = 0; r.out_stride = 0;
   } else if (p.mode == 0) {
     r.K = p.k; r.out = outb; r.out_score = outsb; r.out_rows = p.g; r.out_stride = p.k;
@@ -90,13 +97,22 @@ __device__ __forceinline__ void plan_decode_sequence(const DecodePlan& p, int b,
     dr.kbase = kb;
     dr.kscale = ksb;
     dr.n_vis = p0 + i + 1;
-    dr.K = guarded ? p.k : 0;
+    dr.K = (guarded && !bad) ? p.k : 0;
     dr.out = outb + (size_t)i * p.k;
     dr.out_score = outsb ? outsb + (size_t)i * p.k : nullptr;
     dr.out_rows = 1;
     dr.out_stride = p.k;
     dr.q_map = 0; dr.q_row = b * p.g + i; dr.k_row0 = b * p.Lmax;
     rows[p.B + b * p.g + i] = dr;
+  }
+  return !bad;
+}
+
+// Output rows of a sequence that was not indexed (bad pos0): every entry -1 (scores -inf).
+__device__ __forceinline__ void fill_decode_rows_empty(const DecodePlan& p, int b, int tid, int nthreads) {
+  for (int i = tid; i < p.g * p.k; i += nthreads) {
+    p.out[(size_t)b * p.g * p.k + i] = -1;
+    if (p.out_score) p.out_score[(size_t)b * p.g * p.k + i] = -INFINITY;
   }
 }
 

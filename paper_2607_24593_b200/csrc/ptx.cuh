@@ -74,10 +74,12 @@ constexpr uint64_t kWaitLimitNs = 4000000000ull;  // 4 s: far beyond any legitim
 
 // Waits for the phase with the given parity to complete.  Returns false if `*abort_flag`
 // became non-zero or the time limit ran out (the flag is then set for everybody else).
+// `limit_ns` is the library-wide limit everywhere except in the diagnostic kernel that exists
+// to let this very code path run out on purpose (debug_probe.cu).
 // `backoff_ns` > 0 puts the thread to sleep between polls: single-thread roles (TMA producer,
 // MMA issuer) share a scheduler with epilogue warps and must not eat their issue slots.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          unsigned backoff_ns = 0) {
+                                          unsigned backoff_ns = 0, uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   uint32_t spins = 0;
@@ -86,7 +88,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     if (backoff_ns) __nanosleep(backoff_ns);
     if (*abort_flag) return false;
     if ((++spins & 255u) == 0) {
-      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      if (globaltimer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         return false;
       }
@@ -96,7 +98,8 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 
 // The same bounded wait, polling with test_wait: for the one thread whose wake-up latency is on
 // a kernel's critical path (the MMA issuer).
-__device__ __forceinline__ bool mbar_wait_poll(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_poll(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                               uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_test_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   uint32_t spins = 0;
@@ -104,7 +107,7 @@ __device__ __forceinline__ bool mbar_wait_poll(uint64_t* bar, uint32_t parity, v
     if (mbar_test_wait(bar, parity)) return true;
     if ((++spins & 63u) == 0) {
       if (*abort_flag) return false;
-      if ((spins & 4095u) == 0 && globaltimer_ns() - t0 > kWaitLimitNs) {
+      if ((spins & 4095u) == 0 && globaltimer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         return false;
       }

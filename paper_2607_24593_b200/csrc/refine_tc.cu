@@ -550,13 +550,9 @@ template <int DT, int EPI = 1>
 cudaError_t launch_one(const CUtensorMap& mq, const GroupDesc* groups, int n_groups, int q_rows,
                        const ScanScratch& s, int sms, cudaStream_t st) {
   auto kern = refine_tc_kernel<DT, EPI>;
-  static bool attr_set = false;
+  static bool attr_set[kMaxDevices] = {};
   const size_t smem = rsmem_bytes<DT, EPI>();
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  if (cudaError_t e = opt_in_dynamic_smem(kern, smem, attr_set); e != cudaSuccess) return e;
   const int grid = n_groups < sms ? n_groups : sms;
   kern<<<grid, THREADS, smem, st>>>(mq, groups, n_groups, q_rows, s);
   ++launch_counter();

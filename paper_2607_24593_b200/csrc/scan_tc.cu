@@ -701,13 +701,9 @@ cudaError_t launch_one(const CUtensorMap& mk, const CUtensorMap& mq0, const CUte
                        const RowDesc* rows, int n_rows, const ScanScratch& s, int sms, cudaStream_t st) {
   using C = Cfg<DT, NROWS, EPI>;
   auto kern = scan_select_tc_kernel<DT, NROWS, EPI>;
-  static bool attr_set = false;
+  static bool attr_set[kMaxDevices] = {};
   const size_t smem = smem_bytes<DT, NROWS, EPI>();
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  if (cudaError_t e = opt_in_dynamic_smem(kern, smem, attr_set); e != cudaSuccess) return e;
   const int n_blocks = (n_rows + NROWS - 1) / NROWS;
   const int grid = n_blocks < sms ? n_blocks : sms;
   kern<<<grid, C::THREADS, smem, st>>>(mk, mq0, mq1, mks, rows, n_rows, s);

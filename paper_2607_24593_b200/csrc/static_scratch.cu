@@ -11,6 +11,7 @@
 // exits.  Its name is only a host-side handle: the device address is looked up once per device
 // with cudaGetSymbolAddress (first call on that device) and that address is what the kernels get.
 #include "../../include/pivot.h"
+#include "api_internal.h"
 #include "kernels.h"
 
 using namespace pivot;
@@ -35,20 +36,19 @@ inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
 extern "C" int dense_index_static(const pivot_tensor* q, const float* w, const pivot_tensor* kcache, int L,
                                   int H_I, int d, int k, int32_t* out_idx, pivot_stream_t stream) {
-  if (!q || !w || !kcache || !out_idx || !q->data || !kcache->data) return PIVOT_ERR_INVALID_ARG;
-  if (q->dtype != kcache->dtype || (q->dtype != PIVOT_BF16 && q->dtype != PIVOT_FP8_E4M3))
-    return PIVOT_ERR_INVALID_ARG;
-  if (q->dtype == PIVOT_FP8_E4M3 && (!q->scale || !kcache->scale)) return PIVOT_ERR_INVALID_ARG;
-  if (L < 1 || k < 1) return PIVOT_ERR_INVALID_ARG;
-  if (H_I != kHeads || d != kDim) return PIVOT_ERR_UNSUPPORTED;
+  // the same argument checks as dense_index (pointers, operand types, alignment, shapes)
+  if (int rc = check_operands(q, w, kcache, H_I, d, k, k, PIVOT_REUSE, out_idx)) return rc;
+  if (L < 1) return PIVOT_ERR_INVALID_ARG;
   if (L > kStaticMaxL || k > kStaticMaxK) return PIVOT_ERR_WORKSPACE;   // beyond the built-in scratch
   cudaStream_t st = (cudaStream_t)stream;
 
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return PIVOT_ERR_CUDA;
+  if (int rc = record_cuda(cudaGetDevice(&dev))) return rc;
+  if (dev < 0 || dev >= kMaxDev) return PIVOT_ERR_UNSUPPORTED;
   if (!g_scratch_ptr[dev]) {       // one-time set-up on this device (do it before any stream capture)
     void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return PIVOT_ERR_CUDA;
+    if (int rc = record_cuda(cudaGetSymbolAddress(&p, g_static_scratch))) return rc;
+    if (!p) return PIVOT_ERR_CUDA;
     g_scratch_ptr[dev] = p;
   }
   char* base = (char*)g_scratch_ptr[dev];
@@ -61,7 +61,7 @@ extern "C" int dense_index_static(const pivot_tensor* q, const float* w, const p
 
   // The array keeps whatever the previous call left: the status word must start at zero; row
   // descriptors are rewritten for rows 0..L-1 and candidate cursors start at zero in registers.
-  if (cudaMemsetAsync(status, 0, 2 * sizeof(int), st) != cudaSuccess) return PIVOT_ERR_CUDA;
+  if (int rc = record_cuda(cudaMemsetAsync(status, 0, 2 * sizeof(int), st))) return rc;
 
   PrefillPlan p;
   p.q = q->data; p.w = w; p.qscale = q->scale;
@@ -81,6 +81,6 @@ extern "C" int dense_index_static(const pivot_tensor* q, const float* w, const p
   sc.counter = status + 1;
   // the proxy tensor map needs some valid address; no row refers to it
   ScanOperands op{kcache->data, L, kcache->scale, q->data, L, q->data, 1, q->dtype};
-  if (launch_scan_tc(op, rows, L, 4, sc, kStaticCtas, st) != cudaSuccess) return PIVOT_ERR_CUDA;
-  return cudaGetLastError() == cudaSuccess ? PIVOT_OK : PIVOT_ERR_CUDA;
+  if (int rc = record_cuda(launch_scan_tc(op, rows, L, 4, sc, kStaticCtas, st))) return rc;
+  return record_cuda(cudaGetLastError());
 }

@@ -72,6 +72,51 @@ def test_config3_prefill_128k_fp8(g, mode):
     _run_and_check(131072, "fp8", g, 4096, 2048, mode, n_random=20)
 
 
+def _rows_equal_as_sets(a: torch.Tensor, b: torch.Tensor) -> bool:
+    return bool((torch.sort(a, dim=1).values == torch.sort(b, dim=1).values).all().item())
+
+
+def test_config3_plain_call_and_host_pipeline_at_full_size():
+    """The headline configuration exactly as bench.py times it: the call WITHOUT debug buffers
+    (other store paths in the kernels: staged 16-byte index rows, candidates in the workspace) and
+    the host-buffer pipeline in eight row chunks.  Both must return, row for row, the sets of the
+    call with debug buffers, and those are checked against the oracle on the sampled groups."""
+    import gpu_util
+    from paper_2607_24593_b200 import binding as pv
+    L, g, c, k, mode = 131072, 4, 4096, 2048, po.MODE_REFINE
+    x = _inputs(L, "fp8")
+    d = gpu_util.to_cuda(x)
+    nG = L // g
+    dbg = torch.full((L, k), -7, dtype=torch.int32, device="cuda")
+    cand = torch.full((nG, c), -7, dtype=torch.int32, device="cuda")
+    cs = torch.full((nG, c), float("nan"), dtype=torch.float32, device="cuda")
+    pv.pivot_index_prefill(d["q"], d["w"], d["k"], L, 64, 128, g, c, k, mode, dbg, q_scale=d["qscale"],
+                           k_scale=d["kscale"], dbg_cand=cand, dbg_cand_scores=cs)
+    plain = torch.full((L, k), -7, dtype=torch.int32, device="cuda")
+    pv.pivot_index_prefill(d["q"], d["w"], d["k"], L, 64, 128, g, c, k, mode, plain, q_scale=d["qscale"],
+                           k_scale=d["kscale"])
+    torch.cuda.synchronize()
+    assert pv.pivot_device_status() == 0
+    assert _rows_equal_as_sets(plain, dbg)
+    groups = _sample_groups(L, g, c, 12, seed=99)
+    t = acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=None, out_idx=plain.cpu().numpy(),
+                          cand=cand.cpu().numpy(), cand_scores=cs.cpu().numpy(), groups=groups)
+    print(f"\n[128K plain call] groups={len(groups)} rows={t.rows} exact={t.exact_rows} band_swaps={t.band_swaps}")
+    del cand, cs, dbg
+    # host pipeline (eight chunks at this size)
+    pv.pivot_set_workspace(None)
+    del d
+    torch.cuda.empty_cache()
+    pin = lambda t_: t_.contiguous().pin_memory()
+    hq, hw, hk, hqs, hks = pin(x.q), pin(x.w), pin(x.k), pin(x.qscale), pin(x.kscale)
+    hout = torch.full((L, k), -7, dtype=torch.int32).pin_memory()
+    arena = torch.empty(pv.pivot_prefill_host_arena_bytes(L, 64, 128, g, c, k, pv.FP8_E4M3), dtype=torch.uint8, device="cuda")
+    pv.pivot_index_prefill_host(hq, hw, hk, L, 64, 128, g, c, k, mode, hout, arena, q_scale=hqs, k_scale=hks)
+    assert _rows_equal_as_sets(hout.cuda(), plain)
+    del arena
+    torch.cuda.empty_cache()
+
+
 def test_config5_prefill_256k_fp8_refine():
     _run_and_check(262144, "fp8", 4, 4096, 2048, po.MODE_REFINE, n_random=12)
 

@@ -55,6 +55,28 @@ def test_prefill_small_full_parity(pv, gu, dtype, mode, seed):
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+@pytest.mark.parametrize("mode", [po.MODE_REUSE, po.MODE_REFINE])
+def test_cuda_core_cross_check_kernels_against_the_oracle(pv, gu, dtype, mode):
+    """impl = 1: the plain CUDA-core kernels (one key per thread, radix select) that the library
+    keeps as an on-device cross-check -- config 1, every group against the oracle."""
+    L, g, c, k = 2048, 4, 512, 256
+    x = inputs.make_prefill(L, dtype=dtype, seed=20260724)
+    out, sc, cand, cs = gu.run_prefill(x, g=g, c=c, k=k, mode=mode, impl=pv.IMPL_CUDA_CORE)
+    t = acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=None, out_idx=out,
+                          out_scores=sc, cand=cand, cand_scores=cs)
+    _report(f"CUDA-core kernels {dtype} mode={mode}", t)
+    assert t.exact_rows >= 0.95 * t.rows
+    # and the tensor-core path returns the same sets up to the band swaps both are allowed
+    ref, _, _, _ = gu.run_prefill(x, g=g, c=c, k=k, mode=mode, impl=pv.IMPL_TENSOR_CORE_FP32_HEAD_SUM)
+    same = (_sorted_rows_np(out) == _sorted_rows_np(ref)).all(axis=1).mean()
+    assert same >= 0.9
+
+
+def _sorted_rows_np(a):
+    return np.sort(a, axis=1)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
 def test_dense_small_full_parity(pv, gu, dtype):
     L, k = 1536, 256
     x = inputs.make_prefill(L, dtype=dtype, seed=5)
@@ -351,6 +373,105 @@ def test_decode_paged_argument_errors(pv):
                                     impl=pv.IMPL_CUDA_CORE)
 
 
+# ---------------------------------------------------------------- dense control of a decode step
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+@pytest.mark.parametrize("g", [1, 2, 4, 5])
+def test_dense_decode_control_against_the_oracle(pv, dtype, g):
+    """dense_index_decode: Eq. 1 + TopK for every query of an MTP step.  The query at pos0 + i of
+    sequence b is row pos0 + i of the dense indexer over that sequence's cache: compared with the
+    oracle's dense rows, scores included."""
+    B, k = 5, 96
+    x = inputs.make_decode(B, g, 40, 1500, dtype=dtype, seed=61)        # some sequences with fewer keys than k
+    d = {n: (None if getattr(x, n) is None else getattr(x, n).cuda()) for n in ("q", "qscale", "w", "k", "kscale", "pos0")}
+    Lmax = x.k.shape[1]
+    out = torch.full((B, g, k), -7, dtype=torch.int32, device="cuda")
+    sc = torch.full((B, g, k), float("nan"), dtype=torch.float32, device="cuda")
+    pv.dense_index_decode(d["q"], d["w"], d["k"], d["pos0"], B, Lmax, 64, 128, g, k, out, q_scale=d["qscale"],
+                          k_scale=d["kscale"], dbg_scores=sc)
+    torch.cuda.synchronize()
+    assert pv.pivot_device_status() == 0
+    out, sc = out.cpu().numpy(), sc.cpu().numpy()
+    xc = x.codes()
+    t = acc.Tally()
+    for b in range(B):
+        p0 = int(xc["pos0"][b])
+        nk = p0 + g
+        # the step's queries placed at rows pos0 .. pos0 + g - 1 of a request over this sequence's keys
+        H, dd = xc["q"].shape[2], xc["q"].shape[3]
+        q = np.zeros((nk, H, dd), xc["q"].dtype)
+        w = np.zeros((nk, H), np.float32)
+        q[p0:] = xc["q"][b]
+        w[p0:] = xc["w"][b]
+        qs = None
+        if xc["qscale"] is not None:
+            qs = np.ones((nk, H), np.float32)
+            qs[p0:] = xc["qscale"][b]
+        xb = dict(dtype=dtype, q=q, qscale=qs, w=w, k=xc["k"][b, :nk],
+                  kscale=None if xc["kscale"] is None else xc["kscale"][b, :nk])
+        o = np.full((nk, k), -1, np.int32)
+        s = np.full((nk, k), -np.inf, np.float32)
+        o[p0:], s[p0:] = out[b], sc[b]
+        t.merge(acc.check_dense(xb, k=k, out_idx=o, out_scores=s, rows=range(p0, nk)))
+    _report(f"dense decode {dtype} g={g}", t)
+    assert t.rows == B * g
+
+
+def test_decode_bad_pos0_is_reported_not_read(pv, gu):
+    """pos0 outside [0, Lmax - g]: the sequence is not indexed (rows of -1), the status word says so,
+    the other sequences are unaffected, and a following call is clean."""
+    x = inputs.make_decode(4, 2, 600, 1500, dtype="fp8", seed=62)
+    d = gu.to_cuda(x)
+    Lmax = x.k.shape[1]
+    good, _, _, _ = gu.run_decode(x, c=256, k=128, mode=po.MODE_REFINE)
+    for bad_value in (-1, Lmax - 1, Lmax + 5000):
+        pos = x.pos0.clone()
+        pos[1] = bad_value
+        out = torch.full((4, 2, 128), -7, dtype=torch.int32, device="cuda")
+        pv.pivot_index_decode(d["q"], d["w"], d["k"], pos.cuda(), 4, Lmax, 64, 128, 2, 256, 128, pv.REFINE, out,
+                              q_scale=d["qscale"], k_scale=d["kscale"])
+        torch.cuda.synchronize()
+        assert pv.pivot_device_status() == pv.DEV_BAD_POS
+        assert pv.pivot_device_status() == 0                           # read and cleared
+        o = out.cpu().numpy()
+        assert (o[1] == -1).all()
+        for b in (0, 2, 3):
+            assert np.array_equal(np.sort(o[b], axis=1), np.sort(good[b], axis=1))
+        dn = torch.full((4, 2, 128), -7, dtype=torch.int32, device="cuda")
+        pv.dense_index_decode(d["q"], d["w"], d["k"], pos.cuda(), 4, Lmax, 64, 128, 2, 128, dn, q_scale=d["qscale"],
+                              k_scale=d["kscale"])
+        torch.cuda.synchronize()
+        assert pv.pivot_device_status() == pv.DEV_BAD_POS
+        assert (dn[1] == -1).all() and (dn[0] >= 0).all()
+    again, _, _, _ = gu.run_decode(x, c=256, k=128, mode=po.MODE_REFINE)
+    assert np.array_equal(np.sort(again, axis=2), np.sort(good, axis=2))
+
+
+# ---------------------------------------------------------------- bounded device waits
+
+def test_bounded_wait_runs_out_and_reports_without_hanging(pv, gu):
+    """Failure detection: the kernels' barrier waits are bounded.  A diagnostic kernel waits -- through
+    the library's own wait routines, limit 1 ms -- on a barrier nothing completes: it must return,
+    the status word must read DEV_WAIT_EXPIRED, and the next ordinary call must be clean."""
+    import time
+    x = inputs.make_prefill(600, dtype="fp8", seed=63)
+    gu.run_prefill(x, g=4, c=128, k=64, mode=po.MODE_REFINE)           # registers a workspace
+    t0 = time.perf_counter()
+    pv.pivot_debug_wait_expiry(1_000_000)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    assert pv.pivot_device_status() == pv.DEV_WAIT_EXPIRED
+    assert dt < 1.0, f"the bounded wait took {dt:.3f} s"
+    assert pv.pivot_device_status() == 0                               # cleared by the read
+    out, sc, cand, cs = gu.run_prefill(x, g=4, c=128, k=64, mode=po.MODE_REFINE)
+    acc.check_prefill(x.codes(), g=4, c=128, k=64, mode=po.MODE_REFINE, guard_len=None, out_idx=out,
+                      out_scores=sc, cand=cand, cand_scores=cs)
+    with pytest.raises(pv.PivotError, match="invalid"):
+        pv.pivot_debug_wait_expiry(10)                                  # below 1 us
+    with pytest.raises(pv.PivotError, match="invalid"):
+        pv.pivot_debug_wait_expiry(5_000_000_000)                       # above 1 s
+
+
 # ---------------------------------------------------------------- argument errors (host side)
 
 def test_argument_errors(pv):
@@ -370,6 +491,19 @@ def test_argument_errors(pv):
 
 def _sorted_rows(a):
     return np.sort(a, axis=1)
+
+
+def _oracle_check_plain(gu, x, plain_out, *, g, c, k, mode, groups=None, what=""):
+    """Acceptance rule on the index rows of a call made WITHOUT debug buffers.  Refine's two-stage
+    check needs the candidate sets the kernels produced: they come from a second call on the same
+    inputs that asks for them (every key's score is computed independently of the launch shape, so
+    both calls rank the same candidates; if they did not, stage two would fail here)."""
+    out_d, sc_d, cand, cs = gu.run_prefill(x, g=g, c=c, k=k, mode=mode)
+    t = acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=None, out_idx=plain_out,
+                          cand=cand, cand_scores=cs, groups=groups)
+    _report(what or "plain call vs oracle", t)
+    assert t.rows > 0
+    return t
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "fp8"])
@@ -410,7 +544,7 @@ def test_two_streams_with_their_own_workspaces(pv):
         assert np.array_equal(_sorted_rows(a.cpu().numpy()), _sorted_rows(b.cpu().numpy()))
 
 
-def test_sharded_request_blocks_match_whole_call(pv):
+def test_sharded_request_blocks_match_whole_call(pv, gu):
     """The multi-GPU form of one request (row blocks dealt to ranks in snake order), with the
     ranks' shares indexed one after the other on this GPU: together they give the whole call."""
     from paper_2607_24593_b200 import sharded
@@ -428,11 +562,12 @@ def test_sharded_request_blocks_match_whole_call(pv):
     torch.cuda.synchronize()
     assert covered == L and pv.pivot_device_status() == 0
     assert np.array_equal(_sorted_rows(parts.cpu().numpy()), _sorted_rows(whole.cpu().numpy()))
+    _oracle_check_plain(gu, x, parts.cpu().numpy(), g=g, c=c, k=k, mode=po.MODE_REFINE, what="sharded row blocks")
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "fp8"])
 @pytest.mark.parametrize("mode", [po.MODE_REUSE, po.MODE_REFINE])
-def test_prefill_row_ranges_match_whole_call(pv, dtype, mode):
+def test_prefill_row_ranges_match_whole_call(pv, gu, dtype, mode):
     """Chunks of query rows (row_begin / row_end) give the rows of one whole call: same sets
     (the order inside a row is free), rows outside the chunk untouched."""
     L, g, c, k = 1900, 4, 256, 64
@@ -453,12 +588,13 @@ def test_prefill_row_ranges_match_whole_call(pv, dtype, mode):
         untouched[r0:r1] = False
         assert torch.equal(parts[untouched], before[untouched])
     assert np.array_equal(_sorted_rows(parts.cpu().numpy()), _sorted_rows(whole.cpu().numpy()))
+    _oracle_check_plain(gu, x, parts.cpu().numpy(), g=g, c=c, k=k, mode=mode, what=f"row ranges {dtype} mode={mode}")
     for bad in [(2, 8), (0, 6), (8, 8), (0, L + 4), (-4, 8)]:
         with pytest.raises(pv.PivotError, match="invalid"):
             pv.pivot_index_prefill(q, w, kk, L, 64, 128, g, c, k, mode, parts, rows=bad, **sc)
 
 
-def test_prefill_host_pipeline_matches_device_call(pv):
+def test_prefill_host_pipeline_matches_device_call(pv, gu):
     """The host-buffer entry point (chunked copies overlapping the kernels) returns what the
     device entry point returns for the same request; large enough for several chunks."""
     L, g, c, k = 20000, 4, 512, 128
@@ -475,6 +611,10 @@ def test_prefill_host_pipeline_matches_device_call(pv):
         hout.fill_(-7)
         pv.pivot_index_prefill_host(hq, hw, hk, L, 64, 128, g, c, k, pv.REFINE, hout, arena, q_scale=hqs, k_scale=hks)
         assert np.array_equal(_sorted_rows(hout.numpy()), _sorted_rows(dev.cpu().numpy()))
+    nG = L // g
+    groups = sorted({0, 127, 128, 129, 2499, 2500, 2501, nG // 2, nG - 1} |
+                    set(np.random.default_rng(5).integers(0, nG, 12).tolist()))      # chunk edges at multiples of 2500 groups
+    _oracle_check_plain(gu, x, hout.numpy(), g=g, c=c, k=k, mode=po.MODE_REFINE, groups=groups, what="host pipeline")
 
 
 # ---------------------------------------------------------------- local window (Appendix B)
@@ -509,7 +649,7 @@ def test_local_window_argument_errors(pv):
 # ---------------------------------------------------------------- packed requests (Eq. 2 boundaries)
 
 @pytest.mark.parametrize("dtype", ["bf16", "fp8"])
-def test_prefill_varlen_equals_per_request_calls(pv, dtype):
+def test_prefill_varlen_equals_per_request_calls(pv, gu, dtype):
     """Requests packed back to back give, row for row, what separate calls give: groups and causal
     prefixes stop at the request boundaries, positions are relative to the request."""
     lens = [700, 0, 1028, 300]            # starts at multiples of 4 (FP8 scale rows), one empty request
@@ -532,6 +672,7 @@ def test_prefill_varlen_equals_per_request_calls(pv, dtype):
         got = packed[cu[i]:cu[i + 1]].cpu().numpy()
         assert np.array_equal(_sorted_rows(got), _sorted_rows(one.cpu().numpy())), f"request {i}"
         assert got.max() < lens[i]
+        _oracle_check_plain(gu, x, got, g=g, c=c, k=k, mode=po.MODE_REFINE, what=f"packed request {i} {dtype}")
     if dtype == "fp8":
         with pytest.raises(pv.PivotError, match="invalid"):
             pv.pivot_index_prefill_varlen(q, w, kk, [0, 702, int(cu[-1])], 64, 128, g, c, k, mode, packed, **sc)

@@ -6,6 +6,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import acceptance as acc
 from paper_2607_24593_b200 import inputs
 
 pytestmark = pytest.mark.gpu
@@ -36,6 +37,23 @@ def test_static_scratch_matches_dense_index_twice(dtype):
         for t in (0, 1, k - 1, k, L - 1):
             n = min(k, t + 1)
             assert (np.sort(got[t])[k - n:] >= 0).all() and (got[t] <= t).all()
+        # and against the CPU oracle (Eq. 1 + TopK), under the acceptance rule of the other tests
+        rows = sorted({0, 1, k - 1, k, 127, 128, L // 2, L - 1} | set(np.random.default_rng(seed).integers(0, L, 24).tolist()))
+        tally = acc.check_dense(x.codes(), k=k, out_idx=got, rows=rows)
+        assert tally.rows == len(rows)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+def test_static_scratch_at_its_size_limits(dtype):
+    """L = 4096 and k = 512: the largest request the built-in scratch is sized for."""
+    from paper_2607_24593_b200 import binding as pv
+    L, k = 4096, 512
+    x = inputs.make_prefill(L, dtype=dtype, seed=33)
+    ref, got = _both(pv, x, L, k)
+    np.testing.assert_array_equal(np.sort(got, axis=1), np.sort(ref, axis=1))
+    rows = [0, 511, 512, 513, 2047, 4095]
+    tally = acc.check_dense(x.codes(), k=k, out_idx=got, rows=rows)
+    assert tally.rows == len(rows)
 
 
 def test_static_scratch_rejects_oversize():
