@@ -269,10 +269,10 @@ def decode_bench(pv, dev, steps, warmup, pk):
     torch.cuda.synchronize()
     window_times = timed(step_window, steps)
     assert pv.pivot_device_status() == 0
-    # the dense control of the same step (Eq. 1 + TopK for each of the g queries; the queries of a
-    # sequence share one pass over its keys), same inputs, same GPU
+    # the dense control of the same step (Eq. 1 + TopK for each of the g queries, every query a scan row
+    # of its own on the same key-split kernels), same inputs, same GPU
     dout = torch.empty_like(out)
-    pv.ensure_workspace(B * g, B, k, k, dev, need=pv.pivot_decode_workspace_bytes(B, Lmax, g, max(c, k), k))
+    pv.ensure_workspace(B * g, B * g, k, k, dev, need=pv.pivot_decode_workspace_bytes(B * g, Lmax, 1, k, k))
 
     def step_dense():
         pv.dense_index_decode(q, w, kc, p0, B, Lmax, H, D, g, k, dout, stream, q_scale=qs, k_scale=ks)
@@ -498,7 +498,11 @@ def main():
     from paper_2607_24593_b200 import binding as pv
 
     if args.mma_model:
-        print(json.dumps({"mma_model": pv.pivot_debug_mma_model()}, indent=1))
+        res = {"mma_model": pv.pivot_debug_mma_model(), "key_stream": []}
+        for ctas in (1, 74, 148):
+            for stages in (2, 4, 8, 12):
+                res["key_stream"].append(pv.pivot_debug_key_stream(ctas=ctas, stages=stages))
+        print(json.dumps(res, indent=1))
         return
     if args.sweep:
         sweep(pv, torch.device(f"cuda:{local}"), L, dtype, max(1, min(args.steps, 3)))

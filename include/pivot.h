@@ -229,9 +229,10 @@ int dense_index_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kc
  * Dense control, decode form: Eq. 1 + TopK for each of the g queries of one MTP step (the grouping
  * of Eq. 3) of B sequences -- what a DSA decode step costs without PIVOT.  Arguments as in
  * pivot_index_decode (contiguous cache); the query at position pos0[b] + i ranks keys
- * 0 .. pos0[b] + i of sequence b.  The queries of one sequence share one pass over its keys
- * (rows are packed four to a scan block per sequence).  out_idx [B, g, k] int32.  Workspace:
- * pivot_decode_workspace_bytes(B, Lmax, g, k, k).  opts: dbg_scores, workspace, impl (0 / 2).
+ * 0 .. pos0[b] + i of sequence b.  Runs on the same key-split kernels as pivot_index_decode, every
+ * query as a scan row of its own (its raw codes, effective gate fl32(w * qscale)): the g rows of a
+ * sequence stream that sequence's keys one after the other.  out_idx [B, g, k] int32.  Workspace:
+ * pivot_decode_workspace_bytes(B * g, Lmax, 1, k, k).  opts: dbg_scores, workspace.
  */
 int dense_index_decode(const pivot_tensor* q, const float* w, const pivot_tensor* kcache,
                        const int32_t* pos0, int B, int Lmax, int H_I, int d, int g, int k,
@@ -301,6 +302,16 @@ int pivot_debug_wait_expiry(unsigned long long limit_ns, pivot_stream_t stream);
  * measures time only.
  */
 int pivot_debug_mma_model(long long* out_device, pivot_stream_t stream);
+
+/*
+ * Diagnostic (no counterpart in the paper): `ctas` one-warp CTAs each pull `tiles` consecutive
+ * 16 KB key tiles (the shared scan's TMA box: 128 FP8 keys) of keys_device [n_keys, 128] (device,
+ * n_keys a multiple of 128, L2-sized) through `stages` (1..12) shared-memory stages and discard
+ * them: the rate at which L2 feeds the key stream of Eq. 5's scan to all SMs at once.
+ * out_device[cta] = clocks per tile (int64, device).
+ */
+int pivot_debug_key_stream(const void* keys_device, int n_keys, int ctas, int tiles, int stages,
+                           long long* out_device, pivot_stream_t stream);
 
 /*
  * Per-stage timing, off by default.  While enabled, every call records CUDA events on its own

@@ -26,7 +26,7 @@ SYMBOLS = [
     "pivot_index_decode", "pivot_index_decode_ex", "pivot_index_decode_paged", "dense_index", "dense_index_ex", "dense_index_static",
     "pivot_prefill_host_arena_bytes", "pivot_index_prefill_host", "pivot_device_status",
     "pivot_stage_timing", "pivot_stage_times", "pivot_launch_count_reset", "pivot_status_str", "pivot_last_cuda_error",
-    "dense_index_decode", "dense_index_decode_ex", "pivot_debug_wait_expiry", "pivot_debug_mma_model",
+    "dense_index_decode", "dense_index_decode_ex", "pivot_debug_wait_expiry", "pivot_debug_mma_model", "pivot_debug_key_stream",
 ]
 DEV_OK, DEV_WAIT_EXPIRED, DEV_CAND_OVERFLOW, DEV_BAD_POS, DEV_BOUNDS = 0, 1, 2, 3, 4
 
@@ -71,6 +71,7 @@ def _load():
     lib.dense_index_decode_ex.argtypes = [T, P, T, P, I, I, I, I, I, I, P, P, O]
     lib.pivot_debug_wait_expiry.argtypes = [C.c_ulonglong, P]
     lib.pivot_debug_mma_model.argtypes = [P, P]
+    lib.pivot_debug_key_stream.argtypes = [P, I, I, I, I, P, P]
     lib.pivot_prefill_host_arena_bytes.restype = S
     lib.pivot_prefill_host_arena_bytes.argtypes = [I, I, I, I, I, I, I]
     lib.pivot_index_prefill_host.argtypes = [T, P, T, I, I, I, I, I, I, I, P, P, S, P]
@@ -248,7 +249,7 @@ def dense_index_decode(q, w, kcache, pos0, B, Lmax, H_I, d, g, k, out_idx, strea
     assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and pos0.dtype == torch.int32
     assert out_idx.numel() >= B * g * k
     if workspace is None:
-        ensure_workspace(B * g, B, k, k, q.device, need=pivot_decode_workspace_bytes(B, Lmax, g, k, k))
+        ensure_workspace(B * g, B * g, k, k, q.device, need=pivot_decode_workspace_bytes(B * g, Lmax, 1, k, k))
     o = _opts(None, POOL_MEAN, None, dbg_scores, None, workspace, impl)
     _check(lib.dense_index_decode_ex(C.byref(tq), w.data_ptr(), C.byref(tk), pos0.data_ptr(), B, Lmax, H_I, d, g, k,
                                      out_idx.data_ptr(), _stream(stream), C.byref(o)))
@@ -282,6 +283,17 @@ def pivot_debug_mma_model(stream=None) -> dict:
             d["traffic warps: clk per 256-column pass"] = [x for x in v[ph * 32 + 16: ph * 32 + 24] if x]
         res[pname] = d
     return res
+
+
+def pivot_debug_key_stream(n_keys=131072, ctas=148, tiles=2048, stages=4, stream=None) -> dict:
+    """Key-tile streaming probe (see pivot.h): clocks per 16 KB tile over the CTAs."""
+    keys = torch.zeros((n_keys, 128), dtype=torch.uint8, device="cuda")
+    out = torch.zeros(ctas, dtype=torch.int64, device="cuda")
+    _check(lib.pivot_debug_key_stream(keys.data_ptr(), n_keys, ctas, tiles, stages, out.data_ptr(), _stream(stream)))
+    torch.cuda.synchronize()
+    v = out.cpu().float()
+    return {"n_keys": n_keys, "ctas": ctas, "stages": stages, "tiles_per_cta": tiles,
+            "clk_per_tile_mean": float(v.mean()), "clk_per_tile_min": float(v.min()), "clk_per_tile_max": float(v.max())}
 
 
 def pivot_prefill_host_arena_bytes(L, H_I, d, g, c, k, dtype) -> int:

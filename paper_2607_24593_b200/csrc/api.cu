@@ -270,13 +270,9 @@ size_t pivot_workspace_bytes(int rows, int n_groups, int c, int k) {
   return carve_workspace(nullptr, rows, n_groups, c, k).bytes;
 }
 
-// Row slots of a decode call: the step's B * g queries, padded per sequence to a multiple of four
-// (the dense control packs a sequence's rows into four-row blocks).
-static int decode_row_slots(int B, int g) { return B * ((g + 3) / 4 * 4); }
-
 size_t pivot_decode_workspace_bytes(int B, int Lmax, int g, int c, int k) {
   if (B < 1 || Lmax < 1 || g < 1 || c < 1 || k < 1) return 0;
-  return pivot_workspace_bytes(decode_row_slots(B, g), B, c, k) + decode_fast_bytes(B, Lmax, g, c);
+  return pivot_workspace_bytes(B * g, B, c, k) + decode_fast_bytes(B, Lmax, g, c);
 }
 
 int pivot_set_workspace(void* workspace, size_t bytes) {
@@ -347,10 +343,13 @@ int dense_index(const pivot_tensor* q, const float* w, const pivot_tensor* kcach
 // pool of n_pages pages of 128 keys and block_table [B, Lmax / 128] names each sequence's pages.
 static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor* kcache, const int32_t* pos0,
                       int B, int Lmax, int H_I, int d, int g, int c, int k, int mode, int32_t* out_idx,
-                      pivot_stream_t stream, const pivot_opts* o, const int32_t* block_table, int n_pages) {
+                      pivot_stream_t stream, const pivot_opts* o, const int32_t* block_table, int n_pages,
+                      int dense_share = 0) {
+  // dense_share > 0: the dense control -- B counts the step's queries, each planned as a sequence
+  // of one member (g = 1) scanned with its own raw query; dense_share of them share a key cache
   int rc = check_common(q, w, kcache, H_I, d, c, k, mode, out_idx);
   if (rc) return rc;
-  if (!pos0 || B < 1 || g < 1 || Lmax < g) return PIVOT_ERR_INVALID_ARG;
+  if (!pos0 || B < 1 || g < 1 || Lmax < g || Lmax < dense_share) return PIVOT_ERR_INVALID_ARG;
   // every sequence's scale row must start on a 16-byte boundary (TMA reads it in 128-scale tiles)
   if (q->dtype == PIVOT_FP8_E4M3 && (Lmax & 3)) return PIVOT_ERR_INVALID_ARG;
   if (o && (o->pool < 0 || o->pool > 2)) return PIVOT_ERR_INVALID_ARG;
@@ -362,11 +361,11 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
   const bool paged = block_table != nullptr;
   if (paged && (n_pages < 1 || (Lmax & 127) || (o && o->impl == 1))) return PIVOT_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
-  const size_t base_bytes = pivot_workspace_bytes(decode_row_slots(B, g), B, c, k);
+  const size_t base_bytes = pivot_workspace_bytes(B * g, B, c, k);
   const size_t need = base_bytes + decode_fast_bytes(B, Lmax, g, c);
   void* wsp = nullptr;
   if ((rc = resolve_ws(o, need, &wsp))) return rc;
-  Workspace ws = carve_workspace(wsp, decode_row_slots(B, g), B, c, k);
+  Workspace ws = carve_workspace(wsp, B * g, B, c, k);
   g_dev[cur_device()].last_status = ws.status;
   DecodePlan p;
   p.q = q->data; p.w = w; p.qscale = q->scale;
@@ -380,16 +379,18 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
   p.guard_len = (o && o->guard_len >= 0) ? o->guard_len : c;
   // Paged: a short sequence's dense rows would need a contiguous prefix, so the guardrail is
   // off and short sequences take the proxy path with every visible key as a candidate.
-  if (paged) p.guard_len = 0;
+  if (paged || dense_share) p.guard_len = 0;
+  if (dense_share) { p.kv_share = dense_share; p.raw_q = true; }
   p.block_table = block_table;
   p.n_pages = n_pages;
   p.status = ws.status;
   p.W = W;
-  const long long k_rows = paged ? (long long)n_pages * 128 : (long long)B * Lmax;
+  const long long k_rows = paged ? (long long)n_pages * 128 : (long long)(dense_share ? B / dense_share : B) * Lmax;
   if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 3 * sizeof(int), st)))) return rc;   // status, row counter, prepare ticket
   mark(0, st);
-  launch_proxy_build(q->data, q->scale, w, ws.proxy_q, ws.proxy_w, B * g, g, 0, B, q->dtype,
-                     o ? o->pool : 0, st);
+  if (!dense_share)
+    launch_proxy_build(q->data, q->scale, w, ws.proxy_q, ws.proxy_w, B * g, g, 0, B, q->dtype,
+                       o ? o->pool : 0, st);
   mark(1, st);
   if (o && o->impl == 1) launch_plan_decode(p, ws.rows, ws.groups, st);   // the tensor-core path plans inside its prepare kernel
   mark(2, st);
@@ -400,7 +401,7 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
     DecodeFast df;
     df.plan = p; df.ticket = ws.status + 2;
     df.prox = ws.rows; df.groups = ws.groups;
-    df.kc = kcache->data; df.kscale = kcache->scale; df.q = q->data; df.proxy_q = ws.proxy_q;
+    df.kc = kcache->data; df.kscale = kcache->scale; df.q = q->data; df.proxy_q = dense_share ? q->data : ws.proxy_q;
     df.B = B; df.Lmax = Lmax; df.g = g; df.c = c; df.k = k; df.mode = mode; df.dtype = q->dtype;
     df.k_rows = k_rows;
     df.W = W;
@@ -452,38 +453,11 @@ int pivot_index_decode(const pivot_tensor* q, const float* w, const pivot_tensor
 int dense_index_decode_ex(const pivot_tensor* q, const float* w, const pivot_tensor* kcache, const int32_t* pos0,
                           int B, int Lmax, int H_I, int d, int g, int k, int32_t* out_idx, pivot_stream_t stream,
                           const pivot_opts* o) {
-  int rc = check_common(q, w, kcache, H_I, d, k, k, PIVOT_REUSE, out_idx);
-  if (rc) return rc;
-  if (!pos0 || B < 1 || g < 1 || Lmax < g) return PIVOT_ERR_INVALID_ARG;
-  if (q->dtype == PIVOT_FP8_E4M3 && (Lmax & 3)) return PIVOT_ERR_INVALID_ARG;
-  cudaStream_t st = (cudaStream_t)stream;
-  const int gp = (g + 3) / 4 * 4;
-  const size_t need = pivot_decode_workspace_bytes(B, Lmax, g, k, k);
-  void* wsp = nullptr;
-  if ((rc = resolve_ws(o, need, &wsp))) return rc;
-  Workspace ws = carve_workspace(wsp, decode_row_slots(B, g), B, k, k);
-  g_dev[cur_device()].last_status = ws.status;
-  DecodePlan p;
-  p.q = q->data; p.w = w; p.qscale = q->scale;
-  p.kc = kcache->data; p.kscale = kcache->scale;
-  p.pos0 = pos0;
-  p.proxy_q = nullptr; p.proxy_w = nullptr; p.cand = nullptr; p.cand_score = nullptr;
-  p.out = out_idx; p.out_score = o ? o->dbg_scores : nullptr;
-  p.B = B; p.Lmax = Lmax; p.g = g; p.c = k; p.k = k; p.mode = PIVOT_REUSE; p.dtype = q->dtype;
-  p.guard_len = 0;
-  p.status = ws.status;
-  if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 3 * sizeof(int), st)))) return rc;
-  mark(0, st);
-  mark(1, st);
-  launch_plan_dense_decode(p, ws.rows, gp, st);
-  mark(2, st);
-  // the proxy tensor map needs some valid address; no row refers to it
-  ScanOperands op{kcache->data, (long long)B * Lmax, kcache->scale, q->data, B * g, q->data, 1, q->dtype};
-  if ((rc = check_cuda(launch_scan_tc(op, ws.rows, B * gp, 4, tc_scratch(ws), sm_count(), st, o && o->impl == 2))))
-    return rc;
-  mark(3, st);
-  mark(4, st);
-  return check_cuda(cudaGetLastError());
+  if (B < 1 || g < 1 || (long long)B * g > (1 << 24)) return PIVOT_ERR_INVALID_ARG;
+  if (o && (o->impl == 1 || o->W)) return PIVOT_ERR_INVALID_ARG;
+  // Every query of the step as a sequence of one member on the key-split decode path: Reuse with
+  // g = 1 and the raw query as its own scan row is Eq. 1 + TopK (c plays no part).
+  return run_decode(q, w, kcache, pos0, B * g, Lmax, H_I, d, 1, k, k, PIVOT_REUSE, out_idx, stream, o, nullptr, 0, g);
 }
 
 int dense_index_decode(const pivot_tensor* q, const float* w, const pivot_tensor* kcache, const int32_t* pos0,
@@ -506,6 +480,12 @@ int pivot_debug_wait_expiry(unsigned long long limit_ns, pivot_stream_t stream) 
 int pivot_debug_mma_model(long long* out_device, pivot_stream_t stream) {
   if (!out_device || ((uintptr_t)out_device & 7)) return PIVOT_ERR_INVALID_ARG;
   return check_cuda(launch_mma_model_probe(out_device, (cudaStream_t)stream));
+}
+
+int pivot_debug_key_stream(const void* keys_device, int n_keys, int ctas, int tiles, int stages, long long* out_device,
+                           pivot_stream_t stream) {
+  if (!keys_device || !out_device || ((uintptr_t)keys_device & 15) || ((uintptr_t)out_device & 7)) return PIVOT_ERR_INVALID_ARG;
+  return check_cuda(launch_key_stream_probe(keys_device, n_keys, ctas, tiles, stages, out_device, (cudaStream_t)stream));
 }
 
 size_t pivot_prefill_host_arena_bytes(int L, int H_I, int d, int g, int c, int k, int dtype) {

@@ -7,6 +7,8 @@
 // same two functions, with a short limit passed in -- for a barrier phase that nothing will ever
 // complete, fall through when the limit runs out, and report the status exactly as the real
 // kernels do at their teardown.  Nothing traps and nothing spins without bound.
+#include <cuda.h>
+
 #include "kernels.h"
 #include "ptx.cuh"
 
@@ -264,6 +266,42 @@ __global__ void __launch_bounds__(416, 1) mma_model_probe_kernel(long long* out)
 
 }  // namespace
 
+// Key-tile streaming alone: every CTA pulls 16 KB key tiles (128 keys x 128 B, the scan's TMA box) of
+// one L2-resident key tensor through a ring of `stages` shared-memory stages and does nothing with
+// them -- the rate at which L2 can feed all SMs the scan's key stream.  Each CTA starts at its own
+// offset and walks `tiles` consecutive tiles (wrapping), as the scan's CTAs do.
+__global__ void __launch_bounds__(32, 1) key_stream_probe_kernel(const __grid_constant__ CUtensorMap tm_k, int n_tiles_total,
+                                                                 int tiles, int stages, long long* out) {
+  extern __shared__ uint8_t raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
+  __shared__ uint64_t full[12];
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 12; ++i) ptx::mbar_init(&full[i], 1);
+    abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  __syncwarp();
+  if (threadIdx.x == 0) {
+    ptx::prefetch_tensormap(&tm_k);
+    const int start = (int)(((long long)blockIdx.x * 977) % n_tiles_total);
+    auto issue = [&](int t) {
+      const int s = t % stages;
+      ptx::mbar_arrive_expect_tx(&full[s], 16384);
+      ptx::tma_load_2d(smem + s * 16384, &tm_k, 0, ((start + t) % n_tiles_total) * 128, &full[s]);
+    };
+    for (int t = 0; t < stages && t < tiles; ++t) issue(t);
+    const long long t0 = clock64();
+    for (int t = 0; t < tiles; ++t) {
+      const int s = t % stages;
+      if (!ptx::mbar_wait_poll(&full[s], (uint32_t)((t / stages) & 1), &abort_flag)) break;
+      if (t + stages < tiles) issue(t + stages);
+    }
+    out[blockIdx.x] = (clock64() - t0) / tiles;
+    if (abort_flag) out[blockIdx.x] = -1;
+  }
+}
+
 // out: 256 long longs (device).  [phase * 32 + variant] = tensor-pipe clocks per tile for the issuer variants
 // (phase 0 alone, 1 with ReLU-pass traffic, 2 with load-only traffic from 4 warps, 3 from 8 warps);
 // [phase * 32 + 16 + w] = clocks per 256-column pass of traffic warp w; [128], [129] one-way mbarrier
@@ -273,6 +311,24 @@ cudaError_t launch_mma_model_probe(long long* out, cudaStream_t st) {
   static bool attr[kMaxDevices] = {};
   if (cudaError_t e = opt_in_dynamic_smem(mma_model_probe_kernel, smem, attr); e != cudaSuccess) return e;
   mma_model_probe_kernel<<<1, 416, smem, st>>>(out);
+  ++launch_counter();
+  return cudaGetLastError();
+}
+
+bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows);
+
+// keys: an FP8 key tensor [n_keys, 128] (device), n_keys a multiple of 128; out: one slot per CTA
+// (clocks per tile seen by that CTA).
+cudaError_t launch_key_stream_probe(const void* keys, int n_keys, int ctas, int tiles, int stages, long long* out,
+                                    cudaStream_t st) {
+  if (stages < 1 || stages > 12 || n_keys < 128 || (n_keys & 127) || ctas < 1 || tiles < 1) return cudaErrorInvalidValue;
+  CUtensorMap mk;
+  if (!make_operand_map(&mk, keys, n_keys, DT_FP8, 128)) return cudaErrorInvalidValue;
+  const size_t smem = 1024 + (size_t)stages * 16384;
+  if (cudaError_t e = cudaFuncSetAttribute(key_stream_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      e != cudaSuccess)
+    return e;
+  key_stream_probe_kernel<<<ctas, 32, smem, st>>>(mk, n_keys / 128, tiles, stages, out);
   ++launch_counter();
   return cudaGetLastError();
 }

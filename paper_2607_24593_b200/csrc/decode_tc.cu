@@ -443,6 +443,7 @@ decode_prepare_kernel(DecodePlan p, RowDesc* rows, GroupDesc* plan_groups, uint3
     if (threadIdx.x == 0) seq_ok = plan_decode_sequence(p, b, rows, plan_groups) ? 1 : 0;
     __syncthreads();
     if (!seq_ok) fill_decode_rows_empty(p, b, threadIdx.x, blockDim.x);     // pos0 outside the cache: rows of -1
+    if (p.raw_q) raw_query_gates(p, b, threadIdx.x, blockDim.x);
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) is_last = atomicAdd(ticket, 1) == (int)gridDim.x - 1;

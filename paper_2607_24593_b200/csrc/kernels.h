@@ -80,6 +80,13 @@ struct DecodePlan {
   int n_pages = 0;
   int W = 0;                                            // per-query local window (Appendix B, decode form)
   int* status = nullptr;                                // device status word (a bad pos0 is reported there)
+  // Dense control (Eq. 1 per query): every query of the step is planned as a sequence of its own
+  // with one member.  kv_share consecutive plan slots then share one key cache: slot b reads cache
+  // b / kv_share and sits at position pos0[b / kv_share] + b % kv_share.  raw_q: the scan rows
+  // are the raw queries themselves (no proxy is built); the planner leaves their effective gates
+  // fl32(w * qscale) in proxy_w.
+  int kv_share = 1;
+  bool raw_q = false;
 };
 
 struct ScanScratch {
@@ -144,8 +151,9 @@ long long& launch_counter();
 cudaError_t launch_wait_expiry_probe(int* status, unsigned long long limit_ns, cudaStream_t st);
 // Diagnostic: tensor-pipe / tensor-memory / hand-over timings of one SM (see debug_probe.cu); out = 256 slots.
 cudaError_t launch_mma_model_probe(long long* out, cudaStream_t st);
-// Dense control of a decode step: rows of a sequence padded to blocks of four that share a key stream.
-void launch_plan_dense_decode(const DecodePlan& p, RowDesc* rows, int gp, cudaStream_t st);
+// Diagnostic: rate at which all SMs together can pull the scan's 16 KB key tiles out of L2.
+cudaError_t launch_key_stream_probe(const void* keys, int n_keys, int ctas, int tiles, int stages, long long* out,
+                                    cudaStream_t st);
 
 // The opt-in to more than 48 KB of dynamic shared memory is an attribute of (function, device):
 // remembered per device, so that a process driving several GPUs sets it on each of them.

@@ -92,51 +92,9 @@ void launch_plan_prefill(const PrefillPlan& p, RowDesc* rows, GroupDesc* groups,
 
 __global__ void plan_decode_kernel(DecodePlan p, RowDesc* rows, GroupDesc* groups) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b < p.B && !plan_decode_sequence(p, b, rows, groups)) fill_decode_rows_empty(p, b, 0, 1);
-}
-
-// Dense control of a decode step (Eq. 1 for each of the g queries of every sequence): the rows of
-// sequence b occupy slots b * gp .. b * gp + gp - 1 with gp = g rounded up to a multiple of four, so
-// that a four-row block of the scan never mixes two sequences and the queries of one step share
-// one pass over that sequence's keys.  Padding slots and sequences with a bad pos0 are dead (K = 0).
-__global__ void plan_dense_decode_kernel(DecodePlan p, RowDesc* rows, int gp) {
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= p.B * gp) return;
-  const int b = idx / gp, i = idx % gp;
-  const size_t esz = p.dtype == DT_FP8 ? 1 : 2;
-  const size_t qrow = (size_t)kHeads * kDim * esz;
-  const int p_in = p.pos0[b];
-  const bool bad = p_in < 0 || p_in > p.Lmax - p.g;
-  const int p0 = bad ? 0 : p_in;
-  const int qi = b * p.g + (i < p.g ? i : p.g - 1);        // padding slots point at a real query (never selected from)
-  const bool live = i < p.g && !bad;
-  RowDesc dr;
-  dr.q = (const char*)p.q + (size_t)qi * qrow;
-  dr.w = p.w + (size_t)qi * kHeads;
-  dr.qscale = p.qscale ? p.qscale + (size_t)qi * kHeads : nullptr;
-  dr.kbase = (const char*)p.kc + (size_t)b * p.Lmax * kDim * esz;
-  dr.kscale = p.kscale ? p.kscale + (size_t)b * p.Lmax : nullptr;
-  dr.n_vis = live ? p0 + i + 1 : 0;
-  dr.K = live ? p.k : 0;
-  dr.out = p.out + (size_t)qi * p.k;
-  dr.out_score = p.out_score ? p.out_score + (size_t)qi * p.k : nullptr;
-  dr.out_rows = 1;
-  dr.out_stride = p.k;
-  dr.q_map = 0; dr.q_row = qi; dr.k_row0 = b * p.Lmax;
-  rows[idx] = dr;
-  if (bad && i < p.g) {
-    set_status(p.status, DEV_BAD_POS);
-    for (int j = 0; j < p.k; ++j) {
-      dr.out[j] = -1;
-      if (dr.out_score) dr.out_score[j] = -INFINITY;
-    }
-  }
-}
-
-void launch_plan_dense_decode(const DecodePlan& p, RowDesc* rows, int gp, cudaStream_t st) {
-  const int n = p.B * gp;
-  plan_dense_decode_kernel<<<(n + 127) / 128, 128, 0, st>>>(p, rows, gp);
-  ++launch_counter();
+  if (b >= p.B) return;
+  if (!plan_decode_sequence(p, b, rows, groups)) fill_decode_rows_empty(p, b, 0, 1);
+  if (p.raw_q) raw_query_gates(p, b, 0, 1);
 }
 
 void launch_plan_decode(const DecodePlan& p, RowDesc* rows, GroupDesc* groups, cudaStream_t st) {

@@ -37,27 +37,29 @@ __device__ __forceinline__ void put_group_chunks(GroupDesc* slots, const GroupDe
 __device__ __forceinline__ bool plan_decode_sequence(const DecodePlan& p, int b, RowDesc* rows, GroupDesc* groups) {
   const size_t esz = p.dtype == DT_FP8 ? 1 : 2;
   const size_t qrow = (size_t)kHeads * kDim * esz;
-  const int p_in = p.pos0[b];
-  const bool bad = p_in < 0 || p_in > p.Lmax - p.g;
+  const int cb = b / p.kv_share;                 // whose key cache (and pos0) this slot uses
+  const int p_in = p.pos0[cb];
+  const int step = p.g > p.kv_share ? p.g : p.kv_share;          // queries of the MTP step
+  const bool bad = p_in < 0 || p_in > p.Lmax - step;
   if (bad) set_status(p.status, DEV_BAD_POS);
-  const int p0 = bad ? 0 : p_in;
+  const int p0 = bad ? 0 : p_in + b % p.kv_share;
   const int n0 = p0 + 1;
   const bool guarded = n0 < p.guard_len;
   // Paged cache: descriptors point at the page pool and carry the sequence's block-table row.
   const bool paged = p.block_table != nullptr;
-  const int32_t* pages = paged ? p.block_table + (size_t)b * (p.Lmax / 128) : nullptr;
-  const void* kb = paged ? p.kc : (const char*)p.kc + (size_t)b * p.Lmax * kDim * esz;
-  const float* ksb = !p.kscale ? nullptr : paged ? p.kscale : p.kscale + (size_t)b * p.Lmax;
+  const int32_t* pages = paged ? p.block_table + (size_t)cb * (p.Lmax / 128) : nullptr;
+  const void* kb = paged ? p.kc : (const char*)p.kc + (size_t)cb * p.Lmax * kDim * esz;
+  const float* ksb = !p.kscale ? nullptr : paged ? p.kscale : p.kscale + (size_t)cb * p.Lmax;
   int32_t* outb = p.out + (size_t)b * p.g * p.k;
   float* outsb = p.out_score ? p.out_score + (size_t)b * p.g * p.k : nullptr;
   RowDesc r;
-  r.q = (const char*)p.proxy_q + (size_t)b * qrow;
+  r.q = (const char*)(p.raw_q ? p.q : p.proxy_q) + (size_t)b * qrow;
   r.w = p.proxy_w + (size_t)b * kHeads;
   r.qscale = nullptr;
   r.kbase = kb;
   r.kscale = ksb;
   r.n_vis = n0;
-  r.q_map = 1; r.q_row = b; r.k_row0 = paged ? 0 : b * p.Lmax;
+  r.q_map = p.raw_q ? 0 : 1; r.q_row = b; r.k_row0 = paged ? 0 : cb * p.Lmax;
   r.pages = pages;
   GroupDesc gd;
   gd.pages = pages;
@@ -102,10 +104,19 @@ __device__ __forceinline__ bool plan_decode_sequence(const DecodePlan& p, int b,
     dr.out_score = outsb ? outsb + (size_t)i * p.k : nullptr;
     dr.out_rows = 1;
     dr.out_stride = p.k;
-    dr.q_map = 0; dr.q_row = b * p.g + i; dr.k_row0 = b * p.Lmax;
+    dr.q_map = 0; dr.q_row = b * p.g + i; dr.k_row0 = cb * p.Lmax;
     rows[p.B + b * p.g + i] = dr;
   }
   return !bad;
+}
+
+// Dense control: the scan row of slot b is the raw query b, whose effective gate fl32(w * qscale)
+// (Appendix A: the gate absorbs the query scale) goes where a proxy's gate would be.
+__device__ __forceinline__ void raw_query_gates(const DecodePlan& p, int b, int tid, int nthreads) {
+  for (int j = tid; j < kHeads; j += nthreads) {
+    const size_t i = (size_t)b * kHeads + j;
+    p.proxy_w[i] = p.qscale ? __fmul_rn(p.w[i], p.qscale[i]) : p.w[i];
+  }
 }
 
 // Output rows of a sequence that was not indexed (bad pos0): every entry -1 (scores -inf).
