@@ -499,9 +499,8 @@ def main():
 
     if args.mma_model:
         res = {"mma_model": pv.pivot_debug_mma_model(), "key_stream": []}
-        for ctas in (1, 74, 148):
-            for stages in (2, 4, 8, 12):
-                res["key_stream"].append(pv.pivot_debug_key_stream(ctas=ctas, stages=stages))
+        for ctas, stages, mode in ((1, 4, 0), (148, 2, 0), (148, 4, 0), (148, 8, 0), (148, 4, 1), (148, 4, 2), (1, 4, 2)):
+            res["key_stream"].append(pv.pivot_debug_key_stream(ctas=ctas, stages=stages, mode=mode))
         print(json.dumps(res, indent=1))
         return
     if args.sweep:

@@ -26,7 +26,7 @@ SYMBOLS = [
     "pivot_index_decode", "pivot_index_decode_ex", "pivot_index_decode_paged", "dense_index", "dense_index_ex", "dense_index_static",
     "pivot_prefill_host_arena_bytes", "pivot_index_prefill_host", "pivot_device_status",
     "pivot_stage_timing", "pivot_stage_times", "pivot_launch_count_reset", "pivot_status_str", "pivot_last_cuda_error",
-    "dense_index_decode", "dense_index_decode_ex", "pivot_debug_wait_expiry", "pivot_debug_mma_model", "pivot_debug_key_stream",
+    "dense_index_decode", "dense_index_decode_ex", "pivot_debug_wait_expiry", "pivot_debug_mma_model", "pivot_debug_key_stream", "pivot_debug_scan_profile",
 ]
 DEV_OK, DEV_WAIT_EXPIRED, DEV_CAND_OVERFLOW, DEV_BAD_POS, DEV_BOUNDS = 0, 1, 2, 3, 4
 
@@ -71,7 +71,7 @@ def _load():
     lib.dense_index_decode_ex.argtypes = [T, P, T, P, I, I, I, I, I, I, P, P, O]
     lib.pivot_debug_wait_expiry.argtypes = [C.c_ulonglong, P]
     lib.pivot_debug_mma_model.argtypes = [P, P]
-    lib.pivot_debug_key_stream.argtypes = [P, I, I, I, I, P, P]
+    lib.pivot_debug_key_stream.argtypes = [P, I, I, I, I, I, P, P]
     lib.pivot_prefill_host_arena_bytes.restype = S
     lib.pivot_prefill_host_arena_bytes.argtypes = [I, I, I, I, I, I, I]
     lib.pivot_index_prefill_host.argtypes = [T, P, T, I, I, I, I, I, I, I, P, P, S, P]
@@ -113,7 +113,7 @@ def _stream(stream) -> int:
     return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
 
 
-IMPL_TENSOR_CORE, IMPL_CUDA_CORE, IMPL_TENSOR_CORE_FP32_HEAD_SUM = 0, 1, 2
+IMPL_TENSOR_CORE, IMPL_CUDA_CORE, IMPL_TENSOR_CORE_FP32_HEAD_SUM, IMPL_TENSOR_CORE_BF16_HEAD_SUM = 0, 1, 2, 3
 
 
 def _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl=0, rows=None, W=0) -> pivot_opts:
@@ -285,15 +285,25 @@ def pivot_debug_mma_model(stream=None) -> dict:
     return res
 
 
-def pivot_debug_key_stream(n_keys=131072, ctas=148, tiles=2048, stages=4, stream=None) -> dict:
-    """Key-tile streaming probe (see pivot.h): clocks per 16 KB tile over the CTAs."""
-    keys = torch.zeros((n_keys, 128), dtype=torch.uint8, device="cuda")
-    out = torch.zeros(ctas, dtype=torch.int64, device="cuda")
-    _check(lib.pivot_debug_key_stream(keys.data_ptr(), n_keys, ctas, tiles, stages, out.data_ptr(), _stream(stream)))
+def pivot_debug_scan_profile() -> list:
+    """Cycle counters of the FP8 scan's first CTA (zeros unless built with -DPIVOT_PROF)."""
     torch.cuda.synchronize()
-    v = out.cpu().float()
+    out = (C.c_ulonglong * 64)()
+    _check(lib.pivot_debug_scan_profile(out))
+    return [int(v) for v in out]
+
+
+def pivot_debug_key_stream(n_keys=131072, ctas=148, tiles=2048, stages=4, mode=0, stream=None) -> dict:
+    """Key-tile streaming probe (see pivot.h): clocks per 16 KB tile, mean over the CTAs, per stream."""
+    keys = torch.zeros((n_keys, 128), dtype=torch.uint8, device="cuda")
+    out = torch.zeros(2 * ctas, dtype=torch.int64, device="cuda")
+    _check(lib.pivot_debug_key_stream(keys.data_ptr(), n_keys, ctas, tiles, stages, mode, out.data_ptr(), _stream(stream)))
+    torch.cuda.synchronize()
+    v = out.cpu().float().view(ctas, 2)
     return {"n_keys": n_keys, "ctas": ctas, "stages": stages, "tiles_per_cta": tiles,
-            "clk_per_tile_mean": float(v.mean()), "clk_per_tile_min": float(v.min()), "clk_per_tile_max": float(v.max())}
+            "mode": ["one TMA stream", "two TMA streams", "TMA stream + cp.async stream",
+                     "one thread, four 32-key boxes per tile", "four lanes, one 32-key box each"][mode],
+            "clk_per_tile_stream0": float(v[:, 0].mean()), "clk_per_tile_stream1": float(v[:, 1].mean()) if mode else None}
 
 
 def pivot_prefill_host_arena_bytes(L, H_I, d, g, c, k, dtype) -> int:

@@ -270,35 +270,77 @@ __global__ void __launch_bounds__(416, 1) mma_model_probe_kernel(long long* out)
 // one L2-resident key tensor through a ring of `stages` shared-memory stages and does nothing with
 // them -- the rate at which L2 can feed all SMs the scan's key stream.  Each CTA starts at its own
 // offset and walks `tiles` consecutive tiles (wrapping), as the scan's CTAs do.
-__global__ void __launch_bounds__(32, 1) key_stream_probe_kernel(const __grid_constant__ CUtensorMap tm_k, int n_tiles_total,
-                                                                 int tiles, int stages, long long* out) {
+__global__ void __launch_bounds__(160, 1) key_stream_probe_kernel(const __grid_constant__ CUtensorMap tm_k, const uint8_t* keys,
+                                                                  int n_tiles_total, int tiles, int stages, int mode,
+                                                                  long long* out) {
+  // mode 0: one TMA ring (warp 0).  mode 1: a second, independent TMA ring on warp 1.  mode 2: warp 0's
+  // TMA ring plus warps 1-4 streaming other tiles with 16-byte cp.async (the load/store unit's path).
   extern __shared__ uint8_t raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
-  __shared__ uint64_t full[12];
+  __shared__ uint64_t full[2][12];
   __shared__ int abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 12; ++i) ptx::mbar_init(&full[i], 1);
+    for (int i = 0; i < 24; ++i) ptx::mbar_init(&full[0][0] + i, 1);
     abort_flag = 0;
     ptx::fence_barrier_init();
   }
-  __syncwarp();
-  if (threadIdx.x == 0) {
+  __syncthreads();
+  const int start = (int)(((long long)blockIdx.x * 977) % n_tiles_total);
+  if (mode < 3 && (warp == 0 || (warp == 1 && mode == 1)) && lane == 0) {
     ptx::prefetch_tensormap(&tm_k);
-    const int start = (int)(((long long)blockIdx.x * 977) % n_tiles_total);
+    uint8_t* ring = smem + warp * stages * 16384;
+    const int first = start + warp * (n_tiles_total / 2);
     auto issue = [&](int t) {
       const int s = t % stages;
-      ptx::mbar_arrive_expect_tx(&full[s], 16384);
-      ptx::tma_load_2d(smem + s * 16384, &tm_k, 0, ((start + t) % n_tiles_total) * 128, &full[s]);
+      ptx::mbar_arrive_expect_tx(&full[warp][s], 16384);
+      ptx::tma_load_2d(ring + s * 16384, &tm_k, 0, ((first + t) % n_tiles_total) * 128, &full[warp][s]);
     };
     for (int t = 0; t < stages && t < tiles; ++t) issue(t);
     const long long t0 = clock64();
     for (int t = 0; t < tiles; ++t) {
       const int s = t % stages;
-      if (!ptx::mbar_wait_poll(&full[s], (uint32_t)((t / stages) & 1), &abort_flag)) break;
+      if (!ptx::mbar_wait_poll(&full[warp][s], (uint32_t)((t / stages) & 1), &abort_flag)) break;
       if (t + stages < tiles) issue(t + stages);
     }
-    out[blockIdx.x] = (clock64() - t0) / tiles;
-    if (abort_flag) out[blockIdx.x] = -1;
+    out[blockIdx.x * 2 + warp] = (clock64() - t0) / tiles;
+    if (abort_flag) out[blockIdx.x * 2 + warp] = -1;
+  } else if (mode >= 3 && warp == 0 && (lane == 0 || (mode == 4 && lane < 4))) {
+    // mode 3: one thread issues the tile as four boxes of 32 keys; mode 4: four lanes issue one box each
+    ptx::prefetch_tensormap(&tm_k);
+    auto issue = [&](int t) {
+      const int s = t % stages;
+      if (lane == 0) ptx::mbar_arrive_expect_tx(&full[0][s], 16384);
+      __syncwarp(mode == 4 ? 0xfu : 0x1u);
+      for (int i = (mode == 4 ? lane : 0); i < 4; i += (mode == 4 ? 4 : 1))
+        ptx::tma_load_2d(smem + s * 16384 + i * 4096, &tm_k, 0, ((start + t) % n_tiles_total) * 128 + i * 32, &full[0][s]);
+    };
+    for (int t = 0; t < stages && t < tiles; ++t) issue(t);
+    const long long t0 = clock64();
+    for (int t = 0; t < tiles; ++t) {
+      const int s = t % stages;
+      if (!ptx::mbar_wait_poll(&full[0][s], (uint32_t)((t / stages) & 1), &abort_flag)) break;
+      if (t + stages < tiles) issue(t + stages);
+    }
+    if (lane == 0) out[blockIdx.x * 2] = (clock64() - t0) / tiles;
+  } else if (mode == 2 && warp >= 1) {
+    // four warps share the second stream: warp w copies quarter w of every tile
+    uint8_t* ring = smem + stages * 16384;
+    const int first = start + n_tiles_total / 2;
+    const int wq = warp - 1;
+    const long long t0 = clock64();
+    for (int t = 0; t < tiles; ++t) {
+      const uint8_t* src = keys + (size_t)((first + t) % n_tiles_total) * 16384 + wq * 4096;
+      const uint32_t dst = ptx::smem_u32(ring + (t % stages) * 16384 + wq * 4096);
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (i * 32 + lane) * 16), "l"(src + (i * 32 + lane) * 16)
+                     : "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      asm volatile("cp.async.wait_group 3;" ::: "memory");
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (lane == 0 && wq == 0) out[blockIdx.x * 2 + 1] = (clock64() - t0) / tiles;
   }
 }
 
@@ -318,17 +360,18 @@ cudaError_t launch_mma_model_probe(long long* out, cudaStream_t st) {
 bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows);
 
 // keys: an FP8 key tensor [n_keys, 128] (device), n_keys a multiple of 128; out: one slot per CTA
-// (clocks per tile seen by that CTA).
-cudaError_t launch_key_stream_probe(const void* keys, int n_keys, int ctas, int tiles, int stages, long long* out,
+// (clocks per tile seen by that CTA's first and, with mode 1 / 2, second stream: out[2 cta], out[2 cta + 1]).
+cudaError_t launch_key_stream_probe(const void* keys, int n_keys, int ctas, int tiles, int stages, int mode, long long* out,
                                     cudaStream_t st) {
+  if (mode < 0 || mode > 4 || ((mode == 1 || mode == 2) && stages > 6)) return cudaErrorInvalidValue;
   if (stages < 1 || stages > 12 || n_keys < 128 || (n_keys & 127) || ctas < 1 || tiles < 1) return cudaErrorInvalidValue;
   CUtensorMap mk;
-  if (!make_operand_map(&mk, keys, n_keys, DT_FP8, 128)) return cudaErrorInvalidValue;
-  const size_t smem = 1024 + (size_t)stages * 16384;
+  if (!make_operand_map(&mk, keys, n_keys, DT_FP8, mode >= 3 ? 32 : 128)) return cudaErrorInvalidValue;
+  const size_t smem = 1024 + (size_t)stages * 16384 * ((mode == 1 || mode == 2) ? 2 : 1);
   if (cudaError_t e = cudaFuncSetAttribute(key_stream_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       e != cudaSuccess)
     return e;
-  key_stream_probe_kernel<<<ctas, 32, smem, st>>>(mk, n_keys / 128, tiles, stages, out);
+  key_stream_probe_kernel<<<ctas, 160, smem, st>>>(mk, (const uint8_t*)keys, n_keys / 128, tiles, stages, mode, out);
   ++launch_counter();
   return cudaGetLastError();
 }

@@ -120,8 +120,15 @@ struct ScanOperands {
 // rows_per_block consecutive scan rows share one key stream (4 in prefill, 1 in decode).
 // fp32_head_sum: keep the gate-weighted head sum in fp32 FMAs even where the tensor-core form
 // (FP8, four rows per block) is available.
+// head_sum: how the FP8 four-row configuration sums heads -- HEAD_SUM_I8: 8-bit integer contraction
+// on the tensor core in three-row blocks (scan_i8.cu, the default), HEAD_SUM_FP32: fp32 FMAs,
+// HEAD_SUM_BF16: bf16 contraction on the tensor core in place in the accumulator buffer.
+constexpr int HEAD_SUM_I8 = 0, HEAD_SUM_FP32 = 2, HEAD_SUM_BF16 = 3;
 cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_rows, int rows_per_block,
-                           const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum = false);
+                           const ScanScratch& s, int sms, cudaStream_t st, int head_sum = HEAD_SUM_I8);
+cudaError_t read_scan_prof(unsigned long long* out64_host);
+cudaError_t launch_scan_i8(const ScanOperands& op, const RowDesc* rows, int n_rows, const ScanScratch& s, int sms,
+                           cudaStream_t st);
 
 cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
                              const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum = false,
@@ -152,7 +159,7 @@ cudaError_t launch_wait_expiry_probe(int* status, unsigned long long limit_ns, c
 // Diagnostic: tensor-pipe / tensor-memory / hand-over timings of one SM (see debug_probe.cu); out = 256 slots.
 cudaError_t launch_mma_model_probe(long long* out, cudaStream_t st);
 // Diagnostic: rate at which all SMs together can pull the scan's 16 KB key tiles out of L2.
-cudaError_t launch_key_stream_probe(const void* keys, int n_keys, int ctas, int tiles, int stages, long long* out,
+cudaError_t launch_key_stream_probe(const void* keys, int n_keys, int ctas, int tiles, int stages, int mode, long long* out,
                                     cudaStream_t st);
 
 // The opt-in to more than 48 KB of dynamic shared memory is an attribute of (function, device):

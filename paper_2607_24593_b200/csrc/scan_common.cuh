@@ -1,0 +1,216 @@
+// Parts shared by the shared-scan kernels (scan_tc.cu, scan_i8.cu): the order in which a CTA
+// takes its row blocks, and the streaming select behind the scan (Eq. 6 / Eq. 7) -- survivor
+// queues between the warps that produce scores and one append warp per row, the row histogram
+// that keeps the running threshold, the row's candidate segment, and the final exact selection.
+#pragma once
+#include "kernels.h"
+#include "ptx.cuh"
+#include "segselect.cuh"
+
+namespace pivot {
+namespace scan {
+
+constexpr int TILE_KEYS = 128;
+constexpr int KS_SLOTS = 12;      // key-scale ring: deeper than (key stages + accumulator buffers)
+
+// Block sequence of one CTA: blocks sorted longest-first are dealt in snake order.
+struct BlockIter {
+  int n_blocks, G, cta, round;
+  __device__ BlockIter(int nb, int g, int c) : n_blocks(nb), G(g), cta(c), round(0) {}
+  __device__ int next() {   // block index, or -1
+    const int pos = (round & 1) ? (G - 1 - cta) : cta;
+    const long long d = (long long)round * G + pos;
+    ++round;
+    if (d >= n_blocks) return -1;
+    return n_blocks - 1 - (int)d;
+  }
+};
+
+// Key tiles a block of nrows_blk consecutive scan rows needs (its longest live row), and the
+// first key-tensor row of the block's sequence.
+__device__ __forceinline__ int block_tiles(const RowDesc* rows, int n_rows, int b, int nrows_blk, int* k_row0,
+                                           int* nv_max = nullptr) {
+  int mx = 0;
+  for (int r = 0; r < nrows_blk; ++r) {
+    const int ri = b * nrows_blk + r;
+    if (ri < n_rows) {
+      const int K = rows[ri].K;
+      const int nv = rows[ri].n_vis;
+      if (K > 0 && nv > mx) mx = nv;
+      if (r == 0) *k_row0 = rows[ri].k_row0;
+    }
+  }
+  if (nv_max) *nv_max = mx;
+  return (mx + TILE_KEYS - 1) / TILE_KEYS;
+}
+
+// Shared-memory state of the streaming select of a block of NROWS rows.
+template <int NROWS, int QD>
+struct SelectCtrl {
+  uint32_t rhist[NROWS][kSelBins];      // per row: histogram of every score appended so far
+  uint64_t sc_full[QD], sc_empty[QD];   // survivor queues: score warps -> append warps
+  alignas(16) unsigned long long q[QD][NROWS][4][32];   // [tile % QD][row][lane quarter]: packed entries
+  alignas(16) uint32_t qn[QD][NROWS][4];                // their counts
+  volatile uint32_t thr[NROWS];         // published append threshold of each row (only grows)
+  int rowcnt[NROWS];                    // end of a block: entries held in the row's segment
+  int rowbase[NROWS];                   // ... the row histogram's anchor
+  uint32_t rowthr[NROWS];               // ... and the row's final threshold
+  int abort_code;                       // device status to report besides a timed-out wait
+  SegSelSmem sel[NROWS];                // one per append warp (and per final selection)
+};
+
+// A score warp leaves the survivors of its 32 keys of row r in the tile's queue: compacted by one
+// vote, count beside them.  `take` must already include the causal cut and the threshold test.
+template <int NROWS, int QD>
+__device__ __forceinline__ void push_survivors(SelectCtrl<NROWS, QD>& s, int qb, int r, int lq, int lane, bool take,
+                                               uint32_t key, int s_key) {
+  const uint32_t m = __ballot_sync(0xffffffffu, take);
+  if (take) s.q[qb][r][lq][__popc(m & ((1u << lane) - 1u))] = make_entry(key, s_key);
+  if (lane == 0) s.qn[qb][r][lq] = (uint32_t)__popc(m);
+}
+
+// Score key -> histogram bin: 256 bins per octave (8 mantissa bits), 2048 bins anchored two
+// octaves above the row's first-tile maximum; keys outside land in the end bins.
+__device__ __forceinline__ int select_bin(uint32_t key, int base) {
+  const int b = (int)(key >> 15) - base;
+  return b < 0 ? 0 : (b > kSelBins - 1 ? kSelBins - 1 : b);
+}
+
+// The append warp of row r (one warp, all blocks of this CTA): counts the survivors of every tile
+// in the row histogram, moves them to the row's segment in the L2-resident scratch and keeps the
+// row's threshold fresh -- alone, without barriers.  `rdv` is the barrier it shares with the
+// warps that take the row's final selection at the end of a block.
+template <int NROWS, int QD>
+__device__ __noinline__ void append_role(SelectCtrl<NROWS, QD>& s, int r, int lane, const Team& tm, const Team& rdv,
+                                            const RowDesc* __restrict__ rows, int n_rows, int n_blocks,
+                                            const ScanScratch& sc, volatile int* abort_flag) {
+  SegSelSmem& sel = s.sel[r];
+  const int CAP = sc.cap;                        // entries of this row's candidate segment
+  entry_t* const seg = sc.cand64 + ((size_t)blockIdx.x * NROWS + r) * CAP;
+  uint32_t* const rhist = s.rhist[r];
+  // Lower bound on the K-th best score seen so far, read off the row histogram: the largest
+  // bin edge with at least K scores at or above it.  Returned as a key threshold t such that
+  // only keys > t can still belong to the top K.
+  auto hist_threshold = [&](int K, int base) -> uint32_t {
+    uint32_t b, need_in, pop;
+    if (!warp_hist_boundary<2>(rhist, (uint32_t)K, lane, &b, &need_in, &pop)) return 0u;
+    return b > 0 ? (((uint32_t)((int)b + base)) << 15) - 1u : 0u;
+  };
+  // The threshold is refreshed every CHK tiles; a tile adds at most TILE_KEYS entries, so a
+  // segment checked then always has room until the next check.
+  const int CHK = CAP / (2 * TILE_KEYS) < 32 ? (CAP / (2 * TILE_KEYS) > 0 ? CAP / (2 * TILE_KEYS) : 1) : 32;
+  const int headroom = TILE_KEYS * CHK;
+  BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
+  uint32_t it = 0;
+  for (int b = bi.next(); b >= 0; b = bi.next()) {
+    int k_row0 = 0;
+    const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0);
+    if (ntiles == 0) continue;
+    const int ri = b * NROWS + r;
+    const bool live = ri < n_rows && rows[ri].K > 0;
+    const int K = live ? rows[ri].K : 0;
+    int cnt = 0, base = 0;
+    uint32_t thr = 0;
+    for (int i = lane; i < kSelBins; i += 32) rhist[i] = 0;
+    __syncwarp();
+    for (int t = 0; t < ntiles; ++t, ++it) {
+      if (K > 0 && t > 0 && (t % CHK) == 0) {
+        const uint32_t th = hist_threshold(K, base);
+        thr = th > thr ? th : thr;
+        if (cnt + headroom > CAP) {
+          // nearly full: drop what fell below the threshold; if that is not enough (ties,
+          // adversarial order) compact exactly to the K best
+          const uint32_t tcur = thr;
+          cnt = seg_filter_inplace(seg, cnt, lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
+          if (cnt + headroom > CAP && cnt > K) {
+            entry_t cut;
+            cnt = seg_compact<false>(tm, sel, Seg{seg, cnt}, K, &cut);
+            thr = entry_key(cut) > thr ? entry_key(cut) : thr;
+          }
+        }
+        if (lane == 0) s.thr[r] = thr;
+      }
+      const int sb = it % QD;
+      (void)ptx::mbar_wait(&s.sc_full[sb], (it / QD) & 1, abort_flag);
+      const uint4 n4 = *reinterpret_cast<const uint4*>(&s.qn[sb][r][0]);
+      const uint32_t nq[4] = {n4.x, n4.y, n4.z, n4.w};
+      entry_t e[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) e[j] = (uint32_t)lane < nq[j] ? s.q[sb][r][j][lane] : kPadEntry;
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&s.sc_empty[sb]);
+      if (K <= 0) continue;                    // a dead row still takes part in the handshake
+      if (t == 0) {          // anchor the histogram range on the first tile's maximum
+        uint32_t mx = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) mx = entry_key(e[j]) > mx ? entry_key(e[j]) : mx;
+        mx = __reduce_max_sync(0xffffffffu, mx);
+        const int top = (int)(mx >> 15) + 512 - (kSelBins - 1);
+        base = top > 0 ? top : 0;
+      }
+      // Every entry that reaches the segment is counted: the ones the score warps dropped were
+      // at or below a valid threshold and can never reach a bin edge the threshold could still
+      // move to, so the counts that matter stay exact.
+      int p = cnt + lane;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if ((uint32_t)lane < nq[j]) {
+          atomicAdd(&rhist[select_bin(entry_key(e[j]), base)], 1u);
+          if (p < CAP) seg[p] = e[j];
+          else s.abort_code = DEV_CAND_OVERFLOW;
+        }
+        p += (int)nq[j];
+      }
+      cnt = min(cnt + (int)(nq[0] + nq[1] + nq[2] + nq[3]), CAP);
+    }
+    // ---- end of the block: hand the row to its final select, wait until it is done
+    if (lane == 0) { s.rowcnt[r] = cnt; s.rowbase[r] = base; s.rowthr[r] = thr; }
+    __syncwarp();
+    rdv.sync();
+    if (lane == 0) s.thr[r] = 0u;             // the next block starts from scratch (read after the barrier below)
+    rdv.sync();
+  }
+}
+
+// Final exact selection of row r of block b by a team of four warps (128 threads; warp wq of the
+// team takes the wq-th quarter of the row's segment): the append warp has counted every entry it
+// holds, so the row histogram is exact and one pass over the segment suffices; a boundary bin too
+// crowded to rank takes the general path.  Pads the row with -1 and copies it to the other
+// members of a Reuse group.  Call between the two `rdv` barriers of the append warp.
+template <int NROWS, int QD>
+__device__ __noinline__ void final_select_row(SelectCtrl<NROWS, QD>& s, const Team& tm, int r, int K, const RowDesc& rd,
+                                                 const ScanScratch& sc) {
+  if (K <= 0) return;
+  const int tt = tm.tid, lane = tt & 31, wq = tt >> 5;
+  SegSelSmem& sel = s.sel[r];               // the row's append warp is idle now
+  entry_t* const seg = sc.cand64 + ((size_t)blockIdx.x * NROWS + r) * sc.cap;
+  const int total = s.rowcnt[r];
+  const int rbase = s.rowbase[r];
+  const int lo = (int)(((long long)total * wq) >> 2), hi = (int)(((long long)total * (wq + 1)) >> 2);
+  int mine = hi - lo;                        // this warp's slice of the row segment
+  auto key_bin = [rbase](uint32_t key) { return select_bin(key, rbase); };
+  int n_valid = seg_emit_hist(tm, sel, Seg{seg + lo, mine}, s.rhist[r], key_bin, rd.out, rd.out_score, K);
+  if (n_valid < 0) {
+    const uint32_t tcur = s.rowthr[r];
+    mine = seg_filter_inplace(seg + lo, mine, lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
+    tm.sync();
+    if (tt == 0) sel.total = 0;
+    tm.sync();
+    if (lane == 0) atomicAdd(&sel.total, (uint32_t)mine);
+    tm.sync();
+    n_valid = seg_emit<false>(tm, sel, Seg{seg + lo, mine}, (int)sel.total, rd.out, rd.out_score, K);
+  }
+  for (int i = n_valid + tt; i < K; i += 128) {
+    rd.out[i] = -1;
+    if (rd.out_score) rd.out_score[i] = -INFINITY;
+  }
+  tm.sync();
+  for (int rr = 1; rr < rd.out_rows; ++rr)
+    for (int i = tt; i < K; i += 128) {
+      rd.out[(size_t)rr * rd.out_stride + i] = rd.out[i];
+      if (rd.out_score) rd.out_score[(size_t)rr * rd.out_stride + i] = rd.out_score[i];
+    }
+}
+
+}  // namespace scan
+}  // namespace pivot

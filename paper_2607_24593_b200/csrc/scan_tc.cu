@@ -34,14 +34,17 @@
 
 #include "kernels.h"
 #include "ptx.cuh"
+#include "scan_common.cuh"
 #include "segselect.cuh"
 
 namespace pivot {
 namespace {
 
-constexpr int TILE_KEYS = 128;
+using scan::TILE_KEYS;
+using scan::KS_SLOTS;
+using scan::BlockIter;
+using scan::block_tiles;
 constexpr int MAX_STAGES = 8;
-constexpr int KS_SLOTS = 12;      // key-scale ring: deeper than (key stages + accumulator buffers)
 constexpr int QDEPTH = 4;         // survivor-queue buffers between the score warps and the append warps
 
 // EPI: 1 = the gate-weighted head sum runs on the tensor core where the configuration allows it
@@ -90,21 +93,12 @@ struct Ctrl {
   uint64_t a_ready[2], s_ready[2], w_ready;      // MMA2 handshakes (see the kernel)
   alignas(128) float ks[KS_SLOTS][TILE_KEYS];   // key scales of the tiles in flight (TMA destination)
   alignas(16) float w[4][kHeads];       // effective gates of the block's rows (read as float4)
-  uint32_t rhist[NROWS][kSelBins];      // per row: histogram of every score seen so far
   uint64_t full[MAX_STAGES], empty[MAX_STAGES];
   uint64_t q_full[2], q_empty[2], tmem_full[2], tmem_empty[2];
   uint64_t ks_full[KS_SLOTS];
-  uint64_t sc_full[QD], sc_empty[QD];     // survivor queues: score warps -> append warps
-  alignas(16) unsigned long long q[QD][NROWS][4][32];   // [tile % QD][row][lane quarter]: packed entries
-  alignas(16) uint32_t qn[QD][NROWS][4];                // their counts
-  volatile uint32_t thr[NROWS];         // published append threshold of each row (only grows)
-  int rowcnt[NROWS];                    // end of a block: entries held in the row's segment
-  int rowbase[NROWS];                   // ... the row histogram's anchor
-  uint32_t rowthr[NROWS];               // ... and the row's final threshold
   uint32_t tmem_base;
   int abort;
-  int abort_code;         // device status to report besides a timed-out wait
-  SegSelSmem sel[NROWS];  // one per select warp
+  scan::SelectCtrl<NROWS, QD> s;        // streaming select: queues, row histograms, thresholds
 };
 
 template <int DT, int NROWS, int EPI = 1>
@@ -114,38 +108,6 @@ constexpr size_t smem_bytes() {
 }
 static_assert(smem_bytes<DT_FP8, 4, 1>() <= 232448 && smem_bytes<DT_FP8, 4, 0>() <= 232448 &&
               smem_bytes<DT_BF16, 4>() <= 232448, "shared memory budget");
-
-// Block sequence of one CTA: blocks sorted longest-first are dealt in snake order.
-struct BlockIter {
-  int n_blocks, G, cta, round;
-  __device__ BlockIter(int nb, int g, int c) : n_blocks(nb), G(g), cta(c), round(0) {}
-  __device__ int next() {   // block index, or -1
-    const int pos = (round & 1) ? (G - 1 - cta) : cta;
-    const long long d = (long long)round * G + pos;
-    ++round;
-    if (d >= n_blocks) {
-      // a partial last round can still hold a block for this CTA on the other snake direction
-      return -1;
-    }
-    return n_blocks - 1 - (int)d;
-  }
-};
-
-__device__ __forceinline__ int block_tiles(const RowDesc* rows, int n_rows, int b, int nrows_blk, int* k_row0,
-                                           int* nv_max = nullptr) {
-  int mx = 0;
-  for (int r = 0; r < nrows_blk; ++r) {
-    const int ri = b * nrows_blk + r;
-    if (ri < n_rows) {
-      const int K = rows[ri].K;
-      const int nv = rows[ri].n_vis;
-      if (K > 0 && nv > mx) mx = nv;
-      if (r == 0) *k_row0 = rows[ri].k_row0;
-    }
-  }
-  if (nv_max) *nv_max = mx;
-  return (mx + TILE_KEYS - 1) / TILE_KEYS;
-}
 
 template <int DT, int NROWS, int EPI>
 __global__ void __launch_bounds__(Cfg<DT, NROWS, EPI>::THREADS, 1)
@@ -186,12 +148,12 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     ptx::mbar_init(&ct.w_ready, 1);
     for (int i = 0; i < KS_SLOTS; ++i) ptx::mbar_init(&ct.ks_full[i], 1);
     for (int i = 0; i < QD; ++i) {
-      ptx::mbar_init(&ct.sc_full[i], C::SC_FULL_ARRIVALS);
-      ptx::mbar_init(&ct.sc_empty[i], C::SEL_WARPS);
+      ptx::mbar_init(&ct.s.sc_full[i], C::SC_FULL_ARRIVALS);
+      ptx::mbar_init(&ct.s.sc_empty[i], C::SEL_WARPS);
     }
     ct.abort = 0;
-    ct.abort_code = 0;
-    for (int r = 0; r < NROWS; ++r) ct.thr[r] = 0u;
+    ct.s.abort_code = 0;
+    for (int r = 0; r < NROWS; ++r) ct.s.thr[r] = 0u;
     ptx::fence_barrier_init();
   }
   if (warp == 1) {
@@ -335,7 +297,6 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     const int tt = wq * 32 + lane;                 // rank inside the team (0..127)
     const Team tm{tt, 128, 1 + team};
     const Team rdv{0, C::RDV_THREADS, 7 + team};   // this team and the append warps of its rows
-    const uint32_t lt_mask = (1u << lane) - 1u;
     BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
     uint32_t it = 0;
     // A failed wait never changes this role's control flow (the team barriers below must stay
@@ -455,18 +416,15 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
             const int qb = it % QD;
-            (void)ptx::mbar_wait(&ct.sc_empty[qb], ((it / QD) & 1) ^ 1, abort_flag);
+            (void)ptx::mbar_wait(&ct.s.sc_empty[qb], ((it / QD) & 1) ^ 1, abort_flag);
             const int s_key = t * TILE_KEYS + key_in_tile;
 #pragma unroll
             for (int r = 0; r < NROWS; ++r) {
               const uint32_t key = score_to_key((__uint_as_float(sv[r]) + __uint_as_float(sv[4 + r])) * ksv);
-              const bool take = s_key < nv4[r] && key > ct.thr[r];
-              const uint32_t m = __ballot_sync(0xffffffffu, take);
-              if (take) ct.q[qb][r][lq][__popc(m & lt_mask)] = make_entry(key, s_key);
-              if (lane == 0) ct.qn[qb][r][lq] = (uint32_t)__popc(m);
+              scan::push_survivors(ct.s, qb, r, lq, lane, s_key < nv4[r] && key > ct.s.thr[r], key, s_key);
             }
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&ct.sc_full[qb]);
+            if (lane == 0) ptx::mbar_arrive(&ct.s.sc_full[qb]);
           }
         }
       } else
@@ -528,19 +486,16 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
         // ---- survivors of this warp's 32 keys (key scale applied, Appendix A) go to the row queues
         const int qb = it % QD;
-        (void)ptx::mbar_wait(&ct.sc_empty[qb], ((it / QD) & 1) ^ 1, abort_flag);
+        (void)ptx::mbar_wait(&ct.s.sc_empty[qb], ((it / QD) & 1) ^ 1, abort_flag);
         const int s_key = t * TILE_KEYS + key_in_tile;
 #pragma unroll
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
           const int r = team * C::ROWS_PER_TEAM + rl;
           const uint32_t key = score_to_key(C::FP8 ? score[rl] * ksv : score[rl]);
-          const bool take = s_key < n_vis[rl] && key > ct.thr[r];
-          const uint32_t m = __ballot_sync(0xffffffffu, take);
-          if (take) ct.q[qb][r][lq][__popc(m & lt_mask)] = make_entry(key, s_key);
-          if (lane == 0) ct.qn[qb][r][lq] = (uint32_t)__popc(m);
+          scan::push_survivors(ct.s, qb, r, lq, lane, s_key < n_vis[rl] && key > ct.s.thr[r], key, s_key);
         }
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&ct.sc_full[qb]);
+        if (lane == 0) ptx::mbar_arrive(&ct.s.sc_full[qb]);
       }
       // ---- end of the block: the team takes the final exact select of its rows.  The append
       //      warps have counted every entry they hold, so the row histogram is exact and one pass
@@ -550,140 +505,15 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
         const int r = team * C::ROWS_PER_TEAM + rl;
         const int ri = b * NROWS + r;
-        const int K = Ksel[rl];
-        if (K <= 0) continue;
-        const RowDesc rd = rows[ri];
-        SegSelSmem& sel = ct.sel[r];               // the row's append warp is idle now
-        entry_t* const seg = sc.cand64 + ((size_t)blockIdx.x * NROWS + r) * sc.cap;
-        const int total = ct.rowcnt[r];
-        const int rbase = ct.rowbase[r];
-        const int lo = (int)(((long long)total * wq) >> 2), hi = (int)(((long long)total * (wq + 1)) >> 2);
-        int mine = hi - lo;                        // this warp's slice of the row segment
-        auto key_bin = [rbase](uint32_t key) {
-          const int bb = (int)(key >> 15) - rbase;
-          return bb < 0 ? 0 : (bb > kSelBins - 1 ? kSelBins - 1 : bb);
-        };
-        int n_valid = seg_emit_hist(tm, sel, Seg{seg + lo, mine}, ct.rhist[r], key_bin, rd.out, rd.out_score, K);
-        if (n_valid < 0) {
-          const uint32_t tcur = ct.rowthr[r];
-          mine = seg_filter_inplace(seg + lo, mine, lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
-          tm.sync();
-          if (tt == 0) sel.total = 0;
-          tm.sync();
-          if (lane == 0) atomicAdd(&sel.total, (uint32_t)mine);
-          tm.sync();
-          n_valid = seg_emit<false>(tm, sel, Seg{seg + lo, mine}, (int)sel.total, rd.out, rd.out_score, K);
-        }
-        for (int i = n_valid + tt; i < K; i += 128) {
-          rd.out[i] = -1;
-          if (rd.out_score) rd.out_score[i] = -INFINITY;
-        }
-        tm.sync();
-        for (int rr = 1; rr < rd.out_rows; ++rr)
-          for (int i = tt; i < K; i += 128) {
-            rd.out[(size_t)rr * rd.out_stride + i] = rd.out[i];
-            if (rd.out_score) rd.out_score[(size_t)rr * rd.out_stride + i] = rd.out_score[i];
-          }
+        if (Ksel[rl] > 0) scan::final_select_row(ct.s, tm, r, Ksel[rl], rows[ri], sc);
       }
       rdv.sync();                                  // rows' histograms and segments may be reused
     }
   } else {
     // ------------------------------------------------------------------ append warps: one row each
     const int r = warp - 2 - C::EPI_WARPS;
-    const Team tm{lane, 32, 3 + r};
-    const Team rdv{0, C::RDV_THREADS, 7 + r / C::ROWS_PER_TEAM};
-    SegSelSmem& sel = ct.sel[r];
-    const int CAP = sc.cap;                        // entries of this row's candidate segment
-    entry_t* const seg = sc.cand64 + ((size_t)blockIdx.x * NROWS + r) * CAP;
-    uint32_t* const rhist = ct.rhist[r];
-    // Score key -> histogram bin: 256 bins per octave (8 mantissa bits), 2048 bins anchored two
-    // octaves above the row's first-tile maximum; keys outside land in the end bins.
-    auto key_bin = [](uint32_t key, int base) {
-      const int b = (int)(key >> 15) - base;
-      return b < 0 ? 0 : (b > kSelBins - 1 ? kSelBins - 1 : b);
-    };
-    // Lower bound on the K-th best score seen so far, read off the row histogram: the largest
-    // bin edge with at least K scores at or above it.  Returned as a key threshold t such that
-    // only keys > t can still belong to the top K.
-    auto hist_threshold = [&](int K, int base) -> uint32_t {
-      uint32_t b, need_in, pop;
-      if (!warp_hist_boundary<2>(rhist, (uint32_t)K, lane, &b, &need_in, &pop)) return 0u;
-      return b > 0 ? (((uint32_t)((int)b + base)) << 15) - 1u : 0u;
-    };
-    // The threshold is refreshed every CHK tiles; a tile adds at most TILE_KEYS entries, so a
-    // segment checked then always has room until the next check.
-    const int CHK = CAP / (2 * TILE_KEYS) < 32 ? (CAP / (2 * TILE_KEYS) > 0 ? CAP / (2 * TILE_KEYS) : 1) : 32;
-    const int headroom = TILE_KEYS * CHK;
-    BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
-    uint32_t it = 0;
-    for (int b = bi.next(); b >= 0; b = bi.next()) {
-      int k_row0 = 0;
-      const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0);
-      if (ntiles == 0) continue;
-      const int ri = b * NROWS + r;
-      const bool live = ri < n_rows && rows[ri].K > 0;
-      const int K = live ? rows[ri].K : 0;
-      int cnt = 0, base = 0;
-      uint32_t thr = 0;
-      for (int i = lane; i < kSelBins; i += 32) rhist[i] = 0;
-      __syncwarp();
-      for (int t = 0; t < ntiles; ++t, ++it) {
-        if (K > 0 && t > 0 && (t % CHK) == 0) {
-          const uint32_t th = hist_threshold(K, base);
-          thr = th > thr ? th : thr;
-          if (cnt + headroom > CAP) {
-            // nearly full: drop what fell below the threshold; if that is not enough (ties,
-            // adversarial order) compact exactly to the K best
-            const uint32_t tcur = thr;
-            cnt = seg_filter_inplace(seg, cnt, lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
-            if (cnt + headroom > CAP && cnt > K) {
-              entry_t cut;
-              cnt = seg_compact<false>(tm, sel, Seg{seg, cnt}, K, &cut);
-              thr = entry_key(cut) > thr ? entry_key(cut) : thr;
-            }
-          }
-          if (lane == 0) ct.thr[r] = thr;
-        }
-        const int sb = it % QD;
-        (void)ptx::mbar_wait(&ct.sc_full[sb], (it / QD) & 1, abort_flag);
-        const uint4 n4 = *reinterpret_cast<const uint4*>(&ct.qn[sb][r][0]);
-        const uint32_t nq[4] = {n4.x, n4.y, n4.z, n4.w};
-        entry_t e[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) e[j] = (uint32_t)lane < nq[j] ? ct.q[sb][r][j][lane] : kPadEntry;
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&ct.sc_empty[sb]);
-        if (K <= 0) continue;                    // a dead row still takes part in the handshake
-        if (t == 0) {          // anchor the histogram range on the first tile's maximum
-          uint32_t mx = 0;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) mx = entry_key(e[j]) > mx ? entry_key(e[j]) : mx;
-          mx = __reduce_max_sync(0xffffffffu, mx);
-          const int top = (int)(mx >> 15) + 512 - (kSelBins - 1);
-          base = top > 0 ? top : 0;
-        }
-        // Every entry that reaches the segment is counted: the ones the score warps dropped were
-        // at or below a valid threshold and can never reach a bin edge the threshold could still
-        // move to, so the counts that matter stay exact.
-        int p = cnt + lane;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          if ((uint32_t)lane < nq[j]) {
-            atomicAdd(&rhist[key_bin(entry_key(e[j]), base)], 1u);
-            if (p < CAP) seg[p] = e[j];
-            else ct.abort_code = DEV_CAND_OVERFLOW;
-          }
-          p += (int)nq[j];
-        }
-        cnt = min(cnt + (int)(nq[0] + nq[1] + nq[2] + nq[3]), CAP);
-      }
-      // ---- end of the block: hand the row to the team's final select, wait until it is done
-      if (lane == 0) { ct.rowcnt[r] = cnt; ct.rowbase[r] = base; ct.rowthr[r] = thr; }
-      __syncwarp();
-      rdv.sync();
-      if (lane == 0) ct.thr[r] = 0u;             // the next block starts from scratch (read after the barrier below)
-      rdv.sync();
-    }
+    scan::append_role(ct.s, r, lane, Team{lane, 32, 3 + r}, Team{0, C::RDV_THREADS, 7 + r / C::ROWS_PER_TEAM}, rows, n_rows,
+                      n_blocks, sc, abort_flag);
   }
   // ------------------------------------------------------------------ teardown
   ptx::tc_fence_before();
@@ -691,7 +521,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
   ptx::tc_fence_after();
   if (warp == 1) ptx::tmem_dealloc(tmem_base, C::TMEM_COLS);
   if (threadIdx.x == 0 && ct.abort) set_status(sc.status, DEV_WAIT_EXPIRED);
-  if (threadIdx.x == 0 && ct.abort_code) set_status(sc.status, ct.abort_code);
+  if (threadIdx.x == 0 && ct.s.abort_code) set_status(sc.status, ct.s.abort_code);
 }
 
 // ---------------------------------------------------------------------------- host side
@@ -759,8 +589,10 @@ bool make_scale_map(CUtensorMap* m, const float* base, long long n) {
 
 
 cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_rows, int rows_per_block,
-                           const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum) {
+                           const ScanScratch& s, int sms, cudaStream_t st, int head_sum) {
   if (n_rows <= 0) return cudaSuccess;
+  if (op.dtype == DT_FP8 && rows_per_block == 4 && head_sum == HEAD_SUM_I8) return launch_scan_i8(op, rows, n_rows, s, sms, st);
+  const bool fp32_head_sum = head_sum == HEAD_SUM_FP32;
   CUtensorMap mk, mq0, mq1, mks;
   memset(&mks, 0, sizeof(mks));
   if (op.dtype == DT_FP8 && !make_scale_map(&mks, op.kscale, op.k_rows)) return cudaErrorInvalidValue;
