@@ -89,15 +89,11 @@ typedef struct pivot_tensor {
  *   dbg_cand_scores optional [n_groups, c] fp32: proxy score (Eq. 5) of each dbg_cand entry.
  *   workspace     scratch of at least pivot_workspace_bytes(...) bytes, 256-byte aligned.
  *   impl          0: tensor-core kernels (tcgen05; the product path).  In FP8 prefill the shared
- *                 scan also takes the gate-weighted head sum of Eq. 5 on the tensor core, as an
- *                 8-bit integer contraction: per key and row the ReLU values are scaled to their
- *                 largest head term and rounded to unsigned bytes, the gates enter as three signed
- *                 base-128 digits, the sums are exact integers -- a relative score error of about
- *                 1e-3, inside the FP8 acceptance band.
- *                 2: the same scan with that head sum in fp32 FMAs (slower; the scores then
+ *                 scan also takes the gate-weighted head sum of Eq. 5 on the tensor core: ReLU
+ *                 values rounded to bf16, gates carried as two bf16 terms, fp32 accumulation -- a
+ *                 relative score error of about 2^-9, inside the FP8 acceptance band.
+ *                 2: the same kernels with that head sum in fp32 FMAs (slower; the scores then
  *                 differ from exact arithmetic by fp32 summation order only).
- *                 3: the same scan with the head sum as a bf16 contraction on the tensor core
- *                 (ReLU values rounded to bf16, gates as two bf16 terms; error about 2^-9).
  *                 1: the plain CUDA-core kernels that compute the same thing one key per thread
  *                 -- a slow on-device cross-check, not a fallback: nothing selects it
  *                 automatically.
@@ -306,14 +302,6 @@ int pivot_debug_wait_expiry(unsigned long long limit_ns, pivot_stream_t stream);
  * measures time only.
  */
 int pivot_debug_mma_model(long long* out_device, pivot_stream_t stream);
-
-/*
- * Diagnostic (no counterpart in the paper): cycle accounting of the FP8 shared scan's roles (waits
- * per barrier, busy time per unit) on its first CTA since the previous call, 64 counters into HOST
- * memory.  All zeros unless the library was built with PIVOT_NVCC_FLAGS=-DPIVOT_PROF (the counters
- * cost time, so the default build leaves them out).  Synchronise the stream first.
- */
-int pivot_debug_scan_profile(unsigned long long* out64_host);
 
 /*
  * Diagnostic (no counterpart in the paper): `ctas` CTAs each pull `tiles` consecutive 16 KB key

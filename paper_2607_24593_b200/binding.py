@@ -26,7 +26,7 @@ SYMBOLS = [
     "pivot_index_decode", "pivot_index_decode_ex", "pivot_index_decode_paged", "dense_index", "dense_index_ex", "dense_index_static",
     "pivot_prefill_host_arena_bytes", "pivot_index_prefill_host", "pivot_device_status",
     "pivot_stage_timing", "pivot_stage_times", "pivot_launch_count_reset", "pivot_status_str", "pivot_last_cuda_error",
-    "dense_index_decode", "dense_index_decode_ex", "pivot_debug_wait_expiry", "pivot_debug_mma_model", "pivot_debug_key_stream", "pivot_debug_scan_profile",
+    "dense_index_decode", "dense_index_decode_ex", "pivot_debug_wait_expiry", "pivot_debug_mma_model", "pivot_debug_key_stream",
 ]
 DEV_OK, DEV_WAIT_EXPIRED, DEV_CAND_OVERFLOW, DEV_BAD_POS, DEV_BOUNDS = 0, 1, 2, 3, 4
 
@@ -113,7 +113,7 @@ def _stream(stream) -> int:
     return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
 
 
-IMPL_TENSOR_CORE, IMPL_CUDA_CORE, IMPL_TENSOR_CORE_FP32_HEAD_SUM, IMPL_TENSOR_CORE_BF16_HEAD_SUM = 0, 1, 2, 3
+IMPL_TENSOR_CORE, IMPL_CUDA_CORE, IMPL_TENSOR_CORE_FP32_HEAD_SUM = 0, 1, 2
 
 
 def _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl=0, rows=None, W=0) -> pivot_opts:
@@ -283,14 +283,6 @@ def pivot_debug_mma_model(stream=None) -> dict:
             d["traffic warps: clk per 256-column pass"] = [x for x in v[ph * 32 + 16: ph * 32 + 24] if x]
         res[pname] = d
     return res
-
-
-def pivot_debug_scan_profile() -> list:
-    """Cycle counters of the FP8 scan's first CTA (zeros unless built with -DPIVOT_PROF)."""
-    torch.cuda.synchronize()
-    out = (C.c_ulonglong * 64)()
-    _check(lib.pivot_debug_scan_profile(out))
-    return [int(v) for v in out]
 
 
 def pivot_debug_key_stream(n_keys=131072, ctas=148, tiles=2048, stages=4, mode=0, stream=None) -> dict:

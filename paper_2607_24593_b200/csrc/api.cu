@@ -246,7 +246,7 @@ int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, i
   } else {
     ScanOperands op{kc->data, L, kc->scale, q->data, L, ws.proxy_q, p.n_proxy, q->dtype};
     if ((rc = check_cuda(launch_scan_tc(op, ws.rows, p.n_dense + p.n_proxy, 4, tc_scratch(ws), sm_count(), st,
-                                        o ? o->impl : HEAD_SUM_I8))))
+                                        o && o->impl == 2))))
       return rc;
   }
   mark(3, st);
@@ -289,7 +289,7 @@ int pivot_index_prefill_ex(const pivot_tensor* q, const float* w, const pivot_te
   int rc = check_common(q, w, kcache, H_I, d, c, k, mode, out_idx);
   if (rc) return rc;
   if (L < 1 || g < 1) return PIVOT_ERR_INVALID_ARG;
-  if (opts && (opts->pool < 0 || opts->pool > 2 || opts->impl < 0 || opts->impl > 3))
+  if (opts && (opts->pool < 0 || opts->pool > 2 || opts->impl < 0 || opts->impl > 2))
     return PIVOT_ERR_INVALID_ARG;
   return run_prefill(q, w, kcache, L, g, c, k, mode, false, out_idx, (cudaStream_t)stream, opts);
 }
@@ -475,11 +475,6 @@ int pivot_debug_wait_expiry(unsigned long long limit_ns, pivot_stream_t stream) 
   int rc = check_cuda(cudaMemsetAsync(status, 0, sizeof(int), st));
   if (rc) return rc;
   return check_cuda(launch_wait_expiry_probe(status, limit_ns, st));
-}
-
-int pivot_debug_scan_profile(unsigned long long* out64_host) {
-  if (!out64_host) return PIVOT_ERR_INVALID_ARG;
-  return check_cuda(read_scan_prof(out64_host));
 }
 
 int pivot_debug_mma_model(long long* out_device, pivot_stream_t stream) {

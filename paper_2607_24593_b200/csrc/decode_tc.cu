@@ -567,7 +567,7 @@ cudaError_t launch_scan(const CUtensorMap& mk, const CUtensorMap& mq, const CUte
 }  // namespace
 
 bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows);
-bool make_scale_map(CUtensorMap* m, const float* base, long long n);
+bool make_scale_map(CUtensorMap* m, const float* base, long long n, int box);
 
 size_t decode_fast_bytes(int B, int Lmax, int g, int c) {
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
@@ -604,7 +604,7 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   if (e != cudaSuccess) return e;
   CUtensorMap mk, mq, mks;
   memset(&mks, 0, sizeof(mks));
-  if (d.dtype == DT_FP8 && !make_scale_map(&mks, d.kscale, d.k_rows)) return cudaErrorInvalidValue;
+  if (d.dtype == DT_FP8 && !make_scale_map(&mks, d.kscale, d.k_rows, TILE_KEYS)) return cudaErrorInvalidValue;
   if (!make_operand_map(&mk, d.kc, d.k_rows, d.dtype, TILE_KEYS) ||
       !make_operand_map(&mq, d.proxy_q, (long long)d.B * kHeads, d.dtype, kHeads))
     return cudaErrorInvalidValue;

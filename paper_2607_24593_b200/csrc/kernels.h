@@ -120,15 +120,10 @@ struct ScanOperands {
 // rows_per_block consecutive scan rows share one key stream (4 in prefill, 1 in decode).
 // fp32_head_sum: keep the gate-weighted head sum in fp32 FMAs even where the tensor-core form
 // (FP8, four rows per block) is available.
-// head_sum: how the FP8 four-row configuration sums heads -- HEAD_SUM_I8: 8-bit integer contraction
-// on the tensor core in three-row blocks (scan_i8.cu, the default), HEAD_SUM_FP32: fp32 FMAs,
-// HEAD_SUM_BF16: bf16 contraction on the tensor core in place in the accumulator buffer.
-constexpr int HEAD_SUM_I8 = 0, HEAD_SUM_FP32 = 2, HEAD_SUM_BF16 = 3;
+// fp32_head_sum: keep the gate-weighted head sum in fp32 FMAs even where the tensor-core form
+// (FP8, four rows per block) is available.
 cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_rows, int rows_per_block,
-                           const ScanScratch& s, int sms, cudaStream_t st, int head_sum = HEAD_SUM_I8);
-cudaError_t read_scan_prof(unsigned long long* out64_host);
-cudaError_t launch_scan_i8(const ScanOperands& op, const RowDesc* rows, int n_rows, const ScanScratch& s, int sms,
-                           cudaStream_t st);
+                           const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum = false);
 
 cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
                              const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum = false,

@@ -44,14 +44,18 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                : "memory");
 }
+// One try: the hardware may park the thread until the phase completes or `kTryWaitHintNs` have
+// passed, so a waiting warp leaves its scheduler's issue slots to the warps that have work
+// (a hot polling loop of three waiting warps costs the fourth one three quarters of its issue rate).
+constexpr uint32_t kTryWaitHintNs = 20000u;
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.b32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kTryWaitHintNs)
       : "memory");
   return ok != 0;
 }
@@ -246,12 +250,6 @@ __device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint32_t (&v
         "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
       : "memory");
 }
-// registers -> TMEM, 8 consecutive columns.
-__device__ __forceinline__ void tmem_st_32x8(uint32_t taddr, const uint32_t (&v)[8]) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-               ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
-               : "memory");
-}
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // TMEM -> registers, 8 consecutive columns.
 __device__ __forceinline__ void tmem_ld_32x8(uint32_t taddr, uint32_t (&r)[8]) {
@@ -277,63 +275,5 @@ __device__ __forceinline__ void tc_mma_a_tmem_bf16(uint32_t d_tmem, uint32_t a_t
 __device__ __forceinline__ void tmem_wait_ld() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
-// TMEM -> registers, 16 consecutive columns.
-__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr) : "memory");
-}
-// Instruction descriptor of the 8-bit integer kind: s32 += u8 (A) x s8 (B), both K-major.
-__host__ __device__ constexpr uint32_t make_idesc_u8s8(uint32_t M, uint32_t N) {
-  return (2u << 4) | (0u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
-}
-// MMA of the 8-bit integer kind with the A operand in tensor memory (four K elements per column,
-// the lowest k in the low byte).
-__device__ __forceinline__ void tc_mma_a_tmem_i8(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                                 uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-  float d;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
-// max(x * scale, 0) of four floats, rounded to fp16 and packed in pairs (x0 in the low half of lo).
-__device__ __forceinline__ void relu_scale_pack_f16x2(float x0, float x1, float x2, float x3, float scale, uint32_t& lo,
-                                                      uint32_t& hi) {
-  asm("{\n\t.reg .b64 p, q, o0, o1;\n\t.reg .f32 a0, a1, a2, a3;\n\t"
-      "mov.b64 q, {%6, %6};\n\t"
-      "mov.b64 p, {%2, %3};\n\tmul.rn.f32x2 o0, p, q;\n\t"
-      "mov.b64 p, {%4, %5};\n\tmul.rn.f32x2 o1, p, q;\n\t"
-      "mov.b64 {a0, a1}, o0;\n\tmov.b64 {a2, a3}, o1;\n\t"
-      "cvt.rn.relu.f16x2.f32 %0, a1, a0;\n\tcvt.rn.relu.f16x2.f32 %1, a3, a2;\n\t}"
-      : "=r"(lo), "=r"(hi)
-      : "f"(x0), "f"(x1), "f"(x2), "f"(x3), "f"(scale));
-}
-__device__ __forceinline__ uint32_t max_f16x2(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("max.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-// Two packed pairs of non-negative fp16 values h -> four unsigned 8-bit codes round(h * s), packed
-// with the low half of `lo` in the low byte: h * s + 1024 is formed in fp16, where [1024, 2048) has
-// unit spacing, so the low byte of each half is the rounded code.  Needs h * s < 255.5.
-__device__ __forceinline__ uint32_t quant4_u8_f16(uint32_t lo, uint32_t hi, uint32_t s2) {
-  uint32_t r;
-  asm("{\n\t.reg .b32 z0, z1;\n\t"
-      "fma.rn.f16x2 z0, %1, %3, %4;\n\tfma.rn.f16x2 z1, %2, %3, %4;\n\t"
-      "prmt.b32 %0, z0, z1, 0x6420;\n\t}"
-      : "=r"(r)
-      : "r"(lo), "r"(hi), "r"(s2), "r"(0x64006400u));
-  return r;
-}
-
 }  // namespace ptx
 }  // namespace pivot

@@ -574,28 +574,26 @@ bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtyp
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// 1-D map over an fp32 scale array; box = 128 scales.
-bool make_scale_map(CUtensorMap* m, const float* base, long long n) {
+// 1-D map over an fp32 scale array; box = `box` scales (a TMA box holds at most 256 elements per dimension).
+bool make_scale_map(CUtensorMap* m, const float* base, long long n, int box) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[1] = {(cuuint64_t)n};
   cuuint64_t strides[1] = {0};
-  cuuint32_t box[1] = {(cuuint32_t)TILE_KEYS};
+  cuuint32_t boxd[1] = {(cuuint32_t)box};
   cuuint32_t estr[1] = {1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 1, (void*)base, dims, strides, box, estr,
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 1, (void*)base, dims, strides, boxd, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 
 cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_rows, int rows_per_block,
-                           const ScanScratch& s, int sms, cudaStream_t st, int head_sum) {
+                           const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum) {
   if (n_rows <= 0) return cudaSuccess;
-  if (op.dtype == DT_FP8 && rows_per_block == 4 && head_sum == HEAD_SUM_I8) return launch_scan_i8(op, rows, n_rows, s, sms, st);
-  const bool fp32_head_sum = head_sum == HEAD_SUM_FP32;
   CUtensorMap mk, mq0, mq1, mks;
   memset(&mks, 0, sizeof(mks));
-  if (op.dtype == DT_FP8 && !make_scale_map(&mks, op.kscale, op.k_rows)) return cudaErrorInvalidValue;
+  if (op.dtype == DT_FP8 && !make_scale_map(&mks, op.kscale, op.k_rows, TILE_KEYS)) return cudaErrorInvalidValue;
   if (!make_operand_map(&mk, op.kc, op.k_rows, op.dtype, TILE_KEYS) ||
       !make_operand_map(&mq0, op.q, (long long)op.q_rows * kHeads, op.dtype, kHeads) ||
       !make_operand_map(&mq1, op.proxy_q, (long long)(op.proxy_rows > 0 ? op.proxy_rows : 1) * kHeads, op.dtype, kHeads))

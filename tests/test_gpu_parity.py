@@ -45,18 +45,13 @@ def test_prefill_small_full_parity(pv, gu, dtype, mode, seed):
     # with fp32 head sums; the FP8 scan sums heads on the tensor core with bf16 ReLU values, so keys
     # within ~2^-9 of the cut may trade places (inside the band) in a good part of the rows.
     assert t.exact_rows >= (0.5 if dtype == "fp8" else 0.95) * t.rows
-    assert t.max_score_err <= (0.3 if dtype == "fp8" else 1.0)
-    if dtype == "fp8":       # the fp32 and bf16 head-sum forms of the scan
+    assert t.max_score_err <= (0.25 if dtype == "fp8" else 1.0)
+    if dtype == "fp8":       # the fp32 head-sum form of the same kernels
         out, sc, cand, cs = gu.run_prefill(x, g=g, c=c, k=k, mode=mode, impl=pv.IMPL_TENSOR_CORE_FP32_HEAD_SUM)
         t = acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=None, out_idx=out,
                               out_scores=sc, cand=cand, cand_scores=cs)
         _report(f"prefill fp8 (fp32 head sum) mode={mode} seed={seed}", t)
         assert t.exact_rows >= 0.95 * t.rows
-        out, sc, cand, cs = gu.run_prefill(x, g=g, c=c, k=k, mode=mode, impl=pv.IMPL_TENSOR_CORE_BF16_HEAD_SUM)
-        t = acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=None, out_idx=out,
-                              out_scores=sc, cand=cand, cand_scores=cs)
-        _report(f"prefill fp8 (bf16 head sum) mode={mode} seed={seed}", t)
-        assert t.max_score_err <= 0.25
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "fp8"])
