@@ -13,7 +13,9 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libpivot.so")
+# PIVOT_LIB selects another build of the same sources that sits next to the default one
+# (libpivot_<name>.so from build.build_variant, e.g. the checked -DPIVOT_DEBUG build).
+LIB_PATH = os.path.join(_HERE, os.path.basename(os.environ.get("PIVOT_LIB", "libpivot.so")))
 
 BF16, FP8_E4M3 = 0, 1
 REUSE, REFINE = 0, 1

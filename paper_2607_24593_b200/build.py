@@ -27,6 +27,35 @@ def _stale() -> bool:
     return any(os.path.getmtime(p) > t for p in deps)
 
 
+def build_variant(name: str, extra_flags, force: bool = False) -> str:
+    """Builds csrc/ with extra nvcc flags into libpivot_<name>.so next to the default library (objects
+    under build/<name>/).  The binding loads it when PIVOT_LIB names it.  Used for the checked build
+    (-DPIVOT_DEBUG: bounds checks that set a status code) and for A/B timing of compile-time knobs."""
+    out = os.path.join(HERE, f"libpivot_{name}.so")
+    deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.h")) \
+        + glob.glob(os.path.join(HERE, "..", "include", "*.h"))
+    if not force and os.path.exists(out) and all(os.path.getmtime(p) <= os.path.getmtime(out) for p in deps):
+        return out
+    odir = os.path.join(HERE, "build", name)
+    os.makedirs(odir, exist_ok=True)
+    procs, objs = [], []
+    for src in sources():
+        obj = os.path.join(odir, os.path.basename(src)[:-3] + ".o")
+        procs.append((src, subprocess.Popen([NVCC, *FLAGS, *extra_flags, "-c", src, "-o", obj], stdout=subprocess.PIPE,
+                                            stderr=subprocess.STDOUT, text=True)))
+        objs.append(obj)
+    failed = False
+    for src, p in procs:
+        o, _ = p.communicate()
+        if p.returncode:
+            print(f"--- {os.path.basename(src)}\n{o}", file=sys.stderr)
+        failed |= p.returncode != 0
+    if failed:
+        raise RuntimeError("nvcc failed")
+    subprocess.check_call([NVCC, "-shared", "-o", out, *objs, "-lcudart"])
+    return out
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
@@ -52,4 +81,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--variant" in sys.argv:          # python -m ...build --variant NAME -DFLAG ...
+        i = sys.argv.index("--variant")
+        print(build_variant(sys.argv[i + 1], sys.argv[i + 2:], force=True))
+    else:
+        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

@@ -57,8 +57,11 @@ int cand_cap(int kmax) {
   return (int)align_up((size_t)cap, 64);
 }
 
+#ifndef PIVOT_CAP_FACTOR
+#define PIVOT_CAP_FACTOR 8
+#endif
 int tc_cap(int kmax) {
-  size_t cap = (size_t)8 * kmax;     // eight warp segments of K entries each
+  size_t cap = (size_t)PIVOT_CAP_FACTOR * kmax;     // a tight running threshold admits about K (1 + ln(n / K)) entries
   if (cap < 8192) cap = 8192;
   return (int)align_up(cap, 256);
 }

@@ -12,6 +12,10 @@ namespace scan {
 
 constexpr int TILE_KEYS = 128;
 constexpr int KS_SLOTS = 12;      // key-scale ring: deeper than (key stages + accumulator buffers)
+#ifndef PIVOT_CHK
+#define PIVOT_CHK 32
+#endif
+constexpr int kThresholdRefreshTiles = PIVOT_CHK;   // the append warp re-reads its row's threshold off the histogram this often
 
 // Block sequence of one CTA: blocks sorted longest-first are dealt in snake order.
 struct BlockIter {
@@ -98,7 +102,7 @@ __device__ __noinline__ void append_role(SelectCtrl<NROWS, QD>& s, int r, int la
   };
   // The threshold is refreshed every CHK tiles; a tile adds at most TILE_KEYS entries, so a
   // segment checked then always has room until the next check.
-  const int CHK = CAP / (2 * TILE_KEYS) < 32 ? (CAP / (2 * TILE_KEYS) > 0 ? CAP / (2 * TILE_KEYS) : 1) : 32;
+  const int CHK = CAP / (2 * TILE_KEYS) < kThresholdRefreshTiles ? (CAP / (2 * TILE_KEYS) > 0 ? CAP / (2 * TILE_KEYS) : 1) : kThresholdRefreshTiles;
   const int headroom = TILE_KEYS * CHK;
   BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
   uint32_t it = 0;
