@@ -67,12 +67,17 @@ enum {
  *   scale  NULL for bf16.  FP8: one fp32 scale per d-vector -- queries [L, H_I]
  *          (decode [B, g, H_I]), keys [L] (decode [B, Lmax]); value = code * scale.
  *   dtype  PIVOT_BF16 or PIVOT_FP8_E4M3; q and kcache must agree.
+ *   stride_row  bytes from one row of d elements to the next; 0 = dense (d * element size).  Key
+ *          caches may be padded (a serving engine's cache rows often carry more than the indexer
+ *          key): any multiple of 16 bytes >= the dense row size.  Queries must be dense.  The scale
+ *          arrays are always dense.  Not available with impl = 1 or the host-buffer entry point.
  * data must be 16-byte aligned; the key-cache scale 16-byte aligned, the query scale 4-byte.
  */
 typedef struct pivot_tensor {
   const void* data;
   const float* scale;
   int dtype;
+  size_t stride_row;
 } pivot_tensor;
 
 /*
@@ -115,6 +120,12 @@ typedef struct pivot_tensor {
  *                 W >= g (the window then covers the keys written inside the step) and
  *                 W + g - 1 <= 512.  Sequences under the guardrail are scored densely as usual.
  *                 Not available with impl = 1.
+ *   cand_in       decode, Refine only: a candidate set supplied from outside, [B, c] int32 on the
+ *                 device, valid entries first (min(c, pos0[b] + 1) of them).  The call then skips the
+ *                 shared scan and the top-c select (Eq. 5, Eq. 7) and runs Eq. 8-9 on these
+ *                 candidates -- the second half of a step whose scan was split over several GPUs
+ *                 (pivot_merge_topk builds the set).  Sequences under the guardrail are still
+ *                 scored densely and ignore it.  NULL (the default): the call scans.
  */
 typedef struct pivot_opts {
   int guard_len;
@@ -127,6 +138,7 @@ typedef struct pivot_opts {
   int impl;
   int row_begin, row_end;
   int W;
+  const int32_t* cand_in;
 } pivot_opts;
 
 /* Bytes of scratch a prefill / dense call with these sizes needs: rows = L, n_groups = ceil(L/g)
@@ -214,6 +226,21 @@ int pivot_index_decode_paged(const pivot_tensor* q, const float* w, const pivot_
                              const int32_t* block_table, const int32_t* pos0, int B, int max_pages,
                              int n_pages, int H_I, int d, int g, int c, int k, int mode,
                              int32_t* out_idx, pivot_stream_t stream, const pivot_opts* opts);
+
+/*
+ * TopK (Eq. 7) over the union of several partial candidate lists: the merge step of one decode
+ * sequence whose key axis was split over GPUs -- every part scans its own key range into a local
+ * top-c with proxy scores (pivot_index_decode in Reuse mode with k = c on that range, positions
+ * relative to the range), the parts are exchanged, and the global top-c is the top-c of their union
+ * (a key of the global top-c is in the top-c of its own range).
+ *   scores, idx   [n_seg, seg_len] fp32 / int32, device: part p's entries; idx < 0 marks an empty slot.
+ *   seg_offset    [n_seg] int32, device, or NULL: added to the positions of part p (its range's first key).
+ *   K             entries to keep (at most 8192); order (score desc, position asc), as everywhere.
+ *   out_idx       [K] int32, valid entries first, then -1; out_scores [K] fp32 or NULL.
+ * Uses the registered workspace (at least 256 + 8 * n_seg * seg_len bytes).
+ */
+int pivot_merge_topk(const float* scores, const int32_t* idx, int n_seg, int seg_len, const int32_t* seg_offset,
+                     int K, int32_t* out_idx, float* out_scores, pivot_stream_t stream);
 
 /*
  * Dense control: Eq. 1 + TopK for every query of a request (prefill form) -- the O(L^2) indexer

@@ -28,20 +28,20 @@ SYMBOLS = [
     "pivot_index_decode", "pivot_index_decode_ex", "pivot_index_decode_paged", "dense_index", "dense_index_ex", "dense_index_static",
     "pivot_prefill_host_arena_bytes", "pivot_index_prefill_host", "pivot_device_status",
     "pivot_stage_timing", "pivot_stage_times", "pivot_launch_count_reset", "pivot_status_str", "pivot_last_cuda_error",
-    "dense_index_decode", "dense_index_decode_ex", "pivot_debug_wait_expiry", "pivot_debug_mma_model", "pivot_debug_key_stream",
+    "dense_index_decode", "dense_index_decode_ex", "pivot_debug_wait_expiry", "pivot_debug_mma_model", "pivot_debug_key_stream", "pivot_merge_topk",
 ]
 DEV_OK, DEV_WAIT_EXPIRED, DEV_CAND_OVERFLOW, DEV_BAD_POS, DEV_BOUNDS = 0, 1, 2, 3, 4
 
 
 class pivot_tensor(C.Structure):
-    _fields_ = [("data", C.c_void_p), ("scale", C.c_void_p), ("dtype", C.c_int)]
+    _fields_ = [("data", C.c_void_p), ("scale", C.c_void_p), ("dtype", C.c_int), ("stride_row", C.c_size_t)]
 
 
 class pivot_opts(C.Structure):
     _fields_ = [("guard_len", C.c_int), ("pool", C.c_int), ("dbg_cand", C.c_void_p),
                 ("dbg_scores", C.c_void_p), ("dbg_cand_scores", C.c_void_p),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("impl", C.c_int),
-                ("row_begin", C.c_int), ("row_end", C.c_int), ("W", C.c_int)]
+                ("row_begin", C.c_int), ("row_end", C.c_int), ("W", C.c_int), ("cand_in", C.c_void_p)]
 
 
 class PivotError(RuntimeError):
@@ -74,6 +74,7 @@ def _load():
     lib.pivot_debug_wait_expiry.argtypes = [C.c_ulonglong, P]
     lib.pivot_debug_mma_model.argtypes = [P, P]
     lib.pivot_debug_key_stream.argtypes = [P, I, I, I, I, I, P, P]
+    lib.pivot_merge_topk.argtypes = [P, P, I, I, P, I, P, P, P]
     lib.pivot_prefill_host_arena_bytes.restype = S
     lib.pivot_prefill_host_arena_bytes.argtypes = [I, I, I, I, I, I, I]
     lib.pivot_index_prefill_host.argtypes = [T, P, T, I, I, I, I, I, I, I, P, P, S, P]
@@ -105,8 +106,17 @@ def _dtype_code(t: torch.Tensor) -> int:
 
 
 def _tensor(data: torch.Tensor, scale) -> pivot_tensor:
-    assert data.is_contiguous() and (scale is None or (scale.is_contiguous() and scale.dtype == torch.float32))
-    return pivot_tensor(data.data_ptr(), None if scale is None else scale.data_ptr(), _dtype_code(data))
+    """Dense tensors, or key caches whose rows are padded: a view [..., rows, d] of a wider buffer with
+    unit stride along d and every outer dimension dense over the padded rows (stride_row = bytes per row)."""
+    assert scale is None or (scale.is_contiguous() and scale.dtype == torch.float32)
+    stride_row = 0
+    if not data.is_contiguous():
+        assert data.stride(-1) == 1, "the last dimension must be contiguous"
+        rs = data.stride(-2)
+        for i in range(data.dim() - 2):            # outer dimensions must be dense over the padded rows
+            assert data.stride(i) == rs * int(torch.tensor(data.shape[i + 1:-1]).prod()), "unsupported strides"
+        stride_row = rs * data.element_size()
+    return pivot_tensor(data.data_ptr(), None if scale is None else scale.data_ptr(), _dtype_code(data), stride_row)
 
 
 def _stream(stream) -> int:
@@ -118,12 +128,12 @@ def _stream(stream) -> int:
 IMPL_TENSOR_CORE, IMPL_CUDA_CORE, IMPL_TENSOR_CORE_FP32_HEAD_SUM = 0, 1, 2
 
 
-def _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl=0, rows=None, W=0) -> pivot_opts:
+def _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl=0, rows=None, W=0, cand_in=None) -> pivot_opts:
     p = lambda t: None if t is None else t.data_ptr()
     r0, r1 = (0, 0) if rows is None else rows
     return pivot_opts(-1 if guard_len is None else guard_len, pool, p(dbg_cand), p(dbg_scores),
                       p(dbg_cand_scores), p(workspace), 0 if workspace is None else workspace.numel(), impl,
-                      r0, r1, W)
+                      r0, r1, W, p(cand_in))
 
 
 def pivot_workspace_bytes(rows: int, n_groups: int, c: int, k: int) -> int:
@@ -216,13 +226,15 @@ def dense_index_static(q, w, kcache, L, H_I, d, k, out_idx, stream=None, *, q_sc
 
 def pivot_index_decode(q, w, kcache, pos0, B, Lmax, H_I, d, g, c, k, mode, out_idx, stream=None, *,
                        q_scale=None, k_scale=None, guard_len=None, pool=POOL_MEAN, dbg_cand=None,
-                       dbg_scores=None, dbg_cand_scores=None, workspace=None, impl=0, W=0):
+                       dbg_scores=None, dbg_cand_scores=None, workspace=None, impl=0, W=0, cand_in=None):
+    """cand_in ([B, c] int32, device): Refine on candidate sets supplied from outside (no scan)."""
     tq, tk = _tensor(q, q_scale), _tensor(kcache, k_scale)
     assert w.dtype == torch.float32 and out_idx.dtype == torch.int32 and pos0.dtype == torch.int32
     assert out_idx.numel() >= B * g * k
+    assert cand_in is None or (cand_in.dtype == torch.int32 and cand_in.is_contiguous() and cand_in.numel() >= B * c)
     if workspace is None:
         ensure_workspace(B * g, B, c, k, q.device, need=pivot_decode_workspace_bytes(B, Lmax, g, c, k))
-    o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl, W=W)
+    o = _opts(guard_len, pool, dbg_cand, dbg_scores, dbg_cand_scores, workspace, impl, W=W, cand_in=cand_in)
     _check(lib.pivot_index_decode_ex(C.byref(tq), w.data_ptr(), C.byref(tk), pos0.data_ptr(), B, Lmax,
                                      H_I, d, g, c, k, mode, out_idx.data_ptr(), _stream(stream), C.byref(o)))
     return out_idx
@@ -255,6 +267,24 @@ def dense_index_decode(q, w, kcache, pos0, B, Lmax, H_I, d, g, k, out_idx, strea
     o = _opts(None, POOL_MEAN, None, dbg_scores, None, workspace, impl)
     _check(lib.dense_index_decode_ex(C.byref(tq), w.data_ptr(), C.byref(tk), pos0.data_ptr(), B, Lmax, H_I, d, g, k,
                                      out_idx.data_ptr(), _stream(stream), C.byref(o)))
+    return out_idx
+
+
+def pivot_merge_topk(scores, idx, K, out_idx, out_scores=None, seg_offset=None, stream=None):
+    """Top-K of the union of candidate lists: scores / idx [n_seg, seg_len] (idx < 0 = empty slot), seg_offset [n_seg]
+    int32 added to each list's positions.  Uses the registered workspace."""
+    assert scores.dtype == torch.float32 and idx.dtype == torch.int32 and scores.shape == idx.shape and idx.dim() == 2
+    assert scores.is_contiguous() and idx.is_contiguous() and out_idx.dtype == torch.int32 and out_idx.numel() >= K
+    n_seg, seg_len = idx.shape
+    need = 256 + 8 * n_seg * seg_len
+    dev = idx.device.index if idx.device.index is not None else torch.cuda.current_device()
+    cur = _workspaces.get(dev)
+    if cur is None or cur.numel() < need:
+        with torch.cuda.device(dev):
+            pivot_set_workspace(torch.empty(need, dtype=torch.uint8, device=f"cuda:{dev}"))
+    p = lambda t: None if t is None else t.data_ptr()
+    _check(lib.pivot_merge_topk(scores.data_ptr(), idx.data_ptr(), n_seg, seg_len, p(seg_offset), K, out_idx.data_ptr(),
+                                p(out_scores), _stream(stream)))
     return out_idx
 
 

@@ -177,12 +177,23 @@ int check_operands(const pivot_tensor* q, const float* w, const pivot_tensor* kc
   if ((uintptr_t)kc->scale & 15) return PIVOT_ERR_INVALID_ARG;
   if (H != kHeads || d != kDim) return PIVOT_ERR_UNSUPPORTED;
   if (k > kMaxSel || c > kMaxSel) return PIVOT_ERR_UNSUPPORTED;
+  // rows: queries dense; key rows dense or padded to a multiple of 16 bytes (below 2^31)
+  const size_t row = (size_t)kDim * (q->dtype == PIVOT_FP8_E4M3 ? 1 : 2);
+  if (q->stride_row != 0 && q->stride_row != (size_t)kHeads * row && q->stride_row != row) return PIVOT_ERR_UNSUPPORTED;
+  if (kc->stride_row != 0 && (kc->stride_row < row || (kc->stride_row & 15) || kc->stride_row > (1u << 30)))
+    return PIVOT_ERR_INVALID_ARG;
   return PIVOT_OK;
 }
 
 }  // namespace pivot
 
 namespace {
+
+// Bytes between key rows as the kernels take it: 0 for a dense cache.
+int key_stride(const pivot_tensor* kc) {
+  const size_t row = (size_t)kDim * (kc->dtype == PIVOT_FP8_E4M3 ? 1 : 2);
+  return kc->stride_row == 0 || kc->stride_row == row ? 0 : (int)kc->stride_row;
+}
 
 int resolve_ws(const pivot_opts* o, size_t need, void** ws) {
   void* p = o && o->workspace ? o->workspace : g_dev[cur_device()].ws;
@@ -226,6 +237,8 @@ int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, i
   PrefillPlan p;
   p.q = q->data; p.w = w; p.qscale = q->scale;
   p.kc = kc->data; p.kscale = kc->scale;
+  p.k_stride = key_stride(kc);
+  if (p.k_stride && o && o->impl == 1) return PIVOT_ERR_UNSUPPORTED;
   p.proxy_q = ws.proxy_q; p.proxy_w = ws.proxy_w;
   p.cand = (o && o->dbg_cand) ? o->dbg_cand + (size_t)pg0 * c : ws.cand;
   p.cand_score = (o && o->dbg_cand_scores) ? o->dbg_cand_scores + (size_t)pg0 * c : nullptr;
@@ -248,6 +261,7 @@ int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, i
     launch_scan_simt(ws.rows, p.n_dense + p.n_proxy, q->dtype, ws.scan, st);
   } else {
     ScanOperands op{kc->data, L, kc->scale, q->data, L, ws.proxy_q, p.n_proxy, q->dtype};
+    op.k_stride = p.k_stride;
     if ((rc = check_cuda(launch_scan_tc(op, ws.rows, p.n_dense + p.n_proxy, 4, tc_scratch(ws), sm_count(), st,
                                         o && o->impl == 2))))
       return rc;
@@ -321,8 +335,9 @@ int pivot_index_prefill_varlen(const pivot_tensor* q, const float* w, const pivo
     const size_t r0 = (size_t)cu_seqlens[i];
     const int L = cu_seqlens[i + 1] - cu_seqlens[i];
     if (L == 0) continue;
-    pivot_tensor tq{(const char*)q->data + r0 * H_I * d * esz, q->scale ? q->scale + r0 * H_I : nullptr, q->dtype};
-    pivot_tensor tk{(const char*)kcache->data + r0 * d * esz, kcache->scale ? kcache->scale + r0 : nullptr, q->dtype};
+    const size_t krow = kcache->stride_row ? kcache->stride_row : (size_t)d * esz;
+    pivot_tensor tq{(const char*)q->data + r0 * H_I * d * esz, q->scale ? q->scale + r0 * H_I : nullptr, q->dtype, 0};
+    pivot_tensor tk{(const char*)kcache->data + r0 * krow, kcache->scale ? kcache->scale + r0 : nullptr, q->dtype, kcache->stride_row};
     rc = pivot_index_prefill_ex(&tq, w + r0 * H_I, &tk, L, H_I, d, g, c, k, mode, out_idx + r0 * k, stream, opts);
     if (rc) return rc;
   }
@@ -361,6 +376,8 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
   const int W = o ? o->W : 0;
   if (W < 0 || (W > 0 && (mode != PIVOT_REFINE || W < g || W + g - 1 > kDecodeWinMax || o->impl == 1)))
     return PIVOT_ERR_INVALID_ARG;
+  const int32_t* cand_in = o ? o->cand_in : nullptr;
+  if (cand_in && (mode != PIVOT_REFINE || o->impl == 1 || dense_share || ((uintptr_t)cand_in & 3))) return PIVOT_ERR_INVALID_ARG;
   const bool paged = block_table != nullptr;
   if (paged && (n_pages < 1 || (Lmax & 127) || (o && o->impl == 1))) return PIVOT_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
@@ -373,10 +390,12 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
   DecodePlan p;
   p.q = q->data; p.w = w; p.qscale = q->scale;
   p.kc = kcache->data; p.kscale = kcache->scale;
+  p.k_stride = key_stride(kcache);
+  if (p.k_stride && o && o->impl == 1) return PIVOT_ERR_UNSUPPORTED;
   p.pos0 = pos0;
   p.proxy_q = ws.proxy_q; p.proxy_w = ws.proxy_w;
-  p.cand = (o && o->dbg_cand) ? o->dbg_cand : ws.cand;
-  p.cand_score = o ? o->dbg_cand_scores : nullptr;
+  p.cand = cand_in ? const_cast<int32_t*>(cand_in) : (o && o->dbg_cand) ? o->dbg_cand : ws.cand;
+  p.cand_score = (o && !cand_in) ? o->dbg_cand_scores : nullptr;
   p.out = out_idx; p.out_score = o ? o->dbg_scores : nullptr;
   p.B = B; p.Lmax = Lmax; p.g = g; p.c = c; p.k = k; p.mode = mode; p.dtype = q->dtype;
   p.guard_len = (o && o->guard_len >= 0) ? o->guard_len : c;
@@ -407,7 +426,9 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
     df.kc = kcache->data; df.kscale = kcache->scale; df.q = q->data; df.proxy_q = dense_share ? q->data : ws.proxy_q;
     df.B = B; df.Lmax = Lmax; df.g = g; df.c = c; df.k = k; df.mode = mode; df.dtype = q->dtype;
     df.k_rows = k_rows;
+    df.k_stride = p.k_stride;
     df.W = W;
+    df.skip_scan = cand_in != nullptr;
     df.sms = sm_count();
     df.scratch = (char*)wsp + base_bytes;
     df.scratch_tc = tc_scratch(ws);
@@ -420,6 +441,7 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
     // dense rows of guarded (short) sequences, if any: the generic scan, one row per block
     if (!paged) {
       ScanOperands op{kcache->data, k_rows, kcache->scale, q->data, B * g, ws.proxy_q, B, q->dtype};
+      op.k_stride = p.k_stride;
       if ((rc = check_cuda(launch_scan_tc(op, ws.rows + B, B * g, 1, tc_scratch(ws), sm_count(), st)))) return rc;
     }
   }
@@ -468,6 +490,19 @@ int dense_index_decode(const pivot_tensor* q, const float* w, const pivot_tensor
   return dense_index_decode_ex(q, w, kcache, pos0, B, Lmax, H_I, d, g, k, out_idx, stream, nullptr);
 }
 
+int pivot_merge_topk(const float* scores, const int32_t* idx, int n_seg, int seg_len, const int32_t* seg_offset, int K,
+                     int32_t* out_idx, float* out_scores, pivot_stream_t stream) {
+  if (!scores || !idx || !out_idx || n_seg < 1 || seg_len < 1 || K < 1) return PIVOT_ERR_INVALID_ARG;
+  if (K > kMaxSel || (long long)n_seg * seg_len > (1 << 24)) return PIVOT_ERR_UNSUPPORTED;
+  if (((uintptr_t)scores | (uintptr_t)idx | (uintptr_t)out_idx | (uintptr_t)seg_offset | (uintptr_t)out_scores) & 3)
+    return PIVOT_ERR_INVALID_ARG;
+  DeviceState& ds = g_dev[cur_device()];
+  const size_t need = 256 + (size_t)n_seg * seg_len * sizeof(unsigned long long);
+  if (!ds.ws || ds.ws_bytes < need) return PIVOT_ERR_WORKSPACE;
+  return check_cuda(launch_merge_topk(scores, idx, n_seg, seg_len, seg_offset, (unsigned long long*)((char*)ds.ws + 256), K,
+                                      out_idx, out_scores, (cudaStream_t)stream));
+}
+
 int pivot_debug_wait_expiry(unsigned long long limit_ns, pivot_stream_t stream) {
   if (limit_ns < 1000ull || limit_ns > 1000000000ull) return PIVOT_ERR_INVALID_ARG;      // 1 us .. 1 s
   DeviceState& ds = g_dev[cur_device()];
@@ -512,6 +547,7 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
   // every argument check of the device entry point runs here, before the first copy is enqueued
   int rc = check_common(q, w, kcache, H_I, d, c, k, mode, out_idx);
   if (rc) return rc;
+  if (key_stride(kcache)) return PIVOT_ERR_UNSUPPORTED;          // host arrays are copied as dense blocks
   if (((uintptr_t)arena & 255) || arena_bytes < pivot_prefill_host_arena_bytes(L, H_I, d, g, c, k, q->dtype))
     return PIVOT_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
@@ -577,8 +613,8 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
       return rc;
     if ((rc = check_cuda(cudaEventRecord(ds.ev_in[i], ds.copy_in)))) return rc;
   }
-  pivot_tensor tq{dq, fp8 ? dqs : nullptr, q->dtype};
-  pivot_tensor tk{dk, fp8 ? dks : nullptr, q->dtype};
+  pivot_tensor tq{dq, fp8 ? dqs : nullptr, q->dtype, 0};
+  pivot_tensor tk{dk, fp8 ? dks : nullptr, q->dtype, 0};
   for (int j = 0; j < n_chunks; ++j) {
     const int i = order[j];
     const int r0 = i * chunk_rows, r1 = (r0 + chunk_rows < L) ? r0 + chunk_rows : L;

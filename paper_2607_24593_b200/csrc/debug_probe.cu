@@ -357,7 +357,7 @@ cudaError_t launch_mma_model_probe(long long* out, cudaStream_t st) {
   return cudaGetLastError();
 }
 
-bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows);
+bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows, int row_stride);
 
 // keys: an FP8 key tensor [n_keys, 128] (device), n_keys a multiple of 128; out: one slot per CTA
 // (clocks per tile seen by that CTA's first and, with mode 1 / 2, second stream: out[2 cta], out[2 cta + 1]).
@@ -366,7 +366,7 @@ cudaError_t launch_key_stream_probe(const void* keys, int n_keys, int ctas, int 
   if (mode < 0 || mode > 4 || ((mode == 1 || mode == 2) && stages > 6)) return cudaErrorInvalidValue;
   if (stages < 1 || stages > 12 || n_keys < 128 || (n_keys & 127) || ctas < 1 || tiles < 1) return cudaErrorInvalidValue;
   CUtensorMap mk;
-  if (!make_operand_map(&mk, keys, n_keys, DT_FP8, mode >= 3 ? 32 : 128)) return cudaErrorInvalidValue;
+  if (!make_operand_map(&mk, keys, n_keys, DT_FP8, mode >= 3 ? 32 : 128, 0)) return cudaErrorInvalidValue;
   const size_t smem = 1024 + (size_t)stages * 16384 * ((mode == 1 || mode == 2) ? 2 : 1);
   if (cudaError_t e = cudaFuncSetAttribute(key_stream_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       e != cudaSuccess)

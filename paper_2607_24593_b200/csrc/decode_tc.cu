@@ -424,6 +424,23 @@ __global__ void __launch_bounds__(kBlk, 1) entries_topk_kernel(const EntryList* 
   blk_emit_topk(sm, (const entry_t*)el.list, el.n, el.n, el.K, el.out, el.out_score, 1, el.K);
 }
 
+// Union of candidate lists -> packed entries -> exact top-K, one block.
+__global__ void __launch_bounds__(kBlk, 1)
+merge_topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ idx, int n_seg, int seg_len,
+                  const int32_t* __restrict__ seg_offset, entry_t* __restrict__ entries, int K, int32_t* out_idx,
+                  float* out_scores) {
+  __shared__ BlkSelSmem sm;
+  const int n = n_seg * seg_len;
+  for (int i = threadIdx.x; i < n; i += kBlk) {
+    const int ix = idx[i];
+    const int off = seg_offset ? seg_offset[i / seg_len] : 0;
+    entries[i] = ix < 0 ? kPadEntry : make_entry(score_to_key(scores[i]), ix + off);
+  }
+  __threadfence_block();
+  __syncthreads();
+  blk_emit_topk(sm, entries, n, n, K, out_idx, out_scores, 1, K);
+}
+
 // ------------------------------------------------------------------------------ setup
 
 // One launch prepares a decode step: block b clears sequence b's histogram and list counters and
@@ -566,7 +583,7 @@ cudaError_t launch_scan(const CUtensorMap& mk, const CUtensorMap& mq, const CUte
 
 }  // namespace
 
-bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows);
+bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows, int row_stride);
 bool make_scale_map(CUtensorMap* m, const float* base, long long n, int box);
 
 size_t decode_fast_bytes(int B, int Lmax, int g, int c) {
@@ -577,6 +594,13 @@ size_t decode_fast_bytes(int B, int Lmax, int g, int c) {
   return up(B * Ls * 4) + up((size_t)B * (DHIST + 2) * 4) + up((size_t)(B + 1) * 4) + up((size_t)B * SEL_CAP * 8) +
          up((size_t)B * mc * (ncc + 1) * sizeof(GroupDesc)) + up((size_t)B * g * sizeof(EntryList)) +
          up((size_t)B * kDecodeWinMax * 4) + up((size_t)B * g * (c + kDecodeWinMax) * 8);
+}
+
+cudaError_t launch_merge_topk(const float* scores, const int32_t* idx, int n_seg, int seg_len, const int32_t* seg_offset,
+                              unsigned long long* entries, int K, int32_t* out_idx, float* out_scores, cudaStream_t st) {
+  merge_topk_kernel<<<1, kBlk, 0, st>>>(scores, idx, n_seg, seg_len, seg_offset, entries, K, out_idx, out_scores);
+  ++launch_counter();
+  return cudaGetLastError();
 }
 
 cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
@@ -605,9 +629,12 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   CUtensorMap mk, mq, mks;
   memset(&mks, 0, sizeof(mks));
   if (d.dtype == DT_FP8 && !make_scale_map(&mks, d.kscale, d.k_rows, TILE_KEYS)) return cudaErrorInvalidValue;
-  if (!make_operand_map(&mk, d.kc, d.k_rows, d.dtype, TILE_KEYS) ||
-      !make_operand_map(&mq, d.proxy_q, (long long)d.B * kHeads, d.dtype, kHeads))
+  if (!make_operand_map(&mk, d.kc, d.k_rows, d.dtype, TILE_KEYS, d.k_stride) ||
+      !make_operand_map(&mq, d.proxy_q, (long long)d.B * kHeads, d.dtype, kHeads, 0))
     return cudaErrorInvalidValue;
+  if (d.skip_scan) {
+    if (d.mode != 1) return cudaErrorInvalidValue;
+  } else {
   if (d.ev_scan_begin) cudaEventRecord(d.ev_scan_begin, st);
   e = d.dtype == DT_FP8
           ? launch_scan<DT_FP8>(mk, mq, mks, d.prox, tile_prefix, d.B, Ls, scores, ghist, d.status, d.sms, st)
@@ -619,6 +646,7 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   if ((e = opt_in_dynamic_smem(decode_select_kernel, sel_smem, sel_attr)) != cudaSuccess) return e;
   decode_select_kernel<<<dim3(SEL_SPLIT, d.B), kBlk, sel_smem, st>>>(d.prox, Ls, scores, ghist, glist, sel_ctr);
   ++launch_counter();
+  }
   if (d.mode == 1) {
     if (W > 0) {
       decode_window_kernel<<<d.B, 1024, 0, st>>>(d.groups, mc, d.g, W, wcand);

@@ -17,6 +17,7 @@ struct GroupDesc {
   const float* qscale;  // [m, H] or nullptr
   const void* kbase;
   const float* kscale;
+  int k_stride = 0;     // bytes between key rows (0: dense)
   const int32_t* cand;  // candidate key positions, valid entries first
   int n_cand;           // valid candidates (0: group is skipped)
   int m;                // members (at most kMembersPerDesc per descriptor)
@@ -57,6 +58,7 @@ struct EntryList {
 struct PrefillPlan {
   const void* q; const float* w; const float* qscale;   // raw per-query operands
   const void* kc; const float* kscale;                  // key cache
+  int k_stride = 0;                                     // bytes between key rows (0: dense)
   void* proxy_q; float* proxy_w;                        // [nP, H, d], [nP, H]
   int32_t* cand; float* cand_score;                     // [nP, c] (Refine)
   int32_t* out; float* out_score;                       // [L, k]
@@ -71,6 +73,7 @@ struct PrefillPlan {
 struct DecodePlan {
   const void* q; const float* w; const float* qscale;   // [B, g, H, d] ...
   const void* kc; const float* kscale;                  // [B, Lmax, d], [B, Lmax]
+  int k_stride = 0;                                     // bytes between key rows (0: dense)
   const int32_t* pos0;
   void* proxy_q; float* proxy_w;                        // [B, H, d], [B, H]
   int32_t* cand; float* cand_score;                     // [B, c]
@@ -116,6 +119,7 @@ struct ScanOperands {
   const void* q; int q_rows;               // raw queries [q_rows, H, d]
   const void* proxy_q; int proxy_rows;     // proxies [proxy_rows, H, d]
   int dtype;
+  int k_stride = 0;                        // bytes between key rows (0: dense)
 };
 // rows_per_block consecutive scan rows share one key stream (4 in prefill, 1 in decode).
 // fp32_head_sum: keep the gate-weighted head sum in fp32 FMAs even where the tensor-core form
@@ -138,7 +142,9 @@ struct DecodeFast {
   const void* kc; const float* kscale; const void* q; const void* proxy_q;
   int B, Lmax, g, c, k, mode, dtype, sms;
   long long k_rows;           // rows of the key tensor (B * Lmax, or pool pages * 128 when paged)
+  int k_stride = 0;           // bytes between key rows (0: dense)
   int W = 0;                  // per-query local window (Appendix B, decode form); Refine only
+  bool skip_scan = false;     // the candidate sets come from the caller: no scan, no top-c select
   void* scratch;              // decode_fast_bytes(...) bytes
   ScanScratch scratch_tc;     // candidate scratch of the re-score kernel
   int* status;
@@ -148,6 +154,9 @@ size_t decode_fast_bytes(int B, int Lmax, int g, int c);
 cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st);
 
 long long& launch_counter();
+// Top-K of the union of n_seg candidate lists (see pivot_merge_topk); entries = scratch for n_seg * seg_len packed entries.
+cudaError_t launch_merge_topk(const float* scores, const int32_t* idx, int n_seg, int seg_len, const int32_t* seg_offset,
+                              unsigned long long* entries, int K, int32_t* out_idx, float* out_scores, cudaStream_t st);
 
 // Diagnostic: a kernel whose bounded waits run out after limit_ns (see debug_probe.cu).
 cudaError_t launch_wait_expiry_probe(int* status, unsigned long long limit_ns, cudaStream_t st);

@@ -66,6 +66,7 @@ __global__ void plan_prefill_kernel(PrefillPlan p, RowDesc* rows, GroupDesc* gro
       gd.qscale = p.qscale ? p.qscale + (size_t)t0 * kHeads : nullptr;
       gd.kbase = p.kc;
       gd.kscale = p.kscale;
+      gd.k_stride = p.k_stride;
       gd.cand = r.out;
       gd.n_cand = p.W > 0 ? p.c : min(p.c, r.n_vis);   // with a window every slot is read (pads are skipped)
       gd.m = m;

@@ -48,7 +48,8 @@ __device__ __forceinline__ bool plan_decode_sequence(const DecodePlan& p, int b,
   // Paged cache: descriptors point at the page pool and carry the sequence's block-table row.
   const bool paged = p.block_table != nullptr;
   const int32_t* pages = paged ? p.block_table + (size_t)cb * (p.Lmax / 128) : nullptr;
-  const void* kb = paged ? p.kc : (const char*)p.kc + (size_t)cb * p.Lmax * kDim * esz;
+  const size_t krow = p.k_stride > 0 ? (size_t)p.k_stride : kDim * esz;                       // bytes per key row
+  const void* kb = paged ? p.kc : (const char*)p.kc + (size_t)cb * p.Lmax * krow;
   const float* ksb = !p.kscale ? nullptr : paged ? p.kscale : p.kscale + (size_t)cb * p.Lmax;
   int32_t* outb = p.out + (size_t)b * p.g * p.k;
   float* outsb = p.out_score ? p.out_score + (size_t)b * p.g * p.k : nullptr;
@@ -69,6 +70,7 @@ __device__ __forceinline__ bool plan_decode_sequence(const DecodePlan& p, int b,
   gd.qscale = p.qscale ? p.qscale + (size_t)b * p.g * kHeads : nullptr;
   gd.kbase = kb;
   gd.kscale = ksb;
+  gd.k_stride = p.k_stride;
   gd.cand = p.cand + (size_t)b * p.c;
   gd.n_cand = 0;
   gd.m = p.g;

@@ -268,6 +268,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       const GroupDesc gd = groups[gi];
       const int ntiles = group_tiles(gd);
       if (ntiles == 0) continue;
+      const size_t krow_bytes = gd.k_stride > 0 ? (size_t)gd.k_stride : (size_t)C::ROW_BYTES;   // padded cache rows
       // Candidate positions are fetched three tiles ahead, their rows in the key tensor (a
       // block-table lookup when the cache is paged) two tiles ahead and key scales one tile
       // ahead, so no round trip sits on this thread's issue path.
@@ -308,7 +309,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
           const int rl = i * 4 + sub;                  // row inside this warp's 64
           const int kr = __shfl_sync(0xffffffffu, krow[i >> 3], rl & 31);
           const int row = wrow0 + rl;
-          const uint8_t* src = (const uint8_t*)gd.kbase + (size_t)kr * C::ROW_BYTES + chunk * 16;
+          const uint8_t* src = (const uint8_t*)gd.kbase + (size_t)kr * krow_bytes + chunk * 16;
           const uint32_t dst = dst0 + (uint32_t)row * 128u + (uint32_t)((chunk ^ (row & 7)) << 4);
 #pragma unroll
           for (int h = 0; h < C::KHALVES; ++h) cp_async16(dst + h * C::HALF_TILE_BYTES, src + h * 128);
@@ -561,13 +562,13 @@ cudaError_t launch_one(const CUtensorMap& mq, const GroupDesc* groups, int n_gro
 
 }  // namespace
 
-bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows);
+bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows, int row_stride);
 
 cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
                              const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum, bool chunked) {
   if (n_groups <= 0) return cudaSuccess;
   CUtensorMap mq;
-  if (!make_operand_map(&mq, q, (long long)q_rows * kHeads, dtype, kHeads)) return cudaErrorInvalidValue;
+  if (!make_operand_map(&mq, q, (long long)q_rows * kHeads, dtype, kHeads, 0)) return cudaErrorInvalidValue;
   if (dtype != DT_FP8) return launch_one<DT_BF16>(mq, groups, n_groups, q_rows, s, sms, st);
   if (fp32_head_sum) return launch_one<DT_FP8, 0>(mq, groups, n_groups, q_rows, s, sms, st);
   return chunked ? launch_one<DT_FP8, 2>(mq, groups, n_groups, q_rows, s, sms, st)

@@ -561,12 +561,13 @@ EncodeTiledFn encode_fn() {
 }
 
 // 2-D map over a row-major [rows, 128] operand tensor; box = 128 bytes x box_rows, 128B swizzle.
-bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows) {
+// row_stride: bytes between rows, 0 = dense (a multiple of 16 bytes otherwise: padded key-cache rows).
+bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows, int row_stride) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const bool fp8 = dtype == DT_FP8;
   cuuint64_t dims[2] = {(cuuint64_t)kDim, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)(kDim * (fp8 ? 1 : 2))};
+  cuuint64_t strides[1] = {(cuuint64_t)(row_stride > 0 ? row_stride : kDim * (fp8 ? 1 : 2))};
   cuuint32_t box[2] = {(cuuint32_t)(fp8 ? 128 : 64), (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   return fn(m, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, dims,
@@ -594,9 +595,9 @@ cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_ro
   CUtensorMap mk, mq0, mq1, mks;
   memset(&mks, 0, sizeof(mks));
   if (op.dtype == DT_FP8 && !make_scale_map(&mks, op.kscale, op.k_rows, TILE_KEYS)) return cudaErrorInvalidValue;
-  if (!make_operand_map(&mk, op.kc, op.k_rows, op.dtype, TILE_KEYS) ||
-      !make_operand_map(&mq0, op.q, (long long)op.q_rows * kHeads, op.dtype, kHeads) ||
-      !make_operand_map(&mq1, op.proxy_q, (long long)(op.proxy_rows > 0 ? op.proxy_rows : 1) * kHeads, op.dtype, kHeads))
+  if (!make_operand_map(&mk, op.kc, op.k_rows, op.dtype, TILE_KEYS, op.k_stride) ||
+      !make_operand_map(&mq0, op.q, (long long)op.q_rows * kHeads, op.dtype, kHeads, 0) ||
+      !make_operand_map(&mq1, op.proxy_q, (long long)(op.proxy_rows > 0 ? op.proxy_rows : 1) * kHeads, op.dtype, kHeads, 0))
     return cudaErrorInvalidValue;
   if (op.dtype == DT_FP8) {
     if (rows_per_block != 4) return launch_one<DT_FP8, 1>(mk, mq0, mq1, mks, rows, n_rows, s, sms, st);

@@ -81,6 +81,10 @@ extern "C" int dense_index_static(const pivot_tensor* q, const float* w, const p
   sc.counter = status + 1;
   // the proxy tensor map needs some valid address; no row refers to it
   ScanOperands op{kcache->data, L, kcache->scale, q->data, L, q->data, 1, q->dtype};
+  {
+    const size_t row = (size_t)kDim * (kcache->dtype == PIVOT_FP8_E4M3 ? 1 : 2);
+    op.k_stride = kcache->stride_row == 0 || kcache->stride_row == row ? 0 : (int)kcache->stride_row;
+  }
   if (int rc = record_cuda(launch_scan_tc(op, rows, L, 4, sc, kStaticCtas, st))) return rc;
   return record_cuda(cudaGetLastError());
 }

@@ -104,3 +104,86 @@ def imbalance(L: int, g: int, world: int, block_rows: int = 8192) -> float:
     for i, b in enumerate(blocks):
         cost[owner(i, world)] += block_cost(b)
     return max(cost) / (sum(cost) / world)
+
+
+# ------------------------------------------------------------------------------------------------
+# One decode sequence over several GPUs: the key axis of the shared scan is split.
+#
+# The scan of Eq. 5 is a score per key, so key ranges are independent; a key of the global top-c
+# (Eq. 7) is in the top-c of its own range.  Every rank holds the sequence's key cache, scans its
+# own range into a local top-c with proxy scores, the (score, position) lists are exchanged once
+# (c pairs per rank), every rank merges them into the same global candidate set, and Eq. 8-9 run
+# on that set (on the owner, or on every rank alike).  The exchange is the only collective.
+
+def key_ranges(n_visible: int, world: int, tile: int = 128) -> List[Block]:
+    """Rank r scans keys [k0, k1) of the n_visible keys: whole 128-key tiles dealt evenly, the last
+    range ends at n_visible; ranks beyond the tile count get an empty range."""
+    if n_visible < 1 or world < 1:
+        raise ValueError("n_visible and world must be positive")
+    tiles = (n_visible + tile - 1) // tile
+    per = (tiles + world - 1) // world
+    out = []
+    for r in range(world):
+        t0, t1 = min(r * per, tiles), min((r + 1) * per, tiles)
+        out.append((t0 * tile, min(t1 * tile, n_visible)) if t1 > t0 else (n_visible, n_visible))
+    return out
+
+
+def gather_candidate_lists(scores: torch.Tensor, idx: torch.Tensor, world: int, group=None):
+    """All-gather of the ranks' local lists ([c] each) into [world, c] tensors on every rank."""
+    all_sc = [torch.empty_like(scores) for _ in range(world)]
+    all_ix = [torch.empty_like(idx) for _ in range(world)]
+    dist.all_gather(all_sc, scores, group=group)
+    dist.all_gather(all_ix, idx, group=group)
+    return torch.stack(all_sc), torch.stack(all_ix)
+
+
+def decode_keysplit_local(q, w, kcache, pos0: int, Lmax, H_I, d, c, *, rank: int, world: int, stream=None,
+                          q_scale=None, k_scale=None):
+    """This rank's part of the scan of ONE sequence (q [1, g, H, d], kcache [1, Lmax, d]): the local
+    top-c of the proxy scores over its key range.  Returns (scores [c] fp32, positions [c] int32
+    relative to the range, -1 padded, range start)."""
+    from . import binding as pv
+    g = q.shape[1]
+    k0, k1 = key_ranges(pos0 + 1, world)[rank]
+    dev = q.device
+    sc = torch.full((c,), float("-inf"), dtype=torch.float32, device=dev)
+    ix = torch.full((c,), -1, dtype=torch.int32, device=dev)
+    if k1 > k0:
+        out = torch.empty((1, g, c), dtype=torch.int32, device=dev)
+        osc = torch.empty((1, g, c), dtype=torch.float32, device=dev)
+        view = kcache[:, k0:]                              # one sequence: the range is a contiguous view
+        vks = None if k_scale is None else k_scale[:, k0:]
+        p0 = torch.tensor([k1 - k0 - 1], dtype=torch.int32, device=dev)
+        # Reuse with k = c on the range: the proxy of the step's g queries, its top-c and their scores
+        pv.pivot_index_decode(q, w, view, p0, 1, Lmax - k0, H_I, d, g, c, c, pv.REUSE, out, stream, q_scale=q_scale,
+                              k_scale=vks, guard_len=0, dbg_scores=osc)
+        sc, ix = osc[0, 0].contiguous(), out[0, 0].contiguous()
+    return sc, ix, k0
+
+
+def decode_keysplit_finish(q, w, kcache, pos0_dev, Lmax, H_I, d, c, k, out_idx, all_scores, all_idx, offsets, *,
+                           stream=None, q_scale=None, k_scale=None, cand_out=None):
+    """Merge of the gathered lists ([world, c]) into the global candidate set, then Eq. 8-9 on it.
+    offsets [world] int32 (device): first key of each rank's range."""
+    from . import binding as pv
+    cand = cand_out if cand_out is not None else torch.empty((1, c), dtype=torch.int32, device=q.device)
+    pv.pivot_merge_topk(all_scores, all_idx, c, cand, seg_offset=offsets, stream=stream)
+    g = q.shape[1]
+    pv.pivot_index_decode(q, w, kcache, pos0_dev, 1, Lmax, H_I, d, g, c, k, pv.REFINE, out_idx, stream, q_scale=q_scale,
+                          k_scale=k_scale, guard_len=0, cand_in=cand)
+    return cand
+
+
+def pivot_index_decode_keysplit(q, w, kcache, pos0: int, Lmax, H_I, d, c, k, out_idx, *, rank: int, world: int,
+                                group=None, stream=None, q_scale=None, k_scale=None):
+    """One MTP decode step of ONE sequence with its scan split over `world` ranks (one process per
+    GPU, each holding the sequence's key cache).  Every rank returns the same out_idx [1, g, k]."""
+    sc, ix, _ = decode_keysplit_local(q, w, kcache, pos0, Lmax, H_I, d, c, rank=rank, world=world, stream=stream,
+                                      q_scale=q_scale, k_scale=k_scale)
+    all_sc, all_ix = gather_candidate_lists(sc, ix, world, group) if world > 1 else (sc[None], ix[None])
+    offsets = torch.tensor([r[0] for r in key_ranges(pos0 + 1, world)], dtype=torch.int32, device=q.device)
+    pos0_dev = torch.tensor([pos0], dtype=torch.int32, device=q.device)
+    decode_keysplit_finish(q, w, kcache, pos0_dev, Lmax, H_I, d, c, k, out_idx, all_sc.contiguous(), all_ix.contiguous(),
+                           offsets, stream=stream, q_scale=q_scale, k_scale=k_scale)
+    return out_idx

@@ -447,6 +447,116 @@ def test_decode_bad_pos0_is_reported_not_read(pv, gu):
     assert np.array_equal(np.sort(again, axis=2), np.sort(good, axis=2))
 
 
+# ---------------------------------------------------------------- padded key-cache rows (pivot_tensor.stride_row)
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+@pytest.mark.parametrize("mode", [po.MODE_REUSE, po.MODE_REFINE])
+def test_prefill_with_padded_key_cache_rows(pv, gu, dtype, mode):
+    """A key cache whose rows sit in a wider buffer (a serving engine's cache row carries more than the
+    indexer key): passed as a strided view, scanned through the TMA map's row stride and gathered by
+    the re-score with the same stride -- oracle parity, and the same sets as the dense copy."""
+    L, g, c, k = 1500, 4, 256, 128
+    x = inputs.make_prefill(L, dtype=dtype, seed=81)
+    d = gu.to_cuda(x)
+    pad = 48 if dtype == "fp8" else 24                      # elements: 176-byte / 304-byte rows (multiples of 16)
+    wide = torch.full((L, 128 + pad), 0x7e if dtype == "fp8" else 1.0, dtype=torch.uint8 if dtype == "fp8" else d["k"].dtype,
+                      device="cuda")
+    if dtype == "fp8":
+        wide = wide.view(torch.float8_e4m3fn)
+    wide[:, :128] = d["k"]
+    kview = wide[:, :128]
+    assert not kview.is_contiguous()
+    nG = (L + g - 1) // g
+    out = torch.full((L, k), -7, dtype=torch.int32, device="cuda")
+    sc = torch.full((L, k), float("nan"), dtype=torch.float32, device="cuda")
+    cand = torch.full((nG, c), -7, dtype=torch.int32, device="cuda") if mode == pv.REFINE else None
+    cs = torch.full((nG, c), float("nan"), dtype=torch.float32, device="cuda") if mode == pv.REFINE else None
+    pv.pivot_index_prefill(d["q"], d["w"], kview, L, 64, 128, g, c, k, mode, out, q_scale=d["qscale"], k_scale=d["kscale"],
+                           dbg_scores=sc, dbg_cand=cand, dbg_cand_scores=cs)
+    torch.cuda.synchronize()
+    assert pv.pivot_device_status() == 0
+    f = lambda t_: None if t_ is None else t_.cpu().numpy()
+    t = acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=None, out_idx=f(out), out_scores=f(sc),
+                          cand=f(cand), cand_scores=f(cs))
+    _report(f"padded key rows {dtype} mode={mode}", t)
+    dense, _, _, _ = gu.run_prefill(x, g=g, c=c, k=k, mode=mode)
+    assert np.array_equal(np.sort(f(out), axis=1), np.sort(dense, axis=1))
+    with pytest.raises(pv.PivotError, match="unsupported"):
+        pv.pivot_index_prefill(d["q"], d["w"], kview, L, 64, 128, g, c, k, mode, out, q_scale=d["qscale"],
+                               k_scale=d["kscale"], impl=pv.IMPL_CUDA_CORE)
+
+
+def test_decode_with_padded_key_cache_rows(pv, gu):
+    x = inputs.make_decode(4, 2, 300, 2500, dtype="fp8", seed=82)
+    d = gu.to_cuda(x)
+    B, Lmax = x.k.shape[0], x.k.shape[1]
+    wide = torch.full((B, Lmax, 160), 0x7e, dtype=torch.uint8, device="cuda").view(torch.float8_e4m3fn)
+    wide[:, :, :128] = d["k"]
+    kview = wide[:, :, :128]
+    out = torch.full((B, 2, 128), -7, dtype=torch.int32, device="cuda")
+    cand = torch.full((B, 256), -7, dtype=torch.int32, device="cuda")
+    pv.pivot_index_decode(d["q"], d["w"], kview, d["pos0"], B, Lmax, 64, 128, 2, 256, 128, pv.REFINE, out,
+                          q_scale=d["qscale"], k_scale=d["kscale"], dbg_cand=cand)
+    torch.cuda.synchronize()
+    assert pv.pivot_device_status() == 0
+    acc.check_decode(x.codes(), c=256, k=128, mode=po.MODE_REFINE, guard_len=None, out_idx=out.cpu().numpy(),
+                     cand=cand.cpu().numpy())
+    ref, _, _, _ = gu.run_decode(x, c=256, k=128, mode=po.MODE_REFINE)
+    assert np.array_equal(np.sort(out.cpu().numpy(), axis=2), np.sort(ref, axis=2))
+
+
+# ---------------------------------------------------------------- one decode sequence, key axis split
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+@pytest.mark.parametrize("world", [2, 3, 5])
+def test_decode_key_split_matches_the_single_call_and_the_oracle(pv, gu, dtype, world):
+    """The multi-GPU form of one decode sequence (its scan split along the keys, one exchange of c
+    (score, position) pairs per rank, merge, Eq. 8-9), with the ranks' parts run one after the other
+    on this GPU: same candidate set and index sets as one call, and the oracle agrees."""
+    from paper_2607_24593_b200 import sharded
+    c, k, g = 512, 256, 2
+    x = inputs.make_decode(1, g, 5000, 9000, dtype=dtype, seed=71)
+    d = gu.to_cuda(x)
+    Lmax = x.k.shape[1]
+    p0 = int(x.pos0[0])
+    parts = [sharded.decode_keysplit_local(d["q"], d["w"], d["k"], p0, Lmax, 64, 128, c, rank=r, world=world,
+                                           q_scale=d["qscale"], k_scale=d["kscale"]) for r in range(world)]
+    torch.cuda.synchronize()
+    assert pv.pivot_device_status() == 0
+    all_sc = torch.stack([p[0] for p in parts]).contiguous()
+    all_ix = torch.stack([p[1] for p in parts]).contiguous()
+    offsets = torch.tensor([p[2] for p in parts], dtype=torch.int32, device="cuda")
+    out = torch.full((1, g, k), -7, dtype=torch.int32, device="cuda")
+    cand = torch.full((1, c), -7, dtype=torch.int32, device="cuda")
+    sharded.decode_keysplit_finish(d["q"], d["w"], d["k"], d["pos0"], Lmax, 64, 128, c, k, out, all_sc, all_ix, offsets,
+                                   q_scale=d["qscale"], k_scale=d["kscale"], cand_out=cand)
+    torch.cuda.synchronize()
+    assert pv.pivot_device_status() == 0
+    ref, _, rcand, _ = gu.run_decode(x, c=c, k=k, mode=po.MODE_REFINE, guard_len=0)
+    assert np.array_equal(np.sort(cand.cpu().numpy(), axis=1), np.sort(rcand, axis=1))
+    assert np.array_equal(np.sort(out.cpu().numpy(), axis=2), np.sort(ref, axis=2))
+    t = acc.check_decode(x.codes(), c=c, k=k, mode=po.MODE_REFINE, guard_len=0, out_idx=out.cpu().numpy(),
+                         cand=cand.cpu().numpy())
+    assert t.rows == 1 + g
+
+
+def test_merge_topk_ties_and_empty_slots(pv):
+    """pivot_merge_topk: (score desc, position asc) over the union, empty slots skipped, offsets added."""
+    sc = torch.tensor([[3.0, 1.0, 1.0, 0.0], [1.0, 3.0, 2.0, 9.0]], dtype=torch.float32, device="cuda")
+    ix = torch.tensor([[0, 5, 2, -1], [1, 0, 3, -1]], dtype=torch.int32, device="cuda")
+    off = torch.tensor([0, 100], dtype=torch.int32, device="cuda")
+    out = torch.full((5,), -7, dtype=torch.int32, device="cuda")
+    osc = torch.zeros(5, dtype=torch.float32, device="cuda")
+    pv.pivot_merge_topk(sc, ix, 5, out, osc, seg_offset=off)
+    torch.cuda.synchronize()
+    got = sorted(zip((-osc).tolist(), out.tolist()))
+    assert [p for _, p in got] == [0, 100, 103, 2, 5]          # 3.0 @0, 3.0 @100, 2.0 @103, then the 1.0 tie: 2, 5 (101 is sixth)
+    out7 = torch.full((7,), -7, dtype=torch.int32, device="cuda")
+    pv.pivot_merge_topk(sc, ix, 7, out7, seg_offset=off)
+    torch.cuda.synchronize()
+    assert sorted(out7.tolist()) == [-1, 0, 2, 5, 100, 101, 103]
+
+
 # ---------------------------------------------------------------- bounded device waits
 
 def test_bounded_wait_runs_out_and_reports_without_hanging(pv, gu):
