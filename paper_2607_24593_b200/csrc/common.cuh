@@ -41,6 +41,20 @@ __device__ __forceinline__ void set_status(int* status, int code) {
   if (status) atomicCAS(status, 0, code);
 }
 
+// Checked build (-DPIVOT_DEBUG): indices the kernels derive themselves -- gathered candidate
+// positions, block-table entries, score / entry slots -- are tested before use; a failed test
+// records DEV_BOUNDS in the status word and the access is skipped.  Nothing traps.  (Positions
+// that come from the caller are tested in every build.)
+#ifdef PIVOT_DEBUG
+__device__ __forceinline__ bool bounds_ok(bool ok, int* status) {
+  if (!ok) set_status(status, DEV_BOUNDS);
+  return ok;
+}
+#define PIVOT_BOUNDS(cond, status) ::pivot::bounds_ok((cond), (status))
+#else
+#define PIVOT_BOUNDS(cond, status) (true)
+#endif
+
 // One row of a scan: a (proxy or raw) query of H x d codes, its gates, and where the
 // selection goes.  Filled by the host-side planner kernels.
 struct RowDesc {

@@ -143,6 +143,7 @@ decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         // Row of the tile inside the key tensor.  Paged cache: the sequence's block table names
         // the pool page (a page outside the pool reads as zero fill, like any out-of-range box).
         const int32_t* pages = prox[b].pages;
+        (void)PIVOT_BOUNDS(t * TILE_KEYS < Lmax, status);              // checked build: the tile lies inside the sequence's rows
         const int krow = pages ? __ldg(pages + t) * TILE_KEYS : prox[b].k_row0 + t * TILE_KEYS;
         const int s = it % C::STAGES;
         if (!ptx::mbar_wait(&ct.empty[s], ((it / C::STAGES) & 1) ^ 1, abort_flag, 64)) break;
@@ -263,7 +264,7 @@ decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       float sv = ((ap[0] + an[0]) + (ap[1] + an[1])) + ((ap[2] + an[2]) + (ap[3] + an[3]));
       if (C::FP8) sv *= ksv;
       const int s_key = t * TILE_KEYS + key_in_tile;
-      if (s_key < n_vis) {
+      if (s_key < n_vis && PIVOT_BOUNDS(s_key < Lmax, status)) {
         scores[(size_t)b * Lmax + s_key] = sv;
         atomicAdd(&ct.hist[set][score_to_key(sv) >> (32 - DHIST_BITS)], 1u);
       }

@@ -39,6 +39,9 @@ struct GroupDesc {
   // Per-query window slots (decode form of Appendix B): the member at position t takes a slot
   // only if t - win_span < position <= t.  The default never excludes anything below t.
   int win_span = 1 << 30;
+  // Largest key position a candidate of this group may name (the group's last member); the
+  // gather drops anything beyond it and reports DEV_BOUNDS.
+  int pos_max = 0x7fffffff;
 };
 
 constexpr int kDecodeWinMax = 512;      // most window slots (W + g - 1) of a decode step

@@ -72,6 +72,7 @@ __global__ void plan_prefill_kernel(PrefillPlan p, RowDesc* rows, GroupDesc* gro
       gd.m = m;
       gd.K = p.k;
       gd.first_pos = t0;
+      gd.pos_max = t0 + m - 1;
       gd.q_row = t0;
       gd.out = p.out + (size_t)t0 * p.k;
       gd.out_score = p.out_score ? p.out_score + (size_t)t0 * p.k : nullptr;

@@ -76,6 +76,7 @@ __device__ __forceinline__ bool plan_decode_sequence(const DecodePlan& p, int b,
   gd.m = p.g;
   gd.K = p.k;
   gd.first_pos = p0;
+  gd.pos_max = p0 + p.g - 1;
   gd.q_row = b * p.g;
   gd.out = outb;
   gd.out_score = outsb;

@@ -272,13 +272,20 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       // Candidate positions are fetched three tiles ahead, their rows in the key tensor (a
       // block-table lookup when the cache is paged) two tiles ahead and key scales one tile
       // ahead, so no round trip sits on this thread's issue path.
+      // A candidate position beyond the group's last member (gd.pos_max) cannot come from the scan; it can come
+      // from a caller-supplied candidate set.  Such a slot is dropped like a padding slot and the
+      // status word says so (tested in every build: the gather must never leave the cache).
+      const int pos_limit = gd.pos_max;
       auto load_idx = [&](int tile, int half) -> int {
         const int sl = tile * TILE_KEYS + wrow0 + half * 32 + lane;
-        return (tile < ntiles && sl < gd.n_cand) ? __ldg(gd.cand + sl) : -1;
+        const int ix = (tile < ntiles && sl < gd.n_cand) ? __ldg(gd.cand + sl) : -1;
+        if (ix > pos_limit || ix < -1) { set_status(sc.status, DEV_BOUNDS); return -1; }
+        return ix;
       };
       auto key_row = [&](int ix) -> int {      // -1: padding slot, or a page outside the pool
         if (!gd.pages || ix < 0) return ix;
         const uint32_t pg = (uint32_t)__ldg(gd.pages + (ix >> 7));
+        (void)PIVOT_BOUNDS(pg < (uint32_t)gd.n_pages, sc.status);     // checked build: a hole in the block table is reported
         return pg < (uint32_t)gd.n_pages ? (int)(pg * 128u + (uint32_t)(ix & 127)) : -1;
       };
       auto load_ks = [&](int row) -> float { return (gd.kscale && row >= 0) ? __ldg(gd.kscale + row) : 1.f; };
@@ -387,12 +394,13 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         const int t_r = gd.first_pos + r;
         const bool seen = idx >= 0 && idx <= t_r && idx + gd.win_span > t_r;
         if (smem_sel) {                // key only; the position is looked up again at the end
-          if (r < gd.m) skey[r * SCORE_SLOTS + slot] = seen ? key : 0u;
+          if (r < gd.m && PIVOT_BOUNDS(slot >= 0 && slot < SCORE_SLOTS, sc.status)) skey[r * SCORE_SLOTS + slot] = seen ? key : 0u;
           return;
         }
         const entry_t e = seen ? make_entry(key, idx) : kPadEntry;
         if (gd.ent_out) {              // chunked mode: leave the entries for a later top-k
-          if (r < gd.m && slot < gd.n_cand) gd.ent_out[(size_t)r * gd.ent_stride + gd.slot0 + slot] = e;
+          if (r < gd.m && slot < gd.n_cand && PIVOT_BOUNDS(gd.slot0 + slot < gd.ent_stride, sc.status))
+            gd.ent_out[(size_t)r * gd.ent_stride + gd.slot0 + slot] = e;
         } else if (r < gd.m && t * 32 + lane < SEG) {
           sc.cand64[seg_off(r) + t * 32 + lane] = e;   // entry t*32+lane of segment (r, lane quarter)
         }

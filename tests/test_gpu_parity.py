@@ -557,6 +557,72 @@ def test_merge_topk_ties_and_empty_slots(pv):
     assert sorted(out7.tolist()) == [-1, 0, 2, 5, 100, 101, 103]
 
 
+# ---------------------------------------------------------------- bounds checks
+
+def test_candidate_from_the_caller_outside_the_sequence_is_dropped_and_reported(pv, gu):
+    """pivot_opts.cand_in is the one place where key positions come from outside: an entry beyond the
+    sequence must not be gathered (the read would leave the cache); it is dropped and the status word
+    reads DEV_BOUNDS.  The other rows are unaffected."""
+    x = inputs.make_decode(2, 2, 1500, 2000, dtype="fp8", seed=83)
+    d = gu.to_cuda(x)
+    Lmax = x.k.shape[1]
+    ref, _, rcand, _ = gu.run_decode(x, c=256, k=128, mode=po.MODE_REFINE, guard_len=0)
+    cand = torch.from_numpy(rcand).cuda().contiguous()
+    out = torch.full((2, 2, 128), -7, dtype=torch.int32, device="cuda")
+    run = lambda: pv.pivot_index_decode(d["q"], d["w"], d["k"], d["pos0"], 2, Lmax, 64, 128, 2, 256, 128, pv.REFINE, out,
+                                        q_scale=d["qscale"], k_scale=d["kscale"], guard_len=0, cand_in=cand)
+    run()
+    torch.cuda.synchronize()
+    assert pv.pivot_device_status() == 0
+    assert np.array_equal(np.sort(out.cpu().numpy(), axis=2), np.sort(ref, axis=2))
+    bad = int(cand[1, 7])
+    cand[1, 7] = 5_000_000                        # far outside the cache
+    run()
+    torch.cuda.synchronize()
+    assert pv.pivot_device_status() == pv.DEV_BOUNDS
+    o = out.cpu().numpy()
+    assert np.array_equal(np.sort(o[0], axis=1), np.sort(ref[0], axis=1))
+    assert (o[1] != 5_000_000).all() and (o[1] >= -1).all()
+    assert set(o[1, 0][o[1, 0] >= 0].tolist()) <= set(rcand[1].tolist()) - {bad}
+
+
+def test_checked_build_runs_the_small_parity_cases_clean():
+    """The -DPIVOT_DEBUG build of the same sources (bounds checks on gathered positions, block-table
+    entries, score and entry slots; a failed check sets DEV_BOUNDS and skips the access): small
+    prefill / decode / paged cases in a process of its own -- oracle parity and a clean status word."""
+    import os
+    import subprocess
+    import sys
+    from paper_2607_24593_b200 import build
+    lib = build.build_variant("debug", ["-DPIVOT_DEBUG"])
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = """
+import sys
+sys.path.insert(0, %r); sys.path.insert(0, %r)
+import torch, gpu_util
+from oracle import acceptance as acc, pivot_oracle as po
+from paper_2607_24593_b200 import binding as pv, inputs
+assert pv.LIB_PATH.endswith('libpivot_debug.so')
+for dtype in ('bf16', 'fp8'):
+    x = inputs.make_prefill(1100, dtype=dtype, seed=91)
+    for mode in (po.MODE_REUSE, po.MODE_REFINE):
+        out, sc, cand, cs = gpu_util.run_prefill(x, g=4, c=256, k=128, mode=mode, W=4 if mode else 0)
+        acc.check_prefill(x.codes(), g=4, c=256, k=128, mode=mode, guard_len=None, out_idx=out, out_scores=sc, cand=cand,
+                          cand_scores=cs, W=4 if mode else 0)
+    xd = inputs.make_decode(3, 2, 300, 2600, dtype=dtype, seed=92)
+    out, sc, cand, cs = gpu_util.run_decode(xd, c=256, k=128, mode=po.MODE_REFINE, W=4)
+    acc.check_decode(xd.codes(), c=256, k=128, mode=po.MODE_REFINE, guard_len=None, out_idx=out, out_scores=sc, cand=cand,
+                     cand_scores=cs, W=4)
+    out, sc, cand, cs = gpu_util.run_decode_paged(xd, c=256, k=128, mode=po.MODE_REFINE, seed=3)
+    acc.check_decode(xd.codes(), c=256, k=128, mode=po.MODE_REFINE, guard_len=0, out_idx=out, out_scores=sc, cand=cand,
+                     cand_scores=cs)
+print('checked build ok')
+""" % (root, os.path.join(root, "tests"))
+    env = dict(os.environ, PIVOT_LIB=os.path.basename(lib))
+    r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0 and "checked build ok" in r.stdout, r.stdout[-2000:] + r.stderr[-4000:]
+
+
 # ---------------------------------------------------------------- bounded device waits
 
 def test_bounded_wait_runs_out_and_reports_without_hanging(pv, gu):
