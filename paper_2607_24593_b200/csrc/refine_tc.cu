@@ -268,21 +268,22 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       const GroupDesc gd = groups[gi];
       const int ntiles = group_tiles(gd);
       if (ntiles == 0) continue;
-      const size_t krow_bytes = gd.k_stride > 0 ? (size_t)gd.k_stride : (size_t)C::ROW_BYTES;   // padded cache rows
+      const int krow_bytes = gd.k_stride > 0 ? gd.k_stride : C::ROW_BYTES;   // padded cache rows (32-bit: one wide multiply per address)
       // Candidate positions are fetched three tiles ahead, their rows in the key tensor (a
       // block-table lookup when the cache is paged) two tiles ahead and key scales one tile
       // ahead, so no round trip sits on this thread's issue path.
-      // A candidate position beyond the group's last member (gd.pos_max) cannot come from the scan; it can come
-      // from a caller-supplied candidate set.  Such a slot is dropped like a padding slot and the
-      // status word says so (tested in every build: the gather must never leave the cache).
       const int pos_limit = gd.pos_max;
       auto load_idx = [&](int tile, int half) -> int {
         const int sl = tile * TILE_KEYS + wrow0 + half * 32 + lane;
-        const int ix = (tile < ntiles && sl < gd.n_cand) ? __ldg(gd.cand + sl) : -1;
-        if (ix > pos_limit || ix < -1) { set_status(sc.status, DEV_BOUNDS); return -1; }
-        return ix;
+        return (tile < ntiles && sl < gd.n_cand) ? __ldg(gd.cand + sl) : -1;
       };
+      // A candidate position beyond the group's last member (gd.pos_max) cannot come from the scan; it
+      // can come from a caller-supplied candidate set.  Such a slot is dropped like a padding slot and
+      // the status word says so (tested in every build: the gather must never leave the cache).  The
+      // test sits here, a pipeline stage after the load of the position, so that it does not wait
+      // for that load.
       auto key_row = [&](int ix) -> int {      // -1: padding slot, or a page outside the pool
+        if (ix > pos_limit || ix < -1) { set_status(sc.status, DEV_BOUNDS); return -1; }
         if (!gd.pages || ix < 0) return ix;
         const uint32_t pg = (uint32_t)__ldg(gd.pages + (ix >> 7));
         (void)PIVOT_BOUNDS(pg < (uint32_t)gd.n_pages, sc.status);     // checked build: a hole in the block table is reported
@@ -316,7 +317,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
           const int rl = i * 4 + sub;                  // row inside this warp's 64
           const int kr = __shfl_sync(0xffffffffu, krow[i >> 3], rl & 31);
           const int row = wrow0 + rl;
-          const uint8_t* src = (const uint8_t*)gd.kbase + (size_t)kr * krow_bytes + chunk * 16;
+          const uint8_t* src = (const uint8_t*)gd.kbase + (long long)kr * krow_bytes + chunk * 16;
           const uint32_t dst = dst0 + (uint32_t)row * 128u + (uint32_t)((chunk ^ (row & 7)) << 4);
 #pragma unroll
           for (int h = 0; h < C::KHALVES; ++h) cp_async16(dst + h * C::HALF_TILE_BYTES, src + h * 128);

@@ -15,7 +15,11 @@ constexpr int KS_SLOTS = 12;      // key-scale ring: deeper than (key stages + a
 #ifndef PIVOT_CHK
 #define PIVOT_CHK 32
 #endif
-constexpr int kThresholdRefreshTiles = PIVOT_CHK;   // the append warp re-reads its row's threshold off the histogram this often
+constexpr int kThresholdRefreshTiles = PIVOT_CHK;
+#ifndef PIVOT_COMPACT_EVERY
+#define PIVOT_COMPACT_EVERY 0
+#endif
+constexpr int kCompactEveryTiles = PIVOT_COMPACT_EVERY;   // a multiple of the refresh interval, or 0 = never   // the append warp re-reads its row's threshold off the histogram this often
 
 // Block sequence of one CTA: blocks sorted longest-first are dealt in snake order.
 struct BlockIter {
@@ -121,9 +125,15 @@ __device__ __noinline__ void append_role(SelectCtrl<NROWS, QD>& s, int r, int la
       if (K > 0 && t > 0 && (t % CHK) == 0) {
         const uint32_t th = hist_threshold(K, base);
         thr = th > thr ? th : thr;
-        if (cnt + headroom > CAP) {
-          // nearly full: drop what fell below the threshold; if that is not enough (ties,
-          // adversarial order) compact exactly to the K best
+        // Housekeeping while this warp has slack: every kCompactEveryTiles tiles the entries that fell
+        // below the threshold leave the segment, so that the final selection at the end of the block
+        // (which stalls the whole pipeline) reads a segment of about K entries instead of
+        // K (1 + ln(n / K)).  They lie below every bin the final boundary can be in, so the histogram
+        // stays exact for what the selection looks at.
+        const bool tidy = kCompactEveryTiles > 0 && (t % kCompactEveryTiles) == 0 && cnt > K + K / 2;
+        if (cnt + headroom > CAP || tidy) {
+          // (nearly full: the same filter; if that is not enough -- ties, adversarial order -- compact
+          // exactly to the K best)
           const uint32_t tcur = thr;
           cnt = seg_filter_inplace(seg, cnt, lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
           if (cnt + headroom > CAP && cnt > K) {
