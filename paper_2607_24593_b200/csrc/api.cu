@@ -408,11 +408,10 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
   p.status = ws.status;
   p.W = W;
   const long long k_rows = paged ? (long long)n_pages * 128 : (long long)(dense_share ? B / dense_share : B) * Lmax;
-  if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 3 * sizeof(int), st)))) return rc;   // status, row counter, prepare ticket
+  if ((rc = check_cuda(cudaMemsetAsync(ws.status, 0, 2 * sizeof(int), st)))) return rc;   // status, row counter
   mark(0, st);
-  if (!dense_share)
-    launch_proxy_build(q->data, q->scale, w, ws.proxy_q, ws.proxy_w, B * g, g, 0, B, q->dtype,
-                       o ? o->pool : 0, st);
+  if (!dense_share && o && o->impl == 1)       // the tensor-core path builds the proxies inside its prepare kernel
+    launch_proxy_build(q->data, q->scale, w, ws.proxy_q, ws.proxy_w, B * g, g, 0, B, q->dtype, o->pool, st);
   mark(1, st);
   if (o && o->impl == 1) launch_plan_decode(p, ws.rows, ws.groups, st);   // the tensor-core path plans inside its prepare kernel
   mark(2, st);
@@ -421,7 +420,7 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
   } else {
     // proxy rows: key-tile-split scan, per-sequence select, chunked re-score, final top-k
     DecodeFast df;
-    df.plan = p; df.ticket = ws.status + 2;
+    df.plan = p; df.pool = o ? o->pool : 0;
     df.prox = ws.rows; df.groups = ws.groups;
     df.kc = kcache->data; df.kscale = kcache->scale; df.q = q->data; df.proxy_q = dense_share ? q->data : ws.proxy_q;
     df.B = B; df.Lmax = Lmax; df.g = g; df.c = c; df.k = k; df.mode = mode; df.dtype = q->dtype;

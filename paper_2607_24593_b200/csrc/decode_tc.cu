@@ -29,6 +29,7 @@
 #include "blockselect.cuh"
 #include "kernels.h"
 #include "plan.cuh"
+#include "proxy_math.cuh"
 #include "ptx.cuh"
 
 namespace pivot {
@@ -444,69 +445,72 @@ merge_topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ 
 
 // ------------------------------------------------------------------------------ setup
 
-// One launch prepares a decode step: block b clears sequence b's histogram and list counters and
-// plans the sequence (row and group descriptors, guard test on the device-resident pos0); the
-// block that finishes last -- nobody waits for anybody -- then has every descriptor in front of
-// it and derives what spans sequences: the tile prefix of the key-split scan, the candidate
-// chunks of the re-score and the entry lists of the final top-k.  1024 threads per block.
+// One launch prepares a decode step; block b does everything that concerns sequence b and nobody
+// waits for anybody: it clears the sequence's histogram and list counters, plans the sequence (row
+// and group descriptors, guard test on the device-resident pos0), builds its proxy (Eq. 4), finds
+// its place in the tile order of the key-split scan (the tile counts of the sequences before it,
+// recomputed from their pos0 -- a few loads instead of a hand-over between blocks), and writes its
+// candidate chunks for the re-score and its entry lists for the final top-k.  1024 threads per block.
+__device__ __forceinline__ int decode_live_tiles(const DecodePlan& p, int b) {
+  // tiles of sequence b's proxy scan, as plan_decode_sequence decides them: 0 for a guarded
+  // sequence and for a pos0 outside the cache
+  const int p_in = p.pos0[b / p.kv_share];
+  const int step = p.g > p.kv_share ? p.g : p.kv_share;
+  if (p_in < 0 || p_in > p.Lmax - step) return 0;
+  const int n0 = p_in + b % p.kv_share + 1;
+  return n0 < p.guard_len ? 0 : (n0 + TILE_KEYS - 1) / TILE_KEYS;
+}
+
 __global__ void __launch_bounds__(1024)
-decode_prepare_kernel(DecodePlan p, RowDesc* rows, GroupDesc* plan_groups, uint32_t* ghist, int* ticket, int W,
+decode_prepare_kernel(DecodePlan p, RowDesc* rows, GroupDesc* plan_groups, uint32_t* ghist, int W, int pool,
                       int* tile_prefix, GroupDesc* chunks, EntryList* lists, unsigned long long* entries,
                       const int32_t* wcand) {
-  {
-    const int b = blockIdx.x;
-    for (int i = threadIdx.x; i < DHIST; i += blockDim.x) ghist[(size_t)b * DHIST + i] = 0u;
-    if (threadIdx.x < 2) ghist[(size_t)p.B * DHIST + 2 * b + threadIdx.x] = 0u;      // list length, delivered shares
-    __shared__ int is_last, seq_ok;
-    if (threadIdx.x == 0) seq_ok = plan_decode_sequence(p, b, rows, plan_groups) ? 1 : 0;
-    __syncthreads();
-    if (!seq_ok) fill_decode_rows_empty(p, b, threadIdx.x, blockDim.x);     // pos0 outside the cache: rows of -1
-    if (p.raw_q) raw_query_gates(p, b, threadIdx.x, blockDim.x);
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) is_last = atomicAdd(ticket, 1) == (int)gridDim.x - 1;
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-    if (threadIdx.x == 0) *ticket = 0;              // ready for the next step
-  }
-  const RowDesc* prox = rows;
-  const GroupDesc* groups = plan_groups;
-  const int B = p.B, g = p.g, c = p.c, k = p.k, mode = p.mode;
-  // tile_prefix = exclusive prefix sum of the sequences' tile counts (any B: 1024 at a time)
-  __shared__ int wsum[32];
-  __shared__ int carry;
+  const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  if (tid == 0) carry = 0;
-  __syncthreads();
-  for (int b0 = 0; b0 < B; b0 += 1024) {
-    const int b = b0 + tid;
-    const int v = (b < B && prox[b].K > 0) ? (prox[b].n_vis + TILE_KEYS - 1) / TILE_KEYS : 0;
-    int incl = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int u = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += u;
-    }
-    if (lane == 31) wsum[wid] = incl;
-    __syncthreads();
-    int base = carry;
-    for (int w = 0; w < wid; ++w) base += wsum[w];
-    if (b < B) tile_prefix[b] = base + incl - v;
-    __syncthreads();
-    if (tid == 1023) carry = base + incl;
-    __syncthreads();
+  const int B = p.B, g = p.g, c = p.c, k = p.k, mode = p.mode;
+  for (int i = tid; i < DHIST; i += blockDim.x) ghist[(size_t)b * DHIST + i] = 0u;
+  if (tid < 2) ghist[(size_t)B * DHIST + 2 * b + tid] = 0u;      // list length, delivered shares
+  __shared__ int seq_ok;
+  __shared__ int wsum[32];
+  if (tid == 0) seq_ok = plan_decode_sequence(p, b, rows, plan_groups) ? 1 : 0;
+  // ---- tiles of the sequences before this one
+  int part = 0;
+  for (int bb = tid; bb < b; bb += blockDim.x) part += decode_live_tiles(p, bb);
+  part = __reduce_add_sync(0xffffffffu, part);
+  if (lane == 0) wsum[wid] = part;
+  __syncthreads();                                 // also: the descriptors thread 0 wrote are visible to the block
+  if (tid == 0) {
+    int before = 0;
+    for (int i = 0; i < 32; ++i) before += wsum[i];
+    tile_prefix[b] = before;
+    if (b == B - 1) tile_prefix[B] = before + decode_live_tiles(p, b);
   }
-  if (tid == 0) tile_prefix[B] = carry;
+  if (!seq_ok) fill_decode_rows_empty(p, b, tid, blockDim.x);     // pos0 outside the cache: rows of -1
+  if (p.raw_q) {
+    raw_query_gates(p, b, tid, blockDim.x);
+  } else {
+    // ---- the sequence's proxy: one warp per unit of four (e4m3) or two (bf16) heads
+    if (p.dtype == DT_FP8) {
+      for (int u = wid; u < proxy_units_per_group<DT_FP8>(); u += 32)
+        proxy_build_unit<DT_FP8>(p.q, p.qscale, p.w, p.proxy_q, p.proxy_w, B * g, g, 0, B, pool,
+                                 (long long)b * proxy_units_per_group<DT_FP8>() + u, lane);
+    } else {
+      for (int u = wid; u < proxy_units_per_group<DT_BF16>(); u += 32)
+        proxy_build_unit<DT_BF16>(p.q, p.qscale, p.w, p.proxy_q, p.proxy_w, B * g, g, 0, B, pool,
+                                  (long long)b * proxy_units_per_group<DT_BF16>() + u, lane);
+    }
+  }
   if (mode != 1) return;
   // Refine: split every (sequence, member chunk) into candidate chunks so all SMs re-score,
   // each leaving packed entries; one entry list per query for the final top-k.
+  const GroupDesc* groups = plan_groups;
   const int mc = (g + kMembersPerDesc - 1) / kMembersPerDesc;
   const int ncc = (c + kDecodeCandChunk - 1) / kDecodeCandChunk;
   const int nch = ncc + (W > 0 ? 1 : 0);           // with a window: one more chunk, the window slots
   const int w_g = W > 0 ? W + g - 1 : 0;
   const int stride = c + kDecodeWinMax;            // entries per query
-  for (int i = tid; i < B * mc * nch; i += blockDim.x) {
+  for (int j = tid; j < mc * nch; j += blockDim.x) {
+    const int i = b * mc * nch + j;
     const int gi = i / nch, cc = i % nch;
     GroupDesc gd = groups[gi];
     gd.ent_out = entries + (size_t)gd.q_row * stride;
@@ -524,15 +528,15 @@ decode_prepare_kernel(DecodePlan p, RowDesc* rows, GroupDesc* plan_groups, uint3
     }
     chunks[i] = gd;
   }
-  for (int i = tid; i < B * g; i += blockDim.x) {
-    const int b = i / g;
+  for (int j = tid; j < g; j += blockDim.x) {
+    const int i = b * g + j;
     const GroupDesc gd = groups[b * mc];
     EntryList el;
     el.list = entries + (size_t)i * stride;
     el.n = gd.n_cand > 0 ? gd.n_cand + w_g : 0;
     el.K = gd.n_cand > 0 ? k : 0;
-    el.out = groups[b * mc].out + (size_t)(i - b * g) * gd.out_stride;
-    el.out_score = gd.out_score ? groups[b * mc].out_score + (size_t)(i - b * g) * gd.out_stride : nullptr;
+    el.out = groups[b * mc].out + (size_t)j * gd.out_stride;
+    el.out_score = gd.out_score ? groups[b * mc].out_score + (size_t)j * gd.out_stride : nullptr;
     lists[i] = el;
   }
 }
@@ -622,7 +626,7 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   int32_t* wcand = (int32_t*)p;              p += up((size_t)d.B * kDecodeWinMax * 4);
   unsigned long long* entries = (unsigned long long*)p;
 
-  decode_prepare_kernel<<<d.B, 1024, 0, st>>>(d.plan, d.prox, d.groups, ghist, d.ticket, W, tile_prefix, chunks, lists,
+  decode_prepare_kernel<<<d.B, 1024, 0, st>>>(d.plan, d.prox, d.groups, ghist, W, d.pool, tile_prefix, chunks, lists,
                                               entries, wcand);
   ++launch_counter();
   cudaError_t e = cudaGetLastError();

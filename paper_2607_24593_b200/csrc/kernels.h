@@ -139,7 +139,7 @@ cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDe
 // Decode fast path: key-tile-split scan -> per-sequence select -> chunked re-score -> top-k.
 struct DecodeFast {
   DecodePlan plan;            // the call's geometry: the prepare kernel plans the sequences itself
-  int* ticket;                // one zeroed int (counts the prepare kernel's finished blocks)
+  int pool = 0;               // proxy aggregation (the prepare kernel builds the proxies)
   RowDesc* prox;              // [B + B * g] row slots; [0, B) = proxy rows (K = 0: guarded sequence, skipped)
   GroupDesc* groups;          // [B * group_chunks(g)]
   const void* kc; const float* kscale; const void* q; const void* proxy_q;
