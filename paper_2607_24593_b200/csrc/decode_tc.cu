@@ -462,7 +462,7 @@ __device__ __forceinline__ int decode_live_tiles(const DecodePlan& p, int b) {
 }
 
 __global__ void __launch_bounds__(1024)
-decode_prepare_kernel(DecodePlan p, RowDesc* rows, GroupDesc* plan_groups, uint32_t* ghist, int W, int pool,
+decode_prepare_kernel(DecodePlan p, RowDesc* rows, GroupDesc* plan_groups, uint32_t* ghist, int W, int pool, int chunk,
                       int* tile_prefix, GroupDesc* chunks, EntryList* lists, unsigned long long* entries,
                       const int32_t* wcand) {
   const int b = blockIdx.x;
@@ -505,7 +505,7 @@ decode_prepare_kernel(DecodePlan p, RowDesc* rows, GroupDesc* plan_groups, uint3
   // each leaving packed entries; one entry list per query for the final top-k.
   const GroupDesc* groups = plan_groups;
   const int mc = (g + kMembersPerDesc - 1) / kMembersPerDesc;
-  const int ncc = (c + kDecodeCandChunk - 1) / kDecodeCandChunk;
+  const int ncc = (c + chunk - 1) / chunk;
   const int nch = ncc + (W > 0 ? 1 : 0);           // with a window: one more chunk, the window slots
   const int w_g = W > 0 ? W + g - 1 : 0;
   const int stride = c + kDecodeWinMax;            // entries per query
@@ -516,10 +516,10 @@ decode_prepare_kernel(DecodePlan p, RowDesc* rows, GroupDesc* plan_groups, uint3
     gd.ent_out = entries + (size_t)gd.q_row * stride;
     gd.ent_stride = stride;
     if (cc < ncc) {
-      const int left = gd.n_cand - cc * kDecodeCandChunk;
-      gd.cand = gd.cand + cc * kDecodeCandChunk;
-      gd.n_cand = left > 0 ? (left < kDecodeCandChunk ? left : kDecodeCandChunk) : 0;
-      gd.slot0 = cc * kDecodeCandChunk;
+      const int left = gd.n_cand - cc * chunk;
+      gd.cand = gd.cand + cc * chunk;
+      gd.n_cand = left > 0 ? (left < chunk ? left : chunk) : 0;
+      gd.slot0 = cc * chunk;
     } else {                 // window slots follow the pool's valid entries
       gd.slot0 = gd.n_cand;
       gd.cand = wcand + (size_t)(gi / mc) * kDecodeWinMax;
@@ -618,7 +618,15 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   int* tile_prefix = (int*)p;                p += up((size_t)(d.B + 1) * 4);
   entry_t* glist = (entry_t*)p;              p += up((size_t)d.B * SEL_CAP * 8);
   const int mc = group_chunks(d.g);
-  const int ncc = (d.c + kDecodeCandChunk - 1) / kDecodeCandChunk;
+  // Candidates per re-score work item: as few items as keep every SM busy in ONE wave (each item pays
+  // for its own query load and pipeline ramp), never below kDecodeCandChunk, whole 128-key tiles.
+  int chunk = kDecodeCandChunk;
+  {
+    const int per_group = d.sms / (d.B * mc) > 0 ? d.sms / (d.B * mc) : 1;
+    const int want = ((d.c + per_group - 1) / per_group + TILE_KEYS - 1) / TILE_KEYS * TILE_KEYS;
+    if (want > chunk) chunk = want;
+  }
+  const int ncc = (d.c + chunk - 1) / chunk;
   const int W = d.mode == 1 ? d.W : 0;
   const int nch = ncc + (W > 0 ? 1 : 0);
   GroupDesc* chunks = (GroupDesc*)p;         p += up((size_t)d.B * mc * (ncc + 1) * sizeof(GroupDesc));
@@ -626,7 +634,7 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   int32_t* wcand = (int32_t*)p;              p += up((size_t)d.B * kDecodeWinMax * 4);
   unsigned long long* entries = (unsigned long long*)p;
 
-  decode_prepare_kernel<<<d.B, 1024, 0, st>>>(d.plan, d.prox, d.groups, ghist, W, d.pool, tile_prefix, chunks, lists,
+  decode_prepare_kernel<<<d.B, 1024, 0, st>>>(d.plan, d.prox, d.groups, ghist, W, d.pool, chunk, tile_prefix, chunks, lists,
                                               entries, wcand);
   ++launch_counter();
   cudaError_t e = cudaGetLastError();
