@@ -47,8 +47,8 @@ FLOP_PER_SCORE = 2 * H * D
 # dram__bytes_read.sum + dram__bytes_write.sum per launch: STORED figures from the ncu captures
 # summarised under profiles/ (same workloads as the ones timed here); not re-measured by this run,
 # and labelled so in the line ("traffic_source").
-TRAFFIC_BYTES = {"prefill_128k_fp8_refine_g4": 2780454144 + 4301106432,
-                 "decode_scan_kernel": 403583488 + 12487936}
+TRAFFIC_BYTES = {"prefill_128k_fp8_refine_g4": 2742043648 + 4281856512,
+                 "decode_scan_kernel": 403589888 + 12189440}
 TRAFFIC_SOURCE = "stored ncu capture (profiles/), not re-measured in this run"
 
 
@@ -499,7 +499,7 @@ def main():
 
     if args.mma_model:
         res = {"mma_model": pv.pivot_debug_mma_model(), "key_stream": []}
-        for ctas, stages, mode in ((1, 4, 0), (148, 2, 0), (148, 4, 0), (148, 8, 0), (148, 4, 1), (148, 4, 2), (1, 4, 2)):
+        for ctas, stages, mode in ((1, 4, 0), (148, 2, 0), (148, 4, 0), (148, 12, 0), (148, 4, 1), (148, 4, 2), (1, 4, 2), (148, 4, 3), (148, 4, 4)):
             res["key_stream"].append(pv.pivot_debug_key_stream(ctas=ctas, stages=stages, mode=mode))
         print(json.dumps(res, indent=1))
         return
