@@ -119,6 +119,7 @@ Workspace carve_workspace(void* base, int rows, int n_groups, int c, int k) {
   w.scan.cand_idx = (int32_t*)w.scan.cand64 + simt_entries;
   w.scan.status = w.status;
   w.scan.counter = w.counter;
+  w.scan.rkeys = cv.take<uint32_t>((size_t)sm_count() * 2 * 4 * 4096);
   w.bytes = cv.off;
   return w;
 }
@@ -271,7 +272,7 @@ int run_prefill(const pivot_tensor* q, const float* w, const pivot_tensor* kc, i
     const int nd = p.n_proxy * group_chunks(g);
     if (o && o->impl == 1) launch_refine_simt(ws.groups, nd, q->dtype, ws.scan, st);
     else if ((rc = check_cuda(launch_refine_tc(q->data, L, q->dtype, ws.groups, nd, tc_scratch(ws), sm_count(), st,
-                                               o && o->impl == 2))))
+                                               o && o->impl == 2, false, c))))
       return rc;
   }
   mark(4, st);

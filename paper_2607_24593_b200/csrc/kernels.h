@@ -103,6 +103,7 @@ struct ScanScratch {
   int n_cta;
   int* status;
   int* counter;         // dynamic row scheduler
+  uint32_t* rkeys = nullptr;   // re-score: [SMs][2][4][4096] score keys between the tile loop and the select team
 };
 
 void launch_proxy_build(const void* q, const float* qscale, const float* w, void* proxy_q,
@@ -134,7 +135,7 @@ cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_ro
 
 cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
                              const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum = false,
-                             bool chunked = false);
+                             bool chunked = false, int max_cand = 0);
 
 // Decode fast path: key-tile-split scan -> per-sequence select -> chunked re-score -> top-k.
 struct DecodeFast {

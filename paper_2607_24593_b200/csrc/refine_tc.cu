@@ -9,7 +9,8 @@
 // go to a per-CTA buffer; after the last tile each member's exact top-k is selected from its c
 // scores and written out.
 //
-// Warps: 0 = query TMA, 1 = MMA issuer + TMEM owner, 2-5 = gather producers, 6-13 = epilogue.
+// Warps: 0 = query TMA, 1 = MMA issuer + TMEM owner, 2-3 = gather producers, 4-11 = epilogue,
+// 12-15 (EPI = 3) = select warps, one per member.
 #include <cuda.h>
 
 #include "kernels.h"
@@ -24,17 +25,25 @@ constexpr int MAX_STAGES = 8;
 constexpr int NMEM = 4;                       // members per MMA (N = 256)
 constexpr int GATHER_WARPS = 2;       // each producer thread copies two rows of a tile
 constexpr int EPI_WARPS = 8;
-constexpr int THREADS = (2 + GATHER_WARPS + EPI_WARPS) * 32;   // 384: 168 registers per thread
+constexpr int SEL_WARPS = 4;
 constexpr int N = NMEM * kHeads;
 constexpr int TMEM_COLS = 2 * N;
 
 // EPI: 1 = tensor-core head sum where available (FP8), 0 = fp32 FMA head sum, 2 = as 1 for the
 // candidate chunks of a decode step: those leave packed entries for a later top-k, so the score
 // rows need no shared memory and a second query buffer takes their place (the next chunk's
-// queries load while the current one is re-scored).
+// queries load while the current one is re-scored).  3 = as 1 with the per-member top-k on four
+// warps of their own, one group behind the tile loop: the score rows go through a double buffer
+// in global memory (L2-resident, 128 KB per CTA) instead of shared memory, so the tensor core
+// and the gather keep running while a group's members are selected.  Needs every group of the
+// launch to have at most SCORE_SLOTS candidates.
 template <int DT, int EPI = 1>
 struct RCfg {
   static constexpr bool FP8 = DT == DT_FP8;
+  static constexpr bool OVL = FP8 && EPI == 3;
+  static constexpr int NSEL = OVL ? SEL_WARPS : 2;
+  // 384 threads: 168 registers per thread; 512 (with the select warps): 128
+  static constexpr int THREADS = (2 + GATHER_WARPS + EPI_WARPS + (OVL ? SEL_WARPS : 0)) * 32;
   static constexpr int KHALVES = FP8 ? 1 : 2;
   static constexpr int HALF_TILE_BYTES = TILE_KEYS * 128;
   static constexpr int STAGE_BYTES = KHALVES * HALF_TILE_BYTES;
@@ -44,7 +53,7 @@ struct RCfg {
   // FP8 keeps the group's score keys in shared memory (4 members x 4096 slots x 4 B) for the
   // final top-k; bf16 has no room for that next to 2 x 64 KB of queries and goes through the
   // per-CTA global segments instead.
-  static constexpr bool SMEM_SCORES = FP8 && EPI != 2;
+  static constexpr bool SMEM_SCORES = FP8 && EPI == 1;
   // With the score rows resident, one query buffer (the next group's queries load while the
   // key ring refills) buys two more gather stages, which matter more.
   static constexpr int QBUFS = SMEM_SCORES ? 1 : 2;
@@ -60,6 +69,9 @@ struct RCfg {
   static constexpr int TMEM_EMPTY_ARRIVALS = MMA2 ? 4 : EPI_WARPS;
 };
 
+#ifndef PIVOT_REFINE_OVERLAP
+#define PIVOT_REFINE_OVERLAP 1
+#endif
 constexpr int META_SLOTS = 8;     // key stages in flight (<= 6) + accumulator buffers (2)
 static_assert(META_SLOTS >= 6 + 2, "meta ring");
 constexpr int SCORE_SLOTS = 4096;             // shared-memory score row: candidates per member
@@ -77,7 +89,7 @@ struct KeyMeta {
 // groups is set per slab).
 constexpr int WMAT_BYTES = 5120;
 
-template <bool MMA2>
+template <bool MMA2, int NSEL = 2>
 struct RCtrlT {
   alignas(1024) uint8_t wmat[MMA2 ? WMAT_BYTES : 16];
   uint64_t a_ready[2], s_ready[2], w_ready;      // MMA2 handshakes
@@ -85,18 +97,21 @@ struct RCtrlT {
   KeyMeta meta[META_SLOTS][TILE_KEYS];   // written by the gather warps, read by the epilogue
   uint64_t full[MAX_STAGES], empty[MAX_STAGES];
   uint64_t q_full[2], q_empty[2], tmem_full[2], tmem_empty[2];
+  uint64_t k_full[2], k_free[2];                 // score rows of a group: score warps -> select warps
+  uint32_t kstat[2][NMEM][4];                    // ... and each row's smallest / largest key and filled slots
   uint32_t tmem_base;
   int abort;
-  SegSelSmem sel[2];
+  SegSelSmem sel[NSEL];          // one per selecting team (EPI = 3: per select warp)
 };
 
 template <int DT, int EPI = 1>
 constexpr size_t rsmem_bytes() {
   using C = RCfg<DT, EPI>;
-  return 1024 + C::QBUFS * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(RCtrlT<C::MMA2>) +
+  return 1024 + C::QBUFS * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(RCtrlT<C::MMA2, C::NSEL>) +
          (C::SMEM_SCORES ? (size_t)NMEM * SCORE_SLOTS * 4 : 0);
 }
 static_assert(rsmem_bytes<DT_FP8, 1>() <= 232448 && rsmem_bytes<DT_FP8, 0>() <= 232448 && rsmem_bytes<DT_FP8, 2>() <= 232448 &&
+              rsmem_bytes<DT_FP8, 3>() <= 232448 &&
               rsmem_bytes<DT_BF16>() <= 232448, "shared memory budget");
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -113,7 +128,7 @@ __device__ __forceinline__ int group_tiles(const GroupDesc& gd) {
 }
 
 template <int DT, int EPI>
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__((RCfg<DT, EPI>::THREADS), 1)
 refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __restrict__ groups, int n_groups,
                  int q_rows_total, ScanScratch sc) {
   using C = RCfg<DT, EPI>;
@@ -121,7 +136,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* qbuf = smem;
   uint8_t* kring = smem + C::QBUFS * C::QBUF_BYTES;
-  using RCtrl = RCtrlT<C::MMA2>;
+  using RCtrl = RCtrlT<C::MMA2, C::NSEL>;
   RCtrl& ct = *reinterpret_cast<RCtrl*>(kring + C::STAGES * C::STAGE_BYTES);
   uint32_t* skey = reinterpret_cast<uint32_t*>(kring + C::STAGES * C::STAGE_BYTES + sizeof(RCtrl));   // [NMEM][SCORE_SLOTS]
   volatile int* abort_flag = &ct.abort;
@@ -140,8 +155,15 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       ptx::mbar_init(&ct.tmem_empty[i], C::TMEM_EMPTY_ARRIVALS);
       ptx::mbar_init(&ct.a_ready[i], 4);
       ptx::mbar_init(&ct.s_ready[i], 1);
+      ptx::mbar_init(&ct.k_full[i], 4);
+      ptx::mbar_init(&ct.k_free[i], SEL_WARPS);
     }
     ptx::mbar_init(&ct.w_ready, 1);
+    for (int i = 0; i < 2 * NMEM; ++i) {
+      ct.kstat[i / NMEM][i % NMEM][0] = 0xffffffffu;
+      ct.kstat[i / NMEM][i % NMEM][1] = 0u;
+      ct.kstat[i / NMEM][i % NMEM][2] = 0u;
+    }
     ct.abort = 0;
     ptx::fence_barrier_init();
   }
@@ -331,6 +353,37 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
     }
     cp_async_wait<0>();
     while (pub < it) publish(pub++);
+  } else if (C::OVL && warp >= 2 + GATHER_WARPS + EPI_WARPS) {
+    // ------------------------------------------------------------------ select warps (EPI = 3)
+    // Warp r takes member r's exact top-k of group n while the other warps re-score group n + 1.
+    const int r = warp - (2 + GATHER_WARPS + EPI_WARPS);
+    SegSelSmem& sel = ct.sel[r];
+    const uint32_t* rk = sc.rkeys + (size_t)blockIdx.x * 2 * NMEM * SCORE_SLOTS;
+    uint32_t blk = 0;
+    for (int gi = blockIdx.x; gi < n_groups; gi += gridDim.x) {
+      const GroupDesc gd = groups[gi];
+      const int ntiles = min(group_tiles(gd), SCORE_SLOTS / TILE_KEYS);
+      if (ntiles == 0) continue;
+      const int kb = blk & 1;
+      const uint32_t kph = (blk >> 1) & 1;
+      ++blk;
+      if (!ptx::mbar_wait(&ct.k_full[kb], kph, abort_flag, 64)) break;
+      const uint32_t kmin = ct.kstat[kb][r][0], kmax = ct.kstat[kb][r][1], n_filled = ct.kstat[kb][r][2];
+      __syncwarp();
+      if (lane == 0) { ct.kstat[kb][r][0] = 0xffffffffu; ct.kstat[kb][r][1] = 0u; ct.kstat[kb][r][2] = 0u; }
+      if (r < gd.m) {
+        int32_t* out = gd.out + (size_t)r * gd.out_stride;
+        float* outs = gd.out_score ? gd.out_score + (size_t)r * gd.out_stride : nullptr;
+        const int n_valid = warp_row_topk(sel, rk + (kb * NMEM + r) * SCORE_SLOTS, ntiles * TILE_KEYS, gd.cand,
+                                          gd.n_cand, out, outs, gd.K, lane, kmin, kmax, n_filled);
+        for (int i = n_valid + lane; i < gd.K; i += 32) {
+          out[i] = -1;
+          if (outs) outs[i] = -INFINITY;
+        }
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&ct.k_free[kb]);     // this warp is through with the buffer
+    }
   } else {
     // ------------------------------------------------------------------ epilogue + top-k
     const int ew = warp - (2 + GATHER_WARPS);
@@ -340,17 +393,21 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
     const int tt = (ew & 3) * 32 + lane;
     const Team tm{tt, 128, 1 + team};
     const Team all{ew * 32 + lane, EPI_WARPS * 32, 3};   // both teams
-    SegSelSmem& sel = ct.sel[team];
+    SegSelSmem& sel = ct.sel[C::OVL ? 0 : team];
     const int wq = ew & 3;
     const int SEG = sc.cap >> 2;
     // per-CTA score segments: (member r, warp wq) -> cand64[cta][r][wq][0 .. SEG)
     const size_t cta_base = (size_t)blockIdx.x * NMEM * sc.cap;
     auto seg_off = [&](int r) { return cta_base + ((size_t)r * 4 + wq) * SEG; };
-    uint32_t it = 0;
+    uint32_t it = 0, blk = 0;
+    uint32_t* const rk = C::OVL ? sc.rkeys + (size_t)blockIdx.x * 2 * NMEM * SCORE_SLOTS : nullptr;
     for (int gi = blockIdx.x; gi < n_groups; gi += gridDim.x) {
       const GroupDesc gd = groups[gi];
       const int ntiles = group_tiles(gd);
       if (ntiles == 0) continue;
+      const int kb = blk & 1;                    // score-row buffer of this group (EPI = 3)
+      const uint32_t kph = (blk >> 1) & 1;
+      ++blk;
       const bool smem_sel = C::SMEM_SCORES && !gd.ent_out && ntiles * TILE_KEYS <= SCORE_SLOTS;
       if constexpr (C::MMA2) {
         // team 1 scores all four members (so both teams meet around the tile loop: the other team
@@ -391,9 +448,22 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       // One member row's result: a key never seen by the member (beyond its own position, or
       // before its own window in a chunk of per-query window slots: Appendix B) or a padding
       // slot counts as empty.
+      uint32_t smn[NMEM], smx[NMEM], snv[NMEM];  // EPI = 3: this thread's share of the row statistics
+#pragma unroll
+      for (int r = 0; r < NMEM; ++r) { smn[r] = 0xffffffffu; smx[r] = 0u; snv[r] = 0u; }
       auto put = [&](int r, int t, int slot, int idx, uint32_t key) {
         const int t_r = gd.first_pos + r;
         const bool seen = idx >= 0 && idx <= t_r && idx + gd.win_span > t_r;
+        if constexpr (C::OVL) {        // key only, to this group's score-row buffer
+          if (r < gd.m && slot < SCORE_SLOTS) {
+            const uint32_t kv = seen ? key : 0u;
+            rk[(kb * NMEM + r) * SCORE_SLOTS + slot] = kv;
+            smn[r] = (kv && kv < smn[r]) ? kv : smn[r];
+            smx[r] = kv > smx[r] ? kv : smx[r];
+            snv[r] += kv ? 1u : 0u;
+          }
+          return;
+        }
         if (smem_sel) {                // key only; the position is looked up again at the end
           if (r < gd.m && PIVOT_BOUNDS(slot >= 0 && slot < SCORE_SLOTS, sc.status)) skey[r * SCORE_SLOTS + slot] = seen ? key : 0u;
           return;
@@ -442,6 +512,8 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
           }
         } else {
           // ---- score warps: the four member scores of this thread's key
+          if constexpr (C::OVL)        // the select warps are through with this buffer (two groups back)
+            (void)ptx::mbar_wait(&ct.k_free[kb], kph ^ 1, abort_flag, 64);
           for (int t = 0; t < ntiles; ++t, ++it) {
             const int buf = it & 1;
             const int slot = t * TILE_KEYS + key_in_tile;
@@ -460,6 +532,21 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
               const float sc_r = __uint_as_float(s8[r]) + __uint_as_float(s8[4 + r]);
               put(r, t, slot, mt.idx, score_to_key(gd.kscale ? sc_r * mt.ks : sc_r));
             }
+          }
+          if constexpr (C::OVL) {      // the group's score rows are complete: hand them over
+#pragma unroll
+            for (int r = 0; r < NMEM; ++r) {
+              const uint32_t mn = __reduce_min_sync(0xffffffffu, smn[r]);
+              const uint32_t mx = __reduce_max_sync(0xffffffffu, smx[r]);
+              const uint32_t nv = __reduce_add_sync(0xffffffffu, snv[r]);
+              if (lane == 0 && nv) {
+                atomicMin(&ct.kstat[kb][r][0], mn);
+                atomicMax(&ct.kstat[kb][r][1], mx);
+                atomicAdd(&ct.kstat[kb][r][2], nv);
+              }
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&ct.k_full[kb]);
           }
         }
         all.sync();
@@ -513,7 +600,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       }
       tm.sync();
       }
-      if (gd.ent_out) continue;
+      if (gd.ent_out || C::OVL) continue;
       // ---- per-member exact top-k over the candidate scores
 #pragma unroll
       for (int rl = 0; rl < 2; ++rl) {
@@ -564,7 +651,7 @@ cudaError_t launch_one(const CUtensorMap& mq, const GroupDesc* groups, int n_gro
   const size_t smem = rsmem_bytes<DT, EPI>();
   if (cudaError_t e = opt_in_dynamic_smem(kern, smem, attr_set); e != cudaSuccess) return e;
   const int grid = n_groups < sms ? n_groups : sms;
-  kern<<<grid, THREADS, smem, st>>>(mq, groups, n_groups, q_rows, s);
+  kern<<<grid, RCfg<DT, EPI>::THREADS, smem, st>>>(mq, groups, n_groups, q_rows, s);
   ++launch_counter();
   return cudaGetLastError();
 }
@@ -574,14 +661,18 @@ cudaError_t launch_one(const CUtensorMap& mq, const GroupDesc* groups, int n_gro
 bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtype, int box_rows, int row_stride);
 
 cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
-                             const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum, bool chunked) {
+                             const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum, bool chunked,
+                             int max_cand) {
   if (n_groups <= 0) return cudaSuccess;
   CUtensorMap mq;
   if (!make_operand_map(&mq, q, (long long)q_rows * kHeads, dtype, kHeads, 0)) return cudaErrorInvalidValue;
   if (dtype != DT_FP8) return launch_one<DT_BF16>(mq, groups, n_groups, q_rows, s, sms, st);
   if (fp32_head_sum) return launch_one<DT_FP8, 0>(mq, groups, n_groups, q_rows, s, sms, st);
-  return chunked ? launch_one<DT_FP8, 2>(mq, groups, n_groups, q_rows, s, sms, st)
-                 : launch_one<DT_FP8, 1>(mq, groups, n_groups, q_rows, s, sms, st);
+  if (chunked) return launch_one<DT_FP8, 2>(mq, groups, n_groups, q_rows, s, sms, st);
+  // select overlapped with the next group's tiles where every group's score rows fit the buffers
+  if (PIVOT_REFINE_OVERLAP && s.rkeys && max_cand > 0 && max_cand <= SCORE_SLOTS)
+    return launch_one<DT_FP8, 3>(mq, groups, n_groups, q_rows, s, sms, st);
+  return launch_one<DT_FP8, 1>(mq, groups, n_groups, q_rows, s, sms, st);
 }
 
 }  // namespace pivot

@@ -588,4 +588,123 @@ __device__ __forceinline__ int smem_row_topk(const Team& tm, SegSelSmem& sm, con
   return n_valid < K ? n_valid : K;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Exact top-K of a row of score keys by ONE warp, the row in global memory (written by other
+// warps of the CTA, read through L2).  Slot s holds key keys[s] (0 = empty) and stands for
+// position cand[s] (s < n_cand); the caller knows the smallest and largest filled key and how
+// many slots are filled.  The K best slots under the entry order (key, then the lower position)
+// are found by narrowing a window [lo, hi] of entries: 2048 linear bins over the window, walk
+// from the top to the bin that holds the K-th entry, then either the bin is wanted whole, or it
+// is small enough to rank by brute force, or it becomes the next window (its width shrinks
+// 2048-fold per round, so at most six rounds for 64-bit entries; one round unless many scores
+// tie).  While a bin is wider than 2^32 entries it is a range of keys and the positions are not
+// needed.  The last pass writes every slot above the final bin, lists the bin's own slots and
+// ranks those.  Every pass is a sweep over L2 with U slots per lane in flight: their number is
+// what the select costs.  Writes the selected positions unordered; returns how many:
+// min(K, filled slots).  nslots is a multiple of 32.
+template <int U, bool NEED_POS, typename F>
+__device__ __forceinline__ void warp_row_pass(const uint32_t* keys, int nslots, const int32_t* __restrict__ cand,
+                                              int n_cand, int lane, F f) {
+  for (int s0 = 0; s0 < nslots; s0 += 32 * U) {
+    uint32_t k[U];
+    int ps[U];
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+      const int sl = s0 + j * 32 + lane;
+      k[j] = sl < nslots ? __ldcg(keys + sl) : 0u;
+      ps[j] = (NEED_POS && sl < n_cand) ? __ldg(cand + sl) : -1;
+    }
+    // slots past the end read as empty; no test per slot here, so that the U bodies are one
+    // basic block and their latencies overlap
+#pragma unroll
+    for (int j = 0; j < U; ++j) f(k[j], ps[j]);
+  }
+}
+
+static __device__ __noinline__ int warp_row_topk(SegSelSmem& sm, const uint32_t* keys, int nslots,
+                                                 const int32_t* __restrict__ cand, int n_cand, int32_t* out,
+                                                 float* out_score, int K, int lane, uint32_t kmin, uint32_t kmax,
+                                                 uint32_t n_filled) {
+  const uint32_t lt = (1u << lane) - 1u;
+  // the final bin [blo, bhi]: slots above it go out, its own are ranked unless it is wanted whole
+  entry_t blo = 1ull, bhi = 0ull;            // n_filled <= K: every filled slot is "above"
+  uint32_t need_b = 0;
+  bool whole = false;
+  if (n_filled > (uint32_t)K) {
+    entry_t lo = (entry_t)kmin << 32, hi = ((entry_t)kmax << 32) | 0xffffffffull;
+    uint32_t need = (uint32_t)K;
+    for (int round = 0; round < 8; ++round) {
+      const entry_t span = hi - lo;
+      const int bits = 64 - __clzll((long long)(span | 1ull));
+      const int shift = bits > 11 ? bits - 11 : 0;
+      for (int i = lane; i < kSelBins / 4; i += 32) reinterpret_cast<uint4*>(sm.hist)[i] = make_uint4(0, 0, 0, 0);
+      __syncwarp();
+      if (shift >= 32) {                     // bins are key ranges
+        const uint32_t klo = (uint32_t)(lo >> 32), khi = (uint32_t)(hi >> 32);
+        const int ksh = shift - 32;
+        warp_row_pass<32, false>(keys, nslots, cand, n_cand, lane, [&](uint32_t k, int) {
+          if (k >= klo && k <= khi && k) atomicAdd(&sm.hist[(k - klo) >> ksh], 1u);
+        });
+      } else {
+        warp_row_pass<16, true>(keys, nslots, cand, n_cand, lane, [&](uint32_t k, int ps) {
+          const entry_t e = make_entry(k, ps);
+          if (k && e >= lo && e <= hi) atomicAdd(&sm.hist[(uint32_t)((e - lo) >> shift)], 1u);
+        });
+      }
+      __syncwarp();
+      uint32_t b, pop;
+      warp_hist_boundary(sm.hist, need, lane, &b, &need_b, &pop);
+      blo = lo + ((entry_t)b << shift);
+      bhi = shift ? blo + (((entry_t)1 << shift) - 1ull) : blo;
+      bhi = bhi < hi ? bhi : hi;
+      whole = pop == need_b;
+      if (whole || pop <= (uint32_t)kSelSmall) break;
+      lo = blo; hi = bhi; need = need_b;     // crowded bin (ties): it is the next window
+    }
+  }
+  // Straight-line body: one predicated store per slot (a divergent branch per slot, with its
+  // reconvergence, cost several hundred clocks a slot); the scores, when asked for, take a
+  // sweep of their own afterwards.
+  uint32_t base = 0, ln = 0;
+  if (whole) blo -= 1ull, bhi = blo;         // "above the bin" then includes the bin; nothing is listed
+  const entry_t elo = whole ? ~0ull : blo;   // listed: elo <= e <= bhi
+  warp_row_pass<16, true>(keys, nslots, cand, n_cand, lane, [&](uint32_t k, int ps) {
+    const entry_t e = k ? make_entry(k, ps) : 0ull;
+    const bool em = e > bhi;
+    const bool edge = e >= elo && e <= bhi;
+    const uint32_t m = __ballot_sync(0xffffffffu, em);
+    const uint32_t me = __ballot_sync(0xffffffffu, edge);
+    const uint32_t p = base + __popc(m & lt);
+    const uint32_t q = ln + __popc(me & lt);
+    if (em && p < (uint32_t)K) out[p] = ps;
+    if (edge && q < (uint32_t)kSelSmall) sm.list[q] = e;
+    base += __popc(m);
+    ln += __popc(me);
+  });
+  if (out_score) {
+    uint32_t b2 = 0;
+    warp_row_pass<16, true>(keys, nslots, cand, n_cand, lane, [&](uint32_t k, int ps) {
+      const bool em = (k ? make_entry(k, ps) : 0ull) > bhi;
+      const uint32_t m = __ballot_sync(0xffffffffu, em);
+      const uint32_t p = b2 + __popc(m & lt);
+      if (em && p < (uint32_t)K) out_score[p] = key_to_score(k);
+      b2 += __popc(m);
+    });
+  }
+  __syncwarp();
+  ln = ln < (uint32_t)kSelSmall ? ln : (uint32_t)kSelSmall;
+  for (uint32_t t = lane; t < ln; t += 32) {                      // entries are distinct: ranks are slots
+    const entry_t xt = sm.list[t];
+    uint32_t rank = 0;
+    for (uint32_t u = 0; u < ln; ++u) rank += sm.list[u] > xt ? 1u : 0u;
+    if (rank < need_b && base + rank < (uint32_t)K) {
+      out[base + rank] = entry_pos(xt);
+      if (out_score) out_score[base + rank] = key_to_score(entry_key(xt));
+    }
+  }
+  __syncwarp();
+  const uint32_t n_out = base + (ln < need_b ? ln : need_b);
+  return (int)(n_out < (uint32_t)K ? n_out : (uint32_t)K);
+}
+
 }  // namespace pivot
