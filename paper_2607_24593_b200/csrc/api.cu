@@ -113,7 +113,7 @@ Workspace carve_workspace(void* base, int rows, int n_groups, int c, int k) {
   w.scan.cap = cand_cap(kmax);
   w.tc_cap = tc_cap(kmax);
   const size_t simt_entries = (size_t)w.scan.n_cta * 2 * w.scan.cap;
-  const size_t tc_entries = (size_t)sm_count() * 4 * w.tc_cap;
+  const size_t tc_entries = (size_t)sm_count() * 4 * 2 * w.tc_cap;     // two segments per row (alternate blocks)
   w.scan.cand64 = cv.take<unsigned long long>(simt_entries > tc_entries ? simt_entries : tc_entries);
   w.scan.cand_key = (uint32_t*)w.scan.cand64;
   w.scan.cand_idx = (int32_t*)w.scan.cand64 + simt_entries;

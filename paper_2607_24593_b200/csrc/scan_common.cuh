@@ -1,7 +1,8 @@
-// Parts shared by the shared-scan kernels (scan_tc.cu, scan_i8.cu): the order in which a CTA
-// takes its row blocks, and the streaming select behind the scan (Eq. 6 / Eq. 7) -- survivor
-// queues between the warps that produce scores and one append warp per row, the row histogram
-// that keeps the running threshold, the row's candidate segment, and the final exact selection.
+// Parts of the shared-scan kernel (scan_tc.cu): the order in which a CTA takes its row blocks,
+// and the streaming select behind the scan (Eq. 6 / Eq. 7) -- survivor queues between the warps
+// that produce scores and one append warp per row, the row histogram that keeps the running
+// threshold, the row's candidate segment, and the final exact selection, which finisher warps
+// take one block behind the scan (a row has two segments, used by alternate blocks).
 #pragma once
 #include "kernels.h"
 #include "ptx.cuh"
@@ -11,7 +12,7 @@ namespace pivot {
 namespace scan {
 
 constexpr int TILE_KEYS = 128;
-constexpr int KS_SLOTS = 12;      // key-scale ring: deeper than (key stages + accumulator buffers)
+constexpr int KS_SLOTS = 8;       // key-scale ring: deeper than (key stages + accumulator buffers)
 #ifndef PIVOT_CHK
 #define PIVOT_CHK 32
 #endif
@@ -59,13 +60,34 @@ struct SelectCtrl {
   uint64_t sc_full[QD], sc_empty[QD];   // survivor queues: score warps -> append warps
   alignas(16) unsigned long long q[QD][NROWS][4][32];   // [tile % QD][row][lane quarter]: packed entries
   alignas(16) uint32_t qn[QD][NROWS][4];                // their counts
-  volatile uint32_t thr[NROWS];         // published append threshold of each row (only grows)
-  int rowcnt[NROWS];                    // end of a block: entries held in the row's segment
-  int rowbase[NROWS];                   // ... the row histogram's anchor
-  uint32_t rowthr[NROWS];               // ... and the row's final threshold
+  // published append threshold of each row, (block sequence number << 32) | key: only grows
+  // within a block; a reader that is already in the next block sees a stale tag and takes 0
+  volatile unsigned long long thr[NROWS];
+  // End of a block: what the row's finisher needs (the append warp moves on to the next block
+  // and the row's other segment at once).  Two slots, used by alternate blocks like the segments.
+  struct FinRow {
+    int cnt;                            // entries held in the row's segment
+    int base;                           // the row histogram's anchor
+    int bsel;                           // boundary bin of the exact histogram, -1 = everything is wanted
+    uint32_t need_b, pop;               // entries wanted from that bin, and its population
+  } fin[NROWS][2];
+  uint64_t fin_full[NROWS][2], fin_done[NROWS][2];   // append warp -> finisher -> append warp
   int abort_code;                       // device status to report besides a timed-out wait
-  SegSelSmem sel[NROWS];                // one per append warp (and per final selection)
+  SegSelSmem sel[NROWS];                // the row's append warp (segment overflow) or its finisher
 };
+
+// The threshold the score warps of block sequence number `seq` compare row r's scores with.
+template <int NROWS, int QD>
+__device__ __forceinline__ uint32_t row_threshold(const SelectCtrl<NROWS, QD>& s, int r, uint32_t seq) {
+  const unsigned long long t = s.thr[r];
+  return (uint32_t)(t >> 32) == seq ? (uint32_t)t : 0u;
+}
+
+// Row r's segment for the block with sequence number seq.
+template <int NROWS>
+__device__ __forceinline__ entry_t* row_segment(const ScanScratch& sc, int r, uint32_t seq) {
+  return sc.cand64 + (((size_t)blockIdx.x * NROWS + r) * 2 + (seq & 1u)) * sc.cap;
+}
 
 // A score warp leaves the survivors of its 32 keys of row r in the tile's queue: compacted by one
 // vote, count beside them.  `take` must already include the causal cut and the threshold test.
@@ -86,15 +108,15 @@ __device__ __forceinline__ int select_bin(uint32_t key, int base) {
 
 // The append warp of row r (one warp, all blocks of this CTA): counts the survivors of every tile
 // in the row histogram, moves them to the row's segment in the L2-resident scratch and keeps the
-// row's threshold fresh -- alone, without barriers.  `rdv` is the barrier it shares with the
-// warps that take the row's final selection at the end of a block.
+// row's threshold fresh -- alone, without barriers.  At the end of a block it reads the boundary
+// bin off the (then exact) histogram, hands the segment to the row's finisher and goes on with
+// the next block in the row's other segment.
 template <int NROWS, int QD>
-__device__ __noinline__ void append_role(SelectCtrl<NROWS, QD>& s, int r, int lane, const Team& tm, const Team& rdv,
+__device__ __noinline__ void append_role(SelectCtrl<NROWS, QD>& s, int r, int lane, const Team& tm,
                                             const RowDesc* __restrict__ rows, int n_rows, int n_blocks,
                                             const ScanScratch& sc, volatile int* abort_flag) {
   SegSelSmem& sel = s.sel[r];
   const int CAP = sc.cap;                        // entries of this row's candidate segment
-  entry_t* const seg = sc.cand64 + ((size_t)blockIdx.x * NROWS + r) * CAP;
   uint32_t* const rhist = s.rhist[r];
   // Lower bound on the K-th best score seen so far, read off the row histogram: the largest
   // bin edge with at least K scores at or above it.  Returned as a key threshold t such that
@@ -109,7 +131,7 @@ __device__ __noinline__ void append_role(SelectCtrl<NROWS, QD>& s, int r, int la
   const int CHK = CAP / (2 * TILE_KEYS) < kThresholdRefreshTiles ? (CAP / (2 * TILE_KEYS) > 0 ? CAP / (2 * TILE_KEYS) : 1) : kThresholdRefreshTiles;
   const int headroom = TILE_KEYS * CHK;
   BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
-  uint32_t it = 0;
+  uint32_t it = 0, seq = 0;
   for (int b = bi.next(); b >= 0; b = bi.next()) {
     int k_row0 = 0;
     const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0);
@@ -120,6 +142,12 @@ __device__ __noinline__ void append_role(SelectCtrl<NROWS, QD>& s, int r, int la
     int cnt = 0, base = 0;
     uint32_t thr = 0;
     for (int i = lane; i < kSelBins; i += 32) rhist[i] = 0;
+    if (lane == 0) s.thr[r] = (unsigned long long)seq << 32;
+    // this block's segment was the block's before last: its finisher must be through with it
+    const int fb = seq & 1;
+    (void)ptx::mbar_wait(&s.fin_done[r][fb], ((seq >> 1) & 1) ^ 1, abort_flag, 64);
+    entry_t* const seg = row_segment<NROWS>(sc, r, seq);
+    bool sel_mine = seq == 0;                    // the finisher of the previous block may still use `sel`
     __syncwarp();
     for (int t = 0; t < ntiles; ++t, ++it) {
       if (K > 0 && t > 0 && (t % CHK) == 0) {
@@ -137,12 +165,16 @@ __device__ __noinline__ void append_role(SelectCtrl<NROWS, QD>& s, int r, int la
           const uint32_t tcur = thr;
           cnt = seg_filter_inplace(seg, cnt, lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
           if (cnt + headroom > CAP && cnt > K) {
+            if (!sel_mine) {                     // (rare path: waiting here costs nothing that matters)
+              (void)ptx::mbar_wait(&s.fin_done[r][fb ^ 1], ((seq - 1) >> 1) & 1, abort_flag, 64);
+              sel_mine = true;
+            }
             entry_t cut;
             cnt = seg_compact<false>(tm, sel, Seg{seg, cnt}, K, &cut);
             thr = entry_key(cut) > thr ? entry_key(cut) : thr;
           }
         }
-        if (lane == 0) s.thr[r] = thr;
+        if (lane == 0) s.thr[r] = ((unsigned long long)seq << 32) | thr;
       }
       const int sb = it % QD;
       (void)ptx::mbar_wait(&s.sc_full[sb], (it / QD) & 1, abort_flag);
@@ -177,53 +209,63 @@ __device__ __noinline__ void append_role(SelectCtrl<NROWS, QD>& s, int r, int la
       }
       cnt = min(cnt + (int)(nq[0] + nq[1] + nq[2] + nq[3]), CAP);
     }
-    // ---- end of the block: hand the row to its final select, wait until it is done
-    if (lane == 0) { s.rowcnt[r] = cnt; s.rowbase[r] = base; s.rowthr[r] = thr; }
+    // ---- end of the block: the histogram is exact for everything the segment still holds; read
+    //      the boundary bin off it and hand the row to its finisher
+    uint32_t bb = 0, need_b = 0, pop = 0;
+    const bool found = K > 0 && warp_hist_boundary<0>(rhist, (uint32_t)K, lane, &bb, &need_b, &pop);
+    if (lane == 0) {
+      typename SelectCtrl<NROWS, QD>::FinRow& f = s.fin[r][fb];
+      f.cnt = cnt; f.base = base; f.bsel = found ? (int)bb : -1; f.need_b = need_b; f.pop = pop;
+    }
+    __threadfence_block();
     __syncwarp();
-    rdv.sync();
-    if (lane == 0) s.thr[r] = 0u;             // the next block starts from scratch (read after the barrier below)
-    rdv.sync();
+    if (lane == 0) ptx::mbar_arrive(&s.fin_full[r][fb]);
+    ++seq;
   }
 }
 
-// Final exact selection of row r of block b by a team of four warps (128 threads; warp wq of the
-// team takes the wq-th quarter of the row's segment): the append warp has counted every entry it
-// holds, so the row histogram is exact and one pass over the segment suffices; a boundary bin too
-// crowded to rank takes the general path.  Pads the row with -1 and copies it to the other
-// members of a Reuse group.  Call between the two `rdv` barriers of the append warp.
+// A finisher warp: the final exact selection of rows r0 .. r0 + nr - 1 of every block of this CTA,
+// one block behind the scan.  The append warp has counted every entry the segment holds, so its
+// boundary bin is exact and one sweep over the segment suffices (a boundary bin too crowded to
+// rank takes the general way).  Pads the row with -1 and copies it to the other members of a
+// Reuse group.
 template <int NROWS, int QD>
-__device__ __noinline__ void final_select_row(SelectCtrl<NROWS, QD>& s, const Team& tm, int r, int K, const RowDesc& rd,
-                                                 const ScanScratch& sc) {
-  if (K <= 0) return;
-  const int tt = tm.tid, lane = tt & 31, wq = tt >> 5;
-  SegSelSmem& sel = s.sel[r];               // the row's append warp is idle now
-  entry_t* const seg = sc.cand64 + ((size_t)blockIdx.x * NROWS + r) * sc.cap;
-  const int total = s.rowcnt[r];
-  const int rbase = s.rowbase[r];
-  const int lo = (int)(((long long)total * wq) >> 2), hi = (int)(((long long)total * (wq + 1)) >> 2);
-  int mine = hi - lo;                        // this warp's slice of the row segment
-  auto key_bin = [rbase](uint32_t key) { return select_bin(key, rbase); };
-  int n_valid = seg_emit_hist(tm, sel, Seg{seg + lo, mine}, s.rhist[r], key_bin, rd.out, rd.out_score, K);
-  if (n_valid < 0) {
-    const uint32_t tcur = s.rowthr[r];
-    mine = seg_filter_inplace(seg + lo, mine, lane, [tcur](entry_t x) { return entry_key(x) > tcur; });
-    tm.sync();
-    if (tt == 0) sel.total = 0;
-    tm.sync();
-    if (lane == 0) atomicAdd(&sel.total, (uint32_t)mine);
-    tm.sync();
-    n_valid = seg_emit<false>(tm, sel, Seg{seg + lo, mine}, (int)sel.total, rd.out, rd.out_score, K);
-  }
-  for (int i = n_valid + tt; i < K; i += 128) {
-    rd.out[i] = -1;
-    if (rd.out_score) rd.out_score[i] = -INFINITY;
-  }
-  tm.sync();
-  for (int rr = 1; rr < rd.out_rows; ++rr)
-    for (int i = tt; i < K; i += 128) {
-      rd.out[(size_t)rr * rd.out_stride + i] = rd.out[i];
-      if (rd.out_score) rd.out_score[(size_t)rr * rd.out_stride + i] = rd.out_score[i];
+__device__ __noinline__ void finisher_role(SelectCtrl<NROWS, QD>& s, int r0, int nr, int lane,
+                                              const RowDesc* __restrict__ rows, int n_rows, int n_blocks,
+                                              const ScanScratch& sc, volatile int* abort_flag) {
+  BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
+  uint32_t seq = 0;
+  for (int b = bi.next(); b >= 0; b = bi.next()) {
+    int k_row0 = 0;
+    if (block_tiles(rows, n_rows, b, NROWS, &k_row0) == 0) continue;
+    const int fb = seq & 1;
+    for (int r = r0; r < r0 + nr; ++r) {
+      if (!ptx::mbar_wait(&s.fin_full[r][fb], (seq >> 1) & 1, abort_flag, 64)) return;
+      const int ri = b * NROWS + r;
+      const int K = (ri < n_rows) ? rows[ri].K : 0;
+      if (K > 0) {
+        const RowDesc rd = rows[ri];
+        const typename SelectCtrl<NROWS, QD>::FinRow f = s.fin[r][fb];
+        const int rbase = f.base;
+        auto key_bin = [rbase](uint32_t key) { return select_bin(key, rbase); };
+        const int n_valid = warp_seg_topk_binned(s.sel[r], row_segment<NROWS>(sc, r, seq), f.cnt, key_bin, f.bsel,
+                                                 f.need_b, f.pop, rd.out, rd.out_score, K, lane);
+        for (int i = n_valid + lane; i < K; i += 32) {
+          rd.out[i] = -1;
+          if (rd.out_score) rd.out_score[i] = -INFINITY;
+        }
+        __syncwarp();
+        for (int rr = 1; rr < rd.out_rows; ++rr)
+          for (int i = lane; i < K; i += 32) {
+            rd.out[(size_t)rr * rd.out_stride + i] = rd.out[i];
+            if (rd.out_score) rd.out_score[(size_t)rr * rd.out_stride + i] = rd.out_score[i];
+          }
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&s.fin_done[r][fb]);
     }
+    ++seq;
+  }
 }
 
 }  // namespace scan

@@ -19,8 +19,10 @@
 // barriers.  Splitting the epilogue this way puts more warps on every scheduler within the
 // register file (the score warps carry no select state) and takes the histogram atomics, the
 // global stores and the threshold refresh off the warps that feed the tensor core.  At the end
-// of a block the score-warp teams (128 threads per pair of rows) do the final exact select.
-// Row blocks are dealt to CTAs longest-first in snake order.
+// of a block the append warp hands its row's segment to a FINISHER warp (one per two rows), which
+// takes the final exact select while the other warps are already scanning the next block (a row
+// has two segments, used by alternate blocks).  Row blocks are dealt to CTAs longest-first in
+// snake order.
 //
 // FP8 with four rows per block (the prefill configuration) takes the gate-weighted head sum of
 // Eq. 5 on the tensor core as well: it is the contraction ReLU(X) [128 keys x 256] . W^T with a
@@ -68,8 +70,8 @@ struct Cfg {
   static constexpr int ROWS_PER_TEAM = NROWS == 4 ? 2 : 1;
   static constexpr int TEAMS = EPI_WARPS / 4;
   static constexpr int SEL_WARPS = NROWS;                     // append warps, one per row
-  static constexpr int RDV_THREADS = 128 + ROWS_PER_TEAM * 32; // a team plus the append warps of its rows
-  static constexpr int THREADS = 64 + (EPI_WARPS + SEL_WARPS) * 32;
+  static constexpr int FIN_WARPS = NROWS == 4 ? 2 : 1;        // finisher warps, one per two rows
+  static constexpr int THREADS = 64 + (EPI_WARPS + SEL_WARPS + FIN_WARPS) * 32;
   static constexpr int TMEM_COLS = 2 * N < 32 ? 32 : 2 * N;
   // FP8, four rows: the gate-weighted head sum itself runs on the tensor core (see the kernel
   // header).  Other configurations keep the fp32 FMA epilogue.
@@ -153,7 +155,10 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     }
     ct.abort = 0;
     ct.s.abort_code = 0;
-    for (int r = 0; r < NROWS; ++r) ct.s.thr[r] = 0u;
+    for (int r = 0; r < NROWS; ++r) {
+      ct.s.thr[r] = 0ull;
+      for (int i = 0; i < 2; ++i) { ptx::mbar_init(&ct.s.fin_full[r][i], 1); ptx::mbar_init(&ct.s.fin_done[r][i], 1); }
+    }
     ptx::fence_barrier_init();
   }
   if (warp == 1) {
@@ -296,15 +301,15 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     const int key_in_tile = lq * 32 + lane;
     const int tt = wq * 32 + lane;                 // rank inside the team (0..127)
     const Team tm{tt, 128, 1 + team};
-    const Team rdv{0, C::RDV_THREADS, 7 + team};   // this team and the append warps of its rows
     BlockIter bi(n_blocks, gridDim.x, blockIdx.x);
-    uint32_t it = 0;
+    uint32_t it = 0, seq = 0xffffffffu;            // seq: this block's sequence number in the CTA
     // A failed wait never changes this role's control flow (the team barriers below must stay
     // matched); once the abort flag is up every later wait returns at once.
     for (int b = bi.next(); b >= 0; b = bi.next()) {
       int k_row0 = 0;
       const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0);
       if (ntiles == 0) continue;
+      ++seq;
       // ---- effective gates of this team's rows
       tm.sync();
       if constexpr (C::MMA2) {
@@ -344,13 +349,12 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
           ct.w[r][j] = 0.5f * wv;       // halved: see the ReLU identity below
         }
       }
-      int n_vis[C::ROWS_PER_TEAM], Ksel[C::ROWS_PER_TEAM];
+      int n_vis[C::ROWS_PER_TEAM];
 #pragma unroll
       for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
         const int ri = b * NROWS + team * C::ROWS_PER_TEAM + rl;
         const bool live = ri < n_rows && rows[ri].K > 0;
         n_vis[rl] = live ? rows[ri].n_vis : 0;
-        Ksel[rl] = live ? rows[ri].K : 0;
       }
       tm.sync();
       if constexpr (C::MMA2) {
@@ -421,7 +425,7 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
 #pragma unroll
             for (int r = 0; r < NROWS; ++r) {
               const uint32_t key = score_to_key((__uint_as_float(sv[r]) + __uint_as_float(sv[4 + r])) * ksv);
-              scan::push_survivors(ct.s, qb, r, lq, lane, s_key < nv4[r] && key > ct.s.thr[r], key, s_key);
+              scan::push_survivors(ct.s, qb, r, lq, lane, s_key < nv4[r] && key > scan::row_threshold(ct.s, r, seq), key, s_key);
             }
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&ct.s.sc_full[qb]);
@@ -492,28 +496,22 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
           const int r = team * C::ROWS_PER_TEAM + rl;
           const uint32_t key = score_to_key(C::FP8 ? score[rl] * ksv : score[rl]);
-          scan::push_survivors(ct.s, qb, r, lq, lane, s_key < n_vis[rl] && key > ct.s.thr[r], key, s_key);
+          scan::push_survivors(ct.s, qb, r, lq, lane, s_key < n_vis[rl] && key > scan::row_threshold(ct.s, r, seq), key, s_key);
         }
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&ct.s.sc_full[qb]);
       }
-      // ---- end of the block: the team takes the final exact select of its rows.  The append
-      //      warps have counted every entry they hold, so the row histogram is exact and one pass
-      //      over the segment suffices; a boundary bin too crowded to rank takes the general path.
-      rdv.sync();                                  // append warps are done with the last tile
-#pragma unroll
-      for (int rl = 0; rl < C::ROWS_PER_TEAM; ++rl) {
-        const int r = team * C::ROWS_PER_TEAM + rl;
-        const int ri = b * NROWS + r;
-        if (Ksel[rl] > 0) scan::final_select_row(ct.s, tm, r, Ksel[rl], rows[ri], sc);
-      }
-      rdv.sync();                                  // rows' histograms and segments may be reused
+      // (the rows' final exact select is the finisher warps' business: on to the next block)
     }
-  } else {
+  } else if (warp < 2 + C::EPI_WARPS + C::SEL_WARPS) {
     // ------------------------------------------------------------------ append warps: one row each
     const int r = warp - 2 - C::EPI_WARPS;
-    scan::append_role(ct.s, r, lane, Team{lane, 32, 3 + r}, Team{0, C::RDV_THREADS, 7 + r / C::ROWS_PER_TEAM}, rows, n_rows,
-                      n_blocks, sc, abort_flag);
+    scan::append_role(ct.s, r, lane, Team{lane, 32, 3 + r}, rows, n_rows, n_blocks, sc, abort_flag);
+  } else {
+    // ------------------------------------------------------------------ finisher warps
+    const int f = warp - 2 - C::EPI_WARPS - C::SEL_WARPS;
+    constexpr int RPF = NROWS / C::FIN_WARPS;
+    scan::finisher_role(ct.s, f * RPF, RPF, lane, rows, n_rows, n_blocks, sc, abort_flag);
   }
   // ------------------------------------------------------------------ teardown
   ptx::tc_fence_before();

@@ -363,85 +363,6 @@ __device__ __forceinline__ int seg_emit(const Team& tm, SegSelSmem& sm, const Se
   return n_out > K ? K : n_out;
 }
 
-// Final selection of a row straight from its score histogram: `hist` counted every entry that
-// was ever appended and bin_of(key) is the bin it was counted in.  Entries in bins above the
-// boundary bin are emitted in one pass over the segments; the boundary bin's entries are ranked
-// by brute force.  Returns how many positions were written (K, or fewer when the segments hold
-// fewer than K), or -1 when the boundary bin holds more than kSelSmall entries (the caller then
-// takes the general path; `out` may hold partial results).  All threads of the team call, after
-// a team barrier that follows the last append.
-template <typename BinFn>
-__device__ __forceinline__ int seg_emit_hist(const Team& tm, SegSelSmem& sm, const Seg& seg, const uint32_t* hist,
-                                             BinFn bin_of, int32_t* out, float* out_score, int K) {
-  const int lane = tm.tid & 31;
-  uint32_t b = 0, need_b = 0, pop = 0;
-  const bool found = warp_hist_boundary<0>(hist, (uint32_t)K, lane, &b, &need_b, &pop);
-  const int bsel = found ? (int)b : -1;
-  if (tm.tid == 0) { sm.out_count = 0; sm.list_n = 0; }
-  tm.sync();
-  for (int j0 = 0; j0 < seg.cnt; j0 += 256) {        // eight rows of 32 in flight
-    entry_t x[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int i = j0 + u * 32 + lane;
-      x[u] = i < seg.cnt ? __ldcg(seg.e + i) : kPadEntry;
-    }
-    // one cursor bump per batch: the eight votes first, then a single atomic for their total
-    uint32_t m[8];
-    uint32_t batch = 0;
-    uint32_t emit_bits = 0;
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const bool valid = (j0 + u * 32 + lane) < seg.cnt && entry_pos(x[u]) >= 0;
-      const int bn = (int)bin_of(entry_key(x[u]));
-      const bool emit = valid && bn > bsel;
-      m[u] = __ballot_sync(0xffffffffu, emit);
-      batch += (uint32_t)__popc(m[u]);
-      emit_bits |= emit ? 1u << u : 0u;
-      if (valid && bn == bsel) {
-        const uint32_t q = atomicAdd(&sm.list_n, 1u);
-        if (q < (uint32_t)kSelSmall) sm.list[q] = x[u];
-      }
-    }
-    if (batch) {
-      uint32_t pos = 0;
-      if (lane == 0) pos = atomicAdd(&sm.out_count, batch);
-      pos = __shfl_sync(0xffffffffu, pos, 0);
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        if ((emit_bits >> u) & 1u) {
-          const uint32_t p = pos + __popc(m[u] & ((1u << lane) - 1u));
-          if (p < (uint32_t)K) {
-            out[p] = entry_pos(x[u]);
-            if (out_score) out_score[p] = key_to_score(entry_key(x[u]));
-          }
-        }
-        pos += (uint32_t)__popc(m[u]);
-      }
-    }
-  }
-  tm.sync();
-  if (found) {
-    const uint32_t P = sm.list_n;
-    if (P > (uint32_t)kSelSmall) return -1;
-    for (uint32_t t = tm.tid; t < P; t += tm.nthr) {
-      const entry_t xt = sm.list[t];
-      uint32_t rank = 0;
-      for (uint32_t u = 0; u < P; ++u) rank += sm.list[u] > xt ? 1u : 0u;
-      if (rank < need_b) {
-        const uint32_t p = atomicAdd(&sm.out_count, 1u);
-        if (p < (uint32_t)K) {
-          out[p] = entry_pos(xt);
-          if (out_score) out_score[p] = key_to_score(entry_key(xt));
-        }
-      }
-    }
-    tm.sync();
-  }
-  const int n = (int)sm.out_count;
-  return n < K ? n : K;
-}
-
 // Exact top-K of a row of score keys held in shared memory (0 = padding slot); the position of
 // slot s is cand[s] (s < n_cand).  One linear 2048-bin histogram over the row's key range finds
 // the boundary bin; the slots above it are emitted in a second pass and the boundary bin's
@@ -589,49 +510,133 @@ __device__ __forceinline__ int smem_row_topk(const Team& tm, SegSelSmem& sm, con
 }
 
 // ---------------------------------------------------------------------------------------------
-// Exact top-K of a row of score keys by ONE warp, the row in global memory (written by other
-// warps of the CTA, read through L2).  Slot s holds key keys[s] (0 = empty) and stands for
-// position cand[s] (s < n_cand); the caller knows the smallest and largest filled key and how
-// many slots are filled.  The K best slots under the entry order (key, then the lower position)
-// are found by narrowing a window [lo, hi] of entries: 2048 linear bins over the window, walk
-// from the top to the bin that holds the K-th entry, then either the bin is wanted whole, or it
-// is small enough to rank by brute force, or it becomes the next window (its width shrinks
-// 2048-fold per round, so at most six rounds for 64-bit entries; one round unless many scores
-// tie).  While a bin is wider than 2^32 entries it is a range of keys and the positions are not
-// needed.  The last pass writes every slot above the final bin, lists the bin's own slots and
-// ranks those.  Every pass is a sweep over L2 with U slots per lane in flight: their number is
-// what the select costs.  Writes the selected positions unordered; returns how many:
-// min(K, filled slots).  nslots is a multiple of 32.
-template <int U, bool NEED_POS, typename F>
-__device__ __forceinline__ void warp_row_pass(const uint32_t* keys, int nslots, const int32_t* __restrict__ cand,
-                                              int n_cand, int lane, F f) {
-  for (int s0 = 0; s0 < nslots; s0 += 32 * U) {
-    uint32_t k[U];
-    int ps[U];
+// Exact top-K by ONE warp over entries that lie in global memory (written by other warps of the
+// CTA, read through L2): the rows of score keys the re-score kernel leaves per member, and the
+// candidate segments of the shared scan.  A source sweeps its entries past a functor, U per lane
+// in flight (0 = empty slot).  The sweeps are what the select costs: their bodies carry no branch
+// per entry (a uniform test per entry, let alone a divergent one, makes every entry a basic block
+// of its own and exposes each vote's and each load's latency in turn: measured 320 clocks per
+// entry against 40).
+//
+// The K best entries under the entry order (key, then the lower position) are found by
+// narrowing a window [lo, hi]: 2048 linear bins over the window, walk from the top to the bin
+// that holds the K-th entry, then either the bin is wanted whole, or it is small enough to rank
+// by brute force, or it becomes the next window (its width shrinks 2048-fold per round, so at
+// most six rounds for 64-bit entries; one round unless many scores tie).  While a bin is wider
+// than 2^32 entries it is a range of keys and a source that has to look positions up need not.
+// The last sweep writes every entry above the final bin, lists the bin's own and ranks those.
+// Positions are written unordered; the functions return how many: min(K, entries).
+
+// A row of score keys: slot s holds keys[s] (0 = empty) and stands for position cand[s]
+// (s < n_cand); nslots is a multiple of 32.
+struct KeyRowSrc {
+  static constexpr bool kKeysApart = true;       // keys can be swept without their positions
+  const uint32_t* keys;
+  int nslots;
+  const int32_t* __restrict__ cand;
+  int n_cand;
+  template <int U, typename F>
+  __device__ __forceinline__ void sweep_keys(int lane, F f) const {
+    for (int s0 = 0; s0 < nslots; s0 += 32 * U) {
+      uint32_t k[U];
 #pragma unroll
-    for (int j = 0; j < U; ++j) {
-      const int sl = s0 + j * 32 + lane;
-      k[j] = sl < nslots ? __ldcg(keys + sl) : 0u;
-      ps[j] = (NEED_POS && sl < n_cand) ? __ldg(cand + sl) : -1;
+      for (int j = 0; j < U; ++j) {
+        const int sl = s0 + j * 32 + lane;
+        k[j] = sl < nslots ? __ldcg(keys + sl) : 0u;
+      }
+#pragma unroll
+      for (int j = 0; j < U; ++j) f(k[j]);
     }
-    // slots past the end read as empty; no test per slot here, so that the U bodies are one
-    // basic block and their latencies overlap
-#pragma unroll
-    for (int j = 0; j < U; ++j) f(k[j], ps[j]);
   }
+  template <int U, bool NEED_POS, typename F>
+  __device__ __forceinline__ void sweep(int lane, F f) const {
+    for (int s0 = 0; s0 < nslots; s0 += 32 * U) {
+      uint32_t k[U];
+      int ps[U];
+#pragma unroll
+      for (int j = 0; j < U; ++j) {
+        const int sl = s0 + j * 32 + lane;
+        k[j] = sl < nslots ? __ldcg(keys + sl) : 0u;
+        ps[j] = (NEED_POS && sl < n_cand) ? __ldg(cand + sl) : -1;
+      }
+#pragma unroll
+      for (int j = 0; j < U; ++j) f(k[j] ? make_entry(k[j], ps[j]) : 0ull);   // without positions: low word 0
+    }
+  }
+};
+
+// A segment of packed entries (padding entries, position -1, count as empty).
+struct SegSrc {
+  static constexpr bool kKeysApart = false;
+  const entry_t* e;
+  int cnt;
+  template <int U, bool NEED_POS, typename F>
+  __device__ __forceinline__ void sweep(int lane, F f) const {
+    for (int i0 = 0; i0 < cnt; i0 += 32 * U) {
+      entry_t x[U];
+#pragma unroll
+      for (int j = 0; j < U; ++j) {
+        const int i = i0 + j * 32 + lane;
+        x[j] = i < cnt ? __ldcg(e + i) : 0ull;
+      }
+#pragma unroll
+      for (int j = 0; j < U; ++j) f(entry_pos(x[j]) >= 0 ? x[j] : 0ull);
+    }
+  }
+};
+
+// Last sweep: entries above bhi go out, those in [elo, bhi] are listed and the need_b best of
+// the list follow.  elo > bhi: nothing is listed.
+template <typename Src>
+__device__ __forceinline__ int warp_emit_above(SegSelSmem& sm, const Src& src, entry_t elo, entry_t bhi, uint32_t need_b,
+                                               int32_t* out, float* out_score, int K, int lane) {
+  const uint32_t lt = (1u << lane) - 1u;
+  uint32_t base = 0, ln = 0;
+  src.template sweep<16, true>(lane, [&](entry_t e) {
+    const bool em = e > bhi;
+    const bool edge = e >= elo && e <= bhi;
+    const uint32_t m = __ballot_sync(0xffffffffu, em);
+    const uint32_t me = __ballot_sync(0xffffffffu, edge);
+    const uint32_t p = base + __popc(m & lt);
+    const uint32_t q = ln + __popc(me & lt);
+    if (em && p < (uint32_t)K) out[p] = entry_pos(e);
+    if (edge && q < (uint32_t)kSelSmall) sm.list[q] = e;
+    base += __popc(m);
+    ln += __popc(me);
+  });
+  if (out_score) {                           // the scores, when asked for, take a sweep of their own
+    uint32_t b2 = 0;
+    src.template sweep<16, true>(lane, [&](entry_t e) {
+      const bool em = e > bhi;
+      const uint32_t m = __ballot_sync(0xffffffffu, em);
+      const uint32_t p = b2 + __popc(m & lt);
+      if (em && p < (uint32_t)K) out_score[p] = key_to_score(entry_key(e));
+      b2 += __popc(m);
+    });
+  }
+  __syncwarp();
+  ln = ln < (uint32_t)kSelSmall ? ln : (uint32_t)kSelSmall;
+  for (uint32_t t = lane; t < ln; t += 32) {                      // entries are distinct: ranks are slots
+    const entry_t xt = sm.list[t];
+    uint32_t rank = 0;
+    for (uint32_t u = 0; u < ln; ++u) rank += sm.list[u] > xt ? 1u : 0u;
+    if (rank < need_b && base + rank < (uint32_t)K) {
+      out[base + rank] = entry_pos(xt);
+      if (out_score) out_score[base + rank] = key_to_score(entry_key(xt));
+    }
+  }
+  __syncwarp();
+  const uint32_t n_out = base + (ln < need_b ? ln : need_b);
+  return (int)(n_out < (uint32_t)K ? n_out : (uint32_t)K);
 }
 
-static __device__ __noinline__ int warp_row_topk(SegSelSmem& sm, const uint32_t* keys, int nslots,
-                                                 const int32_t* __restrict__ cand, int n_cand, int32_t* out,
-                                                 float* out_score, int K, int lane, uint32_t kmin, uint32_t kmax,
-                                                 uint32_t n_filled) {
-  const uint32_t lt = (1u << lane) - 1u;
-  // the final bin [blo, bhi]: slots above it go out, its own are ranked unless it is wanted whole
-  entry_t blo = 1ull, bhi = 0ull;            // n_filled <= K: every filled slot is "above"
+// [lo, hi] holds every entry of the source, n_filled of them.
+template <typename Src>
+__device__ __noinline__ int warp_topk_entries(SegSelSmem& sm, const Src src, entry_t lo, entry_t hi, uint32_t n_filled,
+                                              int32_t* out, float* out_score, int K, int lane) {
+  entry_t elo = 1ull, bhi = 0ull;            // n_filled <= K: every entry is "above"
   uint32_t need_b = 0;
-  bool whole = false;
   if (n_filled > (uint32_t)K) {
-    entry_t lo = (entry_t)kmin << 32, hi = ((entry_t)kmax << 32) | 0xffffffffull;
     uint32_t need = (uint32_t)K;
     for (int round = 0; round < 8; ++round) {
       const entry_t span = hi - lo;
@@ -639,61 +644,100 @@ static __device__ __noinline__ int warp_row_topk(SegSelSmem& sm, const uint32_t*
       const int shift = bits > 11 ? bits - 11 : 0;
       for (int i = lane; i < kSelBins / 4; i += 32) reinterpret_cast<uint4*>(sm.hist)[i] = make_uint4(0, 0, 0, 0);
       __syncwarp();
-      if (shift >= 32) {                     // bins are key ranges
-        const uint32_t klo = (uint32_t)(lo >> 32), khi = (uint32_t)(hi >> 32);
-        const int ksh = shift - 32;
-        warp_row_pass<32, false>(keys, nslots, cand, n_cand, lane, [&](uint32_t k, int) {
-          if (k >= klo && k <= khi && k) atomicAdd(&sm.hist[(k - klo) >> ksh], 1u);
-        });
-      } else {
-        warp_row_pass<16, true>(keys, nslots, cand, n_cand, lane, [&](uint32_t k, int ps) {
-          const entry_t e = make_entry(k, ps);
-          if (k && e >= lo && e <= hi) atomicAdd(&sm.hist[(uint32_t)((e - lo) >> shift)], 1u);
-        });
+      auto count = [&](entry_t e) {
+        if (e >= lo && e <= hi && e) atomicAdd(&sm.hist[(uint32_t)((e - lo) >> shift)], 1u);
+      };
+      bool counted = false;
+      if constexpr (Src::kKeysApart) {
+        if (shift >= 32) {                   // bins are key ranges (lo has a zero low word then)
+          const uint32_t klo = (uint32_t)(lo >> 32), khi = (uint32_t)(hi >> 32);
+          const int ksh = shift - 32;
+          src.template sweep_keys<32>(lane, [&](uint32_t k) {
+            if (k >= klo && k <= khi && k) atomicAdd(&sm.hist[(k - klo) >> ksh], 1u);
+          });
+          counted = true;
+        }
       }
+      if (!counted) src.template sweep<16, true>(lane, count);
       __syncwarp();
       uint32_t b, pop;
       warp_hist_boundary(sm.hist, need, lane, &b, &need_b, &pop);
-      blo = lo + ((entry_t)b << shift);
+      const entry_t blo = lo + ((entry_t)b << shift);
       bhi = shift ? blo + (((entry_t)1 << shift) - 1ull) : blo;
       bhi = bhi < hi ? bhi : hi;
-      whole = pop == need_b;
-      if (whole || pop <= (uint32_t)kSelSmall) break;
+      elo = blo;
+      if (pop == need_b) { bhi = blo - 1ull; elo = ~0ull; break; }   // the bin is wanted whole: it counts as "above"
+      if (pop <= (uint32_t)kSelSmall) break;
       lo = blo; hi = bhi; need = need_b;     // crowded bin (ties): it is the next window
     }
   }
-  // Straight-line body: one predicated store per slot (a divergent branch per slot, with its
-  // reconvergence, cost several hundred clocks a slot); the scores, when asked for, take a
-  // sweep of their own afterwards.
+  return warp_emit_above(sm, src, elo, bhi, need_b, out, out_score, K, lane);
+}
+
+__device__ __forceinline__ int warp_row_topk(SegSelSmem& sm, const uint32_t* keys, int nslots,
+                                             const int32_t* __restrict__ cand, int n_cand, int32_t* out,
+                                             float* out_score, int K, int lane, uint32_t kmin, uint32_t kmax,
+                                             uint32_t n_filled) {
+  return warp_topk_entries(sm, KeyRowSrc{keys, nslots, cand, n_cand}, (entry_t)kmin << 32,
+                           ((entry_t)kmax << 32) | 0xffffffffull, n_filled, out, out_score, K, lane);
+}
+
+// A scan row's segment whose entries were all counted in a histogram with bins bin_of(key):
+// bsel = the boundary bin (need_b of its pop entries are wanted), -1 = everything is wanted.
+// One sweep, unless the boundary bin is too crowded to rank (ties): then the general way.
+template <typename BinFn>
+__device__ __noinline__ int warp_seg_topk_binned(SegSelSmem& sm, const entry_t* seg, int cnt, BinFn bin_of, int bsel,
+                                                 uint32_t need_b, uint32_t pop, int32_t* out, float* out_score, int K,
+                                                 int lane) {
+  const SegSrc src{seg, cnt};
+  if (bsel >= 0 && pop != need_b && pop > (uint32_t)kSelSmall) {
+    entry_t mn = ~0ull, mx = 0ull;
+    uint32_t nv = 0;
+    src.template sweep<16, true>(lane, [&](entry_t e) {
+      mn = (e && e < mn) ? e : mn;
+      mx = e > mx ? e : mx;
+      nv += e ? 1u : 0u;
+    });
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const entry_t a = __shfl_xor_sync(0xffffffffu, mn, o), c = __shfl_xor_sync(0xffffffffu, mx, o);
+      mn = a < mn ? a : mn;
+      mx = c > mx ? c : mx;
+    }
+    nv = __reduce_add_sync(0xffffffffu, nv);
+    return warp_topk_entries(sm, src, mn, mx, nv, out, out_score, K, lane);
+  }
+  // the boundary bin as a set of entries: {e : bin_of(key(e)) == bsel}; above it: bin > bsel
+  const uint32_t lt = (1u << lane) - 1u;
+  const bool whole = bsel >= 0 && pop == need_b;
+  const int bcut = whole ? bsel - 1 : bsel;  // a bin wanted whole counts as "above"
   uint32_t base = 0, ln = 0;
-  if (whole) blo -= 1ull, bhi = blo;         // "above the bin" then includes the bin; nothing is listed
-  const entry_t elo = whole ? ~0ull : blo;   // listed: elo <= e <= bhi
-  warp_row_pass<16, true>(keys, nslots, cand, n_cand, lane, [&](uint32_t k, int ps) {
-    const entry_t e = k ? make_entry(k, ps) : 0ull;
-    const bool em = e > bhi;
-    const bool edge = e >= elo && e <= bhi;
+  src.template sweep<16, true>(lane, [&](entry_t e) {
+    const int bn = e ? (int)bin_of(entry_key(e)) : -2;
+    const bool em = bn > bcut;
+    const bool edge = bn == bcut && bsel >= 0 && !whole;
     const uint32_t m = __ballot_sync(0xffffffffu, em);
     const uint32_t me = __ballot_sync(0xffffffffu, edge);
     const uint32_t p = base + __popc(m & lt);
     const uint32_t q = ln + __popc(me & lt);
-    if (em && p < (uint32_t)K) out[p] = ps;
+    if (em && p < (uint32_t)K) out[p] = entry_pos(e);
     if (edge && q < (uint32_t)kSelSmall) sm.list[q] = e;
     base += __popc(m);
     ln += __popc(me);
   });
   if (out_score) {
     uint32_t b2 = 0;
-    warp_row_pass<16, true>(keys, nslots, cand, n_cand, lane, [&](uint32_t k, int ps) {
-      const bool em = (k ? make_entry(k, ps) : 0ull) > bhi;
+    src.template sweep<16, true>(lane, [&](entry_t e) {
+      const bool em = (e ? (int)bin_of(entry_key(e)) : -2) > bcut;
       const uint32_t m = __ballot_sync(0xffffffffu, em);
       const uint32_t p = b2 + __popc(m & lt);
-      if (em && p < (uint32_t)K) out_score[p] = key_to_score(k);
+      if (em && p < (uint32_t)K) out_score[p] = key_to_score(entry_key(e));
       b2 += __popc(m);
     });
   }
   __syncwarp();
   ln = ln < (uint32_t)kSelSmall ? ln : (uint32_t)kSelSmall;
-  for (uint32_t t = lane; t < ln; t += 32) {                      // entries are distinct: ranks are slots
+  for (uint32_t t = lane; t < ln; t += 32) {
     const entry_t xt = sm.list[t];
     uint32_t rank = 0;
     for (uint32_t u = 0; u < ln; ++u) rank += sm.list[u] > xt ? 1u : 0u;

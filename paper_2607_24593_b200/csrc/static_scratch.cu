@@ -21,7 +21,7 @@ namespace {
 constexpr size_t kStaticBytes = (size_t)8 << 20;          // 8 MiB per GPU
 constexpr int kStaticMaxL = 4096;
 constexpr int kStaticMaxK = 512;
-constexpr int kStaticCtas = 48;                           // grid cap: 48 x 4 rows x 4096 entries x 8 B = 6 MiB
+constexpr int kStaticCtas = 24;                           // grid cap: 24 x 4 rows x 2 segments x 4096 entries x 8 B = 6 MiB
 // (4096 entries per row = eight warp segments of 512 = the largest k this entry point accepts)
 constexpr int kStaticCap = 4096;                          // candidate entries per row
 constexpr int kMaxDev = 64;
@@ -56,7 +56,7 @@ extern "C" int dense_index_static(const pivot_tensor* q, const float* w, const p
   int* status = (int*)(base + off);                     off += 256;
   RowDesc* rows = (RowDesc*)(base + off);               off += up256(sizeof(RowDesc) * (size_t)kStaticMaxL);
   unsigned long long* cand = (unsigned long long*)(base + off);
-  off += (size_t)kStaticCtas * 4 * kStaticCap * sizeof(unsigned long long);
+  off += (size_t)kStaticCtas * 4 * 2 * kStaticCap * sizeof(unsigned long long);   // two segments per row
   if (off > kStaticBytes) return PIVOT_ERR_WORKSPACE;
 
   // The array keeps whatever the previous call left: the status word must start at zero; row
