@@ -47,7 +47,7 @@ FLOP_PER_SCORE = 2 * H * D
 # dram__bytes_read.sum + dram__bytes_write.sum per launch: STORED figures from the ncu captures
 # summarised under profiles/ (same workloads as the ones timed here); not re-measured by this run,
 # and labelled so in the line ("traffic_source").
-TRAFFIC_BYTES = {"prefill_128k_fp8_refine_g4": 2742043648 + 4281856512,
+TRAFFIC_BYTES = {"prefill_128k_fp8_refine_g4": 4492556544 + 4826603264,
                  "decode_scan_kernel": 403589888 + 12189440}
 TRAFFIC_SOURCE = "stored ncu capture (profiles/), not re-measured in this run"
 
