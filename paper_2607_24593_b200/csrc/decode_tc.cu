@@ -114,6 +114,10 @@ decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = ct.tmem_base;
+  // everything above touches only this CTA's own shared and tensor memory: it may overlap the
+  // prepare kernel; from here on the plan, the proxies and the cleared histograms are read
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
 
   const int total = tile_prefix[B];
   const int g_lo = (int)((long long)blockIdx.x * total / gridDim.x);
@@ -294,6 +298,8 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Ls, const float* __re
   extern __shared__ uint8_t sel_raw[];
   SelSmem& sm = *reinterpret_cast<SelSmem*>(((uintptr_t)sel_raw + 15) & ~(uintptr_t)15);
   const int split = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();            // the scan's scores and histograms (before any early return)
   const RowDesc rd = prox[b];
   const int K = rd.K, n0 = rd.n_vis;
   if (K <= 0) return;
@@ -421,6 +427,8 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Ls, const float* __re
 
 __global__ void __launch_bounds__(kBlk, 1) entries_topk_kernel(const EntryList* __restrict__ lists) {
   __shared__ BlkSelSmem sm;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();            // the re-score's entries
   const EntryList el = lists[blockIdx.x];
   if (el.K <= 0) return;
   blk_emit_topk(sm, (const entry_t*)el.list, el.n, el.n, el.K, el.out, el.out_score, 1, el.K);
@@ -468,6 +476,7 @@ decode_prepare_kernel(DecodePlan p, RowDesc* rows, GroupDesc* plan_groups, uint3
   const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int B = p.B, g = p.g, c = p.c, k = p.k, mode = p.mode;
+  ptx::grid_launch_dependents();          // the scan may set itself up meanwhile (it waits before it reads)
   for (int i = tid; i < DHIST; i += blockDim.x) ghist[(size_t)b * DHIST + i] = 0u;
   if (tid < 2) ghist[(size_t)B * DHIST + 2 * b + tid] = 0u;      // list length, delivered shares
   __shared__ int seq_ok;
@@ -550,6 +559,8 @@ __global__ void decode_window_kernel(const GroupDesc* __restrict__ groups, int m
                                      int32_t* __restrict__ wcand) {
   __shared__ int dup[kDecodeWinMax];
   const int b = blockIdx.x, tid = threadIdx.x;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();            // the select's candidate sets
   const GroupDesc gd = groups[b * mc];
   if (gd.n_cand <= 0) return;                      // guarded sequence: scored densely
   const int pos0 = gd.first_pos, lo = pos0 - W + 1, w_g = W + g - 1;
@@ -581,9 +592,9 @@ cudaError_t launch_scan(const CUtensorMap& mk, const CUtensorMap& mq, const CUte
   static bool attr_set[kMaxDevices] = {};
   const size_t smem = dsmem_bytes<DT>();
   if (cudaError_t e = opt_in_dynamic_smem(kern, smem, attr_set); e != cudaSuccess) return e;
-  kern<<<sms, D_THREADS, smem, st>>>(mk, mq, mks, prox, tile_prefix, B, Lmax, scores, ghist, status);
   ++launch_counter();
-  return cudaGetLastError();
+  return launch_kernel(kern, dim3(sms), dim3(D_THREADS), smem, st, true, mk, mq, mks, prox, tile_prefix, B, Lmax, scores,
+                       ghist, status);
 }
 
 }  // namespace
@@ -657,18 +668,24 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   static bool sel_attr[kMaxDevices] = {};
   const size_t sel_smem = sizeof(SelSmem) + 16;
   if ((e = opt_in_dynamic_smem(decode_select_kernel, sel_smem, sel_attr)) != cudaSuccess) return e;
-  decode_select_kernel<<<dim3(SEL_SPLIT, d.B), kBlk, sel_smem, st>>>(d.prox, Ls, scores, ghist, glist, sel_ctr);
+  if ((e = launch_kernel(decode_select_kernel, dim3(SEL_SPLIT, d.B), dim3(kBlk), sel_smem, st, true, (const RowDesc*)d.prox,
+                         Ls, (const float*)scores, (const uint32_t*)ghist, glist, sel_ctr)) != cudaSuccess)
+    return e;
   ++launch_counter();
   }
   if (d.mode == 1) {
     if (W > 0) {
-      decode_window_kernel<<<d.B, 1024, 0, st>>>(d.groups, mc, d.g, W, wcand);
+      if ((e = launch_kernel(decode_window_kernel, dim3(d.B), dim3(1024), 0, st, true, (const GroupDesc*)d.groups, mc, d.g,
+                             W, wcand)) != cudaSuccess)
+        return e;
       ++launch_counter();
     }
     ScanScratch sc = d.scratch_tc;
-    e = launch_refine_tc(d.q, d.B * d.g, d.dtype, chunks, d.B * mc * nch, sc, d.sms, st, false, true);
+    e = launch_refine_tc(d.q, d.B * d.g, d.dtype, chunks, d.B * mc * nch, sc, d.sms, st, false, true, 0, true);
     if (e != cudaSuccess) return e;
-    entries_topk_kernel<<<d.B * d.g, kBlk, 0, st>>>(lists);
+    if ((e = launch_kernel(entries_topk_kernel, dim3(d.B * d.g), dim3(kBlk), 0, st, true, (const EntryList*)lists)) !=
+        cudaSuccess)
+      return e;
     ++launch_counter();
   }
   return cudaGetLastError();

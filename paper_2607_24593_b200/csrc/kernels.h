@@ -1,5 +1,6 @@
 // Host-callable launchers of the library's kernels (internal header).
 #pragma once
+#include <utility>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -135,7 +136,7 @@ cudaError_t launch_scan_tc(const ScanOperands& op, const RowDesc* rows, int n_ro
 
 cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
                              const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum = false,
-                             bool chunked = false, int max_cand = 0);
+                             bool chunked = false, int max_cand = 0, bool overlap_prev = false);
 
 // Decode fast path: key-tile-split scan -> per-sequence select -> chunked re-score -> top-k.
 struct DecodeFast {
@@ -183,6 +184,25 @@ inline cudaError_t opt_in_dynamic_smem(Kern kern, size_t bytes, bool (&done)[kMa
   e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
   if (e == cudaSuccess && tracked) done[dev] = true;
   return e;
+}
+
+// Launch with programmatic stream serialisation (`overlap`): the kernel may start before its
+// predecessor in the stream has finished and must call ptx::grid_dependency_wait() before it
+// touches anything the predecessor writes or reads.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool overlap,
+                                 Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(std::forward<Args>(args))...);
 }
 
 }  // namespace pivot

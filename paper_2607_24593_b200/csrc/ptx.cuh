@@ -30,6 +30,16 @@ __device__ __forceinline__ bool elect_one() {
   return pred != 0;
 }
 
+// Programmatic dependent launch.  A kernel launched with programmatic stream serialisation may
+// start while its predecessor in the stream is still running: grid_dependency_wait() returns once
+// the predecessor has completed and its writes are visible (a no-op in a kernel launched the
+// ordinary way), so everything before it must touch neither the predecessor's outputs nor anything
+// it still reads; grid_launch_dependents() lets the successor's blocks be scheduled as soon as
+// every block of this grid has called it or exited.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+
 // ------------------------------------------------------------------ mbarrier
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");

@@ -177,6 +177,9 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = ct.tmem_base;
+  // (a decode step launches this kernel so that the set-up above overlaps the kernel before it)
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ member-query TMA
@@ -645,15 +648,14 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
 
 template <int DT, int EPI = 1>
 cudaError_t launch_one(const CUtensorMap& mq, const GroupDesc* groups, int n_groups, int q_rows,
-                       const ScanScratch& s, int sms, cudaStream_t st) {
+                       const ScanScratch& s, int sms, cudaStream_t st, bool overlap_prev = false) {
   auto kern = refine_tc_kernel<DT, EPI>;
   static bool attr_set[kMaxDevices] = {};
   const size_t smem = rsmem_bytes<DT, EPI>();
   if (cudaError_t e = opt_in_dynamic_smem(kern, smem, attr_set); e != cudaSuccess) return e;
   const int grid = n_groups < sms ? n_groups : sms;
-  kern<<<grid, RCfg<DT, EPI>::THREADS, smem, st>>>(mq, groups, n_groups, q_rows, s);
   ++launch_counter();
-  return cudaGetLastError();
+  return launch_kernel(kern, dim3(grid), dim3(RCfg<DT, EPI>::THREADS), smem, st, overlap_prev, mq, groups, n_groups, q_rows, s);
 }
 
 }  // namespace
@@ -662,13 +664,13 @@ bool make_operand_map(CUtensorMap* m, const void* base, long long rows, int dtyp
 
 cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDesc* groups, int n_groups,
                              const ScanScratch& s, int sms, cudaStream_t st, bool fp32_head_sum, bool chunked,
-                             int max_cand) {
+                             int max_cand, bool overlap_prev) {
   if (n_groups <= 0) return cudaSuccess;
   CUtensorMap mq;
   if (!make_operand_map(&mq, q, (long long)q_rows * kHeads, dtype, kHeads, 0)) return cudaErrorInvalidValue;
   if (dtype != DT_FP8) return launch_one<DT_BF16>(mq, groups, n_groups, q_rows, s, sms, st);
   if (fp32_head_sum) return launch_one<DT_FP8, 0>(mq, groups, n_groups, q_rows, s, sms, st);
-  if (chunked) return launch_one<DT_FP8, 2>(mq, groups, n_groups, q_rows, s, sms, st);
+  if (chunked) return launch_one<DT_FP8, 2>(mq, groups, n_groups, q_rows, s, sms, st, overlap_prev);
   // select overlapped with the next group's tiles where every group's score rows fit the buffers
   if (PIVOT_REFINE_OVERLAP && s.rkeys && max_cand > 0 && max_cand <= SCORE_SLOTS)
     return launch_one<DT_FP8, 3>(mq, groups, n_groups, q_rows, s, sms, st);
