@@ -15,7 +15,10 @@ namespace {
 constexpr int kMaxSel = 8192;
 constexpr int kMaxDevices = 64;
 
-constexpr int kHostChunks = 8;       // query-row chunks of the host-buffer prefill pipeline
+#ifndef PIVOT_HOST_CHUNKS
+#define PIVOT_HOST_CHUNKS 8
+#endif
+constexpr int kHostChunks = PIVOT_HOST_CHUNKS;   // query-row chunks of the host-buffer prefill pipeline
 
 struct DeviceState {
   void* ws = nullptr;
@@ -24,7 +27,7 @@ struct DeviceState {
   int* last_status = nullptr;
   // host-buffer prefill: copy streams and events, created on first use
   cudaStream_t copy_in = nullptr, copy_out = nullptr;
-  cudaEvent_t ev_entry = nullptr, ev_in[kHostChunks] = {}, ev_done[kHostChunks] = {};
+  cudaEvent_t ev_entry = nullptr, ev_in[kHostChunks + 2] = {}, ev_done[kHostChunks + 2] = {};
   // stage-timing events (created on this device on first use) and what the last call recorded
   cudaEvent_t ev[8] = {};
   bool ev_valid = false, ev_decode_scan = false;
@@ -558,7 +561,7 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
     if ((rc = check_cuda(cudaStreamCreateWithFlags(&ds.copy_in, cudaStreamNonBlocking)))) return rc;
     if ((rc = check_cuda(cudaStreamCreateWithFlags(&ds.copy_out, cudaStreamNonBlocking)))) return rc;
     if ((rc = check_cuda(cudaEventCreateWithFlags(&ds.ev_entry, cudaEventDisableTiming)))) return rc;
-    for (int i = 0; i < kHostChunks; ++i) {
+    for (int i = 0; i < kHostChunks + 2; ++i) {
       if ((rc = check_cuda(cudaEventCreateWithFlags(&ds.ev_in[i], cudaEventDisableTiming)))) return rc;
       if ((rc = check_cuda(cudaEventCreateWithFlags(&ds.ev_done[i], cudaEventDisableTiming)))) return rc;
     }
@@ -593,14 +596,29 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
   // while its copies do not.  In row order the first chunks finish long before the next input
   // has arrived; back to front, the last (cheap) chunks finish faster than their results can
   // leave.  Alternating the two ends (last, first, last but one, second, ...) keeps both the
-  // compute stream and the copy-out stream fed.
-  int order[kHostChunks];
-  for (int j = 0; j < n_chunks; ++j) order[j] = (j & 1) ? j / 2 : n_chunks - 1 - j / 2;
-  // queries: chunk by chunk on the copy-in stream
-  const size_t qrow = (size_t)H_I * d * esz;
+  // compute stream and the copy-out stream fed.  The chunk taken first and the chunk taken last
+  // go in two halves: nothing overlaps the first input copy and the last result copy, so those
+  // two are kept short (more chunks throughout cost more in kernel ramps and tails than they save).
+  struct Piece { int r0, r1; };
+  Piece piece[kHostChunks + 2];
+  int n_pieces = 0;
   for (int j = 0; j < n_chunks; ++j) {
-    const int i = order[j];
+    const int i = (j & 1) ? j / 2 : n_chunks - 1 - j / 2;
     const int r0 = i * chunk_rows, r1 = (r0 + chunk_rows < L) ? r0 + chunk_rows : L;
+    // a quarter first (the first input copy) resp. last (the last result copy)
+    const int mid = j == 0 ? r0 + (r1 - r0) / 4 / g * g : r1 - (r1 - r0) / 4 / g * g;
+    if ((j == 0 || j == n_chunks - 1) && n_chunks >= 4 && mid > r0 && mid < r1) {
+      piece[n_pieces++] = Piece{r0, mid};
+      piece[n_pieces++] = Piece{mid, r1};
+    } else {
+      piece[n_pieces++] = Piece{r0, r1};
+    }
+  }
+  // queries: piece by piece on the copy-in stream
+  const size_t qrow = (size_t)H_I * d * esz;
+  for (int j = 0; j < n_pieces; ++j) {
+    const int i = j;
+    const int r0 = piece[j].r0, r1 = piece[j].r1;
     // a chunk's queries, gates and query scales travel together
     if ((rc = check_cuda(cudaMemcpyAsync(dw + (size_t)r0 * H_I, w + (size_t)r0 * H_I, (size_t)(r1 - r0) * H_I * 4,
                                          cudaMemcpyHostToDevice, ds.copy_in))))
@@ -615,15 +633,15 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
   }
   pivot_tensor tq{dq, fp8 ? dqs : nullptr, q->dtype, 0};
   pivot_tensor tk{dk, fp8 ? dks : nullptr, q->dtype, 0};
-  for (int j = 0; j < n_chunks; ++j) {
-    const int i = order[j];
-    const int r0 = i * chunk_rows, r1 = (r0 + chunk_rows < L) ? r0 + chunk_rows : L;
+  for (int j = 0; j < n_pieces; ++j) {
+    const int i = j;
+    const int r0 = piece[j].r0, r1 = piece[j].r1;
     pivot_opts o;
     memset(&o, 0, sizeof(o));
     o.guard_len = -1;
     o.workspace = dws;
     o.workspace_bytes = arena_bytes - cv.off;
-    if (n_chunks > 1) { o.row_begin = r0; o.row_end = r1; }
+    if (n_pieces > 1) { o.row_begin = r0; o.row_end = r1; }
     if ((rc = check_cuda(cudaStreamWaitEvent(st, ds.ev_in[i], 0)))) return rc;
     rc = pivot_index_prefill_ex(&tq, dw, &tk, L, H_I, d, g, c, k, mode, dout, stream, &o);
     if (rc) return rc;
