@@ -207,26 +207,15 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       // MMA2: the head sum of tile it-1 follows the first MMA of tile it (see the shared scan)
       bool pend = false;
       uint32_t pend_it = 0, pend_blk = 0, w_blk = 0xffffffffu;
-#ifdef PIVOT_PROF_REF
-      long long pw[6] = {0, 0, 0, 0, 0, 0};
-      const long long pstart = clock64();
-#define PW(i, stmt) { const long long t_ = clock64(); stmt; pw[i] += clock64() - t_; }
-#else
-#define PW(i, stmt) stmt;
-#endif
       auto issue_mma2 = [&]() -> bool {
         if (pend_blk != w_blk) {                 // first tile of a group: its gate matrix must be in place
-          bool okw;
-          PW(3, okw = ptx::mbar_wait(&ct.w_ready, pend_blk & 1, abort_flag, 0))
-          if (!okw) return false;
+          if (!ptx::mbar_wait(&ct.w_ready, pend_blk & 1, abort_flag, 0)) return false;
           w_blk = pend_blk;
         }
         const int pb = pend_it & 1;
         // no sleep between polls here or on the accumulator / key-stage waits below: this thread's
         // wake-up latency sits on the tile loop's critical path (four handoffs per tile)
-        bool oka;
-        PW(4, oka = ptx::mbar_wait_poll(&ct.a_ready[pb], (pend_it >> 1) & 1, abort_flag))
-        if (!oka) return false;
+        if (!ptx::mbar_wait_poll(&ct.a_ready[pb], (pend_it >> 1) & 1, abort_flag)) return false;
         ptx::tc_fence_after();
         const uint32_t w_addr = ptx::smem_u32(ct.wmat);
         const uint32_t a_tmem = tmem_base + pb * N;
@@ -245,16 +234,16 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         const int ntiles = group_tiles(groups[gi]);
         if (ntiles == 0) continue;
         const int qb = blk % C::QBUFS;
-        PW(0, ok = ptx::mbar_wait(&ct.q_full[qb], (blk / C::QBUFS) & 1, abort_flag, 32))
+        ok = ptx::mbar_wait(&ct.q_full[qb], (blk / C::QBUFS) & 1, abort_flag, 32);
         if (!ok) break;
         const uint32_t q_addr = ptx::smem_u32(qbuf + qb * C::QBUF_BYTES);
         for (int t = 0; t < ntiles; ++t, ++it) {
           const int s = it % C::STAGES;
           const uint32_t ph = (it / C::STAGES) & 1;
           const int buf = it & 1;
-          PW(1, ok = ptx::mbar_wait_poll(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag))
+          ok = ptx::mbar_wait_poll(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag);
           if (!ok) break;
-          PW(2, ok = ptx::mbar_wait_poll(&ct.full[s], ph, abort_flag))
+          ok = ptx::mbar_wait_poll(&ct.full[s], ph, abort_flag);
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t k_addr = ptx::smem_u32(kring + s * C::STAGE_BYTES);
@@ -281,11 +270,6 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         ptx::tc_commit(&ct.q_empty[qb]);
         ++blk;
       }
-#ifdef PIVOT_PROF_REF
-      pw[5] = clock64() - pstart;
-      for (int i = 0; i < 6; ++i) atomicAdd((unsigned long long*)(sc.status + 8 + 2 * i), (unsigned long long)pw[i]);
-      atomicAdd((unsigned long long*)(sc.status + 20), (unsigned long long)it);
-#endif
     }
   } else if (warp < 2 + GATHER_WARPS) {
     // ------------------------------------------------------------------ gather producers
