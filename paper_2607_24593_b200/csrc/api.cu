@@ -122,7 +122,8 @@ Workspace carve_workspace(void* base, int rows, int n_groups, int c, int k) {
   w.scan.cand_idx = (int32_t*)w.scan.cand64 + simt_entries;
   w.scan.status = w.status;
   w.scan.counter = w.counter;
-  w.scan.rkeys = cv.take<uint32_t>((size_t)sm_count() * 2 * 4 * 4096);
+  w.scan.rslots = (c + 127) / 128 * 128;
+  w.scan.rkeys = cv.take<uint32_t>((size_t)sm_count() * 2 * 4 * w.scan.rslots);
   w.bytes = cv.off;
   return w;
 }

@@ -104,7 +104,8 @@ struct ScanScratch {
   int n_cta;
   int* status;
   int* counter;         // dynamic row scheduler
-  uint32_t* rkeys = nullptr;   // re-score: [SMs][2][4][4096] score keys between the tile loop and the select team
+  uint32_t* rkeys = nullptr;   // re-score: [SMs][2][4][rslots] score keys between the tile loop and the select warps
+  int rslots = 0;              // ... slots per row: the candidate budget rounded up to whole 128-key tiles
 };
 
 void launch_proxy_build(const void* q, const float* qscale, const float* w, void* proxy_q,

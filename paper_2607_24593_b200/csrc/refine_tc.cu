@@ -29,14 +29,14 @@ constexpr int SEL_WARPS = 4;
 constexpr int N = NMEM * kHeads;
 constexpr int TMEM_COLS = 2 * N;
 
-// EPI: 1 = tensor-core head sum where available (FP8), 0 = fp32 FMA head sum, 2 = as 1 for the
-// candidate chunks of a decode step: those leave packed entries for a later top-k, so the score
-// rows need no shared memory and a second query buffer takes their place (the next chunk's
-// queries load while the current one is re-scored).  3 = as 1 with the per-member top-k on four
-// warps of their own, one group behind the tile loop: the score rows go through a double buffer
-// in global memory (L2-resident, 128 KB per CTA) instead of shared memory, so the tensor core
-// and the gather keep running while a group's members are selected.  Needs every group of the
-// launch to have at most SCORE_SLOTS candidates.
+// EPI: 0 = fp32 FMA head sum, scores as packed entries in the per-CTA global segments, each
+// member's top-k by the epilogue teams after the group's tiles (bf16 operands; FP8 on request).
+// FP8 otherwise takes the head sum on the tensor core and comes in two forms: 3 = prefill: the
+// per-member top-k runs on four warps of their own, one group behind the tile loop; the score
+// rows go through a double buffer in global memory (L2-resident, 2 x 4 x ScanScratch::rslots keys
+// per CTA), so the tensor core and the gather keep running while a group's members are selected;
+// every group of the launch has at most rslots candidates.  2 = the candidate chunks of a decode
+// step: those leave packed entries for a later top-k kernel.  (1 = the default for bf16, same as 0.)
 template <int DT, int EPI = 1>
 struct RCfg {
   static constexpr bool FP8 = DT == DT_FP8;
@@ -50,13 +50,7 @@ struct RCfg {
   static constexpr int QROW_HALF_BYTES = kHeads * 128;
   static constexpr int QHALF_BYTES = NMEM * QROW_HALF_BYTES;
   static constexpr int QBUF_BYTES = KHALVES * QHALF_BYTES;
-  // FP8 keeps the group's score keys in shared memory (4 members x 4096 slots x 4 B) for the
-  // final top-k; bf16 has no room for that next to 2 x 64 KB of queries and goes through the
-  // per-CTA global segments instead.
-  static constexpr bool SMEM_SCORES = FP8 && EPI == 1;
-  // With the score rows resident, one query buffer (the next group's queries load while the
-  // key ring refills) buys two more gather stages, which matter more.
-  static constexpr int QBUFS = SMEM_SCORES ? 1 : 2;
+  static constexpr int QBUFS = 2;                 // the next group's queries load while this one is re-scored
   static constexpr int STAGES = FP8 ? 6 : 2;
   static constexpr int LOOKAHEAD = FP8 ? 4 : 1;   // gather tiles in flight per producer thread
   static constexpr int ROW_BYTES = FP8 ? 128 : 256;
@@ -69,12 +63,8 @@ struct RCfg {
   static constexpr int TMEM_EMPTY_ARRIVALS = MMA2 ? 4 : EPI_WARPS;
 };
 
-#ifndef PIVOT_REFINE_OVERLAP
-#define PIVOT_REFINE_OVERLAP 1
-#endif
 constexpr int META_SLOTS = 8;     // key stages in flight (<= 6) + accumulator buffers (2)
 static_assert(META_SLOTS >= 6 + 2, "meta ring");
-constexpr int SCORE_SLOTS = 4096;             // shared-memory score row: candidates per member
 
 // What the epilogue needs to know about a gathered key: its position and scale.
 struct KeyMeta {
@@ -107,10 +97,9 @@ struct RCtrlT {
 template <int DT, int EPI = 1>
 constexpr size_t rsmem_bytes() {
   using C = RCfg<DT, EPI>;
-  return 1024 + C::QBUFS * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(RCtrlT<C::MMA2, C::NSEL>) +
-         (C::SMEM_SCORES ? (size_t)NMEM * SCORE_SLOTS * 4 : 0);
+  return 1024 + C::QBUFS * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(RCtrlT<C::MMA2, C::NSEL>);
 }
-static_assert(rsmem_bytes<DT_FP8, 1>() <= 232448 && rsmem_bytes<DT_FP8, 0>() <= 232448 && rsmem_bytes<DT_FP8, 2>() <= 232448 &&
+static_assert(rsmem_bytes<DT_FP8, 0>() <= 232448 && rsmem_bytes<DT_FP8, 2>() <= 232448 &&
               rsmem_bytes<DT_FP8, 3>() <= 232448 &&
               rsmem_bytes<DT_BF16>() <= 232448, "shared memory budget");
 
@@ -138,7 +127,6 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
   uint8_t* kring = smem + C::QBUFS * C::QBUF_BYTES;
   using RCtrl = RCtrlT<C::MMA2, C::NSEL>;
   RCtrl& ct = *reinterpret_cast<RCtrl*>(kring + C::STAGES * C::STAGE_BYTES);
-  uint32_t* skey = reinterpret_cast<uint32_t*>(kring + C::STAGES * C::STAGE_BYTES + sizeof(RCtrl));   // [NMEM][SCORE_SLOTS]
   volatile int* abort_flag = &ct.abort;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -361,11 +349,12 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
     // Warp r takes member r's exact top-k of group n while the other warps re-score group n + 1.
     const int r = warp - (2 + GATHER_WARPS + EPI_WARPS);
     SegSelSmem& sel = ct.sel[r];
-    const uint32_t* rk = sc.rkeys + (size_t)blockIdx.x * 2 * NMEM * SCORE_SLOTS;
+    const int RS = sc.rslots;                    // slots per score row
+    const uint32_t* rk = sc.rkeys + (size_t)blockIdx.x * 2 * NMEM * RS;
     uint32_t blk = 0;
     for (int gi = blockIdx.x; gi < n_groups; gi += gridDim.x) {
       const GroupDesc gd = groups[gi];
-      const int ntiles = min(group_tiles(gd), SCORE_SLOTS / TILE_KEYS);
+      const int ntiles = min(group_tiles(gd), RS / TILE_KEYS);
       if (ntiles == 0) continue;
       const int kb = blk & 1;
       const uint32_t kph = (blk >> 1) & 1;
@@ -377,7 +366,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       if (r < gd.m) {
         int32_t* out = gd.out + (size_t)r * gd.out_stride;
         float* outs = gd.out_score ? gd.out_score + (size_t)r * gd.out_stride : nullptr;
-        const int n_valid = warp_row_topk(sel, rk + (kb * NMEM + r) * SCORE_SLOTS, ntiles * TILE_KEYS, gd.cand,
+        const int n_valid = warp_row_topk(sel, rk + (size_t)(kb * NMEM + r) * RS, ntiles * TILE_KEYS, gd.cand,
                                           gd.n_cand, out, outs, gd.K, lane, kmin, kmax, n_filled);
         for (int i = n_valid + lane; i < gd.K; i += 32) {
           out[i] = -1;
@@ -403,7 +392,8 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
     const size_t cta_base = (size_t)blockIdx.x * NMEM * sc.cap;
     auto seg_off = [&](int r) { return cta_base + ((size_t)r * 4 + wq) * SEG; };
     uint32_t it = 0, blk = 0;
-    uint32_t* const rk = C::OVL ? sc.rkeys + (size_t)blockIdx.x * 2 * NMEM * SCORE_SLOTS : nullptr;
+    const int RS = sc.rslots;
+    uint32_t* const rk = C::OVL ? sc.rkeys + (size_t)blockIdx.x * 2 * NMEM * RS : nullptr;
     for (int gi = blockIdx.x; gi < n_groups; gi += gridDim.x) {
       const GroupDesc gd = groups[gi];
       const int ntiles = group_tiles(gd);
@@ -411,7 +401,6 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       const int kb = blk & 1;                    // score-row buffer of this group (EPI = 3)
       const uint32_t kph = (blk >> 1) & 1;
       ++blk;
-      const bool smem_sel = C::SMEM_SCORES && !gd.ent_out && ntiles * TILE_KEYS <= SCORE_SLOTS;
       if constexpr (C::MMA2) {
         // team 1 scores all four members (so both teams meet around the tile loop: the other team
         // selects from what it wrote) and writes the diagonal blocks of the gate matrix; the last
@@ -458,17 +447,13 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         const int t_r = gd.first_pos + r;
         const bool seen = idx >= 0 && idx <= t_r && idx + gd.win_span > t_r;
         if constexpr (C::OVL) {        // key only, to this group's score-row buffer
-          if (r < gd.m && slot < SCORE_SLOTS) {
+          if (r < gd.m && slot < RS) {
             const uint32_t kv = seen ? key : 0u;
-            rk[(kb * NMEM + r) * SCORE_SLOTS + slot] = kv;
+            rk[(size_t)(kb * NMEM + r) * RS + slot] = kv;
             smn[r] = (kv && kv < smn[r]) ? kv : smn[r];
             smx[r] = kv > smx[r] ? kv : smx[r];
             snv[r] += kv ? 1u : 0u;
           }
-          return;
-        }
-        if (smem_sel) {                // key only; the position is looked up again at the end
-          if (r < gd.m && PIVOT_BOUNDS(slot >= 0 && slot < SCORE_SLOTS, sc.status)) skey[r * SCORE_SLOTS + slot] = seen ? key : 0u;
           return;
         }
         const entry_t e = seen ? make_entry(key, idx) : kPadEntry;
@@ -613,24 +598,9 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         float* outs = gd.out_score ? gd.out_score + (size_t)r * gd.out_stride : nullptr;
         const int segcnt = min(ntiles * 32, SEG);
         const Seg seg{sc.cand64 + seg_off(r), segcnt};
-        int n_valid = -1;
-        if (smem_sel) {
-          const uint32_t* keys = skey + r * SCORE_SLOTS;
-          n_valid = smem_row_topk(tm, sel, keys, ntiles * TILE_KEYS, gd.cand, gd.n_cand, out, outs, gd.K);
-          if (n_valid < 0) {           // crowded boundary bin (ties): spell the entries out and re-select
-            for (int i = 0; i < ntiles; ++i) {
-              const int sl = i * TILE_KEYS + tt;
-              const uint32_t k = keys[sl];
-              const int ci = __ldg(gd.cand + (sl < gd.n_cand ? sl : 0));
-              if (i * 32 + lane < SEG) sc.cand64[seg_off(r) + i * 32 + lane] = k ? make_entry(k, ci) : kPadEntry;
-            }
-            tm.sync();
-          }
-        }
         // 32 entries per lane (c <= 4096) fit the registers this kernel has; beyond that re-read
-        if (n_valid < 0)
-          n_valid = segcnt <= 32 * 32 ? seg_emit<true, 32>(tm, sel, seg, gd.n_cand, out, outs, gd.K)
-                                      : seg_emit<false>(tm, sel, seg, gd.n_cand, out, outs, gd.K);
+        const int n_valid = segcnt <= 32 * 32 ? seg_emit<true, 32>(tm, sel, seg, gd.n_cand, out, outs, gd.K)
+                                              : seg_emit<false>(tm, sel, seg, gd.n_cand, out, outs, gd.K);
         for (int i = n_valid + tt; i < gd.K; i += 128) {
           out[i] = -1;
           if (outs) outs[i] = -INFINITY;
@@ -671,10 +641,9 @@ cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDe
   if (dtype != DT_FP8) return launch_one<DT_BF16>(mq, groups, n_groups, q_rows, s, sms, st);
   if (fp32_head_sum) return launch_one<DT_FP8, 0>(mq, groups, n_groups, q_rows, s, sms, st);
   if (chunked) return launch_one<DT_FP8, 2>(mq, groups, n_groups, q_rows, s, sms, st, overlap_prev);
-  // select overlapped with the next group's tiles where every group's score rows fit the buffers
-  if (PIVOT_REFINE_OVERLAP && s.rkeys && max_cand > 0 && max_cand <= SCORE_SLOTS)
-    return launch_one<DT_FP8, 3>(mq, groups, n_groups, q_rows, s, sms, st);
-  return launch_one<DT_FP8, 1>(mq, groups, n_groups, q_rows, s, sms, st);
+  // the select warps need the caller's score-row buffers, long enough for every group
+  if (!s.rkeys || max_cand <= 0 || max_cand > s.rslots) return cudaErrorInvalidValue;
+  return launch_one<DT_FP8, 3>(mq, groups, n_groups, q_rows, s, sms, st);
 }
 
 }  // namespace pivot

@@ -363,152 +363,6 @@ __device__ __forceinline__ int seg_emit(const Team& tm, SegSelSmem& sm, const Se
   return n_out > K ? K : n_out;
 }
 
-// Exact top-K of a row of score keys held in shared memory (0 = padding slot); the position of
-// slot s is cand[s] (s < n_cand).  One linear 2048-bin histogram over the row's key range finds
-// the boundary bin; the slots above it are emitted in a second pass and the boundary bin's
-// slots are ranked by (key, position).  Returns how many positions were written, or -1 --
-// before writing anything -- when the boundary bin is too crowded to rank (the caller takes the
-// general path).  At most 32 slots per thread (nslots <= 32 x team size, a multiple of the team
-// size); all threads of the team call.
-__device__ __forceinline__ int smem_row_topk(const Team& tm, SegSelSmem& sm, const uint32_t* keys, int nslots,
-                                             const int32_t* __restrict__ cand, int n_cand, int32_t* out,
-                                             float* out_score, int K) {
-  const int lane = tm.tid & 31;
-  const int per = nslots / tm.nthr;       // slots of this thread: i * nthr + tid, i < per
-  // positions first: their global-memory round trip hides behind the histogram passes
-  int ci[32];
-#pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    const int s = i * tm.nthr + tm.tid;
-    ci[i] = (i < per && s < n_cand) ? __ldg(cand + s) : -1;
-  }
-  // ... and the keys: every pass below runs on registers
-  uint32_t kreg[32];
-#pragma unroll
-  for (int i = 0; i < 32; ++i) kreg[i] = i < per ? keys[i * tm.nthr + tm.tid] : 0u;
-  uint32_t mn = 0xffffffffu, mx = 0u, nv = 0u;
-#pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    const uint32_t k = kreg[i];
-    mn = (k && k < mn) ? k : mn;
-    mx = k > mx ? k : mx;
-    nv += k ? 1u : 0u;
-  }
-  if (tm.tid == 0) { sm.kmin = 0xffffffffu; sm.kmax = 0u; sm.total = 0u; sm.out_count = 0u; sm.list_n = 0u; }
-  for (int i = tm.tid; i < kSelBins; i += tm.nthr) sm.hist[i] = 0;
-  tm.sync();
-  mn = __reduce_min_sync(0xffffffffu, mn);
-  mx = __reduce_max_sync(0xffffffffu, mx);
-  nv = __reduce_add_sync(0xffffffffu, nv);
-  if (lane == 0) { atomicMin(&sm.kmin, mn); atomicMax(&sm.kmax, mx); atomicAdd(&sm.total, nv); }
-  tm.sync();
-  const uint32_t lo = sm.kmin, hi = sm.kmax;
-  const int n_valid = (int)sm.total;
-  int bsel = -1;            // emit every bin above bsel
-  uint32_t need_b = 0;
-  bool whole_bin = false;   // the boundary bin is wanted entirely
-  int shift = 0;
-  if (n_valid > K) {
-    const uint32_t span = hi - lo;
-    const int bitsw = span ? 32 - __clz(span) : 0;
-    shift = bitsw > 11 ? bitsw - 11 : 0;
-#pragma unroll
-    for (int i = 0; i < 32; ++i)
-      if (kreg[i]) atomicAdd(&sm.hist[(kreg[i] - lo) >> shift], 1u);
-    tm.sync();
-    uint32_t b, pop;
-    warp_hist_boundary(sm.hist, (uint32_t)K, lane, &b, &need_b, &pop);   // same result in every warp
-    if (pop != need_b && pop > (uint32_t)kSelSmall) return -1;
-    bsel = (int)b;
-    whole_bin = pop == need_b;
-  }
-  // Which of this thread's slots go out: counted first, then a scan over the team hands every
-  // thread a contiguous run of output positions (no atomics, no votes in the write loop).
-  uint32_t emit_mask = 0u, edge_mask = 0u;
-#pragma unroll
-  for (int i = 0; i < 32; ++i) {             // branch-free: two bit masks per thread
-    const uint32_t k = kreg[i];
-    const bool valid = k != 0u;
-    const int bn = valid ? (int)((k - lo) >> shift) : -2;
-    emit_mask |= (valid && (bn > bsel || (whole_bin && bn == bsel))) ? 1u << i : 0u;
-    edge_mask |= (valid && bn == bsel && !whole_bin) ? 1u << i : 0u;
-  }
-  // the boundary bin's slots (a handful per row) go to the list that is ranked below; kept out
-  // of the loop above, where a rarely taken branch per slot cost more than everything else in it
-  while (edge_mask) {
-    const int i = __ffs(edge_mask) - 1;
-    edge_mask &= edge_mask - 1u;
-    const int sl = i * tm.nthr + tm.tid;
-    const uint32_t q = atomicAdd(&sm.list_n, 1u);
-    if (q < (uint32_t)kSelSmall) sm.list[q] = make_entry(keys[sl], sl < n_cand ? __ldg(cand + sl) : -1);
-  }
-  const uint32_t mine = (uint32_t)__popc(emit_mask);
-  uint32_t incl = mine;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += v;
-  }
-  const int wq = tm.tid >> 5;
-  if (lane == 31) sm.wsum[wq] = incl;
-  tm.sync();
-  uint32_t p = incl - mine;
-  for (int w = 0; w < wq; ++w) p += sm.wsum[w];
-  if (tm.tid == tm.nthr - 1) sm.out_count = p + mine;      // emitted so far; the ranked ones follow
-  if (K <= kSelBins && out_score == nullptr) {
-    // Positions are lined up in output order in shared memory first (the histogram is no longer
-    // needed: every warp has its boundary, see the barrier above) and leave as whole 16-byte
-    // rows; written straight from the loop below they would go out as scattered 4-byte stores.
-    int32_t* const stage = reinterpret_cast<int32_t*>(sm.hist);
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      if ((emit_mask >> i) & 1u) {
-        if (p < (uint32_t)K) stage[p] = ci[i];
-        ++p;
-      }
-    }
-    tm.sync();
-    const int n_out = (int)(sm.out_count < (uint32_t)K ? sm.out_count : (uint32_t)K);
-    const int n4 = n_out >> 2;
-    if ((reinterpret_cast<uintptr_t>(out) & 15) == 0) {
-      for (int t = tm.tid; t < n4; t += tm.nthr)
-        reinterpret_cast<int4*>(out)[t] = reinterpret_cast<const int4*>(stage)[t];
-      for (int t = (n4 << 2) + tm.tid; t < n_out; t += tm.nthr) out[t] = stage[t];
-    } else {
-      for (int t = tm.tid; t < n_out; t += tm.nthr) out[t] = stage[t];
-    }
-  } else {
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      if ((emit_mask >> i) & 1u) {
-        if (p < (uint32_t)K) {
-          out[p] = ci[i];
-          if (out_score) out_score[p] = key_to_score(kreg[i]);
-        }
-        ++p;
-      }
-    }
-  }
-  tm.sync();
-  if (bsel >= 0 && !whole_bin) {
-    const uint32_t P = sm.list_n < (uint32_t)kSelSmall ? sm.list_n : (uint32_t)kSelSmall;
-    for (uint32_t t = tm.tid; t < P; t += tm.nthr) {
-      const entry_t xt = sm.list[t];
-      uint32_t rank = 0;
-      for (uint32_t u = 0; u < P; ++u) rank += sm.list[u] > xt ? 1u : 0u;
-      if (rank < need_b) {
-        const uint32_t p = atomicAdd(&sm.out_count, 1u);
-        if (p < (uint32_t)K) {
-          out[p] = entry_pos(xt);
-          if (out_score) out_score[p] = key_to_score(entry_key(xt));
-        }
-      }
-    }
-    tm.sync();
-  }
-  return n_valid < K ? n_valid : K;
-}
-
 // ---------------------------------------------------------------------------------------------
 // Exact top-K by ONE warp over entries that lie in global memory (written by other warps of the
 // CTA, read through L2): the rows of score keys the re-score kernel leaves per member, and the
