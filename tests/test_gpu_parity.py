@@ -106,9 +106,9 @@ def test_prefill_edge_shapes(pv, gu, dtype, L, g, c, k, guard):
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "fp8"])
-def test_prefill_candidate_budget_beyond_the_shared_memory_rows(pv, gu, dtype):
-    """c above 4096 (and not a multiple of the tile): the re-score keeps its score rows in the
-    global segments instead of shared memory, the scan selects more than 4096 per row."""
+def test_prefill_candidate_budget_above_4096(pv, gu, dtype):
+    """c above 4096 (and not a multiple of the tile): the re-score's score rows are longer than
+    4096 slots with a ragged last tile, the scan selects more than 4096 per row."""
     L, g, c, k = 9000, 4, 5000, 2500
     x = inputs.make_prefill(L, dtype=dtype, seed=32)
     out, sc, cand, cs = gu.run_prefill(x, g=g, c=c, k=k, mode=po.MODE_REFINE)
