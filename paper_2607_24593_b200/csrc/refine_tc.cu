@@ -3,11 +3,12 @@
 //
 // One group at a time per persistent CTA.  The group's m <= 4 member queries (m x 64 heads)
 // form the MMA N side and stay in shared memory; the c candidate keys are gathered from the
-// (L2-resident) key cache by four producer warps, 128 keys per tile, written straight into the
+// (L2-resident) key cache by two producer warps, 128 keys per tile, written straight into the
 // 128-byte-swizzled K-major layout the tensor core reads (cp.async, 16 bytes at a time).  The
 // epilogue is the scan's: one key per thread, ReLU, gate-weighted head sum, key scale.  Scores
-// go to a per-CTA buffer; after the last tile each member's exact top-k is selected from its c
-// scores and written out.
+// go to a per-CTA buffer, from which each member's exact top-k is selected and written out:
+// by select warps while the next group is re-scored (FP8 prefill), by the epilogue warps after
+// the group's last tile (bf16), or by a later kernel (the candidate chunks of a decode step).
 //
 // Warps: 0 = query TMA, 1 = MMA issuer + TMEM owner, 2-3 = gather producers, 4-11 = epilogue,
 // 12-15 (EPI = 3) = select warps, one per member.
