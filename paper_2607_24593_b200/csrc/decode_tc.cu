@@ -3,20 +3,20 @@
 // One MTP step scores one proxy per sequence against that sequence's whole key cache, so the
 // step is a single pass over every visible key (128 B + 4 B scale): memory bound.  The work is
 // therefore split by KEY TILES, not by rows:
-//   decode_prepare_kernel one block per sequence clears its histogram and plans it; the block that
-//                        finishes last derives the tile prefix, candidate chunks and entry lists.
+//   decode_prepare_kernel one block per sequence clears its histogram, plans it, builds its proxy
+//                        and writes its share of the tile prefix, candidate chunks and entry lists.
 //   decode_scan_kernel   every SM takes an equal, contiguous share of all (sequence, 128-key
 //                        tile) pairs; per tile: TMA -> tcgen05 MMA (128 keys x 64 heads x d) ->
 //                        epilogue (ReLU, gate-weighted head sum, key scale) -> one fp32 score per
 //                        key to an L2-resident score array (3 % of the bytes read), plus a
 //                        8192-bin histogram of the scores' top 13 key bits per sequence.
-//   decode_select_kernel four 1024-thread CTAs per sequence: the histogram gives the bin holding
-//                        the K-th best score; each CTA collects the survivors of its quarter of
-//                        the score array and appends them to the sequence's list in global
-//                        memory; the CTA that finishes last takes the exact top-K (Eq. 6 / 7) of
-//                        the list in shared memory (nobody waits for anybody).  If the boundary
-//                        bin leaves too many candidates, one CTA alone refines it 12 bits at a
-//                        time with further passes over the scores.
+//   decode_select_kernel a cluster of four 1024-thread CTAs per sequence: the histogram gives the
+//                        bin holding the K-th best score; each CTA collects the survivors of its
+//                        quarter of the score array in its shared memory; after a cluster barrier
+//                        CTA 0 reads the other three lists through distributed shared memory and
+//                        takes the exact top-K (Eq. 6 / 7) of the union.  If the boundary bin
+//                        leaves too many candidates, one CTA alone refines it 12 bits at a time
+//                        with further passes over the scores.
 //   decode_window_kernel (only with a local window, Appendix B) the union of the step's per-query
 //                        windows as one more candidate chunk per sequence, minus the positions
 //                        the pool already holds.
@@ -25,6 +25,8 @@
 //                        over candidates so that all SMs take part).
 #include <cuda.h>
 #include <string.h>
+
+#include <cooperative_groups.h>
 
 #include "blockselect.cuh"
 #include "kernels.h"
@@ -35,6 +37,7 @@
 namespace pivot {
 namespace {
 
+namespace cg = cooperative_groups;
 constexpr int TILE_KEYS = 128;
 constexpr int DKS_SLOTS = 14;
 constexpr int DHIST_BITS = 13;          // histogram digit: top 13 bits of the score key (16 bins per octave)
@@ -290,11 +293,10 @@ struct SelSmem {
   entry_t list[SEL_CAP];
 };
 
-// sel_ctr[2 b] = entries in sequence b's global list, sel_ctr[2 b + 1] = CTAs that have
-// delivered their share (both zeroed with the histograms before every step).
-__global__ void __launch_bounds__(kBlk, 1)
+// The SEL_SPLIT CTAs of a sequence are one thread-block cluster (blockIdx.x = rank in it).
+__global__ void __cluster_dims__(SEL_SPLIT, 1, 1) __launch_bounds__(kBlk, 1)
 decode_select_kernel(const RowDesc* __restrict__ prox, int Ls, const float* __restrict__ scores,
-                     const uint32_t* __restrict__ ghist, entry_t* __restrict__ glist, uint32_t* sel_ctr) {
+                     const uint32_t* __restrict__ ghist) {
   extern __shared__ uint8_t sel_raw[];
   SelSmem& sm = *reinterpret_cast<SelSmem*>(((uintptr_t)sel_raw + 15) & ~(uintptr_t)15);
   const int split = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31;
@@ -316,7 +318,7 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Ls, const float* __re
     // too crowded a boundary bin (every CTA of the sequence sees the same histogram): the
     // refinement passes need the whole score array, CTA 0 takes the sequence alone
     solo = (uint32_t)K - need + pop > (uint32_t)SEL_CAP;
-    if (solo && split != 0) return;
+    if (solo && split != 0) return;          // (the whole cluster takes this branch or none: no cluster barrier follows)
     while ((uint32_t)K - need + pop > (uint32_t)SEL_CAP && pbits < 64) {
       const int wbits = 64 - pbits < 12 ? 64 - pbits : 12;
       __syncthreads();
@@ -355,28 +357,35 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Ls, const float* __re
   const int hi = (solo || split == SEL_SPLIT - 1) ? n0 : (int)(((long long)n0 * (split + 1) / SEL_SPLIT) & ~3ll);
   if (tid == 0) sm.blk.list_n = 0;
   __syncthreads();
-  for (int i0 = lo; i0 < hi; i0 += 16 * kBlk) {        // four 16-byte loads in flight per thread
-    float4 v4[4];
+  for (int i0 = lo; i0 < hi; i0 += 32 * kBlk) {        // eight 16-byte loads in flight per thread
+    float4 v4[8];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < 8; ++u) {
       const int i = i0 + (u * kBlk + tid) * 4;
       v4[u] = i < hi ? __ldcg(reinterpret_cast<const float4*>(sc + i)) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    // One list-cursor bump per warp and pass: each thread counts its keepers among its sixteen
+    // One list-cursor bump per warp and pass: each thread counts its keepers among its 32
     // scores, a warp scan turns the counts into offsets (a bump per keeper group would queue
-    // hundreds of same-address atomics per pass).
-    auto entry_of = [&](int u) -> entry_t {
+    // hundreds of same-address atomics per pass).  The test runs on the 32-bit score key while
+    // the prefix is no longer than that (always, unless a crowded bin was refined further):
+    // the pass is bound by its instruction count, not by the loads.
+    auto score_of = [&](int u) -> float {
       const float4 q4 = v4[u >> 2];
-      const float vu = (u & 3) == 0 ? q4.x : (u & 3) == 1 ? q4.y : (u & 3) == 2 ? q4.z : q4.w;
-      return make_entry(score_to_key(vu), i0 + ((u >> 2) * kBlk + tid) * 4 + (u & 3));
+      return (u & 3) == 0 ? q4.x : (u & 3) == 1 ? q4.y : (u & 3) == 2 ? q4.z : q4.w;
     };
+    auto pos_of = [&](int u) -> int { return i0 + ((u >> 2) * kBlk + tid) * 4 + (u & 3); };
     uint32_t keepmask = 0;
+    if (pbits <= 32) {
+      const uint32_t kthr = pbits ? (uint32_t)prefix << (32 - pbits) : 0u;
 #pragma unroll
-    for (int u = 0; u < 16; ++u) {
-      const int i = i0 + ((u >> 2) * kBlk + tid) * 4 + (u & 3);
-      const entry_t e = entry_of(u);
-      const bool keep = i < hi && (pbits == 0 || (e >> (64 - pbits)) >= prefix);
-      keepmask |= keep ? 1u << u : 0u;
+      for (int u = 0; u < 32; ++u)
+        keepmask |= (pos_of(u) < hi && score_to_key(score_of(u)) >= kthr) ? 1u << u : 0u;
+    } else {
+#pragma unroll
+      for (int u = 0; u < 32; ++u) {
+        const entry_t e = make_entry(score_to_key(score_of(u)), pos_of(u));
+        keepmask |= (pos_of(u) < hi && (e >> (64 - pbits)) >= prefix) ? 1u << u : 0u;
+      }
     }
     const uint32_t cnt = (uint32_t)__popc(keepmask);
     uint32_t incl = cnt;
@@ -391,33 +400,35 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Ls, const float* __re
       if (lane == 31) base = atomicAdd(&sm.blk.list_n, tot);
       base = __shfl_sync(0xffffffffu, base, 31);
       uint32_t p = base + incl - cnt;
+      while (keepmask) {                                 // a few per cent of the scores are kept
+        const int u = __ffs(keepmask) - 1;
+        keepmask &= keepmask - 1u;
+        float vu = 0.f;
 #pragma unroll
-      for (int u = 0; u < 16; ++u) {
-        if ((keepmask >> u) & 1u) {
-          if (p < (uint32_t)SEL_CAP) sm.list[p] = entry_of(u);
-          ++p;
-        }
+        for (int q = 0; q < 32; ++q) vu = q == u ? score_of(q) : vu;
+        if (p < (uint32_t)SEL_CAP) sm.list[p] = make_entry(score_to_key(vu), pos_of(u));
+        ++p;
       }
     }
   }
   __syncthreads();
   int n = min((int)sm.blk.list_n, SEL_CAP);
   if (!solo) {
-    // ---- hand the share over; whoever delivers last holds the complete list
-    entry_t* const gl = glist + (size_t)b * SEL_CAP;
-    if (tid == 0) sm.blk.small_n = n ? atomicAdd(&sel_ctr[2 * b], (uint32_t)n) : 0u;
-    __syncthreads();
-    const uint32_t at = sm.blk.small_n;
-    for (int i = tid; i < n; i += kBlk)
-      if (at + i < (uint32_t)SEL_CAP) gl[at + i] = sm.list[i];
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) sm.blk.small_n = atomicAdd(&sel_ctr[2 * b + 1], 1u);
-    __syncthreads();
-    if (sm.blk.small_n != (uint32_t)(SEL_SPLIT - 1)) return;
-    __threadfence();
-    n = min((int)*reinterpret_cast<volatile uint32_t*>(&sel_ctr[2 * b]), SEL_CAP);
-    for (int i = tid; i < n; i += kBlk) sm.list[i] = __ldcg(gl + i);
+    // ---- hand the shares over: the four CTAs of a sequence form a cluster, and CTA 0 reads the
+    //      others' lists out of their shared memory
+    cg::cluster_group cluster = cg::this_cluster();
+    cluster.sync();                                      // every list is complete
+    if (split == 0) {
+      for (int r = 1; r < SEL_SPLIT; ++r) {
+        const SelSmem* rs = cluster.map_shared_rank(&sm, r);
+        const int nr = min((int)rs->blk.list_n, SEL_CAP);
+        for (int i = tid; i < nr; i += kBlk)
+          if (n + i < SEL_CAP) sm.list[n + i] = rs->list[i];
+        n = min(n + nr, SEL_CAP);
+      }
+    }
+    cluster.sync();                                      // nobody leaves while its list is being read
+    if (split != 0) return;
     __syncthreads();
   }
   blk_emit_topk(sm.blk, sm.list, n, n, K, rd.out, rd.out_score, rd.out_rows, rd.out_stride);
@@ -478,7 +489,6 @@ decode_prepare_kernel(DecodePlan p, RowDesc* rows, GroupDesc* plan_groups, uint3
   const int B = p.B, g = p.g, c = p.c, k = p.k, mode = p.mode;
   ptx::grid_launch_dependents();          // the scan may set itself up meanwhile (it waits before it reads)
   for (int i = tid; i < DHIST; i += blockDim.x) ghist[(size_t)b * DHIST + i] = 0u;
-  if (tid < 2) ghist[(size_t)B * DHIST + 2 * b + tid] = 0u;      // list length, delivered shares
   __shared__ int seq_ok;
   __shared__ int wsum[32];
   if (tid == 0) seq_ok = plan_decode_sequence(p, b, rows, plan_groups) ? 1 : 0;
@@ -607,7 +617,7 @@ size_t decode_fast_bytes(int B, int Lmax, int g, int c) {
   const int mc = group_chunks(g);
   const int ncc = (c + kDecodeCandChunk - 1) / kDecodeCandChunk;
   const size_t Ls = ((size_t)Lmax + 3) & ~(size_t)3;     // score rows start on 16-byte boundaries
-  return up(B * Ls * 4) + up((size_t)B * (DHIST + 2) * 4) + up((size_t)(B + 1) * 4) + up((size_t)B * SEL_CAP * 8) +
+  return up(B * Ls * 4) + up((size_t)B * DHIST * 4) + up((size_t)(B + 1) * 4) +
          up((size_t)B * mc * (ncc + 1) * sizeof(GroupDesc)) + up((size_t)B * g * sizeof(EntryList)) +
          up((size_t)B * kDecodeWinMax * 4) + up((size_t)B * g * (c + kDecodeWinMax) * 8);
 }
@@ -624,10 +634,8 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   char* p = (char*)d.scratch;
   const int Ls = (d.Lmax + 3) & ~3;
   float* scores = (float*)p;                 p += up((size_t)d.B * Ls * 4);
-  uint32_t* ghist = (uint32_t*)p;            p += up((size_t)d.B * (DHIST + 2) * 4);
-  uint32_t* sel_ctr = ghist + (size_t)d.B * DHIST;       // zeroed together with the histograms
+  uint32_t* ghist = (uint32_t*)p;            p += up((size_t)d.B * DHIST * 4);
   int* tile_prefix = (int*)p;                p += up((size_t)(d.B + 1) * 4);
-  entry_t* glist = (entry_t*)p;              p += up((size_t)d.B * SEL_CAP * 8);
   const int mc = group_chunks(d.g);
   // Candidates per re-score work item: as few items as keep every SM busy in ONE wave (each item pays
   // for its own query load and pipeline ramp), never below kDecodeCandChunk, whole 128-key tiles.
@@ -669,7 +677,7 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   const size_t sel_smem = sizeof(SelSmem) + 16;
   if ((e = opt_in_dynamic_smem(decode_select_kernel, sel_smem, sel_attr)) != cudaSuccess) return e;
   if ((e = launch_kernel(decode_select_kernel, dim3(SEL_SPLIT, d.B), dim3(kBlk), sel_smem, st, true, (const RowDesc*)d.prox,
-                         Ls, (const float*)scores, (const uint32_t*)ghist, glist, sel_ctr)) != cudaSuccess)
+                         Ls, (const float*)scores, (const uint32_t*)ghist)) != cudaSuccess)
     return e;
   ++launch_counter();
   }
