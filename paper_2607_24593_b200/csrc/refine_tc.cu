@@ -41,7 +41,7 @@ constexpr int TMEM_COLS = 2 * N;
 template <int DT, int EPI = 1>
 struct RCfg {
   static constexpr bool FP8 = DT == DT_FP8;
-  static constexpr bool OVL = FP8 && EPI == 3;
+  static constexpr bool OVL = EPI == 3;
   static constexpr int NSEL = OVL ? SEL_WARPS : 2;
   // 384 threads: 168 registers per thread; 512 (with the select warps): 128
   static constexpr int THREADS = (2 + GATHER_WARPS + EPI_WARPS + (OVL ? SEL_WARPS : 0)) * 32;
@@ -51,7 +51,9 @@ struct RCfg {
   static constexpr int QROW_HALF_BYTES = kHeads * 128;
   static constexpr int QHALF_BYTES = NMEM * QROW_HALF_BYTES;
   static constexpr int QBUF_BYTES = KHALVES * QHALF_BYTES;
-  static constexpr int QBUFS = 2;                 // the next group's queries load while this one is re-scored
+  // the next group's queries load while this one is re-scored, except where 2 x 64 KB of bf16
+  // queries would leave no room for the select warps' histograms
+  static constexpr int QBUFS = (OVL && !FP8) ? 1 : 2;
   static constexpr int STAGES = FP8 ? 6 : 2;
   static constexpr int LOOKAHEAD = FP8 ? 4 : 1;   // gather tiles in flight per producer thread
   static constexpr int ROW_BYTES = FP8 ? 128 : 256;
@@ -101,7 +103,7 @@ constexpr size_t rsmem_bytes() {
   return 1024 + C::QBUFS * C::QBUF_BYTES + C::STAGES * C::STAGE_BYTES + sizeof(RCtrlT<C::MMA2, C::NSEL>);
 }
 static_assert(rsmem_bytes<DT_FP8, 0>() <= 232448 && rsmem_bytes<DT_FP8, 2>() <= 232448 &&
-              rsmem_bytes<DT_FP8, 3>() <= 232448 &&
+              rsmem_bytes<DT_FP8, 3>() <= 232448 && rsmem_bytes<DT_BF16, 3>() <= 232448 &&
               rsmem_bytes<DT_BF16>() <= 232448, "shared memory budget");
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -144,7 +146,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       ptx::mbar_init(&ct.tmem_empty[i], C::TMEM_EMPTY_ARRIVALS);
       ptx::mbar_init(&ct.a_ready[i], 4);
       ptx::mbar_init(&ct.s_ready[i], 1);
-      ptx::mbar_init(&ct.k_full[i], 4);
+      ptx::mbar_init(&ct.k_full[i], C::MMA2 ? 4 : EPI_WARPS);   // every warp that writes score rows
       ptx::mbar_init(&ct.k_free[i], SEL_WARPS);
     }
     ptx::mbar_init(&ct.w_ready, 1);
@@ -444,16 +446,17 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       uint32_t smn[NMEM], smx[NMEM], snv[NMEM];  // EPI = 3: this thread's share of the row statistics
 #pragma unroll
       for (int r = 0; r < NMEM; ++r) { smn[r] = 0xffffffffu; smx[r] = 0u; snv[r] = 0u; }
-      auto put = [&](int r, int t, int slot, int idx, uint32_t key) {
+      // (si: which of this thread's statistics slots the row uses -- a constant at every call)
+      auto put = [&](int r, int si, int t, int slot, int idx, uint32_t key) {
         const int t_r = gd.first_pos + r;
         const bool seen = idx >= 0 && idx <= t_r && idx + gd.win_span > t_r;
         if constexpr (C::OVL) {        // key only, to this group's score-row buffer
           if (r < gd.m && slot < RS) {
             const uint32_t kv = seen ? key : 0u;
             rk[(size_t)(kb * NMEM + r) * RS + slot] = kv;
-            smn[r] = (kv && kv < smn[r]) ? kv : smn[r];
-            smx[r] = kv > smx[r] ? kv : smx[r];
-            snv[r] += kv ? 1u : 0u;
+            smn[si] = (kv && kv < smn[si]) ? kv : smn[si];
+            smx[si] = kv > smx[si] ? kv : smx[si];
+            snv[si] += kv ? 1u : 0u;
           }
           return;
         }
@@ -519,7 +522,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
 #pragma unroll
             for (int r = 0; r < NMEM; ++r) {
               const float sc_r = __uint_as_float(s8[r]) + __uint_as_float(s8[4 + r]);
-              put(r, t, slot, mt.idx, score_to_key(gd.kscale ? sc_r * mt.ks : sc_r));
+              put(r, r, t, slot, mt.idx, score_to_key(gd.kscale ? sc_r * mt.ks : sc_r));
             }
           }
           if constexpr (C::OVL) {      // the group's score rows are complete: hand them over
@@ -540,6 +543,8 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         }
         all.sync();
       } else {
+      if constexpr (C::OVL)            // the select warps are through with this buffer (two groups back)
+        (void)ptx::mbar_wait(&ct.k_free[kb], kph ^ 1, abort_flag, 64);
       for (int t = 0; t < ntiles; ++t, ++it) {
         const int buf = it & 1;
         const int slot = t * TILE_KEYS + key_in_tile;
@@ -585,7 +590,23 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         if (lane == 0) ptx::mbar_arrive(&ct.tmem_empty[buf]);
 #pragma unroll
         for (int rl = 0; rl < 2; ++rl)
-          put(team * 2 + rl, t, slot, idx, score_to_key(gd.kscale ? score[rl] * ksv : score[rl]));
+          put(team * 2 + rl, rl, t, slot, idx, score_to_key(gd.kscale ? score[rl] * ksv : score[rl]));
+      }
+      if constexpr (C::OVL) {          // this warp's share of its team's two score rows is complete
+#pragma unroll
+        for (int rl = 0; rl < 2; ++rl) {
+          const int r = team * 2 + rl;
+          const uint32_t mn = __reduce_min_sync(0xffffffffu, smn[rl]);
+          const uint32_t mx = __reduce_max_sync(0xffffffffu, smx[rl]);
+          const uint32_t nv = __reduce_add_sync(0xffffffffu, snv[rl]);
+          if (lane == 0 && nv) {
+            atomicMin(&ct.kstat[kb][r][0], mn);
+            atomicMax(&ct.kstat[kb][r][1], mx);
+            atomicAdd(&ct.kstat[kb][r][2], nv);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&ct.k_full[kb]);
       }
       tm.sync();
       }
@@ -639,11 +660,14 @@ cudaError_t launch_refine_tc(const void* q, int q_rows, int dtype, const GroupDe
   if (n_groups <= 0) return cudaSuccess;
   CUtensorMap mq;
   if (!make_operand_map(&mq, q, (long long)q_rows * kHeads, dtype, kHeads, 0)) return cudaErrorInvalidValue;
-  if (dtype != DT_FP8) return launch_one<DT_BF16>(mq, groups, n_groups, q_rows, s, sms, st);
+  // the select warps need the caller's score-row buffers, long enough for every group
+  const bool rows_ok = s.rkeys && max_cand > 0 && max_cand <= s.rslots;
+  if (dtype != DT_FP8)
+    return rows_ok && !chunked ? launch_one<DT_BF16, 3>(mq, groups, n_groups, q_rows, s, sms, st)
+                               : launch_one<DT_BF16>(mq, groups, n_groups, q_rows, s, sms, st);
   if (fp32_head_sum) return launch_one<DT_FP8, 0>(mq, groups, n_groups, q_rows, s, sms, st);
   if (chunked) return launch_one<DT_FP8, 2>(mq, groups, n_groups, q_rows, s, sms, st, overlap_prev);
-  // the select warps need the caller's score-row buffers, long enough for every group
-  if (!s.rkeys || max_cand <= 0 || max_cand > s.rslots) return cudaErrorInvalidValue;
+  if (!rows_ok) return cudaErrorInvalidValue;
   return launch_one<DT_FP8, 3>(mq, groups, n_groups, q_rows, s, sms, st);
 }
 
