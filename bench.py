@@ -195,13 +195,15 @@ def decode_bench(pv, dev, steps, warmup, pk):
     pv.pivot_launch_count_reset()
     times = timed(step, steps)                                         # the step as a caller launches it
     launches = pv.pivot_launch_count_reset()
-    scan_us = []
-    pv.pivot_stage_timing(True)                                        # extra steps with events around the scan launch
+    scan_us, select_us = [], []
+    pv.pivot_stage_timing(True)                                        # extra steps with events around the scan and select launches
     for _ in range(max(3, min(steps, 5))):
         flush.fill_(1)
         step()
         torch.cuda.synchronize()
-        scan_us.append(pv.pivot_stage_times()["decode_scan"] * 1e3)
+        st_ms = pv.pivot_stage_times()
+        scan_us.append(st_ms["decode_scan"] * 1e3)
+        select_us.append(st_ms["decode_select"] * 1e3)
     pv.pivot_stage_timing(False)
     assert pv.pivot_device_status() == 0
     # the same step replayed from a CUDA graph (what a serving loop would do): launch gaps gone
@@ -286,6 +288,7 @@ def decode_bench(pv, dev, steps, warmup, pk):
     scan = float(np.mean(scan_us))
     n0 = (x.pos0.numpy().astype(np.int64) + 1)
     key_bytes = int(n0.sum()) * (D + 4)                      # e4m3 key + fp32 scale, read once per step
+    select_bytes = int(n0.sum()) * 4 + B * 8192 * 4 + B * c * 4   # scores + histograms in, candidate positions out
     # whole step: every visible key once, the c gathered candidates of each sequence once more, and
     # the step's own operands and result (queries, gates, scales, positions, index rows)
     step_bytes = key_bytes + B * c * (D + 4) + B * g * (H * D + 2 * H * 4 + k * 4) + B * 4
@@ -303,6 +306,14 @@ def decode_bench(pv, dev, steps, warmup, pk):
                               "frac": step_bytes / (us * 1e-6) / 1e9 / pk["hbm"], "algorithmic_bytes_per_step": step_bytes,
                               "frac_of_nominal_8TBs": step_bytes / (us * 1e-6) / 8e12,
                               "peak_source": pk["source"] + " STREAM copy"},
+            # the top-c select behind the scan: it reads the fp32 score of every visible key and the
+            # sequence's 8192-bin histogram, and writes c candidate positions per sequence
+            "topk_select": {"kernel": "decode_select_kernel", "bound": "hbm", "kernel_us": float(np.median(select_us)),
+                            "algorithmic_bytes_per_launch": select_bytes,
+                            "achieved": select_bytes / (float(np.median(select_us)) * 1e-6) / 1e9, "peak": pk["hbm"],
+                            "unit": "GB/s", "frac": select_bytes / (float(np.median(select_us)) * 1e-6) / 1e9 / pk["hbm"],
+                            "frac_of_nominal_8TBs": select_bytes / (float(np.median(select_us)) * 1e-6) / 8e12,
+                            "note": "latency-bound: 13 MB per launch; event time includes the launch"},
             "config": {"workload": "decode_mtp_b32_64k-128k_fp8_g2_refine", "B": B, "g": g, "c": c, "k": k,
                        "visible_keys": int(n0.sum()), "l2": "256 MB flush between steps"},
             # dominant kernel: the key-streaming scan; algorithmic bytes = visible keys x 132 B

@@ -349,8 +349,9 @@ int pivot_debug_key_stream(const void* keys_device, int n_keys, int ctas, int ti
  * returns elapsed milliseconds: ms[0] proxy build (Eq. 4), ms[1] planner, ms[2] shared scan +
  * streaming select (Eq. 5-7, and the dense rows), ms[3] gather + re-score + top-k (Eq. 8-9),
  * ms[4] the whole call.  n must be at least 5; with n >= 6, ms[5] is the key-streaming scan kernel
- * of the last decode call (0 if the last call was not a decode call).  For decode calls ms[2]
- * covers scan, select, re-score and top-k together.  Not thread-safe.
+ * of the last decode call (0 if the last call was not a decode call) and, with n >= 7, ms[6] its
+ * per-sequence top-c select kernel (Eq. 6 / Eq. 7).  For decode calls ms[2] covers scan, select,
+ * re-score and top-k together.  Not thread-safe.
  */
 int pivot_stage_timing(int enable);
 int pivot_stage_times(float* ms, int n);

@@ -359,9 +359,10 @@ def pivot_stage_timing(enable: bool):
 
 def pivot_stage_times() -> dict:
     """Elapsed ms of the last call's stages (needs pivot_stage_timing(True) before the call)."""
-    ms = (C.c_float * 6)()
-    _check(lib.pivot_stage_times(ms, 6))
-    return dict(zip(("proxy_build", "plan", "scan_select", "refine", "total", "decode_scan"), [float(v) for v in ms]))
+    ms = (C.c_float * 7)()
+    _check(lib.pivot_stage_times(ms, 7))
+    return dict(zip(("proxy_build", "plan", "scan_select", "refine", "total", "decode_scan", "decode_select"),
+                    [float(v) for v in ms]))
 
 
 def pivot_launch_count_reset() -> int:

@@ -29,7 +29,7 @@ struct DeviceState {
   cudaStream_t copy_in = nullptr, copy_out = nullptr;
   cudaEvent_t ev_entry = nullptr, ev_in[kHostChunks + 2] = {}, ev_done[kHostChunks + 2] = {};
   // stage-timing events (created on this device on first use) and what the last call recorded
-  cudaEvent_t ev[8] = {};
+  cudaEvent_t ev[9] = {};
   bool ev_valid = false, ev_decode_scan = false;
 };
 DeviceState g_dev[kMaxDevices];
@@ -140,7 +140,7 @@ bool g_timing = false;
 cudaEvent_t* timing_events() {
   DeviceState& ds = g_dev[cur_device()];
   if (!ds.ev[0])
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < 9; ++i)
       if (cudaEventCreate(&ds.ev[i]) != cudaSuccess) { ds.ev[0] = nullptr; return nullptr; }
   return ds.ev;
 }
@@ -440,6 +440,7 @@ static int run_decode(const pivot_tensor* q, const float* w, const pivot_tensor*
     cudaEvent_t* tev = g_timing ? timing_events() : nullptr;
     df.ev_scan_begin = tev ? tev[6] : nullptr;
     df.ev_scan_end = tev ? tev[7] : nullptr;
+    df.ev_select_end = tev ? tev[8] : nullptr;
     g_dev[cur_device()].ev_decode_scan = tev != nullptr;
     if ((rc = check_cuda(launch_decode_fast(df, st)))) return rc;
     // dense rows of guarded (short) sequences, if any: the generic scan, one row per block
@@ -695,6 +696,10 @@ int pivot_stage_times(float* ms, int n) {
   if (n >= 6) {
     ms[5] = 0.f;
     if (ds.ev_decode_scan && (rc = check_cuda(cudaEventElapsedTime(&ms[5], ev[6], ev[7])))) return rc;
+  }
+  if (n >= 7) {
+    ms[6] = 0.f;
+    if (ds.ev_decode_scan && (rc = check_cuda(cudaEventElapsedTime(&ms[6], ev[7], ev[8])))) return rc;
   }
   return PIVOT_OK;
 }

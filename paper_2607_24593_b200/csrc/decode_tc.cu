@@ -680,6 +680,7 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
                          Ls, (const float*)scores, (const uint32_t*)ghist)) != cudaSuccess)
     return e;
   ++launch_counter();
+  if (d.ev_scan_end && d.ev_select_end) cudaEventRecord(d.ev_select_end, st);
   }
   if (d.mode == 1) {
     if (W > 0) {

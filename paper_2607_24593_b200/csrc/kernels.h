@@ -155,6 +155,7 @@ struct DecodeFast {
   ScanScratch scratch_tc;     // candidate scratch of the re-score kernel
   int* status;
   cudaEvent_t ev_scan_begin, ev_scan_end;   // optional: recorded around the scan kernel
+  cudaEvent_t ev_select_end = nullptr;      // ... and behind the per-sequence select
 };
 size_t decode_fast_bytes(int B, int Lmax, int g, int c);
 cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st);
