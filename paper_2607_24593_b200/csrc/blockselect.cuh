@@ -21,10 +21,23 @@ struct BlkSelSmem {
 // bin b) / sm.pop (population of bin b); bin = 0, pop = need = 0 if the total is below `need`.
 __device__ __forceinline__ void blk_boundary(BlkSelSmem& sm, const uint32_t* hist, int nbins, uint32_t need) {
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  const int per = nbins >> 10;
+  const int per = nbins >> 10;                // 1 .. 16 bins per thread, walked from the top
   __syncthreads();
+  // this thread's bins in registers, highest first: all loads are issued before the first is used
+  uint32_t h[16];
+  const uint32_t* top = hist + nbins - 1 - per * tid;
+  if (per == 8 && (reinterpret_cast<uintptr_t>(hist) & 15) == 0) {
+    const uint4 a = *reinterpret_cast<const uint4*>(top - 7), c4 = *reinterpret_cast<const uint4*>(top - 3);
+    h[0] = c4.w; h[1] = c4.z; h[2] = c4.y; h[3] = c4.x; h[4] = a.w; h[5] = a.z; h[6] = a.y; h[7] = a.x;
+#pragma unroll
+    for (int i = 8; i < 16; ++i) h[i] = 0u;
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) h[i] = i < per ? top[-i] : 0u;
+  }
   uint32_t s = 0;
-  for (int i = 0; i < per; ++i) s += hist[nbins - 1 - per * tid - i];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) s += h[i];
   uint32_t incl = s;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -34,20 +47,28 @@ __device__ __forceinline__ void blk_boundary(BlkSelSmem& sm, const uint32_t* his
   if (lane == 31) sm.wsum[wid] = incl;
   if (tid == 0) { sm.bin = 0; sm.need = 0; sm.pop = 0; }
   __syncthreads();
-  uint32_t base = 0;
-  for (int w = 0; w < wid; ++w) base += sm.wsum[w];
+  // entries in the warps before this one: a warp scan over the 32 warp totals
+  uint32_t wincl = sm.wsum[lane];
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t v = __shfl_up_sync(0xffffffffu, wincl, o);
+    if (lane >= o) wincl += v;
+  }
+  const uint32_t wtot = sm.wsum[wid];
+  const uint32_t base = __shfl_sync(0xffffffffu, wincl, wid) - wtot;
   const uint32_t excl = base + incl - s;
   if (excl < need && need <= excl + s) {
     uint32_t cum = excl;
-    for (int i = 0; i < per; ++i) {
-      const uint32_t h = hist[nbins - 1 - per * tid - i];
-      if (cum + h >= need) {
+    bool done = false;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      if (!done && i < per && cum + h[i] >= need) {
         sm.bin = (uint32_t)(nbins - 1 - per * tid - i);
         sm.need = need - cum;
-        sm.pop = h;
-        break;
+        sm.pop = h[i];
+        done = true;
       }
-      cum += h;
+      cum += h[i];
     }
   }
   __syncthreads();
