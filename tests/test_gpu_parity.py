@@ -193,6 +193,32 @@ def test_ties_all_equal_scores(pv, gu):
         assert (out[t, n:] == -1).all()
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+def test_heavy_ties_few_distinct_keys(pv, gu, dtype):
+    """Eight distinct key vectors repeated over the whole cache: every row's scores take at most eight
+    values, so the c-th and k-th thresholds always sit inside a tie class of hundreds of keys -- the
+    boundary bins of the scan's finisher, of the re-score's select warps and of their narrowing rounds
+    are as crowded as they get.  Checked with the acceptance rule (any member of a tie class within
+    the tolerance of the threshold is a valid pick) and, where every score is equal, exactly."""
+    L, g, c, k = 2600, 4, 700, 300
+    x = inputs.make_prefill(L, dtype=dtype, seed=41)
+    x.k[:] = x.k[:8].repeat((L + 7) // 8, 1)[:L]
+    if x.kscale is not None:
+        x.kscale[:] = x.kscale[:8].repeat((L + 7) // 8)[:L]
+    for mode in (po.MODE_REUSE, po.MODE_REFINE):
+        out, sc, cand, cs = gu.run_prefill(x, g=g, c=c, k=k, mode=mode)
+        nG = (L + g - 1) // g
+        groups = [0, 1, 174, 175, 176, 300, 449, nG - 1]
+        t = acc.check_prefill(x.codes(), g=g, c=c, k=k, mode=mode, guard_len=None, out_idx=out, out_scores=sc,
+                              cand=cand, cand_scores=cs, groups=groups)
+        _report(f"heavy ties {dtype} mode={mode}", t)
+        # no duplicates, nothing from the future, full rows once enough keys are visible
+        for tq in (299, 300, 1234, L - 1):
+            row = out[tq]
+            vis = row[row >= 0]
+            assert len(set(vis.tolist())) == len(vis) == min(k, tq + 1) and vis.max() <= tq
+
+
 def test_pool_variants(pv, gu):
     x = inputs.make_prefill(600, dtype="fp8", seed=8)
     for pool, name in ((pv.POOL_FIRST, "first"), (pv.POOL_LAST, "last")):
