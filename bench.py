@@ -324,6 +324,49 @@ def decode_bench(pv, dev, steps, warmup, pk):
                          "frac_of_nominal_8TBs": key_bytes / (scan * 1e-6) / 8e12}}
 
 
+def counters_run(pv, dev, wl):
+    """One prefill request and one decode step under the -DPIVOT_PROF build; the kernels' cycle counters,
+    normalised per tile / group / sequence (clocks, averaged over the CTAs)."""
+    L, dtype, g, c, k, mode = WORKLOADS[wl]
+    x = inputs.make_prefill(L, dtype=dtype, seed=rank_seed(0))
+    dq, dw, dk = x.q.to(dev), x.w.to(dev), x.k.to(dev)
+    dqs = None if x.qscale is None else x.qscale.to(dev)
+    dks = None if x.kscale is None else x.kscale.to(dev)
+    out = torch.empty((L, k), dtype=torch.int32, device=dev)
+    pv.ensure_workspace(L, (L + g - 1) // g, c, k, dev)
+    res = {"workload": wl}
+
+    def per(v, a, b, names):
+        n = max(v[b], 1)
+        return {nm: round(v[a + "_" + nm] / n, 1) for nm in names}
+
+    for rep_ in range(2):                       # the first pass also clears whatever the workspace held
+        pv.pivot_index_prefill(dq, dw, dk, L, H, D, g, c, k, mode, out, q_scale=dqs, k_scale=dks)
+        v = pv.pivot_debug_counters()
+    waits = ("wait_queries", "wait_accumulator", "wait_keys", "wait_gates", "wait_relu", "total")
+    res["scan_mma_thread_clocks_per_tile"] = per(v, "scan", "scan_tiles", waits)
+    res["scan_tiles"] = v["scan_tiles"]
+    if v["rescore_tiles"]:
+        res["rescore_mma_thread_clocks_per_tile"] = per(v, "rescore", "rescore_tiles", waits)
+        res["rescore_select_warp_clocks_per_group"] = {
+            "waiting_for_score_rows": round(v["rescore_select_wait"] / max(v["rescore_select_groups"], 1), 1),
+            "selecting": round(v["rescore_select_work"] / max(v["rescore_select_groups"], 1), 1)}
+    B, gd = 32, 2
+    xd = inputs.make_decode(B, gd, 65536, 131072, dtype="fp8")
+    Lmax = xd.k.shape[1]
+    q, w, kc, p0 = xd.q.to(dev), xd.w.to(dev), xd.k.to(dev), xd.pos0.to(dev)
+    qs, ks = xd.qscale.to(dev), xd.kscale.to(dev)
+    od = torch.empty((B, gd, 2048), dtype=torch.int32, device=dev)
+    pv.ensure_workspace(B * gd, B, 4096, 2048, dev, need=pv.pivot_decode_workspace_bytes(B, Lmax, gd, 4096, 2048))
+    for rep_ in range(2):
+        pv.pivot_index_decode(q, w, kc, p0, B, Lmax, H, D, gd, 4096, 2048, pv.REFINE, od, None, q_scale=qs, k_scale=ks)
+        v = pv.pivot_debug_counters()
+    n = max(v["decode_select_sequences"], 1)
+    res["decode_select_clocks_per_sequence"] = {nm: round(v["decode_select_" + nm] / n, 1)
+                                                for nm in ("boundary", "collect", "handover", "topk")}
+    return res
+
+
 def oracle_sample_time(x, L, g, c, k, mode, n_groups, seed):
     """Times the CPU oracle (as it stands) on a uniform random sample of groups; returns
     (estimated seconds for the whole request, seconds spent, groups timed, threads used)."""
@@ -486,12 +529,19 @@ def main():
     ap.add_argument("--mma-model", action="store_true",
                     help="one-SM timing probe behind the per-tile model of the scan (tensor pipe, tensor-memory port, "
                          "hand-overs): prints one JSON object of clocks per tile")
+    ap.add_argument("--counters", action="store_true",
+                    help="build the library with -DPIVOT_PROF (libpivot_prof.so), run one prefill request of the chosen "
+                         "workload and one MTP decode step, and print the kernels' own cycle counters per tile / group / "
+                         "sequence (where the MMA-issuing threads wait, the re-score's select warps, the decode select)")
     ap.add_argument("--sweep", action="store_true",
                     help="g / c / pooling / window sweep with recall of the dense top-k (one JSON line per case)")
     args = ap.parse_args()
     wl = args.workload
     if args.impl == "reference":
         return run_reference(args, wl)
+    if args.counters:
+        from paper_2607_24593_b200 import build as pbuild
+        os.environ["PIVOT_LIB"] = os.path.basename(pbuild.build_variant("prof", ["-DPIVOT_PROF"]))
 
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # started as a plain `python bench.py --gpus N`: become N ranks, one per GPU
@@ -508,6 +558,9 @@ def main():
 
     from paper_2607_24593_b200 import binding as pv
 
+    if args.counters:
+        print(json.dumps(counters_run(pv, torch.device(f"cuda:{local}"), wl), indent=1))
+        return
     if args.mma_model:
         res = {"mma_model": pv.pivot_debug_mma_model(), "key_stream": []}
         for ctas, stages, mode in ((1, 4, 0), (148, 2, 0), (148, 4, 0), (148, 12, 0), (148, 4, 1), (148, 4, 2), (1, 4, 2), (148, 4, 3), (148, 4, 4)):

@@ -344,6 +344,19 @@ int pivot_debug_key_stream(const void* keys_device, int n_keys, int ctas, int ti
                            long long* out_device, pivot_stream_t stream);
 
 /*
+ * Diagnostic (no counterpart in the paper): cycle counters of a library built with -DPIVOT_PROF
+ * (`python -m paper_2607_24593_b200.build --variant prof -DPIVOT_PROF`), summed over all CTAs and
+ * calls since the last read: where the thread that issues the tensor-core instructions of Eq. 5's
+ * scan and of Eq. 8's re-score waits, how long the re-score's select warps take for Eq. 9, and the
+ * phases of the decode step's top-c select (Eq. 7).  out (host) receives the first n <= 28 slots
+ * (ProfSlot in csrc/common.cuh) of the workspace last used on this device and the slots are
+ * cleared; the first read after a workspace is registered returns whatever the memory held.
+ * Synchronises on `stream`.  PIVOT_ERR_UNSUPPORTED in an ordinary build, PIVOT_ERR_WORKSPACE
+ * before any call.
+ */
+int pivot_debug_counters(pivot_stream_t stream, unsigned long long* out, int n);
+
+/*
  * Per-stage timing, off by default.  While enabled, every call records CUDA events on its own
  * stream around its stages; pivot_stage_times synchronises on the last call's final event and
  * returns elapsed milliseconds: ms[0] proxy build (Eq. 4), ms[1] planner, ms[2] shared scan +

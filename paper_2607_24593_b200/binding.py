@@ -28,7 +28,7 @@ SYMBOLS = [
     "pivot_index_decode", "pivot_index_decode_ex", "pivot_index_decode_paged", "dense_index", "dense_index_ex", "dense_index_static",
     "pivot_prefill_host_arena_bytes", "pivot_index_prefill_host", "pivot_device_status",
     "pivot_stage_timing", "pivot_stage_times", "pivot_launch_count_reset", "pivot_status_str", "pivot_last_cuda_error",
-    "dense_index_decode", "dense_index_decode_ex", "pivot_debug_wait_expiry", "pivot_debug_mma_model", "pivot_debug_key_stream", "pivot_merge_topk",
+    "dense_index_decode", "dense_index_decode_ex", "pivot_debug_wait_expiry", "pivot_debug_mma_model", "pivot_debug_key_stream", "pivot_debug_counters", "pivot_merge_topk",
 ]
 DEV_OK, DEV_WAIT_EXPIRED, DEV_CAND_OVERFLOW, DEV_BAD_POS, DEV_BOUNDS = 0, 1, 2, 3, 4
 
@@ -74,6 +74,7 @@ def _load():
     lib.pivot_debug_wait_expiry.argtypes = [C.c_ulonglong, P]
     lib.pivot_debug_mma_model.argtypes = [P, P]
     lib.pivot_debug_key_stream.argtypes = [P, I, I, I, I, I, P, P]
+    lib.pivot_debug_counters.argtypes = [P, C.POINTER(C.c_ulonglong), I]
     lib.pivot_merge_topk.argtypes = [P, P, I, I, P, I, P, P, P]
     lib.pivot_prefill_host_arena_bytes.restype = S
     lib.pivot_prefill_host_arena_bytes.argtypes = [I, I, I, I, I, I, I]
@@ -315,6 +316,23 @@ def pivot_debug_mma_model(stream=None) -> dict:
             d["traffic warps: clk per 256-column pass"] = [x for x in v[ph * 32 + 16: ph * 32 + 24] if x]
         res[pname] = d
     return res
+
+
+PROF_SLOTS = ("scan_wait_queries", "scan_wait_accumulator", "scan_wait_keys", "scan_wait_gates", "scan_wait_relu",
+              "scan_total", "scan_tiles",
+              "rescore_wait_queries", "rescore_wait_accumulator", "rescore_wait_keys", "rescore_wait_gates",
+              "rescore_wait_relu", "rescore_total", "rescore_tiles",
+              "rescore_select_wait", "rescore_select_work", "rescore_select_groups",
+              "decode_select_boundary", "decode_select_collect", "decode_select_handover", "decode_select_topk",
+              "decode_select_sequences")
+
+
+def pivot_debug_counters(stream=None) -> dict:
+    """Cycle counters of a -DPIVOT_PROF build since the last read (read and cleared); raises in an
+    ordinary build."""
+    out = (C.c_ulonglong * len(PROF_SLOTS))()
+    _check(lib.pivot_debug_counters(_stream(stream), out, len(PROF_SLOTS)))
+    return dict(zip(PROF_SLOTS, [int(v) for v in out]))
 
 
 def pivot_debug_key_stream(n_keys=131072, ctas=148, tiles=2048, stages=4, mode=0, stream=None) -> dict:

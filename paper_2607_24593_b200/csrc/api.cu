@@ -677,6 +677,21 @@ int pivot_device_status(pivot_stream_t stream, int* status) {
   return rc;
 }
 
+int pivot_debug_counters(pivot_stream_t stream, unsigned long long* out, int n) {
+#ifdef PIVOT_PROF
+  if (!out || n < 1 || n > 28) return PIVOT_ERR_INVALID_ARG;
+  int* p = g_dev[cur_device()].last_status;
+  if (!p) return PIVOT_ERR_WORKSPACE;
+  int rc = check_cuda(cudaStreamSynchronize((cudaStream_t)stream));
+  if (rc) return rc;
+  if ((rc = check_cuda(cudaMemcpy(out, p + 8, (size_t)n * 8, cudaMemcpyDeviceToHost)))) return rc;
+  return check_cuda(cudaMemset(p + 8, 0, 28 * 8));                   // read and cleared
+#else
+  (void)stream; (void)out; (void)n;
+  return PIVOT_ERR_UNSUPPORTED;                                        // the library was built without -DPIVOT_PROF
+#endif
+}
+
 int pivot_stage_timing(int enable) {
   if (enable && !timing_events()) { (void)check_cuda(cudaGetLastError()); return PIVOT_ERR_CUDA; }
   g_timing = enable != 0;

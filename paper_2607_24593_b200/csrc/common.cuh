@@ -19,6 +19,44 @@ constexpr int DEV_CAND_OVERFLOW = 2;  // a candidate buffer would have overflowe
 constexpr int DEV_BAD_POS = 3;        // decode: a sequence's pos0 lies outside [0, Lmax - g]; its rows are all -1
 constexpr int DEV_BOUNDS = 4;         // PIVOT_DEBUG builds: an index, page or cursor failed its bounds check (access skipped)
 
+// Cycle counters of a -DPIVOT_PROF build (the figures the profiles quote): 64-bit slots in the
+// workspace head, behind the status word and the row counter (ints 8 .. 63), summed over all CTAs
+// and calls until pivot_debug_counters reads and clears them.  An ordinary build has none of it.
+enum ProfSlot {
+  PROF_SCAN_WAIT_QUERIES = 0,   // shared scan, MMA-issuing thread: clocks waiting for the block's queries,
+  PROF_SCAN_WAIT_ACC,           //   a free accumulator buffer,
+  PROF_SCAN_WAIT_KEYS,          //   the key tile,
+  PROF_SCAN_WAIT_GATES,         //   the block's gate matrix,
+  PROF_SCAN_WAIT_RELU,          //   the packed ReLU operand of the second MMA,
+  PROF_SCAN_TOTAL,              //   its whole loop; and
+  PROF_SCAN_TILES,              //   tiles it issued
+  PROF_REF_WAIT_QUERIES,        // re-score, MMA-issuing thread: the same seven
+  PROF_REF_WAIT_ACC,
+  PROF_REF_WAIT_KEYS,
+  PROF_REF_WAIT_GATES,
+  PROF_REF_WAIT_RELU,
+  PROF_REF_TOTAL,
+  PROF_REF_TILES,
+  PROF_REF_SEL_WAIT,            // re-score, select warp of member 0: clocks waiting for a group's score rows,
+  PROF_REF_SEL_WORK,            //   selecting; and
+  PROF_REF_SEL_GROUPS,          //   groups selected
+  PROF_DSEL_BOUNDARY,           // decode select, the CTA that takes the top-c: boundary bin off the histogram,
+  PROF_DSEL_COLLECT,            //   collecting its share of the scores,
+  PROF_DSEL_HANDOVER,           //   cluster barriers + reading the other CTAs' lists,
+  PROF_DSEL_TOPK,               //   exact top-c of the collected entries; and
+  PROF_DSEL_SEQS,               //   sequences
+  PROF_SLOTS
+};
+static_assert(PROF_SLOTS <= 28, "the workspace head holds 28 counters");
+#ifdef PIVOT_PROF
+__device__ __forceinline__ void prof_add(int* status, int slot, long long v) {
+  if (status) atomicAdd(reinterpret_cast<unsigned long long*>(status + 8) + slot, (unsigned long long)v);
+}
+#define PIVOT_PROF_DO(...) __VA_ARGS__
+#else
+#define PIVOT_PROF_DO(...)
+#endif
+
 // fp32 score -> uint32 key whose unsigned order equals the float order (-inf lowest).
 __device__ __forceinline__ uint32_t score_to_key(float s) {
   uint32_t b = __float_as_uint(s);

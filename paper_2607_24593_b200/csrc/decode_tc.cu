@@ -296,12 +296,13 @@ struct SelSmem {
 // The SEL_SPLIT CTAs of a sequence are one thread-block cluster (blockIdx.x = rank in it).
 __global__ void __cluster_dims__(SEL_SPLIT, 1, 1) __launch_bounds__(kBlk, 1)
 decode_select_kernel(const RowDesc* __restrict__ prox, int Ls, const float* __restrict__ scores,
-                     const uint32_t* __restrict__ ghist) {
+                     const uint32_t* __restrict__ ghist, int* status) {
   extern __shared__ uint8_t sel_raw[];
   SelSmem& sm = *reinterpret_cast<SelSmem*>(((uintptr_t)sel_raw + 15) & ~(uintptr_t)15);
   const int split = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31;
   ptx::grid_launch_dependents();
   ptx::grid_dependency_wait();            // the scan's scores and histograms (before any early return)
+  PIVOT_PROF_DO(long long pt[5]; pt[0] = clock64();)
   const RowDesc rd = prox[b];
   const int K = rd.K, n0 = rd.n_vis;
   if (K <= 0) return;
@@ -352,6 +353,7 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Ls, const float* __re
       pbits += wbits;
     }
   }
+  PIVOT_PROF_DO(pt[1] = clock64();)
   // ---- collect them in shared memory: this CTA's share of the scores (multiples of four)
   const int lo = solo ? 0 : (int)(((long long)n0 * split / SEL_SPLIT) & ~3ll);
   const int hi = (solo || split == SEL_SPLIT - 1) ? n0 : (int)(((long long)n0 * (split + 1) / SEL_SPLIT) & ~3ll);
@@ -412,6 +414,7 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Ls, const float* __re
     }
   }
   __syncthreads();
+  PIVOT_PROF_DO(pt[2] = clock64();)
   int n = min((int)sm.blk.list_n, SEL_CAP);
   if (!solo) {
     // ---- hand the shares over: the four CTAs of a sequence form a cluster, and CTA 0 reads the
@@ -431,7 +434,14 @@ decode_select_kernel(const RowDesc* __restrict__ prox, int Ls, const float* __re
     if (split != 0) return;
     __syncthreads();
   }
+  PIVOT_PROF_DO(pt[3] = clock64();)
   blk_emit_topk(sm.blk, sm.list, n, n, K, rd.out, rd.out_score, rd.out_rows, rd.out_stride);
+  PIVOT_PROF_DO(__syncthreads(); if (tid == 0) {
+    pt[4] = clock64();
+    for (int i = 0; i < 4; ++i) prof_add(status, PROF_DSEL_BOUNDARY + i, pt[i + 1] - pt[i]);
+    prof_add(status, PROF_DSEL_SEQS, 1);
+  })
+  (void)status;
 }
 
 // ------------------------------------------------------------------------------ top-k of entry lists
@@ -677,7 +687,7 @@ cudaError_t launch_decode_fast(const DecodeFast& d, cudaStream_t st) {
   const size_t sel_smem = sizeof(SelSmem) + 16;
   if ((e = opt_in_dynamic_smem(decode_select_kernel, sel_smem, sel_attr)) != cudaSuccess) return e;
   if ((e = launch_kernel(decode_select_kernel, dim3(SEL_SPLIT, d.B), dim3(kBlk), sel_smem, st, true, (const RowDesc*)d.prox,
-                         Ls, (const float*)scores, (const uint32_t*)ghist)) != cudaSuccess)
+                         Ls, (const float*)scores, (const uint32_t*)ghist, d.status)) != cudaSuccess)
     return e;
   ++launch_counter();
   if (d.ev_scan_end && d.ev_select_end) cudaEventRecord(d.ev_select_end, st);

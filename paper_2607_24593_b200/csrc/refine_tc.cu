@@ -198,15 +198,26 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       // MMA2: the head sum of tile it-1 follows the first MMA of tile it (see the shared scan)
       bool pend = false;
       uint32_t pend_it = 0, pend_blk = 0, w_blk = 0xffffffffu;
+      // (a -DPIVOT_PROF build times this thread's waits: PW(slot, wait) adds the wait's clocks to pw[slot])
+      PIVOT_PROF_DO(long long pw[6] = {0, 0, 0, 0, 0, 0}; const long long pstart = clock64();)
+#ifdef PIVOT_PROF
+#define PW(i, ...) { const long long t_ = clock64(); __VA_ARGS__; pw[i] += clock64() - t_; }
+#else
+#define PW(i, ...) __VA_ARGS__;
+#endif
       auto issue_mma2 = [&]() -> bool {
         if (pend_blk != w_blk) {                 // first tile of a group: its gate matrix must be in place
-          if (!ptx::mbar_wait(&ct.w_ready, pend_blk & 1, abort_flag, 0)) return false;
+          bool okw;
+          PW(3, okw = ptx::mbar_wait(&ct.w_ready, pend_blk & 1, abort_flag, 0))
+          if (!okw) return false;
           w_blk = pend_blk;
         }
         const int pb = pend_it & 1;
         // no sleep between polls here or on the accumulator / key-stage waits below: this thread's
         // wake-up latency sits on the tile loop's critical path (four handoffs per tile)
-        if (!ptx::mbar_wait_poll(&ct.a_ready[pb], (pend_it >> 1) & 1, abort_flag)) return false;
+        bool oka;
+        PW(4, oka = ptx::mbar_wait_poll(&ct.a_ready[pb], (pend_it >> 1) & 1, abort_flag))
+        if (!oka) return false;
         ptx::tc_fence_after();
         const uint32_t w_addr = ptx::smem_u32(ct.wmat);
         const uint32_t a_tmem = tmem_base + pb * N;
@@ -225,16 +236,16 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         const int ntiles = group_tiles(groups[gi]);
         if (ntiles == 0) continue;
         const int qb = blk % C::QBUFS;
-        ok = ptx::mbar_wait(&ct.q_full[qb], (blk / C::QBUFS) & 1, abort_flag, 32);
+        PW(0, ok = ptx::mbar_wait(&ct.q_full[qb], (blk / C::QBUFS) & 1, abort_flag, 32))
         if (!ok) break;
         const uint32_t q_addr = ptx::smem_u32(qbuf + qb * C::QBUF_BYTES);
         for (int t = 0; t < ntiles; ++t, ++it) {
           const int s = it % C::STAGES;
           const uint32_t ph = (it / C::STAGES) & 1;
           const int buf = it & 1;
-          ok = ptx::mbar_wait_poll(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag);
+          PW(1, ok = ptx::mbar_wait_poll(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag))
           if (!ok) break;
-          ok = ptx::mbar_wait_poll(&ct.full[s], ph, abort_flag);
+          PW(2, ok = ptx::mbar_wait_poll(&ct.full[s], ph, abort_flag))
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t k_addr = ptx::smem_u32(kring + s * C::STAGE_BYTES);
@@ -261,6 +272,12 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         ptx::tc_commit(&ct.q_empty[qb]);
         ++blk;
       }
+#undef PW
+      PIVOT_PROF_DO(if (C::OVL && C::MMA2) {
+        pw[5] = clock64() - pstart;
+        for (int i = 0; i < 6; ++i) prof_add(sc.status, PROF_REF_WAIT_QUERIES + i, pw[i]);
+        prof_add(sc.status, PROF_REF_TILES, it);
+      })
     }
   } else if (warp < 2 + GATHER_WARPS) {
     // ------------------------------------------------------------------ gather producers
@@ -362,7 +379,9 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       const int kb = blk & 1;
       const uint32_t kph = (blk >> 1) & 1;
       ++blk;
+      PIVOT_PROF_DO(const long long pt0 = clock64();)
       if (!ptx::mbar_wait(&ct.k_full[kb], kph, abort_flag, 64)) break;
+      PIVOT_PROF_DO(const long long pt1 = clock64();)
       const uint32_t kmin = ct.kstat[kb][r][0], kmax = ct.kstat[kb][r][1], n_filled = ct.kstat[kb][r][2];
       __syncwarp();
       if (lane == 0) { ct.kstat[kb][r][0] = 0xffffffffu; ct.kstat[kb][r][1] = 0u; ct.kstat[kb][r][2] = 0u; }
@@ -377,6 +396,11 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         }
       }
       __syncwarp();
+      PIVOT_PROF_DO(if (r == 0 && lane == 0) {
+        prof_add(sc.status, PROF_REF_SEL_WAIT, pt1 - pt0);
+        prof_add(sc.status, PROF_REF_SEL_WORK, clock64() - pt1);
+        prof_add(sc.status, PROF_REF_SEL_GROUPS, 1);
+      })
       if (lane == 0) ptx::mbar_arrive(&ct.k_free[kb]);     // this warp is through with the buffer
     }
   } else {

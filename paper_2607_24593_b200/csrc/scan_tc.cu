@@ -233,13 +233,24 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       // bf16 ReLU values in place -- is produced while that MMA runs).
       bool pend = false;
       uint32_t pend_it = 0, pend_blk = 0, w_blk = 0xffffffffu;
+      // (a -DPIVOT_PROF build times this thread's waits: PW(slot, wait) adds the wait's clocks to pw[slot])
+      PIVOT_PROF_DO(long long pw[6] = {0, 0, 0, 0, 0, 0}; const long long pstart = clock64();)
+#ifdef PIVOT_PROF
+#define PW(i, ...) { const long long t_ = clock64(); __VA_ARGS__; pw[i] += clock64() - t_; }
+#else
+#define PW(i, ...) __VA_ARGS__;
+#endif
       auto issue_mma2 = [&]() -> bool {
         if (pend_blk != w_blk) {                 // first tile of a block: its gate matrix must be in place
-          if (!ptx::mbar_wait(&ct.w_ready, pend_blk & 1, abort_flag, 32)) return false;
+          bool okw;
+          PW(3, okw = ptx::mbar_wait(&ct.w_ready, pend_blk & 1, abort_flag, 32))
+          if (!okw) return false;
           w_blk = pend_blk;
         }
         const int pb = pend_it & 1;
-        if (!ptx::mbar_wait(&ct.a_ready[pb], (pend_it >> 1) & 1, abort_flag, 32)) return false;
+        bool oka;
+        PW(4, oka = ptx::mbar_wait(&ct.a_ready[pb], (pend_it >> 1) & 1, abort_flag, 32))
+        if (!oka) return false;
         ptx::tc_fence_after();
         const uint32_t w_addr = ptx::smem_u32(ct.wmat);
         const uint32_t a_tmem = tmem_base + pb * C::N;
@@ -256,16 +267,16 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         const int ntiles = block_tiles(rows, n_rows, b, NROWS, &k_row0);
         if (ntiles == 0) continue;
         const int qb = blk % C::QBUFS;
-        ok = ptx::mbar_wait(&ct.q_full[qb], (blk / C::QBUFS) & 1, abort_flag, 32);
+        PW(0, ok = ptx::mbar_wait(&ct.q_full[qb], (blk / C::QBUFS) & 1, abort_flag, 32))
         if (!ok) break;
         const uint32_t q_addr = ptx::smem_u32(qbuf + qb * C::QBUF_BYTES);
         for (int t = 0; t < ntiles; ++t, ++it) {
           const int s = it % C::STAGES;
           const uint32_t ph = (it / C::STAGES) & 1;
           const int buf = it & 1;
-          ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, 32);
+          PW(1, ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, 32))
           if (!ok) break;
-          ok = ptx::mbar_wait(&ct.full[s], ph, abort_flag, 32);
+          PW(2, ok = ptx::mbar_wait(&ct.full[s], ph, abort_flag, 32))
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t k_addr = ptx::smem_u32(kring + s * C::STAGE_BYTES);
@@ -291,6 +302,12 @@ scan_select_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       if constexpr (C::MMA2) {
         if (pend && ok) (void)issue_mma2();
       }
+#undef PW
+      PIVOT_PROF_DO(if (C::MMA2) {
+        pw[5] = clock64() - pstart;
+        for (int i = 0; i < 6; ++i) prof_add(sc.status, PROF_SCAN_WAIT_QUERIES + i, pw[i]);
+        prof_add(sc.status, PROF_SCAN_TILES, it);
+      })
     }
   } else if (warp < 2 + C::EPI_WARPS) {
     // ------------------------------------------------------------------ score warps
