@@ -90,6 +90,8 @@ struct RCtrlT {
   KeyMeta meta[META_SLOTS][TILE_KEYS];   // written by the gather warps, read by the epilogue
   uint64_t full[MAX_STAGES], empty[MAX_STAGES];
   uint64_t q_full[2], q_empty[2], tmem_full[2], tmem_empty[2];
+  uint64_t g_ready[2];                           // a group's gates are staged (query warp -> score warps)
+  alignas(16) float gstage[2][MMA2 ? NMEM * kHeads : 4];
   uint64_t k_full[2], k_free[2];                 // score rows of a group: score warps -> select warps
   uint32_t kstat[2][NMEM][4];                    // ... and each row's smallest / largest key and filled slots
   uint32_t tmem_base;
@@ -148,6 +150,7 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
       ptx::mbar_init(&ct.s_ready[i], 1);
       ptx::mbar_init(&ct.k_full[i], C::MMA2 ? 4 : EPI_WARPS);   // every warp that writes score rows
       ptx::mbar_init(&ct.k_free[i], SEL_WARPS);
+      ptx::mbar_init(&ct.g_ready[i], 1);
     }
     ptx::mbar_init(&ct.w_ready, 1);
     for (int i = 0; i < 2 * NMEM; ++i) {
@@ -174,21 +177,43 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
 
   if (warp == 0) {
     // ------------------------------------------------------------------ member-query TMA
-    if (ptx::elect_one()) {
-      ptx::prefetch_tensormap(&tm_q);
-      uint32_t blk = 0;
-      for (int gi = blockIdx.x; gi < n_groups; gi += gridDim.x) {
-        const GroupDesc gd = groups[gi];
-        if (group_tiles(gd) == 0) continue;
-        const int qb = blk % C::QBUFS;
-        if (!ptx::mbar_wait(&ct.q_empty[qb], ((blk / C::QBUFS) & 1) ^ 1, abort_flag, 128)) break;
+    // ... and, for the tensor-core head sum, the group's effective gates: fetched here, up to two
+    // groups ahead, into a small staging array, so that the warps that build the gate matrix at
+    // the start of a group find them in shared memory instead of behind two global round trips.
+    // (A staging slot is free when the query buffer of the same parity is: the group that used
+    // it has issued its last MMA, and its gate matrix was built before its first.)
+    const bool leader = ptx::elect_one();
+    if (leader) ptx::prefetch_tensormap(&tm_q);
+    uint32_t blk = 0;
+    for (int gi = blockIdx.x; gi < n_groups; gi += gridDim.x) {
+      const GroupDesc gd = groups[gi];
+      if (group_tiles(gd) == 0) continue;
+      const int qb = blk % C::QBUFS;
+      if (!ptx::mbar_wait(&ct.q_empty[qb], ((blk / C::QBUFS) & 1) ^ 1, abort_flag, 128)) break;
+      if (leader) {
         ptx::mbar_arrive_expect_tx(&ct.q_full[qb], gd.m * C::KHALVES * C::QROW_HALF_BYTES);
         for (int r = 0; r < gd.m; ++r)
           for (int h = 0; h < C::KHALVES; ++h)
             ptx::tma_load_2d(qbuf + qb * C::QBUF_BYTES + h * C::QHALF_BYTES + r * C::QROW_HALF_BYTES, &tm_q,
                              h * 64, (gd.q_row + r) * kHeads, &ct.q_full[qb]);
-        ++blk;
       }
+      if constexpr (C::MMA2) {
+        float wv[NMEM * kHeads / 32];
+#pragma unroll
+        for (int u = 0; u < NMEM * kHeads / 32; ++u) {
+          const int i = u * 32 + lane, r = i >> 6, j = i & 63;
+          wv[u] = 0.f;
+          if (r < gd.m) {
+            wv[u] = gd.w[r * kHeads + j];
+            if (gd.qscale) wv[u] = __fmul_rn(wv[u], gd.qscale[r * kHeads + j]);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < NMEM * kHeads / 32; ++u) ct.gstage[blk & 1][u * 32 + lane] = wv[u];
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&ct.g_ready[blk & 1]);
+      }
+      ++blk;
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -434,14 +459,11 @@ refine_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const GroupDesc* __re
         // second MMA of the previous group is through (its scores have been read)
         all.sync();
         if (team == 1) {
+          (void)ptx::mbar_wait(&ct.g_ready[kb], kph, abort_flag);   // staged by the query warp, usually long ago
 #pragma unroll
           for (int u = 0; u < 2; ++u) {
             const int i = tt + u * 128, r = i >> 6, j = i & 63;
-            float wv = 0.f;
-            if (r < gd.m) {
-              wv = gd.w[r * kHeads + j];
-              if (gd.qscale) wv = __fmul_rn(wv, gd.qscale[r * kHeads + j]);
-            }
+            const float wv = ct.gstage[kb][i];
             const __nv_bfloat16 hi = __float2bfloat16_rn(wv);
             const __nv_bfloat16 lo = __float2bfloat16_rn(wv - __bfloat162float(hi));
             const uint32_t in_row = (j & 7) * 2;
