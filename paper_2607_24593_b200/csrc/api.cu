@@ -729,7 +729,8 @@ const char* pivot_status_str(int code) {
   switch (code) {
     case PIVOT_OK: return "ok";
     case PIVOT_ERR_INVALID_ARG: return "invalid argument";
-    case PIVOT_ERR_UNSUPPORTED: return "unsupported shape (H_I must be 64, d 128, k and c at most 8192)";
+    case PIVOT_ERR_UNSUPPORTED:
+      return "unsupported: shape (H_I must be 64, d 128, k and c at most 8192), layout, or an entry point this build does not carry";
     case PIVOT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case PIVOT_ERR_CUDA: return "CUDA runtime error (see pivot_last_cuda_error)";
     case PIVOT_ERR_DEVICE: return "device-side condition recorded in the status word";

@@ -1,5 +1,6 @@
 """GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded
 inputs, element by element, under the acceptance rule of oracle/acceptance.py."""
+import os
 import numpy as np
 import pytest
 import torch
@@ -675,6 +676,15 @@ def test_bounded_wait_runs_out_and_reports_without_hanging(pv, gu):
 
 
 # ---------------------------------------------------------------- argument errors (host side)
+
+def test_counters_entry_point_is_refused_by_an_ordinary_build(pv):
+    """pivot_debug_counters belongs to the -DPIVOT_PROF build (bench.py --counters); the library the
+    tests load carries no counters and says so instead of returning the workspace head's bytes."""
+    if os.path.basename(os.environ.get("PIVOT_LIB", "libpivot.so")) == "libpivot_prof.so":
+        pytest.skip("counters build loaded")
+    with pytest.raises(pv.PivotError, match="unsupported|not supported"):
+        pv.pivot_debug_counters()
+
 
 def test_argument_errors(pv):
     x = inputs.make_prefill(64, dtype="bf16", seed=1)
