@@ -364,6 +364,11 @@ def counters_run(pv, dev, wl):
     n = max(v["decode_select_sequences"], 1)
     res["decode_select_clocks_per_sequence"] = {nm: round(v["decode_select_" + nm] / n, 1)
                                                 for nm in ("boundary", "collect", "handover", "topk")}
+    nt = max(v["decode_scan_tiles"], 1)
+    res["decode_scan_clocks_per_tile"] = {nm: round(v["decode_scan_" + nm] / nt, 1)
+                                          for nm in ("producer_wait", "wait_accumulator", "wait_keys", "total")}
+    res["decode_scan_tiles"] = v["decode_scan_tiles"]
+    res["decode_scan_loop_clocks_mean_and_longest_cta"] = [round(v["decode_scan_total"] / 148), v["decode_scan_max_total"]]
     return res
 
 
@@ -565,6 +570,9 @@ def main():
         res = {"mma_model": pv.pivot_debug_mma_model(), "key_stream": []}
         for ctas, stages, mode in ((1, 4, 0), (148, 2, 0), (148, 4, 0), (148, 12, 0), (148, 4, 1), (148, 4, 2), (1, 4, 2), (148, 4, 3), (148, 4, 4)):
             res["key_stream"].append(pv.pivot_debug_key_stream(ctas=ctas, stages=stages, mode=mode))
+        # the decode scan's shape without its compute: 148 CTAs x 165 consecutive tiles each out of 410 MB (HBM, not L2)
+        res["key_stream_hbm_decode_shape"] = pv.pivot_debug_key_stream(n_keys=3_200_000 // 128 * 128, ctas=148, tiles=165,
+                                                                       stages=8, mode=0)
         print(json.dumps(res, indent=1))
         return
     if args.sweep:

@@ -324,7 +324,9 @@ PROF_SLOTS = ("scan_wait_queries", "scan_wait_accumulator", "scan_wait_keys", "s
               "rescore_wait_relu", "rescore_total", "rescore_tiles",
               "rescore_select_wait", "rescore_select_work", "rescore_select_groups",
               "decode_select_boundary", "decode_select_collect", "decode_select_handover", "decode_select_topk",
-              "decode_select_sequences")
+              "decode_select_sequences",
+              "decode_scan_producer_wait", "decode_scan_max_total", "decode_scan_wait_accumulator", "decode_scan_wait_keys",
+              "decode_scan_total", "decode_scan_tiles")
 
 
 def pivot_debug_counters(stream=None) -> dict:

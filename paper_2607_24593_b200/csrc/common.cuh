@@ -45,12 +45,21 @@ enum ProfSlot {
   PROF_DSEL_HANDOVER,           //   cluster barriers + reading the other CTAs' lists,
   PROF_DSEL_TOPK,               //   exact top-c of the collected entries; and
   PROF_DSEL_SEQS,               //   sequences
+  PROF_DSCAN_PRODUCER_WAIT,     // decode scan: the key-TMA thread waiting for a free stage,
+  PROF_DSCAN_MAX_TOTAL,         //   the MMA-issuing thread: the longest whole loop of any CTA (a maximum, not a sum),
+  PROF_DSCAN_WAIT_ACC,          //   a free accumulator buffer,
+  PROF_DSCAN_WAIT_KEYS,         //   the key tile,
+  PROF_DSCAN_TOTAL,             //   its whole loop (from the end of the kernel's set-up); and
+  PROF_DSCAN_TILES,             //   tiles
   PROF_SLOTS
 };
 static_assert(PROF_SLOTS <= 28, "the workspace head holds 28 counters");
 #ifdef PIVOT_PROF
 __device__ __forceinline__ void prof_add(int* status, int slot, long long v) {
   if (status) atomicAdd(reinterpret_cast<unsigned long long*>(status + 8) + slot, (unsigned long long)v);
+}
+__device__ __forceinline__ void prof_max(int* status, int slot, long long v) {
+  if (status) atomicMax(reinterpret_cast<unsigned long long*>(status + 8) + slot, (unsigned long long)v);
 }
 #define PIVOT_PROF_DO(...) __VA_ARGS__
 #else

@@ -135,6 +135,7 @@ decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       TileWalk tw(tile_prefix, B);
       int cur_b = -1;
       uint32_t it = 0, blk = 0;
+      PIVOT_PROF_DO(long long pwait = 0;)
       for (int g = g_lo; g < g_hi; ++g, ++it) {
         const int b = tw.seq_of(g);
         const int t = g - tile_prefix[b];
@@ -154,7 +155,9 @@ decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         (void)PIVOT_BOUNDS(t * TILE_KEYS < Lmax, status);              // checked build: the tile lies inside the sequence's rows
         const int krow = pages ? __ldg(pages + t) * TILE_KEYS : prox[b].k_row0 + t * TILE_KEYS;
         const int s = it % C::STAGES;
+        PIVOT_PROF_DO(const long long pw0 = clock64();)
         if (!ptx::mbar_wait(&ct.empty[s], ((it / C::STAGES) & 1) ^ 1, abort_flag, 64)) break;
+        PIVOT_PROF_DO(pwait += clock64() - pw0;)
         ptx::mbar_arrive_expect_tx(&ct.full[s], C::STAGE_BYTES);
         for (int h = 0; h < C::KHALVES; ++h)
           ptx::tma_load_2d(kring + s * C::STAGE_BYTES + h * C::HALF_TILE_BYTES, &tm_k, h * 64, krow, &ct.full[s]);
@@ -164,6 +167,7 @@ decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
           ptx::tma_load_1d(&ct.ks[ksl][0], &tm_ks, krow, &ct.ks_full[ksl]);
         }
       }
+      PIVOT_PROF_DO(prof_add(status, PROF_DSCAN_PRODUCER_WAIT, pwait);)
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -172,21 +176,27 @@ decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       int cur_b = -1, qb = 0;
       uint32_t it = 0, blk = 0;
       bool ok = true;
+      PIVOT_PROF_DO(long long pw[3] = {0, 0, 0}; const long long pstart = clock64();)
+#ifdef PIVOT_PROF
+#define PW(i, ...) { const long long t_ = clock64(); __VA_ARGS__; pw[i] += clock64() - t_; }
+#else
+#define PW(i, ...) __VA_ARGS__;
+#endif
       for (int g = g_lo; g < g_hi && ok; ++g, ++it) {
         const int b = tw.seq_of(g);
         if (b != cur_b) {
           if (cur_b >= 0) ptx::tc_commit(&ct.q_empty[qb]);     // previous proxy no longer needed
           qb = blk & 1;
-          ok = ptx::mbar_wait(&ct.q_full[qb], (blk >> 1) & 1, abort_flag, 32);
+          PW(0, ok = ptx::mbar_wait(&ct.q_full[qb], (blk >> 1) & 1, abort_flag, 32))
           if (!ok) break;
           ++blk;
           cur_b = b;
         }
         const int s = it % C::STAGES;
         const int buf = it & 1;
-        ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, 32);
+        PW(1, ok = ptx::mbar_wait(&ct.tmem_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, 32))
         if (!ok) break;
-        ok = ptx::mbar_wait(&ct.full[s], (it / C::STAGES) & 1, abort_flag, 32);
+        PW(2, ok = ptx::mbar_wait(&ct.full[s], (it / C::STAGES) & 1, abort_flag, 32))
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t k_addr = ptx::smem_u32(kring + s * C::STAGE_BYTES);
@@ -202,6 +212,14 @@ decode_scan_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         ptx::tc_commit(&ct.empty[s]);
         ptx::tc_commit(&ct.tmem_full[buf]);
       }
+#undef PW
+      PIVOT_PROF_DO({
+        prof_add(status, PROF_DSCAN_WAIT_ACC, pw[0] + pw[1]);       // (the proxy wait, a few clocks per tile, is counted here)
+        prof_add(status, PROF_DSCAN_WAIT_KEYS, pw[2]);
+        prof_max(status, PROF_DSCAN_MAX_TOTAL, clock64() - pstart);
+        prof_add(status, PROF_DSCAN_TOTAL, clock64() - pstart);
+        prof_add(status, PROF_DSCAN_TILES, it);
+      })
     }
   } else {
     // ------------------------------------------------------------------ epilogue
