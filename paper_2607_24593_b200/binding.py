@@ -341,6 +341,8 @@ def pivot_debug_key_stream(n_keys=131072, ctas=148, tiles=2048, stages=4, mode=0
     """Key-tile streaming probe (see pivot.h): clocks per 16 KB tile, mean over the CTAs, per stream."""
     keys = torch.zeros((n_keys, 128), dtype=torch.uint8, device="cuda")
     out = torch.zeros(2 * ctas, dtype=torch.int64, device="cuda")
+    if n_keys * 128 > (64 << 20):          # an HBM-sized stream: nothing of it may still sit in L2
+        torch.empty(512 << 20, dtype=torch.uint8, device="cuda").fill_(1)
     _check(lib.pivot_debug_key_stream(keys.data_ptr(), n_keys, ctas, tiles, stages, mode, out.data_ptr(), _stream(stream)))
     torch.cuda.synchronize()
     v = out.cpu().float().view(ctas, 2)
