@@ -55,10 +55,17 @@ __device__ __forceinline__ void proxy_build_unit(const void* __restrict__ q, con
       if (i0 + u < hi) {
         const uint32_t wd[4] = {pk[u].x, pk[u].y, pk[u].z, pk[u].w};
         float x[E];
+        if (FP8) {                           // two codes per conversion (e4m3 -> half is exact, and so is half -> float)
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-          if (FP8) x[e] = __fmul_rn(e4m3_to_float((wd[e >> 2] >> (8 * (e & 3))) & 0xff), sc[u]);
-          else x[e] = bf16_bits_to_float((wd[e >> 1] >> (16 * (e & 1))) & 0xffff);
+          for (int e = 0; e < E; e += 2) {
+            const __half2_raw h2 = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)((wd[e >> 2] >> (8 * (e & 3))) & 0xffff), __NV_E4M3);
+            const float2 f2 = __half22float2(__half2(h2));
+            x[e] = __fmul_rn(f2.x, sc[u]);
+            x[e + 1] = __fmul_rn(f2.y, sc[u]);
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < E; ++e) x[e] = bf16_bits_to_float((wd[e >> 1] >> (16 * (e & 1))) & 0xffff);
         }
         if (i0 + u == lo) {
 #pragma unroll
@@ -93,10 +100,10 @@ __device__ __forceinline__ void proxy_build_unit(const void* __restrict__ q, con
 #pragma unroll
     for (int j = 0; j < 4; ++j) ow[j] = 0u;
 #pragma unroll
-    for (int e = 0; e < E; ++e) {
-      const uint32_t code =
-          (uint32_t)__nv_cvt_float_to_fp8(__fmul_rn(acc[e], inv), __NV_SATFINITE, __NV_E4M3);
-      ow[e >> 2] |= (code & 0xffu) << (8 * (e & 3));
+    for (int e = 0; e < E; e += 2) {         // two values per conversion, same rounding as one at a time
+      const uint32_t code2 = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(acc[e], inv), __fmul_rn(acc[e + 1], inv)),
+                                                                __NV_SATFINITE, __NV_E4M3);
+      ow[e >> 2] |= (code2 & 0xffffu) << (8 * (e & 3));
     }
     if (sub == 0) proxy_w[orow] = __fmul_rn(wacc, sbar);
   } else {
