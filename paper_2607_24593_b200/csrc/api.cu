@@ -16,7 +16,7 @@ constexpr int kMaxSel = 8192;
 constexpr int kMaxDevices = 64;
 
 #ifndef PIVOT_HOST_CHUNKS
-#define PIVOT_HOST_CHUNKS 8
+#define PIVOT_HOST_CHUNKS 7
 #endif
 constexpr int kHostChunks = PIVOT_HOST_CHUNKS;   // query-row chunks of the host-buffer prefill pipeline
 
@@ -608,7 +608,10 @@ int pivot_index_prefill_host(const pivot_tensor* q, const float* w, const pivot_
     const int i = (j & 1) ? j / 2 : n_chunks - 1 - j / 2;
     const int r0 = i * chunk_rows, r1 = (r0 + chunk_rows < L) ? r0 + chunk_rows : L;
     // a quarter first (the first input copy) resp. last (the last result copy)
-    const int mid = j == 0 ? r0 + (r1 - r0) / 4 / g * g : r1 - (r1 - r0) / 4 / g * g;
+#ifndef PIVOT_HOST_SPLIT
+#define PIVOT_HOST_SPLIT 4
+#endif
+    const int mid = j == 0 ? r0 + (r1 - r0) / PIVOT_HOST_SPLIT / g * g : r1 - (r1 - r0) / PIVOT_HOST_SPLIT / g * g;
     if ((j == 0 || j == n_chunks - 1) && n_chunks >= 4 && mid > r0 && mid < r1) {
       piece[n_pieces++] = Piece{r0, mid};
       piece[n_pieces++] = Piece{mid, r1};

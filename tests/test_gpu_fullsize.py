@@ -79,7 +79,7 @@ def _rows_equal_as_sets(a: torch.Tensor, b: torch.Tensor) -> bool:
 def test_config3_plain_call_and_host_pipeline_at_full_size():
     """The headline configuration exactly as bench.py times it: the call WITHOUT debug buffers
     (other store paths in the kernels: staged 16-byte index rows, candidates in the workspace) and
-    the host-buffer pipeline in eight row chunks.  Both must return, row for row, the sets of the
+    the host-buffer pipeline in its row chunks.  Both must return, row for row, the sets of the
     call with debug buffers, and those are checked against the oracle on the sampled groups."""
     import gpu_util
     from paper_2607_24593_b200 import binding as pv
@@ -103,7 +103,7 @@ def test_config3_plain_call_and_host_pipeline_at_full_size():
                           cand=cand.cpu().numpy(), cand_scores=cs.cpu().numpy(), groups=groups)
     print(f"\n[128K plain call] groups={len(groups)} rows={t.rows} exact={t.exact_rows} band_swaps={t.band_swaps}")
     del cand, cs, dbg
-    # host pipeline (eight chunks at this size)
+    # host pipeline (seven chunks at this size, the first and the last cut once more)
     pv.pivot_set_workspace(None)
     del d
     torch.cuda.empty_cache()
